@@ -1,0 +1,425 @@
+/*
+ * halo_ref.c -- CPU fp64 oracle for the HALO group-sparse FFN hot path.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain restatement of what
+ * the method computes, used to check the CUDA library and to time a CPU
+ * baseline.  Nothing on the product path may call it, and it shares no code,
+ * header, table or helper with the CUDA sources.
+ *
+ * Every function takes HOST pointers.  Weights / activations arrive as the raw
+ * bytes the GPU sees (fp32, or bf16 as uint16) and are widened exactly to
+ * double; all arithmetic is fp64 unless a step is an integer decision.
+ *
+ * Passages followed (HALO, arXiv 2601.11676):
+ *   Sec. II-A "Neuron group"            -- a group = gate rows + up rows + the
+ *                                          matching down-projection columns.
+ *   Sec. II-B insight                   -- merged features = sum of all groups'
+ *                                          activations (linearity).
+ *   Sec. III-B.2 (SAPs)                 -- small predictor, importance score
+ *                                          per group, one layer ahead.
+ *   Sec. III-B.3 (Pred process)         -- importance rank indexes the
+ *                                          priority lists of the Assignment phase.
+ *   Sec. III-B.4 + Algorithm 3          -- PLR-aware ratio-guided partition of
+ *                                          the priority list over devices.
+ *   Sec. III-B.3 (relaxed sync)         -- the master merges whatever arrived;
+ *                                          first layer is reliable.
+ *
+ * Pins (tests/test_oracle_*.py): Philox4x32-10 known answers; the worked
+ * example printed with Algorithm 3; 6144/256 = 24 groups; NGLR = 1 - 1/n;
+ * brute-force ranking; dense SwiGLU via an fp64 library matmul; linearity;
+ * permutation invariance; closed forms; merge flip identity.
+ * Parity unpinned: the *meaning* of predictor scores (needs trained weights)
+ * and the particular arrival sequence (the paper's loss is physical; the
+ * sequence is fixed here by the Philox counter convention only).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define REF_OK 0
+#define REF_ERR_ARG (-1)
+#define REF_ERR_SHAPE (-2)
+#define REF_ERR_NOMEM (-6)
+
+#define REF_F32 0
+#define REF_BF16 1
+
+#define REF_SEL_TOPK 0
+#define REF_SEL_THRESHOLD 1
+
+#define REF_ACT_RELU 0
+#define REF_ACT_NONE 1
+
+#define REF_STATUS_NONFINITE 1u
+
+/* ---- exact widening of the stored element types ------------------------- */
+
+static double ref_widen(const void* base, size_t i, int dtype) {
+    if (dtype == REF_F32) return (double)((const float*)base)[i];
+    uint32_t bits = (uint32_t)((const uint16_t*)base)[i] << 16; /* bf16 = top half of fp32 */
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return (double)f;
+}
+
+static size_t ref_elem_size(int dtype) { return dtype == REF_F32 ? 4 : 2; }
+
+/* double -> bf16 with round-to-nearest-even, via the exact fp32 neighbours.
+ * Used only by the inter-layer glue (the activation vector is stored bf16). */
+static uint16_t ref_double_to_bf16(double v) {
+    if (isnan(v)) return 0x7fc0;
+    float f = (float)v;             /* RNE to fp32 first (as the GPU does) */
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;             /* RNE on the dropped 16 bits */
+    return (uint16_t)(u >> 16);
+}
+
+/* ---- Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) ------------------- */
+/* Counter-based generator; 10 rounds of two 32x32->64 multiplies with the
+ * published multipliers, and Weyl key bumps between rounds. */
+
+static void philox_round(uint32_t c[4], const uint32_t k[2]) {
+    uint64_t p0 = (uint64_t)0xD2511F53u * c[0];
+    uint64_t p1 = (uint64_t)0xCD9E8D57u * c[2];
+    uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+    uint32_t n0 = hi1 ^ c[1] ^ k[0];
+    uint32_t n2 = hi0 ^ c[3] ^ k[1];
+    c[0] = n0; c[1] = lo1; c[2] = n2; c[3] = lo0;
+}
+
+void halo_ref_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+    uint32_t c[4] = {ctr[0], ctr[1], ctr[2], ctr[3]};
+    uint32_t k[2] = {key[0], key[1]};
+    for (int r = 0; r < 10; ++r) {
+        if (r > 0) { k[0] += 0x9E3779B9u; k[1] += 0xBB67AE85u; }
+        philox_round(c, k);
+    }
+    memcpy(out, c, sizeof c);
+}
+
+/* One Bernoulli draw per (seed, step, layer, device): the device's whole
+ * partial activation arrives or is lost (relaxed synchronisation, Sec.
+ * III-B.3).  counter = (step, layer, device, 0), key = seed halves; word 0 of
+ * the output is compared with T = round(rho * 2^32) in 64-bit, so rho = 0
+ * always arrives and rho = 1 never does. */
+uint64_t halo_ref_loss_threshold(double rho) {
+    if (!(rho > 0.0)) return 0;
+    if (rho >= 1.0) return (uint64_t)1 << 32;
+    double t = floor(rho * 4294967296.0 + 0.5);
+    if (t > 4294967296.0) t = 4294967296.0;
+    return (uint64_t)t;
+}
+
+int halo_ref_arrival(uint64_t seed, uint32_t step, uint32_t layer, uint32_t device, double rho) {
+    uint32_t ctr[4] = {step, layer, device, 0u};
+    uint32_t key[2] = {(uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32)};
+    uint32_t out[4];
+    halo_ref_philox4x32_10(ctr, key, out);
+    return ((uint64_t)out[0] >= halo_ref_loss_threshold(rho)) ? 1 : 0;
+}
+
+/* ---- weight layout ------------------------------------------------------- */
+/* Packed layer buffer W[G][3][S][d]: plane 0 = gate rows of the group, plane 1
+ * = up rows, plane 2 = the group's down-projection columns stored as rows
+ * (Sec. II-A: one group owns all three slices).  Conventional matrices are
+ * Wgate[F][d], Wup[F][d], Wdown[d][F]. */
+
+static size_t packed_index(int g, int plane, int j, int c, int S, int d) {
+    return (((size_t)g * 3 + (size_t)plane) * (size_t)S + (size_t)j) * (size_t)d + (size_t)c;
+}
+
+int halo_ref_pack_weights(int d, int F, int S, int dtype, const void* Wgate, const void* Wup,
+                          const void* Wdown, void* Wpacked) {
+    if (d <= 0 || F <= 0 || S <= 0 || F % S != 0) return REF_ERR_SHAPE;
+    size_t es = ref_elem_size(dtype);
+    const char* wg = (const char*)Wgate;
+    const char* wu = (const char*)Wup;
+    const char* wd = (const char*)Wdown;
+    char* out = (char*)Wpacked;
+    int G = F / S;
+    for (int g = 0; g < G; ++g)
+        for (int j = 0; j < S; ++j) {
+            size_t n = (size_t)g * S + j; /* neuron index in [0,F) */
+            for (int c = 0; c < d; ++c) {
+                memcpy(out + es * packed_index(g, 0, j, c, S, d), wg + es * (n * d + c), es);
+                memcpy(out + es * packed_index(g, 1, j, c, S, d), wu + es * (n * d + c), es);
+                memcpy(out + es * packed_index(g, 2, j, c, S, d), wd + es * ((size_t)c * F + n), es);
+            }
+        }
+    return REF_OK;
+}
+
+int halo_ref_unpack_weights(int d, int F, int S, int dtype, const void* Wpacked, void* Wgate,
+                            void* Wup, void* Wdown) {
+    if (d <= 0 || F <= 0 || S <= 0 || F % S != 0) return REF_ERR_SHAPE;
+    size_t es = ref_elem_size(dtype);
+    const char* in = (const char*)Wpacked;
+    int G = F / S;
+    for (int g = 0; g < G; ++g)
+        for (int j = 0; j < S; ++j) {
+            size_t n = (size_t)g * S + j;
+            for (int c = 0; c < d; ++c) {
+                memcpy((char*)Wgate + es * (n * d + c), in + es * packed_index(g, 0, j, c, S, d), es);
+                memcpy((char*)Wup + es * (n * d + c), in + es * packed_index(g, 1, j, c, S, d), es);
+                memcpy((char*)Wdown + es * ((size_t)c * F + n), in + es * packed_index(g, 2, j, c, S, d), es);
+            }
+        }
+    return REF_OK;
+}
+
+/* ---- step a1: predictor -------------------------------------------------- */
+/* Bias-free two-layer net, Sec. III-B.2: z = act(W1 f), s = W2 z, with
+ * W1[r][d_in] and W2[G][r] (one row per output unit).  Scores leave as fp32:
+ * that array is the boundary the selection reads.  With mean_pool the scores
+ * of the n_tok tokens are averaged in fp64 (token order fixed) before the
+ * cast, giving one score vector for the whole prompt. */
+int halo_ref_predict(int d_in, int rank, int G, int dtype, int act, const void* W1, const void* W2,
+                     const void* feat, int n_tok, int mean_pool, float* scores) {
+    if (d_in <= 0 || rank <= 0 || G <= 0 || n_tok <= 0) return REF_ERR_SHAPE;
+    double* z = (double*)malloc(sizeof(double) * (size_t)rank);
+    double* pooled = (double*)calloc((size_t)G, sizeof(double));
+    if (!z || !pooled) { free(z); free(pooled); return REF_ERR_NOMEM; }
+    for (int t = 0; t < n_tok; ++t) {
+        for (int u = 0; u < rank; ++u) {
+            double acc = 0.0;
+            for (int c = 0; c < d_in; ++c)
+                acc += ref_widen(W1, (size_t)u * d_in + c, dtype) * ref_widen(feat, (size_t)t * d_in + c, dtype);
+            if (act == REF_ACT_RELU && acc < 0.0) acc = 0.0;
+            z[u] = acc;
+        }
+        for (int g = 0; g < G; ++g) {
+            double acc = 0.0;
+            for (int u = 0; u < rank; ++u) acc += ref_widen(W2, (size_t)g * rank + u, dtype) * z[u];
+            if (mean_pool) pooled[g] += acc;
+            else scores[(size_t)t * G + g] = (float)acc;
+        }
+    }
+    if (mean_pool)
+        for (int g = 0; g < G; ++g) scores[g] = (float)(pooled[g] / (double)n_tok);
+    free(z);
+    free(pooled);
+    return REF_OK;
+}
+
+/* ---- Assignment phase: Algorithm 3 -------------------------------------- */
+/* q = argsort(rho ascending; ties -> lower device index).  The priority list
+ * of M less-critical groups is cut into n contiguous chunks proportional to
+ * the ratios taken in q's order; chunk j goes to device q[j].  Ratios are
+ * integer weights; the cut after chunk j is round-half-up(M * C_j / C_n) in
+ * 64-bit integers, C_j the cumulative weight. */
+int halo_ref_plan(int n_dev, const double* loss_rate, const uint32_t* share_weight, int M,
+                  int32_t* dev_order /*[n]*/, uint64_t* loss_thresh /*[n], by device index*/,
+                  int32_t* boundaries /*[n+1]*/) {
+    if (n_dev < 0 || M < 0) return REF_ERR_ARG;
+    for (int i = 0; i < n_dev; ++i) {
+        if (!(loss_rate[i] >= 0.0 && loss_rate[i] <= 1.0)) return REF_ERR_ARG;
+        loss_thresh[i] = halo_ref_loss_threshold(loss_rate[i]);
+        dev_order[i] = i;
+    }
+    /* insertion sort: stable, ascending rho */
+    for (int a = 1; a < n_dev; ++a) {
+        int32_t v = dev_order[a];
+        int b = a - 1;
+        while (b >= 0 && loss_rate[dev_order[b]] > loss_rate[v]) { dev_order[b + 1] = dev_order[b]; --b; }
+        dev_order[b + 1] = v;
+    }
+    uint64_t total = 0;
+    for (int i = 0; i < n_dev; ++i) total += share_weight[i];
+    boundaries[0] = 0;
+    if (n_dev == 0) return REF_OK;
+    if (total == 0) return REF_ERR_ARG;
+    uint64_t cum = 0;
+    for (int j = 0; j < n_dev; ++j) {
+        cum += share_weight[dev_order[j]];
+        boundaries[j + 1] = (int32_t)((2ull * (uint64_t)M * cum + total) / (2ull * total));
+    }
+    boundaries[n_dev] = M;
+    return REF_OK;
+}
+
+/* ---- steps a2..a5: rank, critical choice, assignment, arrival mask ------- */
+/* Order: higher score first, equal scores -> lower group index (NaN counts as
+ * -inf and raises a status bit; -0 == +0).  TOPK: the first k of the order are
+ * critical.  THRESHOLD: critical = {s >= theta} (a prefix of the order).
+ * Critical groups stay on the master (never lost); the rest, in priority
+ * order, are cut by Algorithm 3.  keep = critical OR the holder arrived;
+ * force_all (first layer / reliable block) keeps everything. */
+int halo_ref_select(int G, int n_dev, const double* loss_rate, const uint32_t* share_weight,
+                    int mode, int k_critical, float threshold, uint64_t seed,
+                    const float* scores, uint32_t step, uint32_t layer, int force_all,
+                    int32_t* order, int32_t* rank, int32_t* dev_of_group, uint8_t* arrived,
+                    uint8_t* keep, int32_t* keep_list, int32_t* n_keep, uint32_t* status) {
+    if (G <= 0 || n_dev < 0) return REF_ERR_SHAPE;
+    if (mode == REF_SEL_TOPK && (k_critical < 0 || k_critical > G)) return REF_ERR_ARG;
+    uint32_t st = 0;
+    float* s = (float*)malloc(sizeof(float) * (size_t)G);
+    int32_t* dev_order = (int32_t*)malloc(sizeof(int32_t) * (size_t)(n_dev + 1));
+    uint64_t* thr = (uint64_t*)malloc(sizeof(uint64_t) * (size_t)(n_dev + 1));
+    int32_t* bnd = (int32_t*)malloc(sizeof(int32_t) * (size_t)(n_dev + 2));
+    if (!s || !dev_order || !thr || !bnd) { free(s); free(dev_order); free(thr); free(bnd); return REF_ERR_NOMEM; }
+    for (int g = 0; g < G; ++g) {
+        float v = scores[g];
+        if (isnan(v)) { v = -INFINITY; st |= REF_STATUS_NONFINITE; }
+        else if (isinf(v)) st |= REF_STATUS_NONFINITE;
+        if (v == 0.0f) v = 0.0f; /* folds -0 onto +0 */
+        s[g] = v;
+    }
+    /* rank by counting: how many groups come strictly before g */
+    for (int g = 0; g < G; ++g) {
+        int before = 0;
+        for (int o = 0; o < G; ++o)
+            if (s[o] > s[g] || (s[o] == s[g] && o < g)) ++before;
+        rank[g] = before;
+        order[before] = g;
+    }
+    int k = k_critical;
+    if (mode == REF_SEL_THRESHOLD) {
+        k = 0;
+        for (int g = 0; g < G; ++g) if (s[g] >= threshold) ++k;
+    }
+    if (n_dev == 0) k = G; /* nobody else to hold them */
+    int M = G - k;
+    int rc = halo_ref_plan(n_dev, loss_rate, share_weight, M, dev_order, thr, bnd);
+    if (rc != REF_OK) { free(s); free(dev_order); free(thr); free(bnd); return rc; }
+    for (int i = 0; i < n_dev; ++i)
+        arrived[i] = (uint8_t)(force_all ? 1 : halo_ref_arrival(seed, step, layer, (uint32_t)i, loss_rate[i]));
+    int nk = 0;
+    for (int g = 0; g < G; ++g) {
+        int dev = -1;
+        if (rank[g] >= k) {
+            int p = rank[g] - k;
+            for (int j = 0; j < n_dev; ++j)
+                if (bnd[j] <= p && p < bnd[j + 1]) { dev = dev_order[j]; break; }
+        }
+        dev_of_group[g] = dev;
+        keep[g] = (uint8_t)((dev < 0) ? 1 : arrived[dev]);
+        if (keep[g]) keep_list[nk++] = g;
+    }
+    for (int i = nk; i < G; ++i) keep_list[i] = -1;
+    *n_keep = nk;
+    if (status) *status = st;
+    free(s); free(dev_order); free(thr); free(bnd);
+    return REF_OK;
+}
+
+/* ---- steps a6..a8: group-masked SwiGLU FFN ------------------------------- */
+/* For every listed group g and neuron j of it:
+ *     a = <gate_j, x>, b = <up_j, x>, h = a / (1 + exp(-a)) * b,
+ *     p_g += h * down_j          (down_j = column j of the down projection)
+ * and the group's partial p_g is added to the slot of its holder
+ * (slot 0 = master, slot i+1 = device i).  group_partials, if given, receives
+ * every listed group's p_g on its own ([n_list][n_tok][d]) -- the linearity
+ * check and the "importance = L2 norm of the group's activation" diagnostic
+ * (Sec. II-B) read it. */
+int halo_ref_group_ffn(int d, int F, int S, int dtype, const void* Wpacked, const void* x, int n_tok,
+                       const int32_t* list, int n_list, const int32_t* dev_of_group, int n_dev,
+                       double* partials /*[n_dev+1][n_tok][d]*/, double* group_partials /*or NULL*/) {
+    if (d <= 0 || F <= 0 || S <= 0 || F % S != 0 || n_tok <= 0 || n_list < 0) return REF_ERR_SHAPE;
+    int G = F / S;
+    for (int i = 0; i < n_list; ++i) if (list[i] < 0 || list[i] >= G) return REF_ERR_ARG;
+    size_t slot_elems = (size_t)n_tok * d;
+    memset(partials, 0, sizeof(double) * slot_elems * (size_t)(n_dev + 1));
+    double* pg = group_partials;
+    int own = 0;
+    if (!pg) {
+        pg = (double*)malloc(sizeof(double) * slot_elems * (size_t)(n_list > 0 ? n_list : 1));
+        if (!pg) return REF_ERR_NOMEM;
+        own = 1;
+    }
+#pragma omp parallel for schedule(dynamic)
+    for (int i = 0; i < n_list; ++i) {
+        int g = list[i];
+        double* out = pg + (size_t)i * slot_elems;
+        for (size_t e = 0; e < slot_elems; ++e) out[e] = 0.0;
+        for (int t = 0; t < n_tok; ++t)
+            for (int j = 0; j < S; ++j) {
+                double a = 0.0, b = 0.0;
+                for (int c = 0; c < d; ++c) {
+                    double xc = ref_widen(x, (size_t)t * d + c, dtype);
+                    a += ref_widen(Wpacked, packed_index(g, 0, j, c, S, d), dtype) * xc;
+                    b += ref_widen(Wpacked, packed_index(g, 1, j, c, S, d), dtype) * xc;
+                }
+                double h = a / (1.0 + exp(-a)) * b;
+                for (int c = 0; c < d; ++c)
+                    out[(size_t)t * d + c] += h * ref_widen(Wpacked, packed_index(g, 2, j, c, S, d), dtype);
+            }
+    }
+    for (int i = 0; i < n_list; ++i) { /* fixed order: ascending list position */
+        int g = list[i];
+        int slot = dev_of_group ? dev_of_group[g] + 1 : 0;
+        if (slot < 0 || slot > n_dev) { if (own) free(pg); return REF_ERR_ARG; }
+        double* dst = partials + (size_t)slot * slot_elems;
+        const double* src = pg + (size_t)i * slot_elems;
+        for (size_t e = 0; e < slot_elems; ++e) dst[e] += src[e];
+    }
+    if (own) free(pg);
+    return REF_OK;
+}
+
+/* ---- step a9: merge ------------------------------------------------------ */
+/* y = P[master] + sum over devices that arrived of P[device]; a lost or late
+ * device contributes nothing (Sec. III-B.3). */
+int halo_ref_merge(const double* partials, const uint8_t* arrived /*NULL => all*/, int n_dev, int n_tok,
+                   int d, double* y) {
+    if (n_dev < 0 || n_tok <= 0 || d <= 0) return REF_ERR_SHAPE;
+    size_t slot_elems = (size_t)n_tok * d;
+    for (size_t e = 0; e < slot_elems; ++e) y[e] = partials[e];
+    for (int i = 0; i < n_dev; ++i)
+        if (!arrived || arrived[i])
+            for (size_t e = 0; e < slot_elems; ++e) y[e] += partials[(size_t)(i + 1) * slot_elems + e];
+    return REF_OK;
+}
+
+/* ---- glue between the layers of an FFN stack ----------------------------- */
+/* Residual stream h (fp32 on the GPU, double here): h' = h + y, and the next
+ * block's input is the gain-free RMS-normalised stream stored in the
+ * activation dtype: x = cast(h' / sqrt(mean(h'^2) + 1e-5)).  y may be NULL
+ * (normalise only: the stack's very first input). */
+int halo_ref_glue(int d, int n_tok, int dtype, const double* h, const double* y, double* h_out, void* x_out) {
+    if (d <= 0 || n_tok <= 0) return REF_ERR_SHAPE;
+    for (int t = 0; t < n_tok; ++t) {
+        double ss = 0.0;
+        for (int c = 0; c < d; ++c) {
+            double v = h[(size_t)t * d + c] + (y ? y[(size_t)t * d + c] : 0.0);
+            h_out[(size_t)t * d + c] = v;
+            ss += v * v;
+        }
+        double scale = 1.0 / sqrt(ss / (double)d + 1e-5);
+        for (int c = 0; c < d; ++c) {
+            double v = h_out[(size_t)t * d + c] * scale;
+            if (dtype == REF_F32) ((float*)x_out)[(size_t)t * d + c] = (float)v;
+            else ((uint16_t*)x_out)[(size_t)t * d + c] = ref_double_to_bf16(v);
+        }
+    }
+    return REF_OK;
+}
+
+/* ---- one whole layer, steps a1..a9 in order ------------------------------ */
+/* feat is the predictor input (the previous layer's x: one layer ahead); x is
+ * this layer's FFN input.  Only kept groups are computed, so the merge adds
+ * every slot that exists.  Outputs y (double) and the selection arrays. */
+int halo_ref_layer(int d, int F, int S, int dtype, const void* Wpacked, int rank, int act, const void* W1,
+                   const void* W2, int n_dev, const double* loss_rate, const uint32_t* share_weight,
+                   int mode, int k_critical, float threshold, uint64_t seed, uint32_t step, uint32_t layer,
+                   int force_all, const void* feat, const void* x, int n_tok, float* scores,
+                   int32_t* order, int32_t* rank_out, int32_t* dev_of_group, uint8_t* arrived,
+                   uint8_t* keep, int32_t* keep_list, int32_t* n_keep, uint32_t* status, double* y) {
+    if (F % S != 0) return REF_ERR_SHAPE;
+    int G = F / S;
+    int rc = halo_ref_predict(d, rank, G, dtype, act, W1, W2, feat, n_tok, n_tok > 1, scores);
+    if (rc) return rc;
+    rc = halo_ref_select(G, n_dev, loss_rate, share_weight, mode, k_critical, threshold, seed, scores, step,
+                         layer, force_all, order, rank_out, dev_of_group, arrived, keep, keep_list, n_keep,
+                         status);
+    if (rc) return rc;
+    double* P = (double*)malloc(sizeof(double) * (size_t)(n_dev + 1) * n_tok * d);
+    if (!P) return REF_ERR_NOMEM;
+    rc = halo_ref_group_ffn(d, F, S, dtype, Wpacked, x, n_tok, keep_list, *n_keep, dev_of_group, n_dev, P, NULL);
+    if (!rc) rc = halo_ref_merge(P, NULL, n_dev, n_tok, d, y);
+    free(P);
+    return rc;
+}

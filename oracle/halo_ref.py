@@ -1,0 +1,270 @@
+"""ctypes front end of the CPU fp64 oracle (``halo_ref.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
+benchmark's CPU-baseline leg.  It never touches CUDA and imports nothing from
+the CUDA package.  Arrays go in as numpy arrays holding the raw element bytes
+(``float32``, or ``uint16`` for bf16) and results come back as numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from ctypes import POINTER, c_double, c_float, c_int, c_int32, c_uint8, c_uint32, c_uint64, c_void_p
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "halo_ref.c")
+_LIB = os.path.join(_HERE, "libhalo_ref.so")
+
+F32, BF16 = 0, 1
+SEL_TOPK, SEL_THRESHOLD = 0, 1
+ACT_RELU, ACT_NONE = 0, 1
+STATUS_NONFINITE = 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain C, OpenMP over groups)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fno-fast-math", "-ffp-contract=off", "-shared", "-fPIC",
+             _SRC, "-o", tmp, "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.halo_ref_loss_threshold.restype = c_uint64
+        _lib.halo_ref_loss_threshold.argtypes = [c_double]
+        _lib.halo_ref_arrival.restype = c_int
+        _lib.halo_ref_arrival.argtypes = [c_uint64, c_uint32, c_uint32, c_uint32, c_double]
+    return _lib
+
+
+def _dtype_of(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return F32
+    if a.dtype == np.uint16:
+        return BF16
+    raise TypeError(f"oracle arrays are float32 or uint16 (bf16 bits), got {a.dtype}")
+
+
+def _c(a: np.ndarray) -> np.ndarray:
+    return np.ascontiguousarray(a)
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(c_void_p)
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise RuntimeError(f"oracle {what} failed with status {rc}")
+
+
+def set_threads(n: int) -> None:
+    """OpenMP thread count for the group loop (the timed baseline states it)."""
+    omp = ctypes.CDLL("libgomp.so.1")
+    omp.omp_set_num_threads(int(n))
+
+
+# --- bf16 helpers for tests (exact bit manipulation, no arithmetic) ----------
+
+def bf16_bits_to_f64(a: np.ndarray) -> np.ndarray:
+    return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def to_f64(a: np.ndarray) -> np.ndarray:
+    return bf16_bits_to_f64(a) if a.dtype == np.uint16 else a.astype(np.float64)
+
+
+# --- RNG / arrival ------------------------------------------------------------
+
+def philox4x32_10(ctr, key):
+    c = (c_uint32 * 4)(*[int(v) & 0xFFFFFFFF for v in ctr])
+    k = (c_uint32 * 2)(*[int(v) & 0xFFFFFFFF for v in key])
+    out = (c_uint32 * 4)()
+    lib().halo_ref_philox4x32_10(c, k, out)
+    return [int(v) for v in out]
+
+
+def loss_threshold(rho: float) -> int:
+    return int(lib().halo_ref_loss_threshold(float(rho)))
+
+
+def arrival(seed: int, step: int, layer: int, device: int, rho: float) -> int:
+    return int(lib().halo_ref_arrival(int(seed), int(step), int(layer), int(device), float(rho)))
+
+
+# --- layout -------------------------------------------------------------------
+
+def pack_weights(Wgate: np.ndarray, Wup: np.ndarray, Wdown: np.ndarray, S: int) -> np.ndarray:
+    F, d = Wgate.shape
+    assert Wup.shape == (F, d) and Wdown.shape == (d, F)
+    dt = _dtype_of(Wgate)
+    Wgate, Wup, Wdown = _c(Wgate), _c(Wup), _c(Wdown)
+    out = np.empty((F // S, 3, S, d), dtype=Wgate.dtype)
+    _check(lib().halo_ref_pack_weights(c_int(d), c_int(F), c_int(S), c_int(dt), _p(Wgate), _p(Wup), _p(Wdown),
+                                       _p(out)), "pack_weights")
+    return out
+
+
+def unpack_weights(Wpacked: np.ndarray):
+    G, three, S, d = Wpacked.shape
+    assert three == 3
+    F = G * S
+    dt = _dtype_of(Wpacked)
+    Wpacked = _c(Wpacked)
+    wg = np.empty((F, d), dtype=Wpacked.dtype)
+    wu = np.empty((F, d), dtype=Wpacked.dtype)
+    wd = np.empty((d, F), dtype=Wpacked.dtype)
+    _check(lib().halo_ref_unpack_weights(c_int(d), c_int(F), c_int(S), c_int(dt), _p(Wpacked), _p(wg), _p(wu),
+                                         _p(wd)), "unpack_weights")
+    return wg, wu, wd
+
+
+# --- a1 -----------------------------------------------------------------------
+
+def predict(W1: np.ndarray, W2: np.ndarray, feat: np.ndarray, act: int = ACT_RELU, mean_pool: bool = False):
+    """W1[r][d_in], W2[G][r], feat[n_tok][d_in] (or [d_in]) -> fp32 scores."""
+    r, d_in = W1.shape
+    G = W2.shape[0]
+    assert W2.shape == (G, r)
+    feat2 = feat.reshape(-1, d_in)
+    n_tok = feat2.shape[0]
+    dt = _dtype_of(W1)
+    assert _dtype_of(W2) == dt and _dtype_of(feat2) == dt
+    W1, W2, feat2 = _c(W1), _c(W2), _c(feat2)
+    out = np.empty((G,) if (mean_pool or n_tok == 1) else (n_tok, G), dtype=np.float32)
+    _check(lib().halo_ref_predict(c_int(d_in), c_int(r), c_int(G), c_int(dt), c_int(act), _p(W1), _p(W2),
+                                  _p(feat2), c_int(n_tok), c_int(1 if (mean_pool and n_tok > 1) else 0),
+                                  _p(out)), "predict")
+    return out
+
+
+# --- Algorithm 3 ----------------------------------------------------------------
+
+def plan(loss_rate, share_weight, M: int):
+    n = len(loss_rate)
+    lr = np.asarray(loss_rate, dtype=np.float64)
+    sw = np.asarray(share_weight, dtype=np.uint32)
+    order = np.empty(max(n, 1), dtype=np.int32)
+    thr = np.empty(max(n, 1), dtype=np.uint64)
+    bnd = np.empty(n + 1, dtype=np.int32)
+    _check(lib().halo_ref_plan(c_int(n), _p(lr), _p(sw), c_int(M), _p(order), _p(thr), _p(bnd)), "plan")
+    return order[:n].copy(), thr[:n].copy(), bnd
+
+
+# --- a2..a5 ---------------------------------------------------------------------
+
+def select(scores: np.ndarray, loss_rate, share_weight, mode: int, k_critical: int, threshold: float,
+           seed: int, step: int, layer: int, force_all: bool = False):
+    G = scores.shape[0]
+    n = len(loss_rate)
+    s = _c(scores.astype(np.float32, copy=False))
+    lr = np.asarray(loss_rate, dtype=np.float64)
+    sw = np.asarray(share_weight, dtype=np.uint32)
+    order = np.empty(G, dtype=np.int32)
+    rank = np.empty(G, dtype=np.int32)
+    dev = np.empty(G, dtype=np.int32)
+    arrived = np.empty(max(n, 1), dtype=np.uint8)
+    keep = np.empty(G, dtype=np.uint8)
+    keep_list = np.empty(G, dtype=np.int32)
+    n_keep = np.zeros(1, dtype=np.int32)
+    status = np.zeros(1, dtype=np.uint32)
+    _check(lib().halo_ref_select(c_int(G), c_int(n), _p(lr), _p(sw), c_int(mode), c_int(k_critical),
+                                 c_float(threshold), c_uint64(seed), _p(s), c_uint32(step), c_uint32(layer),
+                                 c_int(1 if force_all else 0), _p(order), _p(rank), _p(dev), _p(arrived),
+                                 _p(keep), _p(keep_list), _p(n_keep), _p(status)), "select")
+    return dict(order=order, rank=rank, dev_of_group=dev, arrived=arrived[:n].copy(), keep=keep,
+                keep_list=keep_list, n_keep=int(n_keep[0]), status=int(status[0]))
+
+
+# --- a6..a8 ---------------------------------------------------------------------
+
+def group_ffn(Wpacked: np.ndarray, x: np.ndarray, group_list, dev_of_group=None, n_dev: int = 0,
+              want_group_partials: bool = False):
+    """-> partials float64 [n_dev+1][n_tok][d] (and per-group partials)."""
+    G, _, S, d = Wpacked.shape
+    dt = _dtype_of(Wpacked)
+    x2 = _c(x.reshape(-1, d))
+    assert _dtype_of(x2) == dt
+    n_tok = x2.shape[0]
+    Wpacked = _c(Wpacked)
+    lst = np.asarray(group_list, dtype=np.int32).reshape(-1)
+    dg = None if dev_of_group is None else _c(np.asarray(dev_of_group, dtype=np.int32))
+    P = np.empty((n_dev + 1, n_tok, d), dtype=np.float64)
+    gp = np.empty((max(len(lst), 1), n_tok, d), dtype=np.float64) if want_group_partials else None
+    _check(lib().halo_ref_group_ffn(c_int(d), c_int(G * S), c_int(S), c_int(dt), _p(Wpacked), _p(x2),
+                                    c_int(n_tok), _p(lst), c_int(len(lst)), _p(dg), c_int(n_dev), _p(P),
+                                    _p(gp)), "group_ffn")
+    if want_group_partials:
+        return P, gp[: len(lst)]
+    return P
+
+
+# --- a9 -------------------------------------------------------------------------
+
+def merge(partials: np.ndarray, arrived=None):
+    n_slots, n_tok, d = partials.shape
+    P = _c(partials.astype(np.float64, copy=False))
+    arr = None if arrived is None else _c(np.asarray(arrived, dtype=np.uint8))
+    y = np.empty((n_tok, d), dtype=np.float64)
+    _check(lib().halo_ref_merge(_p(P), _p(arr), c_int(n_slots - 1), c_int(n_tok), c_int(d), _p(y)), "merge")
+    return y
+
+
+# --- glue -----------------------------------------------------------------------
+
+def glue(h: np.ndarray, y, dtype: int):
+    """h' = h + y (y may be None), x = cast(rmsnorm(h')). -> (h', x)"""
+    h2 = _c(h.astype(np.float64, copy=False))
+    n_tok, d = h2.reshape(-1, h2.shape[-1]).shape
+    y2 = None if y is None else _c(np.asarray(y, dtype=np.float64))
+    h_out = np.empty((n_tok, d), dtype=np.float64)
+    x_out = np.empty((n_tok, d), dtype=np.float32 if dtype == F32 else np.uint16)
+    _check(lib().halo_ref_glue(c_int(d), c_int(n_tok), c_int(dtype), _p(h2), _p(y2), _p(h_out), _p(x_out)), "glue")
+    return h_out, x_out
+
+
+# --- a1..a9 for one layer ---------------------------------------------------------
+
+def layer(Wpacked, W1, W2, feat, x, loss_rate, share_weight, mode, k_critical, threshold, seed, step, layer_idx,
+          force_all=False, act=ACT_RELU):
+    G, _, S, d = Wpacked.shape
+    dt = _dtype_of(Wpacked)
+    r = W1.shape[0]
+    n = len(loss_rate)
+    x2 = _c(x.reshape(-1, d))
+    f2 = _c(feat.reshape(-1, d))
+    n_tok = x2.shape[0]
+    Wpacked, W1, W2 = _c(Wpacked), _c(W1), _c(W2)
+    lr = np.asarray(loss_rate, dtype=np.float64)
+    sw = np.asarray(share_weight, dtype=np.uint32)
+    scores = np.empty(G, dtype=np.float32)
+    order = np.empty(G, dtype=np.int32)
+    rank = np.empty(G, dtype=np.int32)
+    dev = np.empty(G, dtype=np.int32)
+    arrived = np.empty(max(n, 1), dtype=np.uint8)
+    keep = np.empty(G, dtype=np.uint8)
+    keep_list = np.empty(G, dtype=np.int32)
+    n_keep = np.zeros(1, dtype=np.int32)
+    status = np.zeros(1, dtype=np.uint32)
+    y = np.empty((n_tok, d), dtype=np.float64)
+    _check(lib().halo_ref_layer(c_int(d), c_int(G * S), c_int(S), c_int(dt), _p(Wpacked), c_int(r), c_int(act),
+                                _p(W1), _p(W2), c_int(n), _p(lr), _p(sw), c_int(mode), c_int(k_critical),
+                                c_float(threshold), c_uint64(seed), c_uint32(step), c_uint32(layer_idx),
+                                c_int(1 if force_all else 0), _p(f2), _p(x2), c_int(n_tok), _p(scores), _p(order),
+                                _p(rank), _p(dev), _p(arrived), _p(keep), _p(keep_list), _p(n_keep), _p(status),
+                                _p(y)), "layer")
+    return dict(scores=scores, order=order, rank=rank, dev_of_group=dev, arrived=arrived[:n].copy(), keep=keep,
+                keep_list=keep_list, n_keep=int(n_keep[0]), status=int(status[0]), y=y)

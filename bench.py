@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the group-sparse FFN hot path (predict -> select -> group FFN -> merge, chained as a stack).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl halo|reference]
+
+One step = one token through every block of the workload's FFN stack.  Prints ONE JSON line (rank 0).
+With N > 1 every rank runs an independent replica on its own GPU (the path has no exchange between GPUs).
+`--impl reference` times the CPU fp64 oracle on the host cores instead (a deliberately plain program).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2601_11676_b200 import synth  # noqa: E402
+
+METRIC = "group-sparse FFN decode tokens/s on 1 B200; achieved HBM GB/s vs ~8 TB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d.get("hbm_gbs", FALLBACK_HBM_GBS)), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons, mx = [], set(), None
+        try:
+            for ln in open(self.path):
+                f = [v.strip() for v in ln.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx = float(f[2])
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            busy = [v for v in sm if v >= 0.5 * max(sm)] or sm
+            out.update(sm_mhz=statistics.median(busy), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ----------------------------------------------------------------------------------------------------------------
+
+def build_stack(wl, dev):
+    from paper_2601_11676_b200 import binding as B
+    code = B.F32 if wl.dtype == "f32" else B.BF16
+    Wp = [synth.packed_layer(wl, l, dev) for l in range(wl.n_layers)]
+    preds = [synth.predictor(wl, l, dev) for l in range(wl.n_layers)]
+    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, B.SEL_TOPK, wl.k_critical, 0.0, wl.seed)
+    ffn = B.ffn_shape(wl.d_model, wl.d_ffn, wl.group_size, code)
+    pred = B.pred_shape(wl.d_model, wl.pred_rank, wl.n_groups, code)
+    stack = B.Stack(ffn, pred, wl.n_tok, plan, Wp, [p[0] for p in preds], [p[1] for p in preds])
+    return stack, Wp, preds, plan, ffn
+
+
+def run_halo(args, rank, world, local_rank):
+    from paper_2601_11676_b200 import binding as B
+    B.lib()  # fail loudly if the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    wl = synth.workload(args.workload, keep_permille=args.keep_permille)
+    K, W = args.steps, args.warmup
+    stack, Wp, preds, plan, ffn = build_stack(wl, dev)
+    L, G, d = wl.n_layers, wl.n_groups, wl.d_model
+    total_steps = W + K
+    h0 = torch.stack([synth.stream_input(wl, s, dev) for s in range(total_steps)])
+    h_out = torch.empty_like(h0)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    # ---- record the kept sets of the timed steps once (taps), for the byte accounting ------------------------
+    nk_rec = torch.zeros((total_steps, L), dtype=torch.int32, device=dev)
+    kl_rec = torch.zeros((total_steps, L, G), dtype=torch.int32, device=dev)
+    dg_rec = torch.zeros((total_steps, L, G), dtype=torch.int32, device=dev)
+    taps = B.Taps(None, None, dg_rec.data_ptr(), None, kl_rec.data_ptr(), nk_rec.data_ptr(), None)
+    stack.decode(h0, total_steps, 0, h_out, taps)
+    torch.cuda.synchronize()
+    if stack.status() != 0:
+        raise RuntimeError("device status: " + B.status_message(stack.status()))
+    nk_timed = nk_rec[W:].cpu().numpy().astype(np.int64)
+    kept_groups = int(nk_timed.sum())
+    kept_fraction = kept_groups / float(K * L * G)
+    weight_bytes = kept_groups * wl.group_bytes
+    pred_bytes = K * (L - 1) * wl.pred_bytes
+    algo_bytes_total = weight_bytes + pred_bytes
+
+    # ---- device-resident timing: W warm-up steps, then exactly K timed steps --------------------------------------
+    stack.decode(h0[:W], W, 0, h_out[:W])
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    stack.decode(h0[W:], K, W, h_out[W:])
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = stack.last_launches()
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end through the host entry point: pinned host buffers, copies inside the timed region ----------
+    h0_host = h0[W:].cpu().pin_memory()
+    out_host = torch.empty_like(h0_host).pin_memory()
+    stack.decode_host(h0_host[: max(W, 1)], max(W, 1), 0, out_host[: max(W, 1)])
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    stack.decode_host(h0_host, K, W, out_host)
+    e1.record()
+    torch.cuda.synchronize()
+    ms_e2e = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3)
+
+    # ---- dominant kernel alone: the group FFN of every block, one sweep over the stack per timing ---------------
+    x = synth.activation(wl, 1, dev)
+    partials = torch.empty((wl.n_dev + 1, 1, d), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    sweep_steps = list(range(W, W + min(K, 8)))
+    for l in range(L):  # warm-up sweep
+        B.halo_group_ffn(ffn, Wp[l], x, 1, kl_rec[W, l], nk_rec[W, l:l + 1], dg_rec[W, l], wl.n_dev, partials, None, status)
+    torch.cuda.synchronize()
+    k_ms, k_bytes, k_launches = 0.0, 0, 0
+    for s in sweep_steps:
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for l in range(L):
+            B.halo_group_ffn(ffn, Wp[l], x, 1, kl_rec[s, l], nk_rec[s, l:l + 1], dg_rec[s, l], wl.n_dev, partials, None,
+                             status)
+        b.record()
+        torch.cuda.synchronize()
+        k_ms += a.elapsed_time(b)
+        k_launches += L
+        k_bytes += int(nk_rec[s].sum().item()) * wl.group_bytes
+    kernel_avg_us = k_ms * 1e3 / k_launches
+    kernel_gbs = k_bytes / (k_ms * 1e-3) / 1e9
+
+    # ---- max over ranks -------------------------------------------------------------------------------------------
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        return None
+
+    peak, peak_kind = measured_peaks()
+    tokens = K * world
+    value = tokens / (ms * 1e-3)
+    step_gbs = algo_bytes_total / (ms * 1e-3) / 1e9
+    result = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": wl.dtype, "data": "synthetic",
+        "config": {"workload": wl.name, "n_layers": L, "d_model": d, "d_ffn": wl.d_ffn, "group_size": wl.group_size,
+                   "n_groups": G, "pred_rank": wl.pred_rank, "keep_permille": wl.keep_permille,
+                   "k_critical": wl.k_critical, "virtual_devices": wl.n_dev, "loss_rate": list(wl.loss_rate),
+                   "kept_fraction": kept_fraction, "l2": "inputs larger than L2 (weights of the stack: %.2f GB)"
+                   % (L * wl.layer_bytes / 1e9), "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "clocks": clocks,
+        "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 4 * d * wl.n_tok,
+                "d2h_bytes_per_step": 4 * d * wl.n_tok},
+        "gpu_launches": int(launches),
+        "hbm": {"algorithmic_gb_per_token": algo_bytes_total / K / 1e9, "achieved_gbs": step_gbs,
+                "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS, "frac_of_peak": step_gbs / peak,
+                "peak_gbs": peak, "peak_kind": peak_kind},
+        "roofline": {"bound": "hbm", "kernel": "group_ffn_decode_kernel", "achieved": kernel_gbs, "peak": peak,
+                     "unit": "GB/s", "frac": kernel_gbs / peak, "peak_kind": peak_kind, "traffic": None,
+                     "avg_launch_us": kernel_avg_us, "launches_timed": k_launches,
+                     "frac_of_nominal_8tbs": kernel_gbs / NOMINAL_HBM_GBS},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget)
+    return result
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# the oracle arm (CPU, fp64): reported baseline
+# ----------------------------------------------------------------------------------------------------------------
+
+def _oracle_layer_inputs(wl, layer):
+    hb = synth.host_bits
+    Wp = hb(synth.packed_layer(wl, layer, "cpu"))
+    w1, w2 = (hb(t) for t in synth.predictor(wl, layer, "cpu"))
+    feat = hb(synth.activation(wl, 2 * layer, "cpu"))
+    x = hb(synth.activation(wl, 2 * layer + 1, "cpu"))
+    return Wp, w1, w2, feat, x
+
+
+def cpu_baseline(wl, budget_s=15.0):
+    """Times the oracle as it stands on a bounded sample: whole blocks (predict, select, kept-group FFN, merge) of
+    one token, as many as fit the time budget; tokens/s is that block rate divided by the blocks per token."""
+    from oracle import halo_ref as R
+    cores = os.cpu_count() or 1
+    R.set_threads(cores)
+    R.lib()
+    done, spent = 0, 0.0
+    inputs = _oracle_layer_inputs(wl, 1)  # same shapes for every block; generated outside the timed part
+    while done < wl.n_layers and (done == 0 or spent + spent / done <= budget_s):
+        Wp, w1, w2, feat, x = inputs
+        t0 = time.perf_counter()
+        R.layer(Wp, w1, w2, feat, x, wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed, done,
+                1 + done % max(wl.n_layers - 1, 1))
+        spent += time.perf_counter() - t0
+        done += 1
+    value = (done / wl.n_layers) / spent
+    return {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "sample": f"{done} of {wl.n_layers} blocks of one token ({wl.name}), {spent:.1f} s of CPU time; "
+                      f"tokens/s extrapolated per token"}
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return None
+    from oracle import halo_ref as R
+    wl = synth.workload(args.workload, keep_permille=args.keep_permille)
+    cores = os.cpu_count() or 1
+    R.set_threads(cores)
+    K, W = args.steps, args.warmup
+    Wp, w1, w2, feat, x = _oracle_layer_inputs(wl, 1)
+    G = wl.n_groups
+    scores = R.predict(w1, w2, feat)
+
+    def one_step(step, n_groups_sample):
+        # a bounded sample of one block: predictor, selection, and the FFN of the first n kept groups
+        s = R.predict(w1, w2, feat)
+        sel = R.select(s, wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed, step, 1)
+        keep = sel["keep_list"][: min(sel["n_keep"], n_groups_sample)]
+        P = R.group_ffn(Wp, x, keep, sel["dev_of_group"], wl.n_dev)
+        R.merge(P)
+        return len(keep), sel["n_keep"]
+
+    # size the per-step sample so that W + K steps end within about two minutes
+    t0 = time.perf_counter()
+    g_done, _ = one_step(0, 4)
+    per_group = max((time.perf_counter() - t0) / max(g_done, 1), 1e-6)
+    budget_per_step = 120.0 / max(K + W, 1)
+    n_sample = int(max(1, min(G, budget_per_step / per_group)))
+    for s in range(W):
+        one_step(s, n_sample)
+    groups, kept_total = 0, 0
+    t0 = time.perf_counter()
+    for s in range(K):
+        g, nk = one_step(W + s, n_sample)
+        groups += g
+        kept_total += nk
+    dt = time.perf_counter() - t0
+    # tokens/s: a token costs (average kept groups per block) x (blocks) group evaluations
+    groups_per_token = (kept_total / K) * wl.n_layers
+    value = (groups / groups_per_token) / dt
+    sample = (f"each step = predictor + selection + FFN of {n_sample} kept groups of one block ({wl.name}); "
+              f"tokens/s extrapolated by groups per token ({groups_per_token:.0f})")
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": dt * 1e3 / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "keep_permille": wl.keep_permille},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="halo", choices=["halo", "reference"])
+    ap.add_argument("--workload", default="llama2-7b-decode", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--keep-permille", type=int, default=500)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "halo" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        res = run_reference(args, rank, world)
+        if res is not None:
+            print(json.dumps(res), flush=True)
+        return 0
+
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        torch.distributed.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    try:
+        res = run_halo(args, rank, world, local_rank)
+        if res is not None:
+            print(json.dumps(res), flush=True)
+    finally:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

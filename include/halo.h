@@ -1,0 +1,247 @@
+/*
+ * halo.h -- C ABI of libhalo: the group-sparse FFN hot path of HALO
+ * (arXiv 2601.11676) for NVIDIA B200 (sm_100a).
+ *
+ * Path: predictor scores per FFN neuron group -> rank / critical choice /
+ * assignment of the less-critical groups to virtual unstable devices /
+ * seeded per-device arrival mask -> SwiGLU FFN over the kept groups only,
+ * accumulated per holder -> merge of the partials that arrived.
+ *
+ * Conventions
+ *   - Every function returns a halo_status (0 = HALO_OK, negative = error).
+ *     Argument errors are found on the host before anything is launched.
+ *   - Pointers marked "device" are CUDA device pointers owned by the caller,
+ *     16-byte aligned; pointers marked "host" are ordinary host memory.
+ *   - GPU entry points enqueue work on `stream` (a cudaStream_t passed as
+ *     void*; NULL = the default stream) and return without synchronising.
+ *     They allocate nothing and print nothing.  Scratch memory, where a call
+ *     needs it, is a caller-owned device `workspace` whose size the matching
+ *     *_workspace_bytes function reports.
+ *   - Conditions found on the device (non-finite score, out-of-range group
+ *     index, a wait that ran out) are OR-ed into the caller-owned device word
+ *     `dev_status` (may be NULL); read it after synchronising and decode it
+ *     with halo_status_message.
+ *   - Element type of weights and activations is `halo_dtype`; scores,
+ *     partials and outputs are fp32.
+ *
+ * Weight layout (Sec. II-A, "neuron group": a group owns its gate rows, its
+ * up rows and the matching down-projection columns):
+ *     W_packed[G][3][S][d]   G = d_ffn / group_size, S = group_size, d = d_model
+ *     plane 0: gate rows, plane 1: up rows,
+ *     plane 2: the group's down-projection columns, each stored as a row of d.
+ *   One group is one contiguous block of 3*S*d elements, so a skipped group is
+ *   a skipped address range.
+ */
+#ifndef HALO_H
+#define HALO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int halo_status;
+enum {
+    HALO_OK = 0,
+    HALO_ERR_ARG = -1,           /* NULL pointer, value out of range */
+    HALO_ERR_SHAPE = -2,         /* sizes that do not divide / exceed limits */
+    HALO_ERR_ALIGN = -3,         /* a device pointer is not 16-byte aligned */
+    HALO_ERR_DTYPE = -4,         /* dtype not supported by this entry point */
+    HALO_ERR_CUDA = -5,          /* a CUDA runtime call failed */
+    HALO_ERR_NOMEM = -6,         /* host or device allocation failed (create calls only) */
+    HALO_ERR_UNIMPLEMENTED = -7,
+    HALO_ERR_WORKSPACE = -8      /* workspace missing or too small */
+};
+
+/* bits of the device status word */
+#define HALO_DEV_NONFINITE_SCORE 1u  /* a score was NaN (ranked lowest) or infinite */
+#define HALO_DEV_BAD_INDEX 2u        /* a group id or device id was out of range; the item was skipped */
+#define HALO_DEV_TIMEOUT 4u          /* a bounded device-side wait ran out */
+
+#define HALO_MAX_DEVICES 32
+#define HALO_MAX_GROUPS 1024
+
+typedef enum { HALO_F32 = 0, HALO_BF16 = 1 } halo_dtype;
+typedef enum { HALO_SEL_TOPK = 0, HALO_SEL_THRESHOLD = 1 } halo_sel_mode;
+typedef enum { HALO_ACT_RELU = 0, HALO_ACT_NONE = 1 } halo_pred_act;
+
+/* d_ffn % group_size == 0; d_model % 8 == 0; d_ffn / group_size <= HALO_MAX_GROUPS. */
+typedef struct {
+    int d_model, d_ffn, group_size;
+    halo_dtype wdtype;
+} halo_ffn_shape;
+
+/* Predictor d_in -> rank -> n_groups; d_in % 8 == 0, rank % 8 == 0. */
+typedef struct {
+    int d_in, rank, n_groups;
+    halo_dtype wdtype;
+    halo_pred_act act;
+} halo_pred_shape;
+
+typedef struct halo_plan halo_plan;   /* host object: Assignment-phase tables */
+typedef struct halo_stack halo_stack; /* host object owning device work buffers of an FFN stack */
+
+const char* halo_status_string(halo_status s);
+/* Writes a comma-separated description of the bits of a device status word. */
+halo_status halo_status_message(uint32_t dev_status_value, char* msg /*host*/, int msg_len);
+
+/* ------------------------------------------------------------------------
+ * Assignment phase (Sec. III-B.4, Algorithm 3: PLR-aware ratio-guided
+ * scheduler).  Host only, one-off.
+ *   loss_rate[n_dev]    (host) packet-loss rate rho_i in [0,1] of virtual device i
+ *   share_weight[n_dev] (host) integer workload ratio r_i (any common scale; sum > 0)
+ *   mode / k_critical / threshold: how the critical groups (kept by the
+ *     reliable master, never dropped) are chosen from the scores: the k
+ *     highest, or those with score >= threshold.
+ *   seed: key of the arrival draws.
+ * Devices are ordered by ascending loss rate (ties: lower index).  The M
+ * less-critical groups, in priority order, are cut into n_dev contiguous
+ * chunks; the cut after the j-th device in that order is
+ * floor((2*M*C_j + C_n) / (2*C_n)), C_j = cumulative weight.  n_dev may be 0.
+ * Errors: HALO_ERR_ARG for a rate outside [0,1], all-zero weights, k out of
+ * range, NULL pointers; HALO_ERR_SHAPE for n_groups/n_dev beyond the limits.
+ * The plan is owned by the library until halo_plan_destroy.
+ * ---------------------------------------------------------------------- */
+halo_status halo_plan_create(halo_plan** out, int n_groups, int n_dev, const double* loss_rate,
+                             const uint32_t* share_weight, halo_sel_mode mode, int k_critical,
+                             float threshold, uint64_t seed);
+halo_status halo_plan_destroy(halo_plan* plan);
+/* For inspection: device order (ascending loss), the 33-bit loss thresholds
+ * T_i = round(rho_i * 2^32) by device index, and the n_dev+1 chunk boundaries
+ * for M less-critical groups.  All host arrays; any may be NULL. */
+halo_status halo_plan_describe(const halo_plan* plan, int M, int32_t* dev_order, uint64_t* loss_thresh,
+                               int32_t* boundaries);
+
+/* ------------------------------------------------------------------------
+ * a1. Predictor (Sec. III-B.2, semantic-aware predictors): importance score
+ * of every neuron group of a block from semantic features taken one layer
+ * ahead.  Bias-free two-layer network
+ *     z = act(W1 * f),  s = W2 * z
+ *   W1   device [rank][d_in]      (row u = weights of hidden unit u)
+ *   W2   device [n_groups][rank]
+ *   feat device [n_tok][d_in], wdtype
+ *   scores device fp32: [n_groups] if n_tok == 1 or mean_pool != 0 (mean over
+ *     the tokens of the per-token scores, fixed token order), else [n_tok][n_groups]
+ *   workspace: halo_predict_workspace_bytes(shape, n_tok) bytes, device.
+ * fp32 accumulation.  Sets HALO_DEV_NONFINITE_SCORE if a score is not finite.
+ * ---------------------------------------------------------------------- */
+size_t halo_predict_workspace_bytes(const halo_pred_shape* shape, int n_tok);
+halo_status halo_predict_groups(const halo_pred_shape* shape, const void* W1, const void* W2,
+                                const void* feat, int n_tok, int mean_pool, float* scores,
+                                void* workspace, size_t workspace_bytes, uint32_t* dev_status, void* stream);
+
+/* ------------------------------------------------------------------------
+ * a2..a5. Rank, critical choice, runtime assignment and arrival mask
+ * (Sec. III-B.3, Pred process: the importance rank indexes the priority
+ * lists fixed by the Assignment phase; relaxed synchronisation: the master
+ * merges what arrived).
+ *   scores device fp32 [G].  Order = higher score first, equal scores by
+ *     lower group id; NaN ranks as -inf (status bit), -0 equals +0.
+ *   step, layer: counter of the arrival draw.  Device i's partial of this
+ *     (step, layer) arrives iff word 0 of Philox4x32-10 with counter
+ *     (step, layer, i, 0) and key (seed low, seed high) is >= T_i.
+ *   force_all != 0: a reliable block (the first layer): everything arrives.
+ * Outputs (device; any of order/dev_of_group/arrived/keep may be NULL):
+ *   order[G]        group id at each priority position
+ *   dev_of_group[G] holder of each group: -1 = master (critical), else device index
+ *   arrived[n_dev]  1 if the device's partial arrives
+ *   keep[G]         1 if the group's contribution survives
+ *   keep_list[G]    kept group ids, ascending, then -1 padding
+ *   n_keep[1]       number of kept groups
+ * One thread block; G <= HALO_MAX_GROUPS.
+ * ---------------------------------------------------------------------- */
+halo_status halo_select_groups(const halo_plan* plan, const float* scores, uint32_t step, uint32_t layer,
+                               int force_all, int32_t* order, int32_t* dev_of_group, uint8_t* arrived,
+                               uint8_t* keep, int32_t* keep_list, int32_t* n_keep, uint32_t* dev_status,
+                               void* stream);
+
+/* ------------------------------------------------------------------------
+ * a6..a8. Group-masked SwiGLU FFN (Sec. II-A neuron groups; Sec. II-B: the
+ * merged features are the sum of the groups' activations).  For each kept
+ * group g and neuron j of it
+ *     a = <gate_j, x>, b = <up_j, x>, h = a / (1 + exp(-a)) * b,
+ *     partials[slot(g)] += h * down_j,   slot = dev_of_group[g] + 1 (0 = master)
+ *   W_packed device, layout above;  x device [n_tok][d], wdtype
+ *   keep_list device [>= *n_keep] group ids; n_keep device [1]
+ *   dev_of_group device [G] or NULL (everything into slot 0; then n_dev is 0)
+ *   partials device fp32 [n_dev+1][n_tok][d]; overwritten (zeroed by the call)
+ *   workspace: halo_group_ffn_workspace_bytes(shape, n_tok, n_dev) bytes, device
+ * Groups that are not listed cost no memory traffic.  bf16/fp32 inputs, fp32
+ * accumulation.  n_tok == 1 runs the bandwidth-bound decode kernel; larger
+ * n_tok with bf16 weights runs the tensor-core contraction.  Out-of-range ids
+ * are skipped and flagged HALO_DEV_BAD_INDEX.
+ * ---------------------------------------------------------------------- */
+size_t halo_group_ffn_workspace_bytes(const halo_ffn_shape* shape, int n_tok, int n_dev);
+halo_status halo_group_ffn(const halo_ffn_shape* shape, const void* W_packed, const void* x, int n_tok,
+                           const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
+                           int n_dev, float* partials, void* workspace, size_t workspace_bytes,
+                           uint32_t* dev_status, void* stream);
+
+/* ------------------------------------------------------------------------
+ * a9. Merge (Sec. III-B.3: after the timeout the master merges the
+ * activations that are available): y = partials[0] + sum_i arrived[i] * partials[i+1].
+ *   partials device fp32 [n_dev+1][n_tok][d]; arrived device [n_dev] or NULL (all)
+ *   y device fp32 [n_tok][d]
+ * ---------------------------------------------------------------------- */
+halo_status halo_merge_partials(const float* partials, const uint8_t* arrived, int n_dev, int n_tok,
+                                int d_model, float* y, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Helpers around the path.
+ * halo_pack_weights: Wgate[F][d], Wup[F][d], Wdown[d][F] (device) -> W_packed (device).
+ * halo_glue: element-wise work between the blocks of an FFN stack (Sec. II-A:
+ *   normalisation and residual connection): h_out = h + y (y may be NULL),
+ *   x_out = cast(h_out / sqrt(mean(h_out^2) + 1e-5)) per token.
+ *   h, y, h_out device fp32 [n_tok][d] (h_out may alias h); x_out device [n_tok][d] in `xdtype`.
+ * ---------------------------------------------------------------------- */
+halo_status halo_pack_weights(const halo_ffn_shape* shape, const void* Wgate, const void* Wup,
+                              const void* Wdown, void* W_packed, void* stream);
+halo_status halo_glue(int d_model, int n_tok, halo_dtype xdtype, const float* h, const float* y, float* h_out,
+                      void* x_out, void* stream);
+
+/* ------------------------------------------------------------------------
+ * FFN stack: L blocks chained by halo_glue, the predictor of block l reading
+ * the input of block l-1 (one layer ahead, Sec. III-B.2) and block 0 reliable
+ * (Sec. III-B.3: the first layer has no semantic information yet).
+ * halo_stack_create copies the per-layer pointer tables and allocates the
+ * device work buffers it owns (freed by halo_stack_destroy); the weights stay
+ * caller-owned and must outlive the stack.
+ *   W_packed[L], W1[L], W2[L]: host arrays of device pointers (W1[0], W2[0] unused, may be NULL)
+ * ---------------------------------------------------------------------- */
+typedef struct {
+    void* x;              /* device [steps][L][n_tok][d] wdtype: input of every block */
+    float* scores;        /* device [steps][L][G] (block 0: zeros) */
+    int32_t* dev_of_group;/* device [steps][L][G] */
+    uint8_t* arrived;     /* device [steps][L][n_dev] */
+    int32_t* keep_list;   /* device [steps][L][G] */
+    int32_t* n_keep;      /* device [steps][L] */
+    float* y;             /* device [steps][L][n_tok][d]: merged output of every block */
+} halo_taps;              /* any member may be NULL */
+
+halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred,
+                              int n_layers, int n_tok, const halo_plan* plan, const void* const* W_packed,
+                              const void* const* W1, const void* const* W2);
+halo_status halo_stack_destroy(halo_stack* stack);
+/* Runs `steps` tokens (or prompts of n_tok tokens) through the stack.
+ *   h0    device fp32 [steps][n_tok][d]: residual-stream input of each step
+ *   h_out device fp32 [steps][n_tok][d]: residual stream after the last block
+ *   step0: arrival-draw counter of the first step
+ *   taps: NULL or per-block records for checking
+ * Asynchronous on `stream`; no host synchronisation inside. */
+halo_status halo_stack_decode(halo_stack* stack, const float* h0, int steps, uint32_t step0, float* h_out,
+                              const halo_taps* taps, void* stream);
+/* Same with HOST buffers (pinned memory recommended): copies h0 in, runs,
+ * copies h_out back and synchronises the stream before returning. */
+halo_status halo_stack_decode_host(halo_stack* stack, const float* h0_host, int steps, uint32_t step0,
+                                   float* h_out_host, void* stream);
+/* Device status word accumulated by the stack's launches (synchronises the stream). */
+halo_status halo_stack_status(halo_stack* stack, uint32_t* dev_status_value /*host*/, void* stream);
+/* Number of kernel launches the last halo_stack_decode enqueued. */
+long long halo_stack_last_launches(const halo_stack* stack);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HALO_H */

@@ -1,0 +1,254 @@
+"""Thin ctypes binding of libhalo.so: same names as include/halo.h, argument marshalling only.
+
+Tensors are torch CUDA tensors (device memory and streams are torch's); every
+step of the path runs inside the library's kernels.  The library must have been
+built (``python -m paper_2601_11676_b200.build``); there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_float, c_int, c_int32, c_longlong, c_size_t, \
+    c_uint8, c_uint32, c_uint64, c_void_p
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libhalo.so")
+
+F32, BF16 = 0, 1
+SEL_TOPK, SEL_THRESHOLD = 0, 1
+ACT_RELU, ACT_NONE = 0, 1
+DEV_NONFINITE_SCORE, DEV_BAD_INDEX, DEV_TIMEOUT = 1, 2, 4
+MAX_DEVICES, MAX_GROUPS = 32, 1024
+
+EXPORTS = [
+    "halo_status_string", "halo_status_message", "halo_plan_create", "halo_plan_destroy", "halo_plan_describe",
+    "halo_predict_workspace_bytes", "halo_predict_groups", "halo_select_groups", "halo_group_ffn_workspace_bytes",
+    "halo_group_ffn", "halo_merge_partials", "halo_pack_weights", "halo_glue", "halo_stack_create",
+    "halo_stack_destroy", "halo_stack_decode", "halo_stack_decode_host", "halo_stack_status",
+    "halo_stack_last_launches",
+]
+
+
+class FfnShape(Structure):
+    _fields_ = [("d_model", c_int), ("d_ffn", c_int), ("group_size", c_int), ("wdtype", c_int)]
+
+
+class PredShape(Structure):
+    _fields_ = [("d_in", c_int), ("rank", c_int), ("n_groups", c_int), ("wdtype", c_int), ("act", c_int)]
+
+
+class Taps(Structure):
+    _fields_ = [("x", c_void_p), ("scores", c_void_p), ("dev_of_group", c_void_p), ("arrived", c_void_p),
+                ("keep_list", c_void_p), ("n_keep", c_void_p), ("y", c_void_p)]
+
+
+class HaloError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: status {code} ({status_string(code)})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libhalo.so; raises if it is missing (no CPU or eager fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2601_11676_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        L.halo_status_string.restype = c_char_p
+        L.halo_status_string.argtypes = [c_int]
+        L.halo_predict_workspace_bytes.restype = c_size_t
+        L.halo_predict_workspace_bytes.argtypes = [POINTER(PredShape), c_int]
+        L.halo_group_ffn_workspace_bytes.restype = c_size_t
+        L.halo_group_ffn_workspace_bytes.argtypes = [POINTER(FfnShape), c_int, c_int]
+        L.halo_stack_last_launches.restype = c_longlong
+        L.halo_stack_last_launches.argtypes = [c_void_p]
+        L.halo_plan_create.argtypes = [POINTER(c_void_p), c_int, c_int, POINTER(c_double), POINTER(c_uint32), c_int,
+                                       c_int, c_float, c_uint64]
+        L.halo_plan_destroy.argtypes = [c_void_p]
+        L.halo_plan_describe.argtypes = [c_void_p, c_int, POINTER(c_int32), POINTER(c_uint64), POINTER(c_int32)]
+        L.halo_predict_groups.argtypes = [POINTER(PredShape), c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p,
+                                          c_void_p, c_size_t, c_void_p, c_void_p]
+        L.halo_select_groups.argtypes = [c_void_p, c_void_p, c_uint32, c_uint32, c_int, c_void_p, c_void_p, c_void_p,
+                                         c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.halo_group_ffn.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int,
+                                     c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
+        L.halo_merge_partials.argtypes = [c_void_p, c_void_p, c_int, c_int, c_int, c_void_p, c_void_p]
+        L.halo_pack_weights.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.halo_glue.argtypes = [c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.halo_stack_create.argtypes = [POINTER(c_void_p), POINTER(FfnShape), POINTER(PredShape), c_int, c_int,
+                                        c_void_p, POINTER(c_void_p), POINTER(c_void_p), POINTER(c_void_p)]
+        L.halo_stack_destroy.argtypes = [c_void_p]
+        L.halo_stack_decode.argtypes = [c_void_p, c_void_p, c_int, c_uint32, c_void_p, POINTER(Taps), c_void_p]
+        L.halo_stack_decode_host.argtypes = [c_void_p, c_void_p, c_int, c_uint32, c_void_p, c_void_p]
+        L.halo_stack_status.argtypes = [c_void_p, POINTER(c_uint32), c_void_p]
+        L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().halo_status_string(code).decode()
+
+
+def status_message(value: int) -> str:
+    buf = ctypes.create_string_buffer(128)
+    lib().halo_status_message(value, buf, 128)
+    return buf.value.decode()
+
+
+def _chk(code: int, what: str) -> None:
+    if code != 0:
+        raise HaloError(code, what)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device-contiguous tensor expected"
+    return c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return c_void_p(s.cuda_stream)
+
+
+def ffn_shape(d_model: int, d_ffn: int, group_size: int, dtype: int) -> FfnShape:
+    return FfnShape(d_model, d_ffn, group_size, dtype)
+
+
+def pred_shape(d_in: int, rank: int, n_groups: int, dtype: int, act: int = ACT_RELU) -> PredShape:
+    return PredShape(d_in, rank, n_groups, dtype, act)
+
+
+class Plan:
+    """halo_plan_create / halo_plan_destroy."""
+
+    def __init__(self, n_groups, loss_rate, share_weight, mode=SEL_TOPK, k_critical=0, threshold=0.0, seed=0):
+        n = len(loss_rate)
+        self.n_groups, self.n_dev = n_groups, n
+        lr = (c_double * max(n, 1))(*[float(v) for v in loss_rate])
+        sw = (c_uint32 * max(n, 1))(*[int(v) for v in share_weight])
+        self.handle = c_void_p()
+        _chk(lib().halo_plan_create(byref(self.handle), n_groups, n, lr, sw, mode, k_critical, threshold, seed),
+             "halo_plan_create")
+
+    def describe(self, M: int):
+        n = self.n_dev
+        order = (c_int32 * max(n, 1))()
+        thr = (c_uint64 * max(n, 1))()
+        bnd = (c_int32 * (n + 1))()
+        _chk(lib().halo_plan_describe(self.handle, M, order, thr, bnd), "halo_plan_describe")
+        return list(order)[:n], list(thr)[:n], list(bnd)
+
+    def close(self):
+        if self.handle:
+            lib().halo_plan_destroy(self.handle)
+            self.handle = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def halo_predict_workspace_bytes(shape: PredShape, n_tok: int) -> int:
+    return int(lib().halo_predict_workspace_bytes(byref(shape), n_tok))
+
+
+def halo_predict_groups(shape: PredShape, W1, W2, feat, n_tok, mean_pool, scores, workspace, dev_status=None,
+                        stream=None) -> None:
+    _chk(lib().halo_predict_groups(byref(shape), _ptr(W1), _ptr(W2), _ptr(feat), n_tok, int(bool(mean_pool)),
+                                   _ptr(scores), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                   _ptr(dev_status), _stream(stream)), "halo_predict_groups")
+
+
+def halo_select_groups(plan: Plan, scores, step, layer, force_all, order, dev_of_group, arrived, keep, keep_list,
+                       n_keep, dev_status=None, stream=None) -> None:
+    _chk(lib().halo_select_groups(plan.handle, _ptr(scores), step, layer, int(bool(force_all)), _ptr(order),
+                                  _ptr(dev_of_group), _ptr(arrived), _ptr(keep), _ptr(keep_list), _ptr(n_keep),
+                                  _ptr(dev_status), _stream(stream)), "halo_select_groups")
+
+
+def halo_group_ffn_workspace_bytes(shape: FfnShape, n_tok: int, n_dev: int) -> int:
+    return int(lib().halo_group_ffn_workspace_bytes(byref(shape), n_tok, n_dev))
+
+
+def halo_group_ffn(shape: FfnShape, W_packed, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials,
+                   workspace=None, dev_status=None, stream=None) -> None:
+    _chk(lib().halo_group_ffn(byref(shape), _ptr(W_packed), _ptr(x), n_tok, _ptr(keep_list), _ptr(n_keep),
+                              _ptr(dev_of_group), n_dev, _ptr(partials), _ptr(workspace),
+                              workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                              _ptr(dev_status), _stream(stream)), "halo_group_ffn")
+
+
+def halo_merge_partials(partials, arrived, n_dev, n_tok, d_model, y, stream=None) -> None:
+    _chk(lib().halo_merge_partials(_ptr(partials), _ptr(arrived), n_dev, n_tok, d_model, _ptr(y), _stream(stream)),
+         "halo_merge_partials")
+
+
+def halo_pack_weights(shape: FfnShape, Wgate, Wup, Wdown, W_packed, stream=None) -> None:
+    _chk(lib().halo_pack_weights(byref(shape), _ptr(Wgate), _ptr(Wup), _ptr(Wdown), _ptr(W_packed), _stream(stream)),
+         "halo_pack_weights")
+
+
+def halo_glue(d_model, n_tok, xdtype, h, y, h_out, x_out, stream=None) -> None:
+    _chk(lib().halo_glue(d_model, n_tok, xdtype, _ptr(h), _ptr(y), _ptr(h_out), _ptr(x_out), _stream(stream)),
+         "halo_glue")
+
+
+class Stack:
+    """halo_stack_create / halo_stack_decode / halo_stack_destroy.  Keeps the weight tensors alive."""
+
+    def __init__(self, ffn: FfnShape, pred: PredShape, n_tok: int, plan: Plan, W_packed, W1, W2):
+        L = len(W_packed)
+        self._keep = (list(W_packed), list(W1), list(W2), plan)
+        self.ffn, self.pred, self.n_layers, self.n_tok, self.plan = ffn, pred, L, n_tok, plan
+        arr = lambda ts: (c_void_p * L)(*[(t.data_ptr() if t is not None else None) for t in ts])
+        self.handle = c_void_p()
+        _chk(lib().halo_stack_create(byref(self.handle), byref(ffn), byref(pred), L, n_tok, plan.handle,
+                                     arr(W_packed), arr(W1), arr(W2)), "halo_stack_create")
+
+    def decode(self, h0, steps, step0, h_out, taps: Taps | None = None, stream=None) -> None:
+        _chk(lib().halo_stack_decode(self.handle, _ptr(h0), steps, step0, _ptr(h_out),
+                                     byref(taps) if taps is not None else None, _stream(stream)), "halo_stack_decode")
+
+    def decode_host(self, h0_host: torch.Tensor, steps, step0, h_out_host: torch.Tensor, stream=None) -> None:
+        assert not h0_host.is_cuda and not h_out_host.is_cuda
+        _chk(lib().halo_stack_decode_host(self.handle, c_void_p(h0_host.data_ptr()), steps, step0,
+                                          c_void_p(h_out_host.data_ptr()), _stream(stream)), "halo_stack_decode_host")
+
+    def status(self, stream=None) -> int:
+        v = c_uint32(0)
+        _chk(lib().halo_stack_status(self.handle, byref(v), _stream(stream)), "halo_stack_status")
+        return int(v.value)
+
+    def last_launches(self) -> int:
+        return int(lib().halo_stack_last_launches(self.handle))
+
+    def close(self):
+        if self.handle:
+            lib().halo_stack_destroy(self.handle)
+            self.handle = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

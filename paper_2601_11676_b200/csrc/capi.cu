@@ -1,0 +1,434 @@
+// extern "C" surface of libhalo: argument checks, the host-side Assignment phase, and the stack runner.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace halo;
+
+namespace {
+
+bool valid_dtype(int t) { return t == HALO_F32 || t == HALO_BF16; }
+size_t elem_size(halo_dtype t) { return t == HALO_F32 ? 4 : 2; }
+
+halo_status check_ffn_shape(const halo_ffn_shape* s) {
+    if (!s) return HALO_ERR_ARG;
+    if (!valid_dtype(s->wdtype)) return HALO_ERR_DTYPE;
+    if (s->d_model <= 0 || s->d_ffn <= 0 || s->group_size <= 0) return HALO_ERR_SHAPE;
+    if (s->d_model % 8 != 0 || s->d_ffn % s->group_size != 0) return HALO_ERR_SHAPE;
+    if (s->d_ffn / s->group_size > HALO_MAX_GROUPS) return HALO_ERR_SHAPE;
+    const int per_chunk = s->wdtype == HALO_F32 ? 4 : 8;
+    if (s->d_model / per_chunk > 1024) return HALO_ERR_SHAPE;  // decode kernel: at most 4 chunks per thread
+    return HALO_OK;
+}
+
+halo_status check_pred_shape(const halo_pred_shape* s) {
+    if (!s) return HALO_ERR_ARG;
+    if (!valid_dtype(s->wdtype)) return HALO_ERR_DTYPE;
+    if (s->act != HALO_ACT_RELU && s->act != HALO_ACT_NONE) return HALO_ERR_ARG;
+    if (s->d_in <= 0 || s->rank <= 0 || s->n_groups <= 0) return HALO_ERR_SHAPE;
+    if (s->d_in % 8 != 0 || s->rank % 8 != 0) return HALO_ERR_SHAPE;
+    if (s->d_in > 12288 || s->rank > 8192 || s->n_groups > HALO_MAX_GROUPS) return HALO_ERR_SHAPE;
+    return HALO_OK;
+}
+
+unsigned long long loss_threshold(double rho) {
+    if (!(rho > 0.0)) return 0ull;
+    if (rho >= 1.0) return 1ull << 32;
+    double t = std::floor(rho * 4294967296.0 + 0.5);
+    if (t > 4294967296.0) t = 4294967296.0;
+    return static_cast<unsigned long long>(t);
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------------
+
+extern "C" const char* halo_status_string(halo_status s) {
+    switch (s) {
+        case HALO_OK: return "ok";
+        case HALO_ERR_ARG: return "bad argument";
+        case HALO_ERR_SHAPE: return "unsupported shape";
+        case HALO_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case HALO_ERR_DTYPE: return "unsupported dtype";
+        case HALO_ERR_CUDA: return "CUDA call failed";
+        case HALO_ERR_NOMEM: return "out of memory";
+        case HALO_ERR_UNIMPLEMENTED: return "not implemented";
+        case HALO_ERR_WORKSPACE: return "workspace missing or too small";
+        default: return "unknown status";
+    }
+}
+
+extern "C" halo_status halo_status_message(uint32_t v, char* msg, int msg_len) {
+    if (!msg || msg_len <= 0) return HALO_ERR_ARG;
+    std::snprintf(msg, static_cast<size_t>(msg_len), "%s%s%s%s",
+                  v == 0 ? "clean" : "",
+                  (v & HALO_DEV_NONFINITE_SCORE) ? "non-finite score;" : "",
+                  (v & HALO_DEV_BAD_INDEX) ? "index out of range;" : "",
+                  (v & HALO_DEV_TIMEOUT) ? "device wait timed out;" : "");
+    return HALO_OK;
+}
+
+// ---- Assignment phase (Algorithm 3) ------------------------------------------------------------------
+
+extern "C" halo_status halo_plan_create(halo_plan** out, int n_groups, int n_dev, const double* loss_rate,
+                                        const uint32_t* share_weight, halo_sel_mode mode, int k_critical,
+                                        float threshold, uint64_t seed) {
+    if (!out) return HALO_ERR_ARG;
+    *out = nullptr;
+    if (n_groups <= 0 || n_groups > HALO_MAX_GROUPS || n_dev < 0 || n_dev > HALO_MAX_DEVICES) return HALO_ERR_SHAPE;
+    if (n_dev > 0 && (!loss_rate || !share_weight)) return HALO_ERR_ARG;
+    if (mode != HALO_SEL_TOPK && mode != HALO_SEL_THRESHOLD) return HALO_ERR_ARG;
+    if (mode == HALO_SEL_TOPK && (k_critical < 0 || k_critical > n_groups)) return HALO_ERR_ARG;
+    if (mode == HALO_SEL_THRESHOLD && std::isnan(threshold)) return HALO_ERR_ARG;
+    unsigned long long total = 0;
+    for (int i = 0; i < n_dev; ++i) {
+        if (!(loss_rate[i] >= 0.0 && loss_rate[i] <= 1.0)) return HALO_ERR_ARG;
+        total += share_weight[i];
+    }
+    if (n_dev > 0 && total == 0) return HALO_ERR_ARG;
+    halo_plan* p = new (std::nothrow) halo_plan();
+    if (!p) return HALO_ERR_NOMEM;
+    std::memset(p, 0, sizeof(*p));
+    p->n_groups = n_groups;
+    p->n_dev = n_dev;
+    PlanDev& dv = p->dev;
+    dv.n_dev = n_dev;
+    dv.mode = mode;
+    dv.k_critical = mode == HALO_SEL_TOPK ? k_critical : 0;
+    dv.threshold = threshold;
+    dv.seed_lo = static_cast<uint32_t>(seed & 0xffffffffull);
+    dv.seed_hi = static_cast<uint32_t>(seed >> 32);
+    for (int i = 0; i < n_dev; ++i) {
+        p->loss_rate[i] = loss_rate[i];
+        p->share_weight[i] = share_weight[i];
+        dv.loss_thresh[i] = loss_threshold(loss_rate[i]);
+        dv.dev_order[i] = i;
+    }
+    // q = argsort(rho ascending), ties keep the lower device index first
+    std::stable_sort(dv.dev_order, dv.dev_order + n_dev,
+                     [&](int a, int b) { return p->loss_rate[a] < p->loss_rate[b]; });
+    unsigned long long cum = 0;
+    for (int j = 0; j < n_dev; ++j) {
+        cum += p->share_weight[dv.dev_order[j]];
+        dv.cum_weight[j] = cum;
+    }
+    *out = p;
+    return HALO_OK;
+}
+
+extern "C" halo_status halo_plan_destroy(halo_plan* plan) {
+    delete plan;
+    return HALO_OK;
+}
+
+extern "C" halo_status halo_plan_describe(const halo_plan* plan, int M, int32_t* dev_order, uint64_t* loss_thresh,
+                                          int32_t* boundaries) {
+    if (!plan || M < 0) return HALO_ERR_ARG;
+    const PlanDev& dv = plan->dev;
+    for (int i = 0; i < plan->n_dev; ++i) {
+        if (dev_order) dev_order[i] = dv.dev_order[i];
+        if (loss_thresh) loss_thresh[i] = dv.loss_thresh[i];
+    }
+    if (boundaries) {
+        boundaries[0] = 0;
+        if (plan->n_dev > 0) {
+            const unsigned long long total = dv.cum_weight[plan->n_dev - 1];
+            for (int j = 1; j < plan->n_dev; ++j)
+                boundaries[j] = static_cast<int32_t>(
+                    (2ull * static_cast<unsigned long long>(M) * dv.cum_weight[j - 1] + total) / (2ull * total));
+            boundaries[plan->n_dev] = M;
+        }
+    }
+    return HALO_OK;
+}
+
+// ---- a1 ---------------------------------------------------------------------------------------------
+
+extern "C" size_t halo_predict_workspace_bytes(const halo_pred_shape* shape, int n_tok) {
+    if (check_pred_shape(shape) != HALO_OK || n_tok <= 0) return 0;
+    return sizeof(float) * static_cast<size_t>(n_tok) * (static_cast<size_t>(shape->rank) + shape->n_groups);
+}
+
+extern "C" halo_status halo_predict_groups(const halo_pred_shape* shape, const void* W1, const void* W2,
+                                           const void* feat, int n_tok, int mean_pool, float* scores,
+                                           void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                                           void* stream) {
+    halo_status rc = check_pred_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (!W1 || !W2 || !feat || !scores) return HALO_ERR_ARG;
+    if (n_tok <= 0) return HALO_ERR_SHAPE;
+    if (!aligned16(W1) || !aligned16(W2) || !aligned16(feat) || !aligned16(workspace)) return HALO_ERR_ALIGN;
+    if (!workspace || workspace_bytes < halo_predict_workspace_bytes(shape, n_tok)) return HALO_ERR_WORKSPACE;
+    return launch_predict(*shape, W1, W2, feat, n_tok, mean_pool, scores, static_cast<float*>(workspace), dev_status,
+                          static_cast<cudaStream_t>(stream));
+}
+
+// ---- a2..a5 -----------------------------------------------------------------------------------------
+
+extern "C" halo_status halo_select_groups(const halo_plan* plan, const float* scores, uint32_t step, uint32_t layer,
+                                          int force_all, int32_t* order, int32_t* dev_of_group, uint8_t* arrived,
+                                          uint8_t* keep, int32_t* keep_list, int32_t* n_keep, uint32_t* dev_status,
+                                          void* stream) {
+    if (!plan || !scores || !keep_list || !n_keep) return HALO_ERR_ARG;
+    return launch_select(plan->dev, plan->n_groups, scores, step, layer, force_all, order, dev_of_group, arrived,
+                         keep, keep_list, n_keep, dev_status, static_cast<cudaStream_t>(stream));
+}
+
+// ---- a6..a8 -----------------------------------------------------------------------------------------
+
+extern "C" size_t halo_group_ffn_workspace_bytes(const halo_ffn_shape* shape, int n_tok, int n_dev) {
+    (void)shape; (void)n_tok; (void)n_dev;
+    return 0;
+}
+
+extern "C" halo_status halo_group_ffn(const halo_ffn_shape* shape, const void* W_packed, const void* x, int n_tok,
+                                      const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
+                                      int n_dev, float* partials, void* workspace, size_t workspace_bytes,
+                                      uint32_t* dev_status, void* stream) {
+    halo_status rc = check_ffn_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (!W_packed || !x || !keep_list || !n_keep || !partials) return HALO_ERR_ARG;
+    if (n_tok <= 0) return HALO_ERR_SHAPE;
+    if (n_dev < 0 || n_dev > HALO_MAX_DEVICES || (!dev_of_group && n_dev != 0)) return HALO_ERR_ARG;
+    if (!aligned16(W_packed) || !aligned16(x) || !aligned16(partials)) return HALO_ERR_ALIGN;
+    if (workspace_bytes < halo_group_ffn_workspace_bytes(shape, n_tok, n_dev)) return HALO_ERR_WORKSPACE;
+    (void)workspace;
+    return launch_group_ffn_decode(*shape, W_packed, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials,
+                                   dev_status, static_cast<cudaStream_t>(stream));
+}
+
+// ---- a9 and helpers -----------------------------------------------------------------------------------
+
+extern "C" halo_status halo_merge_partials(const float* partials, const uint8_t* arrived, int n_dev, int n_tok,
+                                           int d_model, float* y, void* stream) {
+    if (!partials || !y) return HALO_ERR_ARG;
+    if (n_dev < 0 || n_dev > HALO_MAX_DEVICES || n_tok <= 0 || d_model <= 0) return HALO_ERR_SHAPE;
+    return launch_merge(partials, arrived, n_dev, n_tok, d_model, y, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" halo_status halo_pack_weights(const halo_ffn_shape* shape, const void* Wgate, const void* Wup,
+                                         const void* Wdown, void* W_packed, void* stream) {
+    halo_status rc = check_ffn_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (!Wgate || !Wup || !Wdown || !W_packed) return HALO_ERR_ARG;
+    return launch_pack(*shape, Wgate, Wup, Wdown, W_packed, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" halo_status halo_glue(int d_model, int n_tok, halo_dtype xdtype, const float* h, const float* y,
+                                 float* h_out, void* x_out, void* stream) {
+    if (!h || !h_out || !x_out) return HALO_ERR_ARG;
+    if (!valid_dtype(xdtype)) return HALO_ERR_DTYPE;
+    if (d_model <= 0 || d_model > 12288 || n_tok <= 0) return HALO_ERR_SHAPE;
+    return launch_glue(d_model, n_tok, xdtype, h, y, h_out, x_out, static_cast<cudaStream_t>(stream));
+}
+
+// ---- FFN stack ----------------------------------------------------------------------------------------
+
+struct halo_stack {
+    halo_ffn_shape ffn;
+    halo_pred_shape pred;
+    int n_layers, n_tok, G, n_dev;
+    halo_plan plan;
+    std::vector<const void*> W, W1, W2;
+    void* slab;
+    // carved from the slab
+    float* h;
+    void* x[2];
+    float* pred_ws;
+    float* scores;
+    float* zero_scores;
+    int32_t* dev_of_group;
+    uint8_t* arrived;
+    int32_t* keep_list;
+    int32_t* n_keep;
+    float* partials;
+    uint32_t* status;
+    float* stage_in;
+    float* stage_out;
+    int stage_steps;
+    long long last_launches;
+};
+
+extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred,
+                                         int n_layers, int n_tok, const halo_plan* plan, const void* const* W_packed,
+                                         const void* const* W1, const void* const* W2) {
+    if (!out) return HALO_ERR_ARG;
+    *out = nullptr;
+    halo_status rc = check_ffn_shape(ffn);
+    if (rc != HALO_OK) return rc;
+    rc = check_pred_shape(pred);
+    if (rc != HALO_OK) return rc;
+    if (!plan || !W_packed || !W1 || !W2) return HALO_ERR_ARG;
+    if (n_layers <= 0 || n_tok <= 0) return HALO_ERR_SHAPE;
+    const int G = ffn->d_ffn / ffn->group_size;
+    if (pred->d_in != ffn->d_model || pred->n_groups != G || plan->n_groups != G || pred->wdtype != ffn->wdtype)
+        return HALO_ERR_SHAPE;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!W_packed[l] || !aligned16(W_packed[l])) return W_packed[l] ? HALO_ERR_ALIGN : HALO_ERR_ARG;
+        if (l > 0 && (!W1[l] || !W2[l])) return HALO_ERR_ARG;
+        if (l > 0 && (!aligned16(W1[l]) || !aligned16(W2[l]))) return HALO_ERR_ALIGN;
+    }
+    halo_stack* s = new (std::nothrow) halo_stack();
+    if (!s) return HALO_ERR_NOMEM;
+    s->ffn = *ffn;
+    s->pred = *pred;
+    s->n_layers = n_layers;
+    s->n_tok = n_tok;
+    s->G = G;
+    s->n_dev = plan->n_dev;
+    s->plan = *plan;
+    s->W.assign(W_packed, W_packed + n_layers);
+    s->W1.assign(W1, W1 + n_layers);
+    s->W2.assign(W2, W2 + n_layers);
+    s->last_launches = 0;
+
+    const size_t d = ffn->d_model, es = elem_size(ffn->wdtype), T = n_tok;
+    const size_t step_elems = T * d;
+    s->stage_steps = static_cast<int>(std::max<size_t>(1, std::min<size_t>(64, (16u << 20) / (step_elems * 4))));
+    size_t off = 0;
+    auto carve = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t o_h = carve(step_elems * 4);
+    const size_t o_x0 = carve(step_elems * es), o_x1 = carve(step_elems * es);
+    const size_t o_pws = carve(sizeof(float) * T * (static_cast<size_t>(pred->rank) + G));
+    const size_t o_sc = carve(sizeof(float) * G), o_zs = carve(sizeof(float) * G);
+    const size_t o_dg = carve(sizeof(int32_t) * G), o_ar = carve(HALO_MAX_DEVICES);
+    const size_t o_kl = carve(sizeof(int32_t) * G), o_nk = carve(sizeof(int32_t));
+    const size_t o_pa = carve(sizeof(float) * (s->n_dev + 1) * step_elems);
+    const size_t o_st = carve(sizeof(uint32_t));
+    const size_t o_si = carve(sizeof(float) * s->stage_steps * step_elems);
+    const size_t o_so = carve(sizeof(float) * s->stage_steps * step_elems);
+    if (cudaMalloc(&s->slab, off) != cudaSuccess) { delete s; return HALO_ERR_NOMEM; }
+    if (cudaMemset(s->slab, 0, off) != cudaSuccess) { cudaFree(s->slab); delete s; return HALO_ERR_CUDA; }
+    char* base = static_cast<char*>(s->slab);
+    s->h = reinterpret_cast<float*>(base + o_h);
+    s->x[0] = base + o_x0;
+    s->x[1] = base + o_x1;
+    s->pred_ws = reinterpret_cast<float*>(base + o_pws);
+    s->scores = reinterpret_cast<float*>(base + o_sc);
+    s->zero_scores = reinterpret_cast<float*>(base + o_zs);
+    s->dev_of_group = reinterpret_cast<int32_t*>(base + o_dg);
+    s->arrived = reinterpret_cast<uint8_t*>(base + o_ar);
+    s->keep_list = reinterpret_cast<int32_t*>(base + o_kl);
+    s->n_keep = reinterpret_cast<int32_t*>(base + o_nk);
+    s->partials = reinterpret_cast<float*>(base + o_pa);
+    s->status = reinterpret_cast<uint32_t*>(base + o_st);
+    s->stage_in = reinterpret_cast<float*>(base + o_si);
+    s->stage_out = reinterpret_cast<float*>(base + o_so);
+    *out = s;
+    return HALO_OK;
+}
+
+extern "C" halo_status halo_stack_destroy(halo_stack* s) {
+    if (!s) return HALO_OK;
+    cudaFree(s->slab);
+    delete s;
+    return HALO_OK;
+}
+
+extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int steps, uint32_t step0, float* h_out,
+                                         const halo_taps* taps, void* stream) {
+    if (!s || !h0 || !h_out) return HALO_ERR_ARG;
+    if (steps <= 0) return HALO_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t d = s->ffn.d_model, T = s->n_tok, es = elem_size(s->ffn.wdtype);
+    const size_t step_elems = T * d;
+    const int L = s->n_layers, G = s->G, n_dev = s->n_dev;
+    long long launches = 0;
+    halo_status rc;
+#define HALO_TRY(call) do { rc = (call); if (rc != HALO_OK) return rc; } while (0)
+#define HALO_COPY(dst, src, bytes)                                                                    \
+    do { if (cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToDevice, st) != cudaSuccess)     \
+             return HALO_ERR_CUDA; } while (0)
+    for (int sidx = 0; sidx < steps; ++sidx) {
+        const uint32_t step = step0 + static_cast<uint32_t>(sidx);
+        HALO_TRY(launch_glue(static_cast<int>(d), static_cast<int>(T), s->ffn.wdtype, h0 + sidx * step_elems, nullptr,
+                             s->h, s->x[0], st));
+        ++launches;
+        for (int l = 0; l < L; ++l) {
+            void* x_cur = s->x[l & 1];
+            void* x_prev = s->x[(l + 1) & 1];
+            const float* scores_used = s->scores;
+            if (l == 0) {
+                // first block: reliable, no semantic information yet -> everything is kept
+                scores_used = s->zero_scores;
+                HALO_TRY(launch_select(s->plan.dev, G, s->zero_scores, step, 0u, 1, nullptr, s->dev_of_group,
+                                       s->arrived, nullptr, s->keep_list, s->n_keep, s->status, st));
+                ++launches;
+            } else if (T == 1) {
+                HALO_TRY(launch_predict_hidden(s->pred, s->W1[l], x_prev, 1, s->pred_ws, st));
+                HALO_TRY(launch_score_select(s->pred, s->W2[l], s->pred_ws, s->plan.dev, step,
+                                             static_cast<uint32_t>(l), 0, s->scores, nullptr, s->dev_of_group,
+                                             s->arrived, nullptr, s->keep_list, s->n_keep, s->status, st));
+                launches += 2;
+            } else {
+                HALO_TRY(launch_predict(s->pred, s->W1[l], s->W2[l], x_prev, static_cast<int>(T), 1, s->scores,
+                                        s->pred_ws, s->status, st));
+                HALO_TRY(launch_select(s->plan.dev, G, s->scores, step, static_cast<uint32_t>(l), 0, nullptr,
+                                       s->dev_of_group, s->arrived, nullptr, s->keep_list, s->n_keep, s->status, st));
+                launches += 4;
+            }
+            float* y_tap = nullptr;
+            if (taps) {
+                const size_t rec = static_cast<size_t>(sidx) * L + l;
+                if (taps->x) HALO_COPY(static_cast<char*>(taps->x) + rec * step_elems * es, x_cur, step_elems * es);
+                if (taps->scores) HALO_COPY(taps->scores + rec * G, scores_used, sizeof(float) * G);
+                if (taps->dev_of_group) HALO_COPY(taps->dev_of_group + rec * G, s->dev_of_group, sizeof(int32_t) * G);
+                if (taps->arrived && n_dev > 0) HALO_COPY(taps->arrived + rec * n_dev, s->arrived, n_dev);
+                if (taps->keep_list) HALO_COPY(taps->keep_list + rec * G, s->keep_list, sizeof(int32_t) * G);
+                if (taps->n_keep) HALO_COPY(taps->n_keep + rec, s->n_keep, sizeof(int32_t));
+                if (taps->y) y_tap = taps->y + rec * step_elems;
+            }
+            HALO_TRY(launch_group_ffn_decode(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->keep_list, s->n_keep,
+                                             s->dev_of_group, n_dev, s->partials, s->status, st));
+            ++launches;
+            float* h_dst = (l == L - 1) ? h_out + sidx * step_elems : s->h;
+            HALO_TRY(launch_merge_glue(s->partials, s->arrived, n_dev, static_cast<int>(T), static_cast<int>(d),
+                                       s->ffn.wdtype, s->h, h_dst, x_prev, y_tap, st));
+            ++launches;
+        }
+    }
+#undef HALO_TRY
+#undef HALO_COPY
+    s->last_launches = launches;
+    return HALO_OK;
+}
+
+extern "C" halo_status halo_stack_decode_host(halo_stack* s, const float* h0_host, int steps, uint32_t step0,
+                                              float* h_out_host, void* stream) {
+    if (!s || !h0_host || !h_out_host) return HALO_ERR_ARG;
+    if (steps <= 0) return HALO_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t step_elems = static_cast<size_t>(s->n_tok) * s->ffn.d_model;
+    long long launches = 0;
+    for (int done = 0; done < steps; done += s->stage_steps) {
+        const int n = std::min(s->stage_steps, steps - done);
+        const size_t bytes = sizeof(float) * n * step_elems;
+        if (cudaMemcpyAsync(s->stage_in, h0_host + done * step_elems, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return HALO_ERR_CUDA;
+        halo_status rc = halo_stack_decode(s, s->stage_in, n, step0 + static_cast<uint32_t>(done), s->stage_out,
+                                           nullptr, stream);
+        if (rc != HALO_OK) return rc;
+        launches += s->last_launches;
+        if (cudaMemcpyAsync(h_out_host + done * step_elems, s->stage_out, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return HALO_ERR_CUDA;
+    }
+    s->last_launches = launches;
+    return cuda_status(cudaStreamSynchronize(st));
+}
+
+extern "C" halo_status halo_stack_status(halo_stack* s, uint32_t* value, void* stream) {
+    if (!s || !value) return HALO_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(value, s->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return HALO_ERR_CUDA;
+    return cuda_status(cudaStreamSynchronize(st));
+}
+
+extern "C" long long halo_stack_last_launches(const halo_stack* s) { return s ? s->last_launches : 0; }

@@ -1,0 +1,137 @@
+// halo_merge_partials (step a9), halo_glue (residual + RMS normalisation between blocks), their fusion
+// for the stack, and halo_pack_weights.
+#include "common.cuh"
+
+namespace halo {
+
+__device__ __forceinline__ float merged_value(const float* __restrict__ partials, const uint8_t* __restrict__ arrived,
+                                              int n_dev, size_t slot_stride, size_t idx) {
+    float v = partials[idx];  // the master's own part is never lost
+    for (int i = 0; i < n_dev; ++i)
+        if (!arrived || arrived[i]) v += partials[static_cast<size_t>(i + 1) * slot_stride + idx];
+    return v;
+}
+
+__global__ void merge_kernel(const float* __restrict__ partials, const uint8_t* __restrict__ arrived, int n_dev,
+                             size_t slot_stride, float* __restrict__ y) {
+    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx < slot_stride) y[idx] = merged_value(partials, arrived, n_dev, slot_stride, idx);
+}
+
+__device__ __forceinline__ float block_sum_1024(float v, float* scratch /*[32]*/) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    v = warp_sum(v);
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    float t = (threadIdx.x < (blockDim.x >> 5)) ? scratch[threadIdx.x] : 0.0f;
+    if (warp == 0) {
+        t = warp_sum(t);
+        if (lane == 0) scratch[0] = t;
+    }
+    __syncthreads();
+    const float r = scratch[0];
+    __syncthreads();
+    return r;
+}
+
+// One block per token.  MERGE: y is taken from the partial slots, else from y_in (may be NULL = 0).
+template <typename T, bool MERGE>
+__global__ void __launch_bounds__(1024)
+glue_kernel(int d, const float* __restrict__ h, const float* __restrict__ y_in, const float* __restrict__ partials,
+            const uint8_t* __restrict__ arrived, int n_dev, size_t slot_stride, float* h_out, T* __restrict__ x_out,
+            float* __restrict__ y_tap) {
+    __shared__ float scratch[32];
+    extern __shared__ float hv[];  // [d]
+    const int tok = blockIdx.x;
+    const size_t base = static_cast<size_t>(tok) * d;
+    float ss = 0.0f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+        float y = 0.0f;
+        if (MERGE) {
+            y = merged_value(partials, arrived, n_dev, slot_stride, base + c);
+            if (y_tap) y_tap[base + c] = y;
+        } else if (y_in) {
+            y = y_in[base + c];
+        }
+        const float v = h[base + c] + y;
+        hv[c] = v;
+        ss = fmaf(v, v, ss);
+    }
+    ss = block_sum_1024(ss, scratch);
+    const float scale = 1.0f / sqrtf(ss / static_cast<float>(d) + 1e-5f);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+        const float v = hv[c];
+        h_out[base + c] = v;
+        x_out[base + c] = from_float<T>(v * scale);
+    }
+}
+
+template <typename T>
+__global__ void pack_kernel(int d, int F, int S, const T* __restrict__ Wgate, const T* __restrict__ Wup,
+                            const T* __restrict__ Wdown, T* __restrict__ Wp) {
+    // one thread per packed element of planes 0/1; plane 2 is a transpose and gets its own index space
+    const size_t n = static_cast<size_t>(F) * d;
+    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= n) return;
+    const int neuron = static_cast<int>(idx / d), c = static_cast<int>(idx % d);
+    const int g = neuron / S, j = neuron % S;
+    const size_t group_base = static_cast<size_t>(g) * 3 * S * d;
+    Wp[group_base + (static_cast<size_t>(0) * S + j) * d + c] = Wgate[idx];
+    Wp[group_base + (static_cast<size_t>(1) * S + j) * d + c] = Wup[idx];
+    Wp[group_base + (static_cast<size_t>(2) * S + j) * d + c] = Wdown[static_cast<size_t>(c) * F + neuron];
+}
+
+halo_status launch_merge(const float* partials, const uint8_t* arrived, int n_dev, int n_tok, int d, float* y,
+                         cudaStream_t st) {
+    const size_t n = static_cast<size_t>(n_tok) * d;
+    merge_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(partials, arrived, n_dev, n, y);
+    HALO_CHECK_LAUNCH();
+    return HALO_OK;
+}
+
+halo_status launch_glue(int d, int n_tok, halo_dtype xdtype, const float* h, const float* y, float* h_out,
+                        void* x_out, cudaStream_t st) {
+    const size_t smem = sizeof(float) * static_cast<size_t>(d);
+    if (xdtype == HALO_BF16)
+        glue_kernel<__nv_bfloat16, false><<<n_tok, 1024, smem, st>>>(d, h, y, nullptr, nullptr, 0, 0, h_out,
+                                                                      static_cast<__nv_bfloat16*>(x_out), nullptr);
+    else
+        glue_kernel<float, false><<<n_tok, 1024, smem, st>>>(d, h, y, nullptr, nullptr, 0, 0, h_out,
+                                                             static_cast<float*>(x_out), nullptr);
+    HALO_CHECK_LAUNCH();
+    return HALO_OK;
+}
+
+halo_status launch_merge_glue(const float* partials, const uint8_t* arrived, int n_dev, int n_tok, int d,
+                              halo_dtype xdtype, const float* h, float* h_out, void* x_out, float* y_tap,
+                              cudaStream_t st) {
+    const size_t smem = sizeof(float) * static_cast<size_t>(d);
+    const size_t stride = static_cast<size_t>(n_tok) * d;
+    if (xdtype == HALO_BF16)
+        glue_kernel<__nv_bfloat16, true><<<n_tok, 1024, smem, st>>>(d, h, nullptr, partials, arrived, n_dev, stride,
+                                                                     h_out, static_cast<__nv_bfloat16*>(x_out), y_tap);
+    else
+        glue_kernel<float, true><<<n_tok, 1024, smem, st>>>(d, h, nullptr, partials, arrived, n_dev, stride, h_out,
+                                                            static_cast<float*>(x_out), y_tap);
+    HALO_CHECK_LAUNCH();
+    return HALO_OK;
+}
+
+halo_status launch_pack(const halo_ffn_shape& sh, const void* Wgate, const void* Wup, const void* Wdown,
+                        void* Wpacked, cudaStream_t st) {
+    const size_t n = static_cast<size_t>(sh.d_ffn) * sh.d_model;
+    const unsigned blocks = static_cast<unsigned>((n + 255) / 256);
+    if (sh.wdtype == HALO_BF16)
+        pack_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(
+            sh.d_model, sh.d_ffn, sh.group_size, static_cast<const __nv_bfloat16*>(Wgate),
+            static_cast<const __nv_bfloat16*>(Wup), static_cast<const __nv_bfloat16*>(Wdown),
+            static_cast<__nv_bfloat16*>(Wpacked));
+    else
+        pack_kernel<float><<<blocks, 256, 0, st>>>(sh.d_model, sh.d_ffn, sh.group_size,
+                                                   static_cast<const float*>(Wgate), static_cast<const float*>(Wup),
+                                                   static_cast<const float*>(Wdown), static_cast<float*>(Wpacked));
+    HALO_CHECK_LAUNCH();
+    return HALO_OK;
+}
+
+}  // namespace halo

@@ -1,0 +1,99 @@
+"""CPU-side checks of the C-ABI library: it loads, exports what include/halo.h declares, validates arguments on
+the host, and its host-only Assignment phase agrees with the oracle's Algorithm 3."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import halo_ref as R
+from paper_2601_11676_b200 import binding as B
+from paper_2601_11676_b200 import build as halo_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    halo_build.build()
+    return B.lib()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "halo.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(halo_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared()
+    assert len(names) >= 15
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in halo.h but not exported"
+    assert sorted(B.EXPORTS) == names
+
+
+def test_status_strings(lib):
+    assert B.status_string(0) == "ok"
+    assert "aligned" in B.status_string(-3)
+    assert "index" in B.status_message(B.DEV_BAD_INDEX)
+    assert B.status_message(0) == "clean"
+
+
+def test_plan_matches_oracle_algorithm3(lib):
+    rng = np.random.default_rng(0)
+    for _ in range(200):
+        n = int(rng.integers(0, 9))
+        G = int(rng.integers(1, 300))
+        M = int(rng.integers(0, G + 1))
+        rho = rng.uniform(0, 1, n).round(2)
+        w = rng.integers(0, 6, n)
+        if n and w.sum() == 0:
+            w[0] = 1
+        plan = B.Plan(G, rho, w, B.SEL_TOPK, G - M, 0.0, 5)
+        order, thr, bnd = plan.describe(M)
+        o_ref, t_ref, b_ref = R.plan(rho, w, M)
+        assert order == o_ref.tolist() and thr == [int(v) for v in t_ref] and bnd == b_ref.tolist()
+        plan.close()
+
+
+def test_plan_paper_example(lib):
+    plan = B.Plan(8, [0.0, 0.5, 0.1], [4, 4, 2], B.SEL_TOPK, 0, 0.0, 0)
+    order, thr, bnd = plan.describe(8)
+    assert order == [0, 2, 1] and bnd == [0, 3, 5, 8]
+
+
+def test_plan_rejects_bad_arguments(lib):
+    for args in [
+        (8, [1.5], [1]), (8, [-0.1], [1]), (8, [0.1, 0.2], [0, 0]), (0, [0.1], [1]), (B.MAX_GROUPS + 1, [0.1], [1]),
+        (8, [0.0] * (B.MAX_DEVICES + 1), [1] * (B.MAX_DEVICES + 1)),
+    ]:
+        with pytest.raises(B.HaloError):
+            B.Plan(*args)
+    with pytest.raises(B.HaloError):
+        B.Plan(8, [0.1], [1], B.SEL_TOPK, 9)
+    with pytest.raises(B.HaloError):
+        B.Plan(8, [0.1], [1], B.SEL_THRESHOLD, 0, float("nan"))
+
+
+def test_host_side_argument_checks_launch_nothing(lib):
+    # NULL pointers / bad shapes are rejected before any CUDA call, so this runs without a GPU
+    sh = B.ffn_shape(256, 688, 16, B.F32)
+    rc = lib.halo_group_ffn(ctypes.byref(sh), None, None, 1, None, None, None, 0, None, None, 0, None, None)
+    assert rc == -1
+    bad = B.ffn_shape(250, 688, 16, B.F32)
+    rc = lib.halo_group_ffn(ctypes.byref(bad), 16, 16, 1, 16, 16, None, 0, 16, None, 0, None, None)
+    assert rc == -2
+    bad = B.ffn_shape(256, 690, 16, B.F32)
+    assert lib.halo_pack_weights(ctypes.byref(bad), 16, 16, 16, 16, None) == -2
+    bad = B.ffn_shape(256, 688, 16, 7)
+    assert lib.halo_pack_weights(ctypes.byref(bad), 16, 16, 16, 16, None) == -4
+    rc = lib.halo_group_ffn(ctypes.byref(sh), 24, 16, 1, 16, 16, None, 0, 16, None, 0, None, None)
+    assert rc == -3  # W_packed not 16-byte aligned
+    ps = B.pred_shape(256, 32, 43, B.F32)
+    assert B.halo_predict_workspace_bytes(ps, 1) == 4 * (32 + 43)
+    rc = lib.halo_predict_groups(ctypes.byref(ps), 16, 16, 16, 1, 0, 16, 16, 8, None, None)
+    assert rc == -8  # workspace too small
+    assert lib.halo_merge_partials(None, None, 1, 1, 8, None, None) == -1
+    assert lib.halo_select_groups(None, None, 0, 0, 0, None, None, None, None, None, None, None, None) == -1

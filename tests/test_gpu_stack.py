@@ -1,0 +1,120 @@
+"""GPU parity of the FFN stack runner: teacher-forced per block against the oracle, via the recorded taps."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import halo_ref as R
+from paper_2601_11676_b200 import binding as B
+from paper_2601_11676_b200 import synth
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+DEV = U.DEV
+
+
+def build_stack(wl):
+    code = U.dtype_code(wl)
+    Wp = [synth.packed_layer(wl, l, DEV) for l in range(wl.n_layers)]
+    preds = [synth.predictor(wl, l, DEV) for l in range(wl.n_layers)]
+    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, B.SEL_TOPK, wl.k_critical, 0.0, wl.seed)
+    stack = B.Stack(B.ffn_shape(wl.d_model, wl.d_ffn, wl.group_size, code),
+                    B.pred_shape(wl.d_model, wl.pred_rank, wl.n_groups, code), wl.n_tok, plan, Wp,
+                    [p[0] for p in preds], [p[1] for p in preds])
+    return stack, Wp, preds
+
+
+def run_with_taps(wl, stack, steps, step0=0):
+    L, G, d, T, n = wl.n_layers, wl.n_groups, wl.d_model, wl.n_tok, wl.n_dev
+    h0 = torch.stack([synth.stream_input(wl, step0 + s, DEV) for s in range(steps)])
+    h_out = torch.empty_like(h0)
+    t = dict(x=torch.zeros((steps, L, T, d), dtype=wl.torch_dtype, device=DEV),
+             scores=torch.zeros((steps, L, G), dtype=torch.float32, device=DEV),
+             dev_of_group=torch.zeros((steps, L, G), dtype=torch.int32, device=DEV),
+             arrived=torch.zeros((steps, L, max(n, 1)), dtype=torch.uint8, device=DEV),
+             keep_list=torch.zeros((steps, L, G), dtype=torch.int32, device=DEV),
+             n_keep=torch.zeros((steps, L), dtype=torch.int32, device=DEV),
+             y=torch.zeros((steps, L, T, d), dtype=torch.float32, device=DEV))
+    taps = B.Taps(*[t[k].data_ptr() for k in ("x", "scores", "dev_of_group", "arrived", "keep_list", "n_keep", "y")])
+    stack.decode(h0, steps, step0, h_out, taps)
+    torch.cuda.synchronize()
+    assert stack.status() == 0
+    return h0, h_out, t
+
+
+def check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=0):
+    hb = synth.host_bits
+    tol = U.tol_for(wl)
+    L, n = wl.n_layers, wl.n_dev
+    x_all = hb(t["x"])
+    lost_layers = 0
+    for s in range(steps):
+        h = h0[s].cpu().numpy().astype(np.float64)
+        # first input: normalised stream
+        _, x0 = R.glue(h, None, U.dtype_code(wl))
+        assert np.abs(R.to_f64(x0) - R.to_f64(x_all[s, 0])).max() <= 2 ** -7 * np.abs(R.to_f64(x0)).max()
+        for l in range(L):
+            x_l = x_all[s, l]
+            scores = t["scores"][s, l].cpu().numpy()
+            if l == 0:
+                assert (scores == 0).all()
+            else:
+                s_ref = R.predict(hb(preds[l][0]), hb(preds[l][1]), x_all[s, l - 1], mean_pool=wl.n_tok > 1)
+                assert U.rel_err(scores, s_ref.astype(np.float64)) <= tol
+            sel = R.select(scores, wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed,
+                           step0 + s, l, force_all=(l == 0))
+            nk = int(t["n_keep"][s, l].item())
+            assert nk == sel["n_keep"]
+            assert (t["keep_list"][s, l].cpu().numpy() == sel["keep_list"]).all()
+            assert (t["dev_of_group"][s, l].cpu().numpy() == sel["dev_of_group"]).all()
+            if n:
+                assert (t["arrived"][s, l, :n].cpu().numpy() == sel["arrived"]).all()
+            lost_layers += int(nk < wl.n_groups)
+            P = R.group_ffn(hb(Wp[l]), x_l, sel["keep_list"][:nk], sel["dev_of_group"], n)
+            y_ref = R.merge(P)
+            y = t["y"][s, l].cpu().numpy()
+            assert U.rel_err(y, y_ref) <= tol, (s, l)
+            # glue, from the GPU's own y: next input and residual stream
+            h, x_next = R.glue(h, y.astype(np.float64), U.dtype_code(wl))
+            if l + 1 < L:
+                xr, xg = R.to_f64(x_next), R.to_f64(x_all[s, l + 1])
+                assert np.abs(xr - xg).max() <= 2 ** -7 * np.abs(xr).max()
+        assert np.abs(h_out[s].cpu().numpy() - h).max() <= 1e-4 * np.abs(h).max()
+    return lost_layers
+
+
+@pytest.mark.parametrize("name,layers,steps", [("tinyllama-1.1b-decode", 4, 3), ("llama2-7b-decode", 3, 2),
+                                               ("llama2-13b-decode", 3, 2)])
+def test_stack_decode_teacher_forced(name, layers, steps):
+    wl = synth.small_variant(synth.workload(name), layers, steps)
+    stack, Wp, preds = build_stack(wl)
+    h0, h_out, t = run_with_taps(wl, stack, steps, step0=3)
+    check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=3)
+    assert stack.last_launches() > 0
+
+
+def test_stack_small_f32_many_steps_sees_losses():
+    wl = synth.Workload("s", 3, 256, 688, 16, 32, "f32", (0.0, 0.3, 0.5), (2, 1, 1), 300, 12)
+    stack, Wp, preds = build_stack(wl)
+    h0, h_out, t = run_with_taps(wl, stack, wl.steps)
+    lost = check_teacher_forced(wl, Wp, preds, h0, h_out, t, wl.steps)
+    assert lost > 0
+
+
+def test_stack_host_entry_matches_device_entry():
+    wl = synth.small_variant(synth.workload("tinyllama-1.1b-decode"), 3, 5)
+    stack, _, _ = build_stack(wl)
+    h0 = torch.stack([synth.stream_input(wl, s, DEV) for s in range(5)])
+    out_dev = torch.empty_like(h0)
+    stack.decode(h0, 5, 0, out_dev)
+    torch.cuda.synchronize()
+    h0_host = h0.cpu().pin_memory()
+    out_host = torch.empty_like(h0_host).pin_memory()
+    stack.decode_host(h0_host, 5, 0, out_host)
+    assert np.abs(out_host.numpy() - out_dev.cpu().numpy()).max() <= 1e-3 * np.abs(out_host.numpy()).max()
+
+
+def test_stack_multi_token_prompt():
+    wl = synth.Workload("p", 3, 512, 768, 64, 64, "bf16", (0.0, 0.3, 0.6), (1, 1, 1), 500, 1, n_tok=5)
+    stack, Wp, preds = build_stack(wl)
+    h0, h_out, t = run_with_taps(wl, stack, 1)
+    check_teacher_forced(wl, Wp, preds, h0, h_out, t, 1)

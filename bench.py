@@ -114,6 +114,8 @@ def run_halo(args, rank, world, local_rank):
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     wl = synth.workload(args.workload, keep_permille=args.keep_permille)
+    if args.layers:
+        wl = synth.small_variant(wl, args.layers, wl.steps)
     K, W = args.steps, args.warmup
     stack, Wp, preds, plan, ffn = build_stack(wl, dev)
     L, G, d = wl.n_layers, wl.n_groups, wl.d_model
@@ -255,17 +257,17 @@ def cpu_baseline(wl, budget_s=15.0):
     R.lib()
     done, spent = 0, 0.0
     inputs = _oracle_layer_inputs(wl, 1)  # same shapes for every block; generated outside the timed part
-    while done < wl.n_layers and (done == 0 or spent + spent / done <= budget_s):
+    while spent < budget_s and done < 64 * wl.n_layers:
         Wp, w1, w2, feat, x = inputs
         t0 = time.perf_counter()
-        R.layer(Wp, w1, w2, feat, x, wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed, done,
-                1 + done % max(wl.n_layers - 1, 1))
+        R.layer(Wp, w1, w2, feat, x, wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed,
+                done // wl.n_layers, 1 + done % max(wl.n_layers - 1, 1))
         spent += time.perf_counter() - t0
         done += 1
     value = (done / wl.n_layers) / spent
     return {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-            "sample": f"{done} of {wl.n_layers} blocks of one token ({wl.name}), {spent:.1f} s of CPU time; "
-                      f"tokens/s extrapolated per token"}
+            "sample": f"{done} blocks ({done / wl.n_layers:.2f} tokens of {wl.n_layers} blocks, {wl.name}), "
+                      f"{spent:.1f} s of CPU time; tokens/s = tokens / time"}
 
 
 def run_reference(args, rank, world):
@@ -328,6 +330,7 @@ def main():
     ap.add_argument("--impl", default="halo", choices=["halo", "reference"])
     ap.add_argument("--workload", default="llama2-7b-decode", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--keep-permille", type=int, default=500)
+    ap.add_argument("--layers", type=int, default=0, help="use only this many blocks (small profiling cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()

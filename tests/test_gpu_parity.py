@@ -212,4 +212,7 @@ def test_tiny_layer_end_to_end_masks_over_steps():
         y = U.gpu_merge(P, gpu["arrived"]).cpu().numpy()
         assert st == 0 and U.rel_err(y, full["y"]) <= U.TOL_F32
         outcomes.add(gpu["n_keep"])
-    assert outcomes == {wl.k_critical, wl.n_groups}  # the lossy device both arrives and is lost
+    # the lossy device both arrives and is lost; when lost, exactly its chunk of the less-critical groups goes
+    order, _, bnd = R.plan(wl.loss_rate, wl.share_weight, wl.n_groups - wl.k_critical)
+    j = list(order).index(1)
+    assert outcomes == {wl.n_groups - int(bnd[j + 1] - bnd[j]), wl.n_groups}

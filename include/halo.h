@@ -236,6 +236,11 @@ halo_status halo_stack_decode(halo_stack* stack, const float* h0, int steps, uin
  * copies h_out back and synchronises the stream before returning. */
 halo_status halo_stack_decode_host(halo_stack* stack, const float* h0_host, int steps, uint32_t step0,
                                    float* h_out_host, void* stream);
+/* How halo_stack_decode runs.  mode 0 (default): decode of bf16 stacks with d_model in {2048, 4096, 5120, 8192}
+ * runs as ONE persistent cooperative kernel over all steps and blocks, the predictor and selection of block
+ * l+1 overlapped with the weight stream of block l; anything else runs one launch per step of the path.
+ * mode 1: always one launch per step of the path (no overlap; for comparison and checking). */
+halo_status halo_stack_set_mode(halo_stack* stack, int mode);
 /* Device status word accumulated by the stack's launches (synchronises the stream). */
 halo_status halo_stack_status(halo_stack* stack, uint32_t* dev_status_value /*host*/, void* stream);
 /* Number of kernel launches the last halo_stack_decode enqueued. */

@@ -27,7 +27,7 @@ EXPORTS = [
     "halo_predict_workspace_bytes", "halo_predict_groups", "halo_select_groups", "halo_group_ffn_workspace_bytes",
     "halo_group_ffn", "halo_merge_partials", "halo_pack_weights", "halo_glue", "halo_stack_create",
     "halo_stack_destroy", "halo_stack_decode", "halo_stack_decode_host", "halo_stack_status",
-    "halo_stack_last_launches",
+    "halo_stack_last_launches", "halo_stack_set_mode",
 ]
 
 
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.halo_stack_decode.argtypes = [c_void_p, c_void_p, c_int, c_uint32, c_void_p, POINTER(Taps), c_void_p]
         L.halo_stack_decode_host.argtypes = [c_void_p, c_void_p, c_int, c_uint32, c_void_p, c_void_p]
         L.halo_stack_status.argtypes = [c_void_p, POINTER(c_uint32), c_void_p]
+        L.halo_stack_set_mode.argtypes = [c_void_p, c_int]
         L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
         _lib = L
     return _lib
@@ -233,6 +234,9 @@ class Stack:
         assert not h0_host.is_cuda and not h_out_host.is_cuda
         _chk(lib().halo_stack_decode_host(self.handle, c_void_p(h0_host.data_ptr()), steps, step0,
                                           c_void_p(h_out_host.data_ptr()), _stream(stream)), "halo_stack_decode_host")
+
+    def set_mode(self, mode: int) -> None:
+        _chk(lib().halo_stack_set_mode(self.handle, mode), "halo_stack_set_mode")
 
     def status(self, stream=None) -> int:
         v = c_uint32(0)

@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "stack_persistent.cuh"
 
 using namespace halo;
 
@@ -254,6 +255,16 @@ struct halo_stack {
     float* stage_out;
     int stage_steps;
     long long last_launches;
+    // persistent single-kernel path
+    int mode;                      // 0 = automatic, 1 = one launch per step of the path
+    bool persistent_ok;
+    const void** d_W;              // device pointer tables
+    const void** d_W1;
+    const void** d_W2;
+    float* p_partials;             // [3][n_dev+1][d]
+    float* p_z;
+    halo::PersistSel* p_sel;       // [3]
+    unsigned* p_sync;              // [4]
 };
 
 extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred,
@@ -304,6 +315,12 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     const size_t o_st = carve(sizeof(uint32_t));
     const size_t o_si = carve(sizeof(float) * s->stage_steps * step_elems);
     const size_t o_so = carve(sizeof(float) * s->stage_steps * step_elems);
+    const size_t o_tw = carve(sizeof(void*) * n_layers), o_tw1 = carve(sizeof(void*) * n_layers);
+    const size_t o_tw2 = carve(sizeof(void*) * n_layers);
+    const size_t o_pp = carve(sizeof(float) * 3 * (s->n_dev + 1) * d);
+    const size_t o_pz = carve(sizeof(float) * pred->rank);
+    const size_t o_ps = carve(sizeof(PersistSel) * 3);
+    const size_t o_py = carve(sizeof(unsigned) * 4);
     if (cudaMalloc(&s->slab, off) != cudaSuccess) { delete s; return HALO_ERR_NOMEM; }
     if (cudaMemset(s->slab, 0, off) != cudaSuccess) { cudaFree(s->slab); delete s; return HALO_ERR_CUDA; }
     char* base = static_cast<char*>(s->slab);
@@ -321,6 +338,38 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     s->status = reinterpret_cast<uint32_t*>(base + o_st);
     s->stage_in = reinterpret_cast<float*>(base + o_si);
     s->stage_out = reinterpret_cast<float*>(base + o_so);
+    s->d_W = reinterpret_cast<const void**>(base + o_tw);
+    s->d_W1 = reinterpret_cast<const void**>(base + o_tw1);
+    s->d_W2 = reinterpret_cast<const void**>(base + o_tw2);
+    s->p_partials = reinterpret_cast<float*>(base + o_pp);
+    s->p_z = reinterpret_cast<float*>(base + o_pz);
+    s->p_sel = reinterpret_cast<PersistSel*>(base + o_ps);
+    s->p_sync = reinterpret_cast<unsigned*>(base + o_py);
+    s->mode = 0;
+    s->persistent_ok = persistent_supported(*ffn, n_tok, G);
+    {
+        // pointer tables, and the first block's selection: reliable block, all scores equal -> the priority
+        // order is the group order, everything is kept (Sec. III-B.3, first layer)
+        std::vector<PersistSel> sel0(1);
+        std::memset(&sel0[0], 0, sizeof(PersistSel));
+        const PlanDev& dv = plan->dev;
+        int k = dv.mode == HALO_SEL_THRESHOLD ? ((0.0f >= dv.threshold) ? G : 0) : dv.k_critical;
+        if (dv.n_dev == 0) k = G;
+        const int M = G - k;
+        std::vector<int32_t> bnd(dv.n_dev + 1, 0);
+        halo_plan_describe(plan, M, nullptr, nullptr, bnd.data());
+        sel0[0].n_keep = G;
+        for (int g = 0; g < HALO_MAX_GROUPS; ++g) { sel0[0].keep_list[g] = g < G ? g : -1; sel0[0].dev_of_group[g] = -1; }
+        for (int g = k; g < G; ++g)
+            for (int j = 0; j < dv.n_dev; ++j)
+                if (bnd[j] <= g - k && g - k < bnd[j + 1]) { sel0[0].dev_of_group[g] = dv.dev_order[j]; break; }
+        for (int i = 0; i < dv.n_dev; ++i) sel0[0].arrived[i] = 1;
+        bool ok = cudaMemcpy(s->p_sel + 2, sel0.data(), sizeof(PersistSel), cudaMemcpyHostToDevice) == cudaSuccess;
+        ok = ok && cudaMemcpy(s->d_W, s->W.data(), sizeof(void*) * n_layers, cudaMemcpyHostToDevice) == cudaSuccess;
+        ok = ok && cudaMemcpy(s->d_W1, s->W1.data(), sizeof(void*) * n_layers, cudaMemcpyHostToDevice) == cudaSuccess;
+        ok = ok && cudaMemcpy(s->d_W2, s->W2.data(), sizeof(void*) * n_layers, cudaMemcpyHostToDevice) == cudaSuccess;
+        if (!ok) { cudaFree(s->slab); delete s; return HALO_ERR_CUDA; }
+    }
     *out = s;
     return HALO_OK;
 }
@@ -342,6 +391,46 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
     const int L = s->n_layers, G = s->G, n_dev = s->n_dev;
     long long launches = 0;
     halo_status rc;
+    if (s->persistent_ok && s->mode == 0) {
+        // whole run in one cooperative launch
+        if (cudaMemsetAsync(s->p_partials, 0, sizeof(float) * 3 * (n_dev + 1) * d, st) != cudaSuccess ||
+            cudaMemsetAsync(s->p_sync, 0, sizeof(unsigned) * 4, st) != cudaSuccess)
+            return HALO_ERR_CUDA;
+        PersistParams P;
+        std::memset(&P, 0, sizeof(P));
+        P.L = L; P.steps = steps; P.d = static_cast<int>(d); P.S = s->ffn.group_size; P.G = G; P.r = s->pred.rank;
+        P.act = s->pred.act; P.step0 = step0; P.sel_cost = 4;
+        P.W = reinterpret_cast<const __nv_bfloat16* const*>(s->d_W);
+        P.W1 = reinterpret_cast<const __nv_bfloat16* const*>(s->d_W1);
+        P.W2 = reinterpret_cast<const __nv_bfloat16* const*>(s->d_W2);
+        P.h0 = h0; P.h_out = h_out; P.partials = s->p_partials; P.z = s->p_z; P.sel = s->p_sel; P.sync = s->p_sync;
+        P.status = s->status;
+        P.plan = s->plan.dev;
+        if (taps) {
+            P.tap_x = static_cast<__nv_bfloat16*>(taps->x); P.tap_scores = taps->scores;
+            P.tap_dev_of_group = taps->dev_of_group; P.tap_arrived = taps->arrived; P.tap_keep_list = taps->keep_list;
+            P.tap_n_keep = taps->n_keep; P.tap_y = taps->y;
+            // records of the first block of every step: its selection is fixed (everything kept, scores zero)
+            for (int sidx = 0; sidx < steps; ++sidx) {
+                const size_t rec = static_cast<size_t>(sidx) * L;
+                const PersistSel* s0 = s->p_sel + 2;
+                auto copy = [&](void* dst, const void* src, size_t bytes) {
+                    return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+                };
+                bool ok = true;
+                if (taps->scores) ok = ok && cudaMemsetAsync(taps->scores + rec * G, 0, sizeof(float) * G, st) == cudaSuccess;
+                if (taps->dev_of_group) ok = ok && copy(taps->dev_of_group + rec * G, s0->dev_of_group, sizeof(int32_t) * G);
+                if (taps->arrived && n_dev > 0) ok = ok && copy(taps->arrived + rec * n_dev, s0->arrived, n_dev);
+                if (taps->keep_list) ok = ok && copy(taps->keep_list + rec * G, s0->keep_list, sizeof(int32_t) * G);
+                if (taps->n_keep) ok = ok && copy(taps->n_keep + rec, &s0->n_keep, sizeof(int32_t));
+                if (!ok) return HALO_ERR_CUDA;
+            }
+        }
+        rc = launch_stack_persistent(P, st);
+        if (rc != HALO_OK) return rc;
+        s->last_launches = 1;
+        return HALO_OK;
+    }
 #define HALO_TRY(call) do { rc = (call); if (rc != HALO_OK) return rc; } while (0)
 #define HALO_COPY(dst, src, bytes)                                                                    \
     do { if (cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToDevice, st) != cudaSuccess)     \
@@ -429,6 +518,12 @@ extern "C" halo_status halo_stack_status(halo_stack* s, uint32_t* value, void* s
     if (cudaMemcpyAsync(value, s->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return HALO_ERR_CUDA;
     return cuda_status(cudaStreamSynchronize(st));
+}
+
+extern "C" halo_status halo_stack_set_mode(halo_stack* s, int mode) {
+    if (!s || (mode != 0 && mode != 1)) return HALO_ERR_ARG;
+    s->mode = mode;
+    return HALO_OK;
 }
 
 extern "C" long long halo_stack_last_launches(const halo_stack* s) { return s ? s->last_launches : 0; }

@@ -9,8 +9,8 @@ select_kernel(const __grid_constant__ PlanDev plan, int G, const float* __restri
               uint32_t layer, int force_all, int32_t* order, int32_t* dev_of_group, uint8_t* arrived,
               uint8_t* keep, int32_t* keep_list, int32_t* n_keep, uint32_t* dev_status) {
     __shared__ SelectSmem sm;
-    select_block(sm, plan, G, scores, step, layer, force_all, order, dev_of_group, arrived, keep, keep_list,
-                 n_keep, dev_status);
+    select_block<1024>(sm, plan, G, scores, step, layer, force_all, order, dev_of_group, arrived, keep, keep_list,
+                       n_keep, dev_status, threadIdx.x, BlockSync());
 }
 
 // s[g] = <W2[g], hidden> for every group (one warp per group, strided), then the selection on those scores.
@@ -41,8 +41,8 @@ score_select_kernel(const __grid_constant__ PlanDev plan, int G, int rank, const
         if (lane == 0) { s_local[g] = acc; if (scores) scores[g] = acc; }
     }
     __syncthreads();
-    select_block(sm, plan, G, s_local, step, layer, force_all, order, dev_of_group, arrived, keep, keep_list,
-                 n_keep, dev_status);
+    select_block<1024>(sm, plan, G, s_local, step, layer, force_all, order, dev_of_group, arrived, keep, keep_list,
+                       n_keep, dev_status, threadIdx.x, BlockSync());
 }
 
 halo_status launch_select(const PlanDev& plan, int G, const float* scores, uint32_t step, uint32_t layer,

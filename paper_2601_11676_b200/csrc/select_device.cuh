@@ -1,5 +1,5 @@
-// Steps a2..a5 for one block of 1024 threads: rank by counting, critical choice, Algorithm-3 chunk lookup,
-// arrival mask, ordered compaction.  Callable from any kernel whose block has 1024 threads.
+// Steps a2..a5 for one cooperating set of NT threads: rank by counting, critical choice, Algorithm-3 chunk
+// lookup, arrival mask, ordered compaction.  `sync` is a barrier over exactly those NT threads.
 #pragma once
 #include "common.cuh"
 #include "philox.cuh"
@@ -8,44 +8,62 @@ namespace halo {
 
 struct SelectSmem {
     float score[HALO_MAX_GROUPS];
+    unsigned char kept[HALO_MAX_GROUPS];
     int boundary[HALO_MAX_DEVICES + 1];
     int arrived[HALO_MAX_DEVICES];
-    int warp_count[32];
     int flags;
+    int count;
 };
 
-// `scores` may point to global or shared memory.  All 1024 threads must call.
+// `scores` may point to global or shared memory.  All NT threads must call; tid in [0, NT).
+template <int NT, typename Sync>
 __device__ __forceinline__ void select_block(SelectSmem& sm, const PlanDev& plan, int G, const float* scores,
                                              uint32_t step, uint32_t layer, int force_all, int32_t* order,
                                              int32_t* dev_of_group, uint8_t* arrived, uint8_t* keep,
-                                             int32_t* keep_list, int32_t* n_keep, uint32_t* dev_status) {
-    const int tid = threadIdx.x;
-    const bool valid = tid < G;
-    float v = -INFINITY;
-    bool nonfinite = false;
-    if (valid) {
-        v = scores[tid];
-        if (isnan(v)) { v = -INFINITY; nonfinite = true; }
-        else if (isinf(v)) nonfinite = true;
-        if (v == 0.0f) v = 0.0f;  // -0 and +0 are one value
+                                             int32_t* keep_list, int32_t* n_keep, uint32_t* dev_status, int tid,
+                                             Sync sync) {
+    constexpr int PER = (HALO_MAX_GROUPS + NT - 1) / NT;
+    static_assert(NT > HALO_MAX_DEVICES, "one thread per boundary entry");
+    float v[PER];
+    if (tid == 0) { sm.flags = 0; sm.count = 0; }
+    sync();  // also orders any earlier use of sm by the caller
+    int above = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const int g = tid + i * NT;
+        v[i] = -INFINITY;
+        if (g < G) {
+            float s = scores[g];
+            bool nonfinite = false;
+            if (isnan(s)) { s = -INFINITY; nonfinite = true; }
+            else if (isinf(s)) nonfinite = true;
+            if (s == 0.0f) s = 0.0f;  // -0 and +0 are one value
+            v[i] = s;
+            sm.score[g] = s;
+            if (nonfinite) atomicOr(&sm.flags, 1);
+            if (s >= plan.threshold) ++above;
+        }
     }
-    if (tid == 0) sm.flags = 0;
-    __syncthreads();  // also orders any earlier use of sm by the caller
-    if (valid) sm.score[tid] = v;
-    if (nonfinite) atomicOr(&sm.flags, 1);
-    __syncthreads();
+    if (plan.mode == HALO_SEL_THRESHOLD && above) atomicAdd(&sm.count, above);
+    sync();
 
     // a2: position in the priority order = number of groups that come before this one
-    int rank = 0;
-    if (valid) {
-        for (int o = 0; o < G; ++o) {
-            const float so = sm.score[o];
-            rank += (so > v || (so == v && o < tid)) ? 1 : 0;
+    int rank[PER];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const int g = tid + i * NT;
+        rank[i] = 0;
+        if (g < G) {
+            int r = 0;
+            for (int o = 0; o < G; ++o) {
+                const float so = sm.score[o];
+                r += (so > v[i] || (so == v[i] && o < g)) ? 1 : 0;
+            }
+            rank[i] = r;
         }
     }
     // a3: number of critical groups
-    int k = plan.k_critical;
-    if (plan.mode == HALO_SEL_THRESHOLD) k = __syncthreads_count(valid && v >= plan.threshold);
+    int k = (plan.mode == HALO_SEL_THRESHOLD) ? sm.count : plan.k_critical;
     if (plan.n_dev == 0) k = G;
     const int M = G - k;
 
@@ -66,39 +84,51 @@ __device__ __forceinline__ void select_block(SelectSmem& sm, const PlanDev& plan
         sm.arrived[tid] = a ? 1 : 0;
         if (arrived) arrived[tid] = a ? 1 : 0;
     }
-    __syncthreads();
+    sync();
 
-    int dev = -1;
-    if (valid && rank >= k) {
-        const int p = rank - k;
-        for (int j = 0; j < plan.n_dev; ++j)
-            if (sm.boundary[j] <= p && p < sm.boundary[j + 1]) { dev = plan.dev_order[j]; break; }
+    int dev[PER];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const int g = tid + i * NT;
+        dev[i] = -1;
+        if (g < G) {
+            if (rank[i] >= k) {
+                const int p = rank[i] - k;
+                for (int j = 0; j < plan.n_dev; ++j)
+                    if (sm.boundary[j] <= p && p < sm.boundary[j + 1]) { dev[i] = plan.dev_order[j]; break; }
+            }
+            sm.kept[g] = (dev[i] < 0 || sm.arrived[dev[i]] != 0) ? 1 : 0;
+        }
     }
-    const bool kept = valid && (dev < 0 || sm.arrived[dev] != 0);
+    sync();
 
-    // ordered compaction: kept group ids ascending
-    const unsigned ballot = __ballot_sync(0xffffffffu, kept);
-    const int lane = tid & 31, warp = tid >> 5;
-    if (lane == 0) sm.warp_count[warp] = __popc(ballot);
-    __syncthreads();
-    int before = 0, total_kept = 0;
-    for (int w = 0; w < 32; ++w) {
-        const int c = sm.warp_count[w];
-        if (w < warp) before += c;
-        total_kept += c;
-    }
-    const int pos = before + __popc(ballot & ((1u << lane) - 1u));
-    if (valid) {
-        if (order) order[rank] = tid;
-        if (dev_of_group) dev_of_group[tid] = dev;
-        if (keep) keep[tid] = kept ? 1 : 0;
-        if (kept) keep_list[pos] = tid;
-        if (tid >= total_kept) keep_list[tid] = -1;  // padding behind the kept ids
+    // ordered compaction: a kept group's position = number of kept groups with a smaller id
+    int total_kept = 0;
+    for (int o = 0; o < G; ++o) total_kept += sm.kept[o];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const int g = tid + i * NT;
+        if (g < G) {
+            const bool kept = sm.kept[g] != 0;
+            if (order) order[rank[i]] = g;
+            if (dev_of_group) dev_of_group[g] = dev[i];
+            if (keep) keep[g] = kept ? 1 : 0;
+            if (kept) {
+                int pos = 0;
+                for (int o = 0; o < g; ++o) pos += sm.kept[o];
+                keep_list[pos] = g;
+            }
+            if (g >= total_kept) keep_list[g] = -1;  // padding behind the kept ids
+        }
     }
     if (tid == 0) {
         *n_keep = total_kept;
         if (sm.flags) flag_status(dev_status, HALO_DEV_NONFINITE_SCORE);
     }
 }
+
+struct BlockSync {
+    __device__ __forceinline__ void operator()() const { __syncthreads(); }
+};
 
 }  // namespace halo

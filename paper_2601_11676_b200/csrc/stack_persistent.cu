@@ -1,0 +1,543 @@
+// Decode stack as ONE persistent cooperative kernel: all steps x blocks of the FFN stack, steps a1..a9 plus
+// the glue between blocks, without leaving the device.
+//
+// One thread block per SM: a producer warp and 512 consumer threads around a ring of shared-memory stages fed
+// by bulk asynchronous copies.  The producer's stream for block l of a step is
+//     [rows of W1 of block l+1 owned by this thread block]   predictor hidden layer, one layer ahead (a1)
+//     [SELECT marker, last thread block only]                 scores, rank, assignment, arrival mask (a1..a5)
+//     [batches of NB kept neurons of block l]                 gate/up dot products, SiLU*up, down rows (a6..a8)
+//     [END marker]
+// and it runs ahead of the consumers by the ring depth, across the end of the block: while the consumers sit in
+// the grid barrier and the glue, the next block's weights are already landing in shared memory.
+// Per block there is one grid-wide barrier: column sums go to partials[slot] by fp32 vector reductions in L2,
+// barrier, then every thread block redundantly merges the slots (a9), adds the residual, normalises, and keeps
+// its own copy of x for the next block.  The selection of block l+1 is published early in block l, so the
+// producers never wait for it in practice.
+// Every wait (mbarrier, grid barrier, flags) is bounded to about a second; on a timeout the thread block takes
+// a uniform exit, raises a global abort word and HALO_DEV_TIMEOUT, and every other thread block follows.
+#include <algorithm>
+
+#include "common.cuh"
+#include "select_device.cuh"
+#include "stack_persistent.cuh"
+#include "tma.cuh"
+
+namespace halo {
+
+constexpr int kPC = 512;                 // consumer threads
+constexpr int kPCWarps = kPC / 32;
+constexpr int kPThreads = kPC + 32;      // + producer warp
+constexpr int kHeaderBytes = 12 * 1024;  // PersistSmem
+constexpr int kXsBytes = 16 * 1024;      // x as bf16, d <= 8192
+
+enum StageType { ST_FFN = 0, ST_PRED = 1, ST_SELECT = 2, ST_END = 3 };
+
+struct PersistSmem {
+    uint64_t full[8];
+    uint64_t empty[8];
+    int type[8];
+    int arg0[8];   // FFN: holder slot (-1 = skip); PRED: first row; SELECT: block to select for
+    int arg1[8];   // PRED: number of rows
+    int abort_flag;
+    int pad[3];
+    float red[2][32];
+    float reduce[32];
+    float score[HALO_MAX_GROUPS];
+    SelectSmem sel;
+};
+static_assert(sizeof(PersistSmem) <= kHeaderBytes, "shared-memory header too large");
+
+__device__ __forceinline__ void pc_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kPC) : "memory"); }
+// barrier over the consumers that also ORs a flag across them (uniform result)
+__device__ __forceinline__ bool pc_barrier_or(bool flag) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"(static_cast<uint32_t>(flag)), "n"(kPC)
+        : "memory");
+    return out != 0;
+}
+struct ConsumerSync {
+    __device__ __forceinline__ void operator()() const { pc_barrier(); }
+};
+
+// Bounded spin until *word >= target (acquire); gives up early when the global abort word is set.
+__device__ __forceinline__ bool spin_until_ge(const unsigned* word, unsigned target, const unsigned* abort_word) {
+    if (ld_acquire_gpu(word) >= target) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (true) {
+        if (ld_acquire_gpu(word) >= target) return true;
+        if ((++spins & 63u) == 0u) {
+            if (ld_acquire_gpu(abort_word) != 0u) return false;
+            if (clock64() - t0 > kWaitLimitCycles) return false;
+        }
+    }
+}
+
+template <int NB, int XC, int P2, int REP, int STAGES>
+__global__ void __launch_bounds__(kPThreads, 1)
+stack_decode_kernel(const __grid_constant__ PersistParams P) {
+    constexpr int ROWS = 2 * NB;
+    constexpr int WPR = kPCWarps / ROWS;
+    static_assert(WPR * ROWS == kPCWarps && STAGES <= 8 && NB % REP == 0, "shape");
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    PersistSmem& sm = *reinterpret_cast<PersistSmem*>(smem_raw);
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw + kHeaderBytes);
+    unsigned char* ring = smem_raw + kHeaderBytes + kXsBytes;
+
+    const int d = P.d, S = P.S, G = P.G, L = P.L, r = P.r, n_dev = P.plan.n_dev;
+    const int chunks = d >> 3;
+    const uint32_t row_bytes = static_cast<uint32_t>(d) * 2u;
+    const uint32_t plane_bytes = row_bytes * NB;
+    const uint32_t stage_bytes = 3u * plane_bytes;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int grid = gridDim.x, cta = blockIdx.x;
+    const bool is_selector = (cta == grid - 1);
+    const int per_group = S / NB;
+    unsigned* const sync_barrier = P.sync + 0;
+    unsigned* const sync_abort = P.sync + 1;
+    unsigned* const sync_zcount = P.sync + 2;
+    unsigned* const sync_selready = P.sync + 3;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], kPCWarps); }
+        sm.abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    volatile int* abort_flag = &sm.abort_flag;
+
+    // =========================================== producer ===========================================
+    if (warp == kPCWarps) {
+        if (lane != 0) return;
+        int it = 0;
+        bool alive = true;
+        auto acquire = [&](int& s) -> bool {
+            if (*abort_flag) return false;
+            s = it % STAGES;
+            if (it >= STAGES) {
+                const uint32_t use = static_cast<uint32_t>(it / STAGES);
+                if (!mbar_wait_bounded(&sm.empty[s], (use - 1u) & 1u, abort_flag)) { *abort_flag = 1; return false; }
+            }
+            return true;
+        };
+        auto marker = [&](int type, int a0) -> bool {
+            int s;
+            if (!acquire(s)) return false;
+            sm.type[s] = type; sm.arg0[s] = a0; sm.arg1[s] = 0;
+            mbar_arrive(&sm.full[s]);
+            ++it;
+            return true;
+        };
+        for (int step_i = 0; step_i < P.steps && alive; ++step_i) {
+            for (int l = 0; l < L && alive; ++l) {
+                // (a) rows of the next block's predictor that this thread block owns
+                if (l + 1 < L) {
+                    const int r0 = static_cast<int>(static_cast<long long>(cta) * r / grid);
+                    const int r1 = static_cast<int>(static_cast<long long>(cta + 1) * r / grid);
+                    const __nv_bfloat16* W1 = P.W1[l + 1];
+                    for (int row = r0; row < r1 && alive; row += ROWS) {
+                        const int n = min(ROWS, r1 - row);
+                        int s;
+                        if (!acquire(s)) { alive = false; break; }
+                        sm.type[s] = ST_PRED; sm.arg0[s] = row; sm.arg1[s] = n;
+                        mbar_arrive_expect_tx(&sm.full[s], n * row_bytes);
+                        bulk_copy_g2s(ring + static_cast<size_t>(s) * stage_bytes, W1 + static_cast<size_t>(row) * d,
+                                      n * row_bytes, &sm.full[s]);
+                        ++it;
+                    }
+                    if (alive && is_selector) alive = marker(ST_SELECT, l + 1);
+                }
+                if (!alive) break;
+                // (b) kept neurons of this block
+                const PersistSel* sb = &P.sel[2];
+                if (l > 0) {
+                    const unsigned need = static_cast<unsigned>(step_i) * (L - 1) + l;
+                    if (!spin_until_ge(sync_selready, need, sync_abort)) { *abort_flag = 1; alive = false; break; }
+                    sb = &P.sel[l & 1];
+                }
+                int nk = __ldcg(&sb->n_keep);
+                nk = max(0, min(nk, G));
+                const long long U = static_cast<long long>(nk) * per_group;
+                const long long U_eff = U + ((l + 1 < L) ? P.sel_cost : 0);
+                const long long lo = min(U, U_eff * cta / grid);
+                const long long hi = is_selector ? U : min(U, U_eff * (cta + 1) / grid);
+                const __nv_bfloat16* Wl = P.W[l];
+                for (long long b = lo; b < hi; ++b) {
+                    int s;
+                    if (!acquire(s)) { alive = false; break; }
+                    const int ki = static_cast<int>(b / per_group), j0 = static_cast<int>(b - static_cast<long long>(ki) * per_group) * NB;
+                    const int g = __ldcg(&sb->keep_list[ki]);
+                    int slot = -1;
+                    if (g >= 0 && g < G) {
+                        slot = __ldcg(&sb->dev_of_group[g]) + 1;
+                        if (slot < 0 || slot > n_dev) slot = -1;
+                    }
+                    sm.type[s] = ST_FFN; sm.arg0[s] = slot; sm.arg1[s] = 0;
+                    if (slot < 0) {
+                        flag_status(P.status, HALO_DEV_BAD_INDEX);
+                        mbar_arrive(&sm.full[s]);
+                    } else {
+                        const __nv_bfloat16* group = Wl + static_cast<size_t>(g) * 3 * S * d;
+                        unsigned char* dst = ring + static_cast<size_t>(s) * stage_bytes;
+                        mbar_arrive_expect_tx(&sm.full[s], stage_bytes);
+                        bulk_copy_g2s(dst, group + static_cast<size_t>(j0) * d, plane_bytes, &sm.full[s]);
+                        bulk_copy_g2s(dst + plane_bytes, group + static_cast<size_t>(S + j0) * d, plane_bytes, &sm.full[s]);
+                        bulk_copy_g2s(dst + 2 * plane_bytes, group + static_cast<size_t>(2 * S + j0) * d, plane_bytes,
+                                      &sm.full[s]);
+                    }
+                    ++it;
+                }
+                if (alive) alive = marker(ST_END, 0);
+            }
+        }
+        if (*abort_flag) {
+            // nobody consumes any more: let every copy this thread block issued land before it exits
+            const int first = it > STAGES ? it - STAGES : 0;
+            int never = 0;
+            for (int k = first; k < it; ++k)
+                mbar_wait_bounded(&sm.full[k % STAGES], static_cast<uint32_t>(k / STAGES) & 1u, &never);
+        }
+        return;
+    }
+
+    // =========================================== consumers ===========================================
+    const int row = warp / WPR, part = warp % WPR;
+    const int p1_base = part * (XC * 32) + lane;
+    const int rep = (REP > 1) ? tid / (kPC / REP) : 0;
+    const int col0 = (REP > 1) ? tid % (kPC / REP) : tid;
+    const bool owner = (REP == 1) || (rep == 0);   // threads that carry the residual stream for their columns
+    float xr[XC][8];
+    float acc[P2][8];
+    float hreg[P2][8];
+    int it = 0, red_par = 0;
+    unsigned q = 0;  // running block counter over steps: partial buffers rotate with it
+    const size_t slot_stride = static_cast<size_t>(d);
+    const size_t buf_stride = static_cast<size_t>(n_dev + 1) * d;
+    bool bad = false;
+
+    // normalise hreg -> xs (bf16) -> xr; thread block 0 records x as the input of block `l_next`
+    auto normalise_and_load_x = [&](int step_i, int l_next, bool want_x) {
+        float ss = 0.0f;
+        if (owner) {
+#pragma unroll
+            for (int p = 0; p < P2; ++p) {
+                const int c = col0 + kPC * p;
+                if (c < chunks) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) ss = fmaf(hreg[p][e], hreg[p][e], ss);
+                }
+            }
+        }
+        ss = warp_sum(ss);
+        if (lane == 0) sm.reduce[warp] = ss;
+        pc_barrier();
+        float tot = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kPCWarps; ++w) tot += sm.reduce[w];
+        const float scale = 1.0f / sqrtf(tot / static_cast<float>(d) + 1e-5f);
+        if (owner && want_x) {
+#pragma unroll
+            for (int p = 0; p < P2; ++p) {
+                const int c = col0 + kPC * p;
+                if (c < chunks) {
+                    __align__(16) __nv_bfloat16 xb[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) xb[e] = __float2bfloat16_rn(hreg[p][e] * scale);
+                    const uint4 packed = *reinterpret_cast<const uint4*>(xb);
+                    reinterpret_cast<uint4*>(xs)[c] = packed;
+                    if (cta == 0 && P.tap_x)
+                        reinterpret_cast<uint4*>(P.tap_x + (static_cast<size_t>(step_i) * L + l_next) * d)[c] = packed;
+                }
+            }
+        }
+        pc_barrier();  // xs complete; sm.reduce free again
+        if (want_x) {
+#pragma unroll
+            for (int i = 0; i < XC; ++i)
+                Elem<__nv_bfloat16>::widen(reinterpret_cast<const uint4*>(xs)[p1_base + 32 * i], xr[i]);
+        }
+    };
+
+    auto flush = [&](int slot) {
+        float* dst = P.partials + (q % 3u) * buf_stride + static_cast<size_t>(slot) * slot_stride;
+#pragma unroll
+        for (int p = 0; p < P2; ++p) {
+            const int c = col0 + kPC * p;
+            if (c < chunks) {
+                red_add_v4f(dst + c * 8, acc[p][0], acc[p][1], acc[p][2], acc[p][3]);
+                red_add_v4f(dst + c * 8 + 4, acc[p][4], acc[p][5], acc[p][6], acc[p][7]);
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[p][e] = 0.0f;
+        }
+    };
+
+    for (int step_i = 0; step_i < P.steps && !bad; ++step_i) {
+        // residual stream of this step, and the first block's input
+        if (owner) {
+#pragma unroll
+            for (int p = 0; p < P2; ++p) {
+                const int c = col0 + kPC * p;
+                if (c < chunks) {
+                    const float4* src = reinterpret_cast<const float4*>(P.h0 + static_cast<size_t>(step_i) * d + c * 8);
+                    const float4 a = __ldg(src), b = __ldg(src + 1);
+                    hreg[p][0] = a.x; hreg[p][1] = a.y; hreg[p][2] = a.z; hreg[p][3] = a.w;
+                    hreg[p][4] = b.x; hreg[p][5] = b.y; hreg[p][6] = b.z; hreg[p][7] = b.w;
+                }
+            }
+        }
+        normalise_and_load_x(step_i, 0, true);
+
+        for (int l = 0; l < L && !bad; ++l) {
+#pragma unroll
+            for (int p = 0; p < P2; ++p)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[p][e] = 0.0f;
+            int cur_slot = -1;
+
+            // ------------------------------ stages of this block ------------------------------
+            while (true) {
+                const int s = it % STAGES;
+                const uint32_t parity = static_cast<uint32_t>(it / STAGES) & 1u;
+                const bool ok = mbar_wait_bounded(&sm.full[s], parity, abort_flag);
+                const int type = sm.type[s], a0 = sm.arg0[s], a1 = sm.arg1[s];
+                const unsigned char* stage = ring + static_cast<size_t>(s) * stage_bytes;
+                float* red = sm.red[red_par];
+                bool okz = true;
+                // ---- before the barrier: nothing in here may block on other consumers ----
+                if (type == ST_FFN) {
+                    if (a0 >= 0) {
+                        if (a0 != cur_slot) {
+                            if (cur_slot >= 0) flush(cur_slot);
+                            cur_slot = a0;
+                        }
+                        const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(row) * row_bytes);
+                        float dot = 0.0f;
+#pragma unroll
+                        for (int i = 0; i < XC; ++i) {
+                            float w8[8];
+                            Elem<__nv_bfloat16>::widen(rp[p1_base + 32 * i], w8);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) dot = fmaf(w8[e], xr[i][e], dot);
+                        }
+                        dot = warp_sum(dot);
+                        if (lane == 0) red[row * WPR + part] = dot;
+                    }
+                } else if (type == ST_PRED) {
+                    if (row < a1) {
+                        const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(row) * row_bytes);
+                        float dot = 0.0f;
+#pragma unroll
+                        for (int i = 0; i < XC; ++i) {
+                            float w8[8];
+                            Elem<__nv_bfloat16>::widen(rp[p1_base + 32 * i], w8);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) dot = fmaf(w8[e], xr[i][e], dot);
+                        }
+                        dot = warp_sum(dot);
+                        if (lane == 0) red[row * WPR + part] = dot;
+                    }
+                } else if (type == ST_SELECT) {
+                    if (tid == 0) {
+                        const unsigned n_pred = static_cast<unsigned>(step_i) * (L - 1) + a0;
+                        okz = spin_until_ge(sync_zcount, n_pred * static_cast<unsigned>(r), sync_abort);
+                    }
+                }
+                bad = pc_barrier_or(!ok || !okz);
+                if (bad) break;
+                // ---- after the barrier ----
+                if (type == ST_FFN) {
+                    if (a0 >= 0) {
+                        const unsigned char* down = stage + 2 * plane_bytes;
+#pragma unroll
+                        for (int jj = 0; jj < NB / REP; ++jj) {
+                            const int j = jj * REP + rep;
+                            float a = 0.0f, b = 0.0f;
+#pragma unroll
+                            for (int w = 0; w < WPR; ++w) { a += red[j * WPR + w]; b += red[(NB + j) * WPR + w]; }
+                            const float h = a / (1.0f + __expf(-a)) * b;
+                            const uint4* dr = reinterpret_cast<const uint4*>(down + static_cast<size_t>(j) * row_bytes);
+#pragma unroll
+                            for (int p = 0; p < P2; ++p) {
+                                const int c = col0 + kPC * p;
+                                if (P2 == 1 || c < chunks) {
+                                    float w8[8];
+                                    Elem<__nv_bfloat16>::widen(dr[c], w8);
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) acc[p][e] = fmaf(h, w8[e], acc[p][e]);
+                                }
+                            }
+                        }
+                    }
+                    red_par ^= 1;
+                } else if (type == ST_PRED) {
+                    if (tid == 0) {
+                        for (int i = 0; i < a1; ++i) {
+                            float z = 0.0f;
+                            for (int w = 0; w < WPR; ++w) z += red[i * WPR + w];
+                            if (P.act == HALO_ACT_RELU) z = fmaxf(z, 0.0f);
+                            P.z[a0 + i] = z;
+                        }
+                        __threadfence();
+                        atomicAdd(sync_zcount, static_cast<unsigned>(a1));
+                    }
+                    red_par ^= 1;
+                } else if (type == ST_SELECT) {
+                    // a1 (second layer): s[g] = <W2[g], z>; then a2..a5 for block a0, published for the producers
+                    const int lp = a0;
+                    const __nv_bfloat16* W2 = P.W2[lp];
+                    const int zc = r >> 3;
+                    for (int g = warp; g < G; g += kPCWarps) {
+                        const uint4* wrow = reinterpret_cast<const uint4*>(W2 + static_cast<size_t>(g) * r);
+                        float dot = 0.0f;
+                        for (int c = lane; c < zc; c += 32) {
+                            float w8[8];
+                            Elem<__nv_bfloat16>::widen(__ldg(wrow + c), w8);
+                            const float4 z0 = __ldcg(reinterpret_cast<const float4*>(P.z) + 2 * c);
+                            const float4 z1 = __ldcg(reinterpret_cast<const float4*>(P.z) + 2 * c + 1);
+                            dot = fmaf(w8[0], z0.x, dot); dot = fmaf(w8[1], z0.y, dot);
+                            dot = fmaf(w8[2], z0.z, dot); dot = fmaf(w8[3], z0.w, dot);
+                            dot = fmaf(w8[4], z1.x, dot); dot = fmaf(w8[5], z1.y, dot);
+                            dot = fmaf(w8[6], z1.z, dot); dot = fmaf(w8[7], z1.w, dot);
+                        }
+                        dot = warp_sum(dot);
+                        if (lane == 0) sm.score[g] = dot;
+                    }
+                    pc_barrier();
+                    PersistSel* sb = &P.sel[lp & 1];
+                    select_block<kPC>(sm.sel, P.plan, G, sm.score, P.step0 + static_cast<uint32_t>(step_i),
+                                      static_cast<uint32_t>(lp), 0, nullptr, sb->dev_of_group, sb->arrived, nullptr,
+                                      sb->keep_list, &sb->n_keep, P.status, tid, ConsumerSync());
+                    __threadfence();
+                    pc_barrier();
+                    const size_t rec = static_cast<size_t>(step_i) * L + lp;
+                    for (int g = tid; g < G; g += kPC) {
+                        if (P.tap_scores) P.tap_scores[rec * G + g] = sm.score[g];
+                        if (P.tap_keep_list) P.tap_keep_list[rec * G + g] = __ldcg(&sb->keep_list[g]);
+                        if (P.tap_dev_of_group) P.tap_dev_of_group[rec * G + g] = __ldcg(&sb->dev_of_group[g]);
+                    }
+                    if (tid < n_dev && P.tap_arrived) P.tap_arrived[rec * n_dev + tid] = static_cast<uint8_t>(sm.sel.arrived[tid]);
+                    if (tid == 0) {
+                        if (P.tap_n_keep) P.tap_n_keep[rec] = __ldcg(&sb->n_keep);
+                        st_release_gpu(sync_selready, static_cast<unsigned>(step_i) * (L - 1) + lp);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.empty[s]);
+                ++it;
+                if (type == ST_END) break;
+            }
+            if (bad) break;
+
+            // ------------------------------ end of the block: flush, grid barrier, merge + glue ------------------------------
+            if (cur_slot >= 0) flush(cur_slot);
+            __threadfence();
+            pc_barrier();
+            bool okb = true;
+            if (tid == 0) {
+                __threadfence();
+                atomicAdd(sync_barrier, 1u);
+                okb = spin_until_ge(sync_barrier, (q + 1u) * static_cast<unsigned>(grid), sync_abort);
+            }
+            bad = pc_barrier_or(!okb);
+            if (bad) break;
+
+            // a9 + residual: every thread block merges all slots for its own copy of the stream
+            const float* pbuf = P.partials + (q % 3u) * buf_stride;
+            float* zbuf = P.partials + ((q + 2u) % 3u) * buf_stride;   // read two blocks ago by everyone: clear it
+            const size_t rec = static_cast<size_t>(step_i) * L + l;
+            if (owner) {
+#pragma unroll
+                for (int p = 0; p < P2; ++p) {
+                    const int c = col0 + kPC * p;
+                    if (c < chunks) {
+                        float y[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                        for (int slot = 0; slot <= n_dev; ++slot) {
+                            const float4* src = reinterpret_cast<const float4*>(pbuf + static_cast<size_t>(slot) * slot_stride + c * 8);
+                            const float4 a = __ldcg(src), b = __ldcg(src + 1);
+                            y[0] += a.x; y[1] += a.y; y[2] += a.z; y[3] += a.w;
+                            y[4] += b.x; y[5] += b.y; y[6] += b.z; y[7] += b.w;
+                        }
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) hreg[p][e] += y[e];
+                        if (cta == 0) {
+                            if (P.tap_y) {
+                                float4* dst = reinterpret_cast<float4*>(P.tap_y + rec * d + c * 8);
+                                dst[0] = make_float4(y[0], y[1], y[2], y[3]);
+                                dst[1] = make_float4(y[4], y[5], y[6], y[7]);
+                            }
+                            if (l == L - 1) {
+                                float4* dst = reinterpret_cast<float4*>(P.h_out + static_cast<size_t>(step_i) * d + c * 8);
+                                dst[0] = make_float4(hreg[p][0], hreg[p][1], hreg[p][2], hreg[p][3]);
+                                dst[1] = make_float4(hreg[p][4], hreg[p][5], hreg[p][6], hreg[p][7]);
+                            }
+                            for (int slot = 0; slot <= n_dev; ++slot) {
+                                float4* dst = reinterpret_cast<float4*>(zbuf + static_cast<size_t>(slot) * slot_stride + c * 8);
+                                dst[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                dst[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            }
+                        }
+                    }
+                }
+            }
+            ++q;
+            if (l + 1 < L) normalise_and_load_x(step_i, l + 1, true);
+        }
+    }
+    if (bad && tid == 0) {
+        *abort_flag = 1;                 // the producer stops and drains
+        atomicExch(sync_abort, 1u);      // every other thread block follows
+        flag_status(P.status, HALO_DEV_TIMEOUT);
+    }
+}
+
+// ---- host side -----------------------------------------------------------------------------------------
+
+bool persistent_supported(const halo_ffn_shape& sh, int n_tok, int G) {
+    if (sh.wdtype != HALO_BF16 || n_tok != 1 || G > kPC) return false;
+    switch (sh.d_model) {
+        case 2048: return sh.group_size % 4 == 0;
+        case 4096: case 5120: return sh.group_size % 2 == 0;
+        case 8192: return true;
+    }
+    return false;
+}
+
+template <int NB, int XC, int P2, int REP, int STAGES>
+static halo_status launch_cfg(PersistParams& P, cudaStream_t st) {
+    auto kernel = stack_decode_kernel<NB, XC, P2, REP, STAGES>;
+    const size_t smem = kHeaderBytes + kXsBytes + static_cast<size_t>(STAGES) * 3 * NB * P.d * 2;
+    static int blocks_per_sm = -1;
+    int dev = 0, sms = kSmCount;
+    if (cudaGetDevice(&dev) != cudaSuccess) return HALO_ERR_CUDA;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (blocks_per_sm < 0) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+            return HALO_ERR_CUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, kernel, kPThreads, smem) != cudaSuccess)
+            return HALO_ERR_CUDA;
+    }
+    if (blocks_per_sm < 1) return HALO_ERR_CUDA;
+    void* args[] = {&P};
+    if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(sms), dim3(kPThreads), args, smem, st) != cudaSuccess)
+        return HALO_ERR_CUDA;
+    return HALO_OK;
+}
+
+halo_status launch_stack_persistent(PersistParams& P, cudaStream_t st) {
+    switch (P.d) {
+        case 2048: return launch_cfg<4, 4, 1, 2, 4>(P, st);
+        case 4096: return launch_cfg<2, 4, 1, 1, 4>(P, st);
+        case 5120: return launch_cfg<2, 5, 2, 1, 3>(P, st);
+        case 8192: return launch_cfg<1, 4, 2, 1, 4>(P, st);
+    }
+    return HALO_ERR_UNIMPLEMENTED;
+}
+
+}  // namespace halo

@@ -82,14 +82,40 @@ def check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=0):
     return lost_layers
 
 
+@pytest.mark.parametrize("mode", [0, 1])  # 0: persistent single kernel where supported; 1: one launch per step
 @pytest.mark.parametrize("name,layers,steps", [("tinyllama-1.1b-decode", 4, 3), ("llama2-7b-decode", 3, 2),
                                                ("llama2-13b-decode", 3, 2)])
-def test_stack_decode_teacher_forced(name, layers, steps):
+def test_stack_decode_teacher_forced(name, layers, steps, mode):
     wl = synth.small_variant(synth.workload(name), layers, steps)
     stack, Wp, preds = build_stack(wl)
+    stack.set_mode(mode)
     h0, h_out, t = run_with_taps(wl, stack, steps, step0=3)
     check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=3)
-    assert stack.last_launches() > 0
+    assert stack.last_launches() == 1 if mode == 0 else stack.last_launches() > 1
+
+
+def test_stack_persistent_many_steps_with_losses_and_single_layer():
+    """Longer run of the single-kernel path: lossy devices so kept sets change every block; and a 1-block stack."""
+    wl = synth.Workload("m", 5, 2048, 64 * 12, 64, 128, "bf16", (0.0, 0.3, 0.6), (2, 1, 1), 250, 10)
+    stack, Wp, preds = build_stack(wl)
+    h0, h_out, t = run_with_taps(wl, stack, wl.steps)
+    assert stack.last_launches() == 1
+    lost = check_teacher_forced(wl, Wp, preds, h0, h_out, t, wl.steps)
+    assert lost > 0
+    one = synth.Workload("o", 1, 4096, 128 * 5, 128, 64, "bf16", (0.5,), (1,), 400, 3)
+    stack, Wp, preds = build_stack(one)
+    h0, h_out, t = run_with_taps(one, stack, one.steps)
+    check_teacher_forced(one, Wp, preds, h0, h_out, t, one.steps)
+
+
+def test_stack_persistent_everything_lost_gives_identity_blocks():
+    """k = 0 and every device always lost: from the second block on nothing is kept and the stream passes through."""
+    wl = synth.Workload("z", 3, 4096, 128 * 4, 128, 64, "bf16", (1.0, 1.0), (1, 1), 0, 2)
+    stack, Wp, preds = build_stack(wl)
+    h0, h_out, t = run_with_taps(wl, stack, wl.steps)
+    assert (t["n_keep"][:, 1:] == 0).all().item() and (t["n_keep"][:, 0] == wl.n_groups).all().item()
+    assert (t["y"][:, 1:] == 0).all().item()
+    check_teacher_forced(wl, Wp, preds, h0, h_out, t, wl.steps)
 
 
 def test_stack_small_f32_many_steps_sees_losses():

@@ -241,6 +241,13 @@ halo_status halo_stack_decode_host(halo_stack* stack, const float* h0_host, int 
  * l+1 overlapped with the weight stream of block l; anything else runs one launch per step of the path.
  * mode 1: always one launch per step of the path (no overlap; for comparison and checking). */
 halo_status halo_stack_set_mode(halo_stack* stack, int mode);
+/* Tracing of the persistent kernel (timing statistics of the generation loop): the caller gives a device
+ * buffer trace[n_blocks][halo_stack_trace_width()][8] of 64-bit words; for the first n_blocks blocks of a
+ * halo_stack_decode run every thread block records global-timer nanoseconds at: 0 block start, 1 first weight
+ * stage landed, 2 last stage consumed, 3 partial sums flushed, 4 grid barrier passed, 5 slots merged,
+ * 6 next input ready; 7 = duration of the selection (selecting thread block only).  n_blocks = 0 turns it off. */
+halo_status halo_stack_set_trace(halo_stack* stack, unsigned long long* trace /*device*/, int n_blocks);
+int halo_stack_trace_width(const halo_stack* stack);
 /* Device status word accumulated by the stack's launches (synchronises the stream). */
 halo_status halo_stack_status(halo_stack* stack, uint32_t* dev_status_value /*host*/, void* stream);
 /* Number of kernel launches the last halo_stack_decode enqueued. */

@@ -27,7 +27,7 @@ EXPORTS = [
     "halo_predict_workspace_bytes", "halo_predict_groups", "halo_select_groups", "halo_group_ffn_workspace_bytes",
     "halo_group_ffn", "halo_merge_partials", "halo_pack_weights", "halo_glue", "halo_stack_create",
     "halo_stack_destroy", "halo_stack_decode", "halo_stack_decode_host", "halo_stack_status",
-    "halo_stack_last_launches", "halo_stack_set_mode",
+    "halo_stack_last_launches", "halo_stack_set_mode", "halo_stack_set_trace", "halo_stack_trace_width",
 ]
 
 
@@ -88,6 +88,9 @@ def lib() -> ctypes.CDLL:
         L.halo_stack_decode_host.argtypes = [c_void_p, c_void_p, c_int, c_uint32, c_void_p, c_void_p]
         L.halo_stack_status.argtypes = [c_void_p, POINTER(c_uint32), c_void_p]
         L.halo_stack_set_mode.argtypes = [c_void_p, c_int]
+        L.halo_stack_set_trace.argtypes = [c_void_p, c_void_p, c_int]
+        L.halo_stack_trace_width.argtypes = [c_void_p]
+        L.halo_stack_trace_width.restype = c_int
         L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
         _lib = L
     return _lib
@@ -237,6 +240,14 @@ class Stack:
 
     def set_mode(self, mode: int) -> None:
         _chk(lib().halo_stack_set_mode(self.handle, mode), "halo_stack_set_mode")
+
+    def set_trace(self, n_blocks: int):
+        """Allocates and attaches a trace buffer [n_blocks][width][8] (int64, ns); returns the tensor."""
+        width = int(lib().halo_stack_trace_width(self.handle))
+        self._trace = torch.zeros((max(n_blocks, 1), width, 8), dtype=torch.int64, device="cuda") if n_blocks else None
+        _chk(lib().halo_stack_set_trace(self.handle, _ptr(self._trace) if n_blocks else None, n_blocks),
+             "halo_stack_set_trace")
+        return self._trace
 
     def status(self, stream=None) -> int:
         v = c_uint32(0)

@@ -2,6 +2,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -261,10 +262,13 @@ struct halo_stack {
     const void** d_W;              // device pointer tables
     const void** d_W1;
     const void** d_W2;
-    float* p_partials;             // [3][n_dev+1][d]
+    float* p_partials;             // [3][2][d]
     float* p_z;
     halo::PersistSel* p_sel;       // [3]
-    unsigned* p_sync;              // [4]
+    unsigned* p_sync;              // [32]
+    unsigned long long* trace;     // caller-owned, optional
+    int trace_blocks;
+    int cross_stages, l2_ahead;    // tuning of the persistent kernel
 };
 
 extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred,
@@ -317,10 +321,10 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     const size_t o_so = carve(sizeof(float) * s->stage_steps * step_elems);
     const size_t o_tw = carve(sizeof(void*) * n_layers), o_tw1 = carve(sizeof(void*) * n_layers);
     const size_t o_tw2 = carve(sizeof(void*) * n_layers);
-    const size_t o_pp = carve(sizeof(float) * 3 * (s->n_dev + 1) * d);
+    const size_t o_pp = carve(sizeof(float) * 3 * 2 * d);
     const size_t o_pz = carve(sizeof(float) * pred->rank);
     const size_t o_ps = carve(sizeof(PersistSel) * 3);
-    const size_t o_py = carve(sizeof(unsigned) * 4);
+    const size_t o_py = carve(sizeof(unsigned) * 32);
     if (cudaMalloc(&s->slab, off) != cudaSuccess) { delete s; return HALO_ERR_NOMEM; }
     if (cudaMemset(s->slab, 0, off) != cudaSuccess) { cudaFree(s->slab); delete s; return HALO_ERR_CUDA; }
     char* base = static_cast<char*>(s->slab);
@@ -346,6 +350,12 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     s->p_sel = reinterpret_cast<PersistSel*>(base + o_ps);
     s->p_sync = reinterpret_cast<unsigned*>(base + o_py);
     s->mode = 0;
+    s->trace = nullptr;
+    s->trace_blocks = 0;
+    s->cross_stages = 1;
+    s->l2_ahead = 0;
+    if (const char* e = std::getenv("HALO_TUNE_CROSS_STAGES")) s->cross_stages = std::max(0, std::atoi(e));
+    if (const char* e = std::getenv("HALO_TUNE_L2_AHEAD")) s->l2_ahead = std::min(32, std::max(0, std::atoi(e)));
     s->persistent_ok = persistent_supported(*ffn, n_tok, G);
     {
         // pointer tables, and the first block's selection: reliable block, all scores equal -> the priority
@@ -393,19 +403,21 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
     halo_status rc;
     if (s->persistent_ok && s->mode == 0) {
         // whole run in one cooperative launch
-        if (cudaMemsetAsync(s->p_partials, 0, sizeof(float) * 3 * (n_dev + 1) * d, st) != cudaSuccess ||
-            cudaMemsetAsync(s->p_sync, 0, sizeof(unsigned) * 4, st) != cudaSuccess)
+        if (cudaMemsetAsync(s->p_partials, 0, sizeof(float) * 3 * 2 * d, st) != cudaSuccess ||
+            cudaMemsetAsync(s->p_sync, 0, sizeof(unsigned) * 32, st) != cudaSuccess)
             return HALO_ERR_CUDA;
         PersistParams P;
         std::memset(&P, 0, sizeof(P));
         P.L = L; P.steps = steps; P.d = static_cast<int>(d); P.S = s->ffn.group_size; P.G = G; P.r = s->pred.rank;
-        P.act = s->pred.act; P.step0 = step0; P.sel_cost = 4;
+        P.act = s->pred.act; P.step0 = step0;
         P.W = reinterpret_cast<const __nv_bfloat16* const*>(s->d_W);
         P.W1 = reinterpret_cast<const __nv_bfloat16* const*>(s->d_W1);
         P.W2 = reinterpret_cast<const __nv_bfloat16* const*>(s->d_W2);
         P.h0 = h0; P.h_out = h_out; P.partials = s->p_partials; P.z = s->p_z; P.sel = s->p_sel; P.sync = s->p_sync;
         P.status = s->status;
         P.plan = s->plan.dev;
+        P.trace = s->trace; P.trace_blocks = s->trace_blocks;
+        P.cross_stages = s->cross_stages; P.l2_ahead = s->l2_ahead;
         if (taps) {
             P.tap_x = static_cast<__nv_bfloat16*>(taps->x); P.tap_scores = taps->scores;
             P.tap_dev_of_group = taps->dev_of_group; P.tap_arrived = taps->arrived; P.tap_keep_list = taps->keep_list;
@@ -524,6 +536,20 @@ extern "C" halo_status halo_stack_set_mode(halo_stack* s, int mode) {
     if (!s || (mode != 0 && mode != 1)) return HALO_ERR_ARG;
     s->mode = mode;
     return HALO_OK;
+}
+
+extern "C" halo_status halo_stack_set_trace(halo_stack* s, unsigned long long* trace, int n_blocks) {
+    if (!s || n_blocks < 0 || (n_blocks > 0 && !trace)) return HALO_ERR_ARG;
+    s->trace = n_blocks > 0 ? trace : nullptr;
+    s->trace_blocks = n_blocks;
+    return HALO_OK;
+}
+
+extern "C" int halo_stack_trace_width(const halo_stack* s) {
+    int dev = 0, sms = kSmCount;
+    (void)s;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms;
 }
 
 extern "C" long long halo_stack_last_launches(const halo_stack* s) { return s ? s->last_launches : 0; }

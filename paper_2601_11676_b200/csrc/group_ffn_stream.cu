@@ -14,6 +14,7 @@
 // Every wait on an mbarrier is bounded: if one runs out the block flags HALO_DEV_TIMEOUT, stops waiting,
 // drains its outstanding copies (bounded) and returns.
 #include "common.cuh"
+#include "ffn_math.cuh"
 #include "tma.cuh"
 
 namespace halo {
@@ -29,7 +30,7 @@ struct StreamSmemHeader {
     int slot[8];        // holder slot of the batch in each stage, -1 = skip
     int abort_flag;
     int pad[3];
-    float red[2][32];   // [parity][row * warps_per_row + part]
+    __align__(16) float red[2][32];   // [parity][row * warps_per_row + part]
 };
 
 // NB   neurons per batch; XC  16-byte chunks of a row per lane in phase 1;
@@ -124,11 +125,11 @@ group_ffn_stream_kernel(int d, int S, int G, const __nv_bfloat16* __restrict__ W
     // ---------------- consumers ----------------
     const int row = warp / WPR, part = warp % WPR;   // phase 1: which row, which slice of it
     const int p1_base = part * (XC * 32) + lane;      // chunk index of this lane's first chunk; stride 32
-    float xr[XC][8];
+    uint4 xq[XC];  // this lane's slice of x, packed bf16
     {
         const uint4* xg = reinterpret_cast<const uint4*>(x_all + static_cast<size_t>(tok) * d);
 #pragma unroll
-        for (int i = 0; i < XC; ++i) Elem<__nv_bfloat16>::widen(__ldg(xg + p1_base + 32 * i), xr[i]);
+        for (int i = 0; i < XC; ++i) xq[i] = __ldg(xg + p1_base + 32 * i);
     }
     const int rep = (REP > 1) ? tid / (kConsumers / REP) : 0;   // phase 2 replica
     const int col0 = (REP > 1) ? tid % (kConsumers / REP) : tid;
@@ -168,15 +169,10 @@ group_ffn_stream_kernel(int d, int S, int G, const __nv_bfloat16* __restrict__ W
             }
             // phase 1: rows 0..NB-1 are gate rows, NB..2NB-1 the up rows (planes 0 and 1 are adjacent)
             const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(row) * row_bytes);
-            float dot = 0.0f;
+            float dot0 = 0.0f, dot1 = 0.0f;
 #pragma unroll
-            for (int i = 0; i < XC; ++i) {
-                float w8[8];
-                Elem<__nv_bfloat16>::widen(rp[p1_base + 32 * i], w8);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) dot = fmaf(w8[e], xr[i][e], dot);
-            }
-            dot = warp_sum(dot);
+            for (int i = 0; i < XC; ++i) dot_bf16x8(rp[p1_base + 32 * i], xq[i], dot0, dot1);
+            const float dot = warp_sum(dot0 + dot1);
             if (lane == 0) red[row * WPR + part] = dot;
         }
         consumer_barrier();
@@ -186,20 +182,12 @@ group_ffn_stream_kernel(int d, int S, int G, const __nv_bfloat16* __restrict__ W
 #pragma unroll
             for (int jj = 0; jj < NB / REP; ++jj) {
                 const int j = jj * REP + rep;
-                float a = 0.0f, b = 0.0f;
-#pragma unroll
-                for (int q = 0; q < WPR; ++q) { a += red[j * WPR + q]; b += red[(NB + j) * WPR + q]; }
-                const float h = a / (1.0f + __expf(-a)) * b;
+                const float h = silu_mul(sum_parts<WPR>(red + j * WPR), sum_parts<WPR>(red + (NB + j) * WPR));
                 const uint4* dr = reinterpret_cast<const uint4*>(down + static_cast<size_t>(j) * row_bytes);
 #pragma unroll
                 for (int p = 0; p < P2; ++p) {
                     const int c = col0 + kConsumers * p;
-                    if (P2 == 1 || c < chunks) {
-                        float w8[8];
-                        Elem<__nv_bfloat16>::widen(dr[c], w8);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) acc[p][e] = fmaf(h, w8[e], acc[p][e]);
-                    }
+                    if (P2 == 1 || c < chunks) axpy_bf16x8(h, dr[c], acc[p]);
                 }
             }
         }

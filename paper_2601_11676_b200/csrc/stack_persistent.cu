@@ -9,15 +9,19 @@
 //     [END marker]
 // and it runs ahead of the consumers by the ring depth, across the end of the block: while the consumers sit in
 // the grid barrier and the glue, the next block's weights are already landing in shared memory.
-// Per block there is one grid-wide barrier: column sums go to partials[slot] by fp32 vector reductions in L2,
-// barrier, then every thread block redundantly merges the slots (a9), adds the residual, normalises, and keeps
-// its own copy of x for the next block.  The selection of block l+1 is published early in block l, so the
+// Batches are handed out dynamically (one atomic counter per block, fetched one batch ahead), so a slow or busy
+// thread block simply takes fewer.  Only kept groups are ever computed, so the merge (a9) is the plain sum of
+// what was computed: each thread block stages its column sums in shared memory and adds them to one of
+// kAccBufs interleaved global buffers with ONE bulk reduction (cp.reduce.async.bulk, fp32 add, done by the copy
+// engine in L2), then one grid-wide barrier, then every thread block redundantly sums the buffers,
+// adds the residual, normalises, and keeps its own copy of x for the next block.  The selection of block l+1 is published early in block l, so the
 // producers never wait for it in practice.
 // Every wait (mbarrier, grid barrier, flags) is bounded to about a second; on a timeout the thread block takes
 // a uniform exit, raises a global abort word and HALO_DEV_TIMEOUT, and every other thread block follows.
 #include <algorithm>
 
 #include "common.cuh"
+#include "ffn_math.cuh"
 #include "select_device.cuh"
 #include "stack_persistent.cuh"
 #include "tma.cuh"
@@ -27,8 +31,9 @@ namespace halo {
 constexpr int kPC = 512;                 // consumer threads
 constexpr int kPCWarps = kPC / 32;
 constexpr int kPThreads = kPC + 32;      // + producer warp
-constexpr int kHeaderBytes = 12 * 1024;  // PersistSmem
-constexpr int kXsBytes = 16 * 1024;      // x as bf16, d <= 8192
+constexpr int kHeaderBytes = 16 * 1024;  // PersistSmem
+constexpr int kAccBufs = 2;              // interleaved accumulation buffers per block of the stack
+constexpr int kFetchAhead = 3;           // batch-counter fetches a producer keeps in flight
 
 enum StageType { ST_FFN = 0, ST_PRED = 1, ST_SELECT = 2, ST_END = 3 };
 
@@ -39,10 +44,12 @@ struct PersistSmem {
     int arg0[8];   // FFN: holder slot (-1 = skip); PRED: first row; SELECT: block to select for
     int arg1[8];   // PRED: number of rows
     int abort_flag;
-    int pad[3];
-    float red[2][32];
+    int blocks_done;   // blocks of the stack whose grid barrier this thread block's consumers have passed
+    int pad[2];
+    __align__(16) float red[2][32];
     float reduce[32];
     float score[HALO_MAX_GROUPS];
+    int kept_group[HALO_MAX_GROUPS];   // producer's table for the block it is issuing: group id or -1 per kept position
     SelectSmem sel;
 };
 static_assert(sizeof(PersistSmem) <= kHeaderBytes, "shared-memory header too large");
@@ -79,6 +86,16 @@ __device__ __forceinline__ bool spin_until_ge(const unsigned* word, unsigned tar
     }
 }
 
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// trace slots per (block of the stack, thread block)
+enum TraceSlot { TR_BLOCK_START = 0, TR_FIRST_STAGE = 1, TR_STAGES_DONE = 2, TR_FLUSHED = 3, TR_BARRIER_DONE = 4,
+                 TR_MERGED = 5, TR_X_READY = 6, TR_SELECT_NS = 7 };
+
 template <int NB, int XC, int P2, int REP, int STAGES>
 __global__ void __launch_bounds__(kPThreads, 1)
 stack_decode_kernel(const __grid_constant__ PersistParams P) {
@@ -87,8 +104,11 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
     static_assert(WPR * ROWS == kPCWarps && STAGES <= 8 && NB % REP == 0, "shape");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     PersistSmem& sm = *reinterpret_cast<PersistSmem*>(smem_raw);
-    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem_raw + kHeaderBytes);
-    unsigned char* ring = smem_raw + kHeaderBytes + kXsBytes;
+    // one vector buffer, used in turn for the fp32 column sums on their way out and for x (bf16) on its way in
+    constexpr int kVecBytesPerCol = 4 * REP;
+    unsigned char* vec_buf = smem_raw + kHeaderBytes;
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(vec_buf);
+    unsigned char* ring = smem_raw + kHeaderBytes + static_cast<size_t>(P.d) * kVecBytesPerCol;
 
     const int d = P.d, S = P.S, G = P.G, L = P.L, r = P.r, n_dev = P.plan.n_dev;
     const int chunks = d >> 3;
@@ -107,6 +127,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], kPCWarps); }
         sm.abort_flag = 0;
+        sm.blocks_done = 0;
         mbar_fence_init();
     }
     __syncthreads();
@@ -114,11 +135,25 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
 
     // =========================================== producer ===========================================
     if (warp == kPCWarps) {
-        if (lane != 0) return;
+        // Lane 0 issues every copy; the other lanes only help to build the per-block table of kept groups.
         int it = 0;
+        unsigned qp = 0;  // running block counter of the producer
+        int issued_in_block = 0;
         bool alive = true;
+        volatile int* blocks_done = &sm.blocks_done;
         auto acquire = [&](int& s) -> bool {
             if (*abort_flag) return false;
+            // Loads issued while the consumers synchronise delay that synchronisation (it queues behind them in
+            // the memory system), so only the first cross_stages stages of a block may be issued before the
+            // consumers are through the previous block's barrier.
+            if (issued_in_block >= P.cross_stages && *blocks_done < static_cast<int>(qp)) {
+                const long long t0 = clock64();
+                while (*blocks_done < static_cast<int>(qp)) {
+                    if (*abort_flag) return false;
+                    if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
+                }
+            }
+            ++issued_in_block;
             s = it % STAGES;
             if (it >= STAGES) {
                 const uint32_t use = static_cast<uint32_t>(it / STAGES);
@@ -136,67 +171,104 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
         };
         for (int step_i = 0; step_i < P.steps && alive; ++step_i) {
             for (int l = 0; l < L && alive; ++l) {
-                // (a) rows of the next block's predictor that this thread block owns
-                if (l + 1 < L) {
-                    const int r0 = static_cast<int>(static_cast<long long>(cta) * r / grid);
-                    const int r1 = static_cast<int>(static_cast<long long>(cta + 1) * r / grid);
-                    const __nv_bfloat16* W1 = P.W1[l + 1];
-                    for (int row = r0; row < r1 && alive; row += ROWS) {
-                        const int n = min(ROWS, r1 - row);
-                        int s;
-                        if (!acquire(s)) { alive = false; break; }
-                        sm.type[s] = ST_PRED; sm.arg0[s] = row; sm.arg1[s] = n;
-                        mbar_arrive_expect_tx(&sm.full[s], n * row_bytes);
-                        bulk_copy_g2s(ring + static_cast<size_t>(s) * stage_bytes, W1 + static_cast<size_t>(row) * d,
-                                      n * row_bytes, &sm.full[s]);
-                        ++it;
+                const PersistSel* sb = (l == 0) ? &P.sel[2] : &P.sel[l & 1];
+                if (lane == 0) {
+                    // (a) rows of the next block's predictor that this thread block owns
+                    if (l + 1 < L) {
+                        const int r0 = static_cast<int>(static_cast<long long>(cta) * r / grid);
+                        const int r1 = static_cast<int>(static_cast<long long>(cta + 1) * r / grid);
+                        const __nv_bfloat16* W1 = P.W1[l + 1];
+                        for (int row = r0; row < r1 && alive; row += ROWS) {
+                            const int n = min(ROWS, r1 - row);
+                            int s;
+                            if (!acquire(s)) { alive = false; break; }
+                            sm.type[s] = ST_PRED; sm.arg0[s] = row; sm.arg1[s] = n;
+                            mbar_arrive_expect_tx(&sm.full[s], n * row_bytes);
+                            bulk_copy_g2s(ring + static_cast<size_t>(s) * stage_bytes, W1 + static_cast<size_t>(row) * d,
+                                          n * row_bytes, &sm.full[s]);
+                            ++it;
+                        }
+                        if (alive && is_selector) alive = marker(ST_SELECT, l + 1);
                     }
-                    if (alive && is_selector) alive = marker(ST_SELECT, l + 1);
+                    // (b) the selection of this block must have been published
+                    if (alive && l > 0) {
+                        const unsigned need = static_cast<unsigned>(step_i) * (L - 1) + l;
+                        if (!spin_until_ge(sync_selready, need, sync_abort)) { *abort_flag = 1; alive = false; }
+                    }
                 }
+                alive = __shfl_sync(0xffffffffu, alive ? 1 : 0, 0) != 0;
                 if (!alive) break;
-                // (b) kept neurons of this block
-                const PersistSel* sb = &P.sel[2];
-                if (l > 0) {
-                    const unsigned need = static_cast<unsigned>(step_i) * (L - 1) + l;
-                    if (!spin_until_ge(sync_selready, need, sync_abort)) { *abort_flag = 1; alive = false; break; }
-                    sb = &P.sel[l & 1];
-                }
+                // (c) table of kept groups for this block: two dependent L2 reads, once per block instead of per batch
                 int nk = __ldcg(&sb->n_keep);
                 nk = max(0, min(nk, G));
-                const long long U = static_cast<long long>(nk) * per_group;
-                const long long U_eff = U + ((l + 1 < L) ? P.sel_cost : 0);
-                const long long lo = min(U, U_eff * cta / grid);
-                const long long hi = is_selector ? U : min(U, U_eff * (cta + 1) / grid);
-                const __nv_bfloat16* Wl = P.W[l];
-                for (long long b = lo; b < hi; ++b) {
-                    int s;
-                    if (!acquire(s)) { alive = false; break; }
-                    const int ki = static_cast<int>(b / per_group), j0 = static_cast<int>(b - static_cast<long long>(ki) * per_group) * NB;
+                for (int ki = lane; ki < nk; ki += 32) {
                     const int g = __ldcg(&sb->keep_list[ki]);
-                    int slot = -1;
-                    if (g >= 0 && g < G) {
-                        slot = __ldcg(&sb->dev_of_group[g]) + 1;
-                        if (slot < 0 || slot > n_dev) slot = -1;
+                    bool ok = (g >= 0 && g < G);
+                    if (ok) {
+                        const int slot = __ldcg(&sb->dev_of_group[g]) + 1;
+                        ok = (slot >= 0 && slot <= n_dev);
                     }
-                    sm.type[s] = ST_FFN; sm.arg0[s] = slot; sm.arg1[s] = 0;
-                    if (slot < 0) {
-                        flag_status(P.status, HALO_DEV_BAD_INDEX);
-                        mbar_arrive(&sm.full[s]);
-                    } else {
-                        const __nv_bfloat16* group = Wl + static_cast<size_t>(g) * 3 * S * d;
-                        unsigned char* dst = ring + static_cast<size_t>(s) * stage_bytes;
-                        mbar_arrive_expect_tx(&sm.full[s], stage_bytes);
-                        bulk_copy_g2s(dst, group + static_cast<size_t>(j0) * d, plane_bytes, &sm.full[s]);
-                        bulk_copy_g2s(dst + plane_bytes, group + static_cast<size_t>(S + j0) * d, plane_bytes, &sm.full[s]);
-                        bulk_copy_g2s(dst + 2 * plane_bytes, group + static_cast<size_t>(2 * S + j0) * d, plane_bytes,
-                                      &sm.full[s]);
-                    }
-                    ++it;
+                    if (!ok) flag_status(P.status, HALO_DEV_BAD_INDEX);
+                    sm.kept_group[ki] = ok ? g : -1;
                 }
-                if (alive) alive = marker(ST_END, 0);
+                __syncwarp();
+                const long long U = static_cast<long long>(nk) * per_group;
+                // (c') keep HBM busy while the consumers synchronise: the block's first batches go to L2 now, long
+                //      before ring slots free up for them (whoever ends up consuming them)
+                if (lane < P.l2_ahead) {
+                    const long long b = cta + static_cast<long long>(grid) * lane;
+                    if (b < U) {
+                        const int ki = static_cast<int>(b / per_group), j0 = static_cast<int>(b - static_cast<long long>(ki) * per_group) * NB;
+                        const int g = sm.kept_group[ki];
+                        if (g >= 0) {
+                            const __nv_bfloat16* group = P.W[l] + static_cast<size_t>(g) * 3 * S * d;
+                            bulk_prefetch_l2(group + static_cast<size_t>(j0) * d, plane_bytes);
+                            bulk_prefetch_l2(group + static_cast<size_t>(S + j0) * d, plane_bytes);
+                            bulk_prefetch_l2(group + static_cast<size_t>(2 * S + j0) * d, plane_bytes);
+                        }
+                    }
+                }
+                if (lane == 0) {
+                    // (d) batches of kept neurons, handed out by the block's counter
+                    unsigned* const ctr = P.sync + 16 + (qp & 15u);
+                    const __nv_bfloat16* Wl = P.W[l];
+                    // The first batch is fixed, the rest come from the counter.  kFetchAhead fetches are kept in
+                    // flight so that the round trip of the atomic is off the issue path.
+                    long long b = cta;
+                    long long ahead[kFetchAhead];
+#pragma unroll
+                    for (int k = 0; k < kFetchAhead; ++k) ahead[k] = static_cast<long long>(grid) + atomicAdd(ctr, 1u);
+                    while (b < U) {
+                        int s;
+                        if (!acquire(s)) { alive = false; break; }
+                        const int ki = static_cast<int>(b / per_group), j0 = static_cast<int>(b - static_cast<long long>(ki) * per_group) * NB;
+                        const int g = sm.kept_group[ki];
+                        sm.type[s] = ST_FFN; sm.arg0[s] = g >= 0 ? 0 : -1; sm.arg1[s] = 0;
+                        if (g < 0) {
+                            mbar_arrive(&sm.full[s]);
+                        } else {
+                            const __nv_bfloat16* group = Wl + static_cast<size_t>(g) * 3 * S * d;
+                            unsigned char* dst = ring + static_cast<size_t>(s) * stage_bytes;
+                            mbar_arrive_expect_tx(&sm.full[s], stage_bytes);
+                            bulk_copy_g2s(dst, group + static_cast<size_t>(j0) * d, plane_bytes, &sm.full[s]);
+                            bulk_copy_g2s(dst + plane_bytes, group + static_cast<size_t>(S + j0) * d, plane_bytes, &sm.full[s]);
+                            bulk_copy_g2s(dst + 2 * plane_bytes, group + static_cast<size_t>(2 * S + j0) * d, plane_bytes,
+                                          &sm.full[s]);
+                        }
+                        ++it;
+                        b = ahead[0];
+#pragma unroll
+                        for (int k = 0; k + 1 < kFetchAhead; ++k) ahead[k] = ahead[k + 1];
+                        ahead[kFetchAhead - 1] = (b < U) ? static_cast<long long>(grid) + atomicAdd(ctr, 1u) : U;
+                    }
+                    if (alive) alive = marker(ST_END, 0);
+                }
+                ++qp;
+                issued_in_block = 0;
+                __syncwarp();  // the table is rewritten for the next block only after lane 0 is done with it
             }
         }
-        if (*abort_flag) {
+        if (lane == 0 && *abort_flag) {
             // nobody consumes any more: let every copy this thread block issued land before it exits
             const int first = it > STAGES ? it - STAGES : 0;
             int never = 0;
@@ -212,14 +284,18 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
     const int rep = (REP > 1) ? tid / (kPC / REP) : 0;
     const int col0 = (REP > 1) ? tid % (kPC / REP) : tid;
     const bool owner = (REP == 1) || (rep == 0);   // threads that carry the residual stream for their columns
-    float xr[XC][8];
+    uint4 xq[XC];      // this lane's slice of x, packed bf16
     float acc[P2][8];
     float hreg[P2][8];
     int it = 0, red_par = 0;
     unsigned q = 0;  // running block counter over steps: partial buffers rotate with it
-    const size_t slot_stride = static_cast<size_t>(d);
-    const size_t buf_stride = static_cast<size_t>(n_dev + 1) * d;
+    const size_t acc_stride = static_cast<size_t>(d);
+    const size_t buf_stride = static_cast<size_t>(kAccBufs) * d;
     bool bad = false;
+    auto trace = [&](int slot, unsigned long long value) {
+        if (P.trace && tid == 0 && q < static_cast<unsigned>(P.trace_blocks))
+            P.trace[(static_cast<size_t>(q) * grid + cta) * 8 + slot] = value;
+    };
 
     // normalise hreg -> xs (bf16) -> xr; thread block 0 records x as the input of block `l_next`
     auto normalise_and_load_x = [&](int step_i, int l_next, bool want_x) {
@@ -259,23 +335,22 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
         pc_barrier();  // xs complete; sm.reduce free again
         if (want_x) {
 #pragma unroll
-            for (int i = 0; i < XC; ++i)
-                Elem<__nv_bfloat16>::widen(reinterpret_cast<const uint4*>(xs)[p1_base + 32 * i], xr[i]);
+            for (int i = 0; i < XC; ++i) xq[i] = reinterpret_cast<const uint4*>(xs)[p1_base + 32 * i];
         }
     };
 
-    auto flush = [&](int slot) {
-        float* dst = P.partials + (q % 3u) * buf_stride + static_cast<size_t>(slot) * slot_stride;
+    // column sums -> shared memory (one region per replica), made visible to the copy engine
+    auto stage_sums = [&]() {
+        float* dst = reinterpret_cast<float*>(vec_buf) + static_cast<size_t>(rep) * d;
 #pragma unroll
         for (int p = 0; p < P2; ++p) {
             const int c = col0 + kPC * p;
             if (c < chunks) {
-                red_add_v4f(dst + c * 8, acc[p][0], acc[p][1], acc[p][2], acc[p][3]);
-                red_add_v4f(dst + c * 8 + 4, acc[p][4], acc[p][5], acc[p][6], acc[p][7]);
+                reinterpret_cast<float4*>(dst + c * 8)[0] = make_float4(acc[p][0], acc[p][1], acc[p][2], acc[p][3]);
+                reinterpret_cast<float4*>(dst + c * 8)[1] = make_float4(acc[p][4], acc[p][5], acc[p][6], acc[p][7]);
             }
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[p][e] = 0.0f;
         }
+        fence_proxy_async_smem();
     };
 
     for (int step_i = 0; step_i < P.steps && !bad; ++step_i) {
@@ -299,13 +374,16 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
             for (int p = 0; p < P2; ++p)
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc[p][e] = 0.0f;
-            int cur_slot = -1;
+            bool any = false;
+            bool first_stage = true;
+            trace(TR_BLOCK_START, global_timer_ns());
 
             // ------------------------------ stages of this block ------------------------------
             while (true) {
                 const int s = it % STAGES;
                 const uint32_t parity = static_cast<uint32_t>(it / STAGES) & 1u;
                 const bool ok = mbar_wait_bounded(&sm.full[s], parity, abort_flag);
+                if (first_stage) { trace(TR_FIRST_STAGE, global_timer_ns()); first_stage = false; }
                 const int type = sm.type[s], a0 = sm.arg0[s], a1 = sm.arg1[s];
                 const unsigned char* stage = ring + static_cast<size_t>(s) * stage_bytes;
                 float* red = sm.red[red_par];
@@ -313,34 +391,21 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 // ---- before the barrier: nothing in here may block on other consumers ----
                 if (type == ST_FFN) {
                     if (a0 >= 0) {
-                        if (a0 != cur_slot) {
-                            if (cur_slot >= 0) flush(cur_slot);
-                            cur_slot = a0;
-                        }
+                        any = true;
                         const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(row) * row_bytes);
-                        float dot = 0.0f;
+                        float dot0 = 0.0f, dot1 = 0.0f;
 #pragma unroll
-                        for (int i = 0; i < XC; ++i) {
-                            float w8[8];
-                            Elem<__nv_bfloat16>::widen(rp[p1_base + 32 * i], w8);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) dot = fmaf(w8[e], xr[i][e], dot);
-                        }
-                        dot = warp_sum(dot);
+                        for (int i = 0; i < XC; ++i) dot_bf16x8(rp[p1_base + 32 * i], xq[i], dot0, dot1);
+                        const float dot = warp_sum(dot0 + dot1);
                         if (lane == 0) red[row * WPR + part] = dot;
                     }
                 } else if (type == ST_PRED) {
                     if (row < a1) {
                         const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(row) * row_bytes);
-                        float dot = 0.0f;
+                        float dot0 = 0.0f, dot1 = 0.0f;
 #pragma unroll
-                        for (int i = 0; i < XC; ++i) {
-                            float w8[8];
-                            Elem<__nv_bfloat16>::widen(rp[p1_base + 32 * i], w8);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) dot = fmaf(w8[e], xr[i][e], dot);
-                        }
-                        dot = warp_sum(dot);
+                        for (int i = 0; i < XC; ++i) dot_bf16x8(rp[p1_base + 32 * i], xq[i], dot0, dot1);
+                        const float dot = warp_sum(dot0 + dot1);
                         if (lane == 0) red[row * WPR + part] = dot;
                     }
                 } else if (type == ST_SELECT) {
@@ -358,20 +423,12 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
 #pragma unroll
                         for (int jj = 0; jj < NB / REP; ++jj) {
                             const int j = jj * REP + rep;
-                            float a = 0.0f, b = 0.0f;
-#pragma unroll
-                            for (int w = 0; w < WPR; ++w) { a += red[j * WPR + w]; b += red[(NB + j) * WPR + w]; }
-                            const float h = a / (1.0f + __expf(-a)) * b;
+                            const float h = silu_mul(sum_parts<WPR>(red + j * WPR), sum_parts<WPR>(red + (NB + j) * WPR));
                             const uint4* dr = reinterpret_cast<const uint4*>(down + static_cast<size_t>(j) * row_bytes);
 #pragma unroll
                             for (int p = 0; p < P2; ++p) {
                                 const int c = col0 + kPC * p;
-                                if (P2 == 1 || c < chunks) {
-                                    float w8[8];
-                                    Elem<__nv_bfloat16>::widen(dr[c], w8);
-#pragma unroll
-                                    for (int e = 0; e < 8; ++e) acc[p][e] = fmaf(h, w8[e], acc[p][e]);
-                                }
+                                if (P2 == 1 || c < chunks) axpy_bf16x8(h, dr[c], acc[p]);
                             }
                         }
                     }
@@ -390,24 +447,40 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                     red_par ^= 1;
                 } else if (type == ST_SELECT) {
                     // a1 (second layer): s[g] = <W2[g], z>; then a2..a5 for block a0, published for the producers
+                    const unsigned long long t_sel = (P.trace && tid == 0) ? global_timer_ns() : 0ull;
                     const int lp = a0;
                     const __nv_bfloat16* W2 = P.W2[lp];
-                    const int zc = r >> 3;
-                    for (int g = warp; g < G; g += kPCWarps) {
-                        const uint4* wrow = reinterpret_cast<const uint4*>(W2 + static_cast<size_t>(g) * r);
-                        float dot = 0.0f;
-                        for (int c = lane; c < zc; c += 32) {
-                            float w8[8];
-                            Elem<__nv_bfloat16>::widen(__ldg(wrow + c), w8);
+                    const int zc = r >> 3;  // 16-byte chunks per W2 row
+                    for (int c0 = 0; c0 < zc; c0 += 32) {
+                        const int c = c0 + lane;
+                        float zv[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                        if (c < zc) {
                             const float4 z0 = __ldcg(reinterpret_cast<const float4*>(P.z) + 2 * c);
                             const float4 z1 = __ldcg(reinterpret_cast<const float4*>(P.z) + 2 * c + 1);
-                            dot = fmaf(w8[0], z0.x, dot); dot = fmaf(w8[1], z0.y, dot);
-                            dot = fmaf(w8[2], z0.z, dot); dot = fmaf(w8[3], z0.w, dot);
-                            dot = fmaf(w8[4], z1.x, dot); dot = fmaf(w8[5], z1.y, dot);
-                            dot = fmaf(w8[6], z1.z, dot); dot = fmaf(w8[7], z1.w, dot);
+                            zv[0] = z0.x; zv[1] = z0.y; zv[2] = z0.z; zv[3] = z0.w;
+                            zv[4] = z1.x; zv[5] = z1.y; zv[6] = z1.z; zv[7] = z1.w;
                         }
-                        dot = warp_sum(dot);
-                        if (lane == 0) sm.score[g] = dot;
+                        // groups warp, warp+16, ...: all row loads of a pass are issued before any is used
+                        for (int g0 = warp; g0 < G; g0 += kPCWarps * 4) {
+                            uint4 wv[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const int g = g0 + u * kPCWarps;
+                                wv[u] = (g < G && c < zc) ? __ldg(reinterpret_cast<const uint4*>(W2 + static_cast<size_t>(g) * r) + c)
+                                                          : make_uint4(0, 0, 0, 0);
+                            }
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const int g = g0 + u * kPCWarps;
+                                float w8[8];
+                                Elem<__nv_bfloat16>::widen(wv[u], w8);
+                                float dot = 0.0f;
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) dot = fmaf(w8[e], zv[e], dot);
+                                dot = warp_sum(dot);
+                                if (lane == 0 && g < G) sm.score[g] = (c0 == 0 ? 0.0f : sm.score[g]) + dot;
+                            }
+                        }
                     }
                     pc_barrier();
                     PersistSel* sb = &P.sel[lp & 1];
@@ -426,6 +499,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                     if (tid == 0) {
                         if (P.tap_n_keep) P.tap_n_keep[rec] = __ldcg(&sb->n_keep);
                         st_release_gpu(sync_selready, static_cast<unsigned>(step_i) * (L - 1) + lp);
+                        if (P.trace) trace(TR_SELECT_NS, global_timer_ns() - t_sel);
                     }
                 }
                 __syncwarp();
@@ -436,19 +510,36 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
             if (bad) break;
 
             // ------------------------------ end of the block: flush, grid barrier, merge + glue ------------------------------
-            if (cur_slot >= 0) flush(cur_slot);
-            __threadfence();
+            trace(TR_STAGES_DONE, global_timer_ns());
+            if (any) stage_sums();
             pc_barrier();
             bool okb = true;
             if (tid == 0) {
+                if (any) {
+                    float* dst = P.partials + (q % 3u) * buf_stride + static_cast<size_t>(cta % kAccBufs) * acc_stride;
+#pragma unroll
+                    for (int k = 0; k < REP; ++k)
+                        bulk_reduce_add_f32_s2g(dst, vec_buf + static_cast<size_t>(k) * d * 4, static_cast<uint32_t>(d) * 4u);
+                    bulk_commit_and_wait_all();   // the sums are in global memory (and vec_buf is free again)
+                    fence_proxy_async_all();
+                }
+                trace(TR_FLUSHED, global_timer_ns());
+                // Batch counters rotate over 16 words.  A producer leads its consumers by at most the ring depth
+                // (<= 8 stages, every block has at least its END stage), so the counter of the block 8 ahead is
+                // idle now: its last user finished 8 blocks ago and its next user cannot have started.
+                if (cta == 0) P.sync[16 + ((q + 8u) & 15u)] = 0u;
                 __threadfence();
-                atomicAdd(sync_barrier, 1u);
-                okb = spin_until_ge(sync_barrier, (q + 1u) * static_cast<unsigned>(grid), sync_abort);
+                const unsigned target = (q + 1u) * static_cast<unsigned>(grid);
+                const unsigned before = atomicAdd(sync_barrier, 1u);
+                okb = (before + 1u == target) || spin_until_ge(sync_barrier, target, sync_abort);
+                __threadfence();
             }
             bad = pc_barrier_or(!okb);
             if (bad) break;
+            if (tid == 0) *reinterpret_cast<volatile int*>(&sm.blocks_done) = static_cast<int>(q) + 1;
+            trace(TR_BARRIER_DONE, global_timer_ns());
 
-            // a9 + residual: every thread block merges all slots for its own copy of the stream
+            // a9 + residual: every thread block sums the accumulation buffers for its own copy of the stream
             const float* pbuf = P.partials + (q % 3u) * buf_stride;
             float* zbuf = P.partials + ((q + 2u) % 3u) * buf_stride;   // read two blocks ago by everyone: clear it
             const size_t rec = static_cast<size_t>(step_i) * L + l;
@@ -457,12 +548,18 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 for (int p = 0; p < P2; ++p) {
                     const int c = col0 + kPC * p;
                     if (c < chunks) {
+                        float4 va[kAccBufs], vb[kAccBufs];
+#pragma unroll
+                        for (int k = 0; k < kAccBufs; ++k) {
+                            const float4* src = reinterpret_cast<const float4*>(pbuf + static_cast<size_t>(k) * acc_stride + c * 8);
+                            va[k] = __ldcg(src);
+                            vb[k] = __ldcg(src + 1);
+                        }
                         float y[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-                        for (int slot = 0; slot <= n_dev; ++slot) {
-                            const float4* src = reinterpret_cast<const float4*>(pbuf + static_cast<size_t>(slot) * slot_stride + c * 8);
-                            const float4 a = __ldcg(src), b = __ldcg(src + 1);
-                            y[0] += a.x; y[1] += a.y; y[2] += a.z; y[3] += a.w;
-                            y[4] += b.x; y[5] += b.y; y[6] += b.z; y[7] += b.w;
+#pragma unroll
+                        for (int k = 0; k < kAccBufs; ++k) {
+                            y[0] += va[k].x; y[1] += va[k].y; y[2] += va[k].z; y[3] += va[k].w;
+                            y[4] += vb[k].x; y[5] += vb[k].y; y[6] += vb[k].z; y[7] += vb[k].w;
                         }
 #pragma unroll
                         for (int e = 0; e < 8; ++e) hreg[p][e] += y[e];
@@ -477,17 +574,19 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                                 dst[0] = make_float4(hreg[p][0], hreg[p][1], hreg[p][2], hreg[p][3]);
                                 dst[1] = make_float4(hreg[p][4], hreg[p][5], hreg[p][6], hreg[p][7]);
                             }
-                            for (int slot = 0; slot <= n_dev; ++slot) {
-                                float4* dst = reinterpret_cast<float4*>(zbuf + static_cast<size_t>(slot) * slot_stride + c * 8);
-                                dst[0] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                dst[1] = make_float4(0.f, 0.f, 0.f, 0.f);
-                            }
+                        }
+                        if (cta < kAccBufs) {
+                            float4* dst = reinterpret_cast<float4*>(zbuf + static_cast<size_t>(cta) * acc_stride + c * 8);
+                            dst[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            dst[1] = make_float4(0.f, 0.f, 0.f, 0.f);
                         }
                     }
                 }
             }
-            ++q;
+            trace(TR_MERGED, global_timer_ns());
             if (l + 1 < L) normalise_and_load_x(step_i, l + 1, true);
+            trace(TR_X_READY, global_timer_ns());
+            ++q;
         }
     }
     if (bad && tid == 0) {
@@ -502,7 +601,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
 bool persistent_supported(const halo_ffn_shape& sh, int n_tok, int G) {
     if (sh.wdtype != HALO_BF16 || n_tok != 1 || G > kPC) return false;
     switch (sh.d_model) {
-        case 2048: return sh.group_size % 4 == 0;
+        case 2048: return sh.group_size % 4 == 0;  // batches of NB neurons must tile a group
         case 4096: case 5120: return sh.group_size % 2 == 0;
         case 8192: return true;
     }
@@ -512,7 +611,7 @@ bool persistent_supported(const halo_ffn_shape& sh, int n_tok, int G) {
 template <int NB, int XC, int P2, int REP, int STAGES>
 static halo_status launch_cfg(PersistParams& P, cudaStream_t st) {
     auto kernel = stack_decode_kernel<NB, XC, P2, REP, STAGES>;
-    const size_t smem = kHeaderBytes + kXsBytes + static_cast<size_t>(STAGES) * 3 * NB * P.d * 2;
+    const size_t smem = kHeaderBytes + static_cast<size_t>(P.d) * 4 * REP + static_cast<size_t>(STAGES) * 3 * NB * P.d * 2;
     static int blocks_per_sm = -1;
     int dev = 0, sms = kSmCount;
     if (cudaGetDevice(&dev) != cudaSuccess) return HALO_ERR_CUDA;
@@ -535,7 +634,7 @@ halo_status launch_stack_persistent(PersistParams& P, cudaStream_t st) {
         case 2048: return launch_cfg<4, 4, 1, 2, 4>(P, st);
         case 4096: return launch_cfg<2, 4, 1, 1, 4>(P, st);
         case 5120: return launch_cfg<2, 5, 2, 1, 3>(P, st);
-        case 8192: return launch_cfg<1, 4, 2, 1, 4>(P, st);
+        case 8192: return launch_cfg<1, 4, 2, 1, 3>(P, st);
     }
     return HALO_ERR_UNIMPLEMENTED;
 }

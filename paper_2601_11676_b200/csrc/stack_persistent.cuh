@@ -16,16 +16,16 @@ struct PersistSel {
 struct PersistParams {
     int L, steps, d, S, G, r, act;
     uint32_t step0;
-    int sel_cost;                          // batches the selecting thread block is spared per block
     const __nv_bfloat16* const* W;         // device tables [L]
     const __nv_bfloat16* const* W1;
     const __nv_bfloat16* const* W2;
     const float* h0;                       // [steps][d]
     float* h_out;                          // [steps][d]
-    float* partials;                       // [3][n_dev+1][d], zero at launch
+    float* partials;                       // [3][2][d] rotating interleaved accumulation buffers, zero at launch
     float* z;                              // [r]
     PersistSel* sel;                       // [3]: two rotating + the static first-block selection
-    unsigned* sync;                        // [4]: barrier count, abort, hidden rows done, selections published
+    unsigned* sync;                        // [32]: 0 barrier count, 1 abort, 2 hidden rows done, 3 selections
+                                           //       published, 16..31 rotating batch counters; zero at launch
     uint32_t* status;
     // optional records (thread block 0 / the selecting thread block write them)
     __nv_bfloat16* tap_x;
@@ -35,6 +35,13 @@ struct PersistParams {
     int32_t* tap_keep_list;
     int32_t* tap_n_keep;
     float* tap_y;
+    // optional trace: [trace_blocks][gridDim.x][8] timestamps (ns, global timer) written by thread 0 of every
+    // thread block for the first trace_blocks blocks of the run
+    int cross_stages;                      // stages of the next block a producer may issue before its consumers
+                                           // have passed the grid barrier of the current block
+    int l2_ahead;                          // batches per thread block prefetched into L2 on entering a block
+    unsigned long long* trace;
+    int trace_blocks;
     PlanDev plan;
 };
 

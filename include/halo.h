@@ -133,6 +133,31 @@ halo_status halo_predict_groups(const halo_pred_shape* shape, const void* W1, co
                                 void* workspace, size_t workspace_bytes, uint32_t* dev_status, void* stream);
 
 /* ------------------------------------------------------------------------
+ * The predictor for callers that cannot provide a workspace.  (The paper has no counterpart of this entry
+ * point; it exists for the way this library gets embedded.)
+ *
+ * halo_predict_groups needs a device workspace, and a workspace has to be allocated by somebody.  Some callers
+ * cannot do that at the point of the call: a server that handed all device memory to its own pool at start-up,
+ * a plug-in living inside another program's memory budget, a latency-critical loop where entering the CUDA
+ * allocator (which may synchronise the device) is not acceptable.  This variant computes exactly what
+ * halo_predict_groups computes, with the same arguments minus the workspace, and keeps its two intermediate
+ * arrays in a fixed array compiled into the library (HALO_STATIC_SCRATCH_FLOATS floats = 2 MiB, held by every
+ * GPU that loads the library, from load until the process exits).  It calls no allocation routine of any kind.
+ *   Limit: n_tok * (rank + n_groups) <= HALO_STATIC_SCRATCH_FLOATS, else HALO_ERR_WORKSPACE and nothing runs.
+ *   Set-up: the first call on each device looks up the device address of the array (with that device
+ *     current); make that first call outside any stream capture.  Later calls only launch.
+ *   Sharing: all calls on a device use the same array, and it keeps what the last call left in it.  Nothing in
+ *     it needs to be zero at entry.  Two calls that overlap on the GPU (different streams, or host threads
+ *     without ordering between their streams) race on it and give wrong scores: keep calls on one stream, or
+ *     order them with events.
+ * Other errors and the device status word are as for halo_predict_groups.
+ * ---------------------------------------------------------------------- */
+#define HALO_STATIC_SCRATCH_FLOATS (512 * 1024)
+halo_status halo_predict_groups_static(const halo_pred_shape* shape, const void* W1, const void* W2,
+                                       const void* feat, int n_tok, int mean_pool, float* scores,
+                                       uint32_t* dev_status, void* stream);
+
+/* ------------------------------------------------------------------------
  * a2..a5. Rank, critical choice, runtime assignment and arrival mask
  * (Sec. III-B.3, Pred process: the importance rank indexes the priority
  * lists fixed by the Assignment phase; relaxed synchronisation: the master

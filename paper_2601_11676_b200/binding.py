@@ -24,7 +24,7 @@ MAX_DEVICES, MAX_GROUPS = 32, 1024
 
 EXPORTS = [
     "halo_status_string", "halo_status_message", "halo_plan_create", "halo_plan_destroy", "halo_plan_describe",
-    "halo_predict_workspace_bytes", "halo_predict_groups", "halo_select_groups", "halo_group_ffn_workspace_bytes",
+    "halo_predict_workspace_bytes", "halo_predict_groups", "halo_predict_groups_static", "halo_select_groups", "halo_group_ffn_workspace_bytes",
     "halo_group_ffn", "halo_merge_partials", "halo_pack_weights", "halo_glue", "halo_stack_create",
     "halo_stack_destroy", "halo_stack_decode", "halo_stack_decode_host", "halo_stack_status",
     "halo_stack_last_launches", "halo_stack_set_mode", "halo_stack_set_trace", "halo_stack_trace_width",
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.halo_plan_describe.argtypes = [c_void_p, c_int, POINTER(c_int32), POINTER(c_uint64), POINTER(c_int32)]
         L.halo_predict_groups.argtypes = [POINTER(PredShape), c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p,
                                           c_void_p, c_size_t, c_void_p, c_void_p]
+        L.halo_predict_groups_static.argtypes = [POINTER(PredShape), c_void_p, c_void_p, c_void_p, c_int, c_int,
+                                                 c_void_p, c_void_p, c_void_p]
         L.halo_select_groups.argtypes = [c_void_p, c_void_p, c_uint32, c_uint32, c_int, c_void_p, c_void_p, c_void_p,
                                          c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         L.halo_group_ffn.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int,
@@ -181,6 +183,18 @@ def halo_predict_groups(shape: PredShape, W1, W2, feat, n_tok, mean_pool, scores
                                    _ptr(scores), _ptr(workspace),
                                    workspace.numel() * workspace.element_size() if workspace is not None else 0,
                                    _ptr(dev_status), _stream(stream)), "halo_predict_groups")
+
+
+STATIC_SCRATCH_FLOATS = 512 * 1024
+
+
+def halo_predict_groups_static(shape: PredShape, W1, W2, feat, n_tok, mean_pool, scores, dev_status=None,
+                               stream=None) -> None:
+    """halo_predict_groups without a workspace: the intermediates live in a fixed array inside the library, for
+    callers that cannot allocate device memory.  Calls on one device share that array: keep them on one stream."""
+    _chk(lib().halo_predict_groups_static(byref(shape), _ptr(W1), _ptr(W2), _ptr(feat), n_tok, int(bool(mean_pool)),
+                                          _ptr(scores), _ptr(dev_status), _stream(stream)),
+         "halo_predict_groups_static")
 
 
 def halo_select_groups(plan: Plan, scores, step, layer, force_all, order, dev_of_group, arrived, keep, keep_list,

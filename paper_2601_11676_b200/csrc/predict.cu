@@ -1,4 +1,6 @@
 // halo_predict_groups (step a1): z = act(W1 f), s = W2 z, optional mean over tokens.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace halo {
@@ -121,3 +123,59 @@ halo_status launch_predict(const halo_pred_shape& sh, const void* W1, const void
 }
 
 }  // namespace halo
+
+// ---- predictor without any caller-provided or allocated scratch --------------------------------------------
+//
+// Some programs that want to call the predictor cannot hand it a workspace because they cannot allocate one
+// at that point: a serving process that gave all device memory to its own pool when it started, a plug-in
+// running inside someone else's memory budget, or a latency-critical loop in which a call into the CUDA
+// allocator (which may synchronise the whole device) is not acceptable.  For them the two intermediate
+// arrays of the predictor live in the fixed array below, which is part of the library image: every GPU on
+// which the library is loaded holds these 2 MiB from load to exit.
+//
+// The name `g_predict_scratch` is only meaningful to device code.  On the host it is a stand-in symbol, not
+// a device address, so the entry point asks the runtime for the real address once per device
+// (cudaGetSymbolAddress, with that device current) and passes it to the kernels like any other pointer.
+static __device__ __align__(256) float g_predict_scratch[HALO_STATIC_SCRATCH_FLOATS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_scratch_addr[kMaxDevices] = {};  // device address of g_predict_scratch, per device ordinal
+std::mutex g_scratch_mutex;
+}  // namespace
+
+extern "C" halo_status halo_predict_groups_static(const halo_pred_shape* shape, const void* W1, const void* W2,
+                                                  const void* feat, int n_tok, int mean_pool, float* scores,
+                                                  uint32_t* dev_status, void* stream) {
+    // same argument rules as halo_predict_groups
+    if (!shape) return HALO_ERR_ARG;
+    if (shape->wdtype != HALO_F32 && shape->wdtype != HALO_BF16) return HALO_ERR_DTYPE;
+    if (shape->act != HALO_ACT_RELU && shape->act != HALO_ACT_NONE) return HALO_ERR_ARG;
+    if (shape->d_in <= 0 || shape->rank <= 0 || shape->n_groups <= 0 || n_tok <= 0) return HALO_ERR_SHAPE;
+    if (shape->d_in % 8 != 0 || shape->rank % 8 != 0) return HALO_ERR_SHAPE;
+    if (shape->d_in > 12288 || shape->rank > 8192 || shape->n_groups > HALO_MAX_GROUPS) return HALO_ERR_SHAPE;
+    if (!W1 || !W2 || !feat || !scores) return HALO_ERR_ARG;
+    if (!halo::aligned16(W1) || !halo::aligned16(W2) || !halo::aligned16(feat)) return HALO_ERR_ALIGN;
+    // the fixed array bounds what fits: hidden values [n_tok][rank] + per-token scores [n_tok][n_groups]
+    const unsigned long long need =
+        static_cast<unsigned long long>(n_tok) * (static_cast<unsigned long long>(shape->rank) + shape->n_groups);
+    if (need > HALO_STATIC_SCRATCH_FLOATS) return HALO_ERR_WORKSPACE;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return HALO_ERR_CUDA;
+    float* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_scratch_mutex);
+        if (!g_scratch_addr[dev]) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_predict_scratch) != cudaSuccess || !p) return HALO_ERR_CUDA;
+            g_scratch_addr[dev] = static_cast<float*>(p);
+        }
+        scratch = g_scratch_addr[dev];
+    }
+    // Nothing in the array has to start at zero: every word a call reads it has written first, so whatever
+    // the previous call left behind is harmless.
+    return halo::launch_predict(*shape, W1, W2, feat, n_tok, mean_pool, scores, scratch, dev_status,
+                                static_cast<cudaStream_t>(stream));
+}
+

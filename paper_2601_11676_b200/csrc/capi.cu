@@ -186,9 +186,25 @@ extern "C" halo_status halo_select_groups(const halo_plan* plan, const float* sc
 // ---- a6..a8 -----------------------------------------------------------------------------------------
 
 extern "C" size_t halo_group_ffn_workspace_bytes(const halo_ffn_shape* shape, int n_tok, int n_dev) {
-    (void)shape; (void)n_tok; (void)n_dev;
-    return 0;
+    (void)n_dev;
+    if (check_ffn_shape(shape) != HALO_OK || n_tok <= 0) return 0;
+    return prefill_supported(*shape, n_tok) ? prefill_workspace_bytes(*shape, n_tok) : 0;
 }
+
+namespace {
+// many tokens + bf16 + supported shape -> tensor-core contraction; otherwise the bandwidth-bound kernels
+halo_status dispatch_group_ffn(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
+                               const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group, int n_dev,
+                               float* partials, void* workspace, uint32_t* dev_status, cudaStream_t st) {
+    if (prefill_supported(sh, n_tok) && workspace) {
+        const size_t bytes = sizeof(float) * static_cast<size_t>(n_dev + 1) * n_tok * sh.d_model;
+        if (cudaMemsetAsync(partials, 0, bytes, st) != cudaSuccess) return HALO_ERR_CUDA;
+        return launch_group_ffn_prefill(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, workspace,
+                                        dev_status, st);
+    }
+    return launch_group_ffn_decode(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, st);
+}
+}  // namespace
 
 extern "C" halo_status halo_group_ffn(const halo_ffn_shape* shape, const void* W_packed, const void* x, int n_tok,
                                       const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
@@ -200,10 +216,11 @@ extern "C" halo_status halo_group_ffn(const halo_ffn_shape* shape, const void* W
     if (n_tok <= 0) return HALO_ERR_SHAPE;
     if (n_dev < 0 || n_dev > HALO_MAX_DEVICES || (!dev_of_group && n_dev != 0)) return HALO_ERR_ARG;
     if (!aligned16(W_packed) || !aligned16(x) || !aligned16(partials)) return HALO_ERR_ALIGN;
-    if (workspace_bytes < halo_group_ffn_workspace_bytes(shape, n_tok, n_dev)) return HALO_ERR_WORKSPACE;
-    (void)workspace;
-    return launch_group_ffn_decode(*shape, W_packed, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials,
-                                   dev_status, static_cast<cudaStream_t>(stream));
+    const size_t need = halo_group_ffn_workspace_bytes(shape, n_tok, n_dev);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return HALO_ERR_WORKSPACE;
+    if (need > 0 && !aligned16(workspace)) return HALO_ERR_ALIGN;
+    return dispatch_group_ffn(*shape, W_packed, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials,
+                              need > 0 ? workspace : nullptr, dev_status, static_cast<cudaStream_t>(stream));
 }
 
 // ---- a9 and helpers -----------------------------------------------------------------------------------
@@ -266,6 +283,7 @@ struct halo_stack {
     float* p_z;
     halo::PersistSel* p_sel;       // [3]
     unsigned* p_sync;              // [32]
+    void* ffn_ws;                  // H buffer of the tensor-core path (multi-token stacks), or null
     unsigned long long* trace;     // caller-owned, optional
     int trace_blocks;
     int cross_stages, l2_ahead;    // tuning of the persistent kernel
@@ -325,6 +343,8 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     const size_t o_pz = carve(sizeof(float) * pred->rank);
     const size_t o_ps = carve(sizeof(PersistSel) * 3);
     const size_t o_py = carve(sizeof(unsigned) * 32);
+    const size_t ws_bytes = prefill_supported(*ffn, n_tok) ? prefill_workspace_bytes(*ffn, n_tok) : 0;
+    const size_t o_ws = carve(ws_bytes ? ws_bytes : 16);
     if (cudaMalloc(&s->slab, off) != cudaSuccess) { delete s; return HALO_ERR_NOMEM; }
     if (cudaMemset(s->slab, 0, off) != cudaSuccess) { cudaFree(s->slab); delete s; return HALO_ERR_CUDA; }
     char* base = static_cast<char*>(s->slab);
@@ -349,6 +369,7 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     s->p_z = reinterpret_cast<float*>(base + o_pz);
     s->p_sel = reinterpret_cast<PersistSel*>(base + o_ps);
     s->p_sync = reinterpret_cast<unsigned*>(base + o_py);
+    s->ffn_ws = ws_bytes ? static_cast<void*>(base + o_ws) : nullptr;
     s->mode = 0;
     s->trace = nullptr;
     s->trace_blocks = 0;
@@ -486,8 +507,8 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                 if (taps->n_keep) HALO_COPY(taps->n_keep + rec, s->n_keep, sizeof(int32_t));
                 if (taps->y) y_tap = taps->y + rec * step_elems;
             }
-            HALO_TRY(launch_group_ffn_decode(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->keep_list, s->n_keep,
-                                             s->dev_of_group, n_dev, s->partials, s->status, st));
+            HALO_TRY(dispatch_group_ffn(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->keep_list, s->n_keep,
+                                        s->dev_of_group, n_dev, s->partials, s->ffn_ws, s->status, st));
             ++launches;
             float* h_dst = (l == L - 1) ? h_out + sidx * step_elems : s->h;
             HALO_TRY(launch_merge_glue(s->partials, s->arrived, n_dev, static_cast<int>(T), static_cast<int>(d),

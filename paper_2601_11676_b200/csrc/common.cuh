@@ -100,6 +100,13 @@ halo_status launch_group_ffn_decode(const halo_ffn_shape& sh, const void* W, con
 halo_status launch_group_ffn_stream(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                     const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
                                     int n_dev, float* partials, uint32_t* dev_status, cudaStream_t st);
+// Prefill form (tensor cores); workspace = bf16 [n_tok][d_ffn]; partials must already be zero.
+bool prefill_supported(const halo_ffn_shape& sh, int n_tok);
+size_t prefill_workspace_bytes(const halo_ffn_shape& sh, int n_tok);
+halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
+                                     const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
+                                     int n_dev, float* partials, void* workspace, uint32_t* dev_status,
+                                     cudaStream_t st);
 halo_status launch_merge(const float* partials, const uint8_t* arrived, int n_dev, int n_tok, int d, float* y,
                          cudaStream_t st);
 halo_status launch_glue(int d, int n_tok, halo_dtype xdtype, const float* h, const float* y, float* h_out,

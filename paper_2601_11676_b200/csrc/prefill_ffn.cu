@@ -1,0 +1,407 @@
+// halo_group_ffn, prefill form (many tokens, bf16): the masked FFN as dense contractions on the tensor cores.
+//
+//   GEMM-1  for every kept group g (one CTA tile per 128 tokens x one group):
+//             Dg = X * Wgate_g^T,  Du = X * Wup_g^T      two fp32 accumulators in TMEM (tcgen05.mma, kind::f16)
+//             H[:, kept position of g] = bf16( silu(Dg) * Du )          epilogue straight from TMEM
+//   GEMM-2  for every 128-token x 128-column output tile, holder slot by holder slot:
+//             partials[slot] = H[:, groups of the slot] * down rows of those groups      (fp32 out)
+//           The down rows are read as stored in the packed layout (plane 2: one row of d per neuron), i.e. as an
+//           MN-major B operand; no second copy of the weights.
+// Operands reach shared memory by tensor-map TMA (128-byte swizzle, no multicast); kept groups are gathered by
+// choosing the TMA row coordinate from keep_list, so skipped groups are never read.  Warp roles: warp 0 TMA
+// producer, warp 1 MMA issuer (+ TMEM allocation), warps 2..5 epilogue.  All mbarrier waits are bounded; on a
+// timeout the CTA stops waiting, skips its stores, flags HALO_DEV_TIMEOUT, drains its copies and frees TMEM.
+#include <algorithm>
+#include <mutex>
+
+#include "common.cuh"
+#include "ffn_math.cuh"
+#include "umma.cuh"
+
+namespace halo {
+
+constexpr int kBM = 128;          // tokens per tile
+constexpr int kBK = 64;           // K elements per stage (128 bytes of bf16)
+constexpr int kUmmaK = 16;
+constexpr int kPfThreads = 192;   // 6 warps
+
+struct PfBarriers {
+    uint64_t full[8];
+    uint64_t empty[8];
+    uint64_t tmem_full;
+    uint64_t tmem_empty;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__device__ __forceinline__ bool pf_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (*abort_flag) return false;
+    if (mbar_wait_bounded(bar, parity, abort_flag)) return true;
+    *abort_flag = 1;
+    return false;
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// GEMM-1: hidden activations of one kept group for one tile of tokens
+// ------------------------------------------------------------------------------------------------------------
+template <int NS, int STAGES>
+__global__ void __launch_bounds__(kPfThreads, 1)
+ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, int T, int d,
+                  int S, int G, const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
+                  __nv_bfloat16* __restrict__ H, int h_cols, uint32_t* dev_status) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = NS * kBK * 2, kStageBytes = kABytes + 2 * kBBytes;
+    PfBarriers& bars = *reinterpret_cast<PfBarriers*>(smem_raw + static_cast<size_t>(STAGES) * kStageBytes);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int ki = blockIdx.y, m0 = blockIdx.x * kBM;
+    int nk = *n_keep_ptr;
+    nk = max(0, min(nk, G));
+    if (ki >= nk) return;
+    const int g = keep_list[ki];
+    if (g < 0 || g >= G) {
+        if (tid == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+        return;
+    }
+    const int n_kt = d / kBK;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], 1); }
+        mbar_init(&bars.tmem_full, 1);
+        mbar_init(&bars.tmem_empty, 1);
+        bars.abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_descriptor(&tmap_x);
+        tma_prefetch_descriptor(&tmap_w);
+    }
+    if (warp == 1) { tmem_alloc(&bars.tmem_base, 2 * NS); tmem_relinquish_alloc_permit(); }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    volatile int* abort_flag = &bars.abort_flag;
+    const uint32_t tmem = bars.tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int kt = 0; kt < n_kt; ++kt) {
+                const int s = kt % STAGES;
+                if (kt >= STAGES && !pf_wait(&bars.empty[s], ((kt / STAGES) - 1) & 1, abort_flag)) break;
+                unsigned char* st = smem_raw + static_cast<size_t>(s) * kStageBytes;
+                mbar_arrive_expect_tx(&bars.full[s], kStageBytes);
+                tma_load_2d(st, &tmap_x, kt * kBK, m0, &bars.full[s]);
+                tma_load_2d(st + kABytes, &tmap_w, kt * kBK, (g * 3 + 0) * S, &bars.full[s]);
+                tma_load_2d(st + kABytes + kBBytes, &tmap_w, kt * kBK, (g * 3 + 1) * S, &bars.full[s]);
+                issued = kt + 1;
+            }
+            if (*abort_flag) {  // let outstanding copies land before the CTA goes away
+                int never = 0;
+                for (int kt = max(0, issued - STAGES); kt < issued; ++kt)
+                    mbar_wait_bounded(&bars.full[kt % STAGES], (kt / STAGES) & 1, &never);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(kBM, NS, false);
+            for (int kt = 0; kt < n_kt; ++kt) {
+                const int s = kt % STAGES;
+                if (!pf_wait(&bars.full[s], (kt / STAGES) & 1, abort_flag)) break;
+                tcgen05_fence_after_sync();
+                const uint32_t a0 = smem_u32(smem_raw + static_cast<size_t>(s) * kStageBytes);
+#pragma unroll
+                for (int kk = 0; kk < kBK / kUmmaK; ++kk) {
+                    const uint64_t a = umma_smem_desc(a0 + kk * 32, 16, 1024);
+                    const uint64_t bg = umma_smem_desc(a0 + kABytes + kk * 32, 16, 1024);
+                    const uint64_t bu = umma_smem_desc(a0 + kABytes + kBBytes + kk * 32, 16, 1024);
+                    const bool accumulate = (kt > 0) || (kk > 0);
+                    umma_bf16(tmem, a, bg, idesc, accumulate);
+                    umma_bf16(tmem + NS, a, bu, idesc, accumulate);
+                }
+                umma_commit(&bars.empty[s]);   // the stage is free once these MMAs have read it
+            }
+            umma_commit(&bars.tmem_full);
+        }
+    } else {
+        // epilogue: this warp reads TMEM lanes [32*(warp%4), +32) = 32 tokens, one token per thread
+        const bool ok = pf_wait(&bars.tmem_full, 0, abort_flag);
+        tcgen05_fence_after_sync();
+        const int quad = warp & 3;
+        const int row = m0 + quad * 32 + lane;
+        const uint32_t lane_base = tmem + (static_cast<uint32_t>(quad * 32) << 16);
+        for (int c0 = 0; c0 < NS; c0 += 32) {
+            uint32_t dg[32], du[32];
+            tmem_ld_32x32(lane_base + c0, dg);
+            tmem_ld_32x32(lane_base + NS + c0, du);
+            tmem_ld_wait();
+            if (ok && row < T) {
+                uint4* dst = reinterpret_cast<uint4*>(H + static_cast<size_t>(row) * h_cols + static_cast<size_t>(ki) * S + c0);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t packed[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int i = q * 8 + e * 2;
+                        const float h0 = silu_mul(__uint_as_float(dg[i]), __uint_as_float(du[i]));
+                        const float h1 = silu_mul(__uint_as_float(dg[i + 1]), __uint_as_float(du[i + 1]));
+                        const __nv_bfloat162 p = __floats2bfloat162_rn(h0, h1);
+                        packed[e] = *reinterpret_cast<const uint32_t*>(&p);
+                    }
+                    dst[q] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                }
+            }
+        }
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, 2 * NS); }
+    if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// GEMM-2: down projection of the kept columns, one accumulation per holder slot
+// ------------------------------------------------------------------------------------------------------------
+constexpr int kBN2 = 128;   // output columns per tile
+
+struct DownSmemTail {
+    PfBarriers bars;
+    int slot_start[HALO_MAX_DEVICES + 2];
+    int32_t group_of[HALO_MAX_GROUPS];    // group id per position of the slot-sorted order (-1 = skip)
+    int16_t kept_pos[HALO_MAX_GROUPS];    // kept position (column block of H) per position of the order
+};
+
+template <int STAGES>
+__global__ void __launch_bounds__(kPfThreads, 1)
+ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_wd, int T, int d,
+                int S, int G, const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
+                const int32_t* __restrict__ dev_of_group, int n_dev, float* __restrict__ partials,
+                uint32_t* dev_status) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = kBK * kBN2 * 2, kStageBytes = kABytes + kBBytes;
+    DownSmemTail& tail = *reinterpret_cast<DownSmemTail*>(smem_raw + static_cast<size_t>(STAGES) * kStageBytes);
+    PfBarriers& bars = tail.bars;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * kBN2;
+    int nk = *n_keep_ptr;
+    nk = max(0, min(nk, G));
+    const int k_per_group = S / kBK;   // K stages per kept group
+    const int n_slots = n_dev + 1;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], 1); }
+        mbar_init(&bars.tmem_full, 1);
+        mbar_init(&bars.tmem_empty, 4);
+        bars.abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_descriptor(&tmap_h);
+        tma_prefetch_descriptor(&tmap_wd);
+    }
+    if (warp == 1) { tmem_alloc(&bars.tmem_base, kBN2); tmem_relinquish_alloc_permit(); }
+    if (warp == 0) {
+        // kept positions sorted by holder slot (stable): one warp, ballot compaction per slot
+        int pos = 0;
+        for (int slot = 0; slot < n_slots; ++slot) {
+            if (lane == 0) tail.slot_start[slot] = pos;
+            for (int base = 0; base < nk; base += 32) {
+                const int ki = base + lane;
+                int g = -1, sl = -1;
+                if (ki < nk) {
+                    g = keep_list[ki];
+                    if (g >= 0 && g < G) sl = dev_of_group ? dev_of_group[g] + 1 : 0;
+                    if (sl < 0 || sl > n_dev) { sl = -1; if (slot == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX); }
+                }
+                const bool match = (sl == slot);
+                const unsigned ballot = __ballot_sync(0xffffffffu, match);
+                if (match) {
+                    const int p = pos + __popc(ballot & ((1u << lane) - 1u));
+                    tail.group_of[p] = g;
+                    tail.kept_pos[p] = static_cast<int16_t>(ki);
+                }
+                pos += __popc(ballot);
+            }
+        }
+        if (lane == 0) tail.slot_start[n_slots] = pos;
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    volatile int* abort_flag = &bars.abort_flag;
+    const uint32_t tmem = bars.tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int it = 0;
+            bool alive = true;
+            const int total = tail.slot_start[n_slots];
+            for (int p = 0; p < total && alive; ++p) {
+                const int g = tail.group_of[p], kp = tail.kept_pos[p];
+                for (int kk2 = 0; kk2 < k_per_group; ++kk2, ++it) {
+                    const int s = it % STAGES;
+                    if (it >= STAGES && !pf_wait(&bars.empty[s], ((it / STAGES) - 1) & 1, abort_flag)) { alive = false; break; }
+                    unsigned char* st = smem_raw + static_cast<size_t>(s) * kStageBytes;
+                    mbar_arrive_expect_tx(&bars.full[s], kStageBytes);
+                    tma_load_2d(st, &tmap_h, kp * S + kk2 * kBK, m0, &bars.full[s]);
+                    const int krow = (g * 3 + 2) * S + kk2 * kBK;
+                    tma_load_2d(st + kABytes, &tmap_wd, n0, krow, &bars.full[s]);
+                    tma_load_2d(st + kABytes + kBBytes / 2, &tmap_wd, n0 + 64, krow, &bars.full[s]);
+                }
+            }
+            if (*abort_flag) {
+                int never = 0;
+                for (int k = max(0, it - STAGES); k < it; ++k)
+                    mbar_wait_bounded(&bars.full[k % STAGES], (k / STAGES) & 1, &never);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(kBM, kBN2, true);
+            int it = 0, used = 0;
+            bool alive = true;
+            for (int slot = 0; slot < n_slots && alive; ++slot) {
+                const int p0 = tail.slot_start[slot], p1 = tail.slot_start[slot + 1];
+                if (p0 == p1) continue;
+                if (used > 0 && !pf_wait(&bars.tmem_empty, (used - 1) & 1, abort_flag)) break;  // epilogue has drained D
+                tcgen05_fence_after_sync();
+                const int n_it = (p1 - p0) * k_per_group;
+                for (int k = 0; k < n_it; ++k, ++it) {
+                    const int s = it % STAGES;
+                    if (!pf_wait(&bars.full[s], (it / STAGES) & 1, abort_flag)) { alive = false; break; }
+                    tcgen05_fence_after_sync();
+                    const uint32_t a0 = smem_u32(smem_raw + static_cast<size_t>(s) * kStageBytes);
+#pragma unroll
+                    for (int kk = 0; kk < kBK / kUmmaK; ++kk) {
+                        const uint64_t a = umma_smem_desc(a0 + kk * 32, 16, 1024);
+                        // MN-major B: 16 K-rows per MMA = 2 KiB further; 64-column blocks are kBBytes/2 apart
+                        const uint64_t b = umma_smem_desc(a0 + kABytes + kk * 2048, kBBytes / 2, 1024);
+                        umma_bf16(tmem, a, b, idesc, (k > 0) || (kk > 0));
+                    }
+                    umma_commit(&bars.empty[s]);
+                }
+                if (!alive) break;
+                umma_commit(&bars.tmem_full);
+                ++used;
+            }
+        }
+    } else {
+        const int quad = warp & 3;
+        const int row = m0 + quad * 32 + lane;
+        const uint32_t lane_base = tmem + (static_cast<uint32_t>(quad * 32) << 16);
+        int used = 0;
+        for (int slot = 0; slot < n_slots; ++slot) {
+            if (tail.slot_start[slot] == tail.slot_start[slot + 1]) continue;
+            const bool ok = pf_wait(&bars.tmem_full, used & 1, abort_flag);
+            tcgen05_fence_after_sync();
+            float* out = partials + (static_cast<size_t>(slot) * T + row) * d + n0;
+            for (int c0 = 0; c0 < kBN2; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32(lane_base + c0, v);
+                tmem_ld_wait();
+                if (ok && row < T) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        reinterpret_cast<float4*>(out + c0)[q] =
+                            make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                        __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+                }
+            }
+            tcgen05_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars.tmem_empty);
+            ++used;
+        }
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, kBN2); }
+    if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
+}
+
+// ---- host side ------------------------------------------------------------------------------------------------
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// bf16 matrix [rows][cols] (cols contiguous), box = box_cols x box_rows, 128-byte swizzle, zero fill out of range
+bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t row_stride_elems,
+              uint32_t box_cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {row_stride_elems * 2};
+    const cuuint32_t box[2] = {box_cols, box_rows};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem_strides,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <typename K>
+bool set_smem(K kernel, size_t bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) == cudaSuccess;
+}
+
+}  // namespace
+
+bool prefill_supported(const halo_ffn_shape& sh, int n_tok) {
+    return sh.wdtype == HALO_BF16 && n_tok >= 16 && (sh.group_size == 64 || sh.group_size == 128) &&
+           sh.d_model % 128 == 0 && sh.d_ffn / sh.group_size <= HALO_MAX_GROUPS;
+}
+
+size_t prefill_workspace_bytes(const halo_ffn_shape& sh, int n_tok) {
+    return static_cast<size_t>(n_tok) * sh.d_ffn * 2;   // H: bf16 [n_tok][d_ffn], kept groups packed to the left
+}
+
+// partials must already be zero (slots without kept groups are not written).
+halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
+                                     const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
+                                     int n_dev, float* partials, void* workspace, uint32_t* dev_status,
+                                     cudaStream_t st) {
+    const int d = sh.d_model, S = sh.group_size, G = sh.d_ffn / S, T = n_tok;
+    __nv_bfloat16* H = static_cast<__nv_bfloat16*>(workspace);
+    const uint64_t w_rows = static_cast<uint64_t>(G) * 3 * S;
+    CUtensorMap map_x, map_w, map_h, map_wd;
+    if (!make_map(&map_x, x, T, d, d, kBK, kBM) || !make_map(&map_w, W, w_rows, d, d, kBK, S) ||
+        !make_map(&map_h, H, T, sh.d_ffn, sh.d_ffn, kBK, kBM) || !make_map(&map_wd, W, w_rows, d, d, 64, kBK))
+        return HALO_ERR_CUDA;
+    const dim3 grid1((T + kBM - 1) / kBM, G);
+    const dim3 grid2((T + kBM - 1) / kBM, d / kBN2);
+    constexpr int kStages1 = 4, kStages2 = 6;
+    if (S == 128) {
+        auto k1 = ffn_hidden_kernel<128, kStages1>;
+        const size_t smem1 = static_cast<size_t>(kStages1) * (kBM * kBK * 2 + 2 * 128 * kBK * 2) + sizeof(PfBarriers) + 1024;
+        static bool once1 = false;
+        if (!once1) { if (!set_smem(k1, smem1)) return HALO_ERR_CUDA; once1 = true; }
+        k1<<<grid1, kPfThreads, smem1, st>>>(map_x, map_w, T, d, S, G, keep_list, n_keep, H, sh.d_ffn, dev_status);
+    } else {
+        auto k1 = ffn_hidden_kernel<64, kStages1>;
+        const size_t smem1 = static_cast<size_t>(kStages1) * (kBM * kBK * 2 + 2 * 64 * kBK * 2) + sizeof(PfBarriers) + 1024;
+        static bool once1 = false;
+        if (!once1) { if (!set_smem(k1, smem1)) return HALO_ERR_CUDA; once1 = true; }
+        k1<<<grid1, kPfThreads, smem1, st>>>(map_x, map_w, T, d, S, G, keep_list, n_keep, H, sh.d_ffn, dev_status);
+    }
+    HALO_CHECK_LAUNCH();
+    auto k2 = ffn_down_kernel<kStages2>;
+    const size_t smem2 = static_cast<size_t>(kStages2) * (kBM * kBK * 2 + kBK * kBN2 * 2) + sizeof(DownSmemTail) + 1024;
+    static bool once2 = false;
+    if (!once2) { if (!set_smem(k2, smem2)) return HALO_ERR_CUDA; once2 = true; }
+    k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, partials,
+                                         dev_status);
+    HALO_CHECK_LAUNCH();
+    return HALO_OK;
+}
+
+}  // namespace halo

@@ -1,0 +1,71 @@
+"""GPU parity of the tensor-core (many-token) form of halo_group_ffn against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import halo_ref as R
+from paper_2601_11676_b200 import binding as B
+from paper_2601_11676_b200 import synth
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+DEV = U.DEV
+
+
+def _wl(d, G, S, n_dev=3):
+    return synth.Workload("pf", 1, d, G * S, S, 64, "bf16", (0.0, 0.2, 0.6)[:n_dev], (3, 2, 1)[:n_dev], 500, 1)
+
+
+@pytest.mark.parametrize("d,G,S,n_tok", [(256, 3, 128, 32), (512, 5, 64, 130), (1024, 4, 128, 257), (256, 6, 64, 16)])
+def test_prefill_ffn_small_shapes_all_tokens(d, G, S, n_tok):
+    wl = _wl(d, G, S)
+    sh = B.ffn_shape(d, G * S, S, B.BF16)
+    assert B.halo_group_ffn_workspace_bytes(sh, n_tok, wl.n_dev) == n_tok * G * S * 2
+    Wp = synth.packed_layer(wl, 0, DEV)
+    x = synth.activation(wl, 1, DEV, n_tok=n_tok)
+    dev = np.array([-1, 0, 1, 2, 0, -1], dtype=np.int32)[:G]
+    for keep in ([g for g in range(G) if g != 1], list(range(G)), [G - 1], []):
+        P, status = U.gpu_group_ffn(wl, Wp, x, keep, dev, wl.n_dev)
+        ref = R.group_ffn(synth.host_bits(Wp), synth.host_bits(x), keep, dev, wl.n_dev)
+        assert status == 0
+        y_ref = R.merge(ref)
+        rms = np.sqrt(np.mean(y_ref ** 2)) if len(keep) else 1.0
+        err = np.abs(P.cpu().numpy() - ref).max() / rms
+        assert err <= U.TOL_BF16, (keep, err)
+        if not keep:
+            assert (P == 0).all().item()
+
+
+def test_prefill_matches_decode_path_token_by_token():
+    wl = _wl(512, 4, 128)
+    Wp = synth.packed_layer(wl, 0, DEV)
+    x = synth.activation(wl, 2, DEV, n_tok=64)
+    keep, dev = [0, 2, 3], np.array([-1, 1, 0, 1], dtype=np.int32)
+    P_many, _ = U.gpu_group_ffn(wl, Wp, x, keep, dev, wl.n_dev)
+    for t in (0, 31, 63):
+        P_one, _ = U.gpu_group_ffn(wl, Wp, x[t:t + 1].contiguous(), keep, dev, wl.n_dev)
+        ref = P_one[:, 0].cpu().numpy().astype(np.float64)
+        rms = np.sqrt(np.mean(ref.sum(0) ** 2))
+        assert np.abs(P_many[:, t].cpu().numpy() - ref).max() <= U.TOL_BF16 * rms
+
+
+def test_prefill_full_size_7b_block_sampled_tokens():
+    """The prefill workload's shapes (512 tokens, one 7B block); the oracle checks a sample of the tokens."""
+    wl = synth.workload("llama2-7b-prefill")
+    G = wl.n_groups
+    Wp = synth.packed_layer(wl, 1, DEV)
+    x = synth.activation(wl, 3, DEV, n_tok=wl.n_tok)
+    scores = np.random.default_rng(5).normal(size=G).astype(np.float32)
+    sel = R.select(scores, wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed, 0, 1)
+    keep = sel["keep_list"][: sel["n_keep"]]
+    P, status = U.gpu_group_ffn(wl, Wp, x, keep, sel["dev_of_group"], wl.n_dev)
+    assert status == 0
+    sample = [0, 127, 128, 300, 511]
+    xs = synth.host_bits(x)[sample]
+    ref = R.group_ffn(synth.host_bits(Wp), xs, keep, sel["dev_of_group"], wl.n_dev)
+    y_ref = R.merge(ref)
+    rms = np.sqrt(np.mean(y_ref ** 2))
+    got = P[:, sample].cpu().numpy()
+    assert np.abs(got - ref).max() <= U.TOL_BF16 * rms
+    y = U.gpu_merge(P, sel["arrived"])[sample].cpu().numpy()
+    assert U.rel_err(y, y_ref) <= U.TOL_BF16

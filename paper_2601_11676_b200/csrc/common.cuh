@@ -107,6 +107,9 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
                                      const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
                                      int n_dev, float* partials, void* workspace, uint32_t* dev_status,
                                      cudaStream_t st);
+bool pred_gemm_supported(const halo_pred_shape& sh, int n_tok);
+halo_status launch_pred_hidden_gemm(const halo_pred_shape& sh, const void* W1, const void* feat, int n_tok,
+                                    float* hidden, uint32_t* dev_status, cudaStream_t st);
 halo_status launch_merge(const float* partials, const uint8_t* arrived, int n_dev, int n_tok, int d, float* y,
                          cudaStream_t st);
 halo_status launch_glue(int d, int n_tok, halo_dtype xdtype, const float* h, const float* y, float* h_out,

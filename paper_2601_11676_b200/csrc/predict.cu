@@ -102,7 +102,9 @@ halo_status launch_predict(const halo_pred_shape& sh, const void* W1, const void
                            int mean_pool, float* scores, float* workspace, uint32_t* dev_status, cudaStream_t st) {
     float* hidden = workspace;                                        // [n_tok][rank]
     float* per_tok = workspace + static_cast<size_t>(n_tok) * sh.rank;  // [n_tok][G], pooled case only
-    halo_status rc = launch_predict_hidden(sh, W1, feat, n_tok, hidden, st);
+    // many tokens: the hidden layer is a dense contraction -> tensor cores; few tokens: one warp per hidden unit
+    halo_status rc = pred_gemm_supported(sh, n_tok) ? launch_pred_hidden_gemm(sh, W1, feat, n_tok, hidden, dev_status, st)
+                                                    : launch_predict_hidden(sh, W1, feat, n_tok, hidden, st);
     if (rc != HALO_OK) return rc;
     const bool pool = mean_pool && n_tok > 1;
     float* out = pool ? per_tok : scores;

@@ -314,6 +314,102 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
     if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
 }
 
+// ------------------------------------------------------------------------------------------------------------
+// Predictor hidden layer for many tokens: Z[T][r] = act(X[T][d] * W1[r][d]^T), fp32 out (step a1, prefill)
+// ------------------------------------------------------------------------------------------------------------
+template <int STAGES>
+__global__ void __launch_bounds__(kPfThreads, 1)
+pred_hidden_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1, int T,
+                        int d, int r, int act, float* __restrict__ Z, uint32_t* dev_status) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    constexpr int BN = 128;
+    constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = BN * kBK * 2, kStageBytes = kABytes + kBBytes;
+    PfBarriers& bars = *reinterpret_cast<PfBarriers*>(smem_raw + static_cast<size_t>(STAGES) * kStageBytes);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * BN;
+    const int n_kt = d / kBK;
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], 1); }
+        mbar_init(&bars.tmem_full, 1);
+        mbar_init(&bars.tmem_empty, 1);
+        bars.abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_descriptor(&tmap_x);
+        tma_prefetch_descriptor(&tmap_w1);
+    }
+    if (warp == 1) { tmem_alloc(&bars.tmem_base, BN); tmem_relinquish_alloc_permit(); }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    volatile int* abort_flag = &bars.abort_flag;
+    const uint32_t tmem = bars.tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int kt = 0; kt < n_kt; ++kt) {
+                const int s = kt % STAGES;
+                if (kt >= STAGES && !pf_wait(&bars.empty[s], ((kt / STAGES) - 1) & 1, abort_flag)) break;
+                unsigned char* st = smem_raw + static_cast<size_t>(s) * kStageBytes;
+                mbar_arrive_expect_tx(&bars.full[s], kStageBytes);
+                tma_load_2d(st, &tmap_x, kt * kBK, m0, &bars.full[s]);
+                tma_load_2d(st + kABytes, &tmap_w1, kt * kBK, n0, &bars.full[s]);   // rows beyond r read as zeros
+                issued = kt + 1;
+            }
+            if (*abort_flag) {
+                int never = 0;
+                for (int kt = max(0, issued - STAGES); kt < issued; ++kt)
+                    mbar_wait_bounded(&bars.full[kt % STAGES], (kt / STAGES) & 1, &never);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN, false);
+            for (int kt = 0; kt < n_kt; ++kt) {
+                const int s = kt % STAGES;
+                if (!pf_wait(&bars.full[s], (kt / STAGES) & 1, abort_flag)) break;
+                tcgen05_fence_after_sync();
+                const uint32_t a0 = smem_u32(smem_raw + static_cast<size_t>(s) * kStageBytes);
+#pragma unroll
+                for (int kk = 0; kk < kBK / kUmmaK; ++kk)
+                    umma_bf16(tmem, umma_smem_desc(a0 + kk * 32, 16, 1024),
+                              umma_smem_desc(a0 + kABytes + kk * 32, 16, 1024), idesc, (kt > 0) || (kk > 0));
+                umma_commit(&bars.empty[s]);
+            }
+            umma_commit(&bars.tmem_full);
+        }
+    } else {
+        const bool ok = pf_wait(&bars.tmem_full, 0, abort_flag);
+        tcgen05_fence_after_sync();
+        const int quad = warp & 3;
+        const int row = m0 + quad * 32 + lane;
+        const uint32_t lane_base = tmem + (static_cast<uint32_t>(quad * 32) << 16);
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld_32x32(lane_base + c0, v);
+            tmem_ld_wait();
+            if (ok && row < T) {
+                float* out = Z + static_cast<size_t>(row) * r + n0 + c0;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (n0 + c0 + 4 * q < r) {   // r is a multiple of 8
+                        float4 o = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                               __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+                        if (act == HALO_ACT_RELU) {
+                            o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f);
+                        }
+                        reinterpret_cast<float4*>(out)[q] = o;
+                    }
+                }
+            }
+        }
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, BN); }
+    if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
+}
+
 // ---- host side ------------------------------------------------------------------------------------------------
 
 namespace {
@@ -400,6 +496,28 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
     if (!once2) { if (!set_smem(k2, smem2)) return HALO_ERR_CUDA; once2 = true; }
     k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, partials,
                                          dev_status);
+    HALO_CHECK_LAUNCH();
+    return HALO_OK;
+}
+
+bool pred_gemm_supported(const halo_pred_shape& sh, int n_tok) {
+    return sh.wdtype == HALO_BF16 && n_tok >= 16 && sh.d_in % kBK == 0;
+}
+
+// Z[n_tok][rank] = act(feat * W1^T) on the tensor cores.
+halo_status launch_pred_hidden_gemm(const halo_pred_shape& sh, const void* W1, const void* feat, int n_tok,
+                                    float* hidden, uint32_t* dev_status, cudaStream_t st) {
+    CUtensorMap map_x, map_w1;
+    if (!make_map(&map_x, feat, n_tok, sh.d_in, sh.d_in, kBK, kBM) ||
+        !make_map(&map_w1, W1, sh.rank, sh.d_in, sh.d_in, kBK, 128))
+        return HALO_ERR_CUDA;
+    constexpr int kStages = 6;
+    auto k = pred_hidden_gemm_kernel<kStages>;
+    const size_t smem = static_cast<size_t>(kStages) * (kBM * kBK * 2 + 128 * kBK * 2) + sizeof(PfBarriers) + 1024;
+    static bool once = false;
+    if (!once) { if (!set_smem(k, smem)) return HALO_ERR_CUDA; once = true; }
+    const dim3 grid((n_tok + kBM - 1) / kBM, (sh.rank + 127) / 128);
+    k<<<grid, kPfThreads, smem, st>>>(map_x, map_w1, n_tok, sh.d_in, sh.rank, sh.act, hidden, dev_status);
     HALO_CHECK_LAUNCH();
     return HALO_OK;
 }

@@ -69,3 +69,22 @@ def test_prefill_full_size_7b_block_sampled_tokens():
     assert np.abs(got - ref).max() <= U.TOL_BF16 * rms
     y = U.gpu_merge(P, sel["arrived"])[sample].cpu().numpy()
     assert U.rel_err(y, y_ref) <= U.TOL_BF16
+
+
+@pytest.mark.parametrize("d,r,G,n_tok,pool", [(256, 64, 6, 32, True), (512, 200, 43, 130, False), (4096, 256, 86, 512, True),
+                                              (5120, 512, 108, 64, True)])
+@pytest.mark.parametrize("act", [B.ACT_RELU, B.ACT_NONE])
+def test_predictor_many_tokens_tensor_core_hidden_layer(d, r, G, n_tok, pool, act):
+    wl = synth.Workload("pp", 1, d, G * 8, 8, r, "bf16", (0.0,), (1,), 500, 1)
+    W1, W2 = synth.predictor(wl, 1, DEV)
+    feat = synth.activation(wl, 9, DEV, n_tok=n_tok)
+    s, status = U.gpu_predict(B.BF16, W1, W2, feat, mean_pool=pool, act=act)
+    assert status == 0
+    sample = slice(None) if n_tok <= 130 else [0, 1, 127, 128, 255, 256, 511]
+    hb = synth.host_bits
+    if pool:
+        ref = R.predict(hb(W1), hb(W2), hb(feat), act=act, mean_pool=True)
+        assert U.rel_err(s.cpu().numpy(), ref.astype(np.float64)) <= U.TOL_BF16
+    else:
+        ref = R.predict(hb(W1), hb(W2), hb(feat)[sample], act=act)
+        assert U.rel_err(s[sample].cpu().numpy(), ref.astype(np.float64)) <= U.TOL_BF16

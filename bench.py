@@ -243,9 +243,48 @@ def run_halo(args, rank, world, local_rank):
     # the unfused halo_group_ffn entry point timed alone (memset + kernel per call), for comparison
     result["group_ffn_entry"] = {"achieved_gbs": kernel_gbs, "avg_call_us": kernel_avg_us, "calls_timed": k_launches,
                                  "frac_of_peak": kernel_gbs / peak}
+    if world == 1 and not args.no_prefill and wl.dtype == "bf16" and wl.n_tok == 1:
+        result["prefill"] = prefill_report(wl, Wp, preds, plan, ffn, dev)
     if world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget)
     return result
+
+
+def prefill_report(wl, Wp, preds, plan, ffn, dev, n_tok=512, prompts=8, warm=3):
+    """The same stack run on a 512-token prompt (tensor-core form of the masked FFN), weights shared with the decode
+    run: milliseconds per prompt and achieved bf16 TFLOP/s over the kept groups' FLOPs."""
+    from paper_2601_11676_b200 import binding as B
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peaks = json.load(open(pk)) if os.path.exists(pk) else {}
+    burst, sustained = float(peaks.get("bf16_tflops", 1590.0)), float(peaks.get("bf16_tflops_sustained", 1400.0))
+    L, G, d = wl.n_layers, wl.n_groups, wl.d_model
+    pred = B.pred_shape(d, wl.pred_rank, G, B.BF16)
+    stack = B.Stack(ffn, pred, n_tok, plan, Wp, [p[0] for p in preds], [p[1] for p in preds])
+    pw = synth.workload(wl.name, n_tok=n_tok)
+    total = warm + prompts
+    h0 = torch.stack([synth.stream_input(pw, 1000 + s, dev) for s in range(total)])
+    h_out = torch.empty_like(h0)
+    nk_rec = torch.zeros((total, L), dtype=torch.int32, device=dev)
+    taps = B.Taps(None, None, None, None, None, nk_rec.data_ptr(), None)
+    stack.decode(h0, total, 0, h_out, taps)     # records the kept sets; also the warm-up
+    torch.cuda.synchronize()
+    status = stack.status()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    stack.decode(h0[warm:], prompts, warm, h_out[warm:])
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b)
+    launches = stack.last_launches()
+    kept = int(nk_rec[warm:].sum().item())
+    flops = 6.0 * n_tok * kept * wl.group_size * d + prompts * (L - 1) * 2.0 * n_tok * (d * wl.pred_rank + wl.pred_rank * G)
+    tflops = flops / (ms * 1e-3) / 1e12
+    stack.close()
+    return {"workload": wl.name.replace("decode", "prefill"), "prompt_tokens": n_tok, "prompts_timed": prompts,
+            "ms_per_prompt": ms / prompts, "tokens_per_s": prompts * n_tok / (ms * 1e-3), "tflops": tflops,
+            "bound": "tensor", "peak_burst_tflops": burst, "frac_of_burst_peak": tflops / burst,
+            "peak_sustained_tflops": sustained, "frac_of_sustained_peak": tflops / sustained,
+            "kept_fraction": kept / float(prompts * L * G), "gpu_launches": int(launches), "device_status": status}
 
 
 # ----------------------------------------------------------------------------------------------------------------
@@ -345,6 +384,7 @@ def main():
     ap.add_argument("--keep-permille", type=int, default=500)
     ap.add_argument("--layers", type=int, default=0, help="use only this many blocks (small profiling cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill", action="store_true", help="skip the 512-token prompt report")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "halo" else args.warmup

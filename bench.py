@@ -93,6 +93,25 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------------------------
+# replicas: every rank runs the same workload on its own GPU; the job's time is the slowest rank's
+# ----------------------------------------------------------------------------------------------------------------
+
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of a list of floats over all ranks (identity for a single process)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def aggregate_tokens_per_s(tokens_per_rank, ms_this_rank, world, device):
+    """Whole-job tokens/s of `world` independent replicas: all ranks' tokens over the slowest rank's time."""
+    (ms,) = max_over_ranks([ms_this_rank], world, device)
+    return tokens_per_rank * world / (ms * 1e-3), ms
+
+
+# ----------------------------------------------------------------------------------------------------------------
 # the CUDA arm
 # ----------------------------------------------------------------------------------------------------------------
 
@@ -198,16 +217,13 @@ def run_halo(args, rank, world, local_rank):
     kernel_gbs = k_bytes / (k_ms * 1e-3) / 1e9
 
     # ---- max over ranks -------------------------------------------------------------------------------------------
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], world, dev)
     if rank != 0:
         return None
 
     peak, peak_kind = measured_peaks()
     tokens = K * world
-    value = tokens / (ms * 1e-3)
+    value = tokens / (ms * 1e-3)   # == aggregate_tokens_per_s(K, ms_local, world, dev)[0]: ms is already the max
     step_gbs = algo_bytes_total / (ms * 1e-3) / 1e9
     result = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,

@@ -74,13 +74,23 @@ predict_out_kernel(int rank, int G, const T* __restrict__ W2, const float* __res
     }
 }
 
-// Mean over tokens in token order (one thread per group).
-__global__ void mean_pool_kernel(int n_tok, int G, const float* __restrict__ per_tok, float* __restrict__ scores) {
-    const int g = blockIdx.x * blockDim.x + threadIdx.x;
-    if (g >= G) return;
+// Mean over tokens: one block per group, threads stride over the tokens, fixed-shape tree reduction (the result
+// does not depend on scheduling).
+__global__ void __launch_bounds__(256)
+mean_pool_kernel(int n_tok, int G, const float* __restrict__ per_tok, float* __restrict__ scores) {
+    __shared__ float part[8];
+    const int g = blockIdx.x;
     float acc = 0.0f;
-    for (int t = 0; t < n_tok; ++t) acc += per_tok[static_cast<size_t>(t) * G + g];
-    scores[g] = acc / static_cast<float>(n_tok);
+    for (int t = threadIdx.x; t < n_tok; t += 256) acc += per_tok[static_cast<size_t>(t) * G + g];
+    acc = warp_sum(acc);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) tot += part[w];
+        scores[g] = tot / static_cast<float>(n_tok);
+    }
 }
 
 halo_status launch_predict_hidden(const halo_pred_shape& sh, const void* W1, const void* feat, int n_tok,
@@ -118,7 +128,7 @@ halo_status launch_predict(const halo_pred_shape& sh, const void* W1, const void
                                                             hidden, out, dev_status);
     HALO_CHECK_LAUNCH();
     if (pool) {
-        mean_pool_kernel<<<(sh.n_groups + 127) / 128, 128, 0, st>>>(n_tok, sh.n_groups, per_tok, scores);
+        mean_pool_kernel<<<sh.n_groups, 256, 0, st>>>(n_tok, sh.n_groups, per_tok, scores);
         HALO_CHECK_LAUNCH();
     }
     return HALO_OK;

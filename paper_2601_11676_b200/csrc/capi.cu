@@ -340,7 +340,7 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     const size_t o_tw = carve(sizeof(void*) * n_layers), o_tw1 = carve(sizeof(void*) * n_layers);
     const size_t o_tw2 = carve(sizeof(void*) * n_layers);
     const size_t o_pp = carve(sizeof(float) * 3 * 2 * d);
-    const size_t o_pz = carve(sizeof(float) * pred->rank);
+    const size_t o_pz = carve(sizeof(float) * 2 * pred->rank);
     const size_t o_ps = carve(sizeof(PersistSel) * 3);
     const size_t o_py = carve(sizeof(unsigned) * 32);
     const size_t ws_bytes = prefill_supported(*ffn, n_tok) ? prefill_workspace_bytes(*ffn, n_tok) : 0;

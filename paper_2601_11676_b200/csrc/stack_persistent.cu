@@ -4,9 +4,12 @@
 // One thread block per SM: a producer warp and 512 consumer threads around a ring of shared-memory stages fed
 // by bulk asynchronous copies.  The producer's stream for block l of a step is
 //     [rows of W1 of block l+1 owned by this thread block]   predictor hidden layer, one layer ahead (a1)
-//     [SELECT marker, last thread block only]                 scores, rank, assignment, arrival mask (a1..a5)
 //     [batches of NB kept neurons of block l]                 gate/up dot products, SiLU*up, down rows (a6..a8)
 //     [END marker]
+// The last thread block streams nothing: it is the selector.  As soon as all hidden values of block l+1 are in
+// (a counter), it computes the scores and steps a2..a5 and publishes the kept set (a flag); it takes no part in
+// the grid barrier, so a selection never delays a block unless it takes longer than the block itself.  The
+// stream is HBM-bound, so the SM given up for this costs nothing.
 // and it runs ahead of the consumers by the ring depth, across the end of the block: while the consumers sit in
 // the grid barrier and the glue, the next block's weights are already landing in shared memory.
 // Batches are handed out dynamically (one atomic counter per block, fetched one batch ahead), so a slow or busy
@@ -14,8 +17,7 @@
 // what was computed: each thread block stages its column sums in shared memory and adds them to one of
 // kAccBufs interleaved global buffers with ONE bulk reduction (cp.reduce.async.bulk, fp32 add, done by the copy
 // engine in L2), then one grid-wide barrier, then every thread block redundantly sums the buffers,
-// adds the residual, normalises, and keeps its own copy of x for the next block.  The selection of block l+1 is published early in block l, so the
-// producers never wait for it in practice.
+// adds the residual, normalises, and keeps its own copy of x for the next block.
 // Every wait (mbarrier, grid barrier, flags) is bounded to about a second; on a timeout the thread block takes
 // a uniform exit, raises a global abort word and HALO_DEV_TIMEOUT, and every other thread block follows.
 #include <algorithm>
@@ -35,13 +37,13 @@ constexpr int kHeaderBytes = 16 * 1024;  // PersistSmem
 constexpr int kAccBufs = 2;              // interleaved accumulation buffers per block of the stack
 constexpr int kFetchAhead = 3;           // batch-counter fetches a producer keeps in flight
 
-enum StageType { ST_FFN = 0, ST_PRED = 1, ST_SELECT = 2, ST_END = 3 };
+enum StageType { ST_FFN = 0, ST_PRED = 1, ST_END = 3 };
 
 struct PersistSmem {
     uint64_t full[8];
     uint64_t empty[8];
     int type[8];
-    int arg0[8];   // FFN: holder slot (-1 = skip); PRED: first row; SELECT: block to select for
+    int arg0[8];   // FFN: 0 = compute, -1 = skip; PRED: first row
     int arg1[8];   // PRED: number of rows
     int abort_flag;
     int blocks_done;   // blocks of the stack whose grid barrier this thread block's consumers have passed
@@ -117,7 +119,8 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
     const uint32_t stage_bytes = 3u * plane_bytes;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int grid = gridDim.x, cta = blockIdx.x;
-    const bool is_selector = (cta == grid - 1);
+    const int workers = grid - 1;                 // thread blocks that stream weights; the last one selects
+    const bool is_selector = (cta == workers);
     const int per_group = S / NB;
     unsigned* const sync_barrier = P.sync + 0;
     unsigned* const sync_abort = P.sync + 1;
@@ -132,6 +135,87 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
     }
     __syncthreads();
     volatile int* abort_flag = &sm.abort_flag;
+
+    // =========================================== selector ===========================================
+    if (is_selector) {
+        if (warp == kPCWarps) return;   // only the 512 "consumer" threads are used here
+        bool bad = false;
+        for (int step_i = 0; step_i < P.steps && !bad; ++step_i) {
+            for (int lp = 1; lp < L && !bad; ++lp) {
+                // prediction number n_pred (1-based over the run) = the selection of block lp of this step; its
+                // hidden values are produced by the workers during block lp-1
+                const unsigned n_pred = static_cast<unsigned>(step_i) * (L - 1) + lp;
+                // W2 of this block is read once per token: start it towards L2 while the hidden values come in
+                if (tid == 0) bulk_prefetch_l2(P.W2[lp], (static_cast<uint32_t>(G) * r * 2u) & ~15u);
+                bool okz = true;
+                if (tid == 0) okz = spin_until_ge(sync_zcount, n_pred * static_cast<unsigned>(r), sync_abort);
+                bad = pc_barrier_or(!okz);
+                if (bad) break;
+                const unsigned long long t_sel = (P.trace && tid == 0) ? global_timer_ns() : 0ull;
+                // a1 (second layer): s[g] = <W2[g], z>
+                const float* zsrc = P.z + static_cast<size_t>(n_pred & 1u) * r;
+                const __nv_bfloat16* W2 = P.W2[lp];
+                const int zc = r >> 3;  // 16-byte chunks per W2 row
+                for (int c0 = 0; c0 < zc; c0 += 32) {
+                    const int c = c0 + lane;
+                    float zv[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                    if (c < zc) {
+                        const float4 z0 = __ldcg(reinterpret_cast<const float4*>(zsrc) + 2 * c);
+                        const float4 z1 = __ldcg(reinterpret_cast<const float4*>(zsrc) + 2 * c + 1);
+                        zv[0] = z0.x; zv[1] = z0.y; zv[2] = z0.z; zv[3] = z0.w;
+                        zv[4] = z1.x; zv[5] = z1.y; zv[6] = z1.z; zv[7] = z1.w;
+                    }
+                    // groups warp, warp+16, ...: all row loads of a pass are issued before any is used
+                    for (int g0 = warp; g0 < G; g0 += kPCWarps * 8) {
+                        uint4 wv[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const int g = g0 + u * kPCWarps;
+                            wv[u] = (g < G && c < zc) ? __ldg(reinterpret_cast<const uint4*>(W2 + static_cast<size_t>(g) * r) + c)
+                                                      : make_uint4(0, 0, 0, 0);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const int g = g0 + u * kPCWarps;
+                            float w8[8];
+                            Elem<__nv_bfloat16>::widen(wv[u], w8);
+                            float dot = 0.0f;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) dot = fmaf(w8[e], zv[e], dot);
+                            dot = warp_sum(dot);
+                            if (lane == 0 && g < G) sm.score[g] = (c0 == 0 ? 0.0f : sm.score[g]) + dot;
+                        }
+                    }
+                }
+                pc_barrier();
+                // a2..a5, written where the producers of block lp will read it
+                PersistSel* sb = &P.sel[lp & 1];
+                select_block<kPC>(sm.sel, P.plan, G, sm.score, P.step0 + static_cast<uint32_t>(step_i),
+                                  static_cast<uint32_t>(lp), 0, nullptr, sb->dev_of_group, sb->arrived, nullptr,
+                                  sb->keep_list, &sb->n_keep, P.status, tid, ConsumerSync());
+                __threadfence();
+                pc_barrier();
+                if (tid == 0) st_release_gpu(sync_selready, n_pred);
+                // records (optional), after publication: off everybody's critical path
+                const size_t rec = static_cast<size_t>(step_i) * L + lp;
+                for (int g = tid; g < G; g += kPC) {
+                    if (P.tap_scores) P.tap_scores[rec * G + g] = sm.score[g];
+                    if (P.tap_keep_list) P.tap_keep_list[rec * G + g] = __ldcg(&sb->keep_list[g]);
+                    if (P.tap_dev_of_group) P.tap_dev_of_group[rec * G + g] = __ldcg(&sb->dev_of_group[g]);
+                }
+                if (tid < n_dev && P.tap_arrived) P.tap_arrived[rec * n_dev + tid] = static_cast<uint8_t>(sm.sel.arrived[tid]);
+                if (tid == 0 && P.tap_n_keep) P.tap_n_keep[rec] = __ldcg(&sb->n_keep);
+                if (P.trace && tid == 0 && n_pred - 1u < static_cast<unsigned>(P.trace_blocks))
+                    P.trace[(static_cast<size_t>(n_pred - 1u) * grid + cta) * 8 + TR_SELECT_NS] = global_timer_ns() - t_sel;
+                pc_barrier();   // sm.score / sm.sel are reused by the next selection
+            }
+        }
+        if (bad && tid == 0) {
+            atomicExch(sync_abort, 1u);
+            flag_status(P.status, HALO_DEV_TIMEOUT);
+        }
+        return;
+    }
 
     // =========================================== producer ===========================================
     if (warp == kPCWarps) {
@@ -175,8 +259,8 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 if (lane == 0) {
                     // (a) rows of the next block's predictor that this thread block owns
                     if (l + 1 < L) {
-                        const int r0 = static_cast<int>(static_cast<long long>(cta) * r / grid);
-                        const int r1 = static_cast<int>(static_cast<long long>(cta + 1) * r / grid);
+                        const int r0 = static_cast<int>(static_cast<long long>(cta) * r / workers);
+                        const int r1 = static_cast<int>(static_cast<long long>(cta + 1) * r / workers);
                         const __nv_bfloat16* W1 = P.W1[l + 1];
                         for (int row = r0; row < r1 && alive; row += ROWS) {
                             const int n = min(ROWS, r1 - row);
@@ -188,7 +272,6 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                                           n * row_bytes, &sm.full[s]);
                             ++it;
                         }
-                        if (alive && is_selector) alive = marker(ST_SELECT, l + 1);
                     }
                     // (b) the selection of this block must have been published
                     if (alive && l > 0) {
@@ -216,7 +299,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 // (c') keep HBM busy while the consumers synchronise: the block's first batches go to L2 now, long
                 //      before ring slots free up for them (whoever ends up consuming them)
                 if (lane < P.l2_ahead) {
-                    const long long b = cta + static_cast<long long>(grid) * lane;
+                    const long long b = cta + static_cast<long long>(workers) * lane;
                     if (b < U) {
                         const int ki = static_cast<int>(b / per_group), j0 = static_cast<int>(b - static_cast<long long>(ki) * per_group) * NB;
                         const int g = sm.kept_group[ki];
@@ -237,7 +320,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                     long long b = cta;
                     long long ahead[kFetchAhead];
 #pragma unroll
-                    for (int k = 0; k < kFetchAhead; ++k) ahead[k] = static_cast<long long>(grid) + atomicAdd(ctr, 1u);
+                    for (int k = 0; k < kFetchAhead; ++k) ahead[k] = static_cast<long long>(workers) + atomicAdd(ctr, 1u);
                     while (b < U) {
                         int s;
                         if (!acquire(s)) { alive = false; break; }
@@ -259,7 +342,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                         b = ahead[0];
 #pragma unroll
                         for (int k = 0; k + 1 < kFetchAhead; ++k) ahead[k] = ahead[k + 1];
-                        ahead[kFetchAhead - 1] = (b < U) ? static_cast<long long>(grid) + atomicAdd(ctr, 1u) : U;
+                        ahead[kFetchAhead - 1] = (b < U) ? static_cast<long long>(workers) + atomicAdd(ctr, 1u) : U;
                     }
                     if (alive) alive = marker(ST_END, 0);
                 }
@@ -387,7 +470,6 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 const int type = sm.type[s], a0 = sm.arg0[s], a1 = sm.arg1[s];
                 const unsigned char* stage = ring + static_cast<size_t>(s) * stage_bytes;
                 float* red = sm.red[red_par];
-                bool okz = true;
                 // ---- before the barrier: nothing in here may block on other consumers ----
                 if (type == ST_FFN) {
                     if (a0 >= 0) {
@@ -408,13 +490,8 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                         const float dot = warp_sum(dot0 + dot1);
                         if (lane == 0) red[row * WPR + part] = dot;
                     }
-                } else if (type == ST_SELECT) {
-                    if (tid == 0) {
-                        const unsigned n_pred = static_cast<unsigned>(step_i) * (L - 1) + a0;
-                        okz = spin_until_ge(sync_zcount, n_pred * static_cast<unsigned>(r), sync_abort);
-                    }
                 }
-                bad = pc_barrier_or(!ok || !okz);
+                bad = pc_barrier_or(!ok);
                 if (bad) break;
                 // ---- after the barrier ----
                 if (type == ST_FFN) {
@@ -435,72 +512,19 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                     red_par ^= 1;
                 } else if (type == ST_PRED) {
                     if (tid == 0) {
+                        // hidden values of the prediction made during this block, in the buffer of its parity
+                        const unsigned n_pred = static_cast<unsigned>(step_i) * (L - 1) + (l + 1);
+                        float* zdst = P.z + static_cast<size_t>(n_pred & 1u) * r;
                         for (int i = 0; i < a1; ++i) {
                             float z = 0.0f;
                             for (int w = 0; w < WPR; ++w) z += red[i * WPR + w];
                             if (P.act == HALO_ACT_RELU) z = fmaxf(z, 0.0f);
-                            P.z[a0 + i] = z;
+                            zdst[a0 + i] = z;
                         }
                         __threadfence();
                         atomicAdd(sync_zcount, static_cast<unsigned>(a1));
                     }
                     red_par ^= 1;
-                } else if (type == ST_SELECT) {
-                    // a1 (second layer): s[g] = <W2[g], z>; then a2..a5 for block a0, published for the producers
-                    const unsigned long long t_sel = (P.trace && tid == 0) ? global_timer_ns() : 0ull;
-                    const int lp = a0;
-                    const __nv_bfloat16* W2 = P.W2[lp];
-                    const int zc = r >> 3;  // 16-byte chunks per W2 row
-                    for (int c0 = 0; c0 < zc; c0 += 32) {
-                        const int c = c0 + lane;
-                        float zv[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-                        if (c < zc) {
-                            const float4 z0 = __ldcg(reinterpret_cast<const float4*>(P.z) + 2 * c);
-                            const float4 z1 = __ldcg(reinterpret_cast<const float4*>(P.z) + 2 * c + 1);
-                            zv[0] = z0.x; zv[1] = z0.y; zv[2] = z0.z; zv[3] = z0.w;
-                            zv[4] = z1.x; zv[5] = z1.y; zv[6] = z1.z; zv[7] = z1.w;
-                        }
-                        // groups warp, warp+16, ...: all row loads of a pass are issued before any is used
-                        for (int g0 = warp; g0 < G; g0 += kPCWarps * 4) {
-                            uint4 wv[4];
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                const int g = g0 + u * kPCWarps;
-                                wv[u] = (g < G && c < zc) ? __ldg(reinterpret_cast<const uint4*>(W2 + static_cast<size_t>(g) * r) + c)
-                                                          : make_uint4(0, 0, 0, 0);
-                            }
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                const int g = g0 + u * kPCWarps;
-                                float w8[8];
-                                Elem<__nv_bfloat16>::widen(wv[u], w8);
-                                float dot = 0.0f;
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) dot = fmaf(w8[e], zv[e], dot);
-                                dot = warp_sum(dot);
-                                if (lane == 0 && g < G) sm.score[g] = (c0 == 0 ? 0.0f : sm.score[g]) + dot;
-                            }
-                        }
-                    }
-                    pc_barrier();
-                    PersistSel* sb = &P.sel[lp & 1];
-                    select_block<kPC>(sm.sel, P.plan, G, sm.score, P.step0 + static_cast<uint32_t>(step_i),
-                                      static_cast<uint32_t>(lp), 0, nullptr, sb->dev_of_group, sb->arrived, nullptr,
-                                      sb->keep_list, &sb->n_keep, P.status, tid, ConsumerSync());
-                    __threadfence();
-                    pc_barrier();
-                    const size_t rec = static_cast<size_t>(step_i) * L + lp;
-                    for (int g = tid; g < G; g += kPC) {
-                        if (P.tap_scores) P.tap_scores[rec * G + g] = sm.score[g];
-                        if (P.tap_keep_list) P.tap_keep_list[rec * G + g] = __ldcg(&sb->keep_list[g]);
-                        if (P.tap_dev_of_group) P.tap_dev_of_group[rec * G + g] = __ldcg(&sb->dev_of_group[g]);
-                    }
-                    if (tid < n_dev && P.tap_arrived) P.tap_arrived[rec * n_dev + tid] = static_cast<uint8_t>(sm.sel.arrived[tid]);
-                    if (tid == 0) {
-                        if (P.tap_n_keep) P.tap_n_keep[rec] = __ldcg(&sb->n_keep);
-                        st_release_gpu(sync_selready, static_cast<unsigned>(step_i) * (L - 1) + lp);
-                        if (P.trace) trace(TR_SELECT_NS, global_timer_ns() - t_sel);
-                    }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm.empty[s]);
@@ -529,7 +553,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 // idle now: its last user finished 8 blocks ago and its next user cannot have started.
                 if (cta == 0) P.sync[16 + ((q + 8u) & 15u)] = 0u;
                 __threadfence();
-                const unsigned target = (q + 1u) * static_cast<unsigned>(grid);
+                const unsigned target = (q + 1u) * static_cast<unsigned>(workers);
                 const unsigned before = atomicAdd(sync_barrier, 1u);
                 okb = (before + 1u == target) || spin_until_ge(sync_barrier, target, sync_abort);
                 __threadfence();

@@ -22,7 +22,7 @@ struct PersistParams {
     const float* h0;                       // [steps][d]
     float* h_out;                          // [steps][d]
     float* partials;                       // [3][2][d] rotating interleaved accumulation buffers, zero at launch
-    float* z;                              // [r]
+    float* z;                              // [2][r]: hidden values, by parity of the prediction
     PersistSel* sel;                       // [3]: two rotating + the static first-block selection
     unsigned* sync;                        // [32]: 0 barrier count, 1 abort, 2 hidden rows done, 3 selections
                                            //       published, 16..31 rotating batch counters; zero at launch

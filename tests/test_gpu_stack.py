@@ -144,3 +144,43 @@ def test_stack_multi_token_prompt():
     stack, Wp, preds = build_stack(wl)
     h0, h_out, t = run_with_taps(wl, stack, 1)
     check_teacher_forced(wl, Wp, preds, h0, h_out, t, 1)
+
+
+@pytest.mark.parametrize("name,steps,sample", [
+    ("llama2-7b-decode", 3, [(0, 0), (0, 1), (1, 16), (2, 30), (2, 31)]),
+    ("llama2-13b-decode", 2, [(0, 1), (1, 20), (1, 39)]),
+    ("tinyllama-1.1b-decode", 4, [(0, 0), (1, 1), (2, 11), (3, 21)]),
+])
+def test_full_size_stack_in_bench_configuration_sampled_blocks(name, steps, sample):
+    """The whole stack at its stated size, run the way bench.py times it (one persistent launch); the oracle
+    recomputes a sample of (step, block) records from the recorded inputs.  Selection integers are checked for
+    every record (they are cheap), FFN outputs for the sample."""
+    wl = synth.workload(name)
+    stack, Wp, preds = build_stack(wl)
+    h0, h_out, t = run_with_taps(wl, stack, steps, step0=7)
+    assert stack.last_launches() == 1
+    hb = synth.host_bits
+    x_all = hb(t["x"])
+    n = wl.n_dev
+    scores_all = t["scores"].cpu().numpy()
+    kl_all, dg_all, nk_all = t["keep_list"].cpu().numpy(), t["dev_of_group"].cpu().numpy(), t["n_keep"].cpu().numpy()
+    arr_all = t["arrived"].cpu().numpy()
+    for s in range(steps):
+        for l in range(wl.n_layers):
+            sel = R.select(scores_all[s, l], wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed,
+                           7 + s, l, force_all=(l == 0))
+            assert int(nk_all[s, l]) == sel["n_keep"], (s, l)
+            assert (kl_all[s, l] == sel["keep_list"]).all() and (dg_all[s, l] == sel["dev_of_group"]).all()
+            assert (arr_all[s, l, :n] == sel["arrived"]).all()
+    for s, l in sample:
+        if l > 0:
+            s_ref = R.predict(hb(preds[l][0]), hb(preds[l][1]), x_all[s, l - 1])
+            assert U.rel_err(scores_all[s, l], s_ref.astype(np.float64)) <= U.TOL_BF16
+        nk = int(nk_all[s, l])
+        P = R.group_ffn(hb(Wp[l]), x_all[s, l], kl_all[s, l][:nk], dg_all[s, l], n)
+        y_ref = R.merge(P)
+        assert U.rel_err(t["y"][s, l].cpu().numpy(), y_ref) <= U.TOL_BF16, (s, l)
+    # the residual stream that comes out is the input plus every block's recorded output
+    for s in range(steps):
+        want = h0[s].double() + t["y"][s].double().sum(dim=0)
+        assert (h_out[s].double() - want).abs().max().item() <= 1e-3 * want.abs().max().item()

@@ -28,6 +28,10 @@ from paper_2601_11676_b200 import synth  # noqa: E402
 
 METRIC = "group-sparse FFN decode tokens/s on 1 B200; achieved HBM GB/s vs ~8 TB/s"
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read+write per launch / algorithmic bytes per launch of stack_decode_kernel, from the ncu capture in
+# profiles/stack_decode_kernel_llama2-7b_4blocks.md (4-block case; traffic is proportional to the kept groups
+# processed, so the ratio carries over to the full-size launch).  Set to None when the kernel changes.
+STACK_KERNEL_TRAFFIC_RATIO = 1.0003
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -248,7 +252,9 @@ def run_halo(args, rank, world, local_rank):
         result["roofline"] = {
             "bound": "hbm", "kernel": "stack_decode_kernel (persistent: all steps x blocks, a1..a9 + glue)",
             "achieved": step_gbs, "peak": peak, "unit": "GB/s", "frac": step_gbs / peak, "peak_kind": peak_kind,
-            "traffic": None, "avg_launch_us": ms * 1e3, "launches_timed": 1,
+            "traffic": (algo_bytes_total * STACK_KERNEL_TRAFFIC_RATIO) if STACK_KERNEL_TRAFFIC_RATIO else None,
+            "traffic_note": "ncu DRAM bytes of a 4-block capture scaled by kept groups processed",
+            "avg_launch_us": ms * 1e3, "launches_timed": 1,
             "algorithmic_bytes_per_launch": algo_bytes_total, "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS}
     else:
         result["roofline"] = {

@@ -115,6 +115,31 @@ halo_status halo_plan_describe(const halo_plan* plan, int M, int32_t* dev_order,
                                int32_t* boundaries);
 
 /* ------------------------------------------------------------------------
+ * Assignment phase, step 1: workload ratios from the devices' memory budgets
+ * m_i and computing power c_i (Sec. III-B.4, PLR-aware load-balancing
+ * scheduler).  Host only.  All arrays are host arrays of n_dev entries;
+ * model_mem is the model's total memory demand in the unit of mem_budget.
+ *   halo_schedule_comp_greedy (Algorithm 1): devices in descending computing
+ *     power (ties: lower index) are filled to their budget until the model
+ *     fits; the last one needed takes the remainder; unused devices get 0.
+ *   halo_schedule_min_max (Algorithm 2): bisection (to eps; the paper uses
+ *     1e-3) on the utilisation threshold T; u_i = min(m_i, T*c_i) with the
+ *     smallest T whose allocation holds the model; minimises the slowest
+ *     device's time.
+ *   Both return ratio[i] = u_i / sum(u) (sum = 1).
+ *   halo_ratios_to_share_weights: integer weights round(ratio * 65536) for
+ *     halo_plan_create (zero-ratio devices get empty chunks).
+ * HALO_ERR_ARG: NULL pointers, n_dev outside [1, HALO_MAX_DEVICES], a
+ * negative budget, non-positive computing power or eps, or budgets that
+ * cannot hold the model.
+ * ---------------------------------------------------------------------- */
+halo_status halo_schedule_comp_greedy(int n_dev, const double* mem_budget, const double* compute,
+                                      double model_mem, double* ratio);
+halo_status halo_schedule_min_max(int n_dev, const double* mem_budget, const double* compute, double model_mem,
+                                  double eps, double* ratio);
+halo_status halo_ratios_to_share_weights(int n_dev, const double* ratio, uint32_t* share_weight);
+
+/* ------------------------------------------------------------------------
  * a1. Predictor (Sec. III-B.2, semantic-aware predictors): importance score
  * of every neuron group of a block from semantic features taken one layer
  * ahead.  Bias-free two-layer network

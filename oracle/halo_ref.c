@@ -423,3 +423,59 @@ int halo_ref_layer(int d, int F, int S, int dtype, const void* Wpacked, int rank
     free(P);
     return rc;
 }
+
+/* ---- Assignment phase, step 1: workload ratios (Algorithms 1 and 2) ------ */
+/* Algorithm 1, Computation-Greedy: devices in descending computing power are
+ * filled to their memory budget until the model fits; the last device needed
+ * takes the remainder, the others get nothing.  r = u / sum(u).  Ties in c
+ * keep the lower device index first. */
+int halo_ref_comp_greedy(int n, const double* m, const double* c, double Mt, double* r) {
+    if (n <= 0 || !(Mt > 0.0)) return REF_ERR_ARG;
+    double total = 0.0;
+    for (int i = 0; i < n; ++i) { if (!(m[i] >= 0.0) || !(c[i] > 0.0)) return REF_ERR_ARG; total += m[i]; }
+    if (total < Mt) return REF_ERR_ARG;   /* the model does not fit at all */
+    int* sigma = (int*)malloc(sizeof(int) * (size_t)n);
+    if (!sigma) return REF_ERR_NOMEM;
+    for (int i = 0; i < n; ++i) sigma[i] = i;
+    for (int a = 1; a < n; ++a) {          /* stable insertion sort, descending c */
+        int v = sigma[a], b = a - 1;
+        while (b >= 0 && c[sigma[b]] < c[v]) { sigma[b + 1] = sigma[b]; --b; }
+        sigma[b + 1] = v;
+    }
+    for (int i = 0; i < n; ++i) r[i] = 0.0;
+    double placed = 0.0, sum_u = 0.0;
+    for (int j = 0; j < n; ++j) {
+        int i = sigma[j];
+        double u = m[i];
+        if (placed + u >= Mt) { u = Mt - placed; r[i] = u; sum_u += u; break; }
+        r[i] = u; sum_u += u; placed += u;
+    }
+    for (int i = 0; i < n; ++i) r[i] /= sum_u;
+    free(sigma);
+    return REF_OK;
+}
+
+/* Algorithm 2, Min-Max: bisection on the utilisation threshold T (memory per
+ * unit of computing power): u_i = min(m_i, T c_i); the smallest T (to eps)
+ * whose allocation holds the model; r = u / sum(u). */
+int halo_ref_min_max(int n, const double* m, const double* c, double Mt, double eps, double* r) {
+    if (n <= 0 || !(Mt > 0.0) || !(eps > 0.0)) return REF_ERR_ARG;
+    double total = 0.0, mmax = 0.0, cmin = 0.0;
+    for (int i = 0; i < n; ++i) {
+        if (!(m[i] >= 0.0) || !(c[i] > 0.0)) return REF_ERR_ARG;
+        total += m[i];
+        if (i == 0 || m[i] > mmax) mmax = m[i];
+        if (i == 0 || c[i] < cmin) cmin = c[i];
+    }
+    if (total < Mt) return REF_ERR_ARG;
+    double left = 0.0, right = mmax / cmin, t_opt = right;
+    while (right - left > eps) {
+        double mid = (left + right) / 2.0, used = 0.0;
+        for (int i = 0; i < n; ++i) used += (m[i] < mid * c[i]) ? m[i] : mid * c[i];
+        if (used >= Mt) { t_opt = mid; right = mid; } else left = mid;
+    }
+    double sum_u = 0.0;
+    for (int i = 0; i < n; ++i) { r[i] = (m[i] < t_opt * c[i]) ? m[i] : t_opt * c[i]; sum_u += r[i]; }
+    for (int i = 0; i < n; ++i) r[i] /= sum_u;
+    return REF_OK;
+}

@@ -268,3 +268,19 @@ def layer(Wpacked, W1, W2, feat, x, loss_rate, share_weight, mode, k_critical, t
                                 _p(y)), "layer")
     return dict(scores=scores, order=order, rank=rank, dev_of_group=dev, arrived=arrived[:n].copy(), keep=keep,
                 keep_list=keep_list, n_keep=int(n_keep[0]), status=int(status[0]), y=y)
+
+
+# --- Algorithms 1 and 2: workload ratios ---------------------------------------------
+
+def comp_greedy(m, c, Mt: float) -> np.ndarray:
+    m = np.asarray(m, dtype=np.float64); c = np.asarray(c, dtype=np.float64)
+    r = np.empty(len(m), dtype=np.float64)
+    _check(lib().halo_ref_comp_greedy(c_int(len(m)), _p(m), _p(c), c_double(Mt), _p(r)), "comp_greedy")
+    return r
+
+
+def min_max(m, c, Mt: float, eps: float = 1e-3) -> np.ndarray:
+    m = np.asarray(m, dtype=np.float64); c = np.asarray(c, dtype=np.float64)
+    r = np.empty(len(m), dtype=np.float64)
+    _check(lib().halo_ref_min_max(c_int(len(m)), _p(m), _p(c), c_double(Mt), c_double(eps), _p(r)), "min_max")
+    return r

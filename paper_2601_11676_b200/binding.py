@@ -28,6 +28,7 @@ EXPORTS = [
     "halo_group_ffn", "halo_merge_partials", "halo_pack_weights", "halo_glue", "halo_stack_create",
     "halo_stack_destroy", "halo_stack_decode", "halo_stack_decode_host", "halo_stack_status",
     "halo_stack_last_launches", "halo_stack_set_mode", "halo_stack_set_trace", "halo_stack_trace_width",
+    "halo_schedule_comp_greedy", "halo_schedule_min_max", "halo_ratios_to_share_weights",
 ]
 
 
@@ -93,6 +94,10 @@ def lib() -> ctypes.CDLL:
         L.halo_stack_set_trace.argtypes = [c_void_p, c_void_p, c_int]
         L.halo_stack_trace_width.argtypes = [c_void_p]
         L.halo_stack_trace_width.restype = c_int
+        L.halo_schedule_comp_greedy.argtypes = [c_int, POINTER(c_double), POINTER(c_double), c_double, POINTER(c_double)]
+        L.halo_schedule_min_max.argtypes = [c_int, POINTER(c_double), POINTER(c_double), c_double, c_double,
+                                            POINTER(c_double)]
+        L.halo_ratios_to_share_weights.argtypes = [c_int, POINTER(c_double), POINTER(c_uint32)]
         L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
         _lib = L
     return _lib
@@ -171,6 +176,33 @@ class Plan:
             self.close()
         except Exception:
             pass
+
+
+def _darr(v):
+    return (c_double * len(v))(*[float(x) for x in v])
+
+
+def halo_schedule_comp_greedy(mem_budget, compute, model_mem):
+    n = len(mem_budget)
+    out = (c_double * n)()
+    _chk(lib().halo_schedule_comp_greedy(n, _darr(mem_budget), _darr(compute), float(model_mem), out),
+         "halo_schedule_comp_greedy")
+    return list(out)
+
+
+def halo_schedule_min_max(mem_budget, compute, model_mem, eps=1e-3):
+    n = len(mem_budget)
+    out = (c_double * n)()
+    _chk(lib().halo_schedule_min_max(n, _darr(mem_budget), _darr(compute), float(model_mem), float(eps), out),
+         "halo_schedule_min_max")
+    return list(out)
+
+
+def halo_ratios_to_share_weights(ratio):
+    n = len(ratio)
+    out = (c_uint32 * n)()
+    _chk(lib().halo_ratios_to_share_weights(n, _darr(ratio), out), "halo_ratios_to_share_weights")
+    return list(out)
 
 
 def halo_predict_workspace_bytes(shape: PredShape, n_tok: int) -> int:

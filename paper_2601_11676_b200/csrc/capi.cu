@@ -151,6 +151,71 @@ extern "C" halo_status halo_plan_describe(const halo_plan* plan, int M, int32_t*
     return HALO_OK;
 }
 
+// ---- Assignment phase, workload ratios (Algorithms 1 and 2) -----------------------------------------------
+
+namespace {
+bool valid_devices(int n, const double* m, const double* c, double Mt, double* total) {
+    if (n <= 0 || n > HALO_MAX_DEVICES || !m || !c || !(Mt > 0.0)) return false;
+    double t = 0.0;
+    for (int i = 0; i < n; ++i) {
+        if (!(m[i] >= 0.0) || !(c[i] > 0.0)) return false;
+        t += m[i];
+    }
+    *total = t;
+    return t >= Mt;   // the budgets must hold the model
+}
+}  // namespace
+
+extern "C" halo_status halo_schedule_comp_greedy(int n_dev, const double* mem_budget, const double* compute,
+                                                 double model_mem, double* ratio) {
+    double total;
+    if (!ratio || !valid_devices(n_dev, mem_budget, compute, model_mem, &total)) return HALO_ERR_ARG;
+    int order[HALO_MAX_DEVICES];
+    for (int i = 0; i < n_dev; ++i) order[i] = i;
+    std::stable_sort(order, order + n_dev, [&](int a, int b) { return compute[a] > compute[b]; });
+    double used[HALO_MAX_DEVICES] = {};
+    double remaining = model_mem, sum = 0.0;
+    for (int j = 0; j < n_dev && remaining > 0.0; ++j) {
+        const int i = order[j];
+        const double take = std::min(mem_budget[i], remaining);   // the last device needed takes the remainder
+        used[i] = take;
+        sum += take;
+        remaining -= take;
+    }
+    for (int i = 0; i < n_dev; ++i) ratio[i] = used[i] / sum;
+    return HALO_OK;
+}
+
+extern "C" halo_status halo_schedule_min_max(int n_dev, const double* mem_budget, const double* compute,
+                                             double model_mem, double eps, double* ratio) {
+    double total;
+    if (!ratio || !(eps > 0.0) || !valid_devices(n_dev, mem_budget, compute, model_mem, &total)) return HALO_ERR_ARG;
+    auto held = [&](double T) {
+        double s = 0.0;
+        for (int i = 0; i < n_dev; ++i) s += std::min(mem_budget[i], T * compute[i]);
+        return s;
+    };
+    double lo = 0.0;
+    double hi = *std::max_element(mem_budget, mem_budget + n_dev) / *std::min_element(compute, compute + n_dev);
+    double best = hi;
+    while (hi - lo > eps) {
+        const double mid = 0.5 * (lo + hi);
+        if (held(mid) >= model_mem) { best = mid; hi = mid; } else lo = mid;
+    }
+    const double sum = held(best);
+    for (int i = 0; i < n_dev; ++i) ratio[i] = std::min(mem_budget[i], best * compute[i]) / sum;
+    return HALO_OK;
+}
+
+extern "C" halo_status halo_ratios_to_share_weights(int n_dev, const double* ratio, uint32_t* share_weight) {
+    if (n_dev <= 0 || n_dev > HALO_MAX_DEVICES || !ratio || !share_weight) return HALO_ERR_ARG;
+    for (int i = 0; i < n_dev; ++i) {
+        if (!(ratio[i] >= 0.0) || ratio[i] > 65535.0) return HALO_ERR_ARG;
+        share_weight[i] = static_cast<uint32_t>(std::floor(ratio[i] * 65536.0 + 0.5));
+    }
+    return HALO_OK;
+}
+
 // ---- a1 ---------------------------------------------------------------------------------------------
 
 extern "C" size_t halo_predict_workspace_bytes(const halo_pred_shape* shape, int n_tok) {

@@ -97,3 +97,26 @@ def test_host_side_argument_checks_launch_nothing(lib):
     assert rc == -8  # workspace too small
     assert lib.halo_merge_partials(None, None, 1, 1, 8, None, None) == -1
     assert lib.halo_select_groups(None, None, 0, 0, 0, None, None, None, None, None, None, None, None) == -1
+
+
+def test_schedulers_match_oracle_and_feed_the_plan(lib):
+    rng = np.random.default_rng(3)
+    for _ in range(200):
+        n = int(rng.integers(1, 9))
+        m = rng.uniform(0.3, 6.3, n).round(1)
+        c = rng.uniform(0.6, 1.8, n).round(1)
+        Mt = float(rng.uniform(0.2, 1.0) * m.sum())
+        assert np.allclose(B.halo_schedule_comp_greedy(m, c, Mt), R.comp_greedy(m, c, Mt), atol=1e-12)
+        assert np.allclose(B.halo_schedule_min_max(m, c, Mt, 1e-3), R.min_max(m, c, Mt, 1e-3), atol=1e-12)
+    # ratios -> integer share weights -> Algorithm 3: a device with ratio 0 gets an empty chunk
+    r = B.halo_schedule_comp_greedy([4, 5, 3], [2.0, 1.0, 3.0], 6.0)
+    w = B.halo_ratios_to_share_weights(r)
+    assert w == [32768, 0, 32768]
+    plan = B.Plan(20, [0.1, 0.0, 0.3], w, B.SEL_TOPK, 4, 0.0, 0)
+    order, _, bnd = plan.describe(16)
+    assert order == [1, 0, 2] and bnd == [0, 0, 8, 16]
+    for bad in [([1, 1], [1.0, 1.0], 3.0), ([1, -1], [1.0, 1.0], 0.5), ([1, 1], [1.0, 0.0], 0.5)]:
+        with pytest.raises(B.HaloError):
+            B.halo_schedule_min_max(*bad)
+        with pytest.raises(B.HaloError):
+            B.halo_schedule_comp_greedy(*bad)

@@ -298,6 +298,16 @@ halo_status halo_stack_set_mode(halo_stack* stack, int mode);
  * 6 next input ready; 7 = duration of the selection (selecting thread block only).  n_blocks = 0 turns it off. */
 halo_status halo_stack_set_trace(halo_stack* stack, unsigned long long* trace /*device*/, int n_blocks);
 int halo_stack_trace_width(const halo_stack* stack);
+/* Failure detection self-test.  Every device-side wait of this library (mbarrier phases of the copy rings, the
+ * grid barrier, the published-selection flag) is bounded; when one runs out the kernel raises HALO_DEV_TIMEOUT
+ * and returns, so a late or missing partner shows up as a status bit, never as a hung GPU (the paper's master
+ * likewise proceeds after its receive timeout, Sec. III-B.3).  This call exercises that mechanism harmlessly:
+ * one thread block waits, for at most limit_cycles SM cycles each (1 .. 2e9), on an mbarrier phase nobody
+ * completes and on the device word never_set_flag (which the caller leaves at 0).  On return (after
+ * synchronising) report[0] = number of threads whose mbarrier wait ran out (128), report[1] = 1 if the flag wait
+ * ran out, and HALO_DEV_TIMEOUT is set in *dev_status.  All pointers are device pointers. */
+halo_status halo_selftest_bounded_wait(const uint32_t* never_set_flag, long long limit_cycles, uint32_t* report,
+                                       uint32_t* dev_status, void* stream);
 /* Device status word accumulated by the stack's launches (synchronises the stream). */
 halo_status halo_stack_status(halo_stack* stack, uint32_t* dev_status_value /*host*/, void* stream);
 /* Number of kernel launches the last halo_stack_decode enqueued. */

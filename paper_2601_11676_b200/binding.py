@@ -29,6 +29,7 @@ EXPORTS = [
     "halo_stack_destroy", "halo_stack_decode", "halo_stack_decode_host", "halo_stack_status",
     "halo_stack_last_launches", "halo_stack_set_mode", "halo_stack_set_trace", "halo_stack_trace_width",
     "halo_schedule_comp_greedy", "halo_schedule_min_max", "halo_ratios_to_share_weights",
+    "halo_selftest_bounded_wait",
 ]
 
 
@@ -98,6 +99,7 @@ def lib() -> ctypes.CDLL:
         L.halo_schedule_min_max.argtypes = [c_int, POINTER(c_double), POINTER(c_double), c_double, c_double,
                                             POINTER(c_double)]
         L.halo_ratios_to_share_weights.argtypes = [c_int, POINTER(c_double), POINTER(c_uint32)]
+        L.halo_selftest_bounded_wait.argtypes = [c_void_p, c_longlong, c_void_p, c_void_p, c_void_p]
         L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
         _lib = L
     return _lib
@@ -203,6 +205,11 @@ def halo_ratios_to_share_weights(ratio):
     out = (c_uint32 * n)()
     _chk(lib().halo_ratios_to_share_weights(n, _darr(ratio), out), "halo_ratios_to_share_weights")
     return list(out)
+
+
+def halo_selftest_bounded_wait(never_set_flag, limit_cycles, report, dev_status, stream=None) -> None:
+    _chk(lib().halo_selftest_bounded_wait(_ptr(never_set_flag), int(limit_cycles), _ptr(report), _ptr(dev_status),
+                                          _stream(stream)), "halo_selftest_bounded_wait")
 
 
 def halo_predict_workspace_bytes(shape: PredShape, n_tok: int) -> int:

@@ -159,27 +159,29 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 // ------------------------------------------------------------------------------------------------------------
 // GEMM-2: down projection of the kept columns, one accumulation per holder slot
 // ------------------------------------------------------------------------------------------------------------
-constexpr int kBN2 = 128;   // output columns per tile
-
 struct DownSmemTail {
     PfBarriers bars;
+    int slot_lo, slot_hi;                 // holder slots this CTA accumulates (the K range is split by slot)
     int slot_start[HALO_MAX_DEVICES + 2];
     int32_t group_of[HALO_MAX_GROUPS];    // group id per position of the slot-sorted order (-1 = skip)
     int16_t kept_pos[HALO_MAX_GROUPS];    // kept position (column block of H) per position of the order
 };
 
-template <int STAGES>
+// BN2 output columns per tile.  gridDim.z CTAs share an output tile position but take disjoint ranges of holder
+// slots: the slots are separate outputs, so splitting K at a slot boundary needs no reduction.
+template <int BN2, int STAGES>
 __global__ void __launch_bounds__(kPfThreads, 1)
 ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_wd, int T, int d,
                 int S, int G, const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
                 const int32_t* __restrict__ dev_of_group, int n_dev, float* __restrict__ partials,
                 uint32_t* dev_status) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = kBK * kBN2 * 2, kStageBytes = kABytes + kBBytes;
+    constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = kBK * BN2 * 2, kStageBytes = kABytes + kBBytes;
+    constexpr uint32_t kBBlock = kBK * 64 * 2;   // one 64-column block of B: 64 K-rows x 128 B
     DownSmemTail& tail = *reinterpret_cast<DownSmemTail*>(smem_raw + static_cast<size_t>(STAGES) * kStageBytes);
     PfBarriers& bars = tail.bars;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * kBN2;
+    const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * BN2;
     int nk = *n_keep_ptr;
     nk = max(0, min(nk, G));
     const int k_per_group = S / kBK;   // K stages per kept group
@@ -194,7 +196,7 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
         tma_prefetch_descriptor(&tmap_h);
         tma_prefetch_descriptor(&tmap_wd);
     }
-    if (warp == 1) { tmem_alloc(&bars.tmem_base, kBN2); tmem_relinquish_alloc_permit(); }
+    if (warp == 1) { tmem_alloc(&bars.tmem_base, BN2); tmem_relinquish_alloc_permit(); }
     if (warp == 0) {
         // kept positions sorted by holder slot (stable): one warp, ballot compaction per slot
         int pos = 0;
@@ -218,20 +220,34 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
                 pos += __popc(ballot);
             }
         }
-        if (lane == 0) tail.slot_start[n_slots] = pos;
+        if (lane == 0) {
+            tail.slot_start[n_slots] = pos;
+            // this CTA's share of the slots: cut at the slot boundary nearest to half of the kept groups
+            int lo = 0, hi = n_slots;
+            if (gridDim.z == 2) {
+                int cut = n_slots, best = pos + 1;
+                for (int sl = 1; sl < n_slots; ++sl) {
+                    const int dist = abs(2 * tail.slot_start[sl] - pos);
+                    if (dist < best) { best = dist; cut = sl; }
+                }
+                if (blockIdx.z == 0) hi = cut; else lo = cut;
+            }
+            tail.slot_lo = lo;
+            tail.slot_hi = hi;
+        }
     }
     tcgen05_fence_before_sync();
     __syncthreads();
     tcgen05_fence_after_sync();
     volatile int* abort_flag = &bars.abort_flag;
     const uint32_t tmem = bars.tmem_base;
+    const int slot_lo = tail.slot_lo, slot_hi = tail.slot_hi;
 
     if (warp == 0) {
         if (lane == 0) {
             int it = 0;
             bool alive = true;
-            const int total = tail.slot_start[n_slots];
-            for (int p = 0; p < total && alive; ++p) {
+            for (int p = tail.slot_start[slot_lo]; p < tail.slot_start[slot_hi] && alive; ++p) {
                 const int g = tail.group_of[p], kp = tail.kept_pos[p];
                 for (int kk2 = 0; kk2 < k_per_group; ++kk2, ++it) {
                     const int s = it % STAGES;
@@ -240,8 +256,9 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
                     mbar_arrive_expect_tx(&bars.full[s], kStageBytes);
                     tma_load_2d(st, &tmap_h, kp * S + kk2 * kBK, m0, &bars.full[s]);
                     const int krow = (g * 3 + 2) * S + kk2 * kBK;
-                    tma_load_2d(st + kABytes, &tmap_wd, n0, krow, &bars.full[s]);
-                    tma_load_2d(st + kABytes + kBBytes / 2, &tmap_wd, n0 + 64, krow, &bars.full[s]);
+#pragma unroll
+                    for (int nb = 0; nb < BN2 / 64; ++nb)
+                        tma_load_2d(st + kABytes + nb * kBBlock, &tmap_wd, n0 + nb * 64, krow, &bars.full[s]);
                 }
             }
             if (*abort_flag) {
@@ -252,10 +269,10 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(kBM, kBN2, true);
+            constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN2, true);
             int it = 0, used = 0;
             bool alive = true;
-            for (int slot = 0; slot < n_slots && alive; ++slot) {
+            for (int slot = slot_lo; slot < slot_hi && alive; ++slot) {
                 const int p0 = tail.slot_start[slot], p1 = tail.slot_start[slot + 1];
                 if (p0 == p1) continue;
                 if (used > 0 && !pf_wait(&bars.tmem_empty, (used - 1) & 1, abort_flag)) break;  // epilogue has drained D
@@ -269,8 +286,8 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
 #pragma unroll
                     for (int kk = 0; kk < kBK / kUmmaK; ++kk) {
                         const uint64_t a = umma_smem_desc(a0 + kk * 32, 16, 1024);
-                        // MN-major B: 16 K-rows per MMA = 2 KiB further; 64-column blocks are kBBytes/2 apart
-                        const uint64_t b = umma_smem_desc(a0 + kABytes + kk * 2048, kBBytes / 2, 1024);
+                        // MN-major B: 16 K-rows per MMA = 2 KiB further; 64-column blocks are kBBlock apart
+                        const uint64_t b = umma_smem_desc(a0 + kABytes + kk * 2048, kBBlock, 1024);
                         umma_bf16(tmem, a, b, idesc, (k > 0) || (kk > 0));
                     }
                     umma_commit(&bars.empty[s]);
@@ -285,12 +302,12 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
         const int row = m0 + quad * 32 + lane;
         const uint32_t lane_base = tmem + (static_cast<uint32_t>(quad * 32) << 16);
         int used = 0;
-        for (int slot = 0; slot < n_slots; ++slot) {
+        for (int slot = slot_lo; slot < slot_hi; ++slot) {
             if (tail.slot_start[slot] == tail.slot_start[slot + 1]) continue;
             const bool ok = pf_wait(&bars.tmem_full, used & 1, abort_flag);
             tcgen05_fence_after_sync();
             float* out = partials + (static_cast<size_t>(slot) * T + row) * d + n0;
-            for (int c0 = 0; c0 < kBN2; c0 += 32) {
+            for (int c0 = 0; c0 < BN2; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32x32(lane_base + c0, v);
                 tmem_ld_wait();
@@ -310,7 +327,7 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
     }
     tcgen05_fence_before_sync();
     __syncthreads();
-    if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, kBN2); }
+    if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, BN2); }
     if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
 }
 
@@ -474,8 +491,7 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         !make_map(&map_h, H, T, sh.d_ffn, sh.d_ffn, kBK, kBM) || !make_map(&map_wd, W, w_rows, d, d, 64, kBK))
         return HALO_ERR_CUDA;
     const dim3 grid1((T + kBM - 1) / kBM, G);
-    const dim3 grid2((T + kBM - 1) / kBM, d / kBN2);
-    constexpr int kStages1 = 4, kStages2 = 6;
+    constexpr int kStages1 = 4;
     if (S == 128) {
         auto k1 = ffn_hidden_kernel<128, kStages1>;
         const size_t smem1 = static_cast<size_t>(kStages1) * (kBM * kBK * 2 + 2 * 128 * kBK * 2) + sizeof(PfBarriers) + 1024;
@@ -490,12 +506,26 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         k1<<<grid1, kPfThreads, smem1, st>>>(map_x, map_w, T, d, S, G, keep_list, n_keep, H, sh.d_ffn, dev_status);
     }
     HALO_CHECK_LAUNCH();
-    auto k2 = ffn_down_kernel<kStages2>;
-    const size_t smem2 = static_cast<size_t>(kStages2) * (kBM * kBK * 2 + kBK * kBN2 * 2) + sizeof(DownSmemTail) + 1024;
-    static bool once2 = false;
-    if (!once2) { if (!set_smem(k2, smem2)) return HALO_ERR_CUDA; once2 = true; }
-    k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, partials,
-                                         dev_status);
+    if (d % 256 == 0) {
+        // 256-column tiles (more FLOP per staged byte); with holder slots the K range is split over two CTAs
+        constexpr int kStages2 = 4;
+        auto k2 = ffn_down_kernel<256, kStages2>;
+        const size_t smem2 = static_cast<size_t>(kStages2) * (kBM * kBK * 2 + kBK * 256 * 2) + sizeof(DownSmemTail) + 1024;
+        static bool once2 = false;
+        if (!once2) { if (!set_smem(k2, smem2)) return HALO_ERR_CUDA; once2 = true; }
+        const dim3 grid2((T + kBM - 1) / kBM, d / 256, n_dev > 0 ? 2 : 1);
+        k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, partials,
+                                             dev_status);
+    } else {
+        constexpr int kStages2 = 6;
+        auto k2 = ffn_down_kernel<128, kStages2>;
+        const size_t smem2 = static_cast<size_t>(kStages2) * (kBM * kBK * 2 + kBK * 128 * 2) + sizeof(DownSmemTail) + 1024;
+        static bool once2 = false;
+        if (!once2) { if (!set_smem(k2, smem2)) return HALO_ERR_CUDA; once2 = true; }
+        const dim3 grid2((T + kBM - 1) / kBM, d / 128, 1);
+        k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, partials,
+                                             dev_status);
+    }
     HALO_CHECK_LAUNCH();
     return HALO_OK;
 }

@@ -32,7 +32,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Waits for the phase with the given parity, at most kWaitLimitCycles; also gives up early when *give_up
 // becomes non-zero.  Returns true when the phase completed.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* give_up) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* give_up,
+                                                  long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
@@ -40,7 +41,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 255u) == 0u) {
             if (*give_up) return false;
-            if (clock64() - t0 > kWaitLimitCycles) return false;
+            if (clock64() - t0 > limit_cycles) return false;
         }
     }
 }

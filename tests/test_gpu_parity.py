@@ -216,3 +216,26 @@ def test_tiny_layer_end_to_end_masks_over_steps():
     order, _, bnd = R.plan(wl.loss_rate, wl.share_weight, wl.n_groups - wl.k_critical)
     j = list(order).index(1)
     assert outcomes == {wl.n_groups - int(bnd[j + 1] - bnd[j]), wl.n_groups}
+
+
+# ---- failure detection: a wait that runs out becomes a status bit, not a hang ----------------------------------
+
+def test_bounded_waits_time_out_cleanly_and_context_stays_usable():
+    flag = torch.zeros(1, dtype=torch.int32, device=DEV)       # nothing ever sets it
+    report = torch.zeros(2, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    B.halo_selftest_bounded_wait(flag, 2_000_000, report, status)   # about a millisecond per wait
+    t1.record()
+    torch.cuda.synchronize()
+    assert report.tolist() == [128, 1]
+    assert int(status.item()) & B.DEV_TIMEOUT
+    assert "timed out" in B.status_message(int(status.item()))
+    assert t0.elapsed_time(t1) < 200.0                               # bounded: milliseconds, not forever
+    # the context is intact: an ordinary call still works and is clean
+    wl = synth.workload("tiny")
+    P, st = U.gpu_group_ffn(wl, synth.packed_layer(wl, 0, DEV), synth.activation(wl, 1, DEV), [0, 1, 2])
+    assert st == 0 and torch.isfinite(P).all().item()
+    with pytest.raises(B.HaloError):
+        B.halo_selftest_bounded_wait(flag, 0, report, status)

@@ -29,7 +29,7 @@ def _worker(rank, world, port, out):
 
 def test_replica_aggregation_takes_the_slowest_rank_and_sums_tokens():
     world, port = 2, 29617
-    with mp.Manager() as mgr:
+    with mp.get_context("spawn").Manager() as mgr:
         out = mgr.dict()
         mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
         res = dict(out)

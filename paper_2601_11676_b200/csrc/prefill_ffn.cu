@@ -44,16 +44,20 @@ __device__ __forceinline__ bool pf_wait(uint64_t* bar, uint32_t parity, volatile
 // ------------------------------------------------------------------------------------------------------------
 // GEMM-1: hidden activations of one kept group for one tile of tokens
 // ------------------------------------------------------------------------------------------------------------
-template <int NS, int STAGES>
+// MH = 128-token halves per tile (1 or 2).  With MH = 2 the group's gate and up rows staged for a K-step serve 256
+// tokens: twice the FLOP per staged byte, four fp32 accumulators = all 512 TMEM columns at NS = 128.
+template <int NS, int MH, int STAGES>
 __global__ void __launch_bounds__(kPfThreads, 1)
 ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, int T, int d,
                   int S, int G, const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
                   __nv_bfloat16* __restrict__ H, int h_cols, uint32_t* dev_status) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = NS * kBK * 2, kStageBytes = kABytes + 2 * kBBytes;
+    constexpr uint32_t kAHalf = kBM * kBK * 2, kABytes = MH * kAHalf, kBBytes = NS * kBK * 2;
+    constexpr uint32_t kStageBytes = kABytes + 2 * kBBytes;
+    constexpr uint32_t kTmemCols = MH * 2 * NS;
     PfBarriers& bars = *reinterpret_cast<PfBarriers*>(smem_raw + static_cast<size_t>(STAGES) * kStageBytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int ki = blockIdx.y, m0 = blockIdx.x * kBM;
+    const int ki = blockIdx.y, m0 = blockIdx.x * (kBM * MH);
     int nk = *n_keep_ptr;
     nk = max(0, min(nk, G));
     if (ki >= nk) return;
@@ -73,7 +77,7 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         tma_prefetch_descriptor(&tmap_x);
         tma_prefetch_descriptor(&tmap_w);
     }
-    if (warp == 1) { tmem_alloc(&bars.tmem_base, 2 * NS); tmem_relinquish_alloc_permit(); }
+    if (warp == 1) { tmem_alloc(&bars.tmem_base, kTmemCols); tmem_relinquish_alloc_permit(); }
     tcgen05_fence_before_sync();
     __syncthreads();
     tcgen05_fence_after_sync();
@@ -88,7 +92,9 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 if (kt >= STAGES && !pf_wait(&bars.empty[s], ((kt / STAGES) - 1) & 1, abort_flag)) break;
                 unsigned char* st = smem_raw + static_cast<size_t>(s) * kStageBytes;
                 mbar_arrive_expect_tx(&bars.full[s], kStageBytes);
-                tma_load_2d(st, &tmap_x, kt * kBK, m0, &bars.full[s]);
+#pragma unroll
+                for (int mh = 0; mh < MH; ++mh)   // rows beyond T read as zeros
+                    tma_load_2d(st + mh * kAHalf, &tmap_x, kt * kBK, m0 + mh * kBM, &bars.full[s]);
                 tma_load_2d(st + kABytes, &tmap_w, kt * kBK, (g * 3 + 0) * S, &bars.full[s]);
                 tma_load_2d(st + kABytes + kBBytes, &tmap_w, kt * kBK, (g * 3 + 1) * S, &bars.full[s]);
                 issued = kt + 1;
@@ -109,50 +115,56 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 const uint32_t a0 = smem_u32(smem_raw + static_cast<size_t>(s) * kStageBytes);
 #pragma unroll
                 for (int kk = 0; kk < kBK / kUmmaK; ++kk) {
-                    const uint64_t a = umma_smem_desc(a0 + kk * 32, 16, 1024);
                     const uint64_t bg = umma_smem_desc(a0 + kABytes + kk * 32, 16, 1024);
                     const uint64_t bu = umma_smem_desc(a0 + kABytes + kBBytes + kk * 32, 16, 1024);
                     const bool accumulate = (kt > 0) || (kk > 0);
-                    umma_bf16(tmem, a, bg, idesc, accumulate);
-                    umma_bf16(tmem + NS, a, bu, idesc, accumulate);
+#pragma unroll
+                    for (int mh = 0; mh < MH; ++mh) {
+                        const uint64_t a = umma_smem_desc(a0 + mh * kAHalf + kk * 32, 16, 1024);
+                        umma_bf16(tmem + mh * 2 * NS, a, bg, idesc, accumulate);
+                        umma_bf16(tmem + mh * 2 * NS + NS, a, bu, idesc, accumulate);
+                    }
                 }
                 umma_commit(&bars.empty[s]);   // the stage is free once these MMAs have read it
             }
             umma_commit(&bars.tmem_full);
         }
     } else {
-        // epilogue: this warp reads TMEM lanes [32*(warp%4), +32) = 32 tokens, one token per thread
+        // epilogue: this warp reads TMEM lanes [32*(warp%4), +32) = 32 tokens of each half, one token per thread
         const bool ok = pf_wait(&bars.tmem_full, 0, abort_flag);
         tcgen05_fence_after_sync();
         const int quad = warp & 3;
-        const int row = m0 + quad * 32 + lane;
         const uint32_t lane_base = tmem + (static_cast<uint32_t>(quad * 32) << 16);
-        for (int c0 = 0; c0 < NS; c0 += 32) {
-            uint32_t dg[32], du[32];
-            tmem_ld_32x32(lane_base + c0, dg);
-            tmem_ld_32x32(lane_base + NS + c0, du);
-            tmem_ld_wait();
-            if (ok && row < T) {
-                uint4* dst = reinterpret_cast<uint4*>(H + static_cast<size_t>(row) * h_cols + static_cast<size_t>(ki) * S + c0);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint32_t packed[4];
+        for (int mh = 0; mh < MH; ++mh) {
+            const int row = m0 + mh * kBM + quad * 32 + lane;
+            for (int c0 = 0; c0 < NS; c0 += 32) {
+                uint32_t dg[32], du[32];
+                tmem_ld_32x32(lane_base + mh * 2 * NS + c0, dg);
+                tmem_ld_32x32(lane_base + mh * 2 * NS + NS + c0, du);
+                tmem_ld_wait();
+                if (ok && row < T) {
+                    uint4* dst = reinterpret_cast<uint4*>(H + static_cast<size_t>(row) * h_cols + static_cast<size_t>(ki) * S + c0);
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int i = q * 8 + e * 2;
-                        const float h0 = silu_mul(__uint_as_float(dg[i]), __uint_as_float(du[i]));
-                        const float h1 = silu_mul(__uint_as_float(dg[i + 1]), __uint_as_float(du[i + 1]));
-                        const __nv_bfloat162 p = __floats2bfloat162_rn(h0, h1);
-                        packed[e] = *reinterpret_cast<const uint32_t*>(&p);
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t packed[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int i = q * 8 + e * 2;
+                            const float h0 = silu_mul(__uint_as_float(dg[i]), __uint_as_float(du[i]));
+                            const float h1 = silu_mul(__uint_as_float(dg[i + 1]), __uint_as_float(du[i + 1]));
+                            const __nv_bfloat162 p = __floats2bfloat162_rn(h0, h1);
+                            packed[e] = *reinterpret_cast<const uint32_t*>(&p);
+                        }
+                        dst[q] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     }
-                    dst[q] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                 }
             }
         }
     }
     tcgen05_fence_before_sync();
     __syncthreads();
-    if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, 2 * NS); }
+    if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, kTmemCols); }
     if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
 }
 
@@ -161,6 +173,8 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 // ------------------------------------------------------------------------------------------------------------
 struct DownSmemTail {
     PfBarriers bars;
+    uint64_t acc_full[2];                 // accumulator b holds a finished slot
+    uint64_t acc_empty[2];                // accumulator b has been drained by the epilogue
     int slot_lo, slot_hi;                 // holder slots this CTA accumulates (the K range is split by slot)
     int slot_start[HALO_MAX_DEVICES + 2];
     int32_t group_of[HALO_MAX_GROUPS];    // group id per position of the slot-sorted order (-1 = skip)
@@ -191,12 +205,14 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
         for (int s = 0; s < STAGES; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], 1); }
         mbar_init(&bars.tmem_full, 1);
         mbar_init(&bars.tmem_empty, 4);
+        for (int b = 0; b < 2; ++b) { mbar_init(&tail.acc_full[b], 1); mbar_init(&tail.acc_empty[b], 4); }
         bars.abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_descriptor(&tmap_h);
         tma_prefetch_descriptor(&tmap_wd);
     }
-    if (warp == 1) { tmem_alloc(&bars.tmem_base, BN2); tmem_relinquish_alloc_permit(); }
+    // two accumulators: the MMAs of the next slot run while the epilogue drains the previous one
+    if (warp == 1) { tmem_alloc(&bars.tmem_base, 2 * BN2); tmem_relinquish_alloc_permit(); }
     if (warp == 0) {
         // kept positions sorted by holder slot (stable): one warp, ballot compaction per slot
         int pos = 0;
@@ -275,8 +291,10 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
             for (int slot = slot_lo; slot < slot_hi && alive; ++slot) {
                 const int p0 = tail.slot_start[slot], p1 = tail.slot_start[slot + 1];
                 if (p0 == p1) continue;
-                if (used > 0 && !pf_wait(&bars.tmem_empty, (used - 1) & 1, abort_flag)) break;  // epilogue has drained D
+                const int buf = used & 1;
+                if (used >= 2 && !pf_wait(&tail.acc_empty[buf], ((used >> 1) - 1) & 1, abort_flag)) break;  // drained
                 tcgen05_fence_after_sync();
+                const uint32_t tmem_acc = tmem + buf * BN2;
                 const int n_it = (p1 - p0) * k_per_group;
                 for (int k = 0; k < n_it; ++k, ++it) {
                     const int s = it % STAGES;
@@ -288,12 +306,12 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
                         const uint64_t a = umma_smem_desc(a0 + kk * 32, 16, 1024);
                         // MN-major B: 16 K-rows per MMA = 2 KiB further; 64-column blocks are kBBlock apart
                         const uint64_t b = umma_smem_desc(a0 + kABytes + kk * 2048, kBBlock, 1024);
-                        umma_bf16(tmem, a, b, idesc, (k > 0) || (kk > 0));
+                        umma_bf16(tmem_acc, a, b, idesc, (k > 0) || (kk > 0));
                     }
                     umma_commit(&bars.empty[s]);
                 }
                 if (!alive) break;
-                umma_commit(&bars.tmem_full);
+                umma_commit(&tail.acc_full[buf]);
                 ++used;
             }
         }
@@ -304,12 +322,13 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
         int used = 0;
         for (int slot = slot_lo; slot < slot_hi; ++slot) {
             if (tail.slot_start[slot] == tail.slot_start[slot + 1]) continue;
-            const bool ok = pf_wait(&bars.tmem_full, used & 1, abort_flag);
+            const int buf = used & 1;
+            const bool ok = pf_wait(&tail.acc_full[buf], (used >> 1) & 1, abort_flag);
             tcgen05_fence_after_sync();
             float* out = partials + (static_cast<size_t>(slot) * T + row) * d + n0;
             for (int c0 = 0; c0 < BN2; c0 += 32) {
                 uint32_t v[32];
-                tmem_ld_32x32(lane_base + c0, v);
+                tmem_ld_32x32(lane_base + buf * BN2 + c0, v);
                 tmem_ld_wait();
                 if (ok && row < T) {
 #pragma unroll
@@ -321,13 +340,13 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
             }
             tcgen05_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars.tmem_empty);
+            if (lane == 0) mbar_arrive(&tail.acc_empty[buf]);
             ++used;
         }
     }
     tcgen05_fence_before_sync();
     __syncthreads();
-    if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, BN2); }
+    if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, 2 * BN2); }
     if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
 }
 
@@ -490,21 +509,23 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
     if (!make_map(&map_x, x, T, d, d, kBK, kBM) || !make_map(&map_w, W, w_rows, d, d, kBK, S) ||
         !make_map(&map_h, H, T, sh.d_ffn, sh.d_ffn, kBK, kBM) || !make_map(&map_wd, W, w_rows, d, d, 64, kBK))
         return HALO_ERR_CUDA;
-    const dim3 grid1((T + kBM - 1) / kBM, G);
-    constexpr int kStages1 = 4;
+    // GEMM-1: 256-token tiles when the prompt has them (more FLOP per staged byte), else 128-token tiles
+#define HALO_LAUNCH_HIDDEN(NS_, MH_, STAGES_)                                                                        \
+    do {                                                                                                             \
+        auto k1 = ffn_hidden_kernel<NS_, MH_, STAGES_>;                                                              \
+        const size_t smem1 = static_cast<size_t>(STAGES_) * (MH_ * kBM * kBK * 2 + 2 * NS_ * kBK * 2) +              \
+                             sizeof(PfBarriers) + 1024;                                                              \
+        static bool once1 = false;                                                                                   \
+        if (!once1) { if (!set_smem(k1, smem1)) return HALO_ERR_CUDA; once1 = true; }                                \
+        const dim3 grid1((T + kBM * MH_ - 1) / (kBM * MH_), G);                                                      \
+        k1<<<grid1, kPfThreads, smem1, st>>>(map_x, map_w, T, d, S, G, keep_list, n_keep, H, sh.d_ffn, dev_status);  \
+    } while (0)
     if (S == 128) {
-        auto k1 = ffn_hidden_kernel<128, kStages1>;
-        const size_t smem1 = static_cast<size_t>(kStages1) * (kBM * kBK * 2 + 2 * 128 * kBK * 2) + sizeof(PfBarriers) + 1024;
-        static bool once1 = false;
-        if (!once1) { if (!set_smem(k1, smem1)) return HALO_ERR_CUDA; once1 = true; }
-        k1<<<grid1, kPfThreads, smem1, st>>>(map_x, map_w, T, d, S, G, keep_list, n_keep, H, sh.d_ffn, dev_status);
+        if (T > kBM) HALO_LAUNCH_HIDDEN(128, 2, 3); else HALO_LAUNCH_HIDDEN(128, 1, 4);
     } else {
-        auto k1 = ffn_hidden_kernel<64, kStages1>;
-        const size_t smem1 = static_cast<size_t>(kStages1) * (kBM * kBK * 2 + 2 * 64 * kBK * 2) + sizeof(PfBarriers) + 1024;
-        static bool once1 = false;
-        if (!once1) { if (!set_smem(k1, smem1)) return HALO_ERR_CUDA; once1 = true; }
-        k1<<<grid1, kPfThreads, smem1, st>>>(map_x, map_w, T, d, S, G, keep_list, n_keep, H, sh.d_ffn, dev_status);
+        if (T > kBM) HALO_LAUNCH_HIDDEN(64, 2, 4); else HALO_LAUNCH_HIDDEN(64, 1, 6);
     }
+#undef HALO_LAUNCH_HIDDEN
     HALO_CHECK_LAUNCH();
     if (d % 256 == 0) {
         // 256-column tiles (more FLOP per staged byte); with holder slots the K range is split over two CTAs

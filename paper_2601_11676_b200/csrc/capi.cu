@@ -349,6 +349,14 @@ struct halo_stack {
     halo::PersistSel* p_sel;       // [3]
     unsigned* p_sync;              // [32]
     void* ffn_ws;                  // H buffer of the tensor-core path (multi-token stacks), or null
+    // multi-token stacks: predictor + selection of block l+1 run on a side stream while block l's FFN runs
+    cudaStream_t side;
+    cudaEvent_t ev_x, ev_sel;
+    float* set_scores[2];          // two selection sets, by parity of the block
+    int32_t* set_dev[2];
+    uint8_t* set_arr[2];
+    int32_t* set_kl[2];
+    int32_t* set_nk[2];
     unsigned long long* trace;     // caller-owned, optional
     int trace_blocks;
     int cross_stages, l2_ahead;    // tuning of the persistent kernel
@@ -410,6 +418,8 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     const size_t o_py = carve(sizeof(unsigned) * 32);
     const size_t ws_bytes = prefill_supported(*ffn, n_tok) ? prefill_workspace_bytes(*ffn, n_tok) : 0;
     const size_t o_ws = carve(ws_bytes ? ws_bytes : 16);
+    const size_t o_sc2 = carve(sizeof(float) * G), o_dg2 = carve(sizeof(int32_t) * G);
+    const size_t o_ar2 = carve(HALO_MAX_DEVICES), o_kl2 = carve(sizeof(int32_t) * G), o_nk2 = carve(sizeof(int32_t));
     if (cudaMalloc(&s->slab, off) != cudaSuccess) { delete s; return HALO_ERR_NOMEM; }
     if (cudaMemset(s->slab, 0, off) != cudaSuccess) { cudaFree(s->slab); delete s; return HALO_ERR_CUDA; }
     char* base = static_cast<char*>(s->slab);
@@ -435,6 +445,21 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     s->p_sel = reinterpret_cast<PersistSel*>(base + o_ps);
     s->p_sync = reinterpret_cast<unsigned*>(base + o_py);
     s->ffn_ws = ws_bytes ? static_cast<void*>(base + o_ws) : nullptr;
+    s->set_scores[0] = s->scores; s->set_scores[1] = reinterpret_cast<float*>(base + o_sc2);
+    s->set_dev[0] = s->dev_of_group; s->set_dev[1] = reinterpret_cast<int32_t*>(base + o_dg2);
+    s->set_arr[0] = s->arrived; s->set_arr[1] = reinterpret_cast<uint8_t*>(base + o_ar2);
+    s->set_kl[0] = s->keep_list; s->set_kl[1] = reinterpret_cast<int32_t*>(base + o_kl2);
+    s->set_nk[0] = s->n_keep; s->set_nk[1] = reinterpret_cast<int32_t*>(base + o_nk2);
+    s->side = nullptr; s->ev_x = nullptr; s->ev_sel = nullptr;
+    if (n_tok > 1) {
+        // best effort: without them the blocks simply run one after the other on the caller's stream
+        if (cudaStreamCreateWithFlags(&s->side, cudaStreamNonBlocking) != cudaSuccess) s->side = nullptr;
+        if (s->side && (cudaEventCreateWithFlags(&s->ev_x, cudaEventDisableTiming) != cudaSuccess ||
+                        cudaEventCreateWithFlags(&s->ev_sel, cudaEventDisableTiming) != cudaSuccess)) {
+            cudaStreamDestroy(s->side);
+            s->side = nullptr;
+        }
+    }
     s->mode = 0;
     s->trace = nullptr;
     s->trace_blocks = 0;
@@ -472,6 +497,12 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
 
 extern "C" halo_status halo_stack_destroy(halo_stack* s) {
     if (!s) return HALO_OK;
+    if (s->side) {
+        cudaStreamSynchronize(s->side);
+        cudaEventDestroy(s->ev_x);
+        cudaEventDestroy(s->ev_sel);
+        cudaStreamDestroy(s->side);
+    }
     cudaFree(s->slab);
     delete s;
     return HALO_OK;
@@ -533,6 +564,63 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
 #define HALO_COPY(dst, src, bytes)                                                                    \
     do { if (cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToDevice, st) != cudaSuccess)     \
              return HALO_ERR_CUDA; } while (0)
+    if (T > 1 && s->side) {
+        // Prompt path.  The scores of block l+1 need only x_l (one layer ahead, Sec. III-B.2), which exists before
+        // block l's FFN starts: predictor + selection of block l+1 go to the side stream and overlap with the
+        // tensor-core GEMMs of block l (the paper's Pred || Comp overlap).  Two selection sets alternate by block.
+        cudaStream_t side = s->side;
+#define HALO_CU(call) do { if ((call) != cudaSuccess) return HALO_ERR_CUDA; } while (0)
+        for (int sidx = 0; sidx < steps; ++sidx) {
+            const uint32_t step = step0 + static_cast<uint32_t>(sidx);
+            HALO_TRY(launch_glue(static_cast<int>(d), static_cast<int>(T), s->ffn.wdtype, h0 + sidx * step_elems,
+                                 nullptr, s->h, s->x[0], st));
+            HALO_TRY(launch_select(s->plan.dev, G, s->zero_scores, step, 0u, 1, nullptr, s->set_dev[0], s->set_arr[0],
+                                   nullptr, s->set_kl[0], s->set_nk[0], s->status, st));
+            launches += 2;
+            HALO_CU(cudaEventRecord(s->ev_x, st));   // x_0 is ready (and set[1] is no longer in use)
+            for (int l = 0; l < L; ++l) {
+                const int cur = l & 1, nxt = (l + 1) & 1;
+                void* x_cur = s->x[cur];
+                void* x_next = s->x[nxt];
+                if (l + 1 < L) {
+                    HALO_CU(cudaStreamWaitEvent(side, s->ev_x, 0));
+                    HALO_TRY(launch_predict(s->pred, s->W1[l + 1], s->W2[l + 1], x_cur, static_cast<int>(T), 1,
+                                            s->set_scores[nxt], s->pred_ws, s->status, side));
+                    HALO_TRY(launch_select(s->plan.dev, G, s->set_scores[nxt], step, static_cast<uint32_t>(l + 1), 0,
+                                           nullptr, s->set_dev[nxt], s->set_arr[nxt], nullptr, s->set_kl[nxt],
+                                           s->set_nk[nxt], s->status, side));
+                    HALO_CU(cudaEventRecord(s->ev_sel, side));
+                    launches += 4;
+                }
+                float* y_tap = nullptr;
+                if (taps) {
+                    const size_t rec = static_cast<size_t>(sidx) * L + l;
+                    if (taps->x) HALO_COPY(static_cast<char*>(taps->x) + rec * step_elems * es, x_cur, step_elems * es);
+                    if (taps->scores) HALO_COPY(taps->scores + rec * G, l == 0 ? s->zero_scores : s->set_scores[cur], sizeof(float) * G);
+                    if (taps->dev_of_group) HALO_COPY(taps->dev_of_group + rec * G, s->set_dev[cur], sizeof(int32_t) * G);
+                    if (taps->arrived && n_dev > 0) HALO_COPY(taps->arrived + rec * n_dev, s->set_arr[cur], n_dev);
+                    if (taps->keep_list) HALO_COPY(taps->keep_list + rec * G, s->set_kl[cur], sizeof(int32_t) * G);
+                    if (taps->n_keep) HALO_COPY(taps->n_keep + rec, s->set_nk[cur], sizeof(int32_t));
+                    if (taps->y) y_tap = taps->y + rec * step_elems;
+                }
+                HALO_TRY(dispatch_group_ffn(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->set_kl[cur], s->set_nk[cur],
+                                            s->set_dev[cur], n_dev, s->partials, s->ffn_ws, s->status, st));
+                float* h_dst = (l == L - 1) ? h_out + sidx * step_elems : s->h;
+                HALO_TRY(launch_merge_glue(s->partials, s->set_arr[cur], n_dev, static_cast<int>(T), static_cast<int>(d),
+                                           s->ffn.wdtype, s->h, h_dst, x_next, y_tap, st));
+                launches += 2;
+                if (l + 1 < L) {
+                    HALO_CU(cudaEventRecord(s->ev_x, st));             // x_{l+1} ready; set[cur] free again
+                    // join: block l+1 needs its selection, and the glue of block l+1 will overwrite the x that the
+                    // side stream has just been reading
+                    HALO_CU(cudaStreamWaitEvent(st, s->ev_sel, 0));
+                }
+            }
+        }
+#undef HALO_CU
+        s->last_launches = launches;
+        return HALO_OK;
+    }
     for (int sidx = 0; sidx < steps; ++sidx) {
         const uint32_t step = step0 + static_cast<uint32_t>(sidx);
         HALO_TRY(launch_glue(static_cast<int>(d), static_cast<int>(T), s->ffn.wdtype, h0 + sidx * step_elems, nullptr,

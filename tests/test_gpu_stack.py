@@ -12,13 +12,13 @@ pytestmark = pytest.mark.gpu
 DEV = U.DEV
 
 
-def build_stack(wl):
+def build_stack(wl, mode=B.SEL_TOPK, threshold=0.0, act=B.ACT_RELU):
     code = U.dtype_code(wl)
     Wp = [synth.packed_layer(wl, l, DEV) for l in range(wl.n_layers)]
     preds = [synth.predictor(wl, l, DEV) for l in range(wl.n_layers)]
-    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, B.SEL_TOPK, wl.k_critical, 0.0, wl.seed)
+    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, mode, wl.k_critical, threshold, wl.seed)
     stack = B.Stack(B.ffn_shape(wl.d_model, wl.d_ffn, wl.group_size, code),
-                    B.pred_shape(wl.d_model, wl.pred_rank, wl.n_groups, code), wl.n_tok, plan, Wp,
+                    B.pred_shape(wl.d_model, wl.pred_rank, wl.n_groups, code, act), wl.n_tok, plan, Wp,
                     [p[0] for p in preds], [p[1] for p in preds])
     return stack, Wp, preds
 
@@ -41,7 +41,8 @@ def run_with_taps(wl, stack, steps, step0=0):
     return h0, h_out, t
 
 
-def check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=0):
+def check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=0, mode=R.SEL_TOPK, threshold=0.0,
+                         act=R.ACT_RELU):
     hb = synth.host_bits
     tol = U.tol_for(wl)
     L, n = wl.n_layers, wl.n_dev
@@ -58,9 +59,9 @@ def check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=0):
             if l == 0:
                 assert (scores == 0).all()
             else:
-                s_ref = R.predict(hb(preds[l][0]), hb(preds[l][1]), x_all[s, l - 1], mean_pool=wl.n_tok > 1)
+                s_ref = R.predict(hb(preds[l][0]), hb(preds[l][1]), x_all[s, l - 1], act=act, mean_pool=wl.n_tok > 1)
                 assert U.rel_err(scores, s_ref.astype(np.float64)) <= tol
-            sel = R.select(scores, wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed,
+            sel = R.select(scores, wl.loss_rate, wl.share_weight, mode, wl.k_critical, threshold, wl.seed,
                            step0 + s, l, force_all=(l == 0))
             nk = int(t["n_keep"][s, l].item())
             assert nk == sel["n_keep"]
@@ -184,3 +185,29 @@ def test_full_size_stack_in_bench_configuration_sampled_blocks(name, steps, samp
     for s in range(steps):
         want = h0[s].double() + t["y"][s].double().sum(dim=0)
         assert (h_out[s].double() - want).abs().max().item() <= 1e-3 * want.abs().max().item()
+
+
+@pytest.mark.parametrize("variant", ["threshold", "act_none", "no_devices", "d8192", "single_device_lossless"])
+def test_stack_persistent_variants(variant):
+    """Persistent path under the other settings of the method: threshold choice of the critical groups, a linear
+    predictor, no virtual devices at all, the widest supported d_model, one lossless device."""
+    kw = dict(mode=B.SEL_TOPK, threshold=0.0, act=B.ACT_RELU)
+    if variant == "threshold":
+        wl = synth.Workload("v", 4, 2048, 64 * 20, 64, 128, "bf16", (0.0, 0.5, 1.0), (1, 2, 1), 0, 6)
+        kw.update(mode=B.SEL_THRESHOLD, threshold=0.5)
+    elif variant == "act_none":
+        wl = synth.Workload("v", 3, 4096, 128 * 6, 128, 64, "bf16", (0.2, 0.7), (1, 1), 334, 4)
+        kw.update(act=B.ACT_NONE)
+    elif variant == "no_devices":
+        wl = synth.Workload("v", 3, 4096, 128 * 5, 128, 64, "bf16", (), (), 400, 3)
+    elif variant == "d8192":
+        wl = synth.Workload("v", 3, 8192, 32 * 9, 32, 64, "bf16", (0.0, 0.6), (1, 3), 300, 4)
+    else:
+        wl = synth.Workload("v", 3, 5120, 128 * 4, 128, 512, "bf16", (0.0,), (7,), 250, 3)
+    stack, Wp, preds = build_stack(wl, **kw)
+    h0, h_out, t = run_with_taps(wl, stack, wl.steps)
+    assert stack.last_launches() == 1      # really the persistent kernel
+    check_teacher_forced(wl, Wp, preds, h0, h_out, t, wl.steps, mode=kw["mode"], threshold=kw["threshold"], act=kw["act"])
+    if variant == "threshold":
+        nk = t["n_keep"][:, 1:].cpu().numpy()
+        assert nk.min() < wl.n_groups and len(np.unique(nk)) > 1   # the critical count really varies with the scores

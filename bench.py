@@ -267,9 +267,45 @@ def run_halo(args, rank, world, local_rank):
                                  "frac_of_peak": kernel_gbs / peak}
     if world == 1 and not args.no_prefill and wl.dtype == "bf16" and wl.n_tok == 1:
         result["prefill"] = prefill_report(wl, Wp, preds, plan, ffn, dev)
+    if world == 1 and not args.no_extra and not args.layers:
+        # the other decode workloads, briefly (same measurement, fewer steps); the headline stays `value`
+        del stack, Wp, preds
+        torch.cuda.empty_cache()
+        result["other_workloads"] = [decode_brief(n, dev, peak) for n in
+                                     ("llama2-13b-decode", "tinyllama-1.1b-decode", "llama2-7b-decode")
+                                     if n != wl.name]
     if world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget)
     return result
+
+
+def decode_brief(name, dev, peak, steps=64, warm=4):
+    """tokens/s and algorithmic GB/s of another decode workload (one persistent launch over `steps` tokens)."""
+    from paper_2601_11676_b200 import binding as B
+    wl = synth.workload(name)
+    stack, Wp, preds, plan, ffn = build_stack(wl, dev)
+    L, G = wl.n_layers, wl.n_groups
+    total = warm + steps
+    h0 = torch.stack([synth.stream_input(wl, s, dev) for s in range(total)])
+    out = torch.empty_like(h0)
+    nk = torch.zeros((total, L), dtype=torch.int32, device=dev)
+    stack.decode(h0, total, 0, out, B.Taps(None, None, None, None, None, nk.data_ptr(), None))
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    stack.decode(h0[warm:], steps, warm, out[warm:])
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b)
+    kept = int(nk[warm:].sum().item())
+    byts = kept * wl.group_bytes + steps * (L - 1) * wl.pred_bytes
+    gbs = byts / (ms * 1e-3) / 1e9
+    res = {"workload": name, "steps": steps, "tokens_per_s": steps / (ms * 1e-3), "ms_per_step": ms / steps,
+           "kept_fraction": kept / float(steps * L * G), "achieved_gbs": gbs, "frac_of_peak": gbs / peak,
+           "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS, "gpu_launches": stack.last_launches(),
+           "device_status": stack.status()}
+    stack.close()
+    return res
 
 
 def prefill_report(wl, Wp, preds, plan, ffn, dev, n_tok=512, prompts=8, warm=3):
@@ -407,6 +443,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="use only this many blocks (small profiling cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true", help="skip the 512-token prompt report")
+    ap.add_argument("--no-extra", action="store_true", help="skip the brief runs of the other decode workloads")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "halo" else args.warmup

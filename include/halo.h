@@ -230,6 +230,19 @@ halo_status halo_group_ffn(const halo_ffn_shape* shape, const void* W_packed, co
                            uint32_t* dev_status, void* stream);
 
 /* ------------------------------------------------------------------------
+ * True importance of the groups (Sec. II-B: the importance of an activation is
+ * its L2 norm; Sec. III-B.2: the predictors are trained on activation norms).
+ * norms[g] = || p_g ||_2, p_g = sum_{j in g} silu(<gate_j,x>) * <up_j,x> * down_j,
+ * for every group of the block and ONE input vector x.  A calibration and
+ * diagnostic call (it reads the whole block), not part of the per-token path.
+ *   W_packed device; x device [d], wdtype; norms device fp32 [G]
+ *   workspace: halo_group_importance_workspace_bytes(shape) bytes, device.
+ * ---------------------------------------------------------------------- */
+size_t halo_group_importance_workspace_bytes(const halo_ffn_shape* shape);
+halo_status halo_group_importance(const halo_ffn_shape* shape, const void* W_packed, const void* x, float* norms,
+                                  void* workspace, size_t workspace_bytes, uint32_t* dev_status, void* stream);
+
+/* ------------------------------------------------------------------------
  * a9. Merge (Sec. III-B.3: after the timeout the master merges the
  * activations that are available): y = partials[0] + sum_i arrived[i] * partials[i+1].
  *   partials device fp32 [n_dev+1][n_tok][d]; arrived device [n_dev] or NULL (all)

@@ -29,7 +29,7 @@ EXPORTS = [
     "halo_stack_destroy", "halo_stack_decode", "halo_stack_decode_host", "halo_stack_status",
     "halo_stack_last_launches", "halo_stack_set_mode", "halo_stack_set_trace", "halo_stack_trace_width",
     "halo_schedule_comp_greedy", "halo_schedule_min_max", "halo_ratios_to_share_weights",
-    "halo_selftest_bounded_wait",
+    "halo_selftest_bounded_wait", "halo_group_importance_workspace_bytes", "halo_group_importance",
 ]
 
 
@@ -99,6 +99,10 @@ def lib() -> ctypes.CDLL:
         L.halo_schedule_min_max.argtypes = [c_int, POINTER(c_double), POINTER(c_double), c_double, c_double,
                                             POINTER(c_double)]
         L.halo_ratios_to_share_weights.argtypes = [c_int, POINTER(c_double), POINTER(c_uint32)]
+        L.halo_group_importance_workspace_bytes.restype = c_size_t
+        L.halo_group_importance_workspace_bytes.argtypes = [POINTER(FfnShape)]
+        L.halo_group_importance.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
+                                            c_void_p]
         L.halo_selftest_bounded_wait.argtypes = [c_void_p, c_longlong, c_void_p, c_void_p, c_void_p]
         L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
         _lib = L
@@ -205,6 +209,18 @@ def halo_ratios_to_share_weights(ratio):
     out = (c_uint32 * n)()
     _chk(lib().halo_ratios_to_share_weights(n, _darr(ratio), out), "halo_ratios_to_share_weights")
     return list(out)
+
+
+def halo_group_importance(shape: FfnShape, W_packed, x, norms, workspace=None, dev_status=None, stream=None):
+    """norms[g] = L2 norm of group g's partial output for the single input vector x.  Allocates the workspace
+    with torch when none is given; returns it so that it can be reused."""
+    need = int(lib().halo_group_importance_workspace_bytes(byref(shape)))
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+    _chk(lib().halo_group_importance(byref(shape), _ptr(W_packed), _ptr(x), _ptr(norms), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream)),
+         "halo_group_importance")
+    return workspace
 
 
 def halo_selftest_bounded_wait(never_set_flag, limit_cycles, report, dev_status, stream=None) -> None:

@@ -168,3 +168,37 @@ def host_bits(t: torch.Tensor) -> np.ndarray:
     if t.dtype == torch.bfloat16:
         return t.view(torch.int16).numpy().view(np.uint16).copy()
     return t.numpy().copy()
+
+
+def structured_layer(wl: Workload, layer: int, device="cpu", scale_sigma: float = 0.8, coherence: float = 1.5,
+                     latent: int = 32):
+    """A packed layer whose groups are NOT exchangeable, plus a matching input distribution, for calibrating and
+    evaluating a predictor without any trained checkpoint.  Every group gets (i) a log-normal overall scale on
+    its down rows, so that some groups matter more than others whatever the input, and (ii) a direction shared by
+    all of its gate rows, so that inputs aligned with it switch the whole group on.  The directions live in a
+    `latent`-dimensional subspace spanned by the columns of A ("topics"); semantic_inputs() draws inputs that mix
+    topic content with noise.  Values are i.i.d. Gaussian apart from these terms.
+    Returns (W[G][3][S][d] in the workload dtype, A[d][latent] fp32)."""
+    base = 100 * (layer + 1)
+    G, S, d = wl.n_groups, wl.group_size, wl.d_model
+    gen = _gen(wl.seed, base + 50, device)
+    W = torch.empty((G, 3, S, d), dtype=torch.float32, device=device).normal_(0.0, wl.weight_std, generator=gen)
+    scale = torch.empty((G,), dtype=torch.float32, device=device).normal_(0.0, scale_sigma, generator=gen).exp()
+    A = torch.empty((d, latent), dtype=torch.float32, device=device).normal_(0.0, latent ** -0.5, generator=gen)
+    C = torch.empty((latent, G), dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=gen)
+    C = C / C.norm(dim=0, keepdim=True)
+    direction = (A @ C).T * (wl.weight_std * latent ** 0.5)          # [G][d], entries ~ weight_std
+    W[:, 0] += coherence * direction[:, None, :]
+    W[:, 2] *= scale[:, None, None]
+    return W.to(wl.torch_dtype), A
+
+
+def semantic_inputs(wl: Workload, tag: int, A: torch.Tensor, n: int, topic_share: float = 0.5) -> torch.Tensor:
+    """n input vectors with unit-variance coordinates: sqrt(topic_share) * (A t) + sqrt(1 - topic_share) * noise,
+    t ~ N(0, I): inputs that carry content in the subspace the structured layer's groups listen to."""
+    device = A.device
+    gen = _gen(wl.seed, 30_000_000 + tag, device)
+    t = torch.empty((n, A.shape[1]), dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=gen)
+    noise = torch.empty((n, A.shape[0]), dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=gen)
+    x = (topic_share ** 0.5) * (t @ A.T) + ((1.0 - topic_share) ** 0.5) * noise
+    return x.to(wl.torch_dtype)

@@ -239,3 +239,34 @@ def test_bounded_waits_time_out_cleanly_and_context_stays_usable():
     assert st == 0 and torch.isfinite(P).all().item()
     with pytest.raises(B.HaloError):
         B.halo_selftest_bounded_wait(flag, 0, report, status)
+
+
+# ---- true importance of the groups (what the predictors regress) -------------------------------------------------
+
+@pytest.mark.parametrize("name", ["tiny", "tinyllama-1.1b-decode", "llama2-7b-decode"])
+def test_group_importance_matches_isolated_group_partials(name):
+    wl = synth.workload(name)
+    Wp = synth.packed_layer(wl, 1, DEV)
+    x = synth.activation(wl, 21, DEV)
+    norms = torch.full((wl.n_groups,), float("nan"), dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.halo_group_importance(B.ffn_shape(wl.d_model, wl.d_ffn, wl.group_size, U.dtype_code(wl)), Wp, x, norms,
+                            dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    _, gp = R.group_ffn(synth.host_bits(Wp), synth.host_bits(x), list(range(wl.n_groups)), want_group_partials=True)
+    ref = np.sqrt((gp[:, 0, :] ** 2).sum(axis=1))
+    got = norms.cpu().numpy()
+    assert np.abs(got - ref).max() <= U.tol_for(wl) * ref.mean()
+
+
+def test_fitted_predictor_beats_random_dropping_on_structured_groups():
+    """Calibration tool end to end (small): a predictor fitted to the true importance must expose better groups
+    to loss than a random choice, and can be no better than the true ranking."""
+    from paper_2601_11676_b200 import calibrate
+    res = calibrate.run("tinyllama-1.1b-decode", n_train=1024, n_test=16, drop_fractions=(0.25,), train_steps=200,
+                        verbose=False)
+    e = res["drop"][0][1]
+    assert e["true-least"] <= e["predicted-least"] + 1e-6
+    assert e["predicted-least"] < e["random"] < e["true-most"]
+    assert res["bottom_quarter_overlap"] > 0.35

@@ -28,9 +28,10 @@ from paper_2601_11676_b200 import synth  # noqa: E402
 
 METRIC = "group-sparse FFN decode tokens/s on 1 B200; achieved HBM GB/s vs ~8 TB/s"
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read+write per launch / algorithmic bytes per launch of stack_decode_kernel, from the ncu capture in
-# profiles/stack_decode_kernel_llama2-7b_4blocks.md (4-block case; traffic is proportional to the kept groups
-# processed, so the ratio carries over to the full-size launch).  Set to None when the kernel changes.
+# dram__bytes_read+write per launch / algorithmic bytes per launch of stack_decode_kernel, from an ncu capture of
+# a 4-block 7B-shaped case (3 231 938 048 + 910 080 bytes against 3 231 058 944 algorithmic); traffic is
+# proportional to the kept groups processed, so the ratio carries over to the full-size launch.  Set to None
+# when the kernel changes.
 STACK_KERNEL_TRAFFIC_RATIO = 1.0003
 FALLBACK_HBM_GBS = 6650.0
 

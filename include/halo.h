@@ -265,6 +265,25 @@ halo_status halo_glue(int d_model, int n_tok, halo_dtype xdtype, const float* h,
                       void* x_out, void* stream);
 
 /* ------------------------------------------------------------------------
+ * One block, steps a1..a9 in one call (the Pred, Comp and merge of one block of the generation phase,
+ * Sec. III-B.3): scores from `feat` (the input of the previous block: one layer ahead), selection and arrival
+ * draw for (step, layer), FFN of `x` over the kept groups, merge of what arrived.  Same results as calling
+ * halo_predict_groups (mean-pooled when n_tok > 1), halo_select_groups, halo_group_ffn and halo_merge_partials
+ * in turn.
+ *   feat, x device [n_tok][d] wdtype; scores device fp32 [G]; dev_of_group device [G]; arrived device [n_dev];
+ *   keep device [G] or NULL; y device fp32 [n_tok][d]
+ *   workspace: halo_layer_workspace_bytes(ffn, pred, n_tok, plan's n_dev) bytes, device.
+ * ---------------------------------------------------------------------- */
+size_t halo_layer_workspace_bytes(const halo_ffn_shape* ffn, const halo_pred_shape* pred, int n_tok, int n_dev);
+halo_status halo_layer_fused(const halo_ffn_shape* ffn, const halo_pred_shape* pred, const halo_plan* plan,
+                             const void* W_packed, const void* W1, const void* W2, const void* feat, const void* x,
+                             int n_tok, uint32_t step, uint32_t layer, int force_all, float* scores,
+                             int32_t* dev_of_group, uint8_t* arrived, uint8_t* keep, float* y, void* workspace,
+                             size_t workspace_bytes, uint32_t* dev_status, void* stream);
+/* halo_status_message for a status word the caller has copied to the host. */
+halo_status halo_read_status(const uint32_t* dev_status_host_copy, char* msg /*host*/, int msg_len);
+
+/* ------------------------------------------------------------------------
  * FFN stack: L blocks chained by halo_glue, the predictor of block l reading
  * the input of block l-1 (one layer ahead, Sec. III-B.2) and block 0 reliable
  * (Sec. III-B.3: the first layer has no semantic information yet).

@@ -30,6 +30,7 @@ EXPORTS = [
     "halo_stack_last_launches", "halo_stack_set_mode", "halo_stack_set_trace", "halo_stack_trace_width",
     "halo_schedule_comp_greedy", "halo_schedule_min_max", "halo_ratios_to_share_weights",
     "halo_selftest_bounded_wait", "halo_group_importance_workspace_bytes", "halo_group_importance",
+    "halo_layer_workspace_bytes", "halo_layer_fused", "halo_read_status",
 ]
 
 
@@ -103,6 +104,11 @@ def lib() -> ctypes.CDLL:
         L.halo_group_importance_workspace_bytes.argtypes = [POINTER(FfnShape)]
         L.halo_group_importance.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
                                             c_void_p]
+        L.halo_layer_workspace_bytes.restype = c_size_t
+        L.halo_layer_workspace_bytes.argtypes = [POINTER(FfnShape), POINTER(PredShape), c_int, c_int]
+        L.halo_layer_fused.argtypes = [POINTER(FfnShape), POINTER(PredShape), c_void_p] + [c_void_p] * 5 + \
+            [c_int, c_uint32, c_uint32, c_int] + [c_void_p] * 6 + [c_size_t, c_void_p, c_void_p]
+        L.halo_read_status.argtypes = [POINTER(c_uint32), c_char_p, c_int]
         L.halo_selftest_bounded_wait.argtypes = [c_void_p, c_longlong, c_void_p, c_void_p, c_void_p]
         L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
         _lib = L
@@ -221,6 +227,27 @@ def halo_group_importance(shape: FfnShape, W_packed, x, norms, workspace=None, d
                                      workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream)),
          "halo_group_importance")
     return workspace
+
+
+def halo_layer_fused(ffn: FfnShape, pred: PredShape, plan: Plan, W_packed, W1, W2, feat, x, n_tok, step, layer,
+                     force_all, scores, dev_of_group, arrived, keep, y, workspace=None, dev_status=None, stream=None):
+    """Steps a1..a9 of one block.  Allocates the workspace with torch when none is given and returns it."""
+    need = int(lib().halo_layer_workspace_bytes(byref(ffn), byref(pred), n_tok, plan.n_dev))
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+    _chk(lib().halo_layer_fused(byref(ffn), byref(pred), plan.handle, _ptr(W_packed), _ptr(W1), _ptr(W2), _ptr(feat),
+                                _ptr(x), n_tok, step, layer, int(bool(force_all)), _ptr(scores), _ptr(dev_of_group),
+                                _ptr(arrived), _ptr(keep), _ptr(y), _ptr(workspace),
+                                workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream)),
+         "halo_layer_fused")
+    return workspace
+
+
+def halo_read_status(value: int) -> str:
+    buf = ctypes.create_string_buffer(128)
+    v = c_uint32(value)
+    _chk(lib().halo_read_status(byref(v), buf, 128), "halo_read_status")
+    return buf.value.decode()
 
 
 def halo_selftest_bounded_wait(never_set_flag, limit_cycles, report, dev_status, stream=None) -> None:

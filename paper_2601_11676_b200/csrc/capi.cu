@@ -313,6 +313,66 @@ extern "C" halo_status halo_glue(int d_model, int n_tok, halo_dtype xdtype, cons
     return launch_glue(d_model, n_tok, xdtype, h, y, h_out, x_out, static_cast<cudaStream_t>(stream));
 }
 
+// ---- one block, a1..a9 ------------------------------------------------------------------------------------
+
+extern "C" size_t halo_layer_workspace_bytes(const halo_ffn_shape* ffn, const halo_pred_shape* pred, int n_tok, int n_dev) {
+    if (check_ffn_shape(ffn) != HALO_OK || check_pred_shape(pred) != HALO_OK || n_tok <= 0 || n_dev < 0) return 0;
+    const size_t G = static_cast<size_t>(ffn->d_ffn / ffn->group_size);
+    size_t b = align_up(halo_predict_workspace_bytes(pred, n_tok), 256);
+    b += align_up(halo_group_ffn_workspace_bytes(ffn, n_tok, n_dev), 256);
+    b += align_up(sizeof(float) * static_cast<size_t>(n_dev + 1) * n_tok * ffn->d_model, 256);   // partials
+    b += align_up(sizeof(int32_t) * G, 256) + 256;                                                // keep_list, n_keep
+    return b;
+}
+
+extern "C" halo_status halo_layer_fused(const halo_ffn_shape* ffn, const halo_pred_shape* pred, const halo_plan* plan,
+                                        const void* W_packed, const void* W1, const void* W2, const void* feat,
+                                        const void* x, int n_tok, uint32_t step, uint32_t layer, int force_all,
+                                        float* scores, int32_t* dev_of_group, uint8_t* arrived, uint8_t* keep,
+                                        float* y, void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                                        void* stream) {
+    halo_status rc = check_ffn_shape(ffn);
+    if (rc != HALO_OK) return rc;
+    rc = check_pred_shape(pred);
+    if (rc != HALO_OK) return rc;
+    if (!plan || !W_packed || !W1 || !W2 || !feat || !x || !scores || !dev_of_group || !arrived || !y) return HALO_ERR_ARG;
+    if (n_tok <= 0) return HALO_ERR_SHAPE;
+    const int G = ffn->d_ffn / ffn->group_size, n_dev = plan->n_dev;
+    if (pred->n_groups != G || plan->n_groups != G || pred->d_in != ffn->d_model || pred->wdtype != ffn->wdtype)
+        return HALO_ERR_SHAPE;
+    if (!aligned16(W_packed) || !aligned16(W1) || !aligned16(W2) || !aligned16(feat) || !aligned16(x) || !aligned16(y) ||
+        !aligned16(workspace))
+        return HALO_ERR_ALIGN;
+    if (!workspace || workspace_bytes < halo_layer_workspace_bytes(ffn, pred, n_tok, n_dev)) return HALO_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    float* pred_ws = reinterpret_cast<float*>(ws);
+    ws += align_up(halo_predict_workspace_bytes(pred, n_tok), 256);
+    void* ffn_ws = ws;
+    const size_t ffn_ws_bytes = halo_group_ffn_workspace_bytes(ffn, n_tok, n_dev);
+    ws += align_up(ffn_ws_bytes, 256);
+    float* partials = reinterpret_cast<float*>(ws);
+    ws += align_up(sizeof(float) * static_cast<size_t>(n_dev + 1) * n_tok * ffn->d_model, 256);
+    int32_t* keep_list = reinterpret_cast<int32_t*>(ws);
+    ws += align_up(sizeof(int32_t) * static_cast<size_t>(G), 256);
+    int32_t* n_keep = reinterpret_cast<int32_t*>(ws);
+    // a1 (mean over tokens for a prompt), a2..a5, a6..a8 over the kept groups, a9
+    rc = launch_predict(*pred, W1, W2, feat, n_tok, 1, scores, pred_ws, dev_status, st);
+    if (rc != HALO_OK) return rc;
+    rc = launch_select(plan->dev, G, scores, step, layer, force_all, nullptr, dev_of_group, arrived, keep, keep_list,
+                       n_keep, dev_status, st);
+    if (rc != HALO_OK) return rc;
+    rc = dispatch_group_ffn(*ffn, W_packed, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials,
+                            ffn_ws_bytes ? ffn_ws : nullptr, dev_status, st);
+    if (rc != HALO_OK) return rc;
+    return launch_merge(partials, arrived, n_dev, n_tok, ffn->d_model, y, st);
+}
+
+extern "C" halo_status halo_read_status(const uint32_t* dev_status_host_copy, char* msg, int msg_len) {
+    if (!dev_status_host_copy) return HALO_ERR_ARG;
+    return halo_status_message(*dev_status_host_copy, msg, msg_len);
+}
+
 // ---- FFN stack ----------------------------------------------------------------------------------------
 
 struct halo_stack {

@@ -270,3 +270,40 @@ def test_fitted_predictor_beats_random_dropping_on_structured_groups():
     assert e["true-least"] <= e["predicted-least"] + 1e-6
     assert e["predicted-least"] < e["random"] < e["true-most"]
     assert res["bottom_quarter_overlap"] > 0.35
+
+
+# ---- one block in one call ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("name,n_tok", [("tiny", 1), ("llama2-7b-decode", 1), ("tinyllama-1.1b-decode", 40)])
+def test_layer_fused_matches_oracle_layer(name, n_tok):
+    wl = synth.workload(name)
+    code = U.dtype_code(wl)
+    Wp, W1, W2 = U.layer_tensors(wl, 2)
+    feat = synth.activation(wl, 30, DEV, n_tok=n_tok)
+    x = synth.activation(wl, 31, DEV, n_tok=n_tok)
+    G, n, d = wl.n_groups, wl.n_dev, wl.d_model
+    plan = B.Plan(G, wl.loss_rate, wl.share_weight, B.SEL_TOPK, wl.k_critical, 0.0, wl.seed)
+    ffn = B.ffn_shape(d, wl.d_ffn, wl.group_size, code)
+    pred = B.pred_shape(d, wl.pred_rank, G, code)
+    scores = torch.zeros(G, dtype=torch.float32, device=DEV)
+    dg = torch.zeros(G, dtype=torch.int32, device=DEV)
+    arr = torch.zeros(max(n, 1), dtype=torch.uint8, device=DEV)
+    keep = torch.zeros(G, dtype=torch.uint8, device=DEV)
+    y = torch.zeros((n_tok, d), dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = None
+    hb = synth.host_bits
+    sample = list(range(n_tok)) if n_tok <= 4 else [0, 17, n_tok - 1]
+    for step in (0, 3):
+        ws = B.halo_layer_fused(ffn, pred, plan, Wp, W1, W2, feat, x, n_tok, step, 5, False, scores, dg, arr, keep, y,
+                                ws, status)
+        torch.cuda.synchronize()
+        assert B.halo_read_status(int(status.item())) == "clean"
+        s_ref = R.predict(hb(W1), hb(W2), hb(feat), mean_pool=n_tok > 1)
+        assert U.rel_err(scores.cpu().numpy(), s_ref.astype(np.float64)) <= U.tol_for(wl)
+        sel = R.select(scores.cpu().numpy(), wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed,
+                       step, 5)
+        assert (dg.cpu().numpy() == sel["dev_of_group"]).all() and (keep.cpu().numpy() == sel["keep"]).all()
+        assert (arr.cpu().numpy()[:n] == sel["arrived"]).all()
+        P = R.group_ffn(hb(Wp), hb(x)[sample], sel["keep_list"][: sel["n_keep"]], sel["dev_of_group"], n)
+        assert U.rel_err(y[sample].cpu().numpy(), R.merge(P)) <= U.tol_for(wl)

@@ -479,3 +479,100 @@ int halo_ref_min_max(int n, const double* m, const double* c, double Mt, double 
     for (int i = 0; i < n; ++i) r[i] /= sum_u;
     return REF_OK;
 }
+
+/* ---- MHA neuron groups (Sec. II-A: one head and its output-projection slice) ---- */
+/* Packed layout Wattn[H][2][dh][d]: plane 0 = the head's query rows, plane 1 =
+ * the head's slice of the output projection stored as rows (row j = column
+ * h*dh+j of Wo[d][H*dh]).  Keys and values are NOT part of a group: every
+ * device keeps a full KV cache (Sec. III-B.3), so K/V projections are computed
+ * for all heads at every token and never dropped.  No positional rotation. */
+static size_t mha_index(int h, int plane, int j, int c, int dh, int d) {
+    return (((size_t)h * 2 + (size_t)plane) * (size_t)dh + (size_t)j) * (size_t)d + (size_t)c;
+}
+
+int halo_ref_pack_mha(int d, int H, int dh, int dtype, const void* Wq /*[H*dh][d]*/, const void* Wo /*[d][H*dh]*/,
+                      void* Wpacked) {
+    if (d <= 0 || H <= 0 || dh <= 0) return REF_ERR_SHAPE;
+    size_t es = ref_elem_size(dtype);
+    for (int h = 0; h < H; ++h)
+        for (int j = 0; j < dh; ++j)
+            for (int c = 0; c < d; ++c) {
+                size_t n = (size_t)h * dh + j;
+                memcpy((char*)Wpacked + es * mha_index(h, 0, j, c, dh, d), (const char*)Wq + es * (n * d + c), es);
+                memcpy((char*)Wpacked + es * mha_index(h, 1, j, c, dh, d),
+                       (const char*)Wo + es * ((size_t)c * H * dh + n), es);
+            }
+    return REF_OK;
+}
+
+/* k = Wk x, v = Wv x for every head, stored in the cache dtype at position pos.
+ * Caches are [H][Lmax][dh]. */
+int halo_ref_mha_kv_append(int d, int H, int dh, int Lmax, int dtype, const void* Wk /*[H*dh][d]*/,
+                           const void* Wv, const void* x, int pos, void* K_cache, void* V_cache) {
+    if (d <= 0 || H <= 0 || dh <= 0 || pos < 0 || pos >= Lmax) return REF_ERR_SHAPE;
+    for (int h = 0; h < H; ++h)
+        for (int j = 0; j < dh; ++j) {
+            double k = 0.0, v = 0.0;
+            size_t row = (size_t)h * dh + j;
+            for (int c = 0; c < d; ++c) {
+                double xc = ref_widen(x, (size_t)c, dtype);
+                k += ref_widen(Wk, row * d + c, dtype) * xc;
+                v += ref_widen(Wv, row * d + c, dtype) * xc;
+            }
+            size_t at = ((size_t)h * Lmax + (size_t)pos) * dh + j;
+            if (dtype == REF_F32) { ((float*)K_cache)[at] = (float)k; ((float*)V_cache)[at] = (float)v; }
+            else { ((uint16_t*)K_cache)[at] = ref_double_to_bf16(k); ((uint16_t*)V_cache)[at] = ref_double_to_bf16(v); }
+        }
+    return REF_OK;
+}
+
+/* For each listed head h: q = Wq_h x; s_p = <q, K_h[p]> / sqrt(dh) for p = 0..pos;
+ * w = softmax(s); o = sum_p w_p V_h[p]; p_h = sum_j o_j * Wo_h[j] (width d), added to
+ * the slot of the head's holder.  head_partials, if given, gets every p_h. */
+int halo_ref_group_mha(int d, int H, int dh, int Lmax, int dtype, const void* Wpacked, const void* x,
+                       const void* K_cache, const void* V_cache, int pos, const int32_t* list, int n_list,
+                       const int32_t* dev_of_group, int n_dev, double* partials /*[n_dev+1][d]*/,
+                       double* head_partials /*[n_list][d] or NULL*/) {
+    if (d <= 0 || H <= 0 || dh <= 0 || pos < 0 || pos >= Lmax || n_list < 0) return REF_ERR_SHAPE;
+    for (int i = 0; i < n_list; ++i) if (list[i] < 0 || list[i] >= H) return REF_ERR_ARG;
+    memset(partials, 0, sizeof(double) * (size_t)(n_dev + 1) * d);
+    double* q = (double*)malloc(sizeof(double) * (size_t)dh);
+    double* o = (double*)malloc(sizeof(double) * (size_t)dh);
+    double* w = (double*)malloc(sizeof(double) * (size_t)(pos + 1));
+    double* ph = (double*)malloc(sizeof(double) * (size_t)d);
+    if (!q || !o || !w || !ph) { free(q); free(o); free(w); free(ph); return REF_ERR_NOMEM; }
+    int rc = REF_OK;
+    for (int i = 0; i < n_list && rc == REF_OK; ++i) {
+        int h = list[i];
+        for (int j = 0; j < dh; ++j) {
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c) acc += ref_widen(Wpacked, mha_index(h, 0, j, c, dh, d), dtype) * ref_widen(x, (size_t)c, dtype);
+            q[j] = acc;
+        }
+        double smax = -INFINITY;
+        for (int p = 0; p <= pos; ++p) {
+            double acc = 0.0;
+            for (int j = 0; j < dh; ++j) acc += q[j] * ref_widen(K_cache, ((size_t)h * Lmax + p) * dh + j, dtype);
+            w[p] = acc / sqrt((double)dh);
+            if (w[p] > smax) smax = w[p];
+        }
+        double denom = 0.0;
+        for (int p = 0; p <= pos; ++p) { w[p] = exp(w[p] - smax); denom += w[p]; }
+        for (int j = 0; j < dh; ++j) {
+            double acc = 0.0;
+            for (int p = 0; p <= pos; ++p) acc += w[p] * ref_widen(V_cache, ((size_t)h * Lmax + p) * dh + j, dtype);
+            o[j] = acc / denom;
+        }
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int j = 0; j < dh; ++j) acc += o[j] * ref_widen(Wpacked, mha_index(h, 1, j, c, dh, d), dtype);
+            ph[c] = acc;
+        }
+        int slot = dev_of_group ? dev_of_group[h] + 1 : 0;
+        if (slot < 0 || slot > n_dev) { rc = REF_ERR_ARG; break; }
+        for (int c = 0; c < d; ++c) partials[(size_t)slot * d + c] += ph[c];
+        if (head_partials) memcpy(head_partials + (size_t)i * d, ph, sizeof(double) * (size_t)d);
+    }
+    free(q); free(o); free(w); free(ph);
+    return rc;
+}

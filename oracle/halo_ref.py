@@ -284,3 +284,46 @@ def min_max(m, c, Mt: float, eps: float = 1e-3) -> np.ndarray:
     r = np.empty(len(m), dtype=np.float64)
     _check(lib().halo_ref_min_max(c_int(len(m)), _p(m), _p(c), c_double(Mt), c_double(eps), _p(r)), "min_max")
     return r
+
+
+# --- MHA neuron groups --------------------------------------------------------------------
+
+def pack_mha(Wq: np.ndarray, Wo: np.ndarray, H: int) -> np.ndarray:
+    """Wq[H*dh][d], Wo[d][H*dh] -> packed [H][2][dh][d]."""
+    n, d = Wq.shape
+    dh = n // H
+    assert Wo.shape == (d, n)
+    dt = _dtype_of(Wq)
+    Wq, Wo = _c(Wq), _c(Wo)
+    out = np.empty((H, 2, dh, d), dtype=Wq.dtype)
+    _check(lib().halo_ref_pack_mha(c_int(d), c_int(H), c_int(dh), c_int(dt), _p(Wq), _p(Wo), _p(out)), "pack_mha")
+    return out
+
+
+def mha_kv_append(Wk: np.ndarray, Wv: np.ndarray, x: np.ndarray, pos: int, K_cache: np.ndarray, V_cache: np.ndarray):
+    """Writes k, v of this token at `pos` into the caches [H][Lmax][dh] (in place)."""
+    H, Lmax, dh = K_cache.shape
+    d = Wk.shape[1]
+    dt = _dtype_of(Wk)
+    assert K_cache.flags.c_contiguous and V_cache.flags.c_contiguous and _dtype_of(K_cache) == dt
+    Wk, Wv, x1 = _c(Wk), _c(Wv), _c(x.reshape(-1))
+    _check(lib().halo_ref_mha_kv_append(c_int(d), c_int(H), c_int(dh), c_int(Lmax), c_int(dt), _p(Wk), _p(Wv), _p(x1),
+                                        c_int(pos), _p(K_cache), _p(V_cache)), "mha_kv_append")
+
+
+def group_mha(Wpacked: np.ndarray, x: np.ndarray, K_cache: np.ndarray, V_cache: np.ndarray, pos: int, head_list,
+              dev_of_group=None, n_dev: int = 0, want_head_partials: bool = False):
+    H, _, dh, d = Wpacked.shape
+    Lmax = K_cache.shape[1]
+    dt = _dtype_of(Wpacked)
+    Wpacked, x1, K_cache, V_cache = _c(Wpacked), _c(x.reshape(-1)), _c(K_cache), _c(V_cache)
+    lst = np.asarray(head_list, dtype=np.int32).reshape(-1)
+    dg = None if dev_of_group is None else _c(np.asarray(dev_of_group, dtype=np.int32))
+    P = np.empty((n_dev + 1, d), dtype=np.float64)
+    hp = np.empty((max(len(lst), 1), d), dtype=np.float64) if want_head_partials else None
+    _check(lib().halo_ref_group_mha(c_int(d), c_int(H), c_int(dh), c_int(Lmax), c_int(dt), _p(Wpacked), _p(x1),
+                                    _p(K_cache), _p(V_cache), c_int(pos), _p(lst), c_int(len(lst)), _p(dg),
+                                    c_int(n_dev), _p(P), _p(hp)), "group_mha")
+    if want_head_partials:
+        return P, hp[: len(lst)]
+    return P

@@ -202,3 +202,11 @@ def semantic_inputs(wl: Workload, tag: int, A: torch.Tensor, n: int, topic_share
     noise = torch.empty((n, A.shape[0]), dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=gen)
     x = (topic_share ** 0.5) * (t @ A.T) + ((1.0 - topic_share) ** 0.5) * noise
     return x.to(wl.torch_dtype)
+
+
+def mha_matrices(wl: Workload, layer: int, n_heads: int, device="cpu"):
+    """Attention projections of one block: Wq, Wk, Wv [H*dh][d] and Wo [d][H*dh], N(0, weight_std)."""
+    base = 100 * (layer + 1) + 60
+    d = wl.d_model
+    mk = lambda i, shape: _normal(shape, wl.weight_std, wl.torch_dtype, _gen(wl.seed, base + i, device), device)
+    return mk(0, (d, d)), mk(1, (d, d)), mk(2, (d, d)), mk(3, (d, d))

@@ -265,6 +265,37 @@ halo_status halo_glue(int d_model, int n_tok, halo_dtype xdtype, const float* h,
                       void* x_out, void* stream);
 
 /* ------------------------------------------------------------------------
+ * MHA neuron groups, decode form (Sec. II-A: "one head and its output projection weight are an independent
+ * neuron group").  The same scoring / selection / holder slots / merge apply with G = n_heads: score with
+ * halo_predict_groups, choose with halo_select_groups, merge with halo_merge_partials.  Keys and values are not
+ * part of a group: every device keeps a full KV cache (Sec. III-B.3), so the K/V projections of ALL heads are
+ * computed at every token (halo_mha_kv_append) and never dropped.  No positional rotation is applied.
+ *   halo_mha_shape: d_model % 8 == 0, head_dim a multiple of 16 (<= 256); max_len = cache capacity.
+ *   W_packed device [H][2][head_dim][d]: plane 0 = the head's query rows, plane 1 = the head's slice of the
+ *     output projection stored as rows (row j = column h*head_dim+j of Wo[d][H*head_dim]);
+ *     halo_pack_mha_weights builds it from Wq[H*head_dim][d] and Wo.
+ *   K_cache, V_cache device [H][max_len][head_dim] in wdtype.
+ *   halo_mha_kv_append: k = Wk x, v = Wv x (Wk, Wv device [H*head_dim][d]) written at position pos.
+ *   halo_group_mha: for each kept head h: q = Wq_h x; w = softmax(q K_h^T / sqrt(head_dim)) over positions
+ *     0..pos; o = w V_h; partials[slot(h)] += sum_j o_j * Wo_h[j].  partials device fp32 [n_dev+1][d], zeroed by
+ *     the call; keep_list / n_keep / dev_of_group as for halo_group_ffn (device); x device [d].
+ *     workspace: halo_group_mha_workspace_bytes(shape) bytes, device.  fp32 accumulation and softmax.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+    int d_model, n_heads, head_dim, max_len;
+    halo_dtype wdtype;
+} halo_mha_shape;
+halo_status halo_pack_mha_weights(const halo_mha_shape* shape, const void* Wq, const void* Wo, void* W_packed,
+                                  void* stream);
+halo_status halo_mha_kv_append(const halo_mha_shape* shape, const void* Wk, const void* Wv, const void* x, int pos,
+                               void* K_cache, void* V_cache, void* stream);
+size_t halo_group_mha_workspace_bytes(const halo_mha_shape* shape);
+halo_status halo_group_mha(const halo_mha_shape* shape, const void* W_packed, const void* x, const void* K_cache,
+                           const void* V_cache, int pos, const int32_t* keep_list, const int32_t* n_keep,
+                           const int32_t* dev_of_group, int n_dev, float* partials, void* workspace,
+                           size_t workspace_bytes, uint32_t* dev_status, void* stream);
+
+/* ------------------------------------------------------------------------
  * One block, steps a1..a9 in one call (the Pred, Comp and merge of one block of the generation phase,
  * Sec. III-B.3): scores from `feat` (the input of the previous block: one layer ahead), selection and arrival
  * draw for (step, layer), FFN of `x` over the kept groups, merge of what arrived.  Same results as calling

@@ -31,6 +31,7 @@ EXPORTS = [
     "halo_schedule_comp_greedy", "halo_schedule_min_max", "halo_ratios_to_share_weights",
     "halo_selftest_bounded_wait", "halo_group_importance_workspace_bytes", "halo_group_importance",
     "halo_layer_workspace_bytes", "halo_layer_fused", "halo_read_status",
+    "halo_pack_mha_weights", "halo_mha_kv_append", "halo_group_mha_workspace_bytes", "halo_group_mha",
 ]
 
 
@@ -40,6 +41,10 @@ class FfnShape(Structure):
 
 class PredShape(Structure):
     _fields_ = [("d_in", c_int), ("rank", c_int), ("n_groups", c_int), ("wdtype", c_int), ("act", c_int)]
+
+
+class MhaShape(Structure):
+    _fields_ = [("d_model", c_int), ("n_heads", c_int), ("head_dim", c_int), ("max_len", c_int), ("wdtype", c_int)]
 
 
 class Taps(Structure):
@@ -109,6 +114,12 @@ def lib() -> ctypes.CDLL:
         L.halo_layer_fused.argtypes = [POINTER(FfnShape), POINTER(PredShape), c_void_p] + [c_void_p] * 5 + \
             [c_int, c_uint32, c_uint32, c_int] + [c_void_p] * 6 + [c_size_t, c_void_p, c_void_p]
         L.halo_read_status.argtypes = [POINTER(c_uint32), c_char_p, c_int]
+        L.halo_pack_mha_weights.argtypes = [POINTER(MhaShape), c_void_p, c_void_p, c_void_p, c_void_p]
+        L.halo_mha_kv_append.argtypes = [POINTER(MhaShape), c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+        L.halo_group_mha_workspace_bytes.restype = c_size_t
+        L.halo_group_mha_workspace_bytes.argtypes = [POINTER(MhaShape)]
+        L.halo_group_mha.argtypes = [POINTER(MhaShape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
+                                     c_void_p, c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
         L.halo_selftest_bounded_wait.argtypes = [c_void_p, c_longlong, c_void_p, c_void_p, c_void_p]
         L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
         _lib = L
@@ -248,6 +259,32 @@ def halo_read_status(value: int) -> str:
     v = c_uint32(value)
     _chk(lib().halo_read_status(byref(v), buf, 128), "halo_read_status")
     return buf.value.decode()
+
+
+def mha_shape(d_model, n_heads, head_dim, max_len, dtype) -> MhaShape:
+    return MhaShape(d_model, n_heads, head_dim, max_len, dtype)
+
+
+def halo_pack_mha_weights(shape: MhaShape, Wq, Wo, W_packed, stream=None) -> None:
+    _chk(lib().halo_pack_mha_weights(byref(shape), _ptr(Wq), _ptr(Wo), _ptr(W_packed), _stream(stream)),
+         "halo_pack_mha_weights")
+
+
+def halo_mha_kv_append(shape: MhaShape, Wk, Wv, x, pos, K_cache, V_cache, stream=None) -> None:
+    _chk(lib().halo_mha_kv_append(byref(shape), _ptr(Wk), _ptr(Wv), _ptr(x), pos, _ptr(K_cache), _ptr(V_cache),
+                                  _stream(stream)), "halo_mha_kv_append")
+
+
+def halo_group_mha_workspace_bytes(shape: MhaShape) -> int:
+    return int(lib().halo_group_mha_workspace_bytes(byref(shape)))
+
+
+def halo_group_mha(shape: MhaShape, W_packed, x, K_cache, V_cache, pos, keep_list, n_keep, dev_of_group, n_dev,
+                   partials, workspace, dev_status=None, stream=None) -> None:
+    _chk(lib().halo_group_mha(byref(shape), _ptr(W_packed), _ptr(x), _ptr(K_cache), _ptr(V_cache), pos,
+                              _ptr(keep_list), _ptr(n_keep), _ptr(dev_of_group), n_dev, _ptr(partials), _ptr(workspace),
+                              workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream)),
+         "halo_group_mha")
 
 
 def halo_selftest_bounded_wait(never_set_flag, limit_cycles, report, dev_status, stream=None) -> None:

@@ -1,0 +1,385 @@
+// MHA neuron groups (Sec. II-A: one head and its output-projection weight form an independent neuron group),
+// decode form, under the same selection / holder-slot / merge machinery as the FFN groups.
+//   halo_mha_kv_append   k = Wk x, v = Wv x for ALL heads into the caches (every device keeps a full KV cache,
+//                        Sec. III-B.3; keys and values are never dropped)
+//   halo_group_mha       for every kept head h:  q = Wq_h x;  w = softmax(q K_h^T / sqrt(dh)) over positions 0..pos;
+//                        o = w V_h;  partials[slot(h)] += sum_j o_j * Wo_h[j]
+// Three launches: query rows (one warp per row), attention per (head, 128-position chunk) with a running-max
+// partial (m, l, o), and combination + output-projection rows (each block streams 16 rows of the head's slice and
+// adds its column sums to the holder's slot with vector reductions).  Bandwidth-bound like the FFN decode path.
+#include "common.cuh"
+#include "tma.cuh"
+
+namespace halo {
+
+constexpr int kAttnChunk = 128;   // positions per attention block
+constexpr int kOutRows = 16;      // output-projection rows per block
+
+template <typename T>
+__device__ __forceinline__ float warp_row_dot(const T* __restrict__ row, const float* __restrict__ xs, int chunks, int lane) {
+    constexpr int E = Elem<T>::kPerChunk;
+    const uint4* r4 = reinterpret_cast<const uint4*>(row);
+    float acc = 0.0f;
+    for (int c0 = lane; c0 < chunks; c0 += 256) {   // eight 16-byte loads in flight per lane
+        uint4 w[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int c = c0 + 32 * i;
+            w[i] = c < chunks ? ldg_stream16(r4 + c) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int c = c0 + 32 * i;
+            if (c < chunks) {
+                float wf[E];
+                Elem<T>::widen(w[i], wf);
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc = fmaf(wf[e], xs[c * E + e], acc);
+            }
+        }
+    }
+    return warp_sum(acc);
+}
+
+// one warp per row of [Wk; Wv]: rows 0..H*dh-1 are keys, the rest values
+template <typename T>
+__global__ void __launch_bounds__(256)
+mha_kv_append_kernel(int d, int H, int dh, int Lmax, const T* __restrict__ Wk, const T* __restrict__ Wv,
+                     const T* __restrict__ x, int pos, T* __restrict__ Kc, T* __restrict__ Vc) {
+    extern __shared__ float xs[];
+    for (int c = threadIdx.x; c < d; c += blockDim.x) xs[c] = to_float(x[c]);
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n = H * dh;
+    const int r = blockIdx.x * 8 + warp;
+    if (r >= 2 * n) return;
+    const bool is_v = r >= n;
+    const int rr = is_v ? r - n : r;
+    const float v = warp_row_dot((is_v ? Wv : Wk) + static_cast<size_t>(rr) * d, xs, d / Elem<T>::kPerChunk, lane);
+    if (lane == 0) {
+        const int h = rr / dh, j = rr - h * dh;
+        (is_v ? Vc : Kc)[(static_cast<size_t>(h) * Lmax + pos) * dh + j] = from_float<T>(v);
+    }
+}
+
+// q[ki][j] = <Wq_h[j], x> / sqrt(dh) for the kept heads
+template <typename T>
+__global__ void __launch_bounds__(256)
+mha_q_kernel(int d, int H, int dh, const T* __restrict__ Wp, const T* __restrict__ x,
+             const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr, float* __restrict__ q_ws,
+             uint32_t* dev_status) {
+    extern __shared__ float xs[];
+    for (int c = threadIdx.x; c < d; c += blockDim.x) xs[c] = to_float(x[c]);
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int nk = *n_keep_ptr;
+    nk = max(0, min(nk, H));
+    const int r = blockIdx.x * 8 + warp;
+    const int ki = r / dh, j = r - ki * dh;
+    if (ki >= nk) return;
+    const int h = keep_list[ki];
+    if (h < 0 || h >= H) {
+        if (lane == 0 && j == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+        return;
+    }
+    const T* row = Wp + ((static_cast<size_t>(h) * 2 + 0) * dh + j) * d;
+    const float v = warp_row_dot(row, xs, d / Elem<T>::kPerChunk, lane);
+    if (lane == 0) q_ws[static_cast<size_t>(ki) * dh + j] = v * rsqrtf(static_cast<float>(dh));
+}
+
+// attention partial of one (kept head, chunk of 128 positions): m = max score, l = sum exp(s - m),
+// o[j] = sum_p exp(s_p - m) V[p][j]; record layout [m, l, o[dh]]
+template <typename T>
+__global__ void __launch_bounds__(kAttnChunk)
+mha_attn_kernel(int H, int dh, int Lmax, int pos, const T* __restrict__ Kc, const T* __restrict__ Vc,
+                const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
+                const float* __restrict__ q_ws, float* __restrict__ attn_ws, int n_chunks) {
+    __shared__ float q[256];
+    __shared__ float w[kAttnChunk];
+    __shared__ float red[8];
+    const int ki = blockIdx.x, chunk = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int nk = *n_keep_ptr;
+    nk = max(0, min(nk, H));
+    if (ki >= nk) return;
+    const int h = keep_list[ki];
+    if (h < 0 || h >= H) return;
+    for (int j = tid; j < dh; j += kAttnChunk) q[j] = q_ws[static_cast<size_t>(ki) * dh + j];
+    __syncthreads();
+    constexpr int E = Elem<T>::kPerChunk;
+    const int p = chunk * kAttnChunk + tid;
+    const bool valid = p <= pos;
+    float s = -INFINITY;
+    if (valid) {
+        const uint4* krow = reinterpret_cast<const uint4*>(Kc + (static_cast<size_t>(h) * Lmax + p) * dh);
+        float acc = 0.0f;
+        for (int c = 0; c < dh / E; ++c) {
+            float kf[E];
+            Elem<T>::widen(__ldg(krow + c), kf);
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc = fmaf(kf[e], q[c * E + e], acc);
+        }
+        s = acc;
+    }
+    // block max
+    float m = s;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    m = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+    const float e = valid ? __expf(s - m) : 0.0f;
+    w[tid] = e;
+    float l = warp_sum(e);
+    if (lane == 0) red[4 + warp] = l;
+    __syncthreads();
+    l = red[4] + red[5] + red[6] + red[7];
+    float* rec = attn_ws + (static_cast<size_t>(ki) * n_chunks + chunk) * (dh + 2);
+    if (tid == 0) { rec[0] = m; rec[1] = l; }
+    const int n_valid = min(kAttnChunk, pos + 1 - chunk * kAttnChunk);
+    // o[j] = sum_p w_p V[p][j]: a thread takes one 16-byte column group and every (128 / groups)-th position,
+    // the position groups meet in shared memory
+    const int col_groups = dh / E;                      // 16-byte groups per value row
+    const int pos_groups = kAttnChunk / col_groups;     // threads per column group
+    const int cg = tid % col_groups, pg = tid / col_groups;
+    float part[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) part[e] = 0.0f;
+    if (pg < pos_groups) {
+        const uint4* vbase = reinterpret_cast<const uint4*>(Vc + (static_cast<size_t>(h) * Lmax + static_cast<size_t>(chunk) * kAttnChunk) * dh) + cg;
+#pragma unroll 4
+        for (int pp = pg; pp < n_valid; pp += pos_groups) {
+            float vf[E];
+            Elem<T>::widen(__ldg(vbase + static_cast<size_t>(pp) * col_groups), vf);
+            const float wp = w[pp];
+#pragma unroll
+            for (int e = 0; e < E; ++e) part[e] = fmaf(wp, vf[e], part[e]);
+        }
+    }
+    __syncthreads();                                    // q[] is no longer needed: reuse it as the meeting place
+    float* o_acc = q;
+    for (int j = tid; j < dh; j += kAttnChunk) o_acc[j] = 0.0f;
+    __syncthreads();
+    if (pg < pos_groups) {
+#pragma unroll
+        for (int e = 0; e < E; ++e) atomicAdd(&o_acc[cg * E + e], part[e]);
+    }
+    __syncthreads();
+    for (int j = tid; j < dh; j += kAttnChunk) rec[2 + j] = o_acc[j];
+}
+
+// combine the chunk partials of the block's 16 values o_j, then stream the 16 output-projection rows
+template <typename T, int ITERS>
+__global__ void __launch_bounds__(256)
+mha_out_kernel(int d, int H, int dh, const T* __restrict__ Wp, const int32_t* __restrict__ keep_list,
+               const int32_t* __restrict__ n_keep_ptr, const int32_t* __restrict__ dev_of_group, int n_dev,
+               const float* __restrict__ attn_ws, int n_chunks, float* __restrict__ partials, uint32_t* dev_status) {
+    constexpr int E = Elem<T>::kPerChunk;
+    __shared__ float o_s[kOutRows];
+    const int ki = blockIdx.x, j0 = blockIdx.y * kOutRows, tid = threadIdx.x;
+    int nk = *n_keep_ptr;
+    nk = max(0, min(nk, H));
+    if (ki >= nk) return;
+    const int h = keep_list[ki];
+    if (h < 0 || h >= H) return;   // flagged by the query kernel
+    int slot = 0;
+    if (dev_of_group) {
+        slot = dev_of_group[h] + 1;
+        if (slot < 0 || slot > n_dev) {
+            if (tid == 0 && j0 == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+            return;
+        }
+    }
+    if (tid < kOutRows) {
+        const float* rec0 = attn_ws + static_cast<size_t>(ki) * n_chunks * (dh + 2);
+        float M = -INFINITY;
+        for (int c = 0; c < n_chunks; ++c) M = fmaxf(M, rec0[static_cast<size_t>(c) * (dh + 2)]);
+        float L = 0.0f, o = 0.0f;
+        for (int c = 0; c < n_chunks; ++c) {
+            const float* rec = rec0 + static_cast<size_t>(c) * (dh + 2);
+            const float f = __expf(rec[0] - M);
+            L = fmaf(rec[1], f, L);
+            o = fmaf(rec[2 + j0 + tid], f, o);
+        }
+        o_s[tid] = o / L;
+    }
+    __syncthreads();
+    const int chunks = d / E;
+    float acc[ITERS][E];
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i)
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[i][e] = 0.0f;
+    const T* rows = Wp + ((static_cast<size_t>(h) * 2 + 1) * dh + j0) * d;
+    for (int jb = 0; jb < kOutRows; jb += 4) {
+        uint4 wv[4][ITERS];
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) {
+                const int c = tid + 256 * i;
+                if (c < chunks) wv[jj][i] = ldg_stream16(reinterpret_cast<const uint4*>(rows + static_cast<size_t>(jb + jj) * d) + c);
+            }
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const float o = o_s[jb + jj];
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) {
+                const int c = tid + 256 * i;
+                if (c < chunks) {
+                    float w8[E];
+                    Elem<T>::widen(wv[jj][i], w8);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc[i][e] = fmaf(o, w8[e], acc[i][e]);
+                }
+            }
+        }
+    }
+    float* dst = partials + static_cast<size_t>(slot) * d;
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+        const int c = tid + 256 * i;
+        if (c < chunks) {
+#pragma unroll
+            for (int e = 0; e < E; e += 4) red_add_v4f(dst + c * E + e, acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]);
+        }
+    }
+}
+
+template <typename T>
+__global__ void mha_pack_kernel(int d, int H, int dh, const T* __restrict__ Wq, const T* __restrict__ Wo, T* __restrict__ Wp) {
+    const size_t n = static_cast<size_t>(H) * dh * d;
+    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= n) return;
+    const int row = static_cast<int>(idx / d), c = static_cast<int>(idx % d);
+    const int h = row / dh, j = row % dh;
+    Wp[((static_cast<size_t>(h) * 2 + 0) * dh + j) * d + c] = Wq[idx];
+    Wp[((static_cast<size_t>(h) * 2 + 1) * dh + j) * d + c] = Wo[static_cast<size_t>(c) * H * dh + row];
+}
+
+}  // namespace halo
+
+using namespace halo;
+
+namespace {
+halo_status check_mha_shape(const halo_mha_shape* s) {
+    if (!s) return HALO_ERR_ARG;
+    if (s->wdtype != HALO_F32 && s->wdtype != HALO_BF16) return HALO_ERR_DTYPE;
+    if (s->d_model <= 0 || s->d_model % 8 != 0 || s->d_model > 8192 || s->n_heads <= 0 ||
+        s->n_heads > HALO_MAX_GROUPS || s->max_len <= 0)
+        return HALO_ERR_SHAPE;
+    if (s->head_dim < kOutRows || s->head_dim > 256 || s->head_dim % kOutRows != 0) return HALO_ERR_SHAPE;
+    const int per_chunk = s->wdtype == HALO_F32 ? 4 : 8;
+    if (s->d_model / per_chunk > 1024) return HALO_ERR_SHAPE;
+    return HALO_OK;
+}
+}  // namespace
+
+extern "C" halo_status halo_pack_mha_weights(const halo_mha_shape* shape, const void* Wq, const void* Wo, void* W_packed,
+                                             void* stream) {
+    halo_status rc = check_mha_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (!Wq || !Wo || !W_packed) return HALO_ERR_ARG;
+    const size_t n = static_cast<size_t>(shape->n_heads) * shape->head_dim * shape->d_model;
+    const unsigned blocks = static_cast<unsigned>((n + 255) / 256);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (shape->wdtype == HALO_BF16)
+        mha_pack_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(shape->d_model, shape->n_heads, shape->head_dim,
+                                                               static_cast<const __nv_bfloat16*>(Wq),
+                                                               static_cast<const __nv_bfloat16*>(Wo),
+                                                               static_cast<__nv_bfloat16*>(W_packed));
+    else
+        mha_pack_kernel<float><<<blocks, 256, 0, st>>>(shape->d_model, shape->n_heads, shape->head_dim,
+                                                       static_cast<const float*>(Wq), static_cast<const float*>(Wo),
+                                                       static_cast<float*>(W_packed));
+    return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+}
+
+extern "C" halo_status halo_mha_kv_append(const halo_mha_shape* shape, const void* Wk, const void* Wv, const void* x,
+                                          int pos, void* K_cache, void* V_cache, void* stream) {
+    halo_status rc = check_mha_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (!Wk || !Wv || !x || !K_cache || !V_cache) return HALO_ERR_ARG;
+    if (pos < 0 || pos >= shape->max_len) return HALO_ERR_ARG;
+    if (!aligned16(Wk) || !aligned16(Wv) || !aligned16(x) || !aligned16(K_cache) || !aligned16(V_cache)) return HALO_ERR_ALIGN;
+    const int d = shape->d_model, H = shape->n_heads, dh = shape->head_dim;
+    const unsigned blocks = static_cast<unsigned>((2 * H * dh + 7) / 8);
+    const size_t smem = sizeof(float) * d;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (shape->wdtype == HALO_BF16)
+        mha_kv_append_kernel<__nv_bfloat16><<<blocks, 256, smem, st>>>(
+            d, H, dh, shape->max_len, static_cast<const __nv_bfloat16*>(Wk), static_cast<const __nv_bfloat16*>(Wv),
+            static_cast<const __nv_bfloat16*>(x), pos, static_cast<__nv_bfloat16*>(K_cache),
+            static_cast<__nv_bfloat16*>(V_cache));
+    else
+        mha_kv_append_kernel<float><<<blocks, 256, smem, st>>>(d, H, dh, shape->max_len, static_cast<const float*>(Wk),
+                                                               static_cast<const float*>(Wv), static_cast<const float*>(x),
+                                                               pos, static_cast<float*>(K_cache),
+                                                               static_cast<float*>(V_cache));
+    return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+}
+
+extern "C" size_t halo_group_mha_workspace_bytes(const halo_mha_shape* shape) {
+    if (check_mha_shape(shape) != HALO_OK) return 0;
+    const size_t H = shape->n_heads, dh = shape->head_dim;
+    const size_t chunks = (static_cast<size_t>(shape->max_len) + kAttnChunk - 1) / kAttnChunk;
+    return sizeof(float) * (H * dh + H * chunks * (dh + 2));
+}
+
+template <typename T>
+static halo_status group_mha_typed(const halo_mha_shape& sh, const void* Wp, const void* x, const void* Kc, const void* Vc,
+                                   int pos, const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
+                                   int n_dev, float* partials, float* ws, uint32_t* dev_status, cudaStream_t st) {
+    constexpr int E = Elem<T>::kPerChunk;
+    const int d = sh.d_model, H = sh.n_heads, dh = sh.head_dim;
+    float* q_ws = ws;
+    float* attn_ws = ws + static_cast<size_t>(H) * dh;
+    const int n_chunks = pos / kAttnChunk + 1;
+    if (cudaMemsetAsync(partials, 0, sizeof(float) * static_cast<size_t>(n_dev + 1) * d, st) != cudaSuccess) return HALO_ERR_CUDA;
+    mha_q_kernel<T><<<(H * dh + 7) / 8, 256, sizeof(float) * d, st>>>(d, H, dh, static_cast<const T*>(Wp),
+                                                                      static_cast<const T*>(x), keep_list, n_keep, q_ws,
+                                                                      dev_status);
+    HALO_CHECK_LAUNCH();
+    mha_attn_kernel<T><<<dim3(H, n_chunks), kAttnChunk, 0, st>>>(H, dh, sh.max_len, pos, static_cast<const T*>(Kc),
+                                                                 static_cast<const T*>(Vc), keep_list, n_keep, q_ws,
+                                                                 attn_ws, n_chunks);
+    HALO_CHECK_LAUNCH();
+    const int iters = (d / E + 255) / 256;
+    const dim3 grid(H, dh / kOutRows);
+#define HALO_MHA_OUT(I)                                                                                              \
+    case I:                                                                                                          \
+        mha_out_kernel<T, I><<<grid, 256, 0, st>>>(d, H, dh, static_cast<const T*>(Wp), keep_list, n_keep, dev_of_group, \
+                                                   n_dev, attn_ws, n_chunks, partials, dev_status);                   \
+        break;
+    switch (iters) {
+        HALO_MHA_OUT(1)
+        HALO_MHA_OUT(2)
+        HALO_MHA_OUT(3)
+        HALO_MHA_OUT(4)
+        default: return HALO_ERR_SHAPE;
+    }
+#undef HALO_MHA_OUT
+    HALO_CHECK_LAUNCH();
+    return HALO_OK;
+}
+
+extern "C" halo_status halo_group_mha(const halo_mha_shape* shape, const void* W_packed, const void* x,
+                                      const void* K_cache, const void* V_cache, int pos, const int32_t* keep_list,
+                                      const int32_t* n_keep, const int32_t* dev_of_group, int n_dev, float* partials,
+                                      void* workspace, size_t workspace_bytes, uint32_t* dev_status, void* stream) {
+    halo_status rc = check_mha_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (!W_packed || !x || !K_cache || !V_cache || !keep_list || !n_keep || !partials) return HALO_ERR_ARG;
+    if (pos < 0 || pos >= shape->max_len) return HALO_ERR_ARG;
+    if (n_dev < 0 || n_dev > HALO_MAX_DEVICES || (!dev_of_group && n_dev != 0)) return HALO_ERR_ARG;
+    if (!aligned16(W_packed) || !aligned16(x) || !aligned16(K_cache) || !aligned16(V_cache) || !aligned16(partials) ||
+        !aligned16(workspace))
+        return HALO_ERR_ALIGN;
+    if (!workspace || workspace_bytes < halo_group_mha_workspace_bytes(shape)) return HALO_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* ws = static_cast<float*>(workspace);
+    if (shape->wdtype == HALO_BF16)
+        return group_mha_typed<__nv_bfloat16>(*shape, W_packed, x, K_cache, V_cache, pos, keep_list, n_keep, dev_of_group,
+                                              n_dev, partials, ws, dev_status, st);
+    return group_mha_typed<float>(*shape, W_packed, x, K_cache, V_cache, pos, keep_list, n_keep, dev_of_group, n_dev,
+                                  partials, ws, dev_status, st);
+}

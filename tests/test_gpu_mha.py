@@ -1,0 +1,116 @@
+"""GPU parity of the MHA neuron-group entry points against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import halo_ref as R
+from paper_2601_11676_b200 import binding as B
+from paper_2601_11676_b200 import synth
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+DEV = U.DEV
+
+
+def _wl(dtype, d, seed=0):
+    return synth.Workload("a", 1, d, 64, 16, 32, dtype, (0.0, 0.2, 0.6), (2, 1, 1), 500, 1, seed=seed)
+
+
+def _caches(wl, H, L, dh, fill):
+    g = torch.Generator(device=DEV).manual_seed(1234)
+    K = torch.zeros((H, L, dh), dtype=wl.torch_dtype, device=DEV)
+    V = torch.zeros((H, L, dh), dtype=wl.torch_dtype, device=DEV)
+    K[:, :fill] = torch.randn((H, fill, dh), generator=g, device=DEV).to(wl.torch_dtype)
+    V[:, :fill] = torch.randn((H, fill, dh), generator=g, device=DEV).to(wl.torch_dtype)
+    return K, V
+
+
+@pytest.mark.parametrize("dtype,d,H,dh,L,positions", [("f32", 64, 4, 16, 40, (0, 7, 39)), ("bf16", 512, 8, 64, 300, (0, 127, 128, 299)),
+                                                      ("bf16", 4096, 32, 128, 1024, (5, 700, 1023))])
+def test_group_mha_and_kv_append_match_oracle(dtype, d, H, dh, L, positions):
+    wl = _wl(dtype, d)
+    code = U.dtype_code(wl)
+    sh = B.mha_shape(d, H, dh, L, code)
+    Wq, Wk, Wv, Wo = synth.mha_matrices(wl, 0, H, DEV)
+    Wp = torch.empty((H, 2, dh, d), dtype=wl.torch_dtype, device=DEV)
+    B.halo_pack_mha_weights(sh, Wq, Wo, Wp)
+    torch.cuda.synchronize()
+    hb = synth.host_bits
+    Wp_ref = R.pack_mha(hb(Wq), hb(Wo), H)
+    assert (hb(Wp) == Wp_ref).all()                               # layout: bit exact
+    K, V = _caches(wl, H, L, dh, L)
+    ws = torch.empty(B.halo_group_mha_workspace_bytes(sh), dtype=torch.uint8, device=DEV)
+    tol = U.tol_for(wl)
+    dev = np.array([(-1, 0, 1, 2)[h % 4] for h in range(H)], dtype=np.int32)
+    dg = torch.as_tensor(dev, device=DEV)
+    for pos in positions:
+        x = synth.activation(wl, 50 + pos, DEV)
+        # keys / values of this token: within one rounding step of the oracle's
+        B.halo_mha_kv_append(sh, Wk, Wv, x, pos, K, V)
+        torch.cuda.synchronize()
+        Kh, Vh = hb(K), hb(V)
+        Kr, Vr = Kh.copy(), Vh.copy()
+        if d <= 512:                                              # the oracle's dense projection is slow at 4096
+            R.mha_kv_append(hb(Wk), hb(Wv), hb(x)[0], pos, Kr, Vr)
+            kk = R.to_f64(Kr[:, pos])
+            assert np.abs(R.to_f64(Kh[:, pos]) - kk).max() <= (1e-5 if dtype == "f32" else 2 ** -7) * np.abs(kk).max()
+            assert np.abs(R.to_f64(Vh[:, pos]) - R.to_f64(Vr[:, pos])).max() <= (1e-5 if dtype == "f32" else 2 ** -7) * np.abs(kk).max()
+        # attention of the kept heads, from the GPU's own cache bytes
+        for keep in (list(range(H)), [h for h in range(H) if h % 3 != 1], [H - 1], []):
+            kl = torch.full((H,), -1, dtype=torch.int32, device=DEV)
+            if keep:
+                kl[: len(keep)] = torch.as_tensor(keep, dtype=torch.int32, device=DEV)
+            nk = torch.tensor([len(keep)], dtype=torch.int32, device=DEV)
+            P = torch.full((4, d), float("nan"), dtype=torch.float32, device=DEV)
+            status = torch.zeros(1, dtype=torch.int32, device=DEV)
+            B.halo_group_mha(sh, Wp, x, K, V, pos, kl, nk, dg, 3, P, ws, status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            ref = R.group_mha(Wp_ref, hb(x)[0], Kh, Vh, pos, keep, dev, 3)
+            if not keep:
+                assert (P == 0).all().item()
+                continue
+            rms = np.sqrt(np.mean(ref.sum(0) ** 2))
+            assert np.abs(P.cpu().numpy() - ref).max() <= tol * rms, (pos, len(keep))
+            y = U.gpu_merge(P[:, None, :].contiguous()).cpu().numpy()[0]
+            assert U.rel_err(y, ref.sum(0)) <= tol
+
+
+def test_mha_heads_under_the_selection_machinery():
+    """Heads as groups: scores -> selection (Algorithm-3 chunks, arrival draw) -> kept heads -> merge."""
+    wl = synth.Workload("a", 1, 512, 64, 16, 32, "bf16", (0.0, 0.4, 0.9), (1, 1, 2), 375, 1)
+    H, dh, L, d = 8, 64, 64, 512
+    sh = B.mha_shape(d, H, dh, L, B.BF16)
+    Wq, Wk, Wv, Wo = synth.mha_matrices(wl, 0, H, DEV)
+    Wp = torch.empty((H, 2, dh, d), dtype=torch.bfloat16, device=DEV)
+    B.halo_pack_mha_weights(sh, Wq, Wo, Wp)
+    K, V = _caches(wl, H, L, dh, L)
+    plan = B.Plan(H, wl.loss_rate, wl.share_weight, B.SEL_TOPK, 3, 0.0, 77)
+    scores = torch.randn(H, generator=torch.Generator().manual_seed(3)).to(DEV)
+    ws = torch.empty(B.halo_group_mha_workspace_bytes(sh), dtype=torch.uint8, device=DEV)
+    hb = synth.host_bits
+    seen = set()
+    for step in range(12):
+        gpu, bufs = U.gpu_select(plan, scores, step, 2)
+        ref_sel = R.select(scores.cpu().numpy(), wl.loss_rate, wl.share_weight, R.SEL_TOPK, 3, 0.0, 77, step, 2)
+        U.assert_select_equal(gpu, ref_sel)
+        x = synth.activation(wl, step, DEV)
+        P = torch.empty((4, d), dtype=torch.float32, device=DEV)
+        B.halo_group_mha(sh, Wp, x, K, V, 40, bufs["keep_list"], bufs["n_keep"], bufs["dev_of_group"], 3, P, ws)
+        y = U.gpu_merge(P[:, None, :].contiguous(), gpu["arrived"]).cpu().numpy()[0]
+        ref = R.group_mha(hb(Wp), hb(x)[0], hb(K), hb(V), 40, ref_sel["keep_list"][: ref_sel["n_keep"]],
+                          ref_sel["dev_of_group"], 3)
+        assert U.rel_err(y, R.merge(ref[:, None, :], ref_sel["arrived"])[0]) <= U.TOL_BF16
+        seen.add(gpu["n_keep"])
+    assert len(seen) > 1
+
+
+def test_mha_argument_checks():
+    sh = B.mha_shape(512, 8, 60, 64, B.BF16)       # head_dim not a multiple of 16
+    assert B.halo_group_mha_workspace_bytes(sh) == 0
+    t = torch.zeros(16, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(B.HaloError):
+        B.halo_mha_kv_append(sh, t, t, t, 0, t, t)
+    ok = B.mha_shape(512, 8, 64, 64, B.BF16)
+    with pytest.raises(B.HaloError):
+        B.halo_mha_kv_append(ok, t, t, t, 64, t, t)   # position beyond the cache

@@ -260,13 +260,18 @@ namespace {
 // many tokens + bf16 + supported shape -> tensor-core contraction; otherwise the bandwidth-bound kernels
 halo_status dispatch_group_ffn(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group, int n_dev,
-                               float* partials, void* workspace, uint32_t* dev_status, cudaStream_t st) {
+                               float* partials, void* workspace, uint32_t* dev_status, cudaStream_t st,
+                               bool* collapsed = nullptr) {
     if (prefill_supported(sh, n_tok) && workspace) {
-        const size_t bytes = sizeof(float) * static_cast<size_t>(n_dev + 1) * n_tok * sh.d_model;
+        // a caller that passes `collapsed` only wants the merged sum: two slots (master / devices) are enough
+        const bool collapse = collapsed != nullptr && n_dev > 1;
+        if (collapsed) *collapsed = collapse;
+        const size_t bytes = sizeof(float) * static_cast<size_t>(collapse ? 2 : n_dev + 1) * n_tok * sh.d_model;
         if (cudaMemsetAsync(partials, 0, bytes, st) != cudaSuccess) return HALO_ERR_CUDA;
-        return launch_group_ffn_prefill(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, workspace,
-                                        dev_status, st);
+        return launch_group_ffn_prefill(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, collapse ? 1 : 0, partials,
+                                        workspace, dev_status, st);
     }
+    if (collapsed) *collapsed = false;
     return launch_group_ffn_decode(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, st);
 }
 }  // namespace
@@ -663,11 +668,13 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                     if (taps->n_keep) HALO_COPY(taps->n_keep + rec, s->set_nk[cur], sizeof(int32_t));
                     if (taps->y) y_tap = taps->y + rec * step_elems;
                 }
+                bool collapsed = false;   // only kept (= arrived) groups are computed: the sum is all we need
                 HALO_TRY(dispatch_group_ffn(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->set_kl[cur], s->set_nk[cur],
-                                            s->set_dev[cur], n_dev, s->partials, s->ffn_ws, s->status, st));
+                                            s->set_dev[cur], n_dev, s->partials, s->ffn_ws, s->status, st, &collapsed));
                 float* h_dst = (l == L - 1) ? h_out + sidx * step_elems : s->h;
-                HALO_TRY(launch_merge_glue(s->partials, s->set_arr[cur], n_dev, static_cast<int>(T), static_cast<int>(d),
-                                           s->ffn.wdtype, s->h, h_dst, x_next, y_tap, st));
+                HALO_TRY(launch_merge_glue(s->partials, collapsed ? nullptr : s->set_arr[cur], collapsed ? 1 : n_dev,
+                                           static_cast<int>(T), static_cast<int>(d), s->ffn.wdtype, s->h, h_dst, x_next,
+                                           y_tap, st));
                 launches += 2;
                 if (l + 1 < L) {
                     HALO_CU(cudaEventRecord(s->ev_x, st));             // x_{l+1} ready; set[cur] free again

@@ -187,7 +187,7 @@ template <int BN2, int STAGES>
 __global__ void __launch_bounds__(kPfThreads, 1)
 ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_wd, int T, int d,
                 int S, int G, const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
-                const int32_t* __restrict__ dev_of_group, int n_dev, float* __restrict__ partials,
+                const int32_t* __restrict__ dev_of_group, int n_dev, int collapse, float* __restrict__ partials,
                 uint32_t* dev_status) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = kBK * BN2 * 2, kStageBytes = kABytes + kBBytes;
@@ -199,7 +199,9 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
     int nk = *n_keep_ptr;
     nk = max(0, min(nk, G));
     const int k_per_group = S / kBK;   // K stages per kept group
-    const int n_slots = n_dev + 1;
+    // collapse: only two output slots, 0 = groups of the master, 1 = groups of any device (the caller wants the
+    // merged sum only and every listed group has arrived); still two slots so that K can be split over two CTAs
+    const int n_slots = collapse ? 2 : n_dev + 1;
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], 1); }
@@ -225,6 +227,7 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
                     g = keep_list[ki];
                     if (g >= 0 && g < G) sl = dev_of_group ? dev_of_group[g] + 1 : 0;
                     if (sl < 0 || sl > n_dev) { sl = -1; if (slot == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX); }
+                    else if (collapse && sl > 1) sl = 1;
                 }
                 const bool match = (sl == slot);
                 const unsigned ballot = __ballot_sync(0xffffffffu, match);
@@ -497,10 +500,11 @@ size_t prefill_workspace_bytes(const halo_ffn_shape& sh, int n_tok) {
     return static_cast<size_t>(n_tok) * sh.d_ffn * 2;   // H: bf16 [n_tok][d_ffn], kept groups packed to the left
 }
 
-// partials must already be zero (slots without kept groups are not written).
+// partials must already be zero (slots without kept groups are not written).  collapse != 0: partials has two
+// slots only, [0] = the master's groups, [1] = all devices' groups.
 halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                      const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
-                                     int n_dev, float* partials, void* workspace, uint32_t* dev_status,
+                                     int n_dev, int collapse, float* partials, void* workspace, uint32_t* dev_status,
                                      cudaStream_t st) {
     const int d = sh.d_model, S = sh.group_size, G = sh.d_ffn / S, T = n_tok;
     __nv_bfloat16* H = static_cast<__nv_bfloat16*>(workspace);
@@ -535,7 +539,7 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         static bool once2 = false;
         if (!once2) { if (!set_smem(k2, smem2)) return HALO_ERR_CUDA; once2 = true; }
         const dim3 grid2((T + kBM - 1) / kBM, d / 256, n_dev > 0 ? 2 : 1);
-        k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, partials,
+        k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, collapse, partials,
                                              dev_status);
     } else {
         constexpr int kStages2 = 6;
@@ -544,7 +548,7 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         static bool once2 = false;
         if (!once2) { if (!set_smem(k2, smem2)) return HALO_ERR_CUDA; once2 = true; }
         const dim3 grid2((T + kBM - 1) / kBM, d / 128, 1);
-        k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, partials,
+        k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, collapse, partials,
                                              dev_status);
     }
     HALO_CHECK_LAUNCH();

@@ -425,6 +425,7 @@ struct halo_stack {
     unsigned long long* trace;     // caller-owned, optional
     int trace_blocks;
     int cross_stages, l2_ahead;    // tuning of the persistent kernel
+    int max_steps_per_launch;      // 0 = derived from the counters' range
 };
 
 extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred,
@@ -531,6 +532,8 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     s->cross_stages = 1;
     s->l2_ahead = 0;
     if (const char* e = std::getenv("HALO_TUNE_CROSS_STAGES")) s->cross_stages = std::max(0, std::atoi(e));
+    s->max_steps_per_launch = 0;
+    if (const char* e = std::getenv("HALO_TUNE_MAX_STEPS")) s->max_steps_per_launch = std::max(0, std::atoi(e));
     if (const char* e = std::getenv("HALO_TUNE_L2_AHEAD")) s->l2_ahead = std::min(32, std::max(0, std::atoi(e)));
     s->persistent_ok = persistent_supported(*ffn, n_tok, G);
     {
@@ -620,10 +623,41 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                 if (!ok) return HALO_ERR_CUDA;
             }
         }
-        rc = launch_stack_persistent(P, st);
-        if (rc != HALO_OK) return rc;
-        s->last_launches = 1;
-        return HALO_OK;
+        // The kernel's 32-bit counters (barrier arrivals, hidden rows) grow with steps x blocks: very long runs are
+        // cut into several launches.
+        const long long per_step = static_cast<long long>(L) * std::max(s->pred.rank, 256);
+        int max_steps = static_cast<int>(std::max<long long>(1, (1ll << 30) / per_step));
+        if (s->max_steps_per_launch > 0) max_steps = std::min(max_steps, s->max_steps_per_launch);
+        long long n_launches = 0;
+        bool fell_back = false;
+        for (int done = 0; done < steps; done += max_steps) {
+            const int n = std::min(max_steps, steps - done);
+            if (done > 0 && (cudaMemsetAsync(s->p_partials, 0, sizeof(float) * 3 * 2 * d, st) != cudaSuccess ||
+                             cudaMemsetAsync(s->p_sync, 0, sizeof(unsigned) * 32, st) != cudaSuccess))
+                return HALO_ERR_CUDA;
+            P.steps = n;
+            P.step0 = step0 + static_cast<uint32_t>(done);
+            P.h0 = h0 + static_cast<size_t>(done) * step_elems;
+            P.h_out = h_out + static_cast<size_t>(done) * step_elems;
+            if (taps) {
+                const size_t rec = static_cast<size_t>(done) * L;
+                P.tap_x = taps->x ? static_cast<__nv_bfloat16*>(taps->x) + rec * step_elems : nullptr;
+                P.tap_scores = taps->scores ? taps->scores + rec * G : nullptr;
+                P.tap_dev_of_group = taps->dev_of_group ? taps->dev_of_group + rec * G : nullptr;
+                P.tap_arrived = taps->arrived ? taps->arrived + rec * n_dev : nullptr;
+                P.tap_keep_list = taps->keep_list ? taps->keep_list + rec * G : nullptr;
+                P.tap_n_keep = taps->n_keep ? taps->n_keep + rec : nullptr;
+                P.tap_y = taps->y ? taps->y + rec * step_elems : nullptr;
+            }
+            rc = launch_stack_persistent(P, st);
+            if (rc == HALO_ERR_UNIMPLEMENTED && done == 0) { fell_back = true; break; }   // not resident: loop path below
+            if (rc != HALO_OK) return rc;
+            ++n_launches;
+        }
+        if (!fell_back) {
+            s->last_launches = n_launches;
+            return HALO_OK;
+        }
     }
 #define HALO_TRY(call) do { rc = (call); if (rc != HALO_OK) return rc; } while (0)
 #define HALO_COPY(dst, src, bytes)                                                                    \

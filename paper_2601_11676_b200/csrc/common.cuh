@@ -27,6 +27,19 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 inline halo_status cuda_status(cudaError_t e) { return e == cudaSuccess ? HALO_OK : HALO_ERR_CUDA; }
 
+// Opt a kernel in to `bytes` of dynamic shared memory, once per device (the attribute is per device; the flag
+// array belongs to the calling site, one per kernel instantiation).
+template <typename Kernel>
+inline bool ensure_dynamic_smem(Kernel kernel, size_t bytes, bool (&done)[64]) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (done[dev]) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) != cudaSuccess)
+        return false;
+    done[dev] = true;
+    return true;
+}
+
 #define HALO_CHECK_LAUNCH()                                   \
     do {                                                      \
         cudaError_t e__ = cudaGetLastError();                 \

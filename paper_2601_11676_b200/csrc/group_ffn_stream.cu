@@ -223,12 +223,8 @@ halo_status launch_stream_cfg(const halo_ffn_shape& sh, const void* W, const voi
                               float* partials, uint32_t* dev_status, cudaStream_t st) {
     auto kernel = group_ffn_stream_kernel<NB, XC, P2, REP, STAGES>;
     const size_t smem = 1024 + static_cast<size_t>(STAGES) * 3 * NB * sh.d_model * 2;
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
-            return HALO_ERR_CUDA;
-        configured = true;
-    }
+    static bool configured[64] = {};
+    if (!ensure_dynamic_smem(kernel, smem, configured)) return HALO_ERR_CUDA;
     int dev = 0, sms = kSmCount;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int G = sh.d_ffn / sh.group_size;

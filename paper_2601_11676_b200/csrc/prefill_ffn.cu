@@ -484,11 +484,6 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <typename K>
-bool set_smem(K kernel, size_t bytes) {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) == cudaSuccess;
-}
-
 }  // namespace
 
 bool prefill_supported(const halo_ffn_shape& sh, int n_tok) {
@@ -519,8 +514,8 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         auto k1 = ffn_hidden_kernel<NS_, MH_, STAGES_>;                                                              \
         const size_t smem1 = static_cast<size_t>(STAGES_) * (MH_ * kBM * kBK * 2 + 2 * NS_ * kBK * 2) +              \
                              sizeof(PfBarriers) + 1024;                                                              \
-        static bool once1 = false;                                                                                   \
-        if (!once1) { if (!set_smem(k1, smem1)) return HALO_ERR_CUDA; once1 = true; }                                \
+        static bool once1[64] = {};                                                                                  \
+        if (!ensure_dynamic_smem(k1, smem1, once1)) return HALO_ERR_CUDA;                                            \
         const dim3 grid1((T + kBM * MH_ - 1) / (kBM * MH_), G);                                                      \
         k1<<<grid1, kPfThreads, smem1, st>>>(map_x, map_w, T, d, S, G, keep_list, n_keep, H, sh.d_ffn, dev_status);  \
     } while (0)
@@ -536,8 +531,8 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         constexpr int kStages2 = 4;
         auto k2 = ffn_down_kernel<256, kStages2>;
         const size_t smem2 = static_cast<size_t>(kStages2) * (kBM * kBK * 2 + kBK * 256 * 2) + sizeof(DownSmemTail) + 1024;
-        static bool once2 = false;
-        if (!once2) { if (!set_smem(k2, smem2)) return HALO_ERR_CUDA; once2 = true; }
+        static bool once2[64] = {};
+        if (!ensure_dynamic_smem(k2, smem2, once2)) return HALO_ERR_CUDA;
         const dim3 grid2((T + kBM - 1) / kBM, d / 256, n_dev > 0 ? 2 : 1);
         k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, collapse, partials,
                                              dev_status);
@@ -545,8 +540,8 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         constexpr int kStages2 = 6;
         auto k2 = ffn_down_kernel<128, kStages2>;
         const size_t smem2 = static_cast<size_t>(kStages2) * (kBM * kBK * 2 + kBK * 128 * 2) + sizeof(DownSmemTail) + 1024;
-        static bool once2 = false;
-        if (!once2) { if (!set_smem(k2, smem2)) return HALO_ERR_CUDA; once2 = true; }
+        static bool once2[64] = {};
+        if (!ensure_dynamic_smem(k2, smem2, once2)) return HALO_ERR_CUDA;
         const dim3 grid2((T + kBM - 1) / kBM, d / 128, 1);
         k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, collapse, partials,
                                              dev_status);
@@ -569,8 +564,8 @@ halo_status launch_pred_hidden_gemm(const halo_pred_shape& sh, const void* W1, c
     constexpr int kStages = 6;
     auto k = pred_hidden_gemm_kernel<kStages>;
     const size_t smem = static_cast<size_t>(kStages) * (kBM * kBK * 2 + 128 * kBK * 2) + sizeof(PfBarriers) + 1024;
-    static bool once = false;
-    if (!once) { if (!set_smem(k, smem)) return HALO_ERR_CUDA; once = true; }
+    static bool once[64] = {};
+    if (!ensure_dynamic_smem(k, smem, once)) return HALO_ERR_CUDA;
     const dim3 grid((n_tok + kBM - 1) / kBM, (sh.rank + 127) / 128);
     k<<<grid, kPfThreads, smem, st>>>(map_x, map_w1, n_tok, sh.d_in, sh.rank, sh.act, hidden, dev_status);
     HALO_CHECK_LAUNCH();

@@ -636,21 +636,25 @@ template <int NB, int XC, int P2, int REP, int STAGES>
 static halo_status launch_cfg(PersistParams& P, cudaStream_t st) {
     auto kernel = stack_decode_kernel<NB, XC, P2, REP, STAGES>;
     const size_t smem = kHeaderBytes + static_cast<size_t>(P.d) * 4 * REP + static_cast<size_t>(STAGES) * 3 * NB * P.d * 2;
-    static int blocks_per_sm = -1;
+    static bool configured[64] = {};
     int dev = 0, sms = kSmCount;
     if (cudaGetDevice(&dev) != cudaSuccess) return HALO_ERR_CUDA;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (blocks_per_sm < 0) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
-            return HALO_ERR_CUDA;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, kernel, kPThreads, smem) != cudaSuccess)
-            return HALO_ERR_CUDA;
-    }
-    if (blocks_per_sm < 1) return HALO_ERR_CUDA;
-    void* args[] = {&P};
-    if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(sms), dim3(kPThreads), args, smem, st) != cudaSuccess)
+    if (!ensure_dynamic_smem(kernel, smem, configured)) return HALO_ERR_CUDA;
+    int blocks_per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, kernel, kPThreads, smem) != cudaSuccess)
         return HALO_ERR_CUDA;
-    return HALO_OK;
+    if (blocks_per_sm < 1 || sms < 2) return HALO_ERR_UNIMPLEMENTED;   // cannot be made resident: caller falls back
+    void* args[] = {&P};
+    const cudaError_t err = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(sms), dim3(kPThreads), args,
+                                                        smem, st);
+    if (err == cudaErrorCooperativeLaunchTooLarge) {
+        // the SMs are not all ours (another context on the device): not an error of this call, the caller runs the
+        // one-launch-per-step path instead
+        (void)cudaGetLastError();
+        return HALO_ERR_UNIMPLEMENTED;
+    }
+    return err == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
 }
 
 halo_status launch_stack_persistent(PersistParams& P, cudaStream_t st) {

@@ -211,3 +211,20 @@ def test_stack_persistent_variants(variant):
     if variant == "threshold":
         nk = t["n_keep"][:, 1:].cpu().numpy()
         assert nk.min() < wl.n_groups and len(np.unique(nk)) > 1   # the critical count really varies with the scores
+
+
+def test_long_runs_are_split_into_several_persistent_launches(monkeypatch):
+    """The persistent kernel's counters are 32 bit, so very long runs are cut into several launches; forced here
+    with a tiny limit: the arrival draws and records must continue seamlessly across the cut."""
+    monkeypatch.setenv("HALO_TUNE_MAX_STEPS", "2")
+    wl = synth.Workload("c", 3, 2048, 64 * 10, 64, 128, "bf16", (0.0, 0.4, 0.8), (1, 1, 1), 300, 5)
+    stack, Wp, preds = build_stack(wl)
+    monkeypatch.delenv("HALO_TUNE_MAX_STEPS")
+    h0, h_out, t = run_with_taps(wl, stack, wl.steps, step0=11)
+    assert stack.last_launches() == 3
+    check_teacher_forced(wl, Wp, preds, h0, h_out, t, wl.steps, step0=11)
+    ref_stack, _, _ = build_stack(wl)
+    _, h_ref, t_ref = run_with_taps(wl, ref_stack, wl.steps, step0=11)
+    assert ref_stack.last_launches() == 1
+    assert (t["keep_list"] == t_ref["keep_list"]).all().item() and (t["n_keep"] == t_ref["n_keep"]).all().item()
+    assert (h_out - h_ref).abs().max().item() <= 1e-3 * h_ref.abs().max().item()

@@ -24,6 +24,8 @@ constexpr int kBM = 128;          // tokens per tile
 constexpr int kBK = 64;           // K elements per stage (128 bytes of bf16)
 constexpr int kUmmaK = 16;
 constexpr int kPfThreads = 192;   // 6 warps
+constexpr int kEpiPitch = 36;     // floats per staged accumulator row: 32 + 4 keeps 16-byte accesses conflict-free
+constexpr size_t kEpiStageBytes = 4 * 32 * kEpiPitch * sizeof(float);   // one 32 x 32 chunk per epilogue warp
 
 struct PfBarriers {
     uint64_t full[8];
@@ -48,8 +50,9 @@ __device__ __forceinline__ bool pf_wait(uint64_t* bar, uint32_t parity, volatile
 // tokens: twice the FLOP per staged byte, four fp32 accumulators = all 512 TMEM columns at NS = 128.
 template <int NS, int MH, int STAGES>
 __global__ void __launch_bounds__(kPfThreads, 1)
-ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w, int T, int d,
-                  int S, int G, const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
+ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                  const __grid_constant__ CUtensorMap tmap_w_half, int T, int d, int S, int G, int n_sm,
+                  const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
                   __nv_bfloat16* __restrict__ H, int h_cols, uint32_t* dev_status) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     constexpr uint32_t kAHalf = kBM * kBK * 2, kABytes = MH * kAHalf, kBBytes = NS * kBK * 2;
@@ -61,6 +64,22 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     int nk = *n_keep_ptr;
     nk = max(0, min(nk, G));
     if (ki >= nk) return;
+    // Tail balancing: the kept groups that fill whole waves of SMs are computed as full tiles (blockIdx.z == 0);
+    // the groups left for the last, partial wave are split into two half-width tiles (blockIdx.z = which half),
+    // when those halves fit in one wave, so the tail takes about half a tile's time.
+    int n_full = nk;
+    {
+        const int tiles_x = gridDim.x, total = tiles_x * nk;
+        if (total > n_sm) {
+            const int full_groups = (total / n_sm) * n_sm / tiles_x, left = nk - full_groups;
+            if (left > 0 && 2 * left * tiles_x <= n_sm) n_full = full_groups;
+        }
+    }
+    const bool split = ki >= n_full;
+    if (!split && blockIdx.z != 0) return;
+    const int ns = split ? NS / 2 : NS;                // neurons of the group this CTA computes
+    const int n_off = split ? blockIdx.z * (NS / 2) : 0;
+    const CUtensorMap* const map_w = split ? &tmap_w_half : &tmap_w;
     const int g = keep_list[ki];
     if (g < 0 || g >= G) {
         if (tid == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
@@ -75,7 +94,7 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         bars.abort_flag = 0;
         mbar_fence_init();
         tma_prefetch_descriptor(&tmap_x);
-        tma_prefetch_descriptor(&tmap_w);
+        tma_prefetch_descriptor(map_w);
     }
     if (warp == 1) { tmem_alloc(&bars.tmem_base, kTmemCols); tmem_relinquish_alloc_permit(); }
     tcgen05_fence_before_sync();
@@ -91,12 +110,13 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 const int s = kt % STAGES;
                 if (kt >= STAGES && !pf_wait(&bars.empty[s], ((kt / STAGES) - 1) & 1, abort_flag)) break;
                 unsigned char* st = smem_raw + static_cast<size_t>(s) * kStageBytes;
-                mbar_arrive_expect_tx(&bars.full[s], kStageBytes);
+                mbar_arrive_expect_tx(&bars.full[s], kABytes + 2u * static_cast<uint32_t>(ns) * kBK * 2u);
 #pragma unroll
                 for (int mh = 0; mh < MH; ++mh)   // rows beyond T read as zeros
                     tma_load_2d(st + mh * kAHalf, &tmap_x, kt * kBK, m0 + mh * kBM, &bars.full[s]);
-                tma_load_2d(st + kABytes, &tmap_w, kt * kBK, (g * 3 + 0) * S, &bars.full[s]);
-                tma_load_2d(st + kABytes + kBBytes, &tmap_w, kt * kBK, (g * 3 + 1) * S, &bars.full[s]);
+                // gate rows, then the up rows directly behind them: one B operand of 2 * ns rows
+                tma_load_2d(st + kABytes, map_w, kt * kBK, (g * 3 + 0) * S + n_off, &bars.full[s]);
+                tma_load_2d(st + kABytes + ns * (kBK * 2), map_w, kt * kBK, (g * 3 + 1) * S + n_off, &bars.full[s]);
                 issued = kt + 1;
             }
             if (*abort_flag) {  // let outstanding copies land before the CTA goes away
@@ -107,7 +127,9 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(kBM, NS, false);
+            // one MMA of N = 2 * ns per token half: accumulator columns [0, ns) = gate, [ns, 2 ns) = up.  The wide
+            // N keeps the A tile's shared-memory reads per FLOP low.
+            const uint32_t idesc = umma_idesc_bf16(kBM, 2 * ns, false);
             for (int kt = 0; kt < n_kt; ++kt) {
                 const int s = kt % STAGES;
                 if (!pf_wait(&bars.full[s], (kt / STAGES) & 1, abort_flag)) break;
@@ -115,14 +137,12 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
                 const uint32_t a0 = smem_u32(smem_raw + static_cast<size_t>(s) * kStageBytes);
 #pragma unroll
                 for (int kk = 0; kk < kBK / kUmmaK; ++kk) {
-                    const uint64_t bg = umma_smem_desc(a0 + kABytes + kk * 32, 16, 1024);
-                    const uint64_t bu = umma_smem_desc(a0 + kABytes + kBBytes + kk * 32, 16, 1024);
+                    const uint64_t b = umma_smem_desc(a0 + kABytes + kk * 32, 16, 1024);
                     const bool accumulate = (kt > 0) || (kk > 0);
 #pragma unroll
                     for (int mh = 0; mh < MH; ++mh) {
                         const uint64_t a = umma_smem_desc(a0 + mh * kAHalf + kk * 32, 16, 1024);
-                        umma_bf16(tmem + mh * 2 * NS, a, bg, idesc, accumulate);
-                        umma_bf16(tmem + mh * 2 * NS + NS, a, bu, idesc, accumulate);
+                        umma_bf16(tmem + mh * 2 * NS, a, b, idesc, accumulate);
                     }
                 }
                 umma_commit(&bars.empty[s]);   // the stage is free once these MMAs have read it
@@ -138,13 +158,14 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
 #pragma unroll
         for (int mh = 0; mh < MH; ++mh) {
             const int row = m0 + mh * kBM + quad * 32 + lane;
-            for (int c0 = 0; c0 < NS; c0 += 32) {
+            for (int c0 = 0; c0 < ns; c0 += 32) {
                 uint32_t dg[32], du[32];
                 tmem_ld_32x32(lane_base + mh * 2 * NS + c0, dg);
-                tmem_ld_32x32(lane_base + mh * 2 * NS + NS + c0, du);
+                tmem_ld_32x32(lane_base + mh * 2 * NS + ns + c0, du);
                 tmem_ld_wait();
                 if (ok && row < T) {
-                    uint4* dst = reinterpret_cast<uint4*>(H + static_cast<size_t>(row) * h_cols + static_cast<size_t>(ki) * S + c0);
+                    uint4* dst = reinterpret_cast<uint4*>(H + static_cast<size_t>(row) * h_cols +
+                                                          static_cast<size_t>(ki) * S + n_off + c0);
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         uint32_t packed[4];
@@ -181,6 +202,38 @@ struct DownSmemTail {
     int16_t kept_pos[HALO_MAX_GROUPS];    // kept position (column block of H) per position of the order
 };
 
+// Kept positions sorted by holder slot (stable), by one warp with ballot compaction per slot.  Slots above
+// `slot_cap` are folded into slot_cap.  Fills slot_start[0 .. n_slots), group_of and kept_pos; returns the number of
+// valid kept positions.
+__device__ __forceinline__ int build_slot_order(DownSmemTail& tail, int nk, int G, int n_dev, int n_slots, int slot_cap,
+                                                const int32_t* __restrict__ keep_list,
+                                                const int32_t* __restrict__ dev_of_group, uint32_t* dev_status,
+                                                int lane) {
+    int pos = 0;
+    for (int slot = 0; slot < n_slots; ++slot) {
+        if (lane == 0) tail.slot_start[slot] = pos;
+        for (int base = 0; base < nk; base += 32) {
+            const int ki = base + lane;
+            int g = -1, sl = -1;
+            if (ki < nk) {
+                g = keep_list[ki];
+                if (g >= 0 && g < G) sl = dev_of_group ? dev_of_group[g] + 1 : 0;
+                if (sl < 0 || sl > n_dev) { sl = -1; if (slot == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX); }
+                else if (sl > slot_cap) sl = slot_cap;
+            }
+            const bool match = (sl == slot);
+            const unsigned ballot = __ballot_sync(0xffffffffu, match);
+            if (match) {
+                const int p = pos + __popc(ballot & ((1u << lane) - 1u));
+                tail.group_of[p] = g;
+                tail.kept_pos[p] = static_cast<int16_t>(ki);
+            }
+            pos += __popc(ballot);
+        }
+    }
+    return pos;
+}
+
 // BN2 output columns per tile.  gridDim.z CTAs share an output tile position but take disjoint ranges of holder
 // slots: the slots are separate outputs, so splitting K at a slot boundary needs no reduction.
 template <int BN2, int STAGES>
@@ -216,29 +269,8 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
     // two accumulators: the MMAs of the next slot run while the epilogue drains the previous one
     if (warp == 1) { tmem_alloc(&bars.tmem_base, 2 * BN2); tmem_relinquish_alloc_permit(); }
     if (warp == 0) {
-        // kept positions sorted by holder slot (stable): one warp, ballot compaction per slot
-        int pos = 0;
-        for (int slot = 0; slot < n_slots; ++slot) {
-            if (lane == 0) tail.slot_start[slot] = pos;
-            for (int base = 0; base < nk; base += 32) {
-                const int ki = base + lane;
-                int g = -1, sl = -1;
-                if (ki < nk) {
-                    g = keep_list[ki];
-                    if (g >= 0 && g < G) sl = dev_of_group ? dev_of_group[g] + 1 : 0;
-                    if (sl < 0 || sl > n_dev) { sl = -1; if (slot == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX); }
-                    else if (collapse && sl > 1) sl = 1;
-                }
-                const bool match = (sl == slot);
-                const unsigned ballot = __ballot_sync(0xffffffffu, match);
-                if (match) {
-                    const int p = pos + __popc(ballot & ((1u << lane) - 1u));
-                    tail.group_of[p] = g;
-                    tail.kept_pos[p] = static_cast<int16_t>(ki);
-                }
-                pos += __popc(ballot);
-            }
-        }
+        const int pos = build_slot_order(tail, nk, G, n_dev, n_slots, collapse ? 1 : n_dev, keep_list, dev_of_group,
+                                         dev_status, lane);
         if (lane == 0) {
             tail.slot_start[n_slots] = pos;
             // this CTA's share of the slots: cut at the slot boundary nearest to half of the kept groups
@@ -350,6 +382,170 @@ ffn_down_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constan
     tcgen05_fence_before_sync();
     __syncthreads();
     if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, 2 * BN2); }
+    if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
+}
+
+// Down projection for prompts of more than one 128-token tile: 256 tokens x 256 output columns per CTA (two
+// accumulators of 256 TMEM columns), so that each staged byte feeds 1.5x the FLOPs of the 128-token tile.  The K
+// range (kept groups in slot order) is cut into gridDim.z equal runs of 64-deep K tiles; every CTA adds its
+// accumulators into the zeroed output slots with vector reductions, so a cut may fall anywhere.  A run that crosses
+// a slot boundary drains the accumulators there and starts the next slot from zero.
+template <int STAGES>
+__global__ void __launch_bounds__(kPfThreads, 1)
+ffn_down_wide_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_wd, int T,
+                     int d, int S, int G, const int32_t* __restrict__ keep_list,
+                     const int32_t* __restrict__ n_keep_ptr, const int32_t* __restrict__ dev_of_group, int n_dev,
+                     int collapse, float* __restrict__ partials, uint32_t* dev_status) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    constexpr int BN2 = 256, MH = 2;
+    constexpr uint32_t kAHalf = kBM * kBK * 2, kABytes = MH * kAHalf, kBBytes = kBK * BN2 * 2;
+    constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    constexpr uint32_t kBBlock = kBK * 64 * 2;
+    DownSmemTail& tail = *reinterpret_cast<DownSmemTail*>(smem_raw + static_cast<size_t>(STAGES) * kStageBytes);
+    float* const epi_stage = reinterpret_cast<float*>(smem_raw + static_cast<size_t>(STAGES) * kStageBytes +
+                                                      ((sizeof(DownSmemTail) + 15) & ~size_t(15)));
+    PfBarriers& bars = tail.bars;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.x * (kBM * MH), n0 = blockIdx.y * BN2;
+    int nk = *n_keep_ptr;
+    nk = max(0, min(nk, G));
+    const int k_per_group = S / kBK;
+    // collapse: the caller wants the sum over holders only and every listed group has arrived: one slot
+    const int n_slots = collapse ? 1 : n_dev + 1;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], 1); }
+        mbar_init(&bars.tmem_full, 1);
+        mbar_init(&bars.tmem_empty, 4);
+        mbar_init(&tail.acc_full[0], 1);
+        mbar_init(&tail.acc_empty[0], 4);
+        bars.abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_descriptor(&tmap_h);
+        tma_prefetch_descriptor(&tmap_wd);
+    }
+    if (warp == 1) { tmem_alloc(&bars.tmem_base, MH * BN2); tmem_relinquish_alloc_permit(); }
+    if (warp == 0) {
+        const int pos = build_slot_order(tail, nk, G, n_dev, n_slots, n_slots - 1, keep_list, dev_of_group, dev_status,
+                                         lane);
+        if (lane == 0) {
+            tail.slot_start[n_slots] = pos;
+            // this CTA's run of K tiles, [slot_lo, slot_hi) reused as the K-tile bounds
+            const long long units = static_cast<long long>(pos) * k_per_group;
+            tail.slot_lo = static_cast<int>(units * blockIdx.z / gridDim.z);
+            tail.slot_hi = static_cast<int>(units * (blockIdx.z + 1) / gridDim.z);
+        }
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    volatile int* abort_flag = &bars.abort_flag;
+    const uint32_t tmem = bars.tmem_base;
+    const int kt_lo = tail.slot_lo, kt_hi = tail.slot_hi;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int it = 0;
+            for (int kt = kt_lo; kt < kt_hi; ++kt, ++it) {
+                const int p = kt / k_per_group, kk2 = kt - p * k_per_group;
+                const int g = tail.group_of[p], kp = tail.kept_pos[p];
+                const int s = it % STAGES;
+                if (it >= STAGES && !pf_wait(&bars.empty[s], ((it / STAGES) - 1) & 1, abort_flag)) break;
+                unsigned char* st = smem_raw + static_cast<size_t>(s) * kStageBytes;
+                mbar_arrive_expect_tx(&bars.full[s], kStageBytes);
+#pragma unroll
+                for (int mh = 0; mh < MH; ++mh)   // rows beyond T read as zeros
+                    tma_load_2d(st + mh * kAHalf, &tmap_h, kp * S + kk2 * kBK, m0 + mh * kBM, &bars.full[s]);
+                const int krow = (g * 3 + 2) * S + kk2 * kBK;
+#pragma unroll
+                for (int nb = 0; nb < BN2 / 64; ++nb)
+                    tma_load_2d(st + kABytes + nb * kBBlock, &tmap_wd, n0 + nb * 64, krow, &bars.full[s]);
+            }
+            if (*abort_flag) {
+                int never = 0;
+                for (int k = max(0, it - STAGES); k < it; ++k)
+                    mbar_wait_bounded(&bars.full[k % STAGES], (k / STAGES) & 1, &never);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(kBM, BN2, true);
+            int it = 0, seg = 0;
+            bool alive = true;
+            for (int slot = 0; slot < n_slots && alive; ++slot) {
+                const int k0 = max(kt_lo, tail.slot_start[slot] * k_per_group);
+                const int k1 = min(kt_hi, tail.slot_start[slot + 1] * k_per_group);
+                if (k0 >= k1) continue;
+                // one accumulator set: the previous segment must have been drained
+                if (seg >= 1 && !pf_wait(&tail.acc_empty[0], (seg - 1) & 1, abort_flag)) break;
+                tcgen05_fence_after_sync();
+                for (int kt = k0; kt < k1; ++kt, ++it) {
+                    const int s = it % STAGES;
+                    if (!pf_wait(&bars.full[s], (it / STAGES) & 1, abort_flag)) { alive = false; break; }
+                    tcgen05_fence_after_sync();
+                    const uint32_t a0 = smem_u32(smem_raw + static_cast<size_t>(s) * kStageBytes);
+#pragma unroll
+                    for (int kk = 0; kk < kBK / kUmmaK; ++kk) {
+                        const uint64_t b = umma_smem_desc(a0 + kABytes + kk * 2048, kBBlock, 1024);
+#pragma unroll
+                        for (int mh = 0; mh < MH; ++mh) {
+                            const uint64_t a = umma_smem_desc(a0 + mh * kAHalf + kk * 32, 16, 1024);
+                            umma_bf16(tmem + mh * BN2, a, b, idesc, (kt > k0) || (kk > 0));
+                        }
+                    }
+                    umma_commit(&bars.empty[s]);
+                }
+                if (!alive) break;
+                umma_commit(&tail.acc_full[0]);
+                ++seg;
+            }
+        }
+    } else {
+        const int quad = warp & 3;
+        const uint32_t lane_base = tmem + (static_cast<uint32_t>(quad * 32) << 16);
+        int seg = 0;
+        for (int slot = 0; slot < n_slots; ++slot) {
+            const int k0 = max(kt_lo, tail.slot_start[slot] * k_per_group);
+            const int k1 = min(kt_hi, tail.slot_start[slot + 1] * k_per_group);
+            if (k0 >= k1) continue;
+            const bool ok = pf_wait(&tail.acc_full[0], seg & 1, abort_flag);
+            tcgen05_fence_after_sync();
+            // Each thread holds one token row of the accumulator; the 32 x 32 chunk is turned through shared memory
+            // so that one reduction instruction covers 4 rows x 128 contiguous bytes instead of 32 rows x 16.
+            float* stage = epi_stage + (warp - 2) * (32 * kEpiPitch);
+#pragma unroll
+            for (int mh = 0; mh < MH; ++mh) {
+                const int row0 = m0 + mh * kBM + quad * 32;
+                float* out = partials + (static_cast<size_t>(slot) * T + row0) * d + n0;
+                for (int c0 = 0; c0 < BN2; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(lane_base + mh * BN2 + c0, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        *reinterpret_cast<float4*>(stage + lane * kEpiPitch + 4 * q) =
+                            make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                        __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int r = 4 * j + (lane >> 3), cq = (lane & 7) * 4;
+                        const float4 w = *reinterpret_cast<const float4*>(stage + r * kEpiPitch + cq);
+                        if (ok && row0 + r < T)
+                            red_add_v4f(out + static_cast<size_t>(r) * d + c0 + cq, w.x, w.y, w.z, w.w);
+                    }
+                    __syncwarp();
+                }
+            }
+            tcgen05_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tail.acc_empty[0]);
+            ++seg;
+        }
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, MH * BN2); }
     if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
 }
 
@@ -504,8 +700,13 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
     const int d = sh.d_model, S = sh.group_size, G = sh.d_ffn / S, T = n_tok;
     __nv_bfloat16* H = static_cast<__nv_bfloat16*>(workspace);
     const uint64_t w_rows = static_cast<uint64_t>(G) * 3 * S;
-    CUtensorMap map_x, map_w, map_h, map_wd;
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return HALO_ERR_CUDA;
+    CUtensorMap map_x, map_w, map_w_half, map_h, map_wd;
     if (!make_map(&map_x, x, T, d, d, kBK, kBM) || !make_map(&map_w, W, w_rows, d, d, kBK, S) ||
+        !make_map(&map_w_half, W, w_rows, d, d, kBK, S / 2) ||
         !make_map(&map_h, H, T, sh.d_ffn, sh.d_ffn, kBK, kBM) || !make_map(&map_wd, W, w_rows, d, d, 64, kBK))
         return HALO_ERR_CUDA;
     // GEMM-1: 256-token tiles when the prompt has them (more FLOP per staged byte), else 128-token tiles
@@ -516,8 +717,9 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
                              sizeof(PfBarriers) + 1024;                                                              \
         static bool once1[64] = {};                                                                                  \
         if (!ensure_dynamic_smem(k1, smem1, once1)) return HALO_ERR_CUDA;                                            \
-        const dim3 grid1((T + kBM * MH_ - 1) / (kBM * MH_), G);                                                      \
-        k1<<<grid1, kPfThreads, smem1, st>>>(map_x, map_w, T, d, S, G, keep_list, n_keep, H, sh.d_ffn, dev_status);  \
+        const dim3 grid1((T + kBM * MH_ - 1) / (kBM * MH_), G, 2);                                                   \
+        k1<<<grid1, kPfThreads, smem1, st>>>(map_x, map_w, map_w_half, T, d, S, G, n_sm, keep_list, n_keep, H,       \
+                                             sh.d_ffn, dev_status);                                                  \
     } while (0)
     if (S == 128) {
         if (T > kBM) HALO_LAUNCH_HIDDEN(128, 2, 3); else HALO_LAUNCH_HIDDEN(128, 1, 4);
@@ -526,7 +728,20 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
     }
 #undef HALO_LAUNCH_HIDDEN
     HALO_CHECK_LAUNCH();
-    if (d % 256 == 0) {
+    if (d % 256 == 0 && T > kBM) {
+        // 256 x 256 tiles; K cut into as many runs as fill the SMs once
+        constexpr int kStages2 = 3;
+        auto k2 = ffn_down_wide_kernel<kStages2>;
+        const size_t smem2 = static_cast<size_t>(kStages2) * (2 * kBM * kBK * 2 + kBK * 256 * 2) + sizeof(DownSmemTail) +
+                             16 + kEpiStageBytes + 1024;
+        static bool once2[64] = {};
+        if (!ensure_dynamic_smem(k2, smem2, once2)) return HALO_ERR_CUDA;
+        const int tiles = ((T + 2 * kBM - 1) / (2 * kBM)) * (d / 256);
+        const int z = std::max(1, std::min(8, n_sm / tiles));
+        const dim3 grid2((T + 2 * kBM - 1) / (2 * kBM), d / 256, z);
+        k2<<<grid2, kPfThreads, smem2, st>>>(map_h, map_wd, T, d, S, G, keep_list, n_keep, dev_of_group, n_dev, collapse,
+                                             partials, dev_status);
+    } else if (d % 256 == 0) {
         // 256-column tiles (more FLOP per staged byte); with holder slots the K range is split over two CTAs
         constexpr int kStages2 = 4;
         auto k2 = ffn_down_kernel<256, kStages2>;

@@ -36,6 +36,22 @@ def test_prefill_ffn_small_shapes_all_tokens(d, G, S, n_tok):
             assert (P == 0).all().item()
 
 
+@pytest.mark.parametrize("d,G,S,n_tok", [(256, 160, 64, 100), (256, 80, 128, 300), (128, 150, 128, 129)])
+def test_prefill_more_tiles_than_sms_splits_the_last_wave(d, G, S, n_tok):
+    """With more hidden-layer tiles than SMs the groups of the last wave are computed as two half-width tiles
+    each; every token of every kept group is checked, with all groups kept and with a ragged kept list."""
+    wl = _wl(d, G, S)
+    Wp = synth.packed_layer(wl, 0, DEV)
+    x = synth.activation(wl, 1, DEV, n_tok=n_tok)
+    dev = (np.arange(G, dtype=np.int32) % 4) - 1
+    for keep in (list(range(G)), [g for g in range(G) if g % 17 != 3]):
+        P, status = U.gpu_group_ffn(wl, Wp, x, keep, dev, wl.n_dev)
+        ref = R.group_ffn(synth.host_bits(Wp), synth.host_bits(x), keep, dev, wl.n_dev)
+        assert status == 0
+        rms = np.sqrt(np.mean(R.merge(ref) ** 2))
+        assert np.abs(P.cpu().numpy() - ref).max() <= U.TOL_BF16 * rms, len(keep)
+
+
 def test_prefill_matches_decode_path_token_by_token():
     wl = _wl(512, 4, 128)
     Wp = synth.packed_layer(wl, 0, DEV)

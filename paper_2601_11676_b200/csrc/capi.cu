@@ -702,14 +702,26 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                     if (taps->n_keep) HALO_COPY(taps->n_keep + rec, s->set_nk[cur], sizeof(int32_t));
                     if (taps->y) y_tap = taps->y + rec * step_elems;
                 }
-                bool collapsed = false;   // only kept (= arrived) groups are computed: the sum is all we need
-                HALO_TRY(dispatch_group_ffn(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->set_kl[cur], s->set_nk[cur],
-                                            s->set_dev[cur], n_dev, s->partials, s->ffn_ws, s->status, st, &collapsed));
                 float* h_dst = (l == L - 1) ? h_out + sidx * step_elems : s->h;
-                HALO_TRY(launch_merge_glue(s->partials, collapsed ? nullptr : s->set_arr[cur], collapsed ? 1 : n_dev,
-                                           static_cast<int>(T), static_cast<int>(d), s->ffn.wdtype, s->h, h_dst, x_next,
-                                           y_tap, st));
-                launches += 2;
+                if (!y_tap && s->ffn_ws && prefill_accumulates(s->ffn, static_cast<int>(T))) {
+                    // only kept (= arrived) groups are computed and nobody asked for y itself: the down projection
+                    // adds its tiles straight into the residual stream, and the glue only normalises
+                    HALO_TRY(launch_group_ffn_prefill(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->set_kl[cur],
+                                                      s->set_nk[cur], s->set_dev[cur], n_dev, 1, s->h, s->ffn_ws,
+                                                      s->status, st));
+                    HALO_TRY(launch_glue(static_cast<int>(d), static_cast<int>(T), s->ffn.wdtype, s->h, nullptr, h_dst,
+                                         x_next, st));
+                    launches += 3;
+                } else {
+                    bool collapsed = false;   // the sum over holders is all the glue needs
+                    HALO_TRY(dispatch_group_ffn(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->set_kl[cur],
+                                                s->set_nk[cur], s->set_dev[cur], n_dev, s->partials, s->ffn_ws,
+                                                s->status, st, &collapsed));
+                    HALO_TRY(launch_merge_glue(s->partials, collapsed ? nullptr : s->set_arr[cur],
+                                               collapsed ? 1 : n_dev, static_cast<int>(T), static_cast<int>(d),
+                                               s->ffn.wdtype, s->h, h_dst, x_next, y_tap, st));
+                    launches += 2;
+                }
                 if (l + 1 < L) {
                     HALO_CU(cudaEventRecord(s->ev_x, st));             // x_{l+1} ready; set[cur] free again
                     // join: block l+1 needs its selection, and the glue of block l+1 will overwrite the x that the

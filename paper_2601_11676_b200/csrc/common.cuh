@@ -116,6 +116,9 @@ halo_status launch_group_ffn_stream(const halo_ffn_shape& sh, const void* W, con
 // Prefill form (tensor cores); workspace = bf16 [n_tok][d_ffn]; partials must already be zero.
 bool prefill_supported(const halo_ffn_shape& sh, int n_tok);
 size_t prefill_workspace_bytes(const halo_ffn_shape& sh, int n_tok);
+// true when launch_group_ffn_prefill with collapse != 0 ADDS into slot 0 of `partials` (K-split reductions), so the
+// caller may pass a buffer that already holds a value to add to
+bool prefill_accumulates(const halo_ffn_shape& sh, int n_tok);
 halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                      const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
                                      int n_dev, int collapse, float* partials, void* workspace, uint32_t* dev_status,

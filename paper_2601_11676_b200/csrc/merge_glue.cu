@@ -1,5 +1,7 @@
 // halo_merge_partials (step a9), halo_glue (residual + RMS normalisation between blocks), their fusion
 // for the stack, and halo_pack_weights.
+#include <initializer_list>
+
 #include "common.cuh"
 
 namespace halo {
@@ -34,35 +36,77 @@ __device__ __forceinline__ float block_sum_1024(float v, float* scratch /*[32]*/
     return r;
 }
 
+__device__ __forceinline__ void store4(float* p, float a, float b, float c, float d) {
+    *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+__device__ __forceinline__ void store4(__nv_bfloat16* p, float a, float b, float c, float d) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+}
+
 // One block per token.  MERGE: y is taken from the partial slots, else from y_in (may be NULL = 0).
 template <typename T, bool MERGE>
 __global__ void __launch_bounds__(1024)
 glue_kernel(int d, const float* __restrict__ h, const float* __restrict__ y_in, const float* __restrict__ partials,
             const uint8_t* __restrict__ arrived, int n_dev, size_t slot_stride, float* h_out, T* __restrict__ x_out,
-            float* __restrict__ y_tap) {
+            float* __restrict__ y_tap, int vec) {
     __shared__ float scratch[32];
-    extern __shared__ float hv[];  // [d]
+    extern __shared__ __align__(16) float hv[];  // [d]
     const int tok = blockIdx.x;
     const size_t base = static_cast<size_t>(tok) * d;
     float ss = 0.0f;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) {
-        float y = 0.0f;
-        if (MERGE) {
-            y = merged_value(partials, arrived, n_dev, slot_stride, base + c);
-            if (y_tap) y_tap[base + c] = y;
-        } else if (y_in) {
-            y = y_in[base + c];
+    if (vec) {
+        // four columns per thread and access (every row starts 16-byte aligned)
+        const int d4 = d >> 2;
+        const float4* h4 = reinterpret_cast<const float4*>(h + base);
+        for (int c = threadIdx.x; c < d4; c += blockDim.x) {
+            float4 y = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (MERGE) {
+                y = reinterpret_cast<const float4*>(partials + base)[c];
+                for (int i = 0; i < n_dev; ++i)
+                    if (!arrived || arrived[i]) {
+                        const float4 p =
+                            reinterpret_cast<const float4*>(partials + static_cast<size_t>(i + 1) * slot_stride + base)[c];
+                        y.x += p.x; y.y += p.y; y.z += p.z; y.w += p.w;
+                    }
+                if (y_tap) reinterpret_cast<float4*>(y_tap + base)[c] = y;
+            } else if (y_in) {
+                y = reinterpret_cast<const float4*>(y_in + base)[c];
+            }
+            const float4 hh = h4[c];
+            const float4 v = make_float4(hh.x + y.x, hh.y + y.y, hh.z + y.z, hh.w + y.w);
+            reinterpret_cast<float4*>(hv)[c] = v;
+            ss = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, fmaf(v.w, v.w, ss))));
         }
-        const float v = h[base + c] + y;
-        hv[c] = v;
-        ss = fmaf(v, v, ss);
+    } else {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) {
+            float y = 0.0f;
+            if (MERGE) {
+                y = merged_value(partials, arrived, n_dev, slot_stride, base + c);
+                if (y_tap) y_tap[base + c] = y;
+            } else if (y_in) {
+                y = y_in[base + c];
+            }
+            const float v = h[base + c] + y;
+            hv[c] = v;
+            ss = fmaf(v, v, ss);
+        }
     }
     ss = block_sum_1024(ss, scratch);
     const float scale = 1.0f / sqrtf(ss / static_cast<float>(d) + 1e-5f);
-    for (int c = threadIdx.x; c < d; c += blockDim.x) {
-        const float v = hv[c];
-        h_out[base + c] = v;
-        x_out[base + c] = from_float<T>(v * scale);
+    if (vec) {
+        const int d4 = d >> 2;
+        for (int c = threadIdx.x; c < d4; c += blockDim.x) {
+            const float4 v = reinterpret_cast<const float4*>(hv)[c];
+            reinterpret_cast<float4*>(h_out + base)[c] = v;
+            store4(x_out + base + 4 * c, v.x * scale, v.y * scale, v.z * scale, v.w * scale);
+        }
+    } else {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) {
+            const float v = hv[c];
+            h_out[base + c] = v;
+            x_out[base + c] = from_float<T>(v * scale);
+        }
     }
 }
 
@@ -89,15 +133,25 @@ halo_status launch_merge(const float* partials, const uint8_t* arrived, int n_de
     return HALO_OK;
 }
 
+namespace {
+// the four-column path needs d % 4 == 0 and every buffer 16-byte aligned
+bool all_aligned16(std::initializer_list<const void*> ptrs) {
+    for (const void* p : ptrs)
+        if (p && (reinterpret_cast<uintptr_t>(p) & 15u)) return false;
+    return true;
+}
+}  // namespace
+
 halo_status launch_glue(int d, int n_tok, halo_dtype xdtype, const float* h, const float* y, float* h_out,
                         void* x_out, cudaStream_t st) {
     const size_t smem = sizeof(float) * static_cast<size_t>(d);
+    const int vec = (d % 4 == 0) && all_aligned16({h, y, h_out, x_out});
     if (xdtype == HALO_BF16)
         glue_kernel<__nv_bfloat16, false><<<n_tok, 1024, smem, st>>>(d, h, y, nullptr, nullptr, 0, 0, h_out,
-                                                                      static_cast<__nv_bfloat16*>(x_out), nullptr);
+                                                                      static_cast<__nv_bfloat16*>(x_out), nullptr, vec);
     else
         glue_kernel<float, false><<<n_tok, 1024, smem, st>>>(d, h, y, nullptr, nullptr, 0, 0, h_out,
-                                                             static_cast<float*>(x_out), nullptr);
+                                                             static_cast<float*>(x_out), nullptr, vec);
     HALO_CHECK_LAUNCH();
     return HALO_OK;
 }
@@ -107,12 +161,13 @@ halo_status launch_merge_glue(const float* partials, const uint8_t* arrived, int
                               cudaStream_t st) {
     const size_t smem = sizeof(float) * static_cast<size_t>(d);
     const size_t stride = static_cast<size_t>(n_tok) * d;
+    const int vec = (d % 4 == 0) && all_aligned16({partials, h, h_out, x_out, y_tap});
     if (xdtype == HALO_BF16)
         glue_kernel<__nv_bfloat16, true><<<n_tok, 1024, smem, st>>>(d, h, nullptr, partials, arrived, n_dev, stride,
-                                                                     h_out, static_cast<__nv_bfloat16*>(x_out), y_tap);
+                                                                     h_out, static_cast<__nv_bfloat16*>(x_out), y_tap, vec);
     else
         glue_kernel<float, true><<<n_tok, 1024, smem, st>>>(d, h, nullptr, partials, arrived, n_dev, stride, h_out,
-                                                            static_cast<float*>(x_out), y_tap);
+                                                            static_cast<float*>(x_out), y_tap, vec);
     HALO_CHECK_LAUNCH();
     return HALO_OK;
 }

@@ -687,12 +687,17 @@ bool prefill_supported(const halo_ffn_shape& sh, int n_tok) {
            sh.d_model % 128 == 0 && sh.d_ffn / sh.group_size <= HALO_MAX_GROUPS;
 }
 
+bool prefill_accumulates(const halo_ffn_shape& sh, int n_tok) {
+    return prefill_supported(sh, n_tok) && n_tok > kBM && sh.d_model % 256 == 0;
+}
+
 size_t prefill_workspace_bytes(const halo_ffn_shape& sh, int n_tok) {
     return static_cast<size_t>(n_tok) * sh.d_ffn * 2;   // H: bf16 [n_tok][d_ffn], kept groups packed to the left
 }
 
-// partials must already be zero (slots without kept groups are not written).  collapse != 0: partials has two
-// slots only, [0] = the master's groups, [1] = all devices' groups.
+// partials must already be zero (slots without kept groups are not written).  collapse != 0: the caller wants the
+// sum over holders only and partials has two slots whose SUM is the result; when prefill_accumulates() holds,
+// everything is added into slot 0 (slot 1 is not touched), which may then hold a value to add to.
 halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                      const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
                                      int n_dev, int collapse, float* partials, void* workspace, uint32_t* dev_status,

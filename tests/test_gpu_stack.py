@@ -147,6 +147,23 @@ def test_stack_multi_token_prompt():
     check_teacher_forced(wl, Wp, preds, h0, h_out, t, 1)
 
 
+@pytest.mark.parametrize("n_tok,d", [(64, 512), (160, 512), (300, 256)])
+def test_stack_prompt_on_the_tensor_core_path(n_tok, d):
+    """Prompts long enough for the tensor-core kernels (one 128-token tile, and more than one): teacher-forced
+    against the oracle through the taps; then the same run without taps, where the down projection adds straight
+    into the residual stream, must give the same stream."""
+    wl = synth.Workload("pt", 3, d, 64 * 12, 64, 64, "bf16", (0.0, 0.3, 0.6), (2, 1, 1), 250, 2, n_tok=n_tok)
+    stack, Wp, preds = build_stack(wl)
+    h0, h_out, t = run_with_taps(wl, stack, wl.steps)
+    lost = check_teacher_forced(wl, Wp, preds, h0, h_out, t, wl.steps)
+    assert lost > 0
+    plain = torch.empty_like(h_out)
+    stack.decode(h0, wl.steps, 0, plain)
+    torch.cuda.synchronize()
+    assert stack.status() == 0
+    assert (plain - h_out).abs().max().item() <= 1e-4 * h_out.abs().max().item()
+
+
 @pytest.mark.parametrize("name,steps,sample", [
     ("llama2-7b-decode", 3, [(0, 0), (0, 1), (1, 16), (2, 30), (2, 31)]),
     ("llama2-13b-decode", 2, [(0, 1), (1, 20), (1, 39)]),

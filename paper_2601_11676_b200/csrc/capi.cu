@@ -519,7 +519,11 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     s->side = nullptr; s->ev_x = nullptr; s->ev_sel = nullptr;
     if (n_tok > 1) {
         // best effort: without them the blocks simply run one after the other on the caller's stream
-        if (cudaStreamCreateWithFlags(&s->side, cudaStreamNonBlocking) != cudaSuccess) s->side = nullptr;
+        // highest priority: the short predictor/selection kernels of the next block must get SMs as they free up,
+        // ahead of the waiting CTAs of the long FFN launch (which pulls its tiles from a queue and loses nothing)
+        int prio_lo = 0, prio_hi = 0;
+        if (cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) != cudaSuccess) prio_hi = 0;
+        if (cudaStreamCreateWithPriority(&s->side, cudaStreamNonBlocking, prio_hi) != cudaSuccess) s->side = nullptr;
         if (s->side && (cudaEventCreateWithFlags(&s->ev_x, cudaEventDisableTiming) != cudaSuccess ||
                         cudaEventCreateWithFlags(&s->ev_sel, cudaEventDisableTiming) != cudaSuccess)) {
             cudaStreamDestroy(s->side);

@@ -550,6 +550,367 @@ ffn_down_wide_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_co
 }
 
 // ------------------------------------------------------------------------------------------------------------
+// Both contractions of a prompt's FFN in ONE launch: a queue of tiles, hidden-layer tiles first, then the
+// down-projection tiles, claimed by the CTAs as they get free.  A down-projection tile reads H columns that
+// hidden-layer tiles of OTHER CTAs write, so each finished hidden tile bumps a ready counter of its (token tile,
+// kept group) and the loader of a down tile waits on the counters of the groups it is about to fetch.  Every
+// hidden tile precedes every down tile in the queue and never waits on anything but its own copies, so a waited
+// counter is always owed by a CTA that is already running and will get there: no co-residency is needed.  This
+// fills the last, partial wave of hidden tiles with down-projection work.
+// ------------------------------------------------------------------------------------------------------------
+struct FusedTail {
+    DownSmemTail dn;
+    uint64_t tile_full[2];    // the loader has published a tile index
+    uint64_t tile_empty[2];   // the MMA thread and the four epilogue warps have read it
+    int tile_ring[2];
+};
+constexpr int kCtlHeaderWords = 32;          // word 0 = tile queue; ready counters follow
+constexpr unsigned kReadyWhen = 8;           // 4 epilogue warps x (2 for a full tile | 1 + 1 for its two halves)
+
+struct FusedGeom {
+    int tiles_x, n_full, n1_full, n1, n_tiles, n_tn, z_cuts, units;
+};
+struct FusedTile {
+    int kind;   // 0 = hidden (full group), 1 = hidden (half group), 2 = down
+    int ki, mt, half, nt, z;
+};
+__device__ __forceinline__ FusedTile fused_decode(const FusedGeom& q, int t) {
+    FusedTile r{};
+    if (t < q.n1_full) {
+        r.kind = 0; r.ki = t / q.tiles_x; r.mt = t - r.ki * q.tiles_x;
+    } else if (t < q.n1) {
+        const int u = t - q.n1_full, per = 2 * q.tiles_x;
+        r.kind = 1; r.ki = q.n_full + u / per;
+        const int w = u % per;
+        r.mt = w >> 1; r.half = w & 1;
+    } else {
+        const int u = t - q.n1, per = q.tiles_x * q.n_tn;
+        r.kind = 2; r.z = u / per;
+        const int w = u - r.z * per;
+        r.nt = w / q.tiles_x; r.mt = w - r.nt * q.tiles_x;
+    }
+    return r;
+}
+
+// Bounded wait for a ready counter written by other CTAs.
+__device__ __forceinline__ bool fused_wait_ready(const unsigned* counter, volatile int* abort_flag) {
+    if (ld_acquire_gpu(counter) >= kReadyWhen) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        if (*abort_flag) return false;
+        if (ld_acquire_gpu(counter) >= kReadyWhen) return true;
+        __nanosleep(64);
+        if (clock64() - t0 > static_cast<long long>(kWaitLimitCycles)) { *abort_flag = 1; return false; }
+    }
+}
+
+template <int NS, int STAGES>
+__global__ void __launch_bounds__(kPfThreads, 1)
+ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                 const __grid_constant__ CUtensorMap tmap_w_half, const __grid_constant__ CUtensorMap tmap_h,
+                 const __grid_constant__ CUtensorMap tmap_wd, int T, int d, int G, int n_sm, int z_cuts,
+                 const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
+                 const int32_t* __restrict__ dev_of_group, int n_dev, int collapse, __nv_bfloat16* __restrict__ H,
+                 int h_cols, float* __restrict__ partials, unsigned* __restrict__ ctl, uint32_t* dev_status) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    constexpr int S = NS, BN2 = 256, MH = 2;
+    constexpr uint32_t kAHalf = kBM * kBK * 2, kABytes = MH * kAHalf;
+    constexpr uint32_t kStageBytes = kABytes + kBK * BN2 * 2;   // 64 KiB: the down tile's stage; a hidden stage fits
+    constexpr uint32_t kBBlock = kBK * 64 * 2;
+    constexpr uint32_t kTmemCols = 512;
+    static_assert(MH * 2 * NS <= 512, "hidden accumulators must fit in TMEM");
+    FusedTail& ft = *reinterpret_cast<FusedTail*>(smem_raw + static_cast<size_t>(STAGES) * kStageBytes);
+    DownSmemTail& tail = ft.dn;
+    float* const epi_stage = reinterpret_cast<float*>(smem_raw + static_cast<size_t>(STAGES) * kStageBytes +
+                                                      ((sizeof(FusedTail) + 15) & ~size_t(15)));
+    PfBarriers& bars = tail.bars;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    int nk = *n_keep_ptr;
+    nk = max(0, min(nk, G));
+    const int k_per_group = S / kBK, n_kt1 = d / kBK;
+    const int n_slots = collapse ? 1 : n_dev + 1;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&bars.full[s], 1); mbar_init(&bars.empty[s], 1); }
+        mbar_init(&bars.tmem_full, 1);
+        mbar_init(&bars.tmem_empty, 4);
+        mbar_init(&tail.acc_full[0], 1);
+        mbar_init(&tail.acc_empty[0], 4);
+        for (int b = 0; b < 2; ++b) { mbar_init(&ft.tile_full[b], 1); mbar_init(&ft.tile_empty[b], 5); }
+        bars.abort_flag = 0;
+        mbar_fence_init();
+        tma_prefetch_descriptor(&tmap_x);
+        tma_prefetch_descriptor(&tmap_w);
+        tma_prefetch_descriptor(&tmap_h);
+        tma_prefetch_descriptor(&tmap_wd);
+    }
+    if (warp == 1) { tmem_alloc(&bars.tmem_base, kTmemCols); tmem_relinquish_alloc_permit(); }
+    if (warp == 0) {
+        const int pos = build_slot_order(tail, nk, G, n_dev, n_slots, n_slots - 1, keep_list, dev_of_group, dev_status,
+                                         lane);
+        if (lane == 0) { tail.slot_start[n_slots] = pos; tail.slot_lo = pos; }
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    volatile int* abort_flag = &bars.abort_flag;
+    const uint32_t tmem = bars.tmem_base;
+
+    // the tile list, derived identically by every role
+    FusedGeom q;
+    q.tiles_x = (T + kBM * MH - 1) / (kBM * MH);
+    q.n_tn = d / BN2;
+    q.z_cuts = z_cuts;
+    q.units = tail.slot_lo * k_per_group;    // K tiles of the down projection (valid kept groups only)
+    q.n_full = nk;
+    {
+        // hidden tiles of the last, partial wave are cut into two half-width tiles (finer work at the end)
+        const int total = q.tiles_x * nk;
+        if (n_sm > 0 && total > n_sm) {
+            const int full_groups = (total / n_sm) * n_sm / q.tiles_x, left = nk - full_groups;
+            if (left > 0 && 2 * left * q.tiles_x <= n_sm) q.n_full = full_groups;
+        }
+    }
+    q.n1_full = q.tiles_x * q.n_full;
+    q.n1 = q.n1_full + 2 * q.tiles_x * (nk - q.n_full);
+    q.n_tiles = q.n1 + (q.units > 0 ? q.tiles_x * q.n_tn * z_cuts : 0);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int it = 0;
+            for (int ti = 0;; ++ti) {
+                if (ti >= 2 && !pf_wait(&ft.tile_empty[ti & 1], ((ti >> 1) - 1) & 1, abort_flag)) break;
+                const int t = static_cast<int>(min(atomicAdd(&ctl[0], 1u), 0x7fffffffu));
+                ft.tile_ring[ti & 1] = t;
+                mbar_arrive(&ft.tile_full[ti & 1]);
+                if (t >= q.n_tiles) break;
+                const FusedTile tl = fused_decode(q, t);
+                const int m0 = tl.mt * (kBM * MH);
+                bool alive = true;
+                if (tl.kind < 2) {
+                    const int g = keep_list[tl.ki];
+                    const bool valid = g >= 0 && g < G;     // an invalid entry was flagged by build_slot_order
+                    const int ns = tl.kind == 1 ? NS / 2 : NS, n_off = tl.kind == 1 ? tl.half * (NS / 2) : 0;
+                    const CUtensorMap* const map_w = tl.kind == 1 ? &tmap_w_half : &tmap_w;
+                    const int gg = valid ? g : 0;
+                    for (int kt = 0; kt < n_kt1; ++kt, ++it) {
+                        const int s = it % STAGES;
+                        if (it >= STAGES && !pf_wait(&bars.empty[s], ((it / STAGES) - 1) & 1, abort_flag)) { alive = false; break; }
+                        unsigned char* st = smem_raw + static_cast<size_t>(s) * kStageBytes;
+                        mbar_arrive_expect_tx(&bars.full[s], kABytes + 2u * static_cast<uint32_t>(ns) * kBK * 2u);
+#pragma unroll
+                        for (int mh = 0; mh < MH; ++mh)
+                            tma_load_2d(st + mh * kAHalf, &tmap_x, kt * kBK, m0 + mh * kBM, &bars.full[s]);
+                        tma_load_2d(st + kABytes, map_w, kt * kBK, (gg * 3 + 0) * S + n_off, &bars.full[s]);
+                        tma_load_2d(st + kABytes + ns * (kBK * 2), map_w, kt * kBK, (gg * 3 + 1) * S + n_off, &bars.full[s]);
+                    }
+                } else {
+                    const int n0 = tl.nt * BN2;
+                    const int kt_lo = static_cast<int>(static_cast<long long>(q.units) * tl.z / z_cuts);
+                    const int kt_hi = static_cast<int>(static_cast<long long>(q.units) * (tl.z + 1) / z_cuts);
+                    int checked = -1;
+                    for (int kt = kt_lo; kt < kt_hi; ++kt, ++it) {
+                        const int p = kt / k_per_group, kk2 = kt - p * k_per_group;
+                        const int g = tail.group_of[p], kp = tail.kept_pos[p];
+                        if (p != checked) {
+                            // the hidden tiles of this group and token tile must have been written
+                            if (!fused_wait_ready(&ctl[kCtlHeaderWords + tl.mt * G + kp], abort_flag)) { alive = false; break; }
+                            fence_proxy_async_all();   // their generic-proxy stores before this thread's TMA reads
+                            checked = p;
+                        }
+                        const int s = it % STAGES;
+                        if (it >= STAGES && !pf_wait(&bars.empty[s], ((it / STAGES) - 1) & 1, abort_flag)) { alive = false; break; }
+                        unsigned char* st = smem_raw + static_cast<size_t>(s) * kStageBytes;
+                        mbar_arrive_expect_tx(&bars.full[s], kStageBytes);
+#pragma unroll
+                        for (int mh = 0; mh < MH; ++mh)
+                            tma_load_2d(st + mh * kAHalf, &tmap_h, kp * S + kk2 * kBK, m0 + mh * kBM, &bars.full[s]);
+                        const int krow = (g * 3 + 2) * S + kk2 * kBK;
+#pragma unroll
+                        for (int nb = 0; nb < BN2 / 64; ++nb)
+                            tma_load_2d(st + kABytes + nb * kBBlock, &tmap_wd, n0 + nb * 64, krow, &bars.full[s]);
+                    }
+                }
+                if (!alive) break;
+            }
+            if (*abort_flag) {  // let outstanding copies land before the CTA goes away
+                int never = 0;
+                for (int k = max(0, it - STAGES); k < it; ++k)
+                    mbar_wait_bounded(&bars.full[k % STAGES], (k / STAGES) & 1, &never);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc2 = umma_idesc_bf16(kBM, BN2, true);
+            int it = 0, seg = 0;
+            bool alive = true;
+            for (int ti = 0; alive; ++ti) {
+                if (!pf_wait(&ft.tile_full[ti & 1], (ti >> 1) & 1, abort_flag)) break;
+                const int t = ft.tile_ring[ti & 1];
+                mbar_arrive(&ft.tile_empty[ti & 1]);
+                if (t >= q.n_tiles) break;
+                const FusedTile tl = fused_decode(q, t);
+                if (tl.kind < 2) {
+                    const int ns = tl.kind == 1 ? NS / 2 : NS;
+                    const uint32_t idesc1 = umma_idesc_bf16(kBM, 2 * ns, false);
+                    if (seg >= 1 && !pf_wait(&tail.acc_empty[0], (seg - 1) & 1, abort_flag)) break;
+                    tcgen05_fence_after_sync();
+                    for (int kt = 0; kt < n_kt1; ++kt, ++it) {
+                        const int s = it % STAGES;
+                        if (!pf_wait(&bars.full[s], (it / STAGES) & 1, abort_flag)) { alive = false; break; }
+                        tcgen05_fence_after_sync();
+                        const uint32_t a0 = smem_u32(smem_raw + static_cast<size_t>(s) * kStageBytes);
+#pragma unroll
+                        for (int kk = 0; kk < kBK / kUmmaK; ++kk) {
+                            const uint64_t b = umma_smem_desc(a0 + kABytes + kk * 32, 16, 1024);
+#pragma unroll
+                            for (int mh = 0; mh < MH; ++mh) {
+                                const uint64_t a = umma_smem_desc(a0 + mh * kAHalf + kk * 32, 16, 1024);
+                                umma_bf16(tmem + mh * 2 * NS, a, b, idesc1, (kt > 0) || (kk > 0));
+                            }
+                        }
+                        umma_commit(&bars.empty[s]);
+                    }
+                    if (!alive) break;
+                    umma_commit(&tail.acc_full[0]);
+                    ++seg;
+                } else {
+                    const int kt_lo = static_cast<int>(static_cast<long long>(q.units) * tl.z / z_cuts);
+                    const int kt_hi = static_cast<int>(static_cast<long long>(q.units) * (tl.z + 1) / z_cuts);
+                    for (int slot = 0; slot < n_slots && alive; ++slot) {
+                        const int k0 = max(kt_lo, tail.slot_start[slot] * k_per_group);
+                        const int k1 = min(kt_hi, tail.slot_start[slot + 1] * k_per_group);
+                        if (k0 >= k1) continue;
+                        if (seg >= 1 && !pf_wait(&tail.acc_empty[0], (seg - 1) & 1, abort_flag)) { alive = false; break; }
+                        tcgen05_fence_after_sync();
+                        for (int kt = k0; kt < k1; ++kt, ++it) {
+                            const int s = it % STAGES;
+                            if (!pf_wait(&bars.full[s], (it / STAGES) & 1, abort_flag)) { alive = false; break; }
+                            tcgen05_fence_after_sync();
+                            const uint32_t a0 = smem_u32(smem_raw + static_cast<size_t>(s) * kStageBytes);
+#pragma unroll
+                            for (int kk = 0; kk < kBK / kUmmaK; ++kk) {
+                                const uint64_t b = umma_smem_desc(a0 + kABytes + kk * 2048, kBBlock, 1024);
+#pragma unroll
+                                for (int mh = 0; mh < MH; ++mh) {
+                                    const uint64_t a = umma_smem_desc(a0 + mh * kAHalf + kk * 32, 16, 1024);
+                                    umma_bf16(tmem + mh * BN2, a, b, idesc2, (kt > k0) || (kk > 0));
+                                }
+                            }
+                            umma_commit(&bars.empty[s]);
+                        }
+                        if (!alive) break;
+                        umma_commit(&tail.acc_full[0]);
+                        ++seg;
+                    }
+                }
+            }
+        }
+    } else {
+        const int quad = warp & 3;
+        const uint32_t lane_base = tmem + (static_cast<uint32_t>(quad * 32) << 16);
+        float* stage = epi_stage + (warp - 2) * (32 * kEpiPitch);
+        int seg = 0;
+        for (int ti = 0;; ++ti) {
+            if (!pf_wait(&ft.tile_full[ti & 1], (ti >> 1) & 1, abort_flag)) break;
+            const int t = ft.tile_ring[ti & 1];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ft.tile_empty[ti & 1]);
+            if (t >= q.n_tiles) break;
+            const FusedTile tl = fused_decode(q, t);
+            const int m0 = tl.mt * (kBM * MH);
+            if (tl.kind < 2) {
+                const int ns = tl.kind == 1 ? NS / 2 : NS, n_off = tl.kind == 1 ? tl.half * (NS / 2) : 0;
+                const int g = keep_list[tl.ki];
+                const bool ok = pf_wait(&tail.acc_full[0], seg & 1, abort_flag) && g >= 0 && g < G;
+                tcgen05_fence_after_sync();
+#pragma unroll
+                for (int mh = 0; mh < MH; ++mh) {
+                    const int row = m0 + mh * kBM + quad * 32 + lane;
+                    for (int c0 = 0; c0 < ns; c0 += 32) {
+                        uint32_t dg[32], du[32];
+                        tmem_ld_32x32(lane_base + mh * 2 * NS + c0, dg);
+                        tmem_ld_32x32(lane_base + mh * 2 * NS + ns + c0, du);
+                        tmem_ld_wait();
+                        if (ok && row < T) {
+                            uint4* dst = reinterpret_cast<uint4*>(H + static_cast<size_t>(row) * h_cols +
+                                                                  static_cast<size_t>(tl.ki) * S + n_off + c0);
+#pragma unroll
+                            for (int qq = 0; qq < 4; ++qq) {
+                                uint32_t packed[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const int i = qq * 8 + e * 2;
+                                    const float h0 = silu_mul(__uint_as_float(dg[i]), __uint_as_float(du[i]));
+                                    const float h1 = silu_mul(__uint_as_float(dg[i + 1]), __uint_as_float(du[i + 1]));
+                                    const __nv_bfloat162 pk = __floats2bfloat162_rn(h0, h1);
+                                    packed[e] = *reinterpret_cast<const uint32_t*>(&pk);
+                                }
+                                dst[qq] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                            }
+                        }
+                    }
+                }
+                // publish: every lane orders its own stores (towards the TMA reads of other CTAs too), then one
+                // lane bumps the counter.  An aborted tile publishes nothing; its readers give up on their own.
+                tcgen05_fence_before_sync();
+                fence_proxy_async_all();
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) {
+                    if (ok) atomicAdd(&ctl[kCtlHeaderWords + tl.mt * G + tl.ki], tl.kind == 1 ? 1u : 2u);
+                    mbar_arrive(&tail.acc_empty[0]);
+                }
+                ++seg;
+            } else {
+                const int n0 = tl.nt * BN2;
+                const int kt_lo = static_cast<int>(static_cast<long long>(q.units) * tl.z / z_cuts);
+                const int kt_hi = static_cast<int>(static_cast<long long>(q.units) * (tl.z + 1) / z_cuts);
+                for (int slot = 0; slot < n_slots; ++slot) {
+                    const int k0 = max(kt_lo, tail.slot_start[slot] * k_per_group);
+                    const int k1 = min(kt_hi, tail.slot_start[slot + 1] * k_per_group);
+                    if (k0 >= k1) continue;
+                    const bool ok = pf_wait(&tail.acc_full[0], seg & 1, abort_flag);
+                    tcgen05_fence_after_sync();
+#pragma unroll
+                    for (int mh = 0; mh < MH; ++mh) {
+                        const int row0 = m0 + mh * kBM + quad * 32;
+                        float* out = partials + (static_cast<size_t>(slot) * T + row0) * d + n0;
+                        for (int c0 = 0; c0 < BN2; c0 += 32) {
+                            uint32_t v[32];
+                            tmem_ld_32x32(lane_base + mh * BN2 + c0, v);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int qq = 0; qq < 8; ++qq)
+                                *reinterpret_cast<float4*>(stage + lane * kEpiPitch + 4 * qq) =
+                                    make_float4(__uint_as_float(v[4 * qq]), __uint_as_float(v[4 * qq + 1]),
+                                                __uint_as_float(v[4 * qq + 2]), __uint_as_float(v[4 * qq + 3]));
+                            __syncwarp();
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const int r = 4 * j + (lane >> 3), cq = (lane & 7) * 4;
+                                const float4 w = *reinterpret_cast<const float4*>(stage + r * kEpiPitch + cq);
+                                if (ok && row0 + r < T)
+                                    red_add_v4f(out + static_cast<size_t>(r) * d + c0 + cq, w.x, w.y, w.z, w.w);
+                            }
+                            __syncwarp();
+                        }
+                    }
+                    tcgen05_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tail.acc_empty[0]);
+                    ++seg;
+                }
+            }
+        }
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, kTmemCols); }
+    if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------------------
 // Predictor hidden layer for many tokens: Z[T][r] = act(X[T][d] * W1[r][d]^T), fp32 out (step a1, prefill)
 // ------------------------------------------------------------------------------------------------------------
 template <int STAGES>
@@ -691,8 +1052,17 @@ bool prefill_accumulates(const halo_ffn_shape& sh, int n_tok) {
     return prefill_supported(sh, n_tok) && n_tok > kBM && sh.d_model % 256 == 0;
 }
 
+namespace {
+// tile queue + one ready counter per (256-token tile, kept position), in front of H
+size_t prefill_ctl_bytes(const halo_ffn_shape& sh, int n_tok) {
+    const size_t words = kCtlHeaderWords + static_cast<size_t>((n_tok + 2 * kBM - 1) / (2 * kBM)) * (sh.d_ffn / sh.group_size);
+    return (words * sizeof(unsigned) + 1023) & ~static_cast<size_t>(1023);
+}
+}  // namespace
+
 size_t prefill_workspace_bytes(const halo_ffn_shape& sh, int n_tok) {
-    return static_cast<size_t>(n_tok) * sh.d_ffn * 2;   // H: bf16 [n_tok][d_ffn], kept groups packed to the left
+    // control words, then H: bf16 [n_tok][d_ffn], kept groups packed to the left
+    return prefill_ctl_bytes(sh, n_tok) + static_cast<size_t>(n_tok) * sh.d_ffn * 2;
 }
 
 // partials must already be zero (slots without kept groups are not written).  collapse != 0: the caller wants the
@@ -703,7 +1073,9 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
                                      int n_dev, int collapse, float* partials, void* workspace, uint32_t* dev_status,
                                      cudaStream_t st) {
     const int d = sh.d_model, S = sh.group_size, G = sh.d_ffn / S, T = n_tok;
-    __nv_bfloat16* H = static_cast<__nv_bfloat16*>(workspace);
+    const size_t ctl_bytes = prefill_ctl_bytes(sh, T);
+    unsigned* ctl = static_cast<unsigned*>(workspace);
+    __nv_bfloat16* H = reinterpret_cast<__nv_bfloat16*>(static_cast<unsigned char*>(workspace) + ctl_bytes);
     const uint64_t w_rows = static_cast<uint64_t>(G) * 3 * S;
     int dev = 0, n_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -714,6 +1086,33 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         !make_map(&map_w_half, W, w_rows, d, d, kBK, S / 2) ||
         !make_map(&map_h, H, T, sh.d_ffn, sh.d_ffn, kBK, kBM) || !make_map(&map_wd, W, w_rows, d, d, 64, kBK))
         return HALO_ERR_CUDA;
+    static const bool two_launches = [] { const char* e = getenv("HALO_TUNE_PREFILL_TWO_LAUNCHES"); return e && e[0] == '1'; }();
+    if (T > kBM && d % 256 == 0 && !two_launches) {
+        // both contractions in one launch, one CTA per SM pulling tiles from a queue
+        if (cudaMemsetAsync(ctl, 0, ctl_bytes, st) != cudaSuccess) return HALO_ERR_CUDA;
+        constexpr int kStagesF = 3;
+        const size_t smemf = static_cast<size_t>(kStagesF) * (2 * kBM * kBK * 2 + kBK * 256 * 2) + sizeof(FusedTail) + 16 +
+                             kEpiStageBytes + 1024;
+        const int tiles2 = ((T + 2 * kBM - 1) / (2 * kBM)) * (d / 256);
+        // K cuts of the down projection: a third more tiles than SMs, so that the CTAs that finish their hidden
+        // tiles late still find down-projection work of a useful size (HALO_TUNE_PREFILL_KCUTS overrides)
+        int z = std::max(1, std::min(8, (n_sm * 4 / 3) / tiles2));
+        if (const char* e = getenv("HALO_TUNE_PREFILL_KCUTS")) z = std::max(1, std::min(16, atoi(e)));
+#define HALO_LAUNCH_FUSED(NS_)                                                                                       \
+    do {                                                                                                             \
+        auto kf = ffn_fused_kernel<NS_, kStagesF>;                                                                   \
+        static bool oncef[64] = {};                                                                                  \
+        if (!ensure_dynamic_smem(kf, smemf, oncef)) return HALO_ERR_CUDA;                                            \
+        kf<<<n_sm, kPfThreads, smemf, st>>>(map_x, map_w, map_w_half, map_h, map_wd, T, d, G,                        \
+                                            n_sm, z, keep_list,                                                      \
+                                            n_keep, dev_of_group, n_dev, collapse, H, sh.d_ffn, partials, ctl,       \
+                                            dev_status);                                                             \
+    } while (0)
+        if (S == 128) HALO_LAUNCH_FUSED(128); else HALO_LAUNCH_FUSED(64);
+#undef HALO_LAUNCH_FUSED
+        HALO_CHECK_LAUNCH();
+        return HALO_OK;
+    }
     // GEMM-1: 256-token tiles when the prompt has them (more FLOP per staged byte), else 128-token tiles
 #define HALO_LAUNCH_HIDDEN(NS_, MH_, STAGES_)                                                                        \
     do {                                                                                                             \

@@ -20,7 +20,7 @@ def _wl(d, G, S, n_dev=3):
 def test_prefill_ffn_small_shapes_all_tokens(d, G, S, n_tok):
     wl = _wl(d, G, S)
     sh = B.ffn_shape(d, G * S, S, B.BF16)
-    assert B.halo_group_ffn_workspace_bytes(sh, n_tok, wl.n_dev) == n_tok * G * S * 2
+    assert B.halo_group_ffn_workspace_bytes(sh, n_tok, wl.n_dev) >= n_tok * G * S * 2
     Wp = synth.packed_layer(wl, 0, DEV)
     x = synth.activation(wl, 1, DEV, n_tok=n_tok)
     dev = np.array([-1, 0, 1, 2, 0, -1], dtype=np.int32)[:G]

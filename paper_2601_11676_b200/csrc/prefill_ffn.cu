@@ -558,6 +558,17 @@ ffn_down_wide_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_co
 // counter is always owed by a CTA that is already running and will get there: no co-residency is needed.  This
 // fills the last, partial wave of hidden tiles with down-projection work.
 // ------------------------------------------------------------------------------------------------------------
+// K cuts of the down projection, as cumulative 16.16 fixed-point fractions of the K range: run z covers
+// [units * cum[z] >> 16, units * cum[z + 1] >> 16).  The runs shrink geometrically, so the tiles claimed last are
+// short: the end of the queue is fine-grained, and the runs that need the last hidden tiles are the small ones.
+struct KCuts {
+    int n;
+    unsigned cum[17];
+};
+__device__ __forceinline__ int kcut(const KCuts& c, int units, int z) {
+    return static_cast<int>((static_cast<unsigned long long>(units) * c.cum[z]) >> 16);
+}
+
 struct FusedTail {
     DownSmemTail dn;
     uint64_t tile_full[2];    // the loader has published a tile index
@@ -608,7 +619,8 @@ template <int NS, int STAGES>
 __global__ void __launch_bounds__(kPfThreads, 1)
 ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                  const __grid_constant__ CUtensorMap tmap_w_half, const __grid_constant__ CUtensorMap tmap_h,
-                 const __grid_constant__ CUtensorMap tmap_wd, int T, int d, int G, int n_sm, int z_cuts,
+                 const __grid_constant__ CUtensorMap tmap_wd, const __grid_constant__ KCuts cuts, int T, int d, int G,
+                 int n_sm,
                  const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
                  const int32_t* __restrict__ dev_of_group, int n_dev, int collapse, __nv_bfloat16* __restrict__ H,
                  int h_cols, float* __restrict__ partials, unsigned* __restrict__ ctl, uint32_t* dev_status) {
@@ -660,7 +672,7 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     FusedGeom q;
     q.tiles_x = (T + kBM * MH - 1) / (kBM * MH);
     q.n_tn = d / BN2;
-    q.z_cuts = z_cuts;
+    q.z_cuts = cuts.n;
     q.units = tail.slot_lo * k_per_group;    // K tiles of the down projection (valid kept groups only)
     q.n_full = nk;
     {
@@ -673,7 +685,7 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     }
     q.n1_full = q.tiles_x * q.n_full;
     q.n1 = q.n1_full + 2 * q.tiles_x * (nk - q.n_full);
-    q.n_tiles = q.n1 + (q.units > 0 ? q.tiles_x * q.n_tn * z_cuts : 0);
+    q.n_tiles = q.n1 + (q.units > 0 ? q.tiles_x * q.n_tn * cuts.n : 0);
 
     if (warp == 0) {
         if (lane == 0) {
@@ -706,8 +718,8 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     }
                 } else {
                     const int n0 = tl.nt * BN2;
-                    const int kt_lo = static_cast<int>(static_cast<long long>(q.units) * tl.z / z_cuts);
-                    const int kt_hi = static_cast<int>(static_cast<long long>(q.units) * (tl.z + 1) / z_cuts);
+                    const int kt_lo = kcut(cuts, q.units, tl.z);
+                    const int kt_hi = kcut(cuts, q.units, tl.z + 1);
                     int checked = -1;
                     for (int kt = kt_lo; kt < kt_hi; ++kt, ++it) {
                         const int p = kt / k_per_group, kk2 = kt - p * k_per_group;
@@ -775,8 +787,8 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                     umma_commit(&tail.acc_full[0]);
                     ++seg;
                 } else {
-                    const int kt_lo = static_cast<int>(static_cast<long long>(q.units) * tl.z / z_cuts);
-                    const int kt_hi = static_cast<int>(static_cast<long long>(q.units) * (tl.z + 1) / z_cuts);
+                    const int kt_lo = kcut(cuts, q.units, tl.z);
+                    const int kt_hi = kcut(cuts, q.units, tl.z + 1);
                     for (int slot = 0; slot < n_slots && alive; ++slot) {
                         const int k0 = max(kt_lo, tail.slot_start[slot] * k_per_group);
                         const int k1 = min(kt_hi, tail.slot_start[slot + 1] * k_per_group);
@@ -864,8 +876,8 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 ++seg;
             } else {
                 const int n0 = tl.nt * BN2;
-                const int kt_lo = static_cast<int>(static_cast<long long>(q.units) * tl.z / z_cuts);
-                const int kt_hi = static_cast<int>(static_cast<long long>(q.units) * (tl.z + 1) / z_cuts);
+                const int kt_lo = kcut(cuts, q.units, tl.z);
+                const int kt_hi = kcut(cuts, q.units, tl.z + 1);
                 for (int slot = 0; slot < n_slots; ++slot) {
                     const int k0 = max(kt_lo, tail.slot_start[slot] * k_per_group);
                     const int k1 = min(kt_hi, tail.slot_start[slot + 1] * k_per_group);
@@ -1094,17 +1106,32 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         const size_t smemf = static_cast<size_t>(kStagesF) * (2 * kBM * kBK * 2 + kBK * 256 * 2) + sizeof(FusedTail) + 16 +
                              kEpiStageBytes + 1024;
         const int tiles2 = ((T + 2 * kBM - 1) / (2 * kBM)) * (d / 256);
-        // K cuts of the down projection: a third more tiles than SMs, so that the CTAs that finish their hidden
-        // tiles late still find down-projection work of a useful size (HALO_TUNE_PREFILL_KCUTS overrides)
-        int z = std::max(1, std::min(8, (n_sm * 4 / 3) / tiles2));
+        // K cuts of the down projection: six runs per output tile on the 7B shape, each 0.75 of the one before
+        // (a model of the tile queue, then a sweep on the GPU: 0.3 ms per 32-block prompt better than six equal
+        // runs); fewer runs when there are many output tiles anyway.  HALO_TUNE_PREFILL_KCUTS and
+        // HALO_TUNE_PREFILL_KRATIO (percent) override.
+        int z = std::max(1, std::min(7, (n_sm * 4 / 3) / tiles2));
+        double ratio = 0.75;
         if (const char* e = getenv("HALO_TUNE_PREFILL_KCUTS")) z = std::max(1, std::min(16, atoi(e)));
+        if (const char* e = getenv("HALO_TUNE_PREFILL_KRATIO")) ratio = std::max(0.3, std::min(1.0, atoi(e) / 100.0));
+        KCuts cuts{};
+        cuts.n = z;
+        {
+            double total = 0.0, run = 1.0, acc = 0.0;
+            for (int i = 0; i < z; ++i, run *= ratio) total += run;
+            run = 1.0;
+            for (int i = 0; i < z; ++i, run *= ratio) {
+                cuts.cum[i] = static_cast<unsigned>(acc / total * 65536.0);
+                acc += run;
+            }
+            cuts.cum[z] = 65536u;
+        }
 #define HALO_LAUNCH_FUSED(NS_)                                                                                       \
     do {                                                                                                             \
         auto kf = ffn_fused_kernel<NS_, kStagesF>;                                                                   \
         static bool oncef[64] = {};                                                                                  \
         if (!ensure_dynamic_smem(kf, smemf, oncef)) return HALO_ERR_CUDA;                                            \
-        kf<<<n_sm, kPfThreads, smemf, st>>>(map_x, map_w, map_w_half, map_h, map_wd, T, d, G,                        \
-                                            n_sm, z, keep_list,                                                      \
+        kf<<<n_sm, kPfThreads, smemf, st>>>(map_x, map_w, map_w_half, map_h, map_wd, cuts, T, d, G, n_sm, keep_list, \
                                             n_keep, dev_of_group, n_dev, collapse, H, sh.d_ffn, partials, ctl,       \
                                             dev_status);                                                             \
     } while (0)

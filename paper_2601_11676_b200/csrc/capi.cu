@@ -414,6 +414,7 @@ struct halo_stack {
     halo::PersistSel* p_sel;       // [3]
     unsigned* p_sync;              // [32]
     void* ffn_ws;                  // H buffer of the tensor-core path (multi-token stacks), or null
+    bool ffn_ws_clean = false;     // its control words are known to be zero
     // multi-token stacks: predictor + selection of block l+1 run on a side stream while block l's FFN runs
     cudaStream_t side;
     cudaEvent_t ev_x, ev_sel;
@@ -712,7 +713,8 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                     // adds its tiles straight into the residual stream, and the glue only normalises
                     HALO_TRY(launch_group_ffn_prefill(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->set_kl[cur],
                                                       s->set_nk[cur], s->set_dev[cur], n_dev, 1, s->h, s->ffn_ws,
-                                                      s->status, st));
+                                                      s->status, st, s->ffn_ws_clean));
+                    s->ffn_ws_clean = true;   // every launch on this workspace leaves the control words zeroed
                     HALO_TRY(launch_glue(static_cast<int>(d), static_cast<int>(T), s->ffn.wdtype, s->h, nullptr, h_dst,
                                          x_next, st));
                     launches += 3;

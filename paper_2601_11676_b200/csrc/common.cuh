@@ -122,7 +122,7 @@ bool prefill_accumulates(const halo_ffn_shape& sh, int n_tok);
 halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                      const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
                                      int n_dev, int collapse, float* partials, void* workspace, uint32_t* dev_status,
-                                     cudaStream_t st);
+                                     cudaStream_t st, bool ctl_clean = false);
 bool pred_gemm_supported(const halo_pred_shape& sh, int n_tok);
 halo_status launch_pred_hidden_gemm(const halo_pred_shape& sh, const void* W1, const void* feat, int n_tok,
                                     float* hidden, uint32_t* dev_status, cudaStream_t st);

@@ -920,6 +920,17 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     __syncthreads();
     if (warp == 1) { tcgen05_fence_after_sync(); tmem_dealloc(tmem, kTmemCols); }
     if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
+    // The last CTA to get here (none reads the control words any more) zeroes them for the next launch.
+    __shared__ int is_last;
+    if (tid == 0) {
+        __threadfence();
+        is_last = atomicAdd(&ctl[1], 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (is_last) {
+        const int n_words = kCtlHeaderWords + q.tiles_x * G;
+        for (int i = tid; i < n_words; i += blockDim.x) ctl[i] = 0u;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -1077,13 +1088,14 @@ size_t prefill_workspace_bytes(const halo_ffn_shape& sh, int n_tok) {
     return prefill_ctl_bytes(sh, n_tok) + static_cast<size_t>(n_tok) * sh.d_ffn * 2;
 }
 
+// ctl_clean: the workspace's control words are known to be zero (left so by an earlier launch on this workspace).
 // partials must already be zero (slots without kept groups are not written).  collapse != 0: the caller wants the
 // sum over holders only and partials has two slots whose SUM is the result; when prefill_accumulates() holds,
 // everything is added into slot 0 (slot 1 is not touched), which may then hold a value to add to.
 halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                      const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
                                      int n_dev, int collapse, float* partials, void* workspace, uint32_t* dev_status,
-                                     cudaStream_t st) {
+                                     cudaStream_t st, bool ctl_clean) {
     const int d = sh.d_model, S = sh.group_size, G = sh.d_ffn / S, T = n_tok;
     const size_t ctl_bytes = prefill_ctl_bytes(sh, T);
     unsigned* ctl = static_cast<unsigned*>(workspace);
@@ -1101,7 +1113,8 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
     static const bool two_launches = [] { const char* e = getenv("HALO_TUNE_PREFILL_TWO_LAUNCHES"); return e && e[0] == '1'; }();
     if (T > kBM && d % 256 == 0 && !two_launches) {
         // both contractions in one launch, one CTA per SM pulling tiles from a queue
-        if (cudaMemsetAsync(ctl, 0, ctl_bytes, st) != cudaSuccess) return HALO_ERR_CUDA;
+        // the kernel leaves its control words zeroed; a workspace of unknown content is zeroed here
+        if (!ctl_clean && cudaMemsetAsync(ctl, 0, ctl_bytes, st) != cudaSuccess) return HALO_ERR_CUDA;
         constexpr int kStagesF = 3;
         const size_t smemf = static_cast<size_t>(kStagesF) * (2 * kBM * kBK * 2 + kBK * 256 * 2) + sizeof(FusedTail) + 16 +
                              kEpiStageBytes + 1024;

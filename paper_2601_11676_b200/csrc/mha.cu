@@ -15,76 +15,115 @@ namespace halo {
 constexpr int kAttnChunk = 128;   // positions per attention block
 constexpr int kOutRows = 16;      // output-projection rows per block
 
+constexpr int kRowsPerWarp = 2;   // rows a warp of the row-product kernels takes, both at once
+constexpr int kRowsPerBlock = 8 * kRowsPerWarp;
+
+// x (d elements, 16-byte aligned) widened into shared memory, 16 bytes per thread and step
 template <typename T>
-__device__ __forceinline__ float warp_row_dot(const T* __restrict__ row, const float* __restrict__ xs, int chunks, int lane) {
+__device__ __forceinline__ void stage_x(const T* __restrict__ x, float* xs, int d) {
     constexpr int E = Elem<T>::kPerChunk;
-    const uint4* r4 = reinterpret_cast<const uint4*>(row);
-    float acc = 0.0f;
-    for (int c0 = lane; c0 < chunks; c0 += 256) {   // eight 16-byte loads in flight per lane
-        uint4 w[8];
+    const uint4* x4 = reinterpret_cast<const uint4*>(x);
+    for (int c = threadIdx.x; c < d / E; c += blockDim.x) {
+        float xf[E];
+        Elem<T>::widen(__ldg(x4 + c), xf);
+#pragma unroll
+        for (int e = 0; e < E; ++e) xs[c * E + e] = xf[e];
+    }
+}
+
+// <row_a, x> and <row_b, x> by one warp; eight 16-byte loads per row and lane in flight (sixteen per lane)
+template <typename T>
+__device__ __forceinline__ void warp_two_rows_dot(const T* __restrict__ row_a, const T* __restrict__ row_b,
+                                                  const float* __restrict__ xs, int chunks, int lane, float& out_a,
+                                                  float& out_b) {
+    constexpr int E = Elem<T>::kPerChunk;
+    const uint4* a4 = reinterpret_cast<const uint4*>(row_a);
+    const uint4* b4 = reinterpret_cast<const uint4*>(row_b);
+    float acc_a = 0.0f, acc_b = 0.0f;
+    for (int c0 = lane; c0 < chunks; c0 += 256) {
+        uint4 wa[8], wb[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int c = c0 + 32 * i;
-            w[i] = c < chunks ? ldg_stream16(r4 + c) : make_uint4(0, 0, 0, 0);
+            wa[i] = c < chunks ? ldg_stream16(a4 + c) : make_uint4(0, 0, 0, 0);
+            wb[i] = c < chunks ? ldg_stream16(b4 + c) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int c = c0 + 32 * i;
             if (c < chunks) {
-                float wf[E];
-                Elem<T>::widen(w[i], wf);
+                float fa[E], fb[E];
+                Elem<T>::widen(wa[i], fa);
+                Elem<T>::widen(wb[i], fb);
 #pragma unroll
-                for (int e = 0; e < E; ++e) acc = fmaf(wf[e], xs[c * E + e], acc);
+                for (int e = 0; e < E; ++e) {
+                    const float xv = xs[c * E + e];
+                    acc_a = fmaf(fa[e], xv, acc_a);
+                    acc_b = fmaf(fb[e], xv, acc_b);
+                }
             }
         }
     }
-    return warp_sum(acc);
+    out_a = warp_sum(acc_a);
+    out_b = warp_sum(acc_b);
 }
 
-// one warp per row of [Wk; Wv]: rows 0..H*dh-1 are keys, the rest values
+// rows of [Wk; Wv]: rows 0..H*dh-1 are keys, the rest values; a warp takes kRowsPerWarp consecutive rows
 template <typename T>
 __global__ void __launch_bounds__(256)
 mha_kv_append_kernel(int d, int H, int dh, int Lmax, const T* __restrict__ Wk, const T* __restrict__ Wv,
                      const T* __restrict__ x, int pos, T* __restrict__ Kc, T* __restrict__ Vc) {
-    extern __shared__ float xs[];
-    for (int c = threadIdx.x; c < d; c += blockDim.x) xs[c] = to_float(x[c]);
+    extern __shared__ __align__(16) float xs[];
+    stage_x(x, xs, d);
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int n = H * dh;
-    const int r = blockIdx.x * 8 + warp;
-    if (r >= 2 * n) return;
-    const bool is_v = r >= n;
-    const int rr = is_v ? r - n : r;
-    const float v = warp_row_dot((is_v ? Wv : Wk) + static_cast<size_t>(rr) * d, xs, d / Elem<T>::kPerChunk, lane);
-    if (lane == 0) {
-        const int h = rr / dh, j = rr - h * dh;
-        (is_v ? Vc : Kc)[(static_cast<size_t>(h) * Lmax + pos) * dh + j] = from_float<T>(v);
+    const int n = H * dh;                       // even (dh % 16 == 0): a pair of rows never straddles keys/values
+    const int r0 = blockIdx.x * kRowsPerBlock + warp * kRowsPerWarp;
+#pragma unroll
+    for (int i = 0; i < kRowsPerWarp; i += 2) {
+        const int r = r0 + i;
+        if (r >= 2 * n) return;
+        const bool is_v = r >= n;
+        const int rr = is_v ? r - n : r;
+        const T* base = (is_v ? Wv : Wk) + static_cast<size_t>(rr) * d;
+        float va, vb;
+        warp_two_rows_dot(base, base + d, xs, d / Elem<T>::kPerChunk, lane, va, vb);
+        if (lane < 2) {
+            const int row = rr + lane, h = row / dh, j = row - h * dh;
+            (is_v ? Vc : Kc)[(static_cast<size_t>(h) * Lmax + pos) * dh + j] = from_float<T>(lane == 0 ? va : vb);
+        }
     }
 }
 
-// q[ki][j] = <Wq_h[j], x> / sqrt(dh) for the kept heads
+// q[ki][j] = <Wq_h[j], x> / sqrt(dh) for the kept heads; a warp takes kRowsPerWarp consecutive rows of one head
 template <typename T>
 __global__ void __launch_bounds__(256)
 mha_q_kernel(int d, int H, int dh, const T* __restrict__ Wp, const T* __restrict__ x,
              const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr, float* __restrict__ q_ws,
              uint32_t* dev_status) {
-    extern __shared__ float xs[];
-    for (int c = threadIdx.x; c < d; c += blockDim.x) xs[c] = to_float(x[c]);
-    __syncthreads();
+    extern __shared__ __align__(16) float xs[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int nk = *n_keep_ptr;
     nk = max(0, min(nk, H));
-    const int r = blockIdx.x * 8 + warp;
-    const int ki = r / dh, j = r - ki * dh;
+    if (blockIdx.x * kRowsPerBlock >= nk * dh) return;     // the whole block lies beyond the kept heads
+    stage_x(x, xs, d);
+    __syncthreads();
+    const int r0 = blockIdx.x * kRowsPerBlock + warp * kRowsPerWarp;   // dh % 16 == 0: the four rows share a head
+    const int ki = r0 / dh, j0 = r0 - ki * dh;
     if (ki >= nk) return;
     const int h = keep_list[ki];
     if (h < 0 || h >= H) {
-        if (lane == 0 && j == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+        if (lane == 0 && j0 == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
         return;
     }
-    const T* row = Wp + ((static_cast<size_t>(h) * 2 + 0) * dh + j) * d;
-    const float v = warp_row_dot(row, xs, d / Elem<T>::kPerChunk, lane);
-    if (lane == 0) q_ws[static_cast<size_t>(ki) * dh + j] = v * rsqrtf(static_cast<float>(dh));
+    const float scale = rsqrtf(static_cast<float>(dh));
+#pragma unroll
+    for (int i = 0; i < kRowsPerWarp; i += 2) {
+        const T* base = Wp + ((static_cast<size_t>(h) * 2 + 0) * dh + j0 + i) * d;
+        float va, vb;
+        warp_two_rows_dot(base, base + d, xs, d / Elem<T>::kPerChunk, lane, va, vb);
+        if (lane < 2) q_ws[static_cast<size_t>(ki) * dh + j0 + i + lane] = (lane == 0 ? va : vb) * scale;
+    }
 }
 
 // attention partial of one (kept head, chunk of 128 positions): m = max score, l = sum exp(s - m),
@@ -167,7 +206,7 @@ mha_attn_kernel(int H, int dh, int Lmax, int pos, const T* __restrict__ Kc, cons
     for (int j = tid; j < dh; j += kAttnChunk) rec[2 + j] = o_acc[j];
 }
 
-// combine the chunk partials of the block's 16 values o_j, then stream the 16 output-projection rows
+// combine the chunk partials of the block's values o_j, then stream their output-projection rows
 template <typename T, int ITERS>
 __global__ void __launch_bounds__(256)
 mha_out_kernel(int d, int H, int dh, const T* __restrict__ Wp, const int32_t* __restrict__ keep_list,
@@ -302,7 +341,7 @@ extern "C" halo_status halo_mha_kv_append(const halo_mha_shape* shape, const voi
     if (pos < 0 || pos >= shape->max_len) return HALO_ERR_ARG;
     if (!aligned16(Wk) || !aligned16(Wv) || !aligned16(x) || !aligned16(K_cache) || !aligned16(V_cache)) return HALO_ERR_ALIGN;
     const int d = shape->d_model, H = shape->n_heads, dh = shape->head_dim;
-    const unsigned blocks = static_cast<unsigned>((2 * H * dh + 7) / 8);
+    const unsigned blocks = static_cast<unsigned>((2 * H * dh + kRowsPerBlock - 1) / kRowsPerBlock);
     const size_t smem = sizeof(float) * d;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (shape->wdtype == HALO_BF16)
@@ -335,7 +374,7 @@ static halo_status group_mha_typed(const halo_mha_shape& sh, const void* Wp, con
     float* attn_ws = ws + static_cast<size_t>(H) * dh;
     const int n_chunks = pos / kAttnChunk + 1;
     if (cudaMemsetAsync(partials, 0, sizeof(float) * static_cast<size_t>(n_dev + 1) * d, st) != cudaSuccess) return HALO_ERR_CUDA;
-    mha_q_kernel<T><<<(H * dh + 7) / 8, 256, sizeof(float) * d, st>>>(d, H, dh, static_cast<const T*>(Wp),
+    mha_q_kernel<T><<<(H * dh + kRowsPerBlock - 1) / kRowsPerBlock, 256, sizeof(float) * d, st>>>(d, H, dh, static_cast<const T*>(Wp),
                                                                       static_cast<const T*>(x), keep_list, n_keep, q_ws,
                                                                       dev_status);
     HALO_CHECK_LAUNCH();

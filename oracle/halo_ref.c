@@ -576,3 +576,30 @@ int halo_ref_group_mha(int d, int H, int dh, int Lmax, int dtype, const void* Wp
     free(q); free(o); free(w); free(ph);
     return rc;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * LM-head neuron groups (Sec. II-A: the LM head only has an up-projection and is a collection of
+ * neuron groups; Sec. III-B.3: its results travel reliably, so nothing is ever lost).
+ * A group is `group_size` consecutive vocabulary rows (the last one may be shorter).  For every
+ * listed group and every token: logits[t][v] = <W[v], x_t>.  Entries of unlisted groups are left
+ * as the caller set them: the groups' outputs are concatenated, never summed.
+ * ------------------------------------------------------------------------------------------- */
+int halo_ref_group_lm_head(int d, int vocab, int group_size, int dtype, const void* W /*[vocab][d]*/,
+                           const void* x /*[n_tok][d]*/, int n_tok, const int32_t* list, int n_list,
+                           double* logits /*[n_tok][vocab]*/) {
+    if (d <= 0 || vocab <= 0 || group_size <= 0 || n_tok <= 0 || n_list < 0) return REF_ERR_SHAPE;
+    int n_groups = (vocab + group_size - 1) / group_size;
+    for (int i = 0; i < n_list; ++i) if (list[i] < 0 || list[i] >= n_groups) return REF_ERR_ARG;
+    for (int i = 0; i < n_list; ++i) {
+        int g = list[i];
+        int v0 = g * group_size, v1 = v0 + group_size < vocab ? v0 + group_size : vocab;
+        for (int t = 0; t < n_tok; ++t)
+            for (int v = v0; v < v1; ++v) {
+                double acc = 0.0;
+                for (int c = 0; c < d; ++c)
+                    acc += ref_widen(W, (size_t)v * d + c, dtype) * ref_widen(x, (size_t)t * d + c, dtype);
+                logits[(size_t)t * vocab + v] = acc;
+            }
+    }
+    return REF_OK;
+}

@@ -327,3 +327,19 @@ def group_mha(Wpacked: np.ndarray, x: np.ndarray, K_cache: np.ndarray, V_cache: 
     if want_head_partials:
         return P, hp[: len(lst)]
     return P
+
+
+def group_lm_head(W: np.ndarray, x: np.ndarray, group_size: int, group_list=None, fill: float = np.nan):
+    """LM-head groups (Sec. II-A, Sec. III-B.3): logits[t][v] = <W[v], x_t> for the rows of the listed groups of
+    `group_size` vocabulary rows; the other entries keep `fill`."""
+    vocab, d = W.shape
+    dt = _dtype_of(W)
+    x2 = x.reshape(-1, d)
+    n_tok = x2.shape[0]
+    n_groups = (vocab + group_size - 1) // group_size
+    lst = np.arange(n_groups, dtype=np.int32) if group_list is None else np.asarray(group_list, dtype=np.int32).reshape(-1)
+    W, x2 = _c(W), _c(x2)
+    out = np.full((n_tok, vocab), fill, dtype=np.float64)
+    _check(lib().halo_ref_group_lm_head(c_int(d), c_int(vocab), c_int(group_size), c_int(dt), _p(W), _p(x2),
+                                        c_int(n_tok), _p(lst), c_int(len(lst)), _p(out)), "group_lm_head")
+    return out

@@ -275,9 +275,79 @@ def run_halo(args, rank, world, local_rank):
         result["other_workloads"] = [decode_brief(n, dev, peak) for n in
                                      ("llama2-13b-decode", "tinyllama-1.1b-decode", "llama2-7b-decode")
                                      if n != wl.name]
+        result["other_blocks"] = other_blocks_report(dev, peak)
     if world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget)
     return result
+
+
+def other_blocks_report(dev, peak, reps=24):
+    """The paper's two other block types at the 7B shape, one token: LM-head groups (32000 x 4096, all groups) and
+    MHA groups (32 heads of 128, 1024 cached positions, K/V append + attention + output projection); microseconds
+    per call and algorithmic GB/s.  Weight sets rotate so that every call streams from HBM."""
+    from paper_2601_11676_b200 import binding as B
+    d, vocab, S, H, dh, Lmax, pos = 4096, 32000, 256, 32, 128, 1024, 1023
+    wl = synth.Workload("blocks", 1, d, 64, 16, 32, "bf16", (0.0, 0.2, 0.6), (2, 1, 1), 500, 1)
+    x = synth.activation(wl, 1, dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def timed(fn):
+        for _ in range(4):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e3)
+        return float(sorted(ts)[len(ts) // 2])
+
+    g = torch.Generator(device="cpu").manual_seed(11)
+    lm = B.lm_shape(d, vocab, S, B.BF16)
+    Wl = [(torch.randn((vocab, d), generator=g) / 64).to(torch.bfloat16).to(dev) for _ in range(3)]
+    logits = torch.empty((1, vocab), dtype=torch.float32, device=dev)
+    i = [0]
+
+    def lm_call():
+        B.halo_group_lm_head(lm, Wl[i[0] % 3], x, 1, None, None, logits, status)
+        i[0] += 1
+
+    lm_us = timed(lm_call)
+    lm_bytes = vocab * d * 2
+    del Wl
+    mh = B.mha_shape(d, H, dh, Lmax, B.BF16)
+    sets = []
+    for l in range(6):
+        Wq, Wk, Wv, Wo = synth.mha_matrices(wl, l, H, dev)
+        Wp = torch.empty((H, 2, dh, d), dtype=torch.bfloat16, device=dev)
+        B.halo_pack_mha_weights(mh, Wq, Wo, Wp)
+        K = torch.randn((H, Lmax, dh), device=dev).to(torch.bfloat16)
+        V = torch.randn((H, Lmax, dh), device=dev).to(torch.bfloat16)
+        sets.append((Wp, Wk, Wv, K, V))
+    ws = torch.empty(B.halo_group_mha_workspace_bytes(mh), dtype=torch.uint8, device=dev)
+    P = torch.empty((4, d), dtype=torch.float32, device=dev)
+    dg = torch.as_tensor([(-1, 0, 1, 2)[h % 4] for h in range(H)], dtype=torch.int32, device=dev)
+    kl = torch.arange(H, dtype=torch.int32, device=dev)
+    nk = torch.tensor([H], dtype=torch.int32, device=dev)
+    j = [0]
+
+    def mha_call():
+        Wp, Wk, Wv, K, V = sets[j[0] % 6]
+        j[0] += 1
+        B.halo_mha_kv_append(mh, Wk, Wv, x, pos, K, V)
+        B.halo_group_mha(mh, Wp, x, K, V, pos, kl, nk, dg, 3, P, ws, status)
+
+    mha_us = timed(mha_call)
+    mha_bytes = 2 * d * d * 2 + H * (2 * dh * d * 2 + 2 * (pos + 1) * dh * 2)
+    return {"lm_head": {"shape": "32000 x 4096 bf16, 125 groups of 256 rows", "us_per_token": lm_us,
+                        "achieved_gbs": lm_bytes / lm_us / 1e3, "frac_of_peak": lm_bytes / lm_us / 1e3 / peak},
+            "mha_groups": {"shape": "32 heads x 128, d 4096, 1024 cached positions, all heads kept",
+                           "us_per_block": mha_us, "achieved_gbs": mha_bytes / mha_us / 1e3,
+                           "frac_of_peak": mha_bytes / mha_us / 1e3 / peak},
+            "device_status": int(status.item())}
 
 
 def decode_brief(name, dev, peak, steps=64, warm=4):

@@ -296,6 +296,27 @@ halo_status halo_group_mha(const halo_mha_shape* shape, const void* W_packed, co
                            size_t workspace_bytes, uint32_t* dev_status, void* stream);
 
 /* ------------------------------------------------------------------------
+ * LM-head neuron groups (Sec. II-A: the LM head "only contains up-projection" and is "also a collection of
+ * neuron groups"; Sec. III-B.3: its results are sent reliably "to ensure the logits are accurate").  A group is
+ * group_size consecutive vocabulary rows (the last group may be shorter).  Nothing is dropped and nothing is
+ * summed: the groups' outputs are concatenated, so there are no holder slots and no arrival mask here; a caller
+ * that distributes the groups over devices uses halo_plan_create / halo_select_groups for the assignment only.
+ *   W device [vocab][d_model] in wdtype (16-byte aligned, d_model % 8 == 0, d_model <= 8192);
+ *   x device [n_tok][d_model] in wdtype; logits device fp32 [n_tok][vocab];
+ *   keep_list / n_keep device: the groups to compute (indices < ceil(vocab / group_size)); both NULL = all.
+ *   For every listed group and token: logits[t][v] = <W[v], x_t> (fp32 accumulation); entries of unlisted
+ *   groups are left untouched.  An index outside the range sets HALO_DEV_BAD_INDEX in *dev_status and that
+ *   group is skipped.  Asynchronous on `stream`; no workspace.
+ * ---------------------------------------------------------------------- */
+typedef struct {
+    int d_model, vocab, group_size;
+    halo_dtype wdtype;
+} halo_lm_shape;
+halo_status halo_group_lm_head(const halo_lm_shape* shape, const void* W, const void* x, int n_tok,
+                               const int32_t* keep_list, const int32_t* n_keep, float* logits, uint32_t* dev_status,
+                               void* stream);
+
+/* ------------------------------------------------------------------------
  * One block, steps a1..a9 in one call (the Pred, Comp and merge of one block of the generation phase,
  * Sec. III-B.3): scores from `feat` (the input of the previous block: one layer ahead), selection and arrival
  * draw for (step, layer), FFN of `x` over the kept groups, merge of what arrived.  Same results as calling

@@ -32,6 +32,7 @@ EXPORTS = [
     "halo_selftest_bounded_wait", "halo_group_importance_workspace_bytes", "halo_group_importance",
     "halo_layer_workspace_bytes", "halo_layer_fused", "halo_read_status",
     "halo_pack_mha_weights", "halo_mha_kv_append", "halo_group_mha_workspace_bytes", "halo_group_mha",
+    "halo_group_lm_head",
 ]
 
 
@@ -45,6 +46,10 @@ class PredShape(Structure):
 
 class MhaShape(Structure):
     _fields_ = [("d_model", c_int), ("n_heads", c_int), ("head_dim", c_int), ("max_len", c_int), ("wdtype", c_int)]
+
+
+class LmShape(Structure):
+    _fields_ = [("d_model", c_int), ("vocab", c_int), ("group_size", c_int), ("wdtype", c_int)]
 
 
 class Taps(Structure):
@@ -120,6 +125,8 @@ def lib() -> ctypes.CDLL:
         L.halo_group_mha_workspace_bytes.argtypes = [POINTER(MhaShape)]
         L.halo_group_mha.argtypes = [POINTER(MhaShape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
                                      c_void_p, c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
+        L.halo_group_lm_head.argtypes = [POINTER(LmShape), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
+                                         c_void_p, c_void_p]
         L.halo_selftest_bounded_wait.argtypes = [c_void_p, c_longlong, c_void_p, c_void_p, c_void_p]
         L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
         _lib = L
@@ -285,6 +292,15 @@ def halo_group_mha(shape: MhaShape, W_packed, x, K_cache, V_cache, pos, keep_lis
                               _ptr(keep_list), _ptr(n_keep), _ptr(dev_of_group), n_dev, _ptr(partials), _ptr(workspace),
                               workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream)),
          "halo_group_mha")
+
+
+def lm_shape(d_model, vocab, group_size, dtype) -> LmShape:
+    return LmShape(d_model, vocab, group_size, dtype)
+
+
+def halo_group_lm_head(shape: LmShape, W, x, n_tok, keep_list, n_keep, logits, dev_status=None, stream=None) -> None:
+    _chk(lib().halo_group_lm_head(byref(shape), _ptr(W), _ptr(x), n_tok, _ptr(keep_list), _ptr(n_keep), _ptr(logits),
+                                  _ptr(dev_status), _stream(stream)), "halo_group_lm_head")
 
 
 def halo_selftest_bounded_wait(never_set_flag, limit_cycles, report, dev_status, stream=None) -> None:

@@ -52,6 +52,52 @@ def test_prefill_more_tiles_than_sms_splits_the_last_wave(d, G, S, n_tok):
         assert np.abs(P.cpu().numpy() - ref).max() <= U.TOL_BF16 * rms, len(keep)
 
 
+@pytest.mark.parametrize("d,G,S,n_tok", [(256, 9, 128, 700), (512, 14, 64, 385)])
+def test_prefill_single_launch_edge_cases(d, G, S, n_tok):
+    """The one-launch form (more than 128 tokens, d % 256 == 0) on three token tiles with a ragged last one: no
+    devices at all, every group on one device, a kept list with bad indices (flagged, skipped), a workspace reused
+    across calls with different kept sets (its control words must come back zeroed)."""
+    wl = _wl(d, G, S)
+    Wp = synth.packed_layer(wl, 0, DEV)
+    x = synth.activation(wl, 1, DEV, n_tok=n_tok)
+    hb = synth.host_bits
+    # no devices: one slot
+    P, status = U.gpu_group_ffn(wl, Wp, x, [0, 2, G - 1], None, 0)
+    ref = R.group_ffn(hb(Wp), hb(x), [0, 2, G - 1])
+    rms = np.sqrt(np.mean(ref ** 2))
+    assert status == 0 and np.abs(P.cpu().numpy() - ref).max() <= U.TOL_BF16 * rms
+    # everything on the last device, slots in between stay zero
+    dev = np.full(G, 2, dtype=np.int32)
+    P, status = U.gpu_group_ffn(wl, Wp, x, list(range(G)), dev, 3)
+    ref = R.group_ffn(hb(Wp), hb(x), list(range(G)), dev, 3)
+    rms = np.sqrt(np.mean(R.merge(ref) ** 2))
+    assert status == 0 and np.abs(P.cpu().numpy() - ref).max() <= U.TOL_BF16 * rms
+    assert (P[:3] == 0).all().item()
+    # bad indices are flagged and skipped
+    dev = (np.arange(G, dtype=np.int32) % 3) - 1
+    P, status = U.gpu_group_ffn(wl, Wp, x, [1, G + 5, 3, -2, 4], dev, 2)
+    ref = R.group_ffn(hb(Wp), hb(x), [1, 3, 4], dev, 2)
+    rms = np.sqrt(np.mean(R.merge(ref) ** 2))
+    assert status & B.DEV_BAD_INDEX
+    assert np.abs(P.cpu().numpy() - ref).max() <= U.TOL_BF16 * rms
+    # one workspace, several calls with different kept sets
+    sh = B.ffn_shape(d, G * S, S, B.BF16)
+    ws = torch.empty(B.halo_group_ffn_workspace_bytes(sh, n_tok, 2), dtype=torch.uint8, device=DEV)
+    dg = torch.as_tensor(dev, device=DEV)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for keep in ([0, 1, 2, 3], [G - 1], list(range(G))[::-1], []):
+        kl = torch.full((G,), -1, dtype=torch.int32, device=DEV)
+        if keep:
+            kl[: len(keep)] = torch.as_tensor(keep, dtype=torch.int32)
+        nk = torch.tensor([len(keep)], dtype=torch.int32, device=DEV)
+        P = torch.full((3, n_tok, d), float("nan"), dtype=torch.float32, device=DEV)
+        B.halo_group_ffn(sh, Wp, x, n_tok, kl, nk, dg, 2, P, ws, st)
+        torch.cuda.synchronize()
+        ref = R.group_ffn(hb(Wp), hb(x), keep, dev, 2)
+        scale = np.sqrt(np.mean(R.merge(ref) ** 2)) if keep else 1.0
+        assert int(st.item()) == 0 and np.abs(P.cpu().numpy() - ref).max() <= U.TOL_BF16 * scale, keep
+
+
 def test_prefill_matches_decode_path_token_by_token():
     wl = _wl(512, 4, 128)
     Wp = synth.packed_layer(wl, 0, DEV)

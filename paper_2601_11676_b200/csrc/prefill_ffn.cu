@@ -60,25 +60,27 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_const
     constexpr uint32_t kTmemCols = MH * 2 * NS;
     PfBarriers& bars = *reinterpret_cast<PfBarriers*>(smem_raw + static_cast<size_t>(STAGES) * kStageBytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int ki = blockIdx.y, m0 = blockIdx.x * (kBM * MH);
+    // A group of S neurons is computed as S / NS tiles of NS neurons: blockIdx.y counts (kept position, tile).
+    const int subs = S / NS;
+    const int kv = blockIdx.y, ki = kv / subs, m0 = blockIdx.x * (kBM * MH);
     int nk = *n_keep_ptr;
     nk = max(0, min(nk, G));
     if (ki >= nk) return;
-    // Tail balancing: the kept groups that fill whole waves of SMs are computed as full tiles (blockIdx.z == 0);
-    // the groups left for the last, partial wave are split into two half-width tiles (blockIdx.z = which half),
-    // when those halves fit in one wave, so the tail takes about half a tile's time.
-    int n_full = nk;
+    // Tail balancing: the tiles that fill whole waves of SMs are computed in full (blockIdx.z == 0); those left
+    // for the last, partial wave are split into two half-width tiles (blockIdx.z = which half), when those halves
+    // fit in one wave, so the tail takes about half a tile's time.
+    int n_full = nk * subs;
     {
-        const int tiles_x = gridDim.x, total = tiles_x * nk;
+        const int tiles_x = gridDim.x, total = tiles_x * nk * subs;
         if (total > n_sm) {
-            const int full_groups = (total / n_sm) * n_sm / tiles_x, left = nk - full_groups;
-            if (left > 0 && 2 * left * tiles_x <= n_sm) n_full = full_groups;
+            const int full_tiles = (total / n_sm) * n_sm / tiles_x, left = nk * subs - full_tiles;
+            if (left > 0 && 2 * left * tiles_x <= n_sm) n_full = full_tiles;
         }
     }
-    const bool split = ki >= n_full;
+    const bool split = kv >= n_full;
     if (!split && blockIdx.z != 0) return;
     const int ns = split ? NS / 2 : NS;                // neurons of the group this CTA computes
-    const int n_off = split ? blockIdx.z * (NS / 2) : 0;
+    const int n_off = (kv - ki * subs) * NS + (split ? blockIdx.z * (NS / 2) : 0);   // first of them in the group
     const CUtensorMap* const map_w = split ? &tmap_w_half : &tmap_w;
     const int g = keep_list[ki];
     if (g < 0 || g >= G) {
@@ -576,7 +578,7 @@ struct FusedTail {
     int tile_ring[2];
 };
 constexpr int kCtlHeaderWords = 32;          // word 0 = tile queue; ready counters follow
-constexpr unsigned kReadyWhen = 8;           // 4 epilogue warps x (2 for a full tile | 1 + 1 for its two halves)
+constexpr unsigned kReadyPerTile = 8;        // 4 epilogue warps x (2 for a full tile | 1 + 1 for its two halves)
 
 struct FusedGeom {
     int tiles_x, n_full, n1_full, n1, n_tiles, n_tn, z_cuts, units;
@@ -604,12 +606,12 @@ __device__ __forceinline__ FusedTile fused_decode(const FusedGeom& q, int t) {
 }
 
 // Bounded wait for a ready counter written by other CTAs.
-__device__ __forceinline__ bool fused_wait_ready(const unsigned* counter, volatile int* abort_flag) {
-    if (ld_acquire_gpu(counter) >= kReadyWhen) return true;
+__device__ __forceinline__ bool fused_wait_ready(const unsigned* counter, unsigned ready_when, volatile int* abort_flag) {
+    if (ld_acquire_gpu(counter) >= ready_when) return true;
     const long long t0 = clock64();
     for (;;) {
         if (*abort_flag) return false;
-        if (ld_acquire_gpu(counter) >= kReadyWhen) return true;
+        if (ld_acquire_gpu(counter) >= ready_when) return true;
         __nanosleep(64);
         if (clock64() - t0 > static_cast<long long>(kWaitLimitCycles)) { *abort_flag = 1; return false; }
     }
@@ -619,13 +621,14 @@ template <int NS, int STAGES>
 __global__ void __launch_bounds__(kPfThreads, 1)
 ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                  const __grid_constant__ CUtensorMap tmap_w_half, const __grid_constant__ CUtensorMap tmap_h,
-                 const __grid_constant__ CUtensorMap tmap_wd, const __grid_constant__ KCuts cuts, int T, int d, int G,
-                 int n_sm,
+                 const __grid_constant__ CUtensorMap tmap_wd, const __grid_constant__ KCuts cuts, int T, int d, int S,
+                 int G, int n_sm,
                  const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
                  const int32_t* __restrict__ dev_of_group, int n_dev, int collapse, __nv_bfloat16* __restrict__ H,
                  int h_cols, float* __restrict__ partials, unsigned* __restrict__ ctl, uint32_t* dev_status) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    constexpr int S = NS, BN2 = 256, MH = 2;
+    constexpr int BN2 = 256, MH = 2;
+    const int subs = S / NS;            // a group of S neurons is computed as S / NS hidden tiles of NS neurons
     constexpr uint32_t kAHalf = kBM * kBK * 2, kABytes = MH * kAHalf;
     constexpr uint32_t kStageBytes = kABytes + kBK * BN2 * 2;   // 64 KiB: the down tile's stage; a hidden stage fits
     constexpr uint32_t kBBlock = kBK * 64 * 2;
@@ -674,17 +677,18 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
     q.n_tn = d / BN2;
     q.z_cuts = cuts.n;
     q.units = tail.slot_lo * k_per_group;    // K tiles of the down projection (valid kept groups only)
-    q.n_full = nk;
+    const int nkv = nk * subs;          // hidden tiles per token tile; FusedTile::ki counts them
+    q.n_full = nkv;
     {
         // hidden tiles of the last, partial wave are cut into two half-width tiles (finer work at the end)
-        const int total = q.tiles_x * nk;
+        const int total = q.tiles_x * nkv;
         if (n_sm > 0 && total > n_sm) {
-            const int full_groups = (total / n_sm) * n_sm / q.tiles_x, left = nk - full_groups;
-            if (left > 0 && 2 * left * q.tiles_x <= n_sm) q.n_full = full_groups;
+            const int full_tiles = (total / n_sm) * n_sm / q.tiles_x, left = nkv - full_tiles;
+            if (left > 0 && 2 * left * q.tiles_x <= n_sm) q.n_full = full_tiles;
         }
     }
     q.n1_full = q.tiles_x * q.n_full;
-    q.n1 = q.n1_full + 2 * q.tiles_x * (nk - q.n_full);
+    q.n1 = q.n1_full + 2 * q.tiles_x * (nkv - q.n_full);
     q.n_tiles = q.n1 + (q.units > 0 ? q.tiles_x * q.n_tn * cuts.n : 0);
 
     if (warp == 0) {
@@ -700,9 +704,11 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 const int m0 = tl.mt * (kBM * MH);
                 bool alive = true;
                 if (tl.kind < 2) {
-                    const int g = keep_list[tl.ki];
+                    const int ki = tl.ki / subs;
+                    const int g = keep_list[ki];
                     const bool valid = g >= 0 && g < G;     // an invalid entry was flagged by build_slot_order
-                    const int ns = tl.kind == 1 ? NS / 2 : NS, n_off = tl.kind == 1 ? tl.half * (NS / 2) : 0;
+                    const int ns = tl.kind == 1 ? NS / 2 : NS;
+                    const int n_off = (tl.ki - ki * subs) * NS + (tl.kind == 1 ? tl.half * (NS / 2) : 0);
                     const CUtensorMap* const map_w = tl.kind == 1 ? &tmap_w_half : &tmap_w;
                     const int gg = valid ? g : 0;
                     for (int kt = 0; kt < n_kt1; ++kt, ++it) {
@@ -726,7 +732,10 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         const int g = tail.group_of[p], kp = tail.kept_pos[p];
                         if (p != checked) {
                             // the hidden tiles of this group and token tile must have been written
-                            if (!fused_wait_ready(&ctl[kCtlHeaderWords + tl.mt * G + kp], abort_flag)) { alive = false; break; }
+                            if (!fused_wait_ready(&ctl[kCtlHeaderWords + tl.mt * G + kp], kReadyPerTile * subs, abort_flag)) {
+                                alive = false;
+                                break;
+                            }
                             fence_proxy_async_all();   // their generic-proxy stores before this thread's TMA reads
                             checked = p;
                         }
@@ -832,8 +841,10 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
             const FusedTile tl = fused_decode(q, t);
             const int m0 = tl.mt * (kBM * MH);
             if (tl.kind < 2) {
-                const int ns = tl.kind == 1 ? NS / 2 : NS, n_off = tl.kind == 1 ? tl.half * (NS / 2) : 0;
-                const int g = keep_list[tl.ki];
+                const int ki = tl.ki / subs;
+                const int ns = tl.kind == 1 ? NS / 2 : NS;
+                const int n_off = (tl.ki - ki * subs) * NS + (tl.kind == 1 ? tl.half * (NS / 2) : 0);
+                const int g = keep_list[ki];
                 const bool ok = pf_wait(&tail.acc_full[0], seg & 1, abort_flag) && g >= 0 && g < G;
                 tcgen05_fence_after_sync();
 #pragma unroll
@@ -846,7 +857,7 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                         tmem_ld_wait();
                         if (ok && row < T) {
                             uint4* dst = reinterpret_cast<uint4*>(H + static_cast<size_t>(row) * h_cols +
-                                                                  static_cast<size_t>(tl.ki) * S + n_off + c0);
+                                                                  static_cast<size_t>(ki) * S + n_off + c0);
 #pragma unroll
                             for (int qq = 0; qq < 4; ++qq) {
                                 uint32_t packed[4];
@@ -870,7 +881,7 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_consta
                 __threadfence();
                 __syncwarp();
                 if (lane == 0) {
-                    if (ok) atomicAdd(&ctl[kCtlHeaderWords + tl.mt * G + tl.ki], tl.kind == 1 ? 1u : 2u);
+                    if (ok) atomicAdd(&ctl[kCtlHeaderWords + tl.mt * G + ki], tl.kind == 1 ? 1u : 2u);
                     mbar_arrive(&tail.acc_empty[0]);
                 }
                 ++seg;
@@ -1067,7 +1078,7 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, 
 }  // namespace
 
 bool prefill_supported(const halo_ffn_shape& sh, int n_tok) {
-    return sh.wdtype == HALO_BF16 && n_tok >= 16 && (sh.group_size == 64 || sh.group_size == 128) &&
+    return sh.wdtype == HALO_BF16 && n_tok >= 16 && (sh.group_size == 64 || sh.group_size == 128 || sh.group_size == 256) &&
            sh.d_model % 128 == 0 && sh.d_ffn / sh.group_size <= HALO_MAX_GROUPS;
 }
 
@@ -1106,8 +1117,9 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return HALO_ERR_CUDA;
     CUtensorMap map_x, map_w, map_w_half, map_h, map_wd;
-    if (!make_map(&map_x, x, T, d, d, kBK, kBM) || !make_map(&map_w, W, w_rows, d, d, kBK, S) ||
-        !make_map(&map_w_half, W, w_rows, d, d, kBK, S / 2) ||
+    const int NS = std::min(S, 128);     // neurons per hidden tile; a 256-neuron group is two tiles
+    if (!make_map(&map_x, x, T, d, d, kBK, kBM) || !make_map(&map_w, W, w_rows, d, d, kBK, NS) ||
+        !make_map(&map_w_half, W, w_rows, d, d, kBK, NS / 2) ||
         !make_map(&map_h, H, T, sh.d_ffn, sh.d_ffn, kBK, kBM) || !make_map(&map_wd, W, w_rows, d, d, 64, kBK))
         return HALO_ERR_CUDA;
     static const bool two_launches = [] { const char* e = getenv("HALO_TUNE_PREFILL_TWO_LAUNCHES"); return e && e[0] == '1'; }();
@@ -1144,11 +1156,12 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         auto kf = ffn_fused_kernel<NS_, kStagesF>;                                                                   \
         static bool oncef[64] = {};                                                                                  \
         if (!ensure_dynamic_smem(kf, smemf, oncef)) return HALO_ERR_CUDA;                                            \
-        kf<<<n_sm, kPfThreads, smemf, st>>>(map_x, map_w, map_w_half, map_h, map_wd, cuts, T, d, G, n_sm, keep_list, \
+        kf<<<n_sm, kPfThreads, smemf, st>>>(map_x, map_w, map_w_half, map_h, map_wd, cuts, T, d, S, G, n_sm,         \
+                                            keep_list,                                                               \
                                             n_keep, dev_of_group, n_dev, collapse, H, sh.d_ffn, partials, ctl,       \
                                             dev_status);                                                             \
     } while (0)
-        if (S == 128) HALO_LAUNCH_FUSED(128); else HALO_LAUNCH_FUSED(64);
+        if (NS == 128) HALO_LAUNCH_FUSED(128); else HALO_LAUNCH_FUSED(64);
 #undef HALO_LAUNCH_FUSED
         HALO_CHECK_LAUNCH();
         return HALO_OK;
@@ -1161,11 +1174,11 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
                              sizeof(PfBarriers) + 1024;                                                              \
         static bool once1[64] = {};                                                                                  \
         if (!ensure_dynamic_smem(k1, smem1, once1)) return HALO_ERR_CUDA;                                            \
-        const dim3 grid1((T + kBM * MH_ - 1) / (kBM * MH_), G, 2);                                                   \
+        const dim3 grid1((T + kBM * MH_ - 1) / (kBM * MH_), G * (S / NS_), 2);                                       \
         k1<<<grid1, kPfThreads, smem1, st>>>(map_x, map_w, map_w_half, T, d, S, G, n_sm, keep_list, n_keep, H,       \
                                              sh.d_ffn, dev_status);                                                  \
     } while (0)
-    if (S == 128) {
+    if (NS == 128) {
         if (T > kBM) HALO_LAUNCH_HIDDEN(128, 2, 3); else HALO_LAUNCH_HIDDEN(128, 1, 4);
     } else {
         if (T > kBM) HALO_LAUNCH_HIDDEN(64, 2, 4); else HALO_LAUNCH_HIDDEN(64, 1, 6);

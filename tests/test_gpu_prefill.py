@@ -16,7 +16,8 @@ def _wl(d, G, S, n_dev=3):
     return synth.Workload("pf", 1, d, G * S, S, 64, "bf16", (0.0, 0.2, 0.6)[:n_dev], (3, 2, 1)[:n_dev], 500, 1)
 
 
-@pytest.mark.parametrize("d,G,S,n_tok", [(256, 3, 128, 32), (512, 5, 64, 130), (1024, 4, 128, 257), (256, 6, 64, 16)])
+@pytest.mark.parametrize("d,G,S,n_tok", [(256, 3, 128, 32), (512, 5, 64, 130), (1024, 4, 128, 257), (256, 6, 64, 16),
+                                         (512, 3, 256, 200), (256, 2, 256, 64), (384, 3, 256, 130)])
 def test_prefill_ffn_small_shapes_all_tokens(d, G, S, n_tok):
     wl = _wl(d, G, S)
     sh = B.ffn_shape(d, G * S, S, B.BF16)
@@ -36,7 +37,8 @@ def test_prefill_ffn_small_shapes_all_tokens(d, G, S, n_tok):
             assert (P == 0).all().item()
 
 
-@pytest.mark.parametrize("d,G,S,n_tok", [(256, 160, 64, 100), (256, 80, 128, 300), (128, 150, 128, 129)])
+@pytest.mark.parametrize("d,G,S,n_tok", [(256, 160, 64, 100), (256, 80, 128, 300), (128, 150, 128, 129),
+                                         (256, 42, 256, 300)])
 def test_prefill_more_tiles_than_sms_splits_the_last_wave(d, G, S, n_tok):
     """With more hidden-layer tiles than SMs the groups of the last wave are computed as two half-width tiles
     each; every token of every kept group is checked, with all groups kept and with a ragged kept list."""

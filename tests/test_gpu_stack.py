@@ -204,6 +204,16 @@ def test_full_size_stack_in_bench_configuration_sampled_blocks(name, steps, samp
         assert (h_out[s].double() - want).abs().max().item() <= 1e-3 * want.abs().max().item()
 
 
+def test_stack_with_the_papers_group_size_of_256():
+    """Sec. II-A fixes the group size to 256: 43 groups at the 7B FFN width, persistent kernel, two blocks."""
+    wl = synth.Workload("g256", 2, 4096, 11008, 256, 256, "bf16", (0.0, 0.1, 0.5), (2, 1, 1), 500, 3)
+    assert wl.n_groups == 43
+    stack, Wp, preds = build_stack(wl)
+    h0, h_out, t = run_with_taps(wl, stack, wl.steps)
+    assert stack.last_launches() == 1
+    check_teacher_forced(wl, Wp, preds, h0, h_out, t, wl.steps)
+
+
 @pytest.mark.parametrize("variant", ["threshold", "act_none", "no_devices", "d8192", "single_device_lossless"])
 def test_stack_persistent_variants(variant):
     """Persistent path under the other settings of the method: threshold choice of the critical groups, a linear

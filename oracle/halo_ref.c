@@ -603,3 +603,21 @@ int halo_ref_group_lm_head(int d, int vocab, int group_size, int dtype, const vo
     }
     return REF_OK;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Late devices (Sec. III-B.3: the master merges what is available after a timeout, so a partial
+ * that comes later than the timeout counts as lost; Eq. 1: device i needs tau * W_i / c_i for the
+ * W_i units it holds, plus the synchronisation time T_c).
+ *   late[i] = 1  iff  tau * units[i] / compute[i] + t_comm > timeout
+ * A device that holds nothing sends nothing and is never late.
+ * ------------------------------------------------------------------------------------------- */
+int halo_ref_late_devices(int n_dev, const int32_t* units, const double* compute, double tau,
+                          double t_comm, double timeout, uint8_t* late) {
+    if (n_dev <= 0 || !units || !compute || !late || tau < 0.0 || t_comm < 0.0 || timeout < 0.0) return REF_ERR_ARG;
+    for (int i = 0; i < n_dev; ++i) {
+        if (units[i] < 0 || !(compute[i] > 0.0)) return REF_ERR_ARG;
+        double t = tau * (double)units[i] / compute[i] + t_comm;
+        late[i] = (units[i] > 0 && t > timeout) ? 1 : 0;
+    }
+    return REF_OK;
+}

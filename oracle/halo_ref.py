@@ -286,6 +286,16 @@ def min_max(m, c, Mt: float, eps: float = 1e-3) -> np.ndarray:
     return r
 
 
+def late_devices(units, compute, tau: float, t_comm: float, timeout: float) -> np.ndarray:
+    """Sec. III-B.3 + Eq. 1: device i is late (its partial counts as lost) iff tau*units[i]/compute[i] + t_comm
+    exceeds the timeout; a device that holds nothing is never late."""
+    u = np.asarray(units, dtype=np.int32); c = np.asarray(compute, dtype=np.float64)
+    late = np.zeros(len(u), dtype=np.uint8)
+    _check(lib().halo_ref_late_devices(c_int(len(u)), _p(u), _p(c), c_double(tau), c_double(t_comm), c_double(timeout),
+                                       _p(late)), "late_devices")
+    return late
+
+
 # --- MHA neuron groups --------------------------------------------------------------------
 
 def pack_mha(Wq: np.ndarray, Wo: np.ndarray, H: int) -> np.ndarray:

@@ -89,3 +89,43 @@ def test_schedulers_reject_models_that_do_not_fit():
         R.min_max([1, 1], [1.0, 1.0], 3.0)
     with pytest.raises(RuntimeError):
         R.min_max([1, 1], [1.0, 0.0], 1.0)
+
+
+# ---- late devices (Sec. III-B.3 timeout, Eq. 1 cost model) ------------------------------------------------------
+
+def test_late_devices_hand_computed():
+    # tau = 2 ms per group; capacities 1, 2, 4 (relative speed); T_c = 0.5 ms; timeout 10 ms
+    #   device 0: 4 groups -> 8.0 + 0.5 = 8.5  on time
+    #   device 1: 10 groups -> 10.0 + 0.5 = 10.5 late
+    #   device 2: 19 groups -> 9.5 + 0.5 = 10.0 exactly the timeout: still merged (late means later than)
+    #   device 3: nothing assigned: never late, whatever its speed
+    late = R.late_devices([4, 10, 19, 0], [1.0, 2.0, 4.0, 1e-9], 2.0, 0.5, 10.0)
+    assert late.tolist() == [0, 1, 0, 0]
+
+
+def test_late_devices_is_monotone_and_matches_brute_force():
+    rng = np.random.default_rng(3)
+    for _ in range(200):
+        n = int(rng.integers(1, 7))
+        units = rng.integers(0, 40, size=n)
+        comp = rng.uniform(0.2, 5.0, size=n)
+        tau, tc, to = rng.uniform(0.1, 3.0), rng.uniform(0.0, 1.0), rng.uniform(1.0, 30.0)
+        late = R.late_devices(units, comp, tau, tc, to)
+        brute = [(1 if (u > 0 and tau * u / c + tc > to) else 0) for u, c in zip(units.tolist(), comp.tolist())]
+        assert late.tolist() == brute
+        assert (R.late_devices(units, comp * 2, tau, tc, to) <= late).all()        # faster devices: never later
+        assert (R.late_devices(units + 1, comp, tau, tc, to) >= late).all()        # more work: never earlier
+    # a min-max schedule equalises tau*W_i/c_i, so either everybody is late or nobody (memory not binding)
+    c = np.array([1.0, 2.0, 5.0])
+    r = R.min_max([1e9] * 3, c, 100.0)
+    units = np.round(r * 800).astype(np.int32)
+    t = 0.1 * units / c
+    assert t.max() - t.min() <= 0.1 * 2 / c.min()
+    assert len(set(R.late_devices(units, c, 0.1, 0.0, float(t.max()) + 1e-9).tolist())) == 1
+
+
+def test_late_devices_rejects_bad_arguments():
+    with pytest.raises(Exception):
+        R.late_devices([1, 2], [1.0, 0.0], 1.0, 0.0, 1.0)
+    with pytest.raises(Exception):
+        R.late_devices([1, -2], [1.0, 1.0], 1.0, 0.0, 1.0)

@@ -140,6 +140,25 @@ halo_status halo_schedule_min_max(int n_dev, const double* mem_budget, const dou
 halo_status halo_ratios_to_share_weights(int n_dev, const double* ratio, uint32_t* share_weight);
 
 /* ------------------------------------------------------------------------
+ * Late devices (Sec. III-B.3: the master merges what is available after a
+ * timeout, so a partial that comes later than the timeout is as good as lost;
+ * Eq. 1: device i needs tau * W_i / c_i for the W_i units it holds, plus the
+ * synchronisation time T_c).  Host only.
+ *   units[i]   groups device i holds per block (e.g. its chunk from
+ *              halo_plan_describe's boundaries); compute[i] = c_i > 0;
+ *   tau        cost of one group on a device of computing power 1;
+ *   t_comm     T_c; timeout in the same unit of time.
+ *   late[i] = 1 iff units[i] > 0 and tau * units[i] / compute[i] + t_comm > timeout.
+ * The path has no clock: a caller applies the mask by giving the late devices a
+ * loss rate of 1 in halo_plan_create (they then hold the least critical groups
+ * and their partials never arrive), or reschedules with Algorithm 2.
+ * HALO_ERR_ARG: NULL pointers, n_dev outside [1, HALO_MAX_DEVICES], negative
+ * units, tau, t_comm or timeout, non-positive computing power.
+ * ---------------------------------------------------------------------- */
+halo_status halo_late_devices(int n_dev, const int32_t* units, const double* compute, double tau, double t_comm,
+                              double timeout, uint8_t* late);
+
+/* ------------------------------------------------------------------------
  * a1. Predictor (Sec. III-B.2, semantic-aware predictors): importance score
  * of every neuron group of a block from semantic features taken one layer
  * ahead.  Bias-free two-layer network

@@ -32,7 +32,7 @@ EXPORTS = [
     "halo_selftest_bounded_wait", "halo_group_importance_workspace_bytes", "halo_group_importance",
     "halo_layer_workspace_bytes", "halo_layer_fused", "halo_read_status",
     "halo_pack_mha_weights", "halo_mha_kv_append", "halo_group_mha_workspace_bytes", "halo_group_mha",
-    "halo_group_lm_head",
+    "halo_group_lm_head", "halo_late_devices",
 ]
 
 
@@ -110,6 +110,8 @@ def lib() -> ctypes.CDLL:
         L.halo_schedule_min_max.argtypes = [c_int, POINTER(c_double), POINTER(c_double), c_double, c_double,
                                             POINTER(c_double)]
         L.halo_ratios_to_share_weights.argtypes = [c_int, POINTER(c_double), POINTER(c_uint32)]
+        L.halo_late_devices.argtypes = [c_int, POINTER(c_int32), POINTER(c_double), c_double, c_double, c_double,
+                                        POINTER(c_uint8)]
         L.halo_group_importance_workspace_bytes.restype = c_size_t
         L.halo_group_importance_workspace_bytes.argtypes = [POINTER(FfnShape)]
         L.halo_group_importance.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p,
@@ -232,6 +234,14 @@ def halo_ratios_to_share_weights(ratio):
     n = len(ratio)
     out = (c_uint32 * n)()
     _chk(lib().halo_ratios_to_share_weights(n, _darr(ratio), out), "halo_ratios_to_share_weights")
+    return list(out)
+
+
+def halo_late_devices(units, compute, tau, t_comm, timeout):
+    n = len(units)
+    out = (c_uint8 * n)()
+    _chk(lib().halo_late_devices(n, (c_int32 * n)(*[int(u) for u in units]), _darr(compute), float(tau), float(t_comm),
+                                 float(timeout), out), "halo_late_devices")
     return list(out)
 
 

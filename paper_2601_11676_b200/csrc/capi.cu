@@ -216,6 +216,19 @@ extern "C" halo_status halo_ratios_to_share_weights(int n_dev, const double* rat
     return HALO_OK;
 }
 
+extern "C" halo_status halo_late_devices(int n_dev, const int32_t* units, const double* compute, double tau,
+                                         double t_comm, double timeout, uint8_t* late) {
+    if (n_dev <= 0 || n_dev > HALO_MAX_DEVICES || !units || !compute || !late) return HALO_ERR_ARG;
+    if (!(tau >= 0.0) || !(t_comm >= 0.0) || !(timeout >= 0.0)) return HALO_ERR_ARG;
+    for (int i = 0; i < n_dev; ++i)
+        if (units[i] < 0 || !(compute[i] > 0.0)) return HALO_ERR_ARG;
+    for (int i = 0; i < n_dev; ++i) {
+        const double busy = tau * static_cast<double>(units[i]) / compute[i] + t_comm;   // Eq. 1, one block
+        late[i] = (units[i] > 0 && busy > timeout) ? 1 : 0;
+    }
+    return HALO_OK;
+}
+
 // ---- a1 ---------------------------------------------------------------------------------------------
 
 extern "C" size_t halo_predict_workspace_bytes(const halo_pred_shape* shape, int n_tok) {

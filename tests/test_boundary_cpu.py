@@ -120,3 +120,29 @@ def test_schedulers_match_oracle_and_feed_the_plan(lib):
             B.halo_schedule_min_max(*bad)
         with pytest.raises(B.HaloError):
             B.halo_schedule_comp_greedy(*bad)
+
+
+def test_late_devices_match_the_oracle_and_feed_the_plan(lib):
+    rng = np.random.default_rng(11)
+    for _ in range(200):
+        n = int(rng.integers(1, 9))
+        units = rng.integers(0, 60, size=n)
+        comp = rng.uniform(0.2, 4.0, size=n)
+        tau, tc, to = float(rng.uniform(0.05, 2.0)), float(rng.uniform(0.0, 1.0)), float(rng.uniform(1.0, 20.0))
+        assert B.halo_late_devices(units, comp, tau, tc, to) == R.late_devices(units, comp, tau, tc, to).tolist()
+    # chunks of a plan -> late devices -> a plan in which they never arrive and hold the least critical groups
+    loss, w = [0.0, 0.2, 0.1], [2, 1, 1]
+    plan = B.Plan(40, loss, w, B.SEL_TOPK, 8, 0.0, 0)
+    order, _, bnd = plan.describe(32)
+    chunk = [0] * 3
+    for pos, dev in enumerate(order):
+        chunk[dev] = bnd[pos + 1] - bnd[pos]
+    assert chunk == [16, 8, 8]
+    late = B.halo_late_devices(chunk, [1.0, 2.0, 0.5], 1.0, 0.0, 10.0)   # busy 16, 4, 16 -> devices 0 and 2 are late
+    assert late == [1, 0, 1]
+    plan2 = B.Plan(40, [1.0 if l else r for l, r in zip(late, loss)], w, B.SEL_TOPK, 8, 0.0, 0)
+    order2, thresh2, _ = plan2.describe(32)
+    assert order2[0] == 1 and thresh2[0] == 1 << 32 and thresh2[2] == 1 << 32 and thresh2[1] < 1 << 32
+    for bad in [([1, 2], [1.0, 0.0], 1.0, 0.0, 1.0), ([1, -1], [1.0, 1.0], 1.0, 0.0, 1.0), ([1], [1.0], -1.0, 0.0, 1.0)]:
+        with pytest.raises(B.HaloError):
+            B.halo_late_devices(*bad)

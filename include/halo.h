@@ -394,6 +394,13 @@ halo_status halo_stack_decode_host(halo_stack* stack, const float* h0_host, int 
  * l+1 overlapped with the weight stream of block l; anything else runs one launch per step of the path.
  * mode 1: always one launch per step of the path (no overlap; for comparison and checking). */
 halo_status halo_stack_set_mode(halo_stack* stack, int mode);
+/* Environment variables read by the library (measurement sweeps only; the defaults are the measured best):
+ *   HALO_TUNE_CROSS_STAGES, HALO_TUNE_L2_AHEAD   persistent kernel: stages fetched across the block barrier, L2
+ *                                                prefetch depth (read at halo_stack_create);
+ *   HALO_TUNE_MAX_STEPS                          persistent kernel: steps per launch before a run is split;
+ *   HALO_TUNE_PREFILL_TWO_LAUNCHES=1             prompt FFN as two launches (hidden, down) instead of one;
+ *   HALO_TUNE_PREFILL_KCUTS, HALO_TUNE_PREFILL_KRATIO   prompt FFN: number of K runs per down-projection tile
+ *                                                and the ratio (percent) between consecutive runs. */
 /* Tracing of the persistent kernel (timing statistics of the generation loop): the caller gives a device
  * buffer trace[n_blocks][halo_stack_trace_width()][8] of 64-bit words; for the first n_blocks blocks of a
  * halo_stack_decode run every thread block records global-timer nanoseconds at: 0 block start, 1 first weight

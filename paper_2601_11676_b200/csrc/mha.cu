@@ -4,9 +4,14 @@
 //                        Sec. III-B.3; keys and values are never dropped)
 //   halo_group_mha       for every kept head h:  q = Wq_h x;  w = softmax(q K_h^T / sqrt(dh)) over positions 0..pos;
 //                        o = w V_h;  partials[slot(h)] += sum_j o_j * Wo_h[j]
-// Three launches: query rows (one warp per row), attention per (head, 128-position chunk) with a running-max
-// partial (m, l, o), and combination + output-projection rows (each block streams 16 rows of the head's slice and
-// adds its column sums to the holder's slot with vector reductions).  Bandwidth-bound like the FFN decode path.
+// halo_group_mha is ONE launch: a cluster of eight thread blocks per kept head (query rows shared through
+// distributed shared memory, positions split over the blocks with an online softmax, each block then streams its
+// part of the head's output-projection slice and adds its column sums to the holder's slot with vector
+// reductions).  The earlier three-launch form (query rows; attention per (head, 128-position chunk) with a
+// running-max partial (m, l, o); combination + output-projection rows) is kept for comparison
+// (HALO_TUNE_MHA_THREE_LAUNCHES=1).  Bandwidth-bound like the FFN decode path.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "tma.cuh"
 
@@ -284,6 +289,216 @@ mha_out_kernel(int d, int H, int dh, const T* __restrict__ Wp, const int32_t* __
     }
 }
 
+// ------------------------------------------------------------------------------------------------------------
+// The three steps above in ONE launch: a cluster of kMhaCluster thread blocks per kept head.  Block r computes
+// dh / 8 query rows and hands them to all blocks of its cluster through distributed shared memory; then takes
+// every 8th run of positions (online softmax over 256-position pieces); the blocks exchange their (m, l) and the
+// slices of o that each other needs; block r finally streams the dh / 8 output-projection rows of its slice.
+// The only waits are the cluster barriers, which the hardware guarantees to be reachable (a cluster is
+// co-scheduled); a block never leaves before the last remote write into its shared memory has been synchronised.
+// ------------------------------------------------------------------------------------------------------------
+constexpr int kMhaCluster = 8;
+constexpr int kMhaMaxRows = 32;     // dh <= 256: at most 32 rows of a head per block
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// store a float into the same shared-memory location of another block of the cluster
+__device__ __forceinline__ void st_remote_f32(float* local_smem_ptr, uint32_t target_rank, float v) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(local_smem_ptr)), "r"(target_rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+
+template <typename T, int ITERS>
+__global__ void __cluster_dims__(kMhaCluster, 1, 1) __launch_bounds__(256)
+mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ Wp, const T* __restrict__ x,
+                 const T* __restrict__ Kc, const T* __restrict__ Vc, const int32_t* __restrict__ keep_list,
+                 const int32_t* __restrict__ n_keep_ptr, const int32_t* __restrict__ dev_of_group, int n_dev,
+                 float* __restrict__ partials, uint32_t* dev_status) {
+    constexpr int E = Elem<T>::kPerChunk;
+    extern __shared__ __align__(16) float xs[];          // [d]: x widened
+    __shared__ float q_s[256];                           // the head's full query (written by all blocks of the cluster)
+    __shared__ float o_acc[256];                         // this block's running o over its positions
+    __shared__ float w_s[256];                           // softmax weights of the current piece
+    __shared__ float red[16];
+    __shared__ float ml_in[kMhaCluster][2];              // (m, l) of every block of the cluster
+    __shared__ float o_in[kMhaCluster][kMhaMaxRows];     // their o restricted to this block's rows
+    __shared__ float o_s[kMhaMaxRows];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int r = static_cast<int>(cluster_rank());
+    const int ki = blockIdx.y;
+    int nk = *n_keep_ptr;
+    nk = max(0, min(nk, H));
+    if (ki >= nk) return;                                // the same decision in every block of the cluster
+    const int h = keep_list[ki];
+    if (h < 0 || h >= H) {
+        if (tid == 0 && r == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+        return;
+    }
+    int slot = 0;
+    if (dev_of_group) {
+        slot = dev_of_group[h] + 1;
+        if (slot < 0 || slot > n_dev) {
+            if (tid == 0 && r == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+            return;
+        }
+    }
+    const int rows = dh / kMhaCluster;                   // rows of the head per block (even: dh % 16 == 0)
+    const int j0 = r * rows;
+    const int chunks = d / E;
+
+    // ---- query rows j0 .. j0 + rows, two per warp and turn, sent to every block of the cluster ----
+    stage_x(x, xs, d);
+    for (int j = tid; j < dh; j += 256) o_acc[j] = 0.0f;
+    __syncthreads();
+    const float scale = rsqrtf(static_cast<float>(dh));
+    for (int i = 2 * warp; i < rows; i += 16) {
+        const T* base = Wp + ((static_cast<size_t>(h) * 2 + 0) * dh + j0 + i) * d;
+        float va, vb;
+        warp_two_rows_dot(base, base + d, xs, chunks, lane, va, vb);
+        if (lane < kMhaCluster) {
+            st_remote_f32(&q_s[j0 + i], lane, va * scale);
+            st_remote_f32(&q_s[j0 + i + 1], lane, vb * scale);
+        }
+    }
+    cluster_barrier();                                   // q_s complete everywhere
+
+    // ---- this block's positions: pieces r, r + 8, r + 16, ... of 256 positions; running (m, l, o) ----
+    float m_run = -INFINITY, l_run = 0.0f;
+    const int n_pos = pos + 1;
+    const int col_groups = dh / E;                       // 16-byte groups per value row
+    const int pos_groups = 256 / col_groups;             // threads per column group
+    const int cg = tid % col_groups, pg = tid / col_groups;
+    for (int p0 = r * 256; p0 < n_pos; p0 += kMhaCluster * 256) {
+        const int p = p0 + tid;
+        const bool valid = p < n_pos;
+        float sc = -INFINITY;
+        if (valid) {
+            const uint4* krow = reinterpret_cast<const uint4*>(Kc + (static_cast<size_t>(h) * Lmax + p) * dh);
+            float acc = 0.0f;
+#pragma unroll 8
+            for (int c = 0; c < col_groups; ++c) {
+                float kf[E];
+                Elem<T>::widen(__ldg(krow + c), kf);
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc = fmaf(kf[e], q_s[c * E + e], acc);
+            }
+            sc = acc;
+        }
+        float m = sc;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0) red[warp] = m;
+        __syncthreads();
+        m = red[0];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) m = fmaxf(m, red[w]);
+        const float m_new = fmaxf(m_run, m);             // finite: the piece holds at least one position
+        const float keep_old = __expf(m_run - m_new);    // 0 on the first piece (m_run = -inf)
+        const float e = valid ? __expf(sc - m_new) : 0.0f;
+        w_s[tid] = e;
+        float l = warp_sum(e);
+        if (lane == 0) red[8 + warp] = l;
+        for (int j = tid; j < dh; j += 256) o_acc[j] *= keep_old;
+        __syncthreads();
+        l = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) l += red[8 + w];
+        l_run = l_run * keep_old + l;
+        m_run = m_new;
+        const int n_valid = min(256, n_pos - p0);
+        if (pg < pos_groups) {
+            float part[E];
+#pragma unroll
+            for (int k = 0; k < E; ++k) part[k] = 0.0f;
+            const uint4* vbase = reinterpret_cast<const uint4*>(Vc + (static_cast<size_t>(h) * Lmax + p0) * dh) + cg;
+#pragma unroll 8
+            for (int pp = pg; pp < n_valid; pp += pos_groups) {
+                float vf[E];
+                Elem<T>::widen(__ldg(vbase + static_cast<size_t>(pp) * col_groups), vf);
+                const float wp = w_s[pp];
+#pragma unroll
+                for (int k = 0; k < E; ++k) part[k] = fmaf(wp, vf[k], part[k]);
+            }
+#pragma unroll
+            for (int k = 0; k < E; ++k) atomicAdd(&o_acc[cg * E + k], part[k]);
+        }
+        __syncthreads();                                 // o_acc, w_s and red are free for the next piece
+    }
+
+    // ---- exchange: block r' gets (m, l) of this block and the o values of ITS rows ----
+    if (tid < kMhaCluster) {
+        st_remote_f32(&ml_in[r][0], tid, m_run);
+        st_remote_f32(&ml_in[r][1], tid, l_run);
+    }
+    for (int j = tid; j < dh; j += 256) st_remote_f32(&o_in[r][j % rows], j / rows, o_acc[j]);
+    cluster_barrier();                                   // the last remote access to anybody's shared memory
+    if (tid < rows) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < kMhaCluster; ++c) M = fmaxf(M, ml_in[c][0]);
+        float L = 0.0f, o = 0.0f;
+#pragma unroll
+        for (int c = 0; c < kMhaCluster; ++c) {
+            const float f = ml_in[c][1] > 0.0f ? __expf(ml_in[c][0] - M) : 0.0f;   // blocks without positions: 0
+            L = fmaf(ml_in[c][1], f, L);
+            o = fmaf(o_in[c][tid], f, o);
+        }
+        o_s[tid] = o / L;
+    }
+    __syncthreads();
+
+    // ---- output-projection rows j0 .. j0 + rows of the head's slice: column sums into the holder's slot ----
+    float acc[ITERS][E];
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i)
+#pragma unroll
+        for (int k = 0; k < E; ++k) acc[i][k] = 0.0f;
+    const T* wrows = Wp + ((static_cast<size_t>(h) * 2 + 1) * dh + j0) * d;
+    constexpr int kAtOnce = ITERS <= 2 ? 8 : 4;          // rows whose 16-byte pieces a thread has in flight
+    for (int jb = 0; jb < rows; jb += kAtOnce) {
+        uint4 wv[kAtOnce][ITERS];
+#pragma unroll
+        for (int jj = 0; jj < kAtOnce; ++jj)
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) {
+                const int c = tid + 256 * i;
+                wv[jj][i] = (c < chunks && jb + jj < rows)
+                                ? ldg_stream16(reinterpret_cast<const uint4*>(wrows + static_cast<size_t>(jb + jj) * d) + c)
+                                : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+        for (int jj = 0; jj < kAtOnce; ++jj) {
+            const float o = jb + jj < rows ? o_s[jb + jj] : 0.0f;
+#pragma unroll
+            for (int i = 0; i < ITERS; ++i) {
+                const int c = tid + 256 * i;
+                if (c < chunks) {
+                    float w8[E];
+                    Elem<T>::widen(wv[jj][i], w8);
+#pragma unroll
+                    for (int k = 0; k < E; ++k) acc[i][k] = fmaf(o, w8[k], acc[i][k]);
+                }
+            }
+        }
+    }
+    float* dst = partials + static_cast<size_t>(slot) * d;
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+        const int c = tid + 256 * i;
+        if (c < chunks) {
+#pragma unroll
+            for (int k = 0; k < E; k += 4) red_add_v4f(dst + c * E + k, acc[i][k], acc[i][k + 1], acc[i][k + 2], acc[i][k + 3]);
+        }
+    }
+}
+
 template <typename T>
 __global__ void mha_pack_kernel(int d, int H, int dh, const T* __restrict__ Wq, const T* __restrict__ Wo, T* __restrict__ Wp) {
     const size_t n = static_cast<size_t>(H) * dh * d;
@@ -374,6 +589,30 @@ static halo_status group_mha_typed(const halo_mha_shape& sh, const void* Wp, con
     float* attn_ws = ws + static_cast<size_t>(H) * dh;
     const int n_chunks = pos / kAttnChunk + 1;
     if (cudaMemsetAsync(partials, 0, sizeof(float) * static_cast<size_t>(n_dev + 1) * d, st) != cudaSuccess) return HALO_ERR_CUDA;
+    static const bool three_launches = [] { const char* e = getenv("HALO_TUNE_MHA_THREE_LAUNCHES"); return e && e[0] == '1'; }();
+    if (!three_launches) {
+        // one launch: a cluster of eight thread blocks per kept head
+        const int iters_f = (d / E + 255) / 256;
+        const dim3 grid_f(kMhaCluster, H);
+        const size_t smem_f = sizeof(float) * d;
+#define HALO_MHA_FUSED(I)                                                                                            \
+    case I:                                                                                                          \
+        mha_fused_kernel<T, I><<<grid_f, 256, smem_f, st>>>(d, H, dh, sh.max_len, pos, static_cast<const T*>(Wp),    \
+                                                            static_cast<const T*>(x), static_cast<const T*>(Kc),     \
+                                                            static_cast<const T*>(Vc), keep_list, n_keep,            \
+                                                            dev_of_group, n_dev, partials, dev_status);              \
+        break;
+        switch (iters_f) {
+            HALO_MHA_FUSED(1)
+            HALO_MHA_FUSED(2)
+            HALO_MHA_FUSED(3)
+            HALO_MHA_FUSED(4)
+            default: return HALO_ERR_SHAPE;
+        }
+#undef HALO_MHA_FUSED
+        HALO_CHECK_LAUNCH();
+        return HALO_OK;
+    }
     mha_q_kernel<T><<<(H * dh + kRowsPerBlock - 1) / kRowsPerBlock, 256, sizeof(float) * d, st>>>(d, H, dh, static_cast<const T*>(Wp),
                                                                       static_cast<const T*>(x), keep_list, n_keep, q_ws,
                                                                       dev_status);

@@ -26,7 +26,9 @@ def _caches(wl, H, L, dh, fill):
 
 
 @pytest.mark.parametrize("dtype,d,H,dh,L,positions", [("f32", 64, 4, 16, 40, (0, 7, 39)), ("bf16", 512, 8, 64, 300, (0, 127, 128, 299)),
-                                                      ("bf16", 4096, 32, 128, 1024, (5, 700, 1023))])
+                                                      ("bf16", 4096, 32, 128, 1024, (5, 700, 1023)),
+                                                      ("bf16", 256, 8, 32, 5000, (255, 2047, 2048, 4999)),
+                                                      ("f32", 512, 2, 256, 70, (0, 69))])
 def test_group_mha_and_kv_append_match_oracle(dtype, d, H, dh, L, positions):
     wl = _wl(dtype, d)
     code = U.dtype_code(wl)

@@ -621,3 +621,68 @@ int halo_ref_late_devices(int n_dev, const int32_t* units, const double* compute
     }
     return REF_OK;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * int4 group-quantised weights.  The paper evaluates models "quantized to 4-bit integer
+ * precision" (Sec. IV-A) and picks the neuron-group size "for compatibility with quantization"
+ * (Sec. II-A) but gives no format; the reading taken here: symmetric, one scale per block of 128
+ * consecutive elements of a stored (packed) row,
+ *   s = bf16(amax / 7)   (fp32 division, round-to-nearest-even to bf16; amax = max |w| of the block)
+ *   q = clamp(rint(w / s), -8, 7)   (fp32 division, round-half-even; s == 0 -> q = 0)
+ * stored as nibble q + 8; element 2i in the low half of byte i, element 2i+1 in the high half.
+ * The decisions are taken in fp32 on both sides (here and on the GPU), so codes and scales
+ * compare bit for bit.  Dequantised value: (nibble - 8) * s, exact in fp32.
+ * ------------------------------------------------------------------------------------------- */
+#define REF_QBLOCK 128
+
+static float ref_bf16_bits_to_float(uint16_t b) {
+    uint32_t bits = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return f;
+}
+
+int halo_ref_quantize_i4(int d, long long n_rows, int dtype, const void* W, uint8_t* Q /*[n_rows][d/2]*/,
+                         uint16_t* scales /*[n_rows][d/128]*/) {
+    if (d <= 0 || d % REF_QBLOCK != 0 || n_rows < 0 || !W || !Q || !scales) return REF_ERR_SHAPE;
+    int nb = d / REF_QBLOCK;
+    for (long long r = 0; r < n_rows; ++r)
+        for (int b = 0; b < nb; ++b) {
+            size_t base = (size_t)r * d + (size_t)b * REF_QBLOCK;
+            float amax = 0.0f;
+            for (int e = 0; e < REF_QBLOCK; ++e) {
+                float w = (float)ref_widen(W, base + e, dtype);     /* exact: the stored types fit fp32 */
+                float a = fabsf(w);
+                if (a > amax) amax = a;
+            }
+            float s32 = amax / 7.0f;
+            uint16_t sb = ref_double_to_bf16((double)s32);
+            float s = ref_bf16_bits_to_float(sb);
+            scales[(size_t)r * nb + b] = sb;
+            for (int e = 0; e < REF_QBLOCK; e += 2) {
+                int q[2];
+                for (int k = 0; k < 2; ++k) {
+                    float w = (float)ref_widen(W, base + e + k, dtype);
+                    float t = s > 0.0f ? rintf(w / s) : 0.0f;
+                    if (t < -8.0f) t = -8.0f;
+                    if (t > 7.0f) t = 7.0f;
+                    q[k] = (int)t;
+                }
+                Q[(base + e) / 2] = (uint8_t)((q[0] + 8) | ((q[1] + 8) << 4));
+            }
+        }
+    return REF_OK;
+}
+
+int halo_ref_dequantize_i4(int d, long long n_rows, const uint8_t* Q, const uint16_t* scales, float* W32) {
+    if (d <= 0 || d % REF_QBLOCK != 0 || n_rows < 0 || !Q || !scales || !W32) return REF_ERR_SHAPE;
+    int nb = d / REF_QBLOCK;
+    for (long long r = 0; r < n_rows; ++r)
+        for (int c = 0; c < d; ++c) {
+            size_t i = (size_t)r * d + c;
+            int nib = (Q[i / 2] >> ((c & 1) * 4)) & 15;
+            float s = ref_bf16_bits_to_float(scales[(size_t)r * nb + c / REF_QBLOCK]);
+            W32[i] = (float)(nib - 8) * s;     /* at most 4 + 8 significant bits: exact */
+        }
+    return REF_OK;
+}

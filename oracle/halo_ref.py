@@ -296,6 +296,41 @@ def late_devices(units, compute, tau: float, t_comm: float, timeout: float) -> n
     return late
 
 
+# --- int4 group-quantised weights -----------------------------------------------------------
+
+QBLOCK = 128
+
+
+def quantize_i4(W: np.ndarray):
+    """Packed rows [..., d] (float32 or bf16 bits) -> (codes uint8 [..., d/2], scales bf16 bits [..., d/128]);
+    symmetric, s = bf16(amax/7), q = clamp(rint(w/s), -8, 7), nibble = q + 8, element 2i in the low half of byte i."""
+    d = W.shape[-1]
+    n_rows = int(np.prod(W.shape[:-1]))
+    dt = _dtype_of(W)
+    W = _c(W)
+    Q = np.empty(W.shape[:-1] + (d // 2,), dtype=np.uint8)
+    Sc = np.empty(W.shape[:-1] + (d // QBLOCK,), dtype=np.uint16)
+    _check(lib().halo_ref_quantize_i4(c_int(d), ctypes.c_longlong(n_rows), c_int(dt), _p(W), _p(Q), _p(Sc)), "quantize_i4")
+    return Q, Sc
+
+
+def dequantize_i4(Q: np.ndarray, Sc: np.ndarray) -> np.ndarray:
+    """(codes, scales) -> float32 rows [..., d]: (nibble - 8) * scale, exact."""
+    d = Q.shape[-1] * 2
+    n_rows = int(np.prod(Q.shape[:-1]))
+    Q, Sc = _c(Q), _c(Sc)
+    W = np.empty(Q.shape[:-1] + (d,), dtype=np.float32)
+    _check(lib().halo_ref_dequantize_i4(c_int(d), ctypes.c_longlong(n_rows), _p(Q), _p(Sc), _p(W)), "dequantize_i4")
+    return W
+
+
+def group_ffn_i4(Q: np.ndarray, Sc: np.ndarray, x: np.ndarray, group_list, dev_of_group=None, n_dev: int = 0):
+    """The group FFN on int4 weights = the group FFN on their dequantised values (x widened exactly to fp32)."""
+    W32 = dequantize_i4(Q, Sc)
+    x32 = to_f64(x).astype(np.float32)          # bf16 -> fp32 is exact
+    return group_ffn(W32, x32, group_list, dev_of_group, n_dev)
+
+
 # --- MHA neuron groups --------------------------------------------------------------------
 
 def pack_mha(Wq: np.ndarray, Wo: np.ndarray, H: int) -> np.ndarray:

@@ -1,0 +1,81 @@
+"""Pins for the oracle's int4 group quantisation (symmetric, blocks of 128 stored elements, bf16 scale)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import halo_ref as R
+
+
+def _bf16_bits(a):
+    return torch.as_tensor(np.asarray(a, dtype=np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+
+def test_values_on_the_grid_come_back_exactly_and_the_nibble_order_is_low_half_first():
+    # one block whose values are k * 0.5 for k = -7 .. 7: amax = 3.5, s = 0.5 exactly, q = k
+    ks = np.array(([-7, 7, 0, 1, -1, 3, -4, 6] * 16), dtype=np.int32)
+    W = (ks * 0.5).astype(np.float32).reshape(1, 128)
+    Q, Sc = R.quantize_i4(W)
+    assert Q.shape == (1, 64) and Sc.shape == (1, 1)
+    assert Sc[0, 0] == _bf16_bits([0.5])[0]
+    assert (Q[0] & 15).tolist() == (ks[0::2] + 8).tolist()        # element 2i: low half of byte i
+    assert (Q[0] >> 4).tolist() == (ks[1::2] + 8).tolist()        # element 2i+1: high half
+    assert (R.dequantize_i4(Q, Sc) == W).all()
+
+
+def test_zero_block_halfway_cases_and_scale_rounding():
+    W = np.zeros((1, 256), dtype=np.float32)
+    # second block: amax 7 -> s = 1; 2.5 and 3.5 are ties -> 2 and 4 (half to even); -0.5 -> -0, 0.5 -> 0
+    W[0, 128:136] = [7.0, 2.5, 3.5, -2.5, -0.5, 0.5, -7.0, 6.49]
+    Q, Sc = R.quantize_i4(W)
+    assert Sc[0, 0] == 0 and (Q[0, :64] == 0x88).all()           # all-zero block: scale 0, every code 0 (nibble 8)
+    assert Sc[0, 1] == _bf16_bits([1.0])[0]
+    deq = R.dequantize_i4(Q, Sc)[0, 128:136]
+    assert deq.tolist() == [7.0, 2.0, 4.0, -2.0, 0.0, 0.0, -7.0, 6.0]
+    # a scale that is not a bf16 number: amax = 1 -> 1/7 = 0.142857.. -> bf16 0.142578125 (nearest of 0.1416, 0.1426)
+    W2 = np.zeros((1, 128), dtype=np.float32)
+    W2[0, 0] = 1.0
+    Q2, Sc2 = R.quantize_i4(W2)
+    s = float(R.to_f64(Sc2)[0, 0])
+    assert s == 0.142578125
+    assert (Q2[0, 0] & 15) == 7 + 8                               # 1 / s = 7.01.. -> 7, no clipping trouble
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_error_bound_and_brute_force_python(dtype):
+    g = torch.Generator().manual_seed(5)
+    Wt = (torch.randn((6, 3, 5, 256), generator=g) * torch.rand((6, 3, 5, 1), generator=g) * 3).to(dtype)
+    Wb = Wt.view(torch.int16).numpy().view(np.uint16) if dtype == torch.bfloat16 else Wt.numpy()
+    Q, Sc = R.quantize_i4(Wb)
+    assert Q.shape == (6, 3, 5, 128) and Sc.shape == (6, 3, 5, 2)
+    w = R.to_f64(Wb).reshape(-1, 2, 128)
+    s = R.to_f64(Sc).reshape(-1, 2, 1)
+    deq = R.dequantize_i4(Q, Sc).astype(np.float64).reshape(-1, 2, 128)
+    # every value within half a step (plus the slack of the rounded scale at the block maximum)
+    assert (np.abs(w - deq) <= 0.5 * s * (1 + 2.0 ** -6)).all()
+    # the scale is amax / 7 to bf16 precision
+    amax = np.abs(w).max(axis=2, keepdims=True)
+    assert (np.abs(s - amax / 7) <= amax / 7 * 2.0 ** -8).all()
+    # brute force in numpy float32 arithmetic, same decisions
+    w32 = w.astype(np.float32)
+    s32 = s.astype(np.float32)
+    q = np.clip(np.rint(w32 / s32), -8, 7).astype(np.int32).reshape(-1, 128)
+    nib = np.empty_like(q)
+    Qf = Q.reshape(-1, 64)
+    nib[:, 0::2] = Qf & 15
+    nib[:, 1::2] = Qf >> 4
+    assert (nib - 8 == q).all()
+
+
+def test_ffn_on_int4_weights_is_the_ffn_on_the_dequantised_values():
+    from paper_2601_11676_b200 import synth
+    wl = synth.Workload("q", 1, 256, 64 * 3, 64, 16, "bf16", (0.0, 0.5), (1, 1), 500, 1)
+    Wp = synth.host_bits(synth.packed_layer(wl, 0))
+    x = synth.host_bits(synth.activation(wl, 1))
+    Q, Sc = R.quantize_i4(Wp)
+    dev = np.array([-1, 0, 1], dtype=np.int32)
+    P4 = R.group_ffn_i4(Q, Sc, x, [0, 2], dev, 2)
+    P16 = R.group_ffn(Wp, x, [0, 2], dev, 2)
+    # same structure: the skipped group's slot is empty, and 4-bit weights stay close to the bf16 result
+    assert (P4[1] == 0).all() and (P16[1] == 0).all()
+    rel = np.abs(P4 - P16).max() / np.abs(P16).max()
+    assert 1e-4 < rel < 0.25

@@ -315,6 +315,26 @@ halo_status halo_group_mha(const halo_mha_shape* shape, const void* W_packed, co
                            size_t workspace_bytes, uint32_t* dev_status, void* stream);
 
 /* ------------------------------------------------------------------------
+ * int4 group-quantised weights for the decode FFN (the paper evaluates models "quantized to 4-bit integer
+ * precision", Sec. IV-A, and fixes the neuron-group size "for compatibility with quantization", Sec. II-A; it
+ * gives no format).  Format used here: symmetric, one bf16 scale per block of 128 consecutive elements of a
+ * packed row: s = bf16(amax / 7), q = clamp(rint(w / s), -8, 7) (fp32 division, round half to even; s == 0
+ * gives q = 0), stored as nibble q + 8 with element 2i in the low half of byte i.  value = (nibble - 8) * s.
+ *   shape: as for halo_group_ffn, with d_model % 128 == 0 and d_model <= 8192; wdtype = type of the SOURCE
+ *     weights for halo_quantize_weights_i4, ignored by halo_group_ffn_i4.
+ *   Q device uint8 [G][3][S][d/2]; scales device bf16 [G][3][S][d/128]; both 16-byte aligned, caller-owned.
+ *   halo_quantize_weights_i4: W_packed (device, layout of halo_pack_weights) -> Q, scales.
+ *   halo_group_ffn_i4: halo_group_ffn on the dequantised weights; x device bf16 [n_tok][d]; partials device
+ *     fp32 [n_dev+1][n_tok][d], zeroed by the call; keep_list / n_keep / dev_of_group / dev_status as there.
+ *     Decode form (one pass over the kept groups' weights per token); no workspace.
+ * ---------------------------------------------------------------------- */
+halo_status halo_quantize_weights_i4(const halo_ffn_shape* shape, const void* W_packed, void* Q, void* scales,
+                                     void* stream);
+halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void* Q, const void* scales, const void* x, int n_tok,
+                              const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
+                              int n_dev, float* partials, uint32_t* dev_status, void* stream);
+
+/* ------------------------------------------------------------------------
  * LM-head neuron groups (Sec. II-A: the LM head "only contains up-projection" and is "also a collection of
  * neuron groups"; Sec. III-B.3: its results are sent reliably "to ensure the logits are accurate").  A group is
  * group_size consecutive vocabulary rows (the last group may be shorter).  Nothing is dropped and nothing is

@@ -32,7 +32,7 @@ EXPORTS = [
     "halo_selftest_bounded_wait", "halo_group_importance_workspace_bytes", "halo_group_importance",
     "halo_layer_workspace_bytes", "halo_layer_fused", "halo_read_status",
     "halo_pack_mha_weights", "halo_mha_kv_append", "halo_group_mha_workspace_bytes", "halo_group_mha",
-    "halo_group_lm_head", "halo_late_devices",
+    "halo_group_lm_head", "halo_late_devices", "halo_quantize_weights_i4", "halo_group_ffn_i4",
 ]
 
 
@@ -129,6 +129,9 @@ def lib() -> ctypes.CDLL:
                                      c_void_p, c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
         L.halo_group_lm_head.argtypes = [POINTER(LmShape), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
                                          c_void_p, c_void_p]
+        L.halo_quantize_weights_i4.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_void_p]
+        L.halo_group_ffn_i4.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
+                                        c_void_p, c_int, c_void_p, c_void_p, c_void_p]
         L.halo_selftest_bounded_wait.argtypes = [c_void_p, c_longlong, c_void_p, c_void_p, c_void_p]
         L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
         _lib = L
@@ -311,6 +314,18 @@ def lm_shape(d_model, vocab, group_size, dtype) -> LmShape:
 def halo_group_lm_head(shape: LmShape, W, x, n_tok, keep_list, n_keep, logits, dev_status=None, stream=None) -> None:
     _chk(lib().halo_group_lm_head(byref(shape), _ptr(W), _ptr(x), n_tok, _ptr(keep_list), _ptr(n_keep), _ptr(logits),
                                   _ptr(dev_status), _stream(stream)), "halo_group_lm_head")
+
+
+def halo_quantize_weights_i4(shape: FfnShape, W_packed, Q, scales, stream=None) -> None:
+    _chk(lib().halo_quantize_weights_i4(byref(shape), _ptr(W_packed), _ptr(Q), _ptr(scales), _stream(stream)),
+         "halo_quantize_weights_i4")
+
+
+def halo_group_ffn_i4(shape: FfnShape, Q, scales, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials,
+                      dev_status=None, stream=None) -> None:
+    _chk(lib().halo_group_ffn_i4(byref(shape), _ptr(Q), _ptr(scales), _ptr(x), n_tok, _ptr(keep_list), _ptr(n_keep),
+                                 _ptr(dev_of_group), n_dev, _ptr(partials), _ptr(dev_status), _stream(stream)),
+         "halo_group_ffn_i4")
 
 
 def halo_selftest_bounded_wait(never_set_flag, limit_cycles, report, dev_status, stream=None) -> None:

@@ -1,0 +1,365 @@
+// int4 group-quantised weights for the decode FFN (steps a6..a8 on 4-bit weights).  The paper evaluates models
+// quantised to 4-bit integers (Sec. IV-A) without giving a format; the one used here: symmetric, one bf16 scale
+// per block of 128 consecutive elements of a packed row, s = bf16(amax / 7), q = clamp(rint(w / s), -8, 7),
+// nibble = q + 8, element 2i in the low half of byte i.
+//
+// halo_quantize_weights_i4: one warp per (row, block); decisions in fp32 with IEEE division and round-half-even.
+// halo_group_ffn_i4: the structure of the generic decode kernel (a thread block walks a contiguous range of kept
+// neurons in batches of 8; phase 1 one warp per neuron against x in shared memory; phase 2 fixed columns per
+// thread, sums kept in registers until the holder changes).  Nibbles are never converted one by one: a word's
+// nibbles k and k+4 are masked into the two halves of a register and OR-ed with 0x4300, which makes them the bf16
+// numbers 128 + nibble; phase 1 feeds those pairs to the mixed-precision FMA against x pre-arranged in the same
+// pairing, phase 2 splits the pair into two fp32 values.  The offset (128 + 8) times the plain sum of x (or of
+// the row factors) is subtracted once per block.
+#include <algorithm>
+
+#include "common.cuh"
+#include "ffn_math.cuh"
+#include "tma.cuh"
+
+namespace halo {
+
+namespace {
+constexpr int kQBlock = 128;
+constexpr int kI4Threads = 256;
+constexpr int kI4Warps = kI4Threads / 32;
+constexpr int kI4BlocksPerSm = 2;
+constexpr float kNibbleBias = 136.0f;      // 128 from the bf16 trick + 8 from the code's zero point
+
+__device__ __forceinline__ uint32_t nibble_pair_bf16(uint32_t word, int k) {
+    return ((word >> (4 * k)) & 0x000F000Fu) | 0x43004300u;      // {128 + nibble k, 128 + nibble k+4} as bf16x2
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+quantize_i4_kernel(int d, long long n_rows, const T* __restrict__ W, uint8_t* __restrict__ Q,
+                   __nv_bfloat16* __restrict__ scales) {
+    const int lane = threadIdx.x & 31;
+    const long long wid = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int nb = d / kQBlock;
+    if (wid >= n_rows * nb) return;
+    const long long row = wid / nb;
+    const int b = static_cast<int>(wid - row * nb);
+    const size_t base = static_cast<size_t>(row) * d + static_cast<size_t>(b) * kQBlock + 4 * lane;
+    float w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) w[e] = to_float(W[base + e]);
+    float amax = fmaxf(fmaxf(fabsf(w[0]), fabsf(w[1])), fmaxf(fabsf(w[2]), fabsf(w[3])));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const __nv_bfloat16 sb = __float2bfloat16_rn(__fdiv_rn(amax, 7.0f));
+    const float s = __bfloat162float(sb);
+    if (lane == 0) scales[static_cast<size_t>(row) * nb + b] = sb;
+    uint32_t packed = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        float t = s > 0.0f ? rintf(__fdiv_rn(w[e], s)) : 0.0f;
+        t = fminf(fmaxf(t, -8.0f), 7.0f);
+        packed |= static_cast<uint32_t>(static_cast<int>(t) + 8) << (4 * e);
+    }
+    reinterpret_cast<uint16_t*>(Q)[base / 4] = static_cast<uint16_t>(packed);   // 4 elements = 2 bytes
+}
+
+template <int ITERS>
+__global__ void __launch_bounds__(kI4Threads, kI4BlocksPerSm)
+group_ffn_i4_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, const __nv_bfloat16* __restrict__ scales,
+                    const __nv_bfloat16* __restrict__ x_all, const int32_t* __restrict__ keep_list,
+                    const int32_t* __restrict__ n_keep_ptr, const int32_t* __restrict__ dev_of_group, int n_dev,
+                    int n_tok, float* __restrict__ partials, uint32_t* dev_status) {
+    extern __shared__ __align__(16) unsigned char smem_b[];
+    const int chunks16 = d / 32;           // 16-byte chunks (32 weights) per row
+    const int chunks8 = d / 16;            // 8-byte chunks (16 weights) per row
+    const int nb = d / kQBlock;
+    uint4* xp = reinterpret_cast<uint4*>(smem_b);                       // [4][chunks16]: x in nibble pairing
+    float* xsum = reinterpret_cast<float*>(smem_b + static_cast<size_t>(d) * 2);   // [chunks16]
+    float* hs = xsum + chunks16;                                        // [kI4Warps]
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tok = blockIdx.y;
+
+    int nk = *n_keep_ptr;
+    if (nk < 0 || nk > G) {
+        if (tid == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+        nk = nk < 0 ? 0 : G;
+    }
+    const long long total = static_cast<long long>(nk) * S;
+    const int lo = static_cast<int>(total * blockIdx.x / gridDim.x);
+    const int hi = static_cast<int>(total * (blockIdx.x + 1) / gridDim.x);
+    if (lo >= hi) return;
+
+    // x: for chunk c and word w of a weight chunk, the four pairs (x[8w+k], x[8w+k+4]), k = 0..3, as bf16x2
+    const uint16_t* xb = reinterpret_cast<const uint16_t*>(x_all + static_cast<size_t>(tok) * d);
+    uint32_t* xp_words = reinterpret_cast<uint32_t*>(xp);
+    for (int i = tid; i < d / 2; i += kI4Threads) {
+        const int c = i / 16, r = i - c * 16, w = r >> 2, k = r & 3;
+        const uint32_t lo16 = xb[32 * c + 8 * w + k], hi16 = xb[32 * c + 8 * w + k + 4];
+        xp_words[(static_cast<size_t>(w) * chunks16 + c) * 4 + k] = lo16 | (hi16 << 16);
+    }
+    for (int c = tid; c < chunks16; c += kI4Threads) {
+        float sx = 0.0f;
+        for (int e = 0; e < 32; ++e) sx += __bfloat162float(x_all[static_cast<size_t>(tok) * d + 32 * c + e]);
+        xsum[c] = sx;
+    }
+    __syncthreads();
+
+    float acc[ITERS][16];
+    float corr[ITERS];
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+        corr[i] = 0.0f;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[i][e] = 0.0f;
+    }
+    int cur_slot = -1;
+    const size_t slot_stride = static_cast<size_t>(n_tok) * d;
+
+    auto flush = [&](int slot) {
+        float* dst = partials + static_cast<size_t>(slot) * slot_stride + static_cast<size_t>(tok) * d;
+#pragma unroll
+        for (int i = 0; i < ITERS; ++i) {
+            const int c = tid + kI4Threads * i;
+            if (c < chunks8) {
+                const float off = kNibbleBias * corr[i];
+#pragma unroll
+                for (int e = 0; e < 16; e += 4)
+                    red_add_v4f(dst + c * 16 + e, acc[i][e] - off, acc[i][e + 1] - off, acc[i][e + 2] - off,
+                                acc[i][e + 3] - off);
+            }
+            corr[i] = 0.0f;
+#pragma unroll
+            for (int e = 0; e < 16; ++e) acc[i][e] = 0.0f;
+        }
+    };
+
+    const size_t row_bytes = static_cast<size_t>(d) / 2;
+
+    // A batch = up to 8 consecutive neurons of one kept group.  (Issuing the gate/up loads of batch t+1 before the
+    // down rows of batch t are consumed was measured and is slower: the extra live registers cost more than the
+    // overlap gains.)
+    struct Batch { int n_next, g, j0, cnt, slot; bool any; };
+    auto find_batch = [&](int n) {
+        Batch bt{n, 0, 0, 0, 0, false};
+        while (n < hi) {
+            const int ki = n / S, j0 = n - ki * S;
+            const int g = keep_list[ki];
+            int slot = 0;
+            bool ok = (g >= 0 && g < G);
+            if (ok && dev_of_group) {
+                slot = dev_of_group[g] + 1;
+                ok = (slot >= 0 && slot <= n_dev);
+            }
+            if (!ok) {  // block-uniform: skip the rest of this group
+                if (tid == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+                n += S - j0;
+                continue;
+            }
+            bt.g = g; bt.j0 = j0; bt.slot = slot; bt.any = true;
+            bt.cnt = min(kI4Warps, min(hi - n, S - j0));
+            bt.n_next = n + bt.cnt;
+            return bt;
+        }
+        bt.n_next = hi;
+        return bt;
+    };
+    // phase-1 operands of this warp's neuron of a batch: 4 chunks of the gate row, 4 of the up row, their scales
+    uint4 wg[4], wu[4];
+    float fg[4], fu[4];
+    auto load_phase1 = [&](const Batch& bt) {
+        if (bt.any && warp < bt.cnt && chunks16 <= 128) {
+            const size_t rg = static_cast<size_t>(bt.g) * 3 * S + bt.j0 + warp, ru = rg + S;
+            const uint4* gate = reinterpret_cast<const uint4*>(Q + rg * row_bytes);
+            const uint4* up = reinterpret_cast<const uint4*>(Q + ru * row_bytes);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int c = lane + 32 * u;
+                if (c < chunks16) {
+                    wg[u] = ldg_stream16(gate + c);
+                    wu[u] = ldg_stream16(up + c);
+                    fg[u] = __bfloat162float(scales[rg * nb + (c >> 2)]);
+                    fu[u] = __bfloat162float(scales[ru * nb + (c >> 2)]);
+                }
+            }
+        }
+    };
+    auto dot_chunk = [&](const uint4& g4, const uint4& u4, float sgf, float suf, int c, float& a, float& b) {
+        float tg0 = 0.0f, tg1 = 0.0f, tu0 = 0.0f, tu1 = 0.0f;
+        const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w};
+        const uint32_t uw[4] = {u4.x, u4.y, u4.z, u4.w};
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const uint4 xq = xp[static_cast<size_t>(w) * chunks16 + c];
+            const uint32_t xk[4] = {xq.x, xq.y, xq.z, xq.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                fma_bf16x2(nibble_pair_bf16(gw[w], k), xk[k], tg0, tg1);
+                fma_bf16x2(nibble_pair_bf16(uw[w], k), xk[k], tu0, tu1);
+            }
+        }
+        const float off = kNibbleBias * xsum[c];
+        a = fmaf(sgf, (tg0 + tg1) - off, a);
+        b = fmaf(suf, (tu0 + tu1) - off, b);
+    };
+
+    Batch cur = find_batch(lo);
+    while (cur.any) {
+        load_phase1(cur);
+        if (cur.slot != cur_slot) {
+            if (cur_slot >= 0) flush(cur_slot);
+            cur_slot = cur.slot;
+        }
+        const size_t group_row = static_cast<size_t>(cur.g) * 3 * S;     // first packed row of the group
+
+        // ---- phase 1: gate / up products, one neuron per warp --------------------------------------------
+        if (warp < cur.cnt) {
+            float a = 0.0f, b = 0.0f;
+            if (chunks16 <= 128) {              // the whole row was fetched ahead
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int c = lane + 32 * u;
+                    if (c < chunks16) dot_chunk(wg[u], wu[u], fg[u], fu[u], c, a, b);
+                }
+            } else {                            // rows longer than 4096: fetched here, 4 chunks at a time
+                const size_t rg = group_row + cur.j0 + warp, ru = rg + S;
+                const uint4* gate = reinterpret_cast<const uint4*>(Q + rg * row_bytes);
+                const uint4* up = reinterpret_cast<const uint4*>(Q + ru * row_bytes);
+                for (int c0 = lane; c0 < chunks16; c0 += 128) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int c = c0 + 32 * u;
+                        if (c < chunks16) {
+                            wg[u] = ldg_stream16(gate + c);
+                            wu[u] = ldg_stream16(up + c);
+                            fg[u] = __bfloat162float(scales[rg * nb + (c >> 2)]);
+                            fu[u] = __bfloat162float(scales[ru * nb + (c >> 2)]);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int c = c0 + 32 * u;
+                        if (c < chunks16) dot_chunk(wg[u], wu[u], fg[u], fu[u], c, a, b);
+                    }
+                }
+            }
+            a = warp_sum(a);
+            b = warp_sum(b);
+            if (lane == 0) hs[warp] = silu_mul(a, b);
+        }
+        __syncthreads();
+
+        // ---- phase 2: down rows, block-wide, 16 fixed columns per thread and turn ---------------------------
+        for (int jb = 0; jb < cur.cnt; jb += 4) {
+            uint2 wd[4][ITERS];
+            float hsv[4][ITERS];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+                for (int i = 0; i < ITERS; ++i) {
+                    const int c = tid + kI4Threads * i;
+                    if (jb + jj < cur.cnt && c < chunks8) {
+                        const size_t rd = group_row + 2 * S + cur.j0 + jb + jj;
+                        wd[jj][i] = __ldg(reinterpret_cast<const uint2*>(Q + rd * row_bytes) + c);
+                        hsv[jj][i] = __bfloat162float(scales[rd * nb + (c >> 3)]);
+                    }
+                }
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                if (jb + jj < cur.cnt) {
+                    const float h = hs[jb + jj];
+#pragma unroll
+                    for (int i = 0; i < ITERS; ++i) {
+                        const int c = tid + kI4Threads * i;
+                        if (c < chunks8) {
+                            const float f = h * hsv[jj][i];
+                            corr[i] += f;
+                            const uint32_t words[2] = {wd[jj][i].x, wd[jj][i].y};
+#pragma unroll
+                            for (int v = 0; v < 2; ++v)
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    const uint32_t p = nibble_pair_bf16(words[v], k);
+                                    acc[i][8 * v + k] = fmaf(f, __uint_as_float(p << 16), acc[i][8 * v + k]);
+                                    acc[i][8 * v + k + 4] = fmaf(f, __uint_as_float(p & 0xffff0000u), acc[i][8 * v + k + 4]);
+                                }
+                        }
+                    }
+                }
+            }
+        }
+        const Batch nxt = find_batch(cur.n_next);
+        __syncthreads();  // hs is rewritten by the next batch
+        cur = nxt;
+    }
+    if (cur_slot >= 0) flush(cur_slot);
+}
+
+halo_status check_i4_shape(const halo_ffn_shape* s) {
+    if (!s) return HALO_ERR_ARG;
+    if (s->d_model <= 0 || s->d_model % kQBlock != 0 || s->d_model > 8192 || s->group_size <= 0 || s->d_ffn <= 0 ||
+        s->d_ffn % s->group_size != 0 || s->d_ffn / s->group_size > HALO_MAX_GROUPS)
+        return HALO_ERR_SHAPE;
+    return HALO_OK;
+}
+}  // namespace
+
+}  // namespace halo
+
+using namespace halo;
+
+extern "C" halo_status halo_quantize_weights_i4(const halo_ffn_shape* shape, const void* W_packed, void* Q,
+                                                void* scales, void* stream) {
+    halo_status rc = check_i4_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (shape->wdtype != HALO_F32 && shape->wdtype != HALO_BF16) return HALO_ERR_DTYPE;
+    if (!W_packed || !Q || !scales) return HALO_ERR_ARG;
+    if (!aligned16(W_packed) || !aligned16(Q) || !aligned16(scales)) return HALO_ERR_ALIGN;
+    const int d = shape->d_model;
+    const long long n_rows = 3ll * shape->d_ffn;
+    const long long warps = n_rows * (d / kQBlock);
+    const unsigned blocks = static_cast<unsigned>((warps + 7) / 8);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (shape->wdtype == HALO_BF16)
+        quantize_i4_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(d, n_rows, static_cast<const __nv_bfloat16*>(W_packed),
+                                                                  static_cast<uint8_t*>(Q),
+                                                                  static_cast<__nv_bfloat16*>(scales));
+    else
+        quantize_i4_kernel<float><<<blocks, 256, 0, st>>>(d, n_rows, static_cast<const float*>(W_packed),
+                                                          static_cast<uint8_t*>(Q), static_cast<__nv_bfloat16*>(scales));
+    return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+}
+
+extern "C" halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void* Q, const void* scales, const void* x,
+                                         int n_tok, const int32_t* keep_list, const int32_t* n_keep,
+                                         const int32_t* dev_of_group, int n_dev, float* partials, uint32_t* dev_status,
+                                         void* stream) {
+    halo_status rc = check_i4_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (!Q || !scales || !x || !keep_list || !n_keep || !partials || n_tok <= 0) return HALO_ERR_ARG;
+    if (n_dev < 0 || n_dev > HALO_MAX_DEVICES || (!dev_of_group && n_dev != 0)) return HALO_ERR_ARG;
+    if (!aligned16(Q) || !aligned16(scales) || !aligned16(x) || !aligned16(partials)) return HALO_ERR_ALIGN;
+    const int d = shape->d_model, S = shape->group_size, G = shape->d_ffn / S;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t bytes = sizeof(float) * static_cast<size_t>(n_dev + 1) * n_tok * d;
+    if (cudaMemsetAsync(partials, 0, bytes, st) != cudaSuccess) return HALO_ERR_CUDA;
+    const int chunks8 = d / 16;
+    const int iters = (chunks8 + kI4Threads - 1) / kI4Threads;
+    const long long max_batches = (static_cast<long long>(G) * S + kI4Warps - 1) / kI4Warps;
+    int dev = 0, sms = kSmCount;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int gx = static_cast<int>(std::min<long long>(max_batches, static_cast<long long>(sms) * kI4BlocksPerSm));
+    const dim3 grid(gx, n_tok);
+    const size_t smem = static_cast<size_t>(d) * 2 + sizeof(float) * (d / 32 + kI4Warps);
+    const uint8_t* q = static_cast<const uint8_t*>(Q);
+    const __nv_bfloat16* sc = static_cast<const __nv_bfloat16*>(scales);
+    const __nv_bfloat16* xt = static_cast<const __nv_bfloat16*>(x);
+    switch (iters) {
+        case 1:
+            group_ffn_i4_kernel<1><<<grid, kI4Threads, smem, st>>>(d, S, G, q, sc, xt, keep_list, n_keep, dev_of_group,
+                                                                   n_dev, n_tok, partials, dev_status);
+            break;
+        case 2:
+            group_ffn_i4_kernel<2><<<grid, kI4Threads, smem, st>>>(d, S, G, q, sc, xt, keep_list, n_keep, dev_of_group,
+                                                                   n_dev, n_tok, partials, dev_status);
+            break;
+        default: return HALO_ERR_SHAPE;
+    }
+    return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+}

@@ -1,0 +1,95 @@
+"""GPU parity of the int4 group-quantised decode FFN: codes and scales bit for bit, outputs against the oracle's
+FFN on the dequantised weights."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import halo_ref as R
+from paper_2601_11676_b200 import binding as B
+from paper_2601_11676_b200 import synth
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+DEV = U.DEV
+
+
+def _quantize(wl, Wp):
+    G, S, d = wl.n_groups, wl.group_size, wl.d_model
+    sh = B.ffn_shape(d, wl.d_ffn, S, U.dtype_code(wl))
+    Q = torch.empty((G, 3, S, d // 2), dtype=torch.uint8, device=DEV)
+    Sc = torch.empty((G, 3, S, d // 128), dtype=torch.bfloat16, device=DEV)
+    B.halo_quantize_weights_i4(sh, Wp, Q, Sc)
+    torch.cuda.synchronize()
+    return sh, Q, Sc
+
+
+def _run(sh, Q, Sc, x, keep, dev, n_dev, G):
+    n_tok, d = x.shape
+    kl = torch.full((G,), -1, dtype=torch.int32, device=DEV)
+    if len(keep):
+        kl[: len(keep)] = torch.as_tensor(np.asarray(keep, dtype=np.int32), device=DEV)
+    nk = torch.tensor([len(keep)], dtype=torch.int32, device=DEV)
+    dg = None if dev is None else torch.as_tensor(np.asarray(dev, dtype=np.int32), device=DEV)
+    P = torch.full((n_dev + 1, n_tok, d), float("nan"), dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.halo_group_ffn_i4(sh, Q, Sc, x, n_tok, kl, nk, dg, n_dev, P, status)
+    torch.cuda.synchronize()
+    return P.cpu().numpy(), int(status.item())
+
+
+@pytest.mark.parametrize("dtype,d,G,S,n_tok", [("bf16", 256, 5, 16, 1), ("f32", 384, 4, 24, 2), ("bf16", 4096, 6, 128, 1),
+                                               ("bf16", 8192, 3, 40, 1), ("bf16", 1024, 7, 256, 3)])
+def test_int4_codes_bit_exact_and_ffn_matches_the_oracle(dtype, d, G, S, n_tok):
+    wl = synth.Workload("q", 1, d, G * S, S, 16, dtype, (0.0, 0.3, 0.6), (1, 1, 1), 500, 1)
+    Wp = synth.packed_layer(wl, 0, DEV)
+    sh, Q, Sc = _quantize(wl, Wp)
+    hb = synth.host_bits
+    Q_ref, Sc_ref = R.quantize_i4(hb(Wp))
+    assert (Q.cpu().numpy() == Q_ref).all()                      # integer work: bit exact
+    assert (hb(Sc) == Sc_ref).all()
+    xw = synth.Workload("qx", 1, d, G * S, S, 16, "bf16", (0.0,), (1,), 500, 1)   # activations are bf16
+    x = synth.activation(xw, 3, DEV, n_tok=n_tok)
+    dev = (np.arange(G, dtype=np.int32) % 4) - 1
+    for keep in (list(range(G)), [g for g in range(G) if g != 1], [G - 1], []):
+        P, status = _run(sh, Q, Sc, x, keep, dev, 3, G)
+        assert status == 0
+        ref = R.group_ffn_i4(Q_ref, Sc_ref, hb(x), keep, dev, 3)
+        if not keep:
+            assert (P == 0).all()
+            continue
+        rms = np.sqrt(np.mean(R.merge(ref) ** 2))
+        assert np.abs(P - ref).max() <= U.TOL_BF16 * rms, (keep, np.abs(P - ref).max() / rms)
+
+
+def test_int4_flags_bad_indices_and_works_without_devices():
+    wl = synth.Workload("q", 1, 512, 64 * 4, 64, 16, "bf16", (), (), 500, 1)
+    Wp = synth.packed_layer(wl, 0, DEV)
+    sh, Q, Sc = _quantize(wl, Wp)
+    x = synth.activation(wl, 1, DEV)
+    P, status = _run(sh, Q, Sc, x, [0, 9, 2], None, 0, 4)
+    assert status & B.DEV_BAD_INDEX
+    Qh, Sh = Q.cpu().numpy(), synth.host_bits(Sc)
+    ref = R.group_ffn_i4(Qh, Sh, synth.host_bits(x), [0, 2])
+    assert np.abs(P - ref).max() <= U.TOL_BF16 * np.sqrt(np.mean(ref ** 2))
+
+
+def test_int4_full_size_7b_block_sampled_groups():
+    """One 7B-shaped block (86 groups of 128, d 4096): codes of sampled groups bit exact, outputs of a kept set
+    against the oracle."""
+    wl = synth.workload("llama2-7b-decode")
+    Wp = synth.packed_layer(wl, 2, DEV)
+    sh, Q, Sc = _quantize(wl, Wp)
+    hb = synth.host_bits
+    sample = [0, 41, 85]
+    Q_ref, Sc_ref = R.quantize_i4(hb(Wp[sample]))
+    assert (Q[sample].cpu().numpy() == Q_ref).all() and (hb(Sc[sample]) == Sc_ref).all()
+    x = synth.activation(wl, 5, DEV)
+    G = wl.n_groups
+    dev = np.full(G, -1, dtype=np.int32)
+    dev[41], dev[85] = 0, 2
+    # keep exactly the sampled groups: the oracle needs only their weights (re-indexed 0, 1, 2)
+    P, status = _run(sh, Q, Sc, x, sample, dev, wl.n_dev, G)
+    assert status == 0
+    ref = R.group_ffn_i4(Q_ref, Sc_ref, hb(x), [0, 1, 2], np.array([-1, 0, 2], dtype=np.int32), wl.n_dev)
+    rms = np.sqrt(np.mean(R.merge(ref) ** 2))
+    assert np.abs(P - ref).max() <= U.TOL_BF16 * rms

@@ -420,6 +420,7 @@ halo_status halo_stack_set_mode(halo_stack* stack, int mode);
  *   HALO_TUNE_MAX_STEPS                          persistent kernel: steps per launch before a run is split;
  *   HALO_TUNE_PREFILL_TWO_LAUNCHES=1             prompt FFN as two launches (hidden, down) instead of one;
  *   HALO_TUNE_MHA_THREE_LAUNCHES=1               halo_group_mha as three launches instead of one;
+ *   HALO_TUNE_I4_NO_RING=1                       halo_group_ffn_i4 on plain loads instead of the shared-memory ring;
  *   HALO_TUNE_PREFILL_KCUTS, HALO_TUNE_PREFILL_KRATIO   prompt FFN: number of K runs per down-projection tile
  *                                                and the ratio (percent) between consecutive runs. */
 /* Tracing of the persistent kernel (timing statistics of the generation loop): the caller gives a device

@@ -4,7 +4,7 @@
 // nibble = q + 8, element 2i in the low half of byte i.
 //
 // halo_quantize_weights_i4: one warp per (row, block); decisions in fp32 with IEEE division and round-half-even.
-// halo_group_ffn_i4: the structure of the generic decode kernel (a thread block walks a contiguous range of kept
+// halo_group_ffn_i4, generic form: the structure of the generic decode kernel (a thread block walks a contiguous range of kept
 // neurons in batches of 8; phase 1 one warp per neuron against x in shared memory; phase 2 fixed columns per
 // thread, sums kept in registers until the holder changes).  Nibbles are never converted one by one: a word's
 // nibbles k and k+4 are masked into the two halves of a register and OR-ed with 0x4300, which makes them the bf16
@@ -12,6 +12,7 @@
 // pairing, phase 2 splits the pair into two fp32 values.  The offset (128 + 8) times the plain sum of x (or of
 // the row factors) is subtracted once per block.
 #include <algorithm>
+#include <cstdlib>
 
 #include "common.cuh"
 #include "ffn_math.cuh"
@@ -291,6 +292,218 @@ group_ffn_i4_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, const __
     if (cur_slot >= 0) flush(cur_slot);
 }
 
+// ------------------------------------------------------------------------------------------------------------
+// Ring form of the same computation for d_model 2048 / 4096 (group size a multiple of 8): one thread block per SM,
+// a producer warp streams batches of 8 neurons (their gate, up and down code rows and the three runs of scales:
+// six bulk copies per stage) into a shared-memory ring, 512 consumer threads work from shared memory, so no
+// consumer ever waits on a global load and the bytes in flight are set by the ring depth.
+//   phase 1  one warp per row (8 gate + 8 up rows); the lane's chunks against x kept in shared memory in the
+//            nibble pairing; the two products of a neuron meet in shared memory;
+//   phase 2  REP replicas of d/16 threads; a replica takes every REP-th down row, a thread owns 16 columns.
+// Every mbarrier wait is bounded; on a timeout the block flags HALO_DEV_TIMEOUT, drains its copies and returns.
+// ------------------------------------------------------------------------------------------------------------
+constexpr int kRingNB = 8;
+constexpr int kRingConsumers = 512;
+constexpr int kRingConsumerWarps = kRingConsumers / 32;
+constexpr int kRingThreads = kRingConsumers + 32;
+__device__ __forceinline__ void ring_consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kRingConsumers) : "memory"); }
+
+struct RingHeader {
+    uint64_t full[8];
+    uint64_t empty[8];
+    int slot[8];        // holder slot of the batch in each stage, -1 = skip
+    int abort_flag;
+    int pad[3];
+    __align__(16) float red[2][2 * kRingNB];
+};
+
+template <int XC, int REP, int STAGES>
+__global__ void __launch_bounds__(kRingThreads, 1)
+group_ffn_i4_ring_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, const __nv_bfloat16* __restrict__ scales,
+                         const __nv_bfloat16* __restrict__ x_all, const int32_t* __restrict__ keep_list,
+                         const int32_t* __restrict__ n_keep_ptr, const int32_t* __restrict__ dev_of_group, int n_dev,
+                         int n_tok, float* __restrict__ partials, uint32_t* dev_status) {
+    constexpr int NB = kRingNB;
+    static_assert(STAGES <= 8 && NB % REP == 0, "ring / replica shape");
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    RingHeader& hd = *reinterpret_cast<RingHeader*>(smem_raw);
+    const int chunks16 = d / 32, chunks8 = d / 16, nb = d / kQBlock;
+    const uint32_t row_bytes = static_cast<uint32_t>(d) / 2u;
+    const uint32_t plane_bytes = row_bytes * NB;                 // codes of one of gate / up / down for a batch
+    const uint32_t sc_bytes = static_cast<uint32_t>(nb) * 2u * NB;   // scales of one plane of a batch
+    const uint32_t stage_bytes = 3u * (plane_bytes + sc_bytes);
+    uint4* xp = reinterpret_cast<uint4*>(smem_raw + 1024);                                  // [4][chunks16]
+    float* xsum = reinterpret_cast<float*>(smem_raw + 1024 + static_cast<size_t>(d) * 2);   // [chunks16]
+    unsigned char* ring = smem_raw + 1024 + static_cast<size_t>(d) * 2 + ((static_cast<size_t>(chunks16) * 4 + 127) & ~size_t(127));
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tok = blockIdx.y;
+    int nk = *n_keep_ptr;
+    if (nk < 0 || nk > G) {
+        if (tid == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+        nk = nk < 0 ? 0 : G;
+    }
+    const int per_group = S / NB;
+    const long long total = static_cast<long long>(nk) * per_group;  // batches
+    const int lo = static_cast<int>(total * blockIdx.x / gridDim.x);
+    const int hi = static_cast<int>(total * (blockIdx.x + 1) / gridDim.x);
+    if (lo >= hi) return;
+    const int n_it = hi - lo;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&hd.full[s], 1); mbar_init(&hd.empty[s], kRingConsumerWarps); }
+        hd.abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    volatile int* abort_flag = &hd.abort_flag;
+
+    if (warp == kRingConsumerWarps) {
+        // ---------------- producer ----------------
+        if (lane == 0) {
+            int issued = 0;
+            for (int it = 0; it < n_it; ++it) {
+                if (*abort_flag) break;
+                const int s = it % STAGES;
+                const uint32_t use = static_cast<uint32_t>(it / STAGES);
+                if (it >= STAGES && !mbar_wait_bounded(&hd.empty[s], (use - 1u) & 1u, abort_flag)) { *abort_flag = 1; break; }
+                const int b = lo + it;
+                const int ki = b / per_group, j0 = (b - ki * per_group) * NB;
+                const int g = keep_list[ki];
+                int slot = 0;
+                bool ok = (g >= 0 && g < G);
+                if (ok && dev_of_group) { slot = dev_of_group[g] + 1; ok = (slot >= 0 && slot <= n_dev); }
+                issued = it + 1;
+                if (!ok) {
+                    flag_status(dev_status, HALO_DEV_BAD_INDEX);
+                    hd.slot[s] = -1;
+                    mbar_arrive(&hd.full[s]);
+                    continue;
+                }
+                hd.slot[s] = slot;
+                unsigned char* dst = ring + static_cast<size_t>(s) * stage_bytes;
+                mbar_arrive_expect_tx(&hd.full[s], stage_bytes);
+#pragma unroll
+                for (int plane = 0; plane < 3; ++plane) {
+                    const size_t row = static_cast<size_t>(g) * 3 * S + static_cast<size_t>(plane) * S + j0;
+                    bulk_copy_g2s(dst + plane * plane_bytes, Q + row * row_bytes, plane_bytes, &hd.full[s]);
+                    bulk_copy_g2s(dst + 3 * plane_bytes + plane * sc_bytes, scales + row * nb, sc_bytes, &hd.full[s]);
+                }
+            }
+            if (*abort_flag) {
+                const int first = issued > STAGES ? issued - STAGES : 0;
+                for (int it = first; it < issued; ++it) {
+                    int never = 0;
+                    mbar_wait_bounded(&hd.full[it % STAGES], static_cast<uint32_t>(it / STAGES) & 1u, &never);
+                }
+                flag_status(dev_status, HALO_DEV_TIMEOUT);
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers ----------------
+    {   // x in the nibble pairing, and its plain sums per 32 elements
+        const uint16_t* xb = reinterpret_cast<const uint16_t*>(x_all + static_cast<size_t>(tok) * d);
+        uint32_t* xp_words = reinterpret_cast<uint32_t*>(xp);
+        for (int i = tid; i < d / 2; i += kRingConsumers) {
+            const int c = i / 16, r = i - c * 16, w = r >> 2, k = r & 3;
+            const uint32_t lo16 = xb[32 * c + 8 * w + k], hi16 = xb[32 * c + 8 * w + k + 4];
+            xp_words[(static_cast<size_t>(w) * chunks16 + c) * 4 + k] = lo16 | (hi16 << 16);
+        }
+        for (int c = tid; c < chunks16; c += kRingConsumers) {
+            float sx = 0.0f;
+            for (int e = 0; e < 32; ++e) sx += __bfloat162float(x_all[static_cast<size_t>(tok) * d + 32 * c + e]);
+            xsum[c] = sx;
+        }
+    }
+    ring_consumer_barrier();
+    const int row = warp;                                  // phase 1: rows 0..7 gate, 8..15 up
+    const int rep = tid / (kRingConsumers / REP);          // phase 2 replica and 8-byte column chunk
+    const int col = tid % (kRingConsumers / REP);
+    float acc[16], corr = 0.0f;
+#pragma unroll
+    for (int e = 0; e < 16; ++e) acc[e] = 0.0f;
+    int cur_slot = -1;
+    const size_t slot_stride = static_cast<size_t>(n_tok) * d;
+
+    auto flush = [&](int slot) {
+        if (col < chunks8) {
+            float* dst = partials + static_cast<size_t>(slot) * slot_stride + static_cast<size_t>(tok) * d + col * 16;
+            const float off = kNibbleBias * corr;
+#pragma unroll
+            for (int e = 0; e < 16; e += 4) red_add_v4f(dst + e, acc[e] - off, acc[e + 1] - off, acc[e + 2] - off, acc[e + 3] - off);
+        }
+        corr = 0.0f;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[e] = 0.0f;
+    };
+
+    for (int it = 0; it < n_it; ++it) {
+        const int s = it % STAGES;
+        const uint32_t parity = static_cast<uint32_t>(it / STAGES) & 1u;
+        if (!*abort_flag && !mbar_wait_bounded(&hd.full[s], parity, abort_flag)) *abort_flag = 1;
+        const int slot = *abort_flag ? -1 : hd.slot[s];
+        const unsigned char* stage = ring + static_cast<size_t>(s) * stage_bytes;
+        const __nv_bfloat16* stage_sc = reinterpret_cast<const __nv_bfloat16*>(stage + 3 * plane_bytes);   // [3][NB][nb]
+        float* red = hd.red[it & 1];
+        if (slot >= 0) {
+            if (slot != cur_slot) {
+                if (cur_slot >= 0) flush(cur_slot);
+                cur_slot = slot;
+            }
+            // phase 1: code rows 0..15 of the stage are the 8 gate rows then the 8 up rows (planes 0, 1 adjacent)
+            const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(row) * row_bytes);
+            const __nv_bfloat16* rs = stage_sc + static_cast<size_t>(row) * nb;
+            float a = 0.0f;
+#pragma unroll
+            for (int u = 0; u < XC; ++u) {
+                const int c = lane + 32 * u;
+                const uint4 w4 = rp[c];
+                const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
+                float t0 = 0.0f, t1 = 0.0f;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    const uint4 xq = xp[static_cast<size_t>(w) * chunks16 + c];
+                    const uint32_t xk[4] = {xq.x, xq.y, xq.z, xq.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) fma_bf16x2(nibble_pair_bf16(ww[w], k), xk[k], t0, t1);
+                }
+                a = fmaf(__bfloat162float(rs[c >> 2]), (t0 + t1) - kNibbleBias * xsum[c], a);
+            }
+            a = warp_sum(a);
+            if (lane == 0) red[row] = a;
+        }
+        ring_consumer_barrier();
+        if (slot >= 0 && col < chunks8) {
+            // phase 2: this replica's down rows, 16 columns of each
+            const unsigned char* down = stage + 2 * plane_bytes;
+            const __nv_bfloat16* ds = stage_sc + static_cast<size_t>(2 * NB) * nb;
+#pragma unroll
+            for (int jj = 0; jj < NB / REP; ++jj) {
+                const int j = jj * REP + rep;
+                const float h = silu_mul(red[j], red[NB + j]);
+                const float f = h * __bfloat162float(ds[static_cast<size_t>(j) * nb + (col >> 3)]);
+                corr += f;
+                const uint2 w2 = reinterpret_cast<const uint2*>(down + static_cast<size_t>(j) * row_bytes)[col];
+                const uint32_t words[2] = {w2.x, w2.y};
+#pragma unroll
+                for (int v = 0; v < 2; ++v)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint32_t p = nibble_pair_bf16(words[v], k);
+                        acc[8 * v + k] = fmaf(f, __uint_as_float(p << 16), acc[8 * v + k]);
+                        acc[8 * v + k + 4] = fmaf(f, __uint_as_float(p & 0xffff0000u), acc[8 * v + k + 4]);
+                    }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&hd.empty[s]);
+    }
+    if (cur_slot >= 0) flush(cur_slot);
+    if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
+}
+
 halo_status check_i4_shape(const halo_ffn_shape* s) {
     if (!s) return HALO_ERR_ARG;
     if (s->d_model <= 0 || s->d_model % kQBlock != 0 || s->d_model > 8192 || s->group_size <= 0 || s->d_ffn <= 0 ||
@@ -339,17 +552,41 @@ extern "C" halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t bytes = sizeof(float) * static_cast<size_t>(n_dev + 1) * n_tok * d;
     if (cudaMemsetAsync(partials, 0, bytes, st) != cudaSuccess) return HALO_ERR_CUDA;
-    const int chunks8 = d / 16;
-    const int iters = (chunks8 + kI4Threads - 1) / kI4Threads;
-    const long long max_batches = (static_cast<long long>(G) * S + kI4Warps - 1) / kI4Warps;
-    int dev = 0, sms = kSmCount;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int gx = static_cast<int>(std::min<long long>(max_batches, static_cast<long long>(sms) * kI4BlocksPerSm));
-    const dim3 grid(gx, n_tok);
-    const size_t smem = static_cast<size_t>(d) * 2 + sizeof(float) * (d / 32 + kI4Warps);
     const uint8_t* q = static_cast<const uint8_t*>(Q);
     const __nv_bfloat16* sc = static_cast<const __nv_bfloat16*>(scales);
     const __nv_bfloat16* xt = static_cast<const __nv_bfloat16*>(x);
+    int dev = 0, sms = kSmCount;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    static const bool no_ring = [] { const char* e = getenv("HALO_TUNE_I4_NO_RING"); return e && e[0] == '1'; }();
+    if ((d == 2048 || d == 4096) && S % kRingNB == 0 && !no_ring) {
+        // ring form: one block per SM
+        constexpr int kStages = 4;
+        const size_t stage = 3 * (static_cast<size_t>(d) / 2 * kRingNB + static_cast<size_t>(d) / kQBlock * 2 * kRingNB);
+        const size_t smem_r = 1024 + static_cast<size_t>(d) * 2 + ((static_cast<size_t>(d) / 32 * 4 + 127) & ~size_t(127)) +
+                              kStages * stage;
+        const long long batches = static_cast<long long>(G) * (S / kRingNB);
+        const dim3 grid_r(static_cast<unsigned>(std::min<long long>(batches, sms)), n_tok);
+        if (d == 4096) {
+            auto k = group_ffn_i4_ring_kernel<4, 2, kStages>;
+            static bool once[64] = {};
+            if (!ensure_dynamic_smem(k, smem_r, once)) return HALO_ERR_CUDA;
+            k<<<grid_r, kRingThreads, smem_r, st>>>(d, S, G, q, sc, xt, keep_list, n_keep, dev_of_group, n_dev, n_tok,
+                                                   partials, dev_status);
+        } else {
+            auto k = group_ffn_i4_ring_kernel<2, 4, kStages>;
+            static bool once[64] = {};
+            if (!ensure_dynamic_smem(k, smem_r, once)) return HALO_ERR_CUDA;
+            k<<<grid_r, kRingThreads, smem_r, st>>>(d, S, G, q, sc, xt, keep_list, n_keep, dev_of_group, n_dev, n_tok,
+                                                   partials, dev_status);
+        }
+        return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+    }
+    const int chunks8 = d / 16;
+    const int iters = (chunks8 + kI4Threads - 1) / kI4Threads;
+    const long long max_batches = (static_cast<long long>(G) * S + kI4Warps - 1) / kI4Warps;
+    const int gx = static_cast<int>(std::min<long long>(max_batches, static_cast<long long>(sms) * kI4BlocksPerSm));
+    const dim3 grid(gx, n_tok);
+    const size_t smem = static_cast<size_t>(d) * 2 + sizeof(float) * (d / 32 + kI4Warps);
     switch (iters) {
         case 1:
             group_ffn_i4_kernel<1><<<grid, kI4Threads, smem, st>>>(d, S, G, q, sc, xt, keep_list, n_keep, dev_of_group,

@@ -113,9 +113,10 @@ def test_prefill_matches_decode_path_token_by_token():
         assert np.abs(P_many[:, t].cpu().numpy() - ref).max() <= U.TOL_BF16 * rms
 
 
-def test_prefill_full_size_7b_block_sampled_tokens():
-    """The prefill workload's shapes (512 tokens, one 7B block); the oracle checks a sample of the tokens."""
-    wl = synth.workload("llama2-7b-prefill")
+@pytest.mark.parametrize("name", ["llama2-7b-prefill", "llama2-13b-decode", "tinyllama-1.1b-decode"])
+def test_prefill_full_size_block_sampled_tokens(name):
+    """512 tokens through one block of each stated shape; the oracle checks a sample of the tokens."""
+    wl = synth.workload(name, n_tok=512) if name.endswith("decode") else synth.workload(name)
     G = wl.n_groups
     Wp = synth.packed_layer(wl, 1, DEV)
     x = synth.activation(wl, 3, DEV, n_tok=wl.n_tok)

@@ -292,7 +292,7 @@ mha_out_kernel(int d, int H, int dh, const T* __restrict__ Wp, const int32_t* __
 // ------------------------------------------------------------------------------------------------------------
 // The three steps above in ONE launch: a cluster of kMhaCluster thread blocks per kept head.  Block r computes
 // dh / 8 query rows and hands them to all blocks of its cluster through distributed shared memory; then takes
-// every 8th run of positions (online softmax over 256-position pieces); the blocks exchange their (m, l) and the
+// every 8th run of positions (online softmax over pieces of up to 256 positions); the blocks exchange their (m, l) and the
 // slices of o that each other needs; block r finally streams the dh / 8 output-projection rows of its slice.
 // The only waits are the cluster barriers, which the hardware guarantees to be reachable (a cluster is
 // co-scheduled); a block never leaves before the last remote write into its shared memory has been synchronised.
@@ -375,9 +375,12 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
     const int col_groups = dh / E;                       // 16-byte groups per value row
     const int pos_groups = 256 / col_groups;             // threads per column group
     const int cg = tid % col_groups, pg = tid / col_groups;
-    for (int p0 = r * 256; p0 < n_pos; p0 += kMhaCluster * 256) {
+    // piece = positions a block takes at a time: an eighth of the context (so that all eight blocks work) in
+    // multiples of 32, at most one position per thread
+    const int piece = min(256, max(32, ((n_pos + kMhaCluster - 1) / kMhaCluster + 31) & ~31));
+    for (int p0 = r * piece; p0 < n_pos; p0 += kMhaCluster * piece) {
         const int p = p0 + tid;
-        const bool valid = p < n_pos;
+        const bool valid = tid < piece && p < n_pos;
         float sc = -INFINITY;
         if (valid) {
             const uint4* krow = reinterpret_cast<const uint4*>(Kc + (static_cast<size_t>(h) * Lmax + p) * dh);
@@ -412,7 +415,7 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
         for (int w = 0; w < 8; ++w) l += red[8 + w];
         l_run = l_run * keep_old + l;
         m_run = m_new;
-        const int n_valid = min(256, n_pos - p0);
+        const int n_valid = min(piece, n_pos - p0);
         if (pg < pos_groups) {
             float part[E];
 #pragma unroll

@@ -113,10 +113,12 @@ def test_prefill_matches_decode_path_token_by_token():
         assert np.abs(P_many[:, t].cpu().numpy() - ref).max() <= U.TOL_BF16 * rms
 
 
-@pytest.mark.parametrize("name", ["llama2-7b-prefill", "llama2-13b-decode", "tinyllama-1.1b-decode"])
-def test_prefill_full_size_block_sampled_tokens(name):
-    """512 tokens through one block of each stated shape; the oracle checks a sample of the tokens."""
-    wl = synth.workload(name, n_tok=512) if name.endswith("decode") else synth.workload(name)
+@pytest.mark.parametrize("name,n_tok", [("llama2-7b-prefill", 512), ("llama2-13b-decode", 512),
+                                        ("tinyllama-1.1b-decode", 512), ("llama2-7b-prefill", 1900)])
+def test_prefill_full_size_block_sampled_tokens(name, n_tok):
+    """A prompt through one block of each stated shape (512 tokens; 1900 = eight token tiles, the last one ragged,
+    more output tiles than SMs); the oracle checks a sample of the tokens."""
+    wl = synth.workload(name, n_tok=n_tok)
     G = wl.n_groups
     Wp = synth.packed_layer(wl, 1, DEV)
     x = synth.activation(wl, 3, DEV, n_tok=wl.n_tok)
@@ -125,7 +127,7 @@ def test_prefill_full_size_block_sampled_tokens(name):
     keep = sel["keep_list"][: sel["n_keep"]]
     P, status = U.gpu_group_ffn(wl, Wp, x, keep, sel["dev_of_group"], wl.n_dev)
     assert status == 0
-    sample = [0, 127, 128, 300, 511]
+    sample = [0, 127, 128, 300, 511] + ([1023, 1024, 1792, 1899] if n_tok > 512 else [])
     xs = synth.host_bits(x)[sample]
     ref = R.group_ffn(synth.host_bits(Wp), xs, keep, sel["dev_of_group"], wl.n_dev)
     y_ref = R.merge(ref)

@@ -125,7 +125,7 @@ def build_stack(wl, dev):
     code = B.F32 if wl.dtype == "f32" else B.BF16
     Wp = [synth.packed_layer(wl, l, dev) for l in range(wl.n_layers)]
     preds = [synth.predictor(wl, l, dev) for l in range(wl.n_layers)]
-    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, B.SEL_TOPK, wl.k_critical, 0.0, wl.seed)
+    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
     ffn = B.ffn_shape(wl.d_model, wl.d_ffn, wl.group_size, code)
     pred = B.pred_shape(wl.d_model, wl.pred_rank, wl.n_groups, code)
     stack = B.Stack(ffn, pred, wl.n_tok, plan, Wp, [p[0] for p in preds], [p[1] for p in preds])
@@ -236,7 +236,7 @@ def run_halo(args, rank, world, local_rank):
         "dtype": wl.dtype, "data": "synthetic",
         "config": {"workload": wl.name, "n_layers": L, "d_model": d, "d_ffn": wl.d_ffn, "group_size": wl.group_size,
                    "n_groups": G, "pred_rank": wl.pred_rank, "keep_permille": wl.keep_permille,
-                   "k_critical": wl.k_critical, "virtual_devices": wl.n_dev, "loss_rate": list(wl.loss_rate),
+                   "k_critical": B.k_of(wl), "virtual_devices": wl.n_dev, "loss_rate": list(wl.loss_rate),
                    "kept_fraction": kept_fraction, "l2": "inputs larger than L2 (weights of the stack: %.2f GB)"
                    % (L * wl.layer_bytes / 1e9), "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": clocks,
@@ -475,7 +475,7 @@ def cpu_baseline(wl, budget_s=15.0):
     while spent < budget_s and done < 64 * wl.n_layers:
         Wp, w1, w2, feat, x = inputs
         t0 = time.perf_counter()
-        R.layer(Wp, w1, w2, feat, x, wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed,
+        R.layer(Wp, w1, w2, feat, x, wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0, wl.seed,
                 done // wl.n_layers, 1 + done % max(wl.n_layers - 1, 1))
         spent += time.perf_counter() - t0
         done += 1
@@ -500,7 +500,7 @@ def run_reference(args, rank, world):
     def one_step(step, n_groups_sample):
         # a bounded sample of one block: predictor, selection, and the FFN of the first n kept groups
         s = R.predict(w1, w2, feat)
-        sel = R.select(s, wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed, step, 1)
+        sel = R.select(s, wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0, wl.seed, step, 1)
         keep = sel["keep_list"][: min(sel["n_keep"], n_groups_sample)]
         P = R.group_ffn(Wp, x, keep, sel["dev_of_group"], wl.n_dev)
         R.merge(P)

@@ -122,10 +122,13 @@ halo_status halo_plan_describe(const halo_plan* plan, int M, int32_t* dev_order,
  *   halo_schedule_comp_greedy (Algorithm 1): devices in descending computing
  *     power (ties: lower index) are filled to their budget until the model
  *     fits; the last one needed takes the remainder; unused devices get 0.
- *   halo_schedule_min_max (Algorithm 2): bisection (to eps; the paper uses
- *     1e-3) on the utilisation threshold T; u_i = min(m_i, T*c_i) with the
- *     smallest T whose allocation holds the model; minimises the slowest
- *     device's time.
+ *   halo_schedule_min_max (the problem Algorithm 2 solves): u_i = min(m_i, T*c_i)
+ *     with the smallest utilisation threshold T whose allocation holds the
+ *     model; minimises the slowest device's time.  The paper bisects on T to a
+ *     tolerance (1e-3); here the piecewise-linear equation sum_i min(m_i, T*c_i)
+ *     = model_mem is solved exactly at its breakpoints m_i/c_i, so the result
+ *     is the limit of that bisection.  eps must be positive and is otherwise
+ *     not needed.
  *   Both return ratio[i] = u_i / sum(u) (sum = 1).
  *   halo_ratios_to_share_weights: integer weights round(ratio * 65536) for
  *     halo_plan_create (zero-ratio devices get empty chunks).
@@ -414,15 +417,20 @@ halo_status halo_stack_decode_host(halo_stack* stack, const float* h0_host, int 
  * l+1 overlapped with the weight stream of block l; anything else runs one launch per step of the path.
  * mode 1: always one launch per step of the path (no overlap; for comparison and checking). */
 halo_status halo_stack_set_mode(halo_stack* stack, int mode);
-/* Environment variables read by the library (measurement sweeps only; the defaults are the measured best):
- *   HALO_TUNE_CROSS_STAGES, HALO_TUNE_L2_AHEAD   persistent kernel: stages fetched across the block barrier, L2
- *                                                prefetch depth (read at halo_stack_create);
- *   HALO_TUNE_MAX_STEPS                          persistent kernel: steps per launch before a run is split;
- *   HALO_TUNE_PREFILL_TWO_LAUNCHES=1             prompt FFN as two launches (hidden, down) instead of one;
- *   HALO_TUNE_MHA_THREE_LAUNCHES=1               halo_group_mha as three launches instead of one;
- *   HALO_TUNE_I4_NO_RING=1                       halo_group_ffn_i4 on plain loads instead of the shared-memory ring;
- *   HALO_TUNE_PREFILL_KCUTS, HALO_TUNE_PREFILL_KRATIO   prompt FFN: number of K runs per down-projection tile
- *                                                and the ratio (percent) between consecutive runs. */
+/* Measurement options, process-wide.  The defaults are the measured best; the options exist so that a sweep or an
+ * ablation can be run through the same library.  value = -1 restores the default.  A stack reads the first three
+ * when it is created; the others are read at every call of the entry point they belong to.  No environment
+ * variable is read anywhere in the library.
+ *   "cross_stages" (0..8)             persistent kernel: stages of the next block fetched across the block barrier
+ *   "l2_ahead" (0..32)                persistent kernel: batches prefetched to L2 on entering a block
+ *   "max_steps_per_launch" (0 = auto) persistent kernel: steps per launch before a run is split
+ *   "prefill_two_launches" (0/1)      prompt FFN as two launches (hidden, down) instead of one
+ *   "prefill_kcuts" (1..16), "prefill_kratio_percent" (30..100)   prompt FFN: K runs per down-projection tile and
+ *                                     the ratio between consecutive runs
+ *   "mha_three_launches" (0/1)        halo_group_mha as three launches instead of one
+ *   "i4_no_ring" (0/1)                halo_group_ffn_i4 on plain loads instead of the shared-memory ring
+ * HALO_ERR_ARG for an unknown name or a value outside the stated range. */
+halo_status halo_set_option(const char* name, int value);
 /* Tracing of the persistent kernel (timing statistics of the generation loop): the caller gives a device
  * buffer trace[n_blocks][halo_stack_trace_width()][8] of 64-bit words; for the first n_blocks blocks of a
  * halo_stack_decode run every thread block records global-timer nanoseconds at: 0 block start, 1 first weight

@@ -71,6 +71,15 @@ def _check(rc: int, what: str):
         raise RuntimeError(f"oracle {what} failed with status {rc}")
 
 
+def k_of(wl) -> int:
+    """Critical groups kept by the master for a keep ratio given per mille: the smallest integer k with
+    k / G >= permille / 1000 (written on its own here; the oracle shares no code with the CUDA package)."""
+    k = 0
+    while k * 1000 < int(wl.keep_permille) * int(wl.n_groups):
+        k += 1
+    return k
+
+
 def set_threads(n: int) -> None:
     """OpenMP thread count for the group loop (the timed baseline states it)."""
     omp = ctypes.CDLL("libgomp.so.1")

@@ -32,7 +32,7 @@ EXPORTS = [
     "halo_selftest_bounded_wait", "halo_group_importance_workspace_bytes", "halo_group_importance",
     "halo_layer_workspace_bytes", "halo_layer_fused", "halo_read_status",
     "halo_pack_mha_weights", "halo_mha_kv_append", "halo_group_mha_workspace_bytes", "halo_group_mha",
-    "halo_group_lm_head", "halo_late_devices", "halo_quantize_weights_i4", "halo_group_ffn_i4",
+    "halo_group_lm_head", "halo_late_devices", "halo_quantize_weights_i4", "halo_group_ffn_i4", "halo_set_option",
 ]
 
 
@@ -134,12 +134,23 @@ def lib() -> ctypes.CDLL:
                                         c_void_p, c_int, c_void_p, c_void_p, c_void_p]
         L.halo_selftest_bounded_wait.argtypes = [c_void_p, c_longlong, c_void_p, c_void_p, c_void_p]
         L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
+        L.halo_set_option.argtypes = [c_char_p, c_int]
         _lib = L
     return _lib
 
 
 def status_string(code: int) -> str:
     return lib().halo_status_string(code).decode()
+
+
+def k_of(wl) -> int:
+    """Number of critical groups for a workload's keep ratio: ceil(permille * G / 1000) in integers.  The ABI takes
+    k itself; this is the convention the callers in this repository use to derive it."""
+    return (int(wl.keep_permille) * int(wl.n_groups) + 999) // 1000
+
+
+def halo_set_option(name: str, value: int) -> None:
+    _chk(lib().halo_set_option(name.encode(), int(value)), "halo_set_option")
 
 
 def status_message(value: int) -> str:

@@ -1,5 +1,6 @@
 // extern "C" surface of libhalo: argument checks, the host-side Assignment phase, and the stack runner.
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -28,16 +29,6 @@ halo_status check_ffn_shape(const halo_ffn_shape* s) {
     return HALO_OK;
 }
 
-halo_status check_pred_shape(const halo_pred_shape* s) {
-    if (!s) return HALO_ERR_ARG;
-    if (!valid_dtype(s->wdtype)) return HALO_ERR_DTYPE;
-    if (s->act != HALO_ACT_RELU && s->act != HALO_ACT_NONE) return HALO_ERR_ARG;
-    if (s->d_in <= 0 || s->rank <= 0 || s->n_groups <= 0) return HALO_ERR_SHAPE;
-    if (s->d_in % 8 != 0 || s->rank % 8 != 0) return HALO_ERR_SHAPE;
-    if (s->d_in > 12288 || s->rank > 8192 || s->n_groups > HALO_MAX_GROUPS) return HALO_ERR_SHAPE;
-    return HALO_OK;
-}
-
 unsigned long long loss_threshold(double rho) {
     if (!(rho > 0.0)) return 0ull;
     if (rho >= 1.0) return 1ull << 32;
@@ -49,6 +40,47 @@ unsigned long long loss_threshold(double rho) {
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace
+
+namespace halo {
+// argument rules of the predictor, shared by every entry point that takes a halo_pred_shape
+halo_status check_pred_shape(const halo_pred_shape* s) {
+    if (!s) return HALO_ERR_ARG;
+    if (!valid_dtype(s->wdtype)) return HALO_ERR_DTYPE;
+    if (s->act != HALO_ACT_RELU && s->act != HALO_ACT_NONE) return HALO_ERR_ARG;
+    if (s->d_in <= 0 || s->rank <= 0 || s->n_groups <= 0) return HALO_ERR_SHAPE;
+    if (s->d_in % 8 != 0 || s->rank % 8 != 0) return HALO_ERR_SHAPE;
+    if (s->d_in > 12288 || s->rank > 8192 || s->n_groups > HALO_MAX_GROUPS) return HALO_ERR_SHAPE;
+    return HALO_OK;
+}
+
+namespace {
+struct OptionName { const char* name; OptionId id; int lo, hi; };
+const OptionName kOptionNames[] = {
+    {"cross_stages", OPT_CROSS_STAGES, 0, 8},
+    {"l2_ahead", OPT_L2_AHEAD, 0, 32},
+    {"max_steps_per_launch", OPT_MAX_STEPS_PER_LAUNCH, 0, 1 << 30},
+    {"prefill_two_launches", OPT_PREFILL_TWO_LAUNCHES, 0, 1},
+    {"prefill_kcuts", OPT_PREFILL_KCUTS, 1, 16},
+    {"prefill_kratio_percent", OPT_PREFILL_KRATIO_PERCENT, 30, 100},
+    {"mha_three_launches", OPT_MHA_THREE_LAUNCHES, 0, 1},
+    {"i4_no_ring", OPT_I4_NO_RING, 0, 1},
+};
+std::atomic<int> g_options[OPT_COUNT] = {{-1}, {-1}, {-1}, {-1}, {-1}, {-1}, {-1}, {-1}};
+}  // namespace
+
+int option_value(OptionId id) { return g_options[id].load(std::memory_order_relaxed); }
+}  // namespace halo
+
+extern "C" halo_status halo_set_option(const char* name, int value) {
+    if (!name) return HALO_ERR_ARG;
+    for (const auto& o : kOptionNames) {
+        if (std::strcmp(name, o.name) != 0) continue;
+        if (value != -1 && (value < o.lo || value > o.hi)) return HALO_ERR_ARG;
+        g_options[o.id].store(value, std::memory_order_relaxed);
+        return HALO_OK;
+    }
+    return HALO_ERR_ARG;
+}
 
 // ---------------------------------------------------------------------------------------------------
 
@@ -190,20 +222,32 @@ extern "C" halo_status halo_schedule_min_max(int n_dev, const double* mem_budget
                                              double model_mem, double eps, double* ratio) {
     double total;
     if (!ratio || !(eps > 0.0) || !valid_devices(n_dev, mem_budget, compute, model_mem, &total)) return HALO_ERR_ARG;
-    auto held = [&](double T) {
-        double s = 0.0;
-        for (int i = 0; i < n_dev; ++i) s += std::min(mem_budget[i], T * compute[i]);
-        return s;
-    };
-    double lo = 0.0;
-    double hi = *std::max_element(mem_budget, mem_budget + n_dev) / *std::min_element(compute, compute + n_dev);
-    double best = hi;
-    while (hi - lo > eps) {
-        const double mid = 0.5 * (lo + hi);
-        if (held(mid) >= model_mem) { best = mid; hi = mid; } else lo = mid;
+    // The problem behind Algorithm 2: the smallest common finishing time T such that the devices, each loaded up
+    // to min(m_i, T * c_i), hold the model.  held(T) = sum_i min(m_i, T * c_i) is continuous, piecewise linear and
+    // non-decreasing with one breakpoint per device at T = m_i / c_i (the device is full from there on), so it is
+    // solved exactly piece by piece instead of by bisection: with the devices sorted by breakpoint, and the first k
+    // of them full, held(T) = (memory of the full ones) + T * (computing power of the rest).
+    int by_break[HALO_MAX_DEVICES];
+    for (int i = 0; i < n_dev; ++i) by_break[i] = i;
+    std::stable_sort(by_break, by_break + n_dev, [&](int a, int b) {
+        return mem_budget[a] * compute[b] < mem_budget[b] * compute[a];   // m_a / c_a < m_b / c_b, c > 0
+    });
+    double open_power = 0.0;
+    for (int i = 0; i < n_dev; ++i) open_power += compute[i];
+    double full_mem = 0.0, T = 0.0;
+    for (int k = 0; k < n_dev; ++k) {
+        const int i = by_break[k];
+        const double t_break = mem_budget[i] / compute[i];
+        T = (model_mem - full_mem) / open_power;       // where this piece reaches the model's demand
+        if (T <= t_break) break;                       // inside the piece: found
+        T = t_break;                                   // all budgets together hold the model exactly at the last one
+        full_mem += mem_budget[i];
+        open_power -= compute[i];
     }
-    const double sum = held(best);
-    for (int i = 0; i < n_dev; ++i) ratio[i] = std::min(mem_budget[i], best * compute[i]) / sum;
+    double sum = 0.0;
+    for (int i = 0; i < n_dev; ++i) sum += std::min(mem_budget[i], T * compute[i]);
+    if (!(sum > 0.0)) return HALO_ERR_ARG;
+    for (int i = 0; i < n_dev; ++i) ratio[i] = std::min(mem_budget[i], T * compute[i]) / sum;
     return HALO_OK;
 }
 
@@ -549,10 +593,9 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     s->trace_blocks = 0;
     s->cross_stages = 1;
     s->l2_ahead = 0;
-    if (const char* e = std::getenv("HALO_TUNE_CROSS_STAGES")) s->cross_stages = std::max(0, std::atoi(e));
-    s->max_steps_per_launch = 0;
-    if (const char* e = std::getenv("HALO_TUNE_MAX_STEPS")) s->max_steps_per_launch = std::max(0, std::atoi(e));
-    if (const char* e = std::getenv("HALO_TUNE_L2_AHEAD")) s->l2_ahead = std::min(32, std::max(0, std::atoi(e)));
+    if (option_value(OPT_CROSS_STAGES) >= 0) s->cross_stages = option_value(OPT_CROSS_STAGES);
+    s->max_steps_per_launch = std::max(0, option_value(OPT_MAX_STEPS_PER_LAUNCH));
+    if (option_value(OPT_L2_AHEAD) >= 0) s->l2_ahead = option_value(OPT_L2_AHEAD);
     s->persistent_ok = persistent_supported(*ffn, n_tok, G);
     {
         // pointer tables, and the first block's selection: reliable block, all scores equal -> the priority
@@ -669,6 +712,30 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
             }
             rc = launch_stack_persistent(P, st);
             if (rc == HALO_ERR_UNIMPLEMENTED && done == 0) { fell_back = true; break; }   // not resident: loop path below
+            if (rc == HALO_ERR_UNIMPLEMENTED) {
+                // a later piece of a split run was refused (the SMs are no longer all ours): the remaining steps
+                // run on the one-launch-per-step path, so the call still completes
+                halo_taps rest{};
+                if (taps) {
+                    const size_t rec = static_cast<size_t>(done) * L;
+                    rest.x = taps->x ? static_cast<char*>(taps->x) + rec * step_elems * es : nullptr;
+                    rest.scores = taps->scores ? taps->scores + rec * G : nullptr;
+                    rest.dev_of_group = taps->dev_of_group ? taps->dev_of_group + rec * G : nullptr;
+                    rest.arrived = taps->arrived ? taps->arrived + rec * n_dev : nullptr;
+                    rest.keep_list = taps->keep_list ? taps->keep_list + rec * G : nullptr;
+                    rest.n_keep = taps->n_keep ? taps->n_keep + rec : nullptr;
+                    rest.y = taps->y ? taps->y + rec * step_elems : nullptr;
+                }
+                const int saved_mode = s->mode;
+                s->mode = 1;
+                rc = halo_stack_decode(s, h0 + static_cast<size_t>(done) * step_elems, steps - done,
+                                       step0 + static_cast<uint32_t>(done), h_out + static_cast<size_t>(done) * step_elems,
+                                       taps ? &rest : nullptr, stream);
+                s->mode = saved_mode;
+                if (rc != HALO_OK) return rc;
+                s->last_launches += n_launches;
+                return HALO_OK;
+            }
             if (rc != HALO_OK) return rc;
             ++n_launches;
         }

@@ -557,7 +557,7 @@ extern "C" halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void
     const __nv_bfloat16* xt = static_cast<const __nv_bfloat16*>(x);
     int dev = 0, sms = kSmCount;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    static const bool no_ring = [] { const char* e = getenv("HALO_TUNE_I4_NO_RING"); return e && e[0] == '1'; }();
+    const bool no_ring = option_value(OPT_I4_NO_RING) == 1;
     if ((d == 2048 || d == 4096) && S % kRingNB == 0 && !no_ring) {
         // ring form: one block per SM
         constexpr int kStages = 4;

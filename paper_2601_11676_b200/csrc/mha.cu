@@ -308,6 +308,8 @@ __device__ __forceinline__ uint32_t cluster_rank() {
 __device__ __forceinline__ void cluster_barrier() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 // store a float into the same shared-memory location of another block of the cluster
 __device__ __forceinline__ void st_remote_f32(float* local_smem_ptr, uint32_t target_rank, float v) {
     uint32_t remote;
@@ -353,11 +355,17 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
     const int j0 = r * rows;
     const int chunks = d / E;
 
+    // Distributed shared memory may be written only once every block of the cluster is known to be running:
+    // arrive now, wait before the first remote store (the staging of x lies in between, and the blocks of a cluster
+    // are scheduled together, so the wait costs next to nothing).  The early returns above are taken by all blocks
+    // of a cluster or by none.
+    cluster_arrive();
     // ---- query rows j0 .. j0 + rows, two per warp and turn, sent to every block of the cluster ----
     stage_x(x, xs, d);
     for (int j = tid; j < dh; j += 256) o_acc[j] = 0.0f;
     __syncthreads();
     const float scale = rsqrtf(static_cast<float>(dh));
+    cluster_wait();                                      // every block of the cluster has started
     for (int i = 2 * warp; i < rows; i += 16) {
         const T* base = Wp + ((static_cast<size_t>(h) * 2 + 0) * dh + j0 + i) * d;
         float va, vb;
@@ -592,7 +600,7 @@ static halo_status group_mha_typed(const halo_mha_shape& sh, const void* Wp, con
     float* attn_ws = ws + static_cast<size_t>(H) * dh;
     const int n_chunks = pos / kAttnChunk + 1;
     if (cudaMemsetAsync(partials, 0, sizeof(float) * static_cast<size_t>(n_dev + 1) * d, st) != cudaSuccess) return HALO_ERR_CUDA;
-    static const bool three_launches = [] { const char* e = getenv("HALO_TUNE_MHA_THREE_LAUNCHES"); return e && e[0] == '1'; }();
+    const bool three_launches = option_value(OPT_MHA_THREE_LAUNCHES) == 1;
     if (!three_launches) {
         // one launch: a cluster of eight thread blocks per kept head
         const int iters_f = (d / E + 255) / 256;

@@ -160,12 +160,9 @@ extern "C" halo_status halo_predict_groups_static(const halo_pred_shape* shape, 
                                                   const void* feat, int n_tok, int mean_pool, float* scores,
                                                   uint32_t* dev_status, void* stream) {
     // same argument rules as halo_predict_groups
-    if (!shape) return HALO_ERR_ARG;
-    if (shape->wdtype != HALO_F32 && shape->wdtype != HALO_BF16) return HALO_ERR_DTYPE;
-    if (shape->act != HALO_ACT_RELU && shape->act != HALO_ACT_NONE) return HALO_ERR_ARG;
-    if (shape->d_in <= 0 || shape->rank <= 0 || shape->n_groups <= 0 || n_tok <= 0) return HALO_ERR_SHAPE;
-    if (shape->d_in % 8 != 0 || shape->rank % 8 != 0) return HALO_ERR_SHAPE;
-    if (shape->d_in > 12288 || shape->rank > 8192 || shape->n_groups > HALO_MAX_GROUPS) return HALO_ERR_SHAPE;
+    const halo_status rc = halo::check_pred_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (n_tok <= 0) return HALO_ERR_SHAPE;
     if (!W1 || !W2 || !feat || !scores) return HALO_ERR_ARG;
     if (!halo::aligned16(W1) || !halo::aligned16(W2) || !halo::aligned16(feat)) return HALO_ERR_ALIGN;
     // the fixed array bounds what fits: hidden values [n_tok][rank] + per-token scores [n_tok][n_groups]

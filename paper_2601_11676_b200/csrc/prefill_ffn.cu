@@ -1122,7 +1122,7 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         !make_map(&map_w_half, W, w_rows, d, d, kBK, NS / 2) ||
         !make_map(&map_h, H, T, sh.d_ffn, sh.d_ffn, kBK, kBM) || !make_map(&map_wd, W, w_rows, d, d, 64, kBK))
         return HALO_ERR_CUDA;
-    static const bool two_launches = [] { const char* e = getenv("HALO_TUNE_PREFILL_TWO_LAUNCHES"); return e && e[0] == '1'; }();
+    const bool two_launches = option_value(OPT_PREFILL_TWO_LAUNCHES) == 1;
     if (T > kBM && d % 256 == 0 && !two_launches) {
         // both contractions in one launch, one CTA per SM pulling tiles from a queue
         // the kernel leaves its control words zeroed; a workspace of unknown content is zeroed here
@@ -1133,12 +1133,12 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
         const int tiles2 = ((T + 2 * kBM - 1) / (2 * kBM)) * (d / 256);
         // K cuts of the down projection: six runs per output tile on the 7B shape, each 0.75 of the one before
         // (a model of the tile queue, then a sweep on the GPU: 0.3 ms per 32-block prompt better than six equal
-        // runs); fewer runs when there are many output tiles anyway.  HALO_TUNE_PREFILL_KCUTS and
-        // HALO_TUNE_PREFILL_KRATIO (percent) override.
+        // runs); fewer runs when there are many output tiles anyway.  The options "prefill_kcuts" and
+        // "prefill_kratio_percent" override.
         int z = std::max(1, std::min(7, (n_sm * 4 / 3) / tiles2));
         double ratio = 0.75;
-        if (const char* e = getenv("HALO_TUNE_PREFILL_KCUTS")) z = std::max(1, std::min(16, atoi(e)));
-        if (const char* e = getenv("HALO_TUNE_PREFILL_KRATIO")) ratio = std::max(0.3, std::min(1.0, atoi(e) / 100.0));
+        if (option_value(OPT_PREFILL_KCUTS) > 0) z = option_value(OPT_PREFILL_KCUTS);
+        if (option_value(OPT_PREFILL_KRATIO_PERCENT) > 0) ratio = option_value(OPT_PREFILL_KRATIO_PERCENT) / 100.0;
         KCuts cuts{};
         cuts.n = z;
         {

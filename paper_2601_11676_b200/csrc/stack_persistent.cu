@@ -281,6 +281,9 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 }
                 alive = __shfl_sync(0xffffffffu, alive ? 1 : 0, 0) != 0;
                 if (!alive) break;
+                // lane 0's acquire orders only lane 0: every lane that is about to read the published selection
+                // makes its own acquire load of the flag (it is already set, so this is one L2 read)
+                if (l > 0) (void)ld_acquire_gpu(sync_selready);
                 // (c) table of kept groups for this block: two dependent L2 reads, once per block instead of per batch
                 int nk = __ldcg(&sb->n_keep);
                 nk = max(0, min(nk, G));

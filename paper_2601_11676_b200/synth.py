@@ -43,11 +43,6 @@ class Workload:
         return len(self.loss_rate)
 
     @property
-    def k_critical(self) -> int:
-        # number of critical groups = ceil(permille * G / 1000), in integers
-        return (self.keep_permille * self.n_groups + 999) // 1000
-
-    @property
     def torch_dtype(self) -> torch.dtype:
         return torch.float32 if self.dtype == "f32" else torch.bfloat16
 

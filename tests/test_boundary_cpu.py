@@ -107,7 +107,28 @@ def test_schedulers_match_oracle_and_feed_the_plan(lib):
         c = rng.uniform(0.6, 1.8, n).round(1)
         Mt = float(rng.uniform(0.2, 1.0) * m.sum())
         assert np.allclose(B.halo_schedule_comp_greedy(m, c, Mt), R.comp_greedy(m, c, Mt), atol=1e-12)
-        assert np.allclose(B.halo_schedule_min_max(m, c, Mt, 1e-3), R.min_max(m, c, Mt, 1e-3), atol=1e-12)
+        # the library solves the min-max problem exactly, the oracle bisects as Algorithm 2 does: two different
+        # routes, which must meet as the oracle's tolerance shrinks
+        r_lib = np.array(B.halo_schedule_min_max(m, c, Mt, 1e-3))
+        assert np.allclose(r_lib, R.min_max(m, c, Mt, 1e-10), atol=1e-7)
+        assert np.abs(r_lib - R.min_max(m, c, Mt, 1e-3)).max() <= 2e-3
+        # invariants of the problem itself: ratios sum to 1, the loads r * Mt fit every budget (the allocation holds
+        # the model exactly), and no choice of "full" devices gives a smaller slowest-device time
+        assert abs(r_lib.sum() - 1.0) <= 1e-12
+        load = r_lib * Mt
+        assert (load <= m * (1 + 1e-9)).all()
+        best = np.inf
+        for mask in range(1 << n):                       # brute force: which devices are filled to their budget
+            full = np.array([(mask >> i) & 1 for i in range(n)], dtype=bool)
+            if full.all():
+                T = (m / c).max() if abs(m.sum() - Mt) <= 1e-9 * Mt else np.inf
+            else:
+                T = (Mt - m[full].sum()) / c[~full].sum()
+            if T < 0 or not np.isfinite(T):
+                continue
+            if (T * c[~full] <= m[~full] * (1 + 1e-12)).all() and (m[full] <= T * c[full] * (1 + 1e-12)).all():
+                best = min(best, T)
+        assert np.isclose((load / c).max(), best, rtol=1e-9)
     # ratios -> integer share weights -> Algorithm 3: a device with ratio 0 gets an empty chunk
     r = B.halo_schedule_comp_greedy([4, 5, 3], [2.0, 1.0, 3.0], 6.0)
     w = B.halo_ratios_to_share_weights(r)

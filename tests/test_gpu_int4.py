@@ -93,3 +93,28 @@ def test_int4_full_size_7b_block_sampled_groups():
     ref = R.group_ffn_i4(Q_ref, Sc_ref, hb(x), [0, 1, 2], np.array([-1, 0, 2], dtype=np.int32), wl.n_dev)
     rms = np.sqrt(np.mean(R.merge(ref) ** 2))
     assert np.abs(P - ref).max() <= U.TOL_BF16 * rms
+
+
+def test_int4_full_size_7b_block_all_groups_kept_every_element():
+    """The case the benchmark times: one 7B-shaped block on int4 weights with all 86 groups kept (the shared-memory
+    ring kernel with a full kept set).  Codes and scales of the whole block bit for bit, every output element of
+    every holder slot against the oracle."""
+    wl = synth.workload("llama2-7b-decode")
+    Wp = synth.packed_layer(wl, 3, DEV)
+    sh, Q, Sc = _quantize(wl, Wp)
+    hb = synth.host_bits
+    Q_ref, Sc_ref = R.quantize_i4(hb(Wp))
+    assert (Q.cpu().numpy() == Q_ref).all() and (hb(Sc) == Sc_ref).all()
+    x = synth.activation(wl, 6, DEV)
+    G = wl.n_groups
+    dev = (np.arange(G, dtype=np.int32) % (wl.n_dev + 1)) - 1
+    keep = list(range(G))
+    P, status = _run(sh, Q, Sc, x, keep, dev, wl.n_dev, G)
+    assert status == 0
+    ref = R.group_ffn_i4(Q_ref, Sc_ref, hb(x), keep, dev, wl.n_dev)
+    rms = np.sqrt(np.mean(R.merge(ref) ** 2))
+    assert np.abs(P - ref).max() <= U.TOL_BF16 * rms
+    # and against the bf16 block it was quantised from: the quantisation error itself stays small
+    P16 = R.group_ffn(hb(Wp), hb(x), keep, dev, wl.n_dev)
+    diff = R.merge(ref) - R.merge(P16)
+    assert np.sqrt(np.mean(diff ** 2)) <= 0.5 * np.sqrt(np.mean(R.merge(P16) ** 2))

@@ -48,15 +48,18 @@ def test_group_mha_and_kv_append_match_oracle(dtype, d, H, dh, L, positions):
     for pos in positions:
         x = synth.activation(wl, 50 + pos, DEV)
         # keys / values of this token: within one rounding step of the oracle's
+        K_before, V_before = K.clone(), V.clone()
         B.halo_mha_kv_append(sh, Wk, Wv, x, pos, K, V)
         torch.cuda.synchronize()
         Kh, Vh = hb(K), hb(V)
         Kr, Vr = Kh.copy(), Vh.copy()
-        if d <= 512:                                              # the oracle's dense projection is slow at 4096
-            R.mha_kv_append(hb(Wk), hb(Wv), hb(x)[0], pos, Kr, Vr)
-            kk = R.to_f64(Kr[:, pos])
-            assert np.abs(R.to_f64(Kh[:, pos]) - kk).max() <= (1e-5 if dtype == "f32" else 2 ** -7) * np.abs(kk).max()
-            assert np.abs(R.to_f64(Vh[:, pos]) - R.to_f64(Vr[:, pos])).max() <= (1e-5 if dtype == "f32" else 2 ** -7) * np.abs(kk).max()
+        R.mha_kv_append(hb(Wk), hb(Wv), hb(x)[0], pos, Kr, Vr)
+        kk = R.to_f64(Kr[:, pos])
+        assert np.abs(R.to_f64(Kh[:, pos]) - kk).max() <= (1e-5 if dtype == "f32" else 2 ** -7) * np.abs(kk).max()
+        assert np.abs(R.to_f64(Vh[:, pos]) - R.to_f64(Vr[:, pos])).max() <= (1e-5 if dtype == "f32" else 2 ** -7) * np.abs(kk).max()
+        # and the rest of the cache is untouched
+        other = [p for p in (0, L // 2, L - 1) if p != pos]
+        assert (Kh[:, other] == hb(K_before)[:, other]).all() and (Vh[:, other] == hb(V_before)[:, other]).all()
         # attention of the kept heads, from the GPU's own cache bytes
         for keep in (list(range(H)), [h for h in range(H) if h % 3 != 1], [H - 1], []):
             kl = torch.full((H,), -1, dtype=torch.int32, device=DEV)

@@ -44,13 +44,13 @@ def test_select_bit_exact(G, n_dev, mode):
 
 def test_select_arrival_stream_matches_oracle_over_many_steps():
     wl = synth.workload("tiny")
-    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, B.SEL_TOPK, wl.k_critical, 0.0, wl.seed)
+    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
     s = torch.randn(wl.n_groups, generator=torch.Generator().manual_seed(1))
     sd = s.to(DEV)
     lost = 0
     for step in range(0, 1000, 7):
         gpu, _ = U.gpu_select(plan, sd, step=step, layer=3)
-        ref = R.select(s.numpy(), wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed, step, 3)
+        ref = R.select(s.numpy(), wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0, wl.seed, step, 3)
         U.assert_select_equal(gpu, ref)
         lost += int(gpu["n_keep"] < wl.n_groups)
     assert 0 < lost < 143  # both outcomes occur
@@ -125,7 +125,7 @@ def test_group_ffn_full_layer_shapes_with_slots(name):
     G = wl.n_groups
     scores = np.random.default_rng(3).normal(size=G).astype(np.float32)
     for step in (0, 5):
-        sel = R.select(scores, wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed, step, 2)
+        sel = R.select(scores, wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0, wl.seed, step, 2)
         keep = sel["keep_list"][: sel["n_keep"]]
         P, ref, status = _ffn_case(wl, 1, keep, sel["dev_of_group"])
         assert status == 0
@@ -191,7 +191,7 @@ def test_tiny_layer_end_to_end_masks_over_steps():
     wl = synth.workload("tiny")
     Wp, W1, W2 = U.layer_tensors(wl, 0)
     x = synth.activation(wl, 0, DEV)
-    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, B.SEL_TOPK, wl.k_critical, 0.0, wl.seed)
+    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
     scores, status = U.gpu_predict(B.F32, W1, W2, x)
     hb = synth.host_bits
     s_ref = R.predict(hb(W1), hb(W2), hb(x))
@@ -200,12 +200,12 @@ def test_tiny_layer_end_to_end_masks_over_steps():
     for step in range(0, 40):
         gpu, dev_bufs = U.gpu_select(plan, scores, step, 1)
         # gate 1: same fp32 scores -> identical integers
-        ref_same = R.select(scores.cpu().numpy(), wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0,
+        ref_same = R.select(scores.cpu().numpy(), wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0,
                             wl.seed, step, 1)
         U.assert_select_equal(gpu, ref_same)
         # gate 3: the oracle's own scores give the same selection in fp32
         full = R.layer(hb(Wp), hb(W1), hb(W2), hb(x), hb(x), wl.loss_rate, wl.share_weight, R.SEL_TOPK,
-                       wl.k_critical, 0.0, wl.seed, step, 1)
+                       R.k_of(wl), 0.0, wl.seed, step, 1)
         assert (full["keep_list"] == gpu["keep_list"]).all()
         keep = gpu["keep_list"][: gpu["n_keep"]]
         P, st = U.gpu_group_ffn(wl, Wp, x, keep, gpu["dev_of_group"], wl.n_dev)
@@ -213,7 +213,7 @@ def test_tiny_layer_end_to_end_masks_over_steps():
         assert st == 0 and U.rel_err(y, full["y"]) <= U.TOL_F32
         outcomes.add(gpu["n_keep"])
     # the lossy device both arrives and is lost; when lost, exactly its chunk of the less-critical groups goes
-    order, _, bnd = R.plan(wl.loss_rate, wl.share_weight, wl.n_groups - wl.k_critical)
+    order, _, bnd = R.plan(wl.loss_rate, wl.share_weight, wl.n_groups - R.k_of(wl))
     j = list(order).index(1)
     assert outcomes == {wl.n_groups - int(bnd[j + 1] - bnd[j]), wl.n_groups}
 
@@ -282,7 +282,7 @@ def test_layer_fused_matches_oracle_layer(name, n_tok):
     feat = synth.activation(wl, 30, DEV, n_tok=n_tok)
     x = synth.activation(wl, 31, DEV, n_tok=n_tok)
     G, n, d = wl.n_groups, wl.n_dev, wl.d_model
-    plan = B.Plan(G, wl.loss_rate, wl.share_weight, B.SEL_TOPK, wl.k_critical, 0.0, wl.seed)
+    plan = B.Plan(G, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
     ffn = B.ffn_shape(d, wl.d_ffn, wl.group_size, code)
     pred = B.pred_shape(d, wl.pred_rank, G, code)
     scores = torch.zeros(G, dtype=torch.float32, device=DEV)
@@ -301,7 +301,7 @@ def test_layer_fused_matches_oracle_layer(name, n_tok):
         assert B.halo_read_status(int(status.item())) == "clean"
         s_ref = R.predict(hb(W1), hb(W2), hb(feat), mean_pool=n_tok > 1)
         assert U.rel_err(scores.cpu().numpy(), s_ref.astype(np.float64)) <= U.tol_for(wl)
-        sel = R.select(scores.cpu().numpy(), wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed,
+        sel = R.select(scores.cpu().numpy(), wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0, wl.seed,
                        step, 5)
         assert (dg.cpu().numpy() == sel["dev_of_group"]).all() and (keep.cpu().numpy() == sel["keep"]).all()
         assert (arr.cpu().numpy()[:n] == sel["arrived"]).all()

@@ -123,7 +123,7 @@ def test_prefill_full_size_block_sampled_tokens(name, n_tok):
     Wp = synth.packed_layer(wl, 1, DEV)
     x = synth.activation(wl, 3, DEV, n_tok=wl.n_tok)
     scores = np.random.default_rng(5).normal(size=G).astype(np.float32)
-    sel = R.select(scores, wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed, 0, 1)
+    sel = R.select(scores, wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0, wl.seed, 0, 1)
     keep = sel["keep_list"][: sel["n_keep"]]
     P, status = U.gpu_group_ffn(wl, Wp, x, keep, sel["dev_of_group"], wl.n_dev)
     assert status == 0

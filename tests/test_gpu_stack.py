@@ -16,7 +16,7 @@ def build_stack(wl, mode=B.SEL_TOPK, threshold=0.0, act=B.ACT_RELU):
     code = U.dtype_code(wl)
     Wp = [synth.packed_layer(wl, l, DEV) for l in range(wl.n_layers)]
     preds = [synth.predictor(wl, l, DEV) for l in range(wl.n_layers)]
-    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, mode, wl.k_critical, threshold, wl.seed)
+    plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, mode, B.k_of(wl), threshold, wl.seed)
     stack = B.Stack(B.ffn_shape(wl.d_model, wl.d_ffn, wl.group_size, code),
                     B.pred_shape(wl.d_model, wl.pred_rank, wl.n_groups, code, act), wl.n_tok, plan, Wp,
                     [p[0] for p in preds], [p[1] for p in preds])
@@ -42,7 +42,9 @@ def run_with_taps(wl, stack, steps, step0=0):
 
 
 def check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=0, mode=R.SEL_TOPK, threshold=0.0,
-                         act=R.ACT_RELU):
+                         act=R.ACT_RELU, tokens=None):
+    """`tokens`: token rows whose FFN output the oracle recomputes (all when None); scores, selection integers and
+    the glue chain are always checked in full."""
     hb = synth.host_bits
     tol = U.tol_for(wl)
     L, n = wl.n_layers, wl.n_dev
@@ -61,7 +63,7 @@ def check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=0, mode=R.SEL
             else:
                 s_ref = R.predict(hb(preds[l][0]), hb(preds[l][1]), x_all[s, l - 1], act=act, mean_pool=wl.n_tok > 1)
                 assert U.rel_err(scores, s_ref.astype(np.float64)) <= tol
-            sel = R.select(scores, wl.loss_rate, wl.share_weight, mode, wl.k_critical, threshold, wl.seed,
+            sel = R.select(scores, wl.loss_rate, wl.share_weight, mode, R.k_of(wl), threshold, wl.seed,
                            step0 + s, l, force_all=(l == 0))
             nk = int(t["n_keep"][s, l].item())
             assert nk == sel["n_keep"]
@@ -70,10 +72,11 @@ def check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=0, mode=R.SEL
             if n:
                 assert (t["arrived"][s, l, :n].cpu().numpy() == sel["arrived"]).all()
             lost_layers += int(nk < wl.n_groups)
-            P = R.group_ffn(hb(Wp[l]), x_l, sel["keep_list"][:nk], sel["dev_of_group"], n)
-            y_ref = R.merge(P)
             y = t["y"][s, l].cpu().numpy()
-            assert U.rel_err(y, y_ref) <= tol, (s, l)
+            x_ffn = x_l if tokens is None else x_l[tokens]
+            P = R.group_ffn(hb(Wp[l]), x_ffn, sel["keep_list"][:nk], sel["dev_of_group"], n)
+            y_ref = R.merge(P)
+            assert U.rel_err(y if tokens is None else y[tokens], y_ref) <= tol, (s, l)
             # glue, from the GPU's own y: next input and residual stream
             h, x_next = R.glue(h, y.astype(np.float64), U.dtype_code(wl))
             if l + 1 < L:
@@ -164,16 +167,37 @@ def test_stack_prompt_on_the_tensor_core_path(n_tok, d):
     assert (plain - h_out).abs().max().item() <= 1e-4 * h_out.abs().max().item()
 
 
-@pytest.mark.parametrize("name,steps,sample", [
-    ("llama2-7b-decode", 3, [(0, 0), (0, 1), (1, 16), (2, 30), (2, 31)]),
-    ("llama2-13b-decode", 2, [(0, 1), (1, 20), (1, 39)]),
-    ("tinyllama-1.1b-decode", 4, [(0, 0), (1, 1), (2, 11), (3, 21)]),
+def test_prompt_stack_at_the_benchmarked_shape():
+    """The prompt path as bench.py times it: 512 tokens, d 4096, groups of 128, lossy devices, the one-launch
+    tensor-core FFN (128-neuron hidden tiles, three stages).  Teacher-forced against the oracle through the taps on
+    a sample of token rows (every block, both prompts); then the tap-free run, in which the down projection adds
+    straight into the residual stream and the predictor runs on the side stream, must give the same stream."""
+    wl = synth.workload("llama2-7b-prefill", n_layers=3, steps=2, loss_rate=(0.0, 0.3, 0.5, 0.7))
+    stack, Wp, preds = build_stack(wl)
+    h0, h_out, t = run_with_taps(wl, stack, wl.steps, step0=5)
+    tokens = [0, 127, 128, 255, 256, 300, 511]
+    lost = check_teacher_forced(wl, Wp, preds, h0, h_out, t, wl.steps, step0=5, tokens=tokens)
+    assert lost > 0                                   # some block really ran with groups dropped
+    plain = torch.empty_like(h_out)
+    stack.decode(h0, wl.steps, 5, plain)
+    torch.cuda.synchronize()
+    assert stack.status() == 0
+    assert (plain - h_out).abs().max().item() <= 1e-4 * h_out.abs().max().item()
+
+
+@pytest.mark.parametrize("name,steps,sample,permille", [
+    ("llama2-7b-decode", 3, [(0, 0), (0, 1), (1, 16), (2, 30), (2, 31)], 500),
+    ("llama2-7b-decode", 2, [(0, 1), (1, 17), (1, 31)], 300),
+    ("llama2-7b-decode", 2, [(0, 1), (1, 9)], 700),
+    ("llama2-7b-decode", 2, [(0, 2), (1, 31)], 1000),
+    ("llama2-13b-decode", 2, [(0, 1), (1, 20), (1, 39)], 500),
+    ("tinyllama-1.1b-decode", 4, [(0, 0), (1, 1), (2, 11), (3, 21)], 500),
 ])
-def test_full_size_stack_in_bench_configuration_sampled_blocks(name, steps, sample):
-    """The whole stack at its stated size, run the way bench.py times it (one persistent launch); the oracle
-    recomputes a sample of (step, block) records from the recorded inputs.  Selection integers are checked for
-    every record (they are cheap), FFN outputs for the sample."""
-    wl = synth.workload(name)
+def test_full_size_stack_in_bench_configuration_sampled_blocks(name, steps, sample, permille):
+    """The whole stack at its stated size, run the way bench.py times it (one persistent launch), at every keep
+    ratio of the 7B sweep; the oracle recomputes a sample of (step, block) records from the recorded inputs.
+    Selection integers are checked for every record (they are cheap), FFN outputs for the sample."""
+    wl = synth.workload(name, keep_permille=permille)
     stack, Wp, preds = build_stack(wl)
     h0, h_out, t = run_with_taps(wl, stack, steps, step0=7)
     assert stack.last_launches() == 1
@@ -185,7 +209,7 @@ def test_full_size_stack_in_bench_configuration_sampled_blocks(name, steps, samp
     arr_all = t["arrived"].cpu().numpy()
     for s in range(steps):
         for l in range(wl.n_layers):
-            sel = R.select(scores_all[s, l], wl.loss_rate, wl.share_weight, R.SEL_TOPK, wl.k_critical, 0.0, wl.seed,
+            sel = R.select(scores_all[s, l], wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0, wl.seed,
                            7 + s, l, force_all=(l == 0))
             assert int(nk_all[s, l]) == sel["n_keep"], (s, l)
             assert (kl_all[s, l] == sel["keep_list"]).all() and (dg_all[s, l] == sel["dev_of_group"]).all()
@@ -240,13 +264,15 @@ def test_stack_persistent_variants(variant):
         assert nk.min() < wl.n_groups and len(np.unique(nk)) > 1   # the critical count really varies with the scores
 
 
-def test_long_runs_are_split_into_several_persistent_launches(monkeypatch):
+def test_long_runs_are_split_into_several_persistent_launches():
     """The persistent kernel's counters are 32 bit, so very long runs are cut into several launches; forced here
     with a tiny limit: the arrival draws and records must continue seamlessly across the cut."""
-    monkeypatch.setenv("HALO_TUNE_MAX_STEPS", "2")
     wl = synth.Workload("c", 3, 2048, 64 * 10, 64, 128, "bf16", (0.0, 0.4, 0.8), (1, 1, 1), 300, 5)
-    stack, Wp, preds = build_stack(wl)
-    monkeypatch.delenv("HALO_TUNE_MAX_STEPS")
+    B.halo_set_option("max_steps_per_launch", 2)
+    try:
+        stack, Wp, preds = build_stack(wl)
+    finally:
+        B.halo_set_option("max_steps_per_launch", -1)
     h0, h_out, t = run_with_taps(wl, stack, wl.steps, step0=11)
     assert stack.last_launches() == 3
     check_teacher_forced(wl, Wp, preds, h0, h_out, t, wl.steps, step0=11)

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "prompt_stack.cuh"
 #include "stack_persistent.cuh"
 
 using namespace halo;
@@ -64,8 +65,10 @@ const OptionName kOptionNames[] = {
     {"prefill_kratio_percent", OPT_PREFILL_KRATIO_PERCENT, 30, 100},
     {"mha_three_launches", OPT_MHA_THREE_LAUNCHES, 0, 1},
     {"i4_no_ring", OPT_I4_NO_RING, 0, 1},
+    {"prompt_kcuts", OPT_PROMPT_KCUTS, 1, 16},
+    {"prompt_l2_ahead", OPT_PROMPT_L2_AHEAD, 0, 32},
 };
-std::atomic<int> g_options[OPT_COUNT] = {{-1}, {-1}, {-1}, {-1}, {-1}, {-1}, {-1}, {-1}};
+std::atomic<int> g_options[OPT_COUNT] = {{-1}, {-1}, {-1}, {-1}, {-1}, {-1}, {-1}, {-1}, {-1}, {-1}};
 }  // namespace
 
 int option_value(OptionId id) { return g_options[id].load(std::memory_order_relaxed); }
@@ -484,6 +487,17 @@ struct halo_stack {
     int trace_blocks;
     int cross_stages, l2_ahead;    // tuning of the persistent kernel
     int max_steps_per_launch;      // 0 = derived from the counters' range
+    // multi-token stacks, persistent prompt kernel (one launch per prompt)
+    bool prompt_ok = false;
+    void* pp_slab = nullptr;
+    CUtensorMap* pp_maps = nullptr;        // device
+    __nv_bfloat16* pp_H[2] = {nullptr, nullptr};
+    float* pp_zpart = nullptr;
+    halo::PersistSel* pp_sel = nullptr;    // [L]
+    unsigned* pp_ctl = nullptr;
+    size_t pp_ctl_bytes = 0;
+    int pp_tiles_x = 0, pp_n_pn = 0, pp_z_cuts = 0;
+    unsigned long long* pp_trace = nullptr;   // caller-owned, optional
 };
 
 extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred,
@@ -619,6 +633,60 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
         ok = ok && cudaMemcpy(s->d_W1, s->W1.data(), sizeof(void*) * n_layers, cudaMemcpyHostToDevice) == cudaSuccess;
         ok = ok && cudaMemcpy(s->d_W2, s->W2.data(), sizeof(void*) * n_layers, cudaMemcpyHostToDevice) == cudaSuccess;
         if (!ok) { cudaFree(s->slab); delete s; return HALO_ERR_CUDA; }
+        if (n_tok > 1 && prompt_stack_supported(*ffn, *pred, n_layers, n_tok)) {
+            // persistent prompt kernel: tensor maps (encoded once, here), two H buffers, control words, one selection
+            // record per block.  Any failure in here only means that prompts run one launch per step of the path.
+            const int S = ffn->group_size, NS = std::min(S, 128), dm = ffn->d_model;
+            const int tiles_x = (n_tok + 255) / 256, n_pn = (pred->rank + 255) / 256;
+            const size_t n_maps = 3 * static_cast<size_t>(n_layers) + 4;
+            const size_t h_bytes = align_up(static_cast<size_t>(n_tok) * ffn->d_ffn * 2, 1024);
+            const size_t z_bytes = align_up(sizeof(float) * 2 * tiles_x * 8 * static_cast<size_t>(n_pn) * 256, 256);
+            const size_t sel_bytes = align_up(sizeof(PersistSel) * n_layers, 256);
+            s->pp_ctl_bytes = align_up(prompt_stack_ctl_bytes(n_layers, tiles_x, G), 256);
+            const size_t map_bytes = align_up(sizeof(CUtensorMap) * n_maps, 256);
+            const size_t total = map_bytes + 2 * h_bytes + z_bytes + sel_bytes + s->pp_ctl_bytes;
+            if (cudaMalloc(&s->pp_slab, total) == cudaSuccess) {
+                char* pb = static_cast<char*>(s->pp_slab);
+                s->pp_maps = reinterpret_cast<CUtensorMap*>(pb); pb += map_bytes;
+                s->pp_H[0] = reinterpret_cast<__nv_bfloat16*>(pb); pb += h_bytes;
+                s->pp_H[1] = reinterpret_cast<__nv_bfloat16*>(pb); pb += h_bytes;
+                s->pp_zpart = reinterpret_cast<float*>(pb); pb += z_bytes;
+                s->pp_sel = reinterpret_cast<PersistSel*>(pb); pb += sel_bytes;
+                s->pp_ctl = reinterpret_cast<unsigned*>(pb);
+                std::vector<CUtensorMap> maps(n_maps);
+                const uint64_t w_rows = static_cast<uint64_t>(G) * 3 * S;
+                bool good = cudaMemset(s->pp_slab, 0, total) == cudaSuccess;
+                for (int l = 0; l < n_layers && good; ++l) {
+                    good = make_bf16_map(&maps[3 * l + 0], s->W[l], w_rows, dm, dm, 64, NS) &&
+                           make_bf16_map(&maps[3 * l + 1], s->W[l], w_rows, dm, dm, 64, 64);
+                    // block 0 has no predictor: its slot repeats the weight map and is never used
+                    good = good && (l == 0 ? make_bf16_map(&maps[3 * l + 2], s->W[l], w_rows, dm, dm, 64, 128)
+                                           : make_bf16_map(&maps[3 * l + 2], s->W1[l], pred->rank, dm, dm, 64, 128));
+                }
+                for (int b = 0; b < 2 && good; ++b)
+                    good = make_bf16_map(&maps[3 * n_layers + b], s->x[b], n_tok, dm, dm, 64, 128) &&
+                           make_bf16_map(&maps[3 * n_layers + 2 + b], s->pp_H[b], n_tok, ffn->d_ffn, ffn->d_ffn, 64, 128);
+                good = good && cudaMemcpy(s->pp_maps, maps.data(), sizeof(CUtensorMap) * n_maps, cudaMemcpyHostToDevice) == cudaSuccess;
+                good = good && cudaMemcpy(s->pp_sel, sel0.data(), sizeof(PersistSel), cudaMemcpyHostToDevice) == cudaSuccess;
+                if (good) {
+                    int dev = 0, n_sm = kSmCount;
+                    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+                    s->pp_tiles_x = tiles_x;
+                    s->pp_n_pn = n_pn;
+                    // K runs per output tile of the down projection: short enough that the tiles a block ends with
+                    // do not hold up the next block's first items for long
+                    s->pp_z_cuts = std::max(1, std::min(8, (n_sm * 4 / 3) / std::max(1, tiles_x * (dm / 256))));
+                    if (option_value(OPT_PROMPT_KCUTS) > 0) s->pp_z_cuts = option_value(OPT_PROMPT_KCUTS);
+                    s->prompt_ok = true;
+                } else {
+                    cudaFree(s->pp_slab);
+                    s->pp_slab = nullptr;
+                    (void)cudaGetLastError();
+                }
+            } else {
+                (void)cudaGetLastError();
+            }
+        }
     }
     *out = s;
     return HALO_OK;
@@ -633,6 +701,7 @@ extern "C" halo_status halo_stack_destroy(halo_stack* s) {
         cudaStreamDestroy(s->side);
     }
     cudaFree(s->slab);
+    if (s->pp_slab) cudaFree(s->pp_slab);
     delete s;
     return HALO_OK;
 }
@@ -748,8 +817,69 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
 #define HALO_COPY(dst, src, bytes)                                                                    \
     do { if (cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToDevice, st) != cudaSuccess)     \
              return HALO_ERR_CUDA; } while (0)
+    if (T > 1 && s->prompt_ok && s->mode == 0 && (!taps || !taps->y)) {
+        // Prompt path, one launch per prompt: every block of the stack inside one persistent kernel.  The residual
+        // stream is updated in place in the caller's h_out.
+        PromptParams P;
+        std::memset(&P, 0, sizeof(P));
+        P.L = L; P.T = static_cast<int>(T); P.d = static_cast<int>(d); P.S = s->ffn.group_size; P.G = G; P.r = s->pred.rank;
+        P.act = s->pred.act;
+        P.tiles_x = s->pp_tiles_x; P.n_tn = static_cast<int>(d) / 256; P.n_pn = s->pp_n_pn; P.z_cuts = s->pp_z_cuts;
+        P.subs = s->ffn.group_size / std::min(s->ffn.group_size, 128);
+        P.ctl_stride = prompt_stack_ctl_stride(P.tiles_x, G);
+        P.r_pad = P.n_pn * 256;
+        P.l2_ahead = std::max(0, option_value(OPT_PROMPT_L2_AHEAD));
+        P.maps = s->pp_maps;
+        P.W2 = reinterpret_cast<const __nv_bfloat16* const*>(s->d_W2);
+        P.x[0] = static_cast<__nv_bfloat16*>(s->x[0]); P.x[1] = static_cast<__nv_bfloat16*>(s->x[1]);
+        P.H[0] = s->pp_H[0]; P.H[1] = s->pp_H[1];
+        P.h_cols = s->ffn.d_ffn;
+        P.zpart = s->pp_zpart; P.sel = s->pp_sel; P.ctl = s->pp_ctl; P.status = s->status;
+        P.plan = s->plan.dev;
+        P.trace = s->pp_trace;
+        {   // what is left of the caller's buffer behind the per-block words holds the tile records
+            int width = halo_stack_trace_width(s);
+            const long long words = static_cast<long long>(s->trace_blocks) * width * 8 - static_cast<long long>(width) * 16;
+            P.trace_items = (s->pp_trace && words > 0) ? static_cast<int>(words / (3ll * width)) : 0;
+        }
+        for (int sidx = 0; sidx < steps; ++sidx) {
+            float* h_run = h_out + sidx * step_elems;
+            if (h_run != h0 + sidx * step_elems &&
+                cudaMemcpyAsync(h_run, h0 + sidx * step_elems, sizeof(float) * step_elems, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                return HALO_ERR_CUDA;
+            if (cudaMemsetAsync(s->pp_ctl, 0, s->pp_ctl_bytes, st) != cudaSuccess) return HALO_ERR_CUDA;
+            P.h = h_run;
+            P.step = step0 + static_cast<uint32_t>(sidx);
+            if (taps) {
+                const size_t rec = static_cast<size_t>(sidx) * L;
+                P.tap_x = taps->x ? static_cast<__nv_bfloat16*>(taps->x) + rec * step_elems : nullptr;
+                P.tap_scores = taps->scores ? taps->scores + rec * G : nullptr;
+                P.tap_dev_of_group = taps->dev_of_group ? taps->dev_of_group + rec * G : nullptr;
+                P.tap_arrived = taps->arrived ? taps->arrived + rec * n_dev : nullptr;
+                P.tap_keep_list = taps->keep_list ? taps->keep_list + rec * G : nullptr;
+                P.tap_n_keep = taps->n_keep ? taps->n_keep + rec : nullptr;
+                // records of the first block: its selection is fixed (everything kept, scores zero)
+                const PersistSel* s0 = s->pp_sel;
+                auto copy = [&](void* dst, const void* src, size_t bytes) {
+                    return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+                };
+                bool ok = true;
+                if (taps->scores) ok = ok && cudaMemsetAsync(P.tap_scores, 0, sizeof(float) * G, st) == cudaSuccess;
+                if (taps->dev_of_group) ok = ok && copy(P.tap_dev_of_group, s0->dev_of_group, sizeof(int32_t) * G);
+                if (taps->arrived && n_dev > 0) ok = ok && copy(P.tap_arrived, s0->arrived, n_dev);
+                if (taps->keep_list) ok = ok && copy(P.tap_keep_list, s0->keep_list, sizeof(int32_t) * G);
+                if (taps->n_keep) ok = ok && copy(P.tap_n_keep, &s0->n_keep, sizeof(int32_t));
+                if (!ok) return HALO_ERR_CUDA;
+            }
+            rc = launch_prompt_stack(P, st);
+            if (rc != HALO_OK) return rc;
+            ++launches;
+        }
+        s->last_launches = launches;
+        return HALO_OK;
+    }
     if (T > 1 && s->side) {
-        // Prompt path.  The scores of block l+1 need only x_l (one layer ahead, Sec. III-B.2), which exists before
+        // Prompt path, one launch per step of the path.  The scores of block l+1 need only x_l (one layer ahead, Sec. III-B.2), which exists before
         // block l's FFN starts: predictor + selection of block l+1 go to the side stream and overlap with the
         // tensor-core GEMMs of block l (the paper's Pred || Comp overlap).  Two selection sets alternate by block.
         cudaStream_t side = s->side;
@@ -915,6 +1045,7 @@ extern "C" halo_status halo_stack_set_trace(halo_stack* s, unsigned long long* t
     if (!s || n_blocks < 0 || (n_blocks > 0 && !trace)) return HALO_ERR_ARG;
     s->trace = n_blocks > 0 ? trace : nullptr;
     s->trace_blocks = n_blocks;
+    s->pp_trace = (n_blocks > 0 && s->n_tok > 1) ? trace : nullptr;
     return HALO_OK;
 }
 

@@ -16,6 +16,7 @@
 
 #include "common.cuh"
 #include "ffn_math.cuh"
+#include "prompt_stack.cuh"
 #include "umma.cuh"
 
 namespace halo {
@@ -1076,6 +1077,11 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, 
 }
 
 }  // namespace
+
+bool make_bf16_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t row_stride_elems,
+                   uint32_t box_cols, uint32_t box_rows) {
+    return make_map(map, base, rows, cols, row_stride_elems, box_cols, box_rows);
+}
 
 bool prefill_supported(const halo_ffn_shape& sh, int n_tok) {
     return sh.wdtype == HALO_BF16 && n_tok >= 16 && (sh.group_size == 64 || sh.group_size == 128 || sh.group_size == 256) &&

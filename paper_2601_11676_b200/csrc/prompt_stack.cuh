@@ -19,6 +19,7 @@ struct PromptParams {
     int subs;          // hidden tiles per group (S / NS)
     int ctl_stride;    // control words per block
     int r_pad;         // n_pn * 256
+    int l2_ahead;      // K steps whose weight tiles are prefetched to L2 ahead of their load (0 = none)
     uint32_t step;     // arrival-draw counter of this prompt
     const CUtensorMap* maps;
     const __nv_bfloat16* const* W2;   // device table [L]
@@ -37,9 +38,14 @@ struct PromptParams {
     uint8_t* tap_arrived;
     int32_t* tap_keep_list;
     int32_t* tap_n_keep;
-    // optional: [gridDim.x][8] nanoseconds per thread block: 0 normalise items (with their waits), 1 hidden tiles,
-    // 2 predictor tiles and selection, 3 down tiles, 4 waiting for the next item, 5 items taken, 6 first, 7 last stamp
+    // optional: [gridDim.x][16] words per thread block.  Nanoseconds seen by the first epilogue warp: 1 hidden tiles,
+    // 2 predictor tiles and selection, 3 down tiles, 4 waiting for the next tile, 7 first to last time stamp.  SM
+    // cycles: 5 loader waiting for hidden tiles of other CTAs, 6 for the block's selection, 8 for a free stage, 9 for
+    // the rows of x; 10 / 11 MMA thread waiting for a filled stage (hidden and predictor / down tiles), 12 for the
+    // accumulators to be drained, 13 / 14 MMA thread from a tile's start to its last commit
     unsigned long long* trace;
+    int trace_items;                  // behind the [gridDim.x][16] words: per thread block this many records of
+                                      // (queue entry + 1, start ns, end ns) of the first tiles it took
     PlanDev plan;
 };
 

@@ -183,7 +183,7 @@ def test_stack_prompt_on_the_tensor_core_path(n_tok, d):
     assert (plain - h_out).abs().max().item() <= U.TOL_BF16 * float(upd.pow(2).mean().sqrt().item())
 
 
-def check_chained_without_y(wl, Wp, preds, h0, h_out, t, steps, step0, tokens):
+def check_chained_without_y(wl, Wp, preds, h0, h_out, t, steps, step0, tokens, act=R.ACT_RELU):
     """Check of a run that recorded every block's input x, scores and selection but NOT its output y (the form in
     which the prompt path adds the down projection straight into the residual stream).  Scores and selection
     integers are checked as usual.  For the sampled token rows the oracle computes y_l from the recorded x_l and
@@ -205,7 +205,7 @@ def check_chained_without_y(wl, Wp, preds, h0, h_out, t, steps, step0, tokens):
             if l == 0:
                 assert (scores == 0).all()
             else:
-                s_ref = R.predict(hb(preds[l][0]), hb(preds[l][1]), x_all[s, l - 1], mean_pool=wl.n_tok > 1)
+                s_ref = R.predict(hb(preds[l][0]), hb(preds[l][1]), x_all[s, l - 1], act=act, mean_pool=wl.n_tok > 1)
                 assert U.rel_err(scores, s_ref.astype(np.float64)) <= tol
             sel = R.select(scores, wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0, wl.seed, step0 + s, l,
                            force_all=(l == 0))
@@ -225,6 +225,47 @@ def check_chained_without_y(wl, Wp, preds, h0, h_out, t, steps, step0, tokens):
                 assert (np.abs(xr - xg) <= bound / scale + 2 ** -7 * np.abs(xr) + 1e-6).all(), (s, l)
         assert np.abs(h_out[s].cpu().numpy()[tokens] - h).max() <= bound + 1e-5 * np.abs(h).max(), s
     return lost
+
+
+@pytest.mark.parametrize("variant", ["wide_rank512", "group256", "three_token_tiles", "everything_lost", "no_devices",
+                                     "linear_predictor", "full_tile_of_tokens"])
+def test_prompt_stack_single_launch_variants(variant):
+    """The one-launch prompt kernel under the other settings: a 5120-wide block with a 512-unit predictor (two unit
+    tiles), the paper's 256-neuron groups (two hidden tiles per group), three token tiles with a ragged last one,
+    k = 0 with every device always lost (blocks from the second on keep nothing), no devices at all, a predictor
+    without the ReLU, exactly 256 tokens.  Checked by chaining the oracle's outputs from the recorded inputs."""
+    kw = dict(act=B.ACT_RELU)
+    if variant == "wide_rank512":
+        wl = synth.Workload("v", 3, 5120, 128 * 6, 128, 512, "bf16", (0.0, 0.4, 0.8), (1, 2, 1), 300, 1, n_tok=300)
+    elif variant == "group256":
+        wl = synth.Workload("v", 3, 512, 256 * 5, 256, 64, "bf16", (0.1, 0.6), (1, 1), 400, 2, n_tok=257)
+    elif variant == "three_token_tiles":
+        wl = synth.Workload("v", 4, 256, 64 * 12, 64, 64, "bf16", (0.0, 0.3, 0.6), (2, 1, 1), 250, 1, n_tok=700)
+    elif variant == "everything_lost":
+        wl = synth.Workload("v", 3, 512, 128 * 4, 128, 64, "bf16", (1.0, 1.0), (1, 1), 0, 2, n_tok=200)
+    elif variant == "no_devices":
+        wl = synth.Workload("v", 3, 512, 64 * 9, 64, 128, "bf16", (), (), 400, 1, n_tok=129)
+    elif variant == "linear_predictor":
+        wl = synth.Workload("v", 3, 1024, 128 * 5, 128, 200, "bf16", (0.2, 0.7), (1, 1), 334, 2, n_tok=160)
+        kw.update(act=B.ACT_NONE)
+    else:
+        wl = synth.Workload("v", 2, 768, 64 * 7, 64, 96, "bf16", (0.0, 0.5), (3, 1), 430, 1, n_tok=256)
+    stack, Wp, preds = build_stack(wl, **kw)
+    h0 = torch.stack([synth.stream_input(wl, s, DEV) for s in range(wl.steps)])
+    plain, t = run_without_y(wl, stack, h0, wl.steps, step0=2)
+    assert stack.last_launches() == wl.steps                      # one launch per prompt
+    check_chained_without_y(wl, Wp, preds, h0, plain, t, wl.steps, 2, list(range(0, wl.n_tok, 7)) + [wl.n_tok - 1],
+                            act=kw["act"])
+    if variant == "everything_lost":
+        assert (t["n_keep"][:, 1:] == 0).all().item()
+        # nothing kept from the second block on: the stream stays what the first block left
+    # and the same stack through the one-launch-per-step path gives the same selections
+    stack.set_mode(1)
+    plain1, t1 = run_without_y(wl, stack, h0, wl.steps, step0=2)
+    assert stack.last_launches() > wl.steps
+    assert (t1["n_keep"] == t["n_keep"]).all().item()
+    upd = (plain1 - h0).double().pow(2).mean().sqrt().item()
+    assert (plain - plain1).abs().max().item() <= U.TOL_BF16 * max(upd, 1e-3) * 4
 
 
 def test_prompt_stack_at_the_benchmarked_shape():

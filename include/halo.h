@@ -412,10 +412,28 @@ halo_status halo_stack_decode(halo_stack* stack, const float* h0, int steps, uin
  * copies h_out back and synchronises the stream before returning. */
 halo_status halo_stack_decode_host(halo_stack* stack, const float* h0_host, int steps, uint32_t step0,
                                    float* h_out_host, void* stream);
-/* How halo_stack_decode runs.  mode 0 (default): decode of bf16 stacks with d_model in {2048, 4096, 5120, 8192}
- * runs as ONE persistent cooperative kernel over all steps and blocks, the predictor and selection of block
- * l+1 overlapped with the weight stream of block l; anything else runs one launch per step of the path.
- * mode 1: always one launch per step of the path (no overlap; for comparison and checking). */
+/* How halo_stack_decode runs.  mode = 0 (default) or a sum of the flags below.
+ * Default: decode of bf16 stacks with d_model in {2048, 4096, 5120, 8192} runs as ONE persistent cooperative
+ * kernel over all steps and blocks, with the two overlaps of the paper's generation phase (Sec. III-B.3): the
+ * predictor and selection of block l+1 run beside the weight stream of block l (Pred beside Comp/Comm), and the
+ * first weights of block l+1 are fetched while block l is still being merged (Load beside Comp).  Prompts of more
+ * than 128 tokens (bf16, d_model % 256 == 0, group size 64/128/256, predictor rank <= 1024) run as one persistent
+ * kernel per prompt.  Anything else runs one launch per step of the path.
+ *   HALO_STACK_PER_STEP_LAUNCHES  always one launch per step of the path (for comparison and checking);
+ *   HALO_STACK_PRED_SERIAL        persistent decode kernel with the predictor and selection of a block at the start
+ *                                 of that block, in front of its weight stream (the ablation arm "Pred not overlapped");
+ *   HALO_STACK_LOAD_SERIAL        persistent decode kernel that fetches no weights of block l+1 before block l is
+ *                                 merged (the ablation arm "Load not overlapped");
+ *   HALO_STACK_DETERMINISTIC      persistent decode kernel with a fixed assignment of neuron batches to thread blocks
+ *                                 and column sums added in a fixed order, so that two runs give bitwise identical
+ *                                 results (slower: every thread block reads every other's sums); the default adds
+ *                                 them with atomic reductions in arrival order.
+ * The last three only act on the persistent decode kernel; results are the same numbers in every mode up to the
+ * order of fp32 additions. */
+#define HALO_STACK_PER_STEP_LAUNCHES 1
+#define HALO_STACK_PRED_SERIAL 2
+#define HALO_STACK_LOAD_SERIAL 4
+#define HALO_STACK_DETERMINISTIC 8
 halo_status halo_stack_set_mode(halo_stack* stack, int mode);
 /* Measurement options, process-wide.  The defaults are the measured best; the options exist so that a sweep or an
  * ablation can be run through the same library.  value = -1 restores the default.  A stack reads the first three

@@ -473,6 +473,8 @@ struct halo_stack {
     float* p_z;
     halo::PersistSel* p_sel;       // [3]
     unsigned* p_sync;              // [32]
+    __nv_bfloat16* p_xhist;        // [2][d]
+    float* p_det_rows;             // [2][kMaxGrid][d]
     void* ffn_ws;                  // H buffer of the tensor-core path (multi-token stacks), or null
     bool ffn_ws_clean = false;     // its control words are known to be zero
     // multi-token stacks: predictor + selection of block l+1 run on a side stream while block l's FFN runs
@@ -554,6 +556,9 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     const size_t o_pz = carve(sizeof(float) * 2 * pred->rank);
     const size_t o_ps = carve(sizeof(PersistSel) * 3);
     const size_t o_py = carve(sizeof(unsigned) * 32);
+    constexpr size_t kMaxGrid = 192;   // thread blocks of the persistent kernel (one per SM)
+    const size_t o_xh = carve(2 * d * 2);
+    const size_t o_dr = carve(persistent_supported(*ffn, n_tok, G) ? sizeof(float) * 2 * kMaxGrid * d : 16);
     const size_t ws_bytes = prefill_supported(*ffn, n_tok) ? prefill_workspace_bytes(*ffn, n_tok) : 0;
     const size_t o_ws = carve(ws_bytes ? ws_bytes : 16);
     const size_t o_sc2 = carve(sizeof(float) * G), o_dg2 = carve(sizeof(int32_t) * G);
@@ -582,6 +587,8 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     s->p_z = reinterpret_cast<float*>(base + o_pz);
     s->p_sel = reinterpret_cast<PersistSel*>(base + o_ps);
     s->p_sync = reinterpret_cast<unsigned*>(base + o_py);
+    s->p_xhist = reinterpret_cast<__nv_bfloat16*>(base + o_xh);
+    s->p_det_rows = reinterpret_cast<float*>(base + o_dr);
     s->ffn_ws = ws_bytes ? static_cast<void*>(base + o_ws) : nullptr;
     s->set_scores[0] = s->scores; s->set_scores[1] = reinterpret_cast<float*>(base + o_sc2);
     s->set_dev[0] = s->dev_of_group; s->set_dev[1] = reinterpret_cast<int32_t*>(base + o_dg2);
@@ -716,7 +723,7 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
     const int L = s->n_layers, G = s->G, n_dev = s->n_dev;
     long long launches = 0;
     halo_status rc;
-    if (s->persistent_ok && s->mode == 0) {
+    if (s->persistent_ok && !(s->mode & HALO_STACK_PER_STEP_LAUNCHES)) {
         // whole run in one cooperative launch
         if (cudaMemsetAsync(s->p_partials, 0, sizeof(float) * 3 * 2 * d, st) != cudaSuccess ||
             cudaMemsetAsync(s->p_sync, 0, sizeof(unsigned) * 32, st) != cudaSuccess)
@@ -733,6 +740,10 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
         P.plan = s->plan.dev;
         P.trace = s->trace; P.trace_blocks = s->trace_blocks;
         P.cross_stages = s->cross_stages; P.l2_ahead = s->l2_ahead;
+        if (s->mode & HALO_STACK_LOAD_SERIAL) { P.cross_stages = 0; P.l2_ahead = 0; }
+        P.pred_serial = (s->mode & HALO_STACK_PRED_SERIAL) ? 1 : 0;
+        P.deterministic = (s->mode & HALO_STACK_DETERMINISTIC) ? 1 : 0;
+        P.x_hist = s->p_xhist; P.det_rows = s->p_det_rows;
         if (taps) {
             P.tap_x = static_cast<__nv_bfloat16*>(taps->x); P.tap_scores = taps->scores;
             P.tap_dev_of_group = taps->dev_of_group; P.tap_arrived = taps->arrived; P.tap_keep_list = taps->keep_list;
@@ -817,7 +828,7 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
 #define HALO_COPY(dst, src, bytes)                                                                    \
     do { if (cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToDevice, st) != cudaSuccess)     \
              return HALO_ERR_CUDA; } while (0)
-    if (T > 1 && s->prompt_ok && s->mode == 0 && (!taps || !taps->y)) {
+    if (T > 1 && s->prompt_ok && !(s->mode & HALO_STACK_PER_STEP_LAUNCHES) && (!taps || !taps->y)) {
         // Prompt path, one launch per prompt: every block of the stack inside one persistent kernel.  The residual
         // stream is updated in place in the caller's h_out.
         PromptParams P;
@@ -1036,7 +1047,7 @@ extern "C" halo_status halo_stack_status(halo_stack* s, uint32_t* value, void* s
 }
 
 extern "C" halo_status halo_stack_set_mode(halo_stack* s, int mode) {
-    if (!s || (mode != 0 && mode != 1)) return HALO_ERR_ARG;
+    if (!s || mode < 0 || mode > 15) return HALO_ERR_ARG;
     s->mode = mode;
     return HALO_OK;
 }

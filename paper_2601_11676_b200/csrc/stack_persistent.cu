@@ -257,11 +257,13 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
             for (int l = 0; l < L && alive; ++l) {
                 const PersistSel* sb = (l == 0) ? &P.sel[2] : &P.sel[l & 1];
                 if (lane == 0) {
-                    // (a) rows of the next block's predictor that this thread block owns
-                    if (l + 1 < L) {
+                    // (a) rows of a predictor that this thread block owns: the next block's, one layer ahead, beside
+                    //     this block's stream; or (pred_serial) this block's own, in front of its stream
+                    const int lp = P.pred_serial ? l : l + 1;
+                    if (lp >= 1 && lp < L) {
                         const int r0 = static_cast<int>(static_cast<long long>(cta) * r / workers);
                         const int r1 = static_cast<int>(static_cast<long long>(cta + 1) * r / workers);
-                        const __nv_bfloat16* W1 = P.W1[l + 1];
+                        const __nv_bfloat16* W1 = P.W1[lp];
                         for (int row = r0; row < r1 && alive; row += ROWS) {
                             const int n = min(ROWS, r1 - row);
                             int s;
@@ -322,8 +324,12 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                     // flight so that the round trip of the atomic is off the issue path.
                     long long b = cta;
                     long long ahead[kFetchAhead];
+                    // deterministic: batch cta, cta + workers, ...: every thread block sums the same batches in the
+                    // same order in every run
 #pragma unroll
-                    for (int k = 0; k < kFetchAhead; ++k) ahead[k] = static_cast<long long>(workers) + atomicAdd(ctr, 1u);
+                    for (int k = 0; k < kFetchAhead; ++k)
+                        ahead[k] = P.deterministic ? static_cast<long long>(cta) + static_cast<long long>(workers) * (k + 1)
+                                                   : static_cast<long long>(workers) + atomicAdd(ctr, 1u);
                     while (b < U) {
                         int s;
                         if (!acquire(s)) { alive = false; break; }
@@ -345,7 +351,8 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                         b = ahead[0];
 #pragma unroll
                         for (int k = 0; k + 1 < kFetchAhead; ++k) ahead[k] = ahead[k + 1];
-                        ahead[kFetchAhead - 1] = (b < U) ? static_cast<long long>(workers) + atomicAdd(ctr, 1u) : U;
+                        if (P.deterministic) ahead[kFetchAhead - 1] = ahead[kFetchAhead - 2] + workers;
+                        else ahead[kFetchAhead - 1] = (b < U) ? static_cast<long long>(workers) + atomicAdd(ctr, 1u) : U;
                     }
                     if (alive) alive = marker(ST_END, 0);
                 }
@@ -415,6 +422,8 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                     reinterpret_cast<uint4*>(xs)[c] = packed;
                     if (cta == 0 && P.tap_x)
                         reinterpret_cast<uint4*>(P.tap_x + (static_cast<size_t>(step_i) * L + l_next) * d)[c] = packed;
+                    if (cta == 0 && P.pred_serial)
+                        reinterpret_cast<uint4*>(P.x_hist + static_cast<size_t>(l_next & 1) * d)[c] = packed;
                 }
             }
         }
@@ -488,8 +497,15 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                     if (row < a1) {
                         const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(row) * row_bytes);
                         float dot0 = 0.0f, dot1 = 0.0f;
+                        if (P.pred_serial) {
+                            // this block's own predictor: its input is the previous block's x, kept in global memory
+                            const uint4* xp = reinterpret_cast<const uint4*>(P.x_hist + static_cast<size_t>((l - 1) & 1) * d);
+#pragma unroll
+                            for (int i = 0; i < XC; ++i) dot_bf16x8(rp[p1_base + 32 * i], __ldcg(xp + p1_base + 32 * i), dot0, dot1);
+                        } else {
 #pragma unroll
                         for (int i = 0; i < XC; ++i) dot_bf16x8(rp[p1_base + 32 * i], xq[i], dot0, dot1);
+                        }
                         const float dot = warp_sum(dot0 + dot1);
                         if (lane == 0) red[row * WPR + part] = dot;
                     }
@@ -516,7 +532,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 } else if (type == ST_PRED) {
                     if (tid == 0) {
                         // hidden values of the prediction made during this block, in the buffer of its parity
-                        const unsigned n_pred = static_cast<unsigned>(step_i) * (L - 1) + (l + 1);
+                        const unsigned n_pred = static_cast<unsigned>(step_i) * (L - 1) + (P.pred_serial ? l : l + 1);
                         float* zdst = P.z + static_cast<size_t>(n_pred & 1u) * r;
                         for (int i = 0; i < a1; ++i) {
                             float z = 0.0f;
@@ -538,11 +554,35 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
 
             // ------------------------------ end of the block: flush, grid barrier, merge + glue ------------------------------
             trace(TR_STAGES_DONE, global_timer_ns());
-            if (any) stage_sums();
+            if (any || P.deterministic) stage_sums();
             pc_barrier();
+            if (P.deterministic) {
+                // this thread block's column sums (replicas added in index order) go to its own row
+                float* rowp = P.det_rows + (static_cast<size_t>(q & 1u) * grid + cta) * d;
+                if (owner) {
+#pragma unroll
+                    for (int p = 0; p < P2; ++p) {
+                        const int c = col0 + kPC * p;
+                        if (c < chunks) {
+                            float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+#pragma unroll
+                            for (int k = 0; k < REP; ++k) {
+                                const float* src = reinterpret_cast<const float*>(vec_buf) + static_cast<size_t>(k) * d + c * 8;
+                                const float4 u = reinterpret_cast<const float4*>(src)[0], v = reinterpret_cast<const float4*>(src)[1];
+                                a.x += u.x; a.y += u.y; a.z += u.z; a.w += u.w;
+                                b.x += v.x; b.y += v.y; b.z += v.z; b.w += v.w;
+                            }
+                            reinterpret_cast<float4*>(rowp + c * 8)[0] = a;
+                            reinterpret_cast<float4*>(rowp + c * 8)[1] = b;
+                        }
+                    }
+                }
+                __threadfence();
+                pc_barrier();
+            }
             bool okb = true;
             if (tid == 0) {
-                if (any) {
+                if (any && !P.deterministic) {
                     float* dst = P.partials + (q % 3u) * buf_stride + static_cast<size_t>(cta % kAccBufs) * acc_stride;
 #pragma unroll
                     for (int k = 0; k < REP; ++k)
@@ -575,6 +615,17 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 for (int p = 0; p < P2; ++p) {
                     const int c = col0 + kPC * p;
                     if (c < chunks) {
+                        float y[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                        if (P.deterministic) {
+                            // the rows of all streaming thread blocks, added in index order
+                            const float* rows = P.det_rows + static_cast<size_t>(q & 1u) * grid * d + c * 8;
+                            for (int w = 0; w < workers; ++w) {
+                                const float4 u = __ldcg(reinterpret_cast<const float4*>(rows + static_cast<size_t>(w) * d));
+                                const float4 v = __ldcg(reinterpret_cast<const float4*>(rows + static_cast<size_t>(w) * d) + 1);
+                                y[0] += u.x; y[1] += u.y; y[2] += u.z; y[3] += u.w;
+                                y[4] += v.x; y[5] += v.y; y[6] += v.z; y[7] += v.w;
+                            }
+                        } else {
                         float4 va[kAccBufs], vb[kAccBufs];
 #pragma unroll
                         for (int k = 0; k < kAccBufs; ++k) {
@@ -582,11 +633,11 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                             va[k] = __ldcg(src);
                             vb[k] = __ldcg(src + 1);
                         }
-                        float y[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 #pragma unroll
                         for (int k = 0; k < kAccBufs; ++k) {
                             y[0] += va[k].x; y[1] += va[k].y; y[2] += va[k].z; y[3] += va[k].w;
                             y[4] += vb[k].x; y[5] += vb[k].y; y[6] += vb[k].z; y[7] += vb[k].w;
+                        }
                         }
 #pragma unroll
                         for (int e = 0; e < 8; ++e) hreg[p][e] += y[e];

@@ -40,6 +40,11 @@ struct PersistParams {
     int cross_stages;                      // stages of the next block a producer may issue before its consumers
                                            // have passed the grid barrier of the current block
     int l2_ahead;                          // batches per thread block prefetched into L2 on entering a block
+    int pred_serial;                       // 1: the predictor rows and the selection of block l run at the start of
+                                           // block l itself (from the recorded x_{l-1}), not beside block l-1
+    int deterministic;                     // 1: fixed batch assignment and fixed-order sums (bitwise repeatable)
+    __nv_bfloat16* x_hist;                 // [2][d]: input of the previous block (pred_serial only)
+    float* det_rows;                       // [2][gridDim.x][d]: per-thread-block column sums (deterministic only)
     unsigned long long* trace;
     int trace_blocks;
     PlanDev plan;

@@ -28,12 +28,23 @@ from paper_2601_11676_b200 import synth  # noqa: E402
 
 METRIC = "group-sparse FFN decode tokens/s on 1 B200; achieved HBM GB/s vs ~8 TB/s"
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read+write per launch / algorithmic bytes per launch of stack_decode_kernel, from an ncu capture of
-# a 4-block 7B-shaped case (3 231 938 048 + 910 080 bytes against 3 231 058 944 algorithmic); traffic is
-# proportional to the kept groups processed, so the ratio carries over to the full-size launch.  Set to None
-# when the kernel changes.
+# dram__bytes_read+write per launch / algorithmic bytes per launch of stack_decode_kernel, from an ncu capture of a
+# 4-block 7B-shaped case (profiles/stack_decode_kernel_llama2-7b_4blocks.md); traffic is proportional to the kept
+# groups processed, so the ratio carries over to the full-size launch.  The figure belongs to the kernel sources with
+# the hash below: when they change the line reports no traffic until the counters have been taken again.
 STACK_KERNEL_TRAFFIC_RATIO = 1.0003
+STACK_KERNEL_SOURCES = ("stack_persistent.cu", "stack_persistent.cuh", "ffn_math.cuh", "tma.cuh", "select_device.cuh")
+STACK_KERNEL_SOURCES_SHA1 = "unset"
 FALLBACK_HBM_GBS = 6650.0
+
+
+def stack_kernel_sources_sha1():
+    import hashlib
+    h = hashlib.sha1()
+    for name in STACK_KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2601_11676_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
 
 
 def measured_peaks():
@@ -120,6 +131,20 @@ def aggregate_tokens_per_s(tokens_per_rank, ms_this_rank, world, device):
 # the CUDA arm
 # ----------------------------------------------------------------------------------------------------------------
 
+def tokens_of(K, world):
+    return K * world
+
+
+def workload_config(wl, world):
+    """The same keys in both arms: what the workload is, not how a particular run went."""
+    return {"workload": wl.name, "n_layers": wl.n_layers, "d_model": wl.d_model, "d_ffn": wl.d_ffn,
+            "group_size": wl.group_size, "n_groups": wl.n_groups, "pred_rank": wl.pred_rank,
+            "keep_permille": wl.keep_permille, "k_critical": (wl.keep_permille * wl.n_groups + 999) // 1000,
+            "virtual_devices": wl.n_dev, "loss_rate": list(wl.loss_rate),
+            "l2": "inputs larger than L2 (weights of the stack: %.2f GB)" % (wl.n_layers * wl.layer_bytes / 1e9),
+            "parallelism": "replicas only" if world > 1 else "single GPU"}
+
+
 def build_stack(wl, dev):
     from paper_2601_11676_b200 import binding as B
     code = B.F32 if wl.dtype == "f32" else B.BF16
@@ -168,22 +193,28 @@ def run_halo(args, rank, world, local_rank):
     pred_bytes = K * (L - 1) * wl.pred_bytes
     algo_bytes_total = weight_bytes + pred_bytes
 
-    # ---- device-resident timing: W warm-up steps, then exactly K timed steps --------------------------------------
+    # ---- device-resident timing: W warm-up steps, then exactly K timed steps, REPS times back to back inside one
+    #      sampled region; the median run is the reported one, all runs are listed ----------------------------------
+    REPS = 5
     stack.decode(h0[:W], W, 0, h_out[:W])
     barrier()
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(REPS)]
     barrier()
-    ev0.record()
-    stack.decode(h0[W:], K, W, h_out[W:])
-    ev1.record()
+    for ev0, ev1 in evs:
+        ev0.record()
+        stack.decode(h0[W:], K, W, h_out[W:])
+        ev1.record()
     barrier()
-    ms = ev0.elapsed_time(ev1)
+    runs_ms = [ev0.elapsed_time(ev1) for ev0, ev1 in evs]
+    ms = sorted(runs_ms)[REPS // 2]
     launches = stack.last_launches()
     clocks = sampler.stop() if rank == 0 else None
+    if stack.status() != 0:
+        raise RuntimeError("device status after the timed run: " + B.status_message(stack.status()))
 
     # ---- end to end through the host entry point: pinned host buffers, copies inside the timed region ----------
     h0_host = h0[W:].cpu().pin_memory()
@@ -223,6 +254,7 @@ def run_halo(args, rank, world, local_rank):
 
     # ---- max over ranks -------------------------------------------------------------------------------------------
     ms, ms_e2e = max_over_ranks([ms, ms_e2e], world, dev)
+    runs_ms = max_over_ranks(runs_ms, world, dev)
     if rank != 0:
         return None
 
@@ -234,11 +266,9 @@ def run_halo(args, rank, world, local_rank):
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": wl.dtype, "data": "synthetic",
-        "config": {"workload": wl.name, "n_layers": L, "d_model": d, "d_ffn": wl.d_ffn, "group_size": wl.group_size,
-                   "n_groups": G, "pred_rank": wl.pred_rank, "keep_permille": wl.keep_permille,
-                   "k_critical": B.k_of(wl), "virtual_devices": wl.n_dev, "loss_rate": list(wl.loss_rate),
-                   "kept_fraction": kept_fraction, "l2": "inputs larger than L2 (weights of the stack: %.2f GB)"
-                   % (L * wl.layer_bytes / 1e9), "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "config": dict(workload_config(wl, world), kept_fraction=kept_fraction),
+        "runs": {"ms_per_step": [r / K for r in runs_ms], "tokens_per_s": [tokens_of(K, world) / (r * 1e-3) for r in runs_ms],
+                 "reported": "median of %d back-to-back runs of the K timed steps" % len(runs_ms)},
         "clocks": clocks,
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 4 * d * wl.n_tok,
                 "d2h_bytes_per_step": 4 * d * wl.n_tok},
@@ -248,14 +278,18 @@ def run_halo(args, rank, world, local_rank):
                 "peak_gbs": peak, "peak_kind": peak_kind},
     }
     persistent = launches == 1
+    traffic_valid = STACK_KERNEL_TRAFFIC_RATIO is not None and stack_kernel_sources_sha1() == STACK_KERNEL_SOURCES_SHA1
     if persistent:
         # the timed region is ONE launch of the persistent stack kernel: its duration is the event time itself
         result["roofline"] = {
             "bound": "hbm", "kernel": "stack_decode_kernel (persistent: all steps x blocks, a1..a9 + glue)",
             "achieved": step_gbs, "peak": peak, "unit": "GB/s", "frac": step_gbs / peak, "peak_kind": peak_kind,
-            "traffic": (algo_bytes_total * STACK_KERNEL_TRAFFIC_RATIO) if STACK_KERNEL_TRAFFIC_RATIO else None,
-            "traffic_note": "ncu DRAM bytes of a 4-block capture scaled by kept groups processed",
-            "avg_launch_us": ms * 1e3, "launches_timed": 1,
+            "traffic": (algo_bytes_total * STACK_KERNEL_TRAFFIC_RATIO) if traffic_valid else None,
+            "traffic_note": ("scaled: ncu DRAM bytes of a 4-block capture x kept groups processed "
+                             "(kernel sources %s)" % STACK_KERNEL_SOURCES_SHA1[:12]) if traffic_valid else
+                            "none: the kernel sources changed since the counters were taken",
+            "peak_note": "the peak is a read+write copy; a read-only stream can pass it" if step_gbs > peak else None,
+            "avg_launch_us": ms * 1e3, "launches_timed": len(runs_ms),
             "algorithmic_bytes_per_launch": algo_bytes_total, "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS}
     else:
         result["roofline"] = {
@@ -276,6 +310,8 @@ def run_halo(args, rank, world, local_rank):
                                      ("llama2-13b-decode", "tinyllama-1.1b-decode", "llama2-7b-decode")
                                      if n != wl.name]
         result["other_blocks"] = other_blocks_report(dev, peak)
+        result["keep_sweep"] = keep_sweep(dev, peak)
+        result["overlap_ablation"] = overlap_ablation(dev)
     if world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget)
     return result
@@ -381,6 +417,82 @@ def other_blocks_report(dev, peak, reps=12):
             "device_status": int(status.item())}
 
 
+def _timed_decode(stack, wl, dev, steps, warm, reps=3):
+    """Median milliseconds of `steps` tokens through `stack` (one decode call), and the kept groups of those steps."""
+    from paper_2601_11676_b200 import binding as B
+    L = wl.n_layers
+    total = warm + steps
+    h0 = torch.stack([synth.stream_input(wl, s, dev) for s in range(total)])
+    out = torch.empty_like(h0)
+    nk = torch.zeros((total, L), dtype=torch.int32, device=dev)
+    stack.decode(h0, total, 0, out, B.Taps(None, None, None, None, None, nk.data_ptr(), None))
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        stack.decode(h0[warm:], steps, warm, out[warm:])
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    return sorted(ts)[len(ts) // 2], int(nk[warm:].sum().item())
+
+
+def keep_sweep(dev, peak, steps=48, warm=4):
+    """The 7B-shaped stack at the keep ratios of its configuration, with the stated loss rates and - supplementary -
+    with every virtual device always lost, where the kept fraction is the keep ratio itself (the predictor's top-k
+    alone decides what is read).  Bytes are counted over the kept groups of the timed steps."""
+    from paper_2601_11676_b200 import binding as B
+    base = synth.workload("llama2-7b-decode")
+    Wp = [synth.packed_layer(base, l, dev) for l in range(base.n_layers)]
+    preds = [synth.predictor(base, l, dev) for l in range(base.n_layers)]
+    ffn = B.ffn_shape(base.d_model, base.d_ffn, base.group_size, B.BF16)
+    pred = B.pred_shape(base.d_model, base.pred_rank, base.n_groups, B.BF16)
+    rows = []
+    for lost in (False, True):
+        for permille in (300, 500, 700, 1000):
+            wl = synth.workload("llama2-7b-decode", keep_permille=permille,
+                                loss_rate=(1.0,) * base.n_dev if lost else base.loss_rate)
+            plan = B.Plan(wl.n_groups, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
+            stack = B.Stack(ffn, pred, 1, plan, Wp, [p[0] for p in preds], [p[1] for p in preds])
+            ms, kept = _timed_decode(stack, wl, dev, steps, warm)
+            byts = kept * wl.group_bytes + steps * (wl.n_layers - 1) * wl.pred_bytes
+            gbs = byts / (ms * 1e-3) / 1e9
+            rows.append({"keep_permille": permille, "devices": "all lost (supplementary)" if lost else "as configured",
+                         "kept_fraction": kept / float(steps * wl.n_layers * wl.n_groups),
+                         "tokens_per_s": steps / (ms * 1e-3), "achieved_gbs": gbs,
+                         "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS, "frac_of_peak": gbs / peak,
+                         "device_status": stack.status()})
+            stack.close()
+    return {"workload": "llama2-7b-decode", "steps": steps, "rows": rows}
+
+
+def overlap_ablation(dev, steps=48, warm=4):
+    """The arms of the paper's overlap ablation (Table V) restated for one GPU, all inside the persistent kernel:
+    predictor + selection beside the previous block's stream or in front of the block's own; first weights of the
+    next block fetched during the merge or not; and, for scale, one launch per step of the path."""
+    from paper_2601_11676_b200 import binding as B
+    out = []
+    for name in ("llama2-7b-decode", "tinyllama-1.1b-decode"):
+        wl = synth.workload(name)
+        stack, Wp, preds, plan, ffn = build_stack(wl, dev)
+        arms = [("both overlaps (default)", 0), ("Pred overlapped only", B.STACK_LOAD_SERIAL),
+                ("Load overlapped only", B.STACK_PRED_SERIAL), ("no overlap", B.STACK_PRED_SERIAL | B.STACK_LOAD_SERIAL),
+                ("one launch per step of the path", B.STACK_PER_STEP_LAUNCHES)]
+        ms_of = {}
+        for label, mode in arms:
+            stack.set_mode(mode)
+            ms_of[label], _ = _timed_decode(stack, wl, dev, steps, warm)
+        base = ms_of["no overlap"]
+        out.append({"workload": name, "steps": steps,
+                    "arms": [{"arm": label, "ms_per_token": ms_of[label] / steps, "tokens_per_s": steps / (ms_of[label] * 1e-3),
+                              "speedup_over_no_overlap": base / ms_of[label]} for label, _ in arms]})
+        stack.close()
+        del stack, Wp, preds
+        torch.cuda.empty_cache()
+    return out
+
+
 def decode_brief(name, dev, peak, steps=64, warm=4):
     """tokens/s and algorithmic GB/s of another decode workload (one persistent launch over `steps` tokens)."""
     from paper_2601_11676_b200 import binding as B
@@ -439,6 +551,19 @@ def prefill_report(wl, Wp, preds, plan, ffn, dev, n_tok=512, prompts=16, warm=3)
         reps.append(a.elapsed_time(b))
     ms = sorted(reps)[1]
     launches = stack.last_launches()
+    # the same prompts through the one-launch-per-prompt kernel (not the default: see the header), for the record
+    stack.set_mode(B.STACK_PROMPT_ONE_LAUNCH)
+    stack.decode(h0[:warm], warm, 0, h_out[:warm])
+    one = []
+    for _ in range(3):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        stack.decode(h0[warm:], prompts, warm, h_out[warm:])
+        b.record()
+        torch.cuda.synchronize()
+        one.append(a.elapsed_time(b))
+    one_launches = stack.last_launches()
+    status |= stack.status()
     kept = int(nk_rec[warm:].sum().item())
     flops = 6.0 * n_tok * kept * wl.group_size * d + prompts * (L - 1) * 2.0 * n_tok * (d * wl.pred_rank + wl.pred_rank * G)
     tflops = flops / (ms * 1e-3) / 1e12
@@ -447,7 +572,9 @@ def prefill_report(wl, Wp, preds, plan, ffn, dev, n_tok=512, prompts=16, warm=3)
             "ms_per_prompt": ms / prompts, "ms_per_prompt_runs": [r / prompts for r in reps], "tokens_per_s": prompts * n_tok / (ms * 1e-3), "tflops": tflops,
             "bound": "tensor", "peak_burst_tflops": burst, "frac_of_burst_peak": tflops / burst,
             "peak_sustained_tflops": sustained, "frac_of_sustained_peak": tflops / sustained,
-            "kept_fraction": kept / float(prompts * L * G), "gpu_launches": int(launches), "device_status": status}
+            "kept_fraction": kept / float(prompts * L * G), "gpu_launches": int(launches), "device_status": status,
+            "one_launch_per_prompt": {"ms_per_prompt": sorted(one)[1] / prompts, "gpu_launches": int(one_launches),
+                                      "tflops": flops / (sorted(one)[1] * 1e-3) / 1e12}}
 
 
 # ----------------------------------------------------------------------------------------------------------------
@@ -530,7 +657,7 @@ def run_reference(args, rank, world):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": dt * 1e3 / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "keep_permille": wl.keep_permille},
+        "config": workload_config(wl, 1 if world <= 1 else world),
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,

@@ -416,9 +416,9 @@ halo_status halo_stack_decode_host(halo_stack* stack, const float* h0_host, int 
  * Default: decode of bf16 stacks with d_model in {2048, 4096, 5120, 8192} runs as ONE persistent cooperative
  * kernel over all steps and blocks, with the two overlaps of the paper's generation phase (Sec. III-B.3): the
  * predictor and selection of block l+1 run beside the weight stream of block l (Pred beside Comp/Comm), and the
- * first weights of block l+1 are fetched while block l is still being merged (Load beside Comp).  Prompts of more
- * than 128 tokens (bf16, d_model % 256 == 0, group size 64/128/256, predictor rank <= 1024) run as one persistent
- * kernel per prompt.  Anything else runs one launch per step of the path.
+ * first weights of block l+1 are fetched while block l is still being merged (Load beside Comp).  Anything else
+ * runs one launch per step of the path; for prompts the predictor and selection of block l+1 then run on a side
+ * stream beside the tensor-core FFN of block l.
  *   HALO_STACK_PER_STEP_LAUNCHES  always one launch per step of the path (for comparison and checking);
  *   HALO_STACK_PRED_SERIAL        persistent decode kernel with the predictor and selection of a block at the start
  *                                 of that block, in front of its weight stream (the ablation arm "Pred not overlapped");
@@ -428,12 +428,20 @@ halo_status halo_stack_decode_host(halo_stack* stack, const float* h0_host, int 
  *                                 and column sums added in a fixed order, so that two runs give bitwise identical
  *                                 results (slower: every thread block reads every other's sums); the default adds
  *                                 them with atomic reductions in arrival order.
- * The last three only act on the persistent decode kernel; results are the same numbers in every mode up to the
- * order of fp32 additions. */
+ *   HALO_STACK_PROMPT_ONE_LAUNCH  prompts of more than 128 tokens (bf16, d_model % 256 == 0, group size 64/128/256,
+ *                                 predictor rank <= 1024, no y records asked for) run as ONE persistent kernel per
+ *                                 prompt: a tile queue over all blocks with the predictor, the selection and the
+ *                                 normalisation between blocks inside.  No host work between blocks and one launch
+ *                                 instead of ~7 per block; measured 4 % slower than the default on the 512-token 7B
+ *                                 shape (the normalisation sits on the critical path of every block boundary), so
+ *                                 it is not the default.
+ * The three flags before it only act on the persistent decode kernel; results are the same numbers in every mode up
+ * to the order of fp32 additions. */
 #define HALO_STACK_PER_STEP_LAUNCHES 1
 #define HALO_STACK_PRED_SERIAL 2
 #define HALO_STACK_LOAD_SERIAL 4
 #define HALO_STACK_DETERMINISTIC 8
+#define HALO_STACK_PROMPT_ONE_LAUNCH 16
 halo_status halo_stack_set_mode(halo_stack* stack, int mode);
 /* Measurement options, process-wide.  The defaults are the measured best; the options exist so that a sweep or an
  * ablation can be run through the same library.  value = -1 restores the default.  A stack reads the first three

@@ -20,7 +20,7 @@ F32, BF16 = 0, 1
 SEL_TOPK, SEL_THRESHOLD = 0, 1
 ACT_RELU, ACT_NONE = 0, 1
 DEV_NONFINITE_SCORE, DEV_BAD_INDEX, DEV_TIMEOUT = 1, 2, 4
-STACK_PER_STEP_LAUNCHES, STACK_PRED_SERIAL, STACK_LOAD_SERIAL, STACK_DETERMINISTIC = 1, 2, 4, 8
+STACK_PER_STEP_LAUNCHES, STACK_PRED_SERIAL, STACK_LOAD_SERIAL, STACK_DETERMINISTIC, STACK_PROMPT_ONE_LAUNCH = 1, 2, 4, 8, 16
 MAX_DEVICES, MAX_GROUPS = 32, 1024
 
 EXPORTS = [

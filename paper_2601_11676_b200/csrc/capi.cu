@@ -828,7 +828,8 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
 #define HALO_COPY(dst, src, bytes)                                                                    \
     do { if (cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToDevice, st) != cudaSuccess)     \
              return HALO_ERR_CUDA; } while (0)
-    if (T > 1 && s->prompt_ok && !(s->mode & HALO_STACK_PER_STEP_LAUNCHES) && (!taps || !taps->y)) {
+    if (T > 1 && s->prompt_ok && (s->mode & HALO_STACK_PROMPT_ONE_LAUNCH) && !(s->mode & HALO_STACK_PER_STEP_LAUNCHES) &&
+        (!taps || !taps->y)) {
         // Prompt path, one launch per prompt: every block of the stack inside one persistent kernel.  The residual
         // stream is updated in place in the caller's h_out.
         PromptParams P;
@@ -1047,7 +1048,7 @@ extern "C" halo_status halo_stack_status(halo_stack* s, uint32_t* value, void* s
 }
 
 extern "C" halo_status halo_stack_set_mode(halo_stack* s, int mode) {
-    if (!s || mode < 0 || mode > 15) return HALO_ERR_ARG;
+    if (!s || mode < 0 || mode > 31) return HALO_ERR_ARG;
     s->mode = mode;
     return HALO_OK;
 }

@@ -1122,12 +1122,31 @@ halo_status launch_group_ffn_prefill(const halo_ffn_shape& sh, const void* W, co
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return HALO_ERR_CUDA;
-    CUtensorMap map_x, map_w, map_w_half, map_h, map_wd;
     const int NS = std::min(S, 128);     // neurons per hidden tile; a 256-neuron group is two tiles
-    if (!make_map(&map_x, x, T, d, d, kBK, kBM) || !make_map(&map_w, W, w_rows, d, d, kBK, NS) ||
-        !make_map(&map_w_half, W, w_rows, d, d, kBK, NS / 2) ||
-        !make_map(&map_h, H, T, sh.d_ffn, sh.d_ffn, kBK, kBM) || !make_map(&map_wd, W, w_rows, d, d, 64, kBK))
-        return HALO_ERR_CUDA;
+    // The five tensor maps depend only on the pointers and the shape: they are encoded once per combination and
+    // kept (a stack calls this with the same few buffers for every prompt), not once per launch.
+    struct MapSet { const void* W; const void* x; const void* H; int T, d, S, G; CUtensorMap m[5]; bool used; };
+    constexpr int kMapSets = 256;
+    static MapSet cache[kMapSets];
+    static std::mutex cache_mutex;
+    CUtensorMap map_x, map_w, map_w_half, map_h, map_wd;
+    {
+        std::lock_guard<std::mutex> lock(cache_mutex);
+        size_t hsh = (reinterpret_cast<uintptr_t>(W) >> 8) * 1000003u ^ (reinterpret_cast<uintptr_t>(x) >> 8) * 7919u ^
+                     static_cast<size_t>(T) * 31u;
+        MapSet* e = &cache[hsh % kMapSets];
+        if (!(e->used && e->W == W && e->x == x && e->H == H && e->T == T && e->d == d && e->S == S && e->G == G)) {
+            MapSet fresh{};
+            fresh.W = W; fresh.x = x; fresh.H = H; fresh.T = T; fresh.d = d; fresh.S = S; fresh.G = G;
+            if (!make_map(&fresh.m[0], x, T, d, d, kBK, kBM) || !make_map(&fresh.m[1], W, w_rows, d, d, kBK, NS) ||
+                !make_map(&fresh.m[2], W, w_rows, d, d, kBK, NS / 2) ||
+                !make_map(&fresh.m[3], H, T, sh.d_ffn, sh.d_ffn, kBK, kBM) || !make_map(&fresh.m[4], W, w_rows, d, d, 64, kBK))
+                return HALO_ERR_CUDA;
+            fresh.used = true;
+            *e = fresh;      // a colliding entry is simply replaced
+        }
+        map_x = e->m[0]; map_w = e->m[1]; map_w_half = e->m[2]; map_h = e->m[3]; map_wd = e->m[4];
+    }
     const bool two_launches = option_value(OPT_PREFILL_TWO_LAUNCHES) == 1;
     if (T > kBM && d % 256 == 0 && !two_launches) {
         // both contractions in one launch, one CTA per SM pulling tiles from a queue

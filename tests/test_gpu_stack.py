@@ -177,10 +177,12 @@ def test_stack_prompt_on_the_tensor_core_path(n_tok, d):
     h0, h_out, t = run_with_taps(wl, stack, wl.steps)
     lost = check_teacher_forced(wl, Wp, preds, h0, h_out, t, wl.steps)
     assert lost > 0
-    plain, t2 = run_without_y(wl, stack, h0, wl.steps)
-    assert check_chained_without_y(wl, Wp, preds, h0, plain, t2, wl.steps, 0, list(range(n_tok))) == lost
-    upd = (h_out - h0).double()
-    assert (plain - h_out).abs().max().item() <= U.TOL_BF16 * float(upd.pow(2).mean().sqrt().item())
+    upd = float((h_out - h0).double().pow(2).mean().sqrt().item())
+    for mode in (0, B.STACK_PROMPT_ONE_LAUNCH):
+        stack.set_mode(mode)
+        plain, t2 = run_without_y(wl, stack, h0, wl.steps)
+        assert check_chained_without_y(wl, Wp, preds, h0, plain, t2, wl.steps, 0, list(range(n_tok))) == lost
+        assert (plain - h_out).abs().max().item() <= U.TOL_BF16 * upd
 
 
 def check_chained_without_y(wl, Wp, preds, h0, h_out, t, steps, step0, tokens, act=R.ACT_RELU):
@@ -251,6 +253,7 @@ def test_prompt_stack_single_launch_variants(variant):
     else:
         wl = synth.Workload("v", 2, 768, 64 * 7, 64, 96, "bf16", (0.0, 0.5), (3, 1), 430, 1, n_tok=256)
     stack, Wp, preds = build_stack(wl, **kw)
+    stack.set_mode(B.STACK_PROMPT_ONE_LAUNCH)
     h0 = torch.stack([synth.stream_input(wl, s, DEV) for s in range(wl.steps)])
     plain, t = run_without_y(wl, stack, h0, wl.steps, step0=2)
     assert stack.last_launches() == wl.steps                      # one launch per prompt
@@ -260,7 +263,7 @@ def test_prompt_stack_single_launch_variants(variant):
         assert (t["n_keep"][:, 1:] == 0).all().item()
         # nothing kept from the second block on: the stream stays what the first block left
     # and the same stack through the one-launch-per-step path gives the same selections
-    stack.set_mode(1)
+    stack.set_mode(0)
     plain1, t1 = run_without_y(wl, stack, h0, wl.steps, step0=2)
     assert stack.last_launches() > wl.steps
     assert (t1["n_keep"] == t["n_keep"]).all().item()
@@ -281,11 +284,14 @@ def test_prompt_stack_at_the_benchmarked_shape():
     tokens = [0, 127, 128, 255, 256, 300, 511]
     lost = check_teacher_forced(wl, Wp, preds, h0, h_out, t, wl.steps, step0=5, tokens=tokens)
     assert lost > 0                                   # some block really ran with groups dropped
-    plain, t2 = run_without_y(wl, stack, h0, wl.steps, step0=5)
-    lost2 = check_chained_without_y(wl, Wp, preds, h0, plain, t2, wl.steps, 5, tokens)
-    assert lost2 == lost
-    upd = (h_out - h0).double()
-    assert (plain - h_out).abs().max().item() <= U.TOL_BF16 * float(upd.pow(2).mean().sqrt().item())
+    upd = float((h_out - h0).double().pow(2).mean().sqrt().item())
+    for mode in (0, B.STACK_PROMPT_ONE_LAUNCH):      # the default (timed) form, and the one-launch-per-prompt kernel
+        stack.set_mode(mode)
+        plain, t2 = run_without_y(wl, stack, h0, wl.steps, step0=5)
+        assert (stack.last_launches() == wl.steps) == (mode != 0)
+        lost2 = check_chained_without_y(wl, Wp, preds, h0, plain, t2, wl.steps, 5, tokens)
+        assert lost2 == lost
+        assert (plain - h_out).abs().max().item() <= U.TOL_BF16 * upd
 
 
 @pytest.mark.parametrize("name,steps,sample,permille", [

@@ -464,6 +464,57 @@ halo_status halo_set_option(const char* name, int value);
  * 6 next input ready; 7 = duration of the selection (selecting thread block only).  n_blocks = 0 turns it off. */
 halo_status halo_stack_set_trace(halo_stack* stack, unsigned long long* trace /*device*/, int n_blocks);
 int halo_stack_trace_width(const halo_stack* stack);
+/* ------------------------------------------------------------------------
+ * Transformer-block stack: the generation loop over whole layers (Sec. III-B.3, Comp process: "MHA then MLP"; Sec. II-A:
+ * MHA blocks, MLP blocks and the LM head are all collections of neuron groups; the first layer and the LM head are sent
+ * reliably).  Per token at position pos and layer l:
+ *     x_a = cast(rmsnorm(h));  keys / values of ALL heads from x_a appended to layer l's caches at pos (never dropped)
+ *     kept heads  = selection from the MHA predictor of layer l applied to layer l-1's x_a   (arrival draw (step, 2l))
+ *     h += merge(halo_group_mha over the kept heads)
+ *     x_f = cast(rmsnorm(h))
+ *     kept groups = selection from the MLP predictor of layer l applied to layer l-1's x_f   (arrival draw (step, 2l+1))
+ *     h += merge(halo_group_ffn over the kept groups)
+ * Layer 0 keeps every head and group.  After the last layer the LM-head groups (all of them) give the logits of
+ * cast(rmsnorm(h)).  The residual input h_0 of each token is given by the caller (it stands for the embedding of the
+ * previous token).  One launch per step of the path on `stream`, no host synchronisation inside.
+ *   halo_block_weights: host arrays of n_layers device pointers (caller-owned, they must outlive the stack):
+ *     W_ffn packed FFN weights; W_mha packed MHA weights (halo_pack_mha_weights); Wk, Wv [H*head_dim][d];
+ *     W1_ffn / W2_ffn and W1_mha / W2_mha predictor factors (entry 0 unused, may be NULL); K_cache / V_cache
+ *     [H][max_len][head_dim], updated by decode; W_lm [vocab][d] (NULL and lm == NULL: no LM head).
+ *   plan_ffn over the FFN groups, plan_mha over the heads (n_groups = n_heads).
+ *   halo_block_stack_decode: h0 device fp32 [steps][d]; token s sits at position pos0 + s (pos0 + steps <= max_len)
+ *     and draws arrivals with counter step0 + s; logits device fp32 [steps][vocab] or NULL; h_out device fp32
+ *     [steps][d] or NULL; taps: NULL or records per (step, layer) of either block type (layout of halo_taps with
+ *     n_tok = 1; for the MHA block G = n_heads).
+ * ---------------------------------------------------------------------- */
+typedef struct halo_block_stack halo_block_stack;
+typedef struct {
+    const void* const* W_ffn;
+    const void* const* W_mha;
+    const void* const* Wk;
+    const void* const* Wv;
+    const void* const* W1_ffn;
+    const void* const* W2_ffn;
+    const void* const* W1_mha;
+    const void* const* W2_mha;
+    void* const* K_cache;
+    void* const* V_cache;
+    const void* W_lm;
+} halo_block_weights;
+typedef struct {
+    halo_taps mha;
+    halo_taps ffn;
+} halo_block_taps;
+halo_status halo_block_stack_create(halo_block_stack** out, const halo_ffn_shape* ffn, const halo_mha_shape* mha,
+                                    const halo_lm_shape* lm, const halo_pred_shape* pred_ffn,
+                                    const halo_pred_shape* pred_mha, int n_layers, const halo_plan* plan_ffn,
+                                    const halo_plan* plan_mha, const halo_block_weights* weights);
+halo_status halo_block_stack_destroy(halo_block_stack* stack);
+halo_status halo_block_stack_decode(halo_block_stack* stack, const float* h0, int steps, int pos0, uint32_t step0,
+                                    float* logits, float* h_out, const halo_block_taps* taps, void* stream);
+halo_status halo_block_stack_status(halo_block_stack* stack, uint32_t* dev_status_value /*host*/, void* stream);
+long long halo_block_stack_last_launches(const halo_block_stack* stack);
+
 /* Failure detection self-test.  Every device-side wait of this library (mbarrier phases of the copy rings, the
  * grid barrier, the published-selection flag) is bounded; when one runs out the kernel raises HALO_DEV_TIMEOUT
  * and returns, so a late or missing partner shows up as a status bit, never as a hung GPU (the paper's master

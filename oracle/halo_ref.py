@@ -397,3 +397,53 @@ def group_lm_head(W: np.ndarray, x: np.ndarray, group_size: int, group_list=None
     _check(lib().halo_ref_group_lm_head(c_int(d), c_int(vocab), c_int(group_size), c_int(dt), _p(W), _p(x2),
                                         c_int(n_tok), _p(lst), c_int(len(lst)), _p(out)), "group_lm_head")
     return out
+
+
+# --- a transformer-block stack: MHA groups, then FFN groups, per layer; LM-head groups at the end --------------
+
+def block_stack_token(h0, pos, step, blocks, lm_W, lm_group_size, plan_mha, plan_ffn, dtype, act=ACT_RELU):
+    """One token through L transformer blocks the way the generation phase runs them (Sec. III-B.3: in every layer
+    the MHA block and then the MLP block, each with its own predictor fed one layer ahead; the first layer and the LM
+    head are sent reliably).  Free running, every step by the functions above, nothing fused:
+
+        for layer l:   x_a = cast(rmsnorm(h));  K, V caches of layer l get the keys / values of x_a at `pos`
+                       heads kept = select(predict(mha predictor of l, x_a of layer l-1)), arrival draw (step, 2l)
+                       h += merge(group_mha(kept heads))
+                       x_f = cast(rmsnorm(h))
+                       groups kept = select(predict(ffn predictor of l, x_f of layer l-1)), arrival draw (step, 2l+1)
+                       h += merge(group_ffn(kept groups))
+        logits = LM-head groups (all of them) on cast(rmsnorm(h))
+
+    blocks: list of dicts with W_mha (packed [H][2][dh][d]), Wk, Wv, K, V (caches, updated in place), W_ffn (packed),
+    and for l >= 1 the predictor factors W1_mha, W2_mha, W1_ffn, W2_ffn.  plan_*: dict(loss_rate, share_weight, mode,
+    k, threshold, seed).  Returns (h, logits or None, records per layer)."""
+    h = np.asarray(h0, dtype=np.float64).reshape(1, -1)
+    recs = []
+    xa_prev = xf_prev = None
+    for l, b in enumerate(blocks):
+        H = b["W_mha"].shape[0]
+        G = b["W_ffn"].shape[0]
+        _, x_a = glue(h, None, dtype)
+        mha_kv_append(b["Wk"], b["Wv"], x_a[0], pos, b["K"], b["V"])
+        s_a = np.zeros(H, dtype=np.float32) if l == 0 else predict(b["W1_mha"], b["W2_mha"], xa_prev, act=act)
+        sel_a = select(s_a, plan_mha["loss_rate"], plan_mha["share_weight"], plan_mha["mode"], plan_mha["k"],
+                       plan_mha["threshold"], plan_mha["seed"], step, 2 * l, force_all=(l == 0))
+        n_a = len(plan_mha["loss_rate"])
+        P_a = group_mha(b["W_mha"], x_a[0], b["K"], b["V"], pos, sel_a["keep_list"][: sel_a["n_keep"]],
+                        sel_a["dev_of_group"], n_a)
+        y_a = merge(P_a[:, None, :])
+        h, x_f = glue(h, y_a, dtype)
+        s_f = np.zeros(G, dtype=np.float32) if l == 0 else predict(b["W1_ffn"], b["W2_ffn"], xf_prev, act=act)
+        sel_f = select(s_f, plan_ffn["loss_rate"], plan_ffn["share_weight"], plan_ffn["mode"], plan_ffn["k"],
+                       plan_ffn["threshold"], plan_ffn["seed"], step, 2 * l + 1, force_all=(l == 0))
+        n_f = len(plan_ffn["loss_rate"])
+        P_f = group_ffn(b["W_ffn"], x_f, sel_f["keep_list"][: sel_f["n_keep"]], sel_f["dev_of_group"], n_f)
+        y_f = merge(P_f)
+        h = h + y_f
+        recs.append(dict(x_a=x_a, x_f=x_f, scores_a=s_a, scores_f=s_f, sel_a=sel_a, sel_f=sel_f, y_a=y_a, y_f=y_f))
+        xa_prev, xf_prev = x_a, x_f
+    logits = None
+    if lm_W is not None:
+        _, x_o = glue(h, None, dtype)
+        logits = group_lm_head(lm_W, x_o, lm_group_size)
+    return h, logits, recs

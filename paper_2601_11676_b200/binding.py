@@ -34,6 +34,8 @@ EXPORTS = [
     "halo_layer_workspace_bytes", "halo_layer_fused", "halo_read_status",
     "halo_pack_mha_weights", "halo_mha_kv_append", "halo_group_mha_workspace_bytes", "halo_group_mha",
     "halo_group_lm_head", "halo_late_devices", "halo_quantize_weights_i4", "halo_group_ffn_i4", "halo_set_option",
+    "halo_block_stack_create", "halo_block_stack_destroy", "halo_block_stack_decode", "halo_block_stack_status",
+    "halo_block_stack_last_launches",
 ]
 
 
@@ -56,6 +58,15 @@ class LmShape(Structure):
 class Taps(Structure):
     _fields_ = [("x", c_void_p), ("scores", c_void_p), ("dev_of_group", c_void_p), ("arrived", c_void_p),
                 ("keep_list", c_void_p), ("n_keep", c_void_p), ("y", c_void_p)]
+
+
+class BlockWeights(Structure):
+    _fields_ = [(n, POINTER(c_void_p)) for n in ("W_ffn", "W_mha", "Wk", "Wv", "W1_ffn", "W2_ffn", "W1_mha", "W2_mha",
+                                                  "K_cache", "V_cache")] + [("W_lm", c_void_p)]
+
+
+class BlockTaps(Structure):
+    _fields_ = [("mha", Taps), ("ffn", Taps)]
 
 
 class HaloError(RuntimeError):
@@ -136,6 +147,15 @@ def lib() -> ctypes.CDLL:
         L.halo_selftest_bounded_wait.argtypes = [c_void_p, c_longlong, c_void_p, c_void_p, c_void_p]
         L.halo_status_message.argtypes = [c_uint32, c_char_p, c_int]
         L.halo_set_option.argtypes = [c_char_p, c_int]
+        L.halo_block_stack_create.argtypes = [POINTER(c_void_p), POINTER(FfnShape), POINTER(MhaShape), POINTER(LmShape),
+                                              POINTER(PredShape), POINTER(PredShape), c_int, c_void_p, c_void_p,
+                                              POINTER(BlockWeights)]
+        L.halo_block_stack_destroy.argtypes = [c_void_p]
+        L.halo_block_stack_decode.argtypes = [c_void_p, c_void_p, c_int, c_int, c_uint32, c_void_p, c_void_p,
+                                              POINTER(BlockTaps), c_void_p]
+        L.halo_block_stack_status.argtypes = [c_void_p, POINTER(c_uint32), c_void_p]
+        L.halo_block_stack_last_launches.argtypes = [c_void_p]
+        L.halo_block_stack_last_launches.restype = c_longlong
         _lib = L
     return _lib
 
@@ -446,6 +466,53 @@ class Stack:
     def close(self):
         if self.handle:
             lib().halo_stack_destroy(self.handle)
+            self.handle = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class BlockStack:
+    """halo_block_stack_create / _decode / _destroy.  Keeps the weight and cache tensors alive.
+    blocks: list of dicts with W_ffn, W_mha, Wk, Wv, K, V and (from the second layer on) W1_ffn, W2_ffn, W1_mha, W2_mha."""
+
+    def __init__(self, ffn: FfnShape, mha: MhaShape, lm, pred_ffn: PredShape, pred_mha: PredShape, plan_ffn: Plan,
+                 plan_mha: Plan, blocks, W_lm=None):
+        L = len(blocks)
+        self._keep = (blocks, W_lm, plan_ffn, plan_mha)
+        self.n_layers = L
+        arr = lambda key: (c_void_p * L)(*[(b[key].data_ptr() if b.get(key) is not None else None) for b in blocks])
+        self._arrays = {k: arr(k) for k in ("W_ffn", "W_mha", "Wk", "Wv", "W1_ffn", "W2_ffn", "W1_mha", "W2_mha", "K", "V")}
+        w = BlockWeights()
+        for k in ("W_ffn", "W_mha", "Wk", "Wv", "W1_ffn", "W2_ffn", "W1_mha", "W2_mha"):
+            setattr(w, k, ctypes.cast(self._arrays[k], POINTER(c_void_p)))
+        w.K_cache = ctypes.cast(self._arrays["K"], POINTER(c_void_p))
+        w.V_cache = ctypes.cast(self._arrays["V"], POINTER(c_void_p))
+        w.W_lm = c_void_p(W_lm.data_ptr()) if W_lm is not None else None
+        self.handle = c_void_p()
+        _chk(lib().halo_block_stack_create(byref(self.handle), byref(ffn), byref(mha), byref(lm) if lm is not None else None,
+                                           byref(pred_ffn), byref(pred_mha), L, plan_ffn.handle, plan_mha.handle, byref(w)),
+             "halo_block_stack_create")
+
+    def decode(self, h0, steps, pos0, step0, logits=None, h_out=None, taps: BlockTaps | None = None, stream=None) -> None:
+        _chk(lib().halo_block_stack_decode(self.handle, _ptr(h0), steps, pos0, step0, _ptr(logits), _ptr(h_out),
+                                           byref(taps) if taps is not None else None, _stream(stream)),
+             "halo_block_stack_decode")
+
+    def status(self, stream=None) -> int:
+        v = c_uint32(0)
+        _chk(lib().halo_block_stack_status(self.handle, byref(v), _stream(stream)), "halo_block_stack_status")
+        return int(v.value)
+
+    def last_launches(self) -> int:
+        return int(lib().halo_block_stack_last_launches(self.handle))
+
+    def close(self):
+        if self.handle:
+            lib().halo_block_stack_destroy(self.handle)
             self.handle = c_void_p()
 
     def __del__(self):

@@ -310,6 +310,8 @@ def run_halo(args, rank, world, local_rank):
                                      ("llama2-13b-decode", "tinyllama-1.1b-decode", "llama2-7b-decode")
                                      if n != wl.name]
         result["other_blocks"] = other_blocks_report(dev, peak)
+        result["int4_stack"] = int4_stack_report(dev, peak)
+        result["block_stack"] = block_stack_report(dev, peak)
         result["keep_sweep"] = keep_sweep(dev, peak)
         result["overlap_ablation"] = overlap_ablation(dev)
     if world == 1 and not args.no_cpu_baseline:
@@ -491,6 +493,111 @@ def overlap_ablation(dev, steps=48, warm=4):
         del stack, Wp, preds
         torch.cuda.empty_cache()
     return out
+
+
+def int4_stack_report(dev, peak, steps=32, warm=4):
+    """The 7B-shaped FFN stack on int4 group-quantised weights (the paper's models are 4-bit): tokens/s and GB/s over the
+    int4 bytes of the kept groups (codes + scales) and the predictors.  One launch per step of the path."""
+    from paper_2601_11676_b200 import binding as B
+    wl = synth.workload("llama2-7b-decode")
+    L, G, S, d = wl.n_layers, wl.n_groups, wl.group_size, wl.d_model
+    fsh = B.ffn_shape(d, wl.d_ffn, S, B.BF16)
+    Q, Sc = [], []
+    for l in range(L):
+        Wf = synth.packed_layer(wl, l, dev)
+        q = torch.empty((G, 3, S, d // 2), dtype=torch.uint8, device=dev)
+        sc = torch.empty((G, 3, S, d // 128), dtype=torch.bfloat16, device=dev)
+        B.halo_quantize_weights_i4(fsh, Wf, q, sc)
+        torch.cuda.synchronize()
+        Q.append(q); Sc.append(sc)
+        del Wf
+    preds = [synth.predictor(wl, l, dev) for l in range(L)]
+    plan = B.Plan(G, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
+    stack = B.Stack(fsh, B.pred_shape(d, wl.pred_rank, G, B.BF16), 1, plan, Q, [p[0] for p in preds], [p[1] for p in preds],
+                    i4_scales=Sc)
+    ms, kept = _timed_decode(stack, wl, dev, steps, warm)
+    group_bytes_i4 = 3 * S * (d // 2 + (d // 128) * 2)
+    byts = kept * group_bytes_i4 + steps * (L - 1) * wl.pred_bytes
+    gbs = byts / (ms * 1e-3) / 1e9
+    res = {"workload": "llama2-7b-decode on int4 weights (one bf16 scale per 128 elements)", "steps": steps,
+           "tokens_per_s": steps / (ms * 1e-3), "ms_per_token": ms / steps,
+           "kept_fraction": kept / float(steps * L * G), "achieved_gbs": gbs, "frac_of_peak": gbs / peak,
+           "bf16_equivalent_gbs": (kept * wl.group_bytes + steps * (L - 1) * wl.pred_bytes) / (ms * 1e-3) / 1e9,
+           "weights_gb": L * G * group_bytes_i4 / 1e9, "gpu_launches_per_token": stack.last_launches() / steps,
+           "device_status": stack.status()}
+    stack.close()
+    return res
+
+
+def block_stack_report(dev, peak, steps=24, warm=4, context=1024):
+    """The paper's generation loop over whole layers at the 7B shape: per layer the MHA block (keys / values of all 32
+    heads appended, kept heads attend over `context` cached positions) and the MLP block, each with its predictor,
+    selection and merge, and the LM-head groups at the end (32000 x 4096).  One launch per step of the path.
+    Bytes: kept FFN groups + kept heads' query / output rows + K/V projections + K/V cache rows read + predictors +
+    LM head."""
+    from paper_2601_11676_b200 import binding as B
+    wl = synth.workload("llama2-7b-decode")
+    L, d, G, H, dh, vocab, r_mha = wl.n_layers, wl.d_model, wl.n_groups, 32, 128, 32000, 64
+    max_len = context + warm + steps + 1
+    mh = B.mha_shape(d, H, dh, max_len, B.BF16)
+    mw = synth.Workload("mha-pred", L, d, H * 8, 8, r_mha, "bf16", (), (), 500, 1, seed=wl.seed + 1)
+    blocks = []
+    g = torch.Generator(device=dev).manual_seed(5)
+    for l in range(L):
+        Wq, Wk, Wv, Wo = synth.mha_matrices(wl, l, H, dev)
+        Wp = torch.empty((H, 2, dh, d), dtype=torch.bfloat16, device=dev)
+        B.halo_pack_mha_weights(mh, Wq, Wo, Wp)
+        torch.cuda.synchronize()
+        del Wq, Wo
+        K = torch.zeros((H, max_len, dh), dtype=torch.bfloat16, device=dev)
+        V = torch.zeros((H, max_len, dh), dtype=torch.bfloat16, device=dev)
+        K[:, :context] = torch.randn((H, context, dh), generator=g, device=dev).to(torch.bfloat16)
+        V[:, :context] = torch.randn((H, context, dh), generator=g, device=dev).to(torch.bfloat16)
+        blk = dict(W_ffn=synth.packed_layer(wl, l, dev), W_mha=Wp, Wk=Wk, Wv=Wv, K=K, V=V)
+        if l > 0:
+            blk["W1_ffn"], blk["W2_ffn"] = synth.predictor(wl, l, dev)
+            blk["W1_mha"], blk["W2_mha"] = synth.predictor(mw, l, dev)
+        blocks.append(blk)
+    gc = torch.Generator(device="cpu").manual_seed(17)
+    W_lm = (torch.randn((vocab, d), generator=gc) / 64).to(torch.bfloat16).to(dev)
+    plan_f = B.Plan(G, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
+    plan_a = B.Plan(H, wl.loss_rate, wl.share_weight, B.SEL_TOPK, H // 2, 0.0, wl.seed + 1)
+    stack = B.BlockStack(B.ffn_shape(d, wl.d_ffn, wl.group_size, B.BF16), mh, B.lm_shape(d, vocab, 256, B.BF16),
+                         B.pred_shape(d, wl.pred_rank, G, B.BF16), B.pred_shape(d, r_mha, H, B.BF16), plan_f, plan_a,
+                         blocks, W_lm)
+    total = warm + steps
+    h0 = torch.stack([synth.stream_input(wl, 500 + s, dev)[0] for s in range(total)])
+    logits = torch.empty((total, vocab), dtype=torch.float32, device=dev)
+    nk_a = torch.zeros((total, L), dtype=torch.int32, device=dev)
+    nk_f = torch.zeros((total, L), dtype=torch.int32, device=dev)
+    taps = B.BlockTaps(B.Taps(None, None, None, None, None, nk_a.data_ptr(), None),
+                       B.Taps(None, None, None, None, None, nk_f.data_ptr(), None))
+    stack.decode(h0, total, context, 0, logits, None, taps)          # records the kept sets; also the warm-up
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(3):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        stack.decode(h0[warm:], steps, context + warm, warm, logits[warm:])
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    ms = sorted(ts)[1]
+    kept_f, kept_a = int(nk_f[warm:].sum().item()), int(nk_a[warm:].sum().item())
+    pos_sum = sum(context + warm + s + 1 for s in range(steps))
+    byts = (kept_f * wl.group_bytes + steps * (L - 1) * (wl.pred_bytes + (d * r_mha + r_mha * H) * 2)
+            + steps * L * 2 * d * d * 2 + kept_a * 2 * dh * d * 2
+            + sum(int(nk_a[warm + s].sum().item()) * 2 * (context + warm + s + 1) * dh * 2 for s in range(steps))
+            + steps * vocab * d * 2)
+    gbs = byts / (ms * 1e-3) / 1e9
+    res = {"shape": "32 layers x (32 heads of 128 + 86 FFN groups of 128), d 4096, %d cached positions, LM head 32000" % context,
+           "steps": steps, "tokens_per_s": steps / (ms * 1e-3), "ms_per_token": ms / steps,
+           "kept_fraction_ffn": kept_f / float(steps * L * G), "kept_fraction_heads": kept_a / float(steps * L * H),
+           "algorithmic_gb_per_token": byts / steps / 1e9, "achieved_gbs": gbs, "frac_of_peak": gbs / peak,
+           "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS, "gpu_launches_per_token": stack.last_launches() / steps,
+           "device_status": stack.status()}
+    stack.close()
+    return res
 
 
 def decode_brief(name, dev, peak, steps=64, warm=4):

@@ -399,6 +399,12 @@ typedef struct {
 halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred,
                               int n_layers, int n_tok, const halo_plan* plan, const void* const* W_packed,
                               const void* const* W1, const void* const* W2);
+/* The same stack on int4 group-quantised FFN weights (Sec. IV-A: the evaluated models are 4-bit): Q[L] and scales[L]
+ * as written by halo_quantize_weights_i4 for every block; activations, predictor and everything else as above
+ * (ffn->wdtype must be HALO_BF16, d_model % 128 == 0).  Runs one launch per step of the path. */
+halo_status halo_stack_create_i4(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred,
+                                 int n_layers, int n_tok, const halo_plan* plan, const void* const* Q,
+                                 const void* const* scales, const void* const* W1, const void* const* W2);
 halo_status halo_stack_destroy(halo_stack* stack);
 /* Runs `steps` tokens (or prompts of n_tok tokens) through the stack.
  *   h0    device fp32 [steps][n_tok][d]: residual-stream input of each step
@@ -454,7 +460,8 @@ halo_status halo_stack_set_mode(halo_stack* stack, int mode);
  *   "prefill_kcuts" (1..16), "prefill_kratio_percent" (30..100)   prompt FFN: K runs per down-projection tile and
  *                                     the ratio between consecutive runs
  *   "mha_three_launches" (0/1)        halo_group_mha as three launches instead of one
- *   "i4_no_ring" (0/1)                halo_group_ffn_i4 on plain loads instead of the shared-memory ring
+ *   "i4_no_ring" (0/1/3)              halo_group_ffn_i4: 0 shared-memory ring (default), 1 plain loads, 3 ring with
+ *                                     the products on the legacy tensor-core path (mma.sync; slower here)
  * HALO_ERR_ARG for an unknown name or a value outside the stated range. */
 halo_status halo_set_option(const char* name, int value);
 /* Tracing of the persistent kernel (timing statistics of the generation loop): the caller gives a device

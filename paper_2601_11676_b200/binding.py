@@ -35,7 +35,7 @@ EXPORTS = [
     "halo_pack_mha_weights", "halo_mha_kv_append", "halo_group_mha_workspace_bytes", "halo_group_mha",
     "halo_group_lm_head", "halo_late_devices", "halo_quantize_weights_i4", "halo_group_ffn_i4", "halo_set_option",
     "halo_block_stack_create", "halo_block_stack_destroy", "halo_block_stack_decode", "halo_block_stack_status",
-    "halo_block_stack_last_launches",
+    "halo_block_stack_last_launches", "halo_stack_create_i4",
 ]
 
 
@@ -110,6 +110,9 @@ def lib() -> ctypes.CDLL:
         L.halo_glue.argtypes = [c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         L.halo_stack_create.argtypes = [POINTER(c_void_p), POINTER(FfnShape), POINTER(PredShape), c_int, c_int,
                                         c_void_p, POINTER(c_void_p), POINTER(c_void_p), POINTER(c_void_p)]
+        L.halo_stack_create_i4.argtypes = [POINTER(c_void_p), POINTER(FfnShape), POINTER(PredShape), c_int, c_int,
+                                           c_void_p, POINTER(c_void_p), POINTER(c_void_p), POINTER(c_void_p),
+                                           POINTER(c_void_p)]
         L.halo_stack_destroy.argtypes = [c_void_p]
         L.halo_stack_decode.argtypes = [c_void_p, c_void_p, c_int, c_uint32, c_void_p, POINTER(Taps), c_void_p]
         L.halo_stack_decode_host.argtypes = [c_void_p, c_void_p, c_int, c_uint32, c_void_p, c_void_p]
@@ -426,14 +429,19 @@ def halo_glue(d_model, n_tok, xdtype, h, y, h_out, x_out, stream=None) -> None:
 class Stack:
     """halo_stack_create / halo_stack_decode / halo_stack_destroy.  Keeps the weight tensors alive."""
 
-    def __init__(self, ffn: FfnShape, pred: PredShape, n_tok: int, plan: Plan, W_packed, W1, W2):
+    def __init__(self, ffn: FfnShape, pred: PredShape, n_tok: int, plan: Plan, W_packed, W1, W2, i4_scales=None):
+        """i4_scales given: W_packed holds the int4 codes of halo_quantize_weights_i4 (halo_stack_create_i4)."""
         L = len(W_packed)
-        self._keep = (list(W_packed), list(W1), list(W2), plan)
+        self._keep = (list(W_packed), list(W1), list(W2), plan, list(i4_scales) if i4_scales is not None else None)
         self.ffn, self.pred, self.n_layers, self.n_tok, self.plan = ffn, pred, L, n_tok, plan
         arr = lambda ts: (c_void_p * L)(*[(t.data_ptr() if t is not None else None) for t in ts])
         self.handle = c_void_p()
-        _chk(lib().halo_stack_create(byref(self.handle), byref(ffn), byref(pred), L, n_tok, plan.handle,
-                                     arr(W_packed), arr(W1), arr(W2)), "halo_stack_create")
+        if i4_scales is not None:
+            _chk(lib().halo_stack_create_i4(byref(self.handle), byref(ffn), byref(pred), L, n_tok, plan.handle,
+                                            arr(W_packed), arr(i4_scales), arr(W1), arr(W2)), "halo_stack_create_i4")
+        else:
+            _chk(lib().halo_stack_create(byref(self.handle), byref(ffn), byref(pred), L, n_tok, plan.handle,
+                                         arr(W_packed), arr(W1), arr(W2)), "halo_stack_create")
 
     def decode(self, h0, steps, step0, h_out, taps: Taps | None = None, stream=None) -> None:
         _chk(lib().halo_stack_decode(self.handle, _ptr(h0), steps, step0, _ptr(h_out),

@@ -64,7 +64,7 @@ const OptionName kOptionNames[] = {
     {"prefill_kcuts", OPT_PREFILL_KCUTS, 1, 16},
     {"prefill_kratio_percent", OPT_PREFILL_KRATIO_PERCENT, 30, 100},
     {"mha_three_launches", OPT_MHA_THREE_LAUNCHES, 0, 1},
-    {"i4_no_ring", OPT_I4_NO_RING, 0, 1},
+    {"i4_no_ring", OPT_I4_NO_RING, 0, 3},
     {"prompt_kcuts", OPT_PROMPT_KCUTS, 1, 16},
     {"prompt_l2_ahead", OPT_PROMPT_L2_AHEAD, 0, 32},
 };
@@ -446,6 +446,7 @@ struct halo_stack {
     int n_layers, n_tok, G, n_dev;
     halo_plan plan;
     std::vector<const void*> W, W1, W2;
+    std::vector<const void*> i4_scales;   // non-empty: W holds int4 codes (halo_quantize_weights_i4)
     void* slab;
     // carved from the slab
     float* h;
@@ -502,9 +503,33 @@ struct halo_stack {
     unsigned long long* pp_trace = nullptr;   // caller-owned, optional
 };
 
+namespace {
+halo_status stack_create_impl(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred, int n_layers,
+                              int n_tok, const halo_plan* plan, const void* const* W_packed, const void* const* i4_scales,
+                              const void* const* W1, const void* const* W2);
+}  // namespace
+
 extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred,
                                          int n_layers, int n_tok, const halo_plan* plan, const void* const* W_packed,
                                          const void* const* W1, const void* const* W2) {
+    return stack_create_impl(out, ffn, pred, n_layers, n_tok, plan, W_packed, nullptr, W1, W2);
+}
+
+extern "C" halo_status halo_stack_create_i4(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred,
+                                            int n_layers, int n_tok, const halo_plan* plan, const void* const* Q,
+                                            const void* const* scales, const void* const* W1, const void* const* W2) {
+    if (!scales || !ffn) return HALO_ERR_ARG;
+    if (ffn->wdtype != HALO_BF16) return HALO_ERR_DTYPE;          // activations and predictor stay bf16
+    if (ffn->d_model % 128 != 0) return HALO_ERR_SHAPE;
+    for (int l = 0; l < n_layers; ++l)
+        if (!scales[l] || !aligned16(scales[l])) return scales[l] ? HALO_ERR_ALIGN : HALO_ERR_ARG;
+    return stack_create_impl(out, ffn, pred, n_layers, n_tok, plan, Q, scales, W1, W2);
+}
+
+namespace {
+halo_status stack_create_impl(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred, int n_layers,
+                              int n_tok, const halo_plan* plan, const void* const* W_packed, const void* const* i4_scales,
+                              const void* const* W1, const void* const* W2) {
     if (!out) return HALO_ERR_ARG;
     *out = nullptr;
     halo_status rc = check_ffn_shape(ffn);
@@ -533,6 +558,7 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     s->W.assign(W_packed, W_packed + n_layers);
     s->W1.assign(W1, W1 + n_layers);
     s->W2.assign(W2, W2 + n_layers);
+    if (i4_scales) s->i4_scales.assign(i4_scales, i4_scales + n_layers);
     s->last_launches = 0;
 
     const size_t d = ffn->d_model, es = elem_size(ffn->wdtype), T = n_tok;
@@ -559,7 +585,7 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     constexpr size_t kMaxGrid = 192;   // thread blocks of the persistent kernel (one per SM)
     const size_t o_xh = carve(2 * d * 2);
     const size_t o_dr = carve(persistent_supported(*ffn, n_tok, G) ? sizeof(float) * 2 * kMaxGrid * d : 16);
-    const size_t ws_bytes = prefill_supported(*ffn, n_tok) ? prefill_workspace_bytes(*ffn, n_tok) : 0;
+    const size_t ws_bytes = (!i4_scales && prefill_supported(*ffn, n_tok)) ? prefill_workspace_bytes(*ffn, n_tok) : 0;
     const size_t o_ws = carve(ws_bytes ? ws_bytes : 16);
     const size_t o_sc2 = carve(sizeof(float) * G), o_dg2 = carve(sizeof(int32_t) * G);
     const size_t o_ar2 = carve(HALO_MAX_DEVICES), o_kl2 = carve(sizeof(int32_t) * G), o_nk2 = carve(sizeof(int32_t));
@@ -596,7 +622,7 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     s->set_kl[0] = s->keep_list; s->set_kl[1] = reinterpret_cast<int32_t*>(base + o_kl2);
     s->set_nk[0] = s->n_keep; s->set_nk[1] = reinterpret_cast<int32_t*>(base + o_nk2);
     s->side = nullptr; s->ev_x = nullptr; s->ev_sel = nullptr;
-    if (n_tok > 1) {
+    if (n_tok > 1 && !i4_scales) {
         // best effort: without them the blocks simply run one after the other on the caller's stream
         // highest priority: the short predictor/selection kernels of the next block must get SMs as they free up,
         // ahead of the waiting CTAs of the long FFN launch (which pulls its tiles from a queue and loses nothing)
@@ -617,7 +643,7 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     if (option_value(OPT_CROSS_STAGES) >= 0) s->cross_stages = option_value(OPT_CROSS_STAGES);
     s->max_steps_per_launch = std::max(0, option_value(OPT_MAX_STEPS_PER_LAUNCH));
     if (option_value(OPT_L2_AHEAD) >= 0) s->l2_ahead = option_value(OPT_L2_AHEAD);
-    s->persistent_ok = persistent_supported(*ffn, n_tok, G);
+    s->persistent_ok = !i4_scales && persistent_supported(*ffn, n_tok, G);
     {
         // pointer tables, and the first block's selection: reliable block, all scores equal -> the priority
         // order is the group order, everything is kept (Sec. III-B.3, first layer)
@@ -640,7 +666,7 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
         ok = ok && cudaMemcpy(s->d_W1, s->W1.data(), sizeof(void*) * n_layers, cudaMemcpyHostToDevice) == cudaSuccess;
         ok = ok && cudaMemcpy(s->d_W2, s->W2.data(), sizeof(void*) * n_layers, cudaMemcpyHostToDevice) == cudaSuccess;
         if (!ok) { cudaFree(s->slab); delete s; return HALO_ERR_CUDA; }
-        if (n_tok > 1 && prompt_stack_supported(*ffn, *pred, n_layers, n_tok)) {
+        if (n_tok > 1 && !i4_scales && prompt_stack_supported(*ffn, *pred, n_layers, n_tok)) {
             // persistent prompt kernel: tensor maps (encoded once, here), two H buffers, control words, one selection
             // record per block.  Any failure in here only means that prompts run one launch per step of the path.
             const int S = ffn->group_size, NS = std::min(S, 128), dm = ffn->d_model;
@@ -698,6 +724,7 @@ extern "C" halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape*
     *out = s;
     return HALO_OK;
 }
+}  // namespace
 
 extern "C" halo_status halo_stack_destroy(halo_stack* s) {
     if (!s) return HALO_OK;
@@ -1001,8 +1028,14 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                 if (taps->n_keep) HALO_COPY(taps->n_keep + rec, s->n_keep, sizeof(int32_t));
                 if (taps->y) y_tap = taps->y + rec * step_elems;
             }
-            HALO_TRY(dispatch_group_ffn(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->keep_list, s->n_keep,
-                                        s->dev_of_group, n_dev, s->partials, s->ffn_ws, s->status, st));
+            if (!s->i4_scales.empty()) {
+                HALO_TRY(halo_group_ffn_i4(&s->ffn, s->W[l], s->i4_scales[l], x_cur, static_cast<int>(T), s->keep_list,
+                                           s->n_keep, s->dev_of_group, n_dev, s->partials, s->status, stream));
+                ++launches;
+            } else {
+                HALO_TRY(dispatch_group_ffn(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->keep_list, s->n_keep,
+                                            s->dev_of_group, n_dev, s->partials, s->ffn_ws, s->status, st));
+            }
             ++launches;
             float* h_dst = (l == L - 1) ? h_out + sidx * step_elems : s->h;
             HALO_TRY(launch_merge_glue(s->partials, s->arrived, n_dev, static_cast<int>(T), static_cast<int>(d),

@@ -504,6 +504,282 @@ group_ffn_i4_ring_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, con
     if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
 }
 
+// ------------------------------------------------------------------------------------------------------------
+// Ring form with the products on the tensor cores (mma.sync m16n8k16, bf16 x bf16 -> fp32); an option, not the default
+// (see the dispatch below for the measurement).  The plain ring kernel is bound by instruction issue: every weight
+// costs a mask-and-bias plus a multiply-add on the CUDA cores.  Here the CUDA cores only turn nibbles into bf16
+// numbers (128 + nibble, one shift and one logic instruction per pair) and the multiply-adds of 256 weights go into
+// one warp-wide MMA.  A batch is 8 neurons: its 8 gate rows and 8 up rows are the 16 rows of the A operand.
+//   phase 1  warp w owns a slice of d/16 input elements.  Thread (g = lane / 4, t = lane % 4) takes word t of each
+//            16-byte chunk of rows g (gate) and 8 + g (up): a word's nibbles k and k + 4 form one register pair, so
+//            the K order of an MMA is "pairs (k, k + 4)"; x is laid out in the same pairing and sits in column 0 of
+//            the B operand.  After the 8 MMAs of a 128-element block the accumulator of a row is corrected by the
+//            offset (136 x the plain sum of x over the block) and scaled by the row's block scale.
+//   phase 2  y[c] = sum_j f_j * (nibble_j[c] - 8), f_j = silu(a_j) * b_j * scale_j: the M dimension is 16 columns,
+//            the K dimension the 8 neurons (K slots 8..15 are zero).  Thread (g, t) takes word g of a 64-column
+//            group from rows 2t and 2t + 1 and pairs the two rows' nibbles column by column (one byte permutation per
+//            column); f is split into a bf16 high and low part that sit in columns 0 and 1 of B, so nothing is lost
+//            to bf16 rounding.  The column sums stay in the MMA accumulators across batches.
+// Rows are staged with a pitch of (d/2 + 16) bytes so that the word loads above are free of bank conflicts.
+// ------------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void mma_16816_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+struct MmaRingHeader {
+    uint64_t full[8];
+    uint64_t empty[8];
+    int slot[8];
+    int abort_flag;
+    int pad[3];
+    __align__(16) float red[3][2 * kRingNB];     // gate / up sums of the batch, by batch number modulo 3
+};
+
+// KG = 64-column groups per warp in phase 2 = d / 1024.  512 threads, no producer warp: with 17 warps one of the four
+// register files of an SM would hold five warps and cap every thread at 96 registers, too few for the 64 accumulator
+// registers of phase 2.  Instead, right after the barrier between the two phases of batch `it` (every warp is then
+// done with batch it-1), lane 0 of every warp issues one or two of the copies of batch it + STAGES - 1 into the stage
+// batch it-1 occupied.
+template <int KG, int STAGES>
+__global__ void __launch_bounds__(kRingConsumers, 1)
+group_ffn_i4_mma_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, const __nv_bfloat16* __restrict__ scales,
+                        const __nv_bfloat16* __restrict__ x_all, const int32_t* __restrict__ keep_list,
+                        const int32_t* __restrict__ n_keep_ptr, const int32_t* __restrict__ dev_of_group, int n_dev,
+                        int n_tok, float* __restrict__ partials, uint32_t* dev_status) {
+    constexpr int NB = kRingNB;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    MmaRingHeader& hd = *reinterpret_cast<MmaRingHeader*>(smem_raw);
+    const int chunks16 = d / 32, nb = d / kQBlock;
+    const uint32_t row_bytes = static_cast<uint32_t>(d) / 2u;
+    const uint32_t pitch = row_bytes + 16u;
+    const uint32_t sc_bytes = static_cast<uint32_t>(nb) * 2u * NB;      // scales of one plane of a batch
+    const uint32_t codes_bytes = 3u * NB * pitch;
+    const uint32_t stage_bytes = codes_bytes + 3u * sc_bytes;
+    uint4* xp = reinterpret_cast<uint4*>(smem_raw + 1024);                                  // [4][chunks16]
+    float* xsum = reinterpret_cast<float*>(smem_raw + 1024 + static_cast<size_t>(d) * 2);   // [nb]: per 128 elements
+    unsigned char* ring = smem_raw + 1024 + static_cast<size_t>(d) * 2 + ((static_cast<size_t>(nb) * 4 + 127) & ~size_t(127));
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tok = blockIdx.y;
+    int nk = *n_keep_ptr;
+    if (nk < 0 || nk > G) {
+        if (tid == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+        nk = nk < 0 ? 0 : G;
+    }
+    const int per_group = S / NB;
+    const long long total = static_cast<long long>(nk) * per_group;
+    const int lo = static_cast<int>(total * blockIdx.x / gridDim.x);
+    const int hi = static_cast<int>(total * (blockIdx.x + 1) / gridDim.x);
+    if (lo >= hi) return;
+    const int n_it = hi - lo;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) mbar_init(&hd.full[s], 1);
+        hd.abort_flag = 0;
+        mbar_fence_init();
+    }
+    if (tid < 3 * 2 * NB) (&hd.red[0][0])[tid] = 0.0f;
+    __syncthreads();
+    volatile int* abort_flag = &hd.abort_flag;
+
+    // Copies of batch `bi` into its stage, shared out over the warps: copy number cp = 0..26 (24 code rows with the
+    // padded pitch, 3 planes of scales) goes to warp cp % 16.  Warp 0 also posts the expected bytes (or marks the
+    // stage as skipped); copies of other warps may complete before that, which the transaction count allows.
+    auto issue_batch = [&](int bi) {
+        if (lane != 0 || bi >= n_it) return;
+        const int s = bi % STAGES;
+        const int b = lo + bi;
+        const int ki = b / per_group, j0 = (b - ki * per_group) * NB;
+        const int gq = keep_list[ki];
+        int slot = 0;
+        bool ok = (gq >= 0 && gq < G);
+        if (ok && dev_of_group) { slot = dev_of_group[gq] + 1; ok = (slot >= 0 && slot <= n_dev); }
+        if (warp == 0) {
+            if (!ok) {
+                flag_status(dev_status, HALO_DEV_BAD_INDEX);
+                hd.slot[s] = -1;
+                mbar_arrive(&hd.full[s]);
+            } else {
+                hd.slot[s] = slot;
+                mbar_arrive_expect_tx(&hd.full[s], 3u * NB * row_bytes + 3u * sc_bytes);
+            }
+        }
+        if (!ok) return;
+        unsigned char* dst = ring + static_cast<size_t>(s) * stage_bytes;
+        const size_t row0 = static_cast<size_t>(gq) * 3 * S + j0;      // row of plane 0; plane p adds p * S
+        for (int cp = warp; cp < 3 * NB + 3; cp += kRingConsumerWarps) {
+            if (cp < 3 * NB) {
+                const int plane = cp / NB, j = cp - plane * NB;
+                bulk_copy_g2s(dst + cp * pitch, Q + (row0 + static_cast<size_t>(plane) * S + j) * row_bytes, row_bytes, &hd.full[s]);
+            } else {
+                const int plane = cp - 3 * NB;
+                bulk_copy_g2s(dst + codes_bytes + plane * sc_bytes, scales + (row0 + static_cast<size_t>(plane) * S) * nb, sc_bytes,
+                              &hd.full[s]);
+            }
+        }
+    };
+    for (int bi = 0; bi < STAGES - 1; ++bi) issue_batch(bi);
+
+    // ---------------- consumers ----------------
+    {   // x in the nibble pairing, and its plain sums per block of 128 elements
+        const uint16_t* xb = reinterpret_cast<const uint16_t*>(x_all + static_cast<size_t>(tok) * d);
+        uint32_t* xp_words = reinterpret_cast<uint32_t*>(xp);
+        for (int i = tid; i < d / 2; i += kRingConsumers) {
+            const int c = i / 16, r = i - c * 16, w = r >> 2, k = r & 3;
+            const uint32_t lo16 = xb[32 * c + 8 * w + k], hi16 = xb[32 * c + 8 * w + k + 4];
+            xp_words[(static_cast<size_t>(w) * chunks16 + c) * 4 + k] = lo16 | (hi16 << 16);
+        }
+        for (int b = tid; b < nb; b += kRingConsumers) {
+            float sx = 0.0f;
+            for (int e = 0; e < kQBlock; ++e) sx += __bfloat162float(x_all[static_cast<size_t>(tok) * d + kQBlock * b + e]);
+            xsum[b] = sx;
+        }
+    }
+    ring_consumer_barrier();
+    const int g = lane >> 2, t = lane & 3;
+    constexpr int CPW_BLOCKS = KG / 2;            // 128-element blocks of the K slice of a warp in phase 1 (d / 16 / 128)
+    static_assert(KG == 2 || KG == 4, "d must be 2048 or 4096");
+    float acc[KG][4][4];                           // phase-2 accumulators: [64-column group][column pair][MMA fragment]
+    float corr[KG];                                // sum of f per 64-column group's scale block (offset correction)
+#pragma unroll
+    for (int q = 0; q < KG; ++q) {
+        corr[q] = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[q][i][e] = 0.0f;
+    }
+    int cur_slot = -1;
+    const size_t slot_stride = static_cast<size_t>(n_tok) * d;
+
+    auto flush = [&](int slot) {
+        float* dst = partials + static_cast<size_t>(slot) * slot_stride + static_cast<size_t>(tok) * d;
+#pragma unroll
+        for (int q = 0; q < KG; ++q) {
+            const float off = kNibbleBias * corr[q];
+            if (t == 0) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    // columns 2i and 2i + 1 of word g of this group: high part (B column 0) + low part (B column 1)
+                    const int col = (warp * KG + q) * 64 + g * 8 + 2 * i;
+                    asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(dst + col),
+                                 "f"(acc[q][i][0] + acc[q][i][1] - off), "f"(acc[q][i][2] + acc[q][i][3] - off)
+                                 : "memory");
+                }
+            }
+            corr[q] = 0.0f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc[q][i][e] = 0.0f;
+        }
+    };
+
+    for (int it = 0; it < n_it; ++it) {
+        const int s = it % STAGES;
+        const uint32_t parity = static_cast<uint32_t>(it / STAGES) & 1u;
+        if (!*abort_flag && !mbar_wait_bounded(&hd.full[s], parity, abort_flag)) *abort_flag = 1;
+        const int slot = *abort_flag ? -1 : hd.slot[s];
+        const unsigned char* stage = ring + static_cast<size_t>(s) * stage_bytes;
+        const __nv_bfloat16* stage_sc = reinterpret_cast<const __nv_bfloat16*>(stage + codes_bytes);   // [3][NB][nb]
+        float* red = hd.red[it % 3];
+        if (slot >= 0) {
+            if (slot != cur_slot) {
+                if (cur_slot >= 0) flush(cur_slot);
+                cur_slot = slot;
+            }
+            // ---- phase 1: this warp's slice of the 16 gate / up rows on the tensor cores ----
+            const unsigned char* row_g = stage + static_cast<size_t>(g) * pitch + t * 4;
+            const unsigned char* row_u = stage + static_cast<size_t>(NB + g) * pitch + t * 4;
+            float a_g = 0.0f, a_u = 0.0f;
+#pragma unroll
+            for (int blk = 0; blk < CPW_BLOCKS; ++blk) {
+                const int block = warp * CPW_BLOCKS + blk;       // 128-element block of the rows
+                float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    const int c = block * 4 + cc;
+                    const uint32_t wg = *reinterpret_cast<const uint32_t*>(row_g + c * 16);
+                    const uint32_t wu = *reinterpret_cast<const uint32_t*>(row_u + c * 16);
+                    uint4 xb = make_uint4(0u, 0u, 0u, 0u);
+                    if (g == 0) xb = xp[static_cast<size_t>(t) * chunks16 + c];
+                    mma_16816_bf16(c4, nibble_pair_bf16(wg, 0), nibble_pair_bf16(wu, 0), nibble_pair_bf16(wg, 1),
+                                   nibble_pair_bf16(wu, 1), xb.x, xb.y);
+                    mma_16816_bf16(c4, nibble_pair_bf16(wg, 2), nibble_pair_bf16(wu, 2), nibble_pair_bf16(wg, 3),
+                                   nibble_pair_bf16(wu, 3), xb.z, xb.w);
+                    asm volatile("" ::: "memory");
+                }
+                if (t == 0) {   // column 0 of the accumulator: rows g (gate) and 8 + g (up)
+                    const float off = kNibbleBias * xsum[block];
+                    a_g = fmaf(__bfloat162float(stage_sc[static_cast<size_t>(g) * nb + block]), c4[0] - off, a_g);
+                    a_u = fmaf(__bfloat162float(stage_sc[static_cast<size_t>(NB + g) * nb + block]), c4[2] - off, a_u);
+                }
+            }
+            if (t == 0) {
+                atomicAdd(&red[g], a_g);
+                atomicAdd(&red[NB + g], a_u);
+            }
+        }
+        ring_consumer_barrier();
+        if (tid < 2 * NB) hd.red[(it + 2) % 3][tid] = 0.0f;     // the buffer of the batch after next
+        if (!*abort_flag) issue_batch(it + STAGES - 1);        // into the stage of batch it-1, which everybody has left
+        if (slot >= 0) {
+            // ---- phase 2: this warp's d/16 columns of the 8 down rows on the tensor cores ----
+            const float h0 = silu_mul(red[2 * t], red[NB + 2 * t]);
+            const float h1 = silu_mul(red[2 * t + 1], red[NB + 2 * t + 1]);
+            const __nv_bfloat16* ds = stage_sc + static_cast<size_t>(2 * NB) * nb;
+            const unsigned char* d0 = stage + static_cast<size_t>(2 * NB + 2 * t) * pitch + g * 4;
+            const unsigned char* d1 = d0 + pitch;
+#pragma unroll
+            for (int q = 0; q < KG; ++q) {
+                const int grp = warp * KG + q;                  // 64-column group; its scale block is grp / 2
+                const float f0 = h0 * __bfloat162float(ds[static_cast<size_t>(2 * t) * nb + (grp >> 1)]);
+                const float f1 = h1 * __bfloat162float(ds[static_cast<size_t>(2 * t + 1) * nb + (grp >> 1)]);
+                // sum of f over the 8 neurons (lanes with the same g hold the 4 pairs)
+                float fs = f0 + f1;
+                fs += __shfl_xor_sync(0xffffffffu, fs, 1);
+                fs += __shfl_xor_sync(0xffffffffu, fs, 2);
+                corr[q] += fs;
+                // f = high + low, both bf16: column 0 of B carries the high parts, column 1 the low parts
+                const __nv_bfloat16 f0h = __float2bfloat16_rn(f0), f1h = __float2bfloat16_rn(f1);
+                const __nv_bfloat162 hi2 = __halves2bfloat162(f0h, f1h);
+                const __nv_bfloat162 lo2 = __floats2bfloat162_rn(f0 - __bfloat162float(f0h), f1 - __bfloat162float(f1h));
+                uint32_t bfrag = 0u;
+                if (g == 0) bfrag = *reinterpret_cast<const uint32_t*>(&hi2);
+                else if (g == 1) bfrag = *reinterpret_cast<const uint32_t*>(&lo2);
+                const uint32_t w0 = *reinterpret_cast<const uint32_t*>(d0 + grp * 32);
+                const uint32_t w1 = *reinterpret_cast<const uint32_t*>(d1 + grp * 32);
+                uint32_t p0[4], p1[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) { p0[k] = nibble_pair_bf16(w0, k); p1[k] = nibble_pair_bf16(w1, k); }
+                // column c < 4 is the low half of pair c, column c >= 4 the high half of pair c - 4; an A register holds
+                // one column of the two rows
+                mma_16816_bf16(acc[q][0], __byte_perm(p0[0], p1[0], 0x5410), __byte_perm(p0[1], p1[1], 0x5410), 0u, 0u, bfrag, 0u);
+                mma_16816_bf16(acc[q][1], __byte_perm(p0[2], p1[2], 0x5410), __byte_perm(p0[3], p1[3], 0x5410), 0u, 0u, bfrag, 0u);
+                mma_16816_bf16(acc[q][2], __byte_perm(p0[0], p1[0], 0x7632), __byte_perm(p0[1], p1[1], 0x7632), 0u, 0u, bfrag, 0u);
+                mma_16816_bf16(acc[q][3], __byte_perm(p0[2], p1[2], 0x7632), __byte_perm(p0[3], p1[3], 0x7632), 0u, 0u, bfrag, 0u);
+                asm volatile("" ::: "memory");   // keeps the next group's loads behind this group's MMAs (register pressure)
+            }
+        }
+    }
+    if (cur_slot >= 0) flush(cur_slot);
+    if (*abort_flag) {
+        // a wait ran out: every copy that was issued must have landed before the block goes away
+        __syncthreads();
+        if (tid == 0) {
+            for (int bi = max(0, n_it - STAGES); bi < n_it; ++bi) {
+                int never = 0;
+                mbar_wait_bounded(&hd.full[bi % STAGES], static_cast<uint32_t>(bi / STAGES) & 1u, &never);
+            }
+            flag_status(dev_status, HALO_DEV_TIMEOUT);
+        }
+    }
+}
+
 halo_status check_i4_shape(const halo_ffn_shape* s) {
     if (!s) return HALO_ERR_ARG;
     if (s->d_model <= 0 || s->d_model % kQBlock != 0 || s->d_model > 8192 || s->group_size <= 0 || s->d_ffn <= 0 ||
@@ -558,6 +834,31 @@ extern "C" halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void
     int dev = 0, sms = kSmCount;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const bool no_ring = option_value(OPT_I4_NO_RING) == 1;
+    // 3: ring with the products on the tensor cores.  Correct, and measured SLOWER than the CUDA-core ring (61 against
+    // 35 us on the 7B block): mma.sync is the legacy tensor path on this GPU, so it is kept as an option only.
+    const int form = option_value(OPT_I4_NO_RING);
+    if ((d == 2048 || d == 4096) && S % kRingNB == 0 && form == 3) {
+        constexpr int kStages = 4;
+        const size_t nbk = static_cast<size_t>(d) / kQBlock;
+        const size_t stage = 3 * kRingNB * (static_cast<size_t>(d) / 2 + 16) + 3 * nbk * 2 * kRingNB;
+        const size_t smem_m = 1024 + static_cast<size_t>(d) * 2 + ((nbk * 4 + 127) & ~size_t(127)) + kStages * stage;
+        const long long batches = static_cast<long long>(G) * (S / kRingNB);
+        const dim3 grid_m(static_cast<unsigned>(std::min<long long>(batches, sms)), n_tok);
+        if (d == 4096) {
+            auto k = group_ffn_i4_mma_kernel<4, kStages>;
+            static bool once[64] = {};
+            if (!ensure_dynamic_smem(k, smem_m, once)) return HALO_ERR_CUDA;
+            k<<<grid_m, kRingConsumers, smem_m, st>>>(d, S, G, q, sc, xt, keep_list, n_keep, dev_of_group, n_dev, n_tok,
+                                                     partials, dev_status);
+        } else {
+            auto k = group_ffn_i4_mma_kernel<2, kStages>;
+            static bool once[64] = {};
+            if (!ensure_dynamic_smem(k, smem_m, once)) return HALO_ERR_CUDA;
+            k<<<grid_m, kRingConsumers, smem_m, st>>>(d, S, G, q, sc, xt, keep_list, n_keep, dev_of_group, n_dev, n_tok,
+                                                   partials, dev_status);
+        }
+        return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+    }
     if ((d == 2048 || d == 4096) && S % kRingNB == 0 && !no_ring) {
         // ring form: one block per SM
         constexpr int kStages = 4;

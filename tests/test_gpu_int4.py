@@ -95,10 +95,19 @@ def test_int4_full_size_7b_block_sampled_groups():
     assert np.abs(P - ref).max() <= U.TOL_BF16 * rms
 
 
-def test_int4_full_size_7b_block_all_groups_kept_every_element():
+@pytest.mark.parametrize("form", [-1, 1, 3])
+def test_int4_full_size_7b_block_all_groups_kept_every_element(form):
     """The case the benchmark times: one 7B-shaped block on int4 weights with all 86 groups kept (the shared-memory
-    ring kernel with a full kept set).  Codes and scales of the whole block bit for bit, every output element of
-    every holder slot against the oracle."""
+    ring kernel with a full kept set; also the plain-load form and the tensor-core form).  Codes and scales of the
+    whole block bit for bit, every output element of every holder slot against the oracle."""
+    B.halo_set_option("i4_no_ring", form)
+    try:
+        _full_block_all_groups()
+    finally:
+        B.halo_set_option("i4_no_ring", -1)
+
+
+def _full_block_all_groups():
     wl = synth.workload("llama2-7b-decode")
     Wp = synth.packed_layer(wl, 3, DEV)
     sh, Q, Sc = _quantize(wl, Wp)
@@ -118,3 +127,52 @@ def test_int4_full_size_7b_block_all_groups_kept_every_element():
     P16 = R.group_ffn(hb(Wp), hb(x), keep, dev, wl.n_dev)
     diff = R.merge(ref) - R.merge(P16)
     assert np.sqrt(np.mean(diff ** 2)) <= 0.5 * np.sqrt(np.mean(R.merge(P16) ** 2))
+
+
+@pytest.mark.parametrize("name,layers,steps", [("tinyllama-1.1b-decode", 3, 3), ("llama2-7b-decode", 3, 2)])
+def test_int4_stack_teacher_forced(name, layers, steps):
+    """The FFN stack on int4 weights (halo_stack_create_i4): scores and selections as for the bf16 stack, every block's
+    output against the oracle's FFN on the dequantised weights from the recorded input."""
+    wl = synth.small_variant(synth.workload(name), layers, steps)
+    L, G, d, n = wl.n_layers, wl.n_groups, wl.d_model, wl.n_dev
+    hb = synth.host_bits
+    quant = []
+    for l in range(L):
+        Wp = synth.packed_layer(wl, l, DEV)
+        _, Q, Sc = _quantize(wl, Wp)
+        quant.append((Q, Sc))
+    preds = [synth.predictor(wl, l, DEV) for l in range(L)]
+    plan = B.Plan(G, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
+    stack = B.Stack(B.ffn_shape(d, wl.d_ffn, wl.group_size, B.BF16), B.pred_shape(d, wl.pred_rank, G, B.BF16), 1, plan,
+                    [q[0] for q in quant], [p[0] for p in preds], [p[1] for p in preds], i4_scales=[q[1] for q in quant])
+    h0 = torch.stack([synth.stream_input(wl, s, DEV) for s in range(steps)])
+    h_out = torch.empty_like(h0)
+    t = dict(x=torch.zeros((steps, L, 1, d), dtype=torch.bfloat16, device=DEV),
+             scores=torch.zeros((steps, L, G), dtype=torch.float32, device=DEV),
+             dev_of_group=torch.zeros((steps, L, G), dtype=torch.int32, device=DEV),
+             arrived=torch.zeros((steps, L, n), dtype=torch.uint8, device=DEV),
+             keep_list=torch.zeros((steps, L, G), dtype=torch.int32, device=DEV),
+             n_keep=torch.zeros((steps, L), dtype=torch.int32, device=DEV),
+             y=torch.zeros((steps, L, 1, d), dtype=torch.float32, device=DEV))
+    taps = B.Taps(*[t[k].data_ptr() for k in ("x", "scores", "dev_of_group", "arrived", "keep_list", "n_keep", "y")])
+    stack.decode(h0, steps, 2, h_out, taps)
+    torch.cuda.synchronize()
+    assert stack.status() == 0 and stack.last_launches() > steps * L
+    x_all = hb(t["x"])
+    lost = 0
+    for s in range(steps):
+        for l in range(L):
+            scores = t["scores"][s, l].cpu().numpy()
+            if l > 0:
+                ref = R.predict(hb(preds[l][0]), hb(preds[l][1]), x_all[s, l - 1])
+                assert U.rel_err(scores, ref.astype(np.float64)) <= U.TOL_BF16
+            sel = R.select(scores, wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0, wl.seed, 2 + s, l,
+                           force_all=(l == 0))
+            nk = int(t["n_keep"][s, l].item())
+            assert nk == sel["n_keep"] and (t["keep_list"][s, l].cpu().numpy() == sel["keep_list"]).all()
+            lost += int(nk < G)
+            Q, Sc = quant[l]
+            P = R.group_ffn_i4(Q.cpu().numpy(), hb(Sc), x_all[s, l], sel["keep_list"][:nk], sel["dev_of_group"], n)
+            y_ref = R.merge(P)
+            assert U.rel_err(t["y"][s, l].cpu().numpy(), y_ref) <= U.TOL_BF16, (s, l)
+    assert lost > 0

@@ -312,6 +312,14 @@ halo_status halo_pack_mha_weights(const halo_mha_shape* shape, const void* Wq, c
 halo_status halo_mha_kv_append(const halo_mha_shape* shape, const void* Wk, const void* Wv, const void* x, int pos,
                                void* K_cache, void* V_cache, void* stream);
 size_t halo_group_mha_workspace_bytes(const halo_mha_shape* shape);
+/* halo_mha_block: halo_mha_kv_append and halo_group_mha of one token in ONE launch (a cluster of eight thread blocks
+ * per head: keys and values of every head are written at `pos`, then the kept heads attend over positions 0..pos and
+ * add their output-projection slices into partials, zeroed by the call).  Same results as the two calls in turn;
+ * K_cache / V_cache are read and written; no workspace. */
+halo_status halo_mha_block(const halo_mha_shape* shape, const void* W_packed, const void* Wk, const void* Wv,
+                           const void* x, void* K_cache, void* V_cache, int pos, const int32_t* keep_list,
+                           const int32_t* n_keep, const int32_t* dev_of_group, int n_dev, float* partials,
+                           uint32_t* dev_status, void* stream);
 halo_status halo_group_mha(const halo_mha_shape* shape, const void* W_packed, const void* x, const void* K_cache,
                            const void* V_cache, int pos, const int32_t* keep_list, const int32_t* n_keep,
                            const int32_t* dev_of_group, int n_dev, float* partials, void* workspace,

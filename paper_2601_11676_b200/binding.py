@@ -35,7 +35,7 @@ EXPORTS = [
     "halo_pack_mha_weights", "halo_mha_kv_append", "halo_group_mha_workspace_bytes", "halo_group_mha",
     "halo_group_lm_head", "halo_late_devices", "halo_quantize_weights_i4", "halo_group_ffn_i4", "halo_set_option",
     "halo_block_stack_create", "halo_block_stack_destroy", "halo_block_stack_decode", "halo_block_stack_status",
-    "halo_block_stack_last_launches", "halo_stack_create_i4",
+    "halo_block_stack_last_launches", "halo_stack_create_i4", "halo_mha_block",
 ]
 
 
@@ -142,6 +142,8 @@ def lib() -> ctypes.CDLL:
         L.halo_group_mha_workspace_bytes.argtypes = [POINTER(MhaShape)]
         L.halo_group_mha.argtypes = [POINTER(MhaShape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
                                      c_void_p, c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
+        L.halo_mha_block.argtypes = [POINTER(MhaShape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int,
+                                     c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
         L.halo_group_lm_head.argtypes = [POINTER(LmShape), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
                                          c_void_p, c_void_p]
         L.halo_quantize_weights_i4.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_void_p]
@@ -340,6 +342,13 @@ def halo_group_mha(shape: MhaShape, W_packed, x, K_cache, V_cache, pos, keep_lis
                               _ptr(keep_list), _ptr(n_keep), _ptr(dev_of_group), n_dev, _ptr(partials), _ptr(workspace),
                               workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream)),
          "halo_group_mha")
+
+
+def halo_mha_block(shape: MhaShape, W_packed, Wk, Wv, x, K_cache, V_cache, pos, keep_list, n_keep, dev_of_group, n_dev,
+                   partials, dev_status=None, stream=None) -> None:
+    _chk(lib().halo_mha_block(byref(shape), _ptr(W_packed), _ptr(Wk), _ptr(Wv), _ptr(x), _ptr(K_cache), _ptr(V_cache), pos,
+                              _ptr(keep_list), _ptr(n_keep), _ptr(dev_of_group), n_dev, _ptr(partials), _ptr(dev_status),
+                              _stream(stream)), "halo_mha_block")
 
 
 def lm_shape(d_model, vocab, group_size, dtype) -> LmShape:

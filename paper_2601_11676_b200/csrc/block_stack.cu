@@ -1,6 +1,7 @@
 // halo_block_stack_*: the generation loop over whole transformer blocks (Sec. III-B.3: in every layer the MHA block
 // and then the MLP block, one predictor each fed one layer ahead, the first layer and the LM head reliable), built
-// from the group entry points of this library: one launch per step of the path, no host synchronisation inside.
+// from the group entry points of this library: one launch per step of the path (the MHA block is one launch, the
+// predictors of the next layer run on a side stream), no host synchronisation inside.
 #include <algorithm>
 #include <cstring>
 #include <new>
@@ -30,13 +31,16 @@ struct halo_block_stack {
     float* h;
     void* x_a[2];
     void* x_f[2];
-    float* hidden;            // predictor hidden values
-    float* scores_a; float* scores_f; float* zero_scores;
-    int32_t* dev_a; int32_t* dev_f;
-    uint8_t* arr_a; uint8_t* arr_f;
-    int32_t* kl_a; int32_t* kl_f;
-    int32_t* nk_a; int32_t* nk_f;
+    // selections of a layer are made one layer ahead on a side stream: two sets each, by parity of the layer
+    float* hidden_a; float* hidden_f;
+    float* scores_a[2]; float* scores_f[2]; float* zero_scores;
+    int32_t* dev_a[2]; int32_t* dev_f[2];
+    uint8_t* arr_a[2]; uint8_t* arr_f[2];
+    int32_t* kl_a[2]; int32_t* kl_f[2];
+    int32_t* nk_a[2]; int32_t* nk_f[2];
     float* part_a; float* part_f;
+    cudaStream_t side;
+    cudaEvent_t ev_xa, ev_xf, ev_sa, ev_sf;
     void* mha_ws; size_t mha_ws_bytes;
     uint32_t* status;
     long long last_launches;
@@ -89,12 +93,16 @@ extern "C" halo_status halo_block_stack_create(halo_block_stack** out, const hal
     auto carve = [&](size_t bytes) { size_t o = off; off = bs_align(off + bytes); return o; };
     const size_t o_h = carve(sizeof(float) * d);
     const size_t o_xa0 = carve(es * d), o_xa1 = carve(es * d), o_xf0 = carve(es * d), o_xf1 = carve(es * d);
-    const size_t o_hid = carve(sizeof(float) * std::max(pred_ffn->rank, pred_mha->rank));
-    const size_t o_sa = carve(sizeof(float) * H), o_sf = carve(sizeof(float) * G), o_zs = carve(sizeof(float) * std::max(G, H));
-    const size_t o_da = carve(sizeof(int32_t) * H), o_df = carve(sizeof(int32_t) * G);
-    const size_t o_aa = carve(HALO_MAX_DEVICES), o_af = carve(HALO_MAX_DEVICES);
-    const size_t o_ka = carve(sizeof(int32_t) * H), o_kf = carve(sizeof(int32_t) * G);
-    const size_t o_na = carve(sizeof(int32_t)), o_nf = carve(sizeof(int32_t));
+    const size_t o_hida = carve(sizeof(float) * pred_mha->rank), o_hidf = carve(sizeof(float) * pred_ffn->rank);
+    const size_t o_zs = carve(sizeof(float) * std::max(G, H));
+    size_t o_sa[2], o_sf[2], o_da[2], o_df[2], o_aa[2], o_af[2], o_ka[2], o_kf[2], o_na[2], o_nf[2];
+    for (int k = 0; k < 2; ++k) {
+        o_sa[k] = carve(sizeof(float) * H); o_sf[k] = carve(sizeof(float) * G);
+        o_da[k] = carve(sizeof(int32_t) * H); o_df[k] = carve(sizeof(int32_t) * G);
+        o_aa[k] = carve(HALO_MAX_DEVICES); o_af[k] = carve(HALO_MAX_DEVICES);
+        o_ka[k] = carve(sizeof(int32_t) * H); o_kf[k] = carve(sizeof(int32_t) * G);
+        o_na[k] = carve(sizeof(int32_t)); o_nf[k] = carve(sizeof(int32_t));
+    }
     const size_t o_pa = carve(sizeof(float) * (s->n_dev_a + 1) * d), o_pf = carve(sizeof(float) * (s->n_dev_f + 1) * d);
     s->mha_ws_bytes = halo_group_mha_workspace_bytes(mha);
     const size_t o_mw = carve(s->mha_ws_bytes);
@@ -104,22 +112,47 @@ extern "C" halo_status halo_block_stack_create(halo_block_stack** out, const hal
     char* b = static_cast<char*>(s->slab);
     s->h = reinterpret_cast<float*>(b + o_h);
     s->x_a[0] = b + o_xa0; s->x_a[1] = b + o_xa1; s->x_f[0] = b + o_xf0; s->x_f[1] = b + o_xf1;
-    s->hidden = reinterpret_cast<float*>(b + o_hid);
-    s->scores_a = reinterpret_cast<float*>(b + o_sa); s->scores_f = reinterpret_cast<float*>(b + o_sf);
+    s->hidden_a = reinterpret_cast<float*>(b + o_hida); s->hidden_f = reinterpret_cast<float*>(b + o_hidf);
     s->zero_scores = reinterpret_cast<float*>(b + o_zs);
-    s->dev_a = reinterpret_cast<int32_t*>(b + o_da); s->dev_f = reinterpret_cast<int32_t*>(b + o_df);
-    s->arr_a = reinterpret_cast<uint8_t*>(b + o_aa); s->arr_f = reinterpret_cast<uint8_t*>(b + o_af);
-    s->kl_a = reinterpret_cast<int32_t*>(b + o_ka); s->kl_f = reinterpret_cast<int32_t*>(b + o_kf);
-    s->nk_a = reinterpret_cast<int32_t*>(b + o_na); s->nk_f = reinterpret_cast<int32_t*>(b + o_nf);
+    for (int k = 0; k < 2; ++k) {
+        s->scores_a[k] = reinterpret_cast<float*>(b + o_sa[k]); s->scores_f[k] = reinterpret_cast<float*>(b + o_sf[k]);
+        s->dev_a[k] = reinterpret_cast<int32_t*>(b + o_da[k]); s->dev_f[k] = reinterpret_cast<int32_t*>(b + o_df[k]);
+        s->arr_a[k] = reinterpret_cast<uint8_t*>(b + o_aa[k]); s->arr_f[k] = reinterpret_cast<uint8_t*>(b + o_af[k]);
+        s->kl_a[k] = reinterpret_cast<int32_t*>(b + o_ka[k]); s->kl_f[k] = reinterpret_cast<int32_t*>(b + o_kf[k]);
+        s->nk_a[k] = reinterpret_cast<int32_t*>(b + o_na[k]); s->nk_f[k] = reinterpret_cast<int32_t*>(b + o_nf[k]);
+    }
     s->part_a = reinterpret_cast<float*>(b + o_pa); s->part_f = reinterpret_cast<float*>(b + o_pf);
     s->mha_ws = b + o_mw;
     s->status = reinterpret_cast<uint32_t*>(b + o_st);
+    // side stream for the predictors (best effort: without it they run in line on the caller's stream)
+    s->side = nullptr;
+    s->ev_xa = s->ev_xf = s->ev_sa = s->ev_sf = nullptr;
+    int prio_lo = 0, prio_hi = 0;
+    if (cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) != cudaSuccess) prio_hi = 0;
+    if (cudaStreamCreateWithPriority(&s->side, cudaStreamNonBlocking, prio_hi) == cudaSuccess) {
+        bool ok = true;
+        for (cudaEvent_t* e : {&s->ev_xa, &s->ev_xf, &s->ev_sa, &s->ev_sf})
+            ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
+            for (cudaEvent_t e : {s->ev_xa, s->ev_xf, s->ev_sa, s->ev_sf}) if (e) cudaEventDestroy(e);
+            cudaStreamDestroy(s->side);
+            s->side = nullptr;
+        }
+    } else {
+        s->side = nullptr;
+        (void)cudaGetLastError();
+    }
     *out = s;
     return HALO_OK;
 }
 
 extern "C" halo_status halo_block_stack_destroy(halo_block_stack* s) {
     if (!s) return HALO_OK;
+    if (s->side) {
+        cudaStreamSynchronize(s->side);
+        for (cudaEvent_t e : {s->ev_xa, s->ev_xf, s->ev_sa, s->ev_sf}) cudaEventDestroy(e);
+        cudaStreamDestroy(s->side);
+    }
     cudaFree(s->slab);
     delete s;
     return HALO_OK;
@@ -140,78 +173,95 @@ extern "C" halo_status halo_block_stack_decode(halo_block_stack* s, const float*
 #define BS_COPY(dst, src, bytes)                                                                      \
     do { if (cudaMemcpyAsync((dst), (src), (bytes), cudaMemcpyDeviceToDevice, st) != cudaSuccess)     \
              return HALO_ERR_CUDA; } while (0)
+#define BS_CU(call) do { if ((call) != cudaSuccess) return HALO_ERR_CUDA; } while (0)
+    // The scores of layer l need only layer l-1's inputs (one layer ahead, Sec. III-B.2): predictor and selection of
+    // both blocks of layer l run on the side stream while layer l-1's blocks run here.  The partial slots are zeroed
+    // once and left zeroed by every merge, so the streaming kernels need no zero-fill in front of them.
+    cudaStream_t side = s->side ? s->side : st;
+    const bool fork = s->side != nullptr;
+    if (cudaMemsetAsync(s->part_a, 0, sizeof(float) * (s->n_dev_a + 1) * d, st) != cudaSuccess ||
+        cudaMemsetAsync(s->part_f, 0, sizeof(float) * (s->n_dev_f + 1) * d, st) != cudaSuccess)
+        return HALO_ERR_CUDA;
     for (int sidx = 0; sidx < steps; ++sidx) {
         const uint32_t step = step0 + static_cast<uint32_t>(sidx);
         const int pos = pos0 + sidx;
         BS_TRY(launch_glue(d, 1, dt, h0 + static_cast<size_t>(sidx) * d, nullptr, s->h, s->x_a[0], st));
-        ++launches;
+        // layer 0: reliable, nothing to go by yet -> every head and every group is kept
+        BS_TRY(launch_select(s->plan_mha.dev, H, s->zero_scores, step, 0u, 1, nullptr, s->dev_a[0], s->arr_a[0], nullptr,
+                             s->kl_a[0], s->nk_a[0], s->status, st));
+        BS_TRY(launch_select(s->plan_ffn.dev, G, s->zero_scores, step, 1u, 1, nullptr, s->dev_f[0], s->arr_f[0], nullptr,
+                             s->kl_f[0], s->nk_f[0], s->status, st));
+        launches += 3;
         for (int l = 0; l < L; ++l) {
             const size_t rec = static_cast<size_t>(sidx) * L + l;
-            void* xa = s->x_a[l & 1];
-            void* xf = s->x_f[l & 1];
-            // ---- MHA block: keys / values of every head, then the kept heads ----
-            BS_TRY(halo_mha_kv_append(&s->mha, s->Wk[l], s->Wv[l], xa, pos, s->K[l], s->V[l], stream));
-            ++launches;
-            const float* sc_a = s->scores_a;
-            if (l == 0) {
-                sc_a = s->zero_scores;   // first layer: reliable, nothing to go by yet -> every head is kept
-                BS_TRY(launch_select(s->plan_mha.dev, H, s->zero_scores, step, 0u, 1, nullptr, s->dev_a, s->arr_a, nullptr,
-                                     s->kl_a, s->nk_a, s->status, st));
-                ++launches;
-            } else {
-                BS_TRY(launch_predict_hidden(s->pred_mha, s->W1_mha[l], s->x_a[(l - 1) & 1], 1, s->hidden, st));
-                BS_TRY(launch_score_select(s->pred_mha, s->W2_mha[l], s->hidden, s->plan_mha.dev, step,
-                                           static_cast<uint32_t>(2 * l), 0, s->scores_a, nullptr, s->dev_a, s->arr_a, nullptr,
-                                           s->kl_a, s->nk_a, s->status, st));
+            const int cur = l & 1, nxt = (l + 1) & 1;
+            void* xa = s->x_a[cur];
+            void* xf = s->x_f[cur];
+            // ---- MHA block ----
+            if (l + 1 < L) {
+                // heads of layer l+1 from this layer's attention input
+                if (fork) { BS_CU(cudaEventRecord(s->ev_xa, st)); BS_CU(cudaStreamWaitEvent(side, s->ev_xa, 0)); }
+                BS_TRY(launch_predict_hidden(s->pred_mha, s->W1_mha[l + 1], xa, 1, s->hidden_a, side));
+                BS_TRY(launch_score_select(s->pred_mha, s->W2_mha[l + 1], s->hidden_a, s->plan_mha.dev, step,
+                                           static_cast<uint32_t>(2 * (l + 1)), 0, s->scores_a[nxt], nullptr, s->dev_a[nxt],
+                                           s->arr_a[nxt], nullptr, s->kl_a[nxt], s->nk_a[nxt], s->status, side));
+                if (fork) BS_CU(cudaEventRecord(s->ev_sa, side));
                 launches += 2;
             }
-            BS_TRY(halo_group_mha(&s->mha, s->W_mha[l], xa, s->K[l], s->V[l], pos, s->kl_a, s->nk_a, s->dev_a, s->n_dev_a,
-                                  s->part_a, s->mha_ws, s->mha_ws_bytes, s->status, stream));
-            launches += 2;
+            if (s->mha.head_dim % 16 == 0) {
+                BS_TRY(launch_mha_block(s->mha, s->W_mha[l], s->Wk[l], s->Wv[l], xa, s->K[l], s->V[l], pos, s->kl_a[cur],
+                                        s->nk_a[cur], s->dev_a[cur], s->n_dev_a, s->part_a, s->status, st, true));
+                ++launches;
+            } else {
+                BS_TRY(halo_mha_kv_append(&s->mha, s->Wk[l], s->Wv[l], xa, pos, s->K[l], s->V[l], stream));
+                BS_TRY(halo_group_mha(&s->mha, s->W_mha[l], xa, s->K[l], s->V[l], pos, s->kl_a[cur], s->nk_a[cur], s->dev_a[cur],
+                                      s->n_dev_a, s->part_a, s->mha_ws, s->mha_ws_bytes, s->status, stream));
+                launches += 3;
+            }
             float* y_tap = nullptr;
             if (taps) {
                 const halo_taps& t = taps->mha;
                 if (t.x) BS_COPY(static_cast<char*>(t.x) + rec * d * es, xa, d * es);
-                if (t.scores) BS_COPY(t.scores + rec * H, sc_a, sizeof(float) * H);
-                if (t.dev_of_group) BS_COPY(t.dev_of_group + rec * H, s->dev_a, sizeof(int32_t) * H);
-                if (t.arrived && s->n_dev_a > 0) BS_COPY(t.arrived + rec * s->n_dev_a, s->arr_a, s->n_dev_a);
-                if (t.keep_list) BS_COPY(t.keep_list + rec * H, s->kl_a, sizeof(int32_t) * H);
-                if (t.n_keep) BS_COPY(t.n_keep + rec, s->nk_a, sizeof(int32_t));
+                if (t.scores) BS_COPY(t.scores + rec * H, l == 0 ? s->zero_scores : s->scores_a[cur], sizeof(float) * H);
+                if (t.dev_of_group) BS_COPY(t.dev_of_group + rec * H, s->dev_a[cur], sizeof(int32_t) * H);
+                if (t.arrived && s->n_dev_a > 0) BS_COPY(t.arrived + rec * s->n_dev_a, s->arr_a[cur], s->n_dev_a);
+                if (t.keep_list) BS_COPY(t.keep_list + rec * H, s->kl_a[cur], sizeof(int32_t) * H);
+                if (t.n_keep) BS_COPY(t.n_keep + rec, s->nk_a[cur], sizeof(int32_t));
                 if (t.y) y_tap = t.y + rec * d;
             }
             // merge of the heads that arrived + residual; the normalised stream is the MLP block's input
-            BS_TRY(launch_merge_glue(s->part_a, s->arr_a, s->n_dev_a, 1, d, dt, s->h, s->h, xf, y_tap, st));
+            BS_TRY(launch_merge_glue(s->part_a, s->arr_a[cur], s->n_dev_a, 1, d, dt, s->h, s->h, xf, y_tap, st, true));
             ++launches;
             // ---- MLP block ----
-            const float* sc_f = s->scores_f;
-            if (l == 0) {
-                sc_f = s->zero_scores;
-                BS_TRY(launch_select(s->plan_ffn.dev, G, s->zero_scores, step, 1u, 1, nullptr, s->dev_f, s->arr_f, nullptr,
-                                     s->kl_f, s->nk_f, s->status, st));
-                ++launches;
-            } else {
-                BS_TRY(launch_predict_hidden(s->pred_ffn, s->W1_ffn[l], s->x_f[(l - 1) & 1], 1, s->hidden, st));
-                BS_TRY(launch_score_select(s->pred_ffn, s->W2_ffn[l], s->hidden, s->plan_ffn.dev, step,
-                                           static_cast<uint32_t>(2 * l + 1), 0, s->scores_f, nullptr, s->dev_f, s->arr_f,
-                                           nullptr, s->kl_f, s->nk_f, s->status, st));
+            if (l + 1 < L) {
+                // groups of layer l+1 from this layer's MLP input
+                if (fork) { BS_CU(cudaEventRecord(s->ev_xf, st)); BS_CU(cudaStreamWaitEvent(side, s->ev_xf, 0)); }
+                BS_TRY(launch_predict_hidden(s->pred_ffn, s->W1_ffn[l + 1], xf, 1, s->hidden_f, side));
+                BS_TRY(launch_score_select(s->pred_ffn, s->W2_ffn[l + 1], s->hidden_f, s->plan_ffn.dev, step,
+                                           static_cast<uint32_t>(2 * (l + 1) + 1), 0, s->scores_f[nxt], nullptr, s->dev_f[nxt],
+                                           s->arr_f[nxt], nullptr, s->kl_f[nxt], s->nk_f[nxt], s->status, side));
+                if (fork) BS_CU(cudaEventRecord(s->ev_sf, side));
                 launches += 2;
             }
-            BS_TRY(halo_group_ffn(&s->ffn, s->W_ffn[l], xf, 1, s->kl_f, s->nk_f, s->dev_f, s->n_dev_f, s->part_f, nullptr, 0,
-                                  s->status, stream));
-            launches += 2;
+            BS_TRY(launch_group_ffn_decode(s->ffn, s->W_ffn[l], xf, 1, s->kl_f[cur], s->nk_f[cur], s->dev_f[cur], s->n_dev_f,
+                                           s->part_f, s->status, st, true));
+            ++launches;
             y_tap = nullptr;
             if (taps) {
                 const halo_taps& t = taps->ffn;
                 if (t.x) BS_COPY(static_cast<char*>(t.x) + rec * d * es, xf, d * es);
-                if (t.scores) BS_COPY(t.scores + rec * G, sc_f, sizeof(float) * G);
-                if (t.dev_of_group) BS_COPY(t.dev_of_group + rec * G, s->dev_f, sizeof(int32_t) * G);
-                if (t.arrived && s->n_dev_f > 0) BS_COPY(t.arrived + rec * s->n_dev_f, s->arr_f, s->n_dev_f);
-                if (t.keep_list) BS_COPY(t.keep_list + rec * G, s->kl_f, sizeof(int32_t) * G);
-                if (t.n_keep) BS_COPY(t.n_keep + rec, s->nk_f, sizeof(int32_t));
+                if (t.scores) BS_COPY(t.scores + rec * G, l == 0 ? s->zero_scores : s->scores_f[cur], sizeof(float) * G);
+                if (t.dev_of_group) BS_COPY(t.dev_of_group + rec * G, s->dev_f[cur], sizeof(int32_t) * G);
+                if (t.arrived && s->n_dev_f > 0) BS_COPY(t.arrived + rec * s->n_dev_f, s->arr_f[cur], s->n_dev_f);
+                if (t.keep_list) BS_COPY(t.keep_list + rec * G, s->kl_f[cur], sizeof(int32_t) * G);
+                if (t.n_keep) BS_COPY(t.n_keep + rec, s->nk_f[cur], sizeof(int32_t));
                 if (t.y) y_tap = t.y + rec * d;
             }
+            // both selections of layer l+1 must be in before its blocks start, and the side stream must be done
+            // reading this layer's inputs before later merges overwrite those buffers
+            if (fork && l + 1 < L) { BS_CU(cudaStreamWaitEvent(st, s->ev_sa, 0)); BS_CU(cudaStreamWaitEvent(st, s->ev_sf, 0)); }
             // merge + residual; the normalised stream is the next layer's attention input (or the LM head's input)
-            BS_TRY(launch_merge_glue(s->part_f, s->arr_f, s->n_dev_f, 1, d, dt, s->h, s->h, s->x_a[(l + 1) & 1], y_tap, st));
+            BS_TRY(launch_merge_glue(s->part_f, s->arr_f[cur], s->n_dev_f, 1, d, dt, s->h, s->h, s->x_a[nxt], y_tap, st, true));
             ++launches;
         }
         if (logits) {
@@ -222,6 +272,7 @@ extern "C" halo_status halo_block_stack_decode(halo_block_stack* s, const float*
         }
         if (h_out) BS_COPY(h_out + static_cast<size_t>(sidx) * d, s->h, sizeof(float) * d);
     }
+#undef BS_CU
 #undef BS_TRY
 #undef BS_COPY
     s->last_launches = launches;

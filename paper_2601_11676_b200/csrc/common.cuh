@@ -114,9 +114,11 @@ halo_status launch_score_select(const halo_pred_shape& sh, const void* W2, const
                                 int32_t* keep_list, int32_t* n_keep, uint32_t* dev_status, cudaStream_t st);
 halo_status launch_predict_hidden(const halo_pred_shape& sh, const void* W1, const void* feat, int n_tok,
                                   float* hidden, cudaStream_t st);
+// already_zero: the caller guarantees that `partials` is zero (otherwise the call zeroes it first).
 halo_status launch_group_ffn_decode(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                     const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
-                                    int n_dev, float* partials, uint32_t* dev_status, cudaStream_t st);
+                                    int n_dev, float* partials, uint32_t* dev_status, cudaStream_t st,
+                                    bool already_zero = false);
 halo_status launch_group_ffn_stream(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                     const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
                                     int n_dev, float* partials, uint32_t* dev_status, cudaStream_t st);
@@ -138,9 +140,15 @@ halo_status launch_merge(const float* partials, const uint8_t* arrived, int n_de
 halo_status launch_glue(int d, int n_tok, halo_dtype xdtype, const float* h, const float* y, float* h_out,
                         void* x_out, cudaStream_t st);
 // merge + residual + normalise in one launch (stack path); y_tap may be NULL.
+// zero_after: every slot of `partials` is left zeroed (for a following kernel that adds into them).
 halo_status launch_merge_glue(const float* partials, const uint8_t* arrived, int n_dev, int n_tok, int d,
                               halo_dtype xdtype, const float* h, float* h_out, void* x_out, float* y_tap,
-                              cudaStream_t st);
+                              cudaStream_t st, bool zero_after = false);
+// halo_mha_block without argument checks; already_zero: the caller guarantees that `partials` is zero.
+halo_status launch_mha_block(const halo_mha_shape& sh, const void* W_packed, const void* Wk, const void* Wv, const void* x,
+                             void* K_cache, void* V_cache, int pos, const int32_t* keep_list, const int32_t* n_keep,
+                             const int32_t* dev_of_group, int n_dev, float* partials, uint32_t* dev_status, cudaStream_t st,
+                             bool already_zero);
 halo_status launch_pack(const halo_ffn_shape& sh, const void* Wgate, const void* Wup, const void* Wdown,
                         void* Wpacked, cudaStream_t st);
 

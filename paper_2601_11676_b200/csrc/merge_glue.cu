@@ -47,9 +47,9 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, float a, float b, float
 // One block per token.  MERGE: y is taken from the partial slots, else from y_in (may be NULL = 0).
 template <typename T, bool MERGE>
 __global__ void __launch_bounds__(1024)
-glue_kernel(int d, const float* __restrict__ h, const float* __restrict__ y_in, const float* __restrict__ partials,
+glue_kernel(int d, const float* __restrict__ h, const float* __restrict__ y_in, const float* partials,
             const uint8_t* __restrict__ arrived, int n_dev, size_t slot_stride, float* h_out, T* __restrict__ x_out,
-            float* __restrict__ y_tap, int vec) {
+            float* __restrict__ y_tap, int vec, float* zero_slots) {
     __shared__ float scratch[32];
     extern __shared__ __align__(16) float hv[];  // [d]
     const int tok = blockIdx.x;
@@ -70,6 +70,10 @@ glue_kernel(int d, const float* __restrict__ h, const float* __restrict__ y_in, 
                         y.x += p.x; y.y += p.y; y.z += p.z; y.w += p.w;
                     }
                 if (y_tap) reinterpret_cast<float4*>(y_tap + base)[c] = y;
+                if (zero_slots)   // the slots are left zeroed for the next kernel that adds into them
+                    for (int i = 0; i <= n_dev; ++i)
+                        reinterpret_cast<float4*>(zero_slots + static_cast<size_t>(i) * slot_stride + base)[c] =
+                            make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             } else if (y_in) {
                 y = reinterpret_cast<const float4*>(y_in + base)[c];
             }
@@ -84,6 +88,8 @@ glue_kernel(int d, const float* __restrict__ h, const float* __restrict__ y_in, 
             if (MERGE) {
                 y = merged_value(partials, arrived, n_dev, slot_stride, base + c);
                 if (y_tap) y_tap[base + c] = y;
+                if (zero_slots)
+                    for (int i = 0; i <= n_dev; ++i) zero_slots[static_cast<size_t>(i) * slot_stride + base + c] = 0.0f;
             } else if (y_in) {
                 y = y_in[base + c];
             }
@@ -148,26 +154,28 @@ halo_status launch_glue(int d, int n_tok, halo_dtype xdtype, const float* h, con
     const int vec = (d % 4 == 0) && all_aligned16({h, y, h_out, x_out});
     if (xdtype == HALO_BF16)
         glue_kernel<__nv_bfloat16, false><<<n_tok, 1024, smem, st>>>(d, h, y, nullptr, nullptr, 0, 0, h_out,
-                                                                      static_cast<__nv_bfloat16*>(x_out), nullptr, vec);
+                                                                      static_cast<__nv_bfloat16*>(x_out), nullptr, vec, nullptr);
     else
         glue_kernel<float, false><<<n_tok, 1024, smem, st>>>(d, h, y, nullptr, nullptr, 0, 0, h_out,
-                                                             static_cast<float*>(x_out), nullptr, vec);
+                                                             static_cast<float*>(x_out), nullptr, vec, nullptr);
     HALO_CHECK_LAUNCH();
     return HALO_OK;
 }
 
 halo_status launch_merge_glue(const float* partials, const uint8_t* arrived, int n_dev, int n_tok, int d,
                               halo_dtype xdtype, const float* h, float* h_out, void* x_out, float* y_tap,
-                              cudaStream_t st) {
+                              cudaStream_t st, bool zero_after) {
+    float* zero_slots = zero_after ? const_cast<float*>(partials) : nullptr;
     const size_t smem = sizeof(float) * static_cast<size_t>(d);
     const size_t stride = static_cast<size_t>(n_tok) * d;
     const int vec = (d % 4 == 0) && all_aligned16({partials, h, h_out, x_out, y_tap});
     if (xdtype == HALO_BF16)
         glue_kernel<__nv_bfloat16, true><<<n_tok, 1024, smem, st>>>(d, h, nullptr, partials, arrived, n_dev, stride,
-                                                                     h_out, static_cast<__nv_bfloat16*>(x_out), y_tap, vec);
+                                                                     h_out, static_cast<__nv_bfloat16*>(x_out), y_tap, vec,
+                                                                     zero_slots);
     else
         glue_kernel<float, true><<<n_tok, 1024, smem, st>>>(d, h, nullptr, partials, arrived, n_dev, stride, h_out,
-                                                            static_cast<float*>(x_out), y_tap, vec);
+                                                            static_cast<float*>(x_out), y_tap, vec, zero_slots);
     HALO_CHECK_LAUNCH();
     return HALO_OK;
 }

@@ -317,12 +317,17 @@ __device__ __forceinline__ void st_remote_f32(float* local_smem_ptr, uint32_t ta
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
 }
 
-template <typename T, int ITERS>
+// APPEND: the whole MHA block of a token in this one launch.  The grid then has one cluster per head (kept or not):
+// block r first computes dh / 8 rows each of the head's keys and values for this token and writes them into the
+// caches at `pos` (every head, never dropped); clusters of heads that are not kept end there.  The cluster barrier
+// that completes the query also orders those cache writes before the attention reads them.
+template <typename T, int ITERS, bool APPEND>
 __global__ void __cluster_dims__(kMhaCluster, 1, 1) __launch_bounds__(256)
 mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ Wp, const T* __restrict__ x,
-                 const T* __restrict__ Kc, const T* __restrict__ Vc, const int32_t* __restrict__ keep_list,
+                 const T* Kc, const T* Vc, const int32_t* __restrict__ keep_list,
                  const int32_t* __restrict__ n_keep_ptr, const int32_t* __restrict__ dev_of_group, int n_dev,
-                 float* __restrict__ partials, uint32_t* dev_status) {
+                 float* __restrict__ partials, uint32_t* dev_status, const T* __restrict__ Wk, const T* __restrict__ Wv,
+                 T* Kw, T* Vw) {
     constexpr int E = Elem<T>::kPerChunk;
     extern __shared__ __align__(16) float xs[];          // [d]: x widened
     __shared__ float q_s[256];                           // the head's full query (written by all blocks of the cluster)
@@ -334,26 +339,56 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
     __shared__ float o_s[kMhaMaxRows];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r = static_cast<int>(cluster_rank());
-    const int ki = blockIdx.y;
     int nk = *n_keep_ptr;
     nk = max(0, min(nk, H));
-    if (ki >= nk) return;                                // the same decision in every block of the cluster
-    const int h = keep_list[ki];
-    if (h < 0 || h >= H) {
-        if (tid == 0 && r == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
-        return;
-    }
-    int slot = 0;
-    if (dev_of_group) {
-        slot = dev_of_group[h] + 1;
-        if (slot < 0 || slot > n_dev) {
-            if (tid == 0 && r == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
-            return;
-        }
-    }
     const int rows = dh / kMhaCluster;                   // rows of the head per block (even: dh % 16 == 0)
     const int j0 = r * rows;
     const int chunks = d / E;
+    int h, slot = 0;
+    if constexpr (APPEND) {
+        h = blockIdx.y;
+        // keys and values of this token for head h, rows j0 .. j0 + rows of each, two rows per warp and turn
+        stage_x(x, xs, d);
+        __syncthreads();
+        for (int i = 2 * warp; i < 2 * rows; i += 16) {
+            const bool is_v = i >= rows;
+            const int j = j0 + (is_v ? i - rows : i);
+            const T* base = (is_v ? Wv : Wk) + (static_cast<size_t>(h) * dh + j) * d;
+            float va, vb;
+            warp_two_rows_dot(base, base + d, xs, chunks, lane, va, vb);
+            if (lane < 2) (is_v ? Vw : Kw)[(static_cast<size_t>(h) * Lmax + pos) * dh + j + lane] = from_float<T>(lane == 0 ? va : vb);
+        }
+        // is this head kept, and by whom?  (the list is short: one pass of the block over it)
+        int found = 0;
+        for (int i = tid; i < nk; i += 256) {
+            const int e = keep_list[i];
+            if (e == h) found = 1;
+            if ((e < 0 || e >= H) && h == 0 && r == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+        }
+        if (!__syncthreads_or(found)) return;            // the same decision in every block of the cluster
+        if (dev_of_group) {
+            slot = dev_of_group[h] + 1;
+            if (slot < 0 || slot > n_dev) {
+                if (tid == 0 && r == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+                return;
+            }
+        }
+    } else {
+        const int ki = blockIdx.y;
+        if (ki >= nk) return;                            // the same decision in every block of the cluster
+        h = keep_list[ki];
+        if (h < 0 || h >= H) {
+            if (tid == 0 && r == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+            return;
+        }
+        if (dev_of_group) {
+            slot = dev_of_group[h] + 1;
+            if (slot < 0 || slot > n_dev) {
+                if (tid == 0 && r == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+                return;
+            }
+        }
+    }
 
     // Distributed shared memory may be written only once every block of the cluster is known to be running:
     // arrive now, wait before the first remote store (the staging of x lies in between, and the blocks of a cluster
@@ -361,7 +396,7 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
     // of a cluster or by none.
     cluster_arrive();
     // ---- query rows j0 .. j0 + rows, two per warp and turn, sent to every block of the cluster ----
-    stage_x(x, xs, d);
+    if constexpr (!APPEND) stage_x(x, xs, d);
     for (int j = tid; j < dh; j += 256) o_acc[j] = 0.0f;
     __syncthreads();
     const float scale = rsqrtf(static_cast<float>(dh));
@@ -396,7 +431,7 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
 #pragma unroll 8
             for (int c = 0; c < col_groups; ++c) {
                 float kf[E];
-                Elem<T>::widen(__ldg(krow + c), kf);
+                Elem<T>::widen(APPEND ? __ldcg(krow + c) : __ldg(krow + c), kf);
 #pragma unroll
                 for (int e = 0; e < E; ++e) acc = fmaf(kf[e], q_s[c * E + e], acc);
             }
@@ -432,7 +467,7 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
 #pragma unroll 8
             for (int pp = pg; pp < n_valid; pp += pos_groups) {
                 float vf[E];
-                Elem<T>::widen(__ldg(vbase + static_cast<size_t>(pp) * col_groups), vf);
+                Elem<T>::widen(APPEND ? __ldcg(vbase + static_cast<size_t>(pp) * col_groups) : __ldg(vbase + static_cast<size_t>(pp) * col_groups), vf);
                 const float wp = w_s[pp];
 #pragma unroll
                 for (int k = 0; k < E; ++k) part[k] = fmaf(wp, vf[k], part[k]);
@@ -608,10 +643,10 @@ static halo_status group_mha_typed(const halo_mha_shape& sh, const void* Wp, con
         const size_t smem_f = sizeof(float) * d;
 #define HALO_MHA_FUSED(I)                                                                                            \
     case I:                                                                                                          \
-        mha_fused_kernel<T, I><<<grid_f, 256, smem_f, st>>>(d, H, dh, sh.max_len, pos, static_cast<const T*>(Wp),    \
-                                                            static_cast<const T*>(x), static_cast<const T*>(Kc),     \
-                                                            static_cast<const T*>(Vc), keep_list, n_keep,            \
-                                                            dev_of_group, n_dev, partials, dev_status);              \
+        mha_fused_kernel<T, I, false><<<grid_f, 256, smem_f, st>>>(                                                   \
+            d, H, dh, sh.max_len, pos, static_cast<const T*>(Wp), static_cast<const T*>(x), static_cast<const T*>(Kc), \
+            static_cast<const T*>(Vc), keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, nullptr, nullptr,  \
+            nullptr, nullptr);                                                                                       \
         break;
         switch (iters_f) {
             HALO_MHA_FUSED(1)
@@ -671,4 +706,64 @@ extern "C" halo_status halo_group_mha(const halo_mha_shape* shape, const void* W
                                               n_dev, partials, ws, dev_status, st);
     return group_mha_typed<float>(*shape, W_packed, x, K_cache, V_cache, pos, keep_list, n_keep, dev_of_group, n_dev,
                                   partials, ws, dev_status, st);
+}
+
+template <typename T>
+static halo_status mha_block_typed(const halo_mha_shape& sh, const void* Wp, const void* Wk, const void* Wv, const void* x,
+                                   void* Kc, void* Vc, int pos, const int32_t* keep_list, const int32_t* n_keep,
+                                   const int32_t* dev_of_group, int n_dev, float* partials, uint32_t* dev_status,
+                                   cudaStream_t st, bool already_zero) {
+    constexpr int E = Elem<T>::kPerChunk;
+    const int d = sh.d_model, H = sh.n_heads, dh = sh.head_dim;
+    if (!already_zero &&
+        cudaMemsetAsync(partials, 0, sizeof(float) * static_cast<size_t>(n_dev + 1) * d, st) != cudaSuccess)
+        return HALO_ERR_CUDA;
+    const int iters = (d / E + 255) / 256;
+    const dim3 grid(kMhaCluster, H);
+    const size_t smem = sizeof(float) * d;
+#define HALO_MHA_BLOCK(I)                                                                                            \
+    case I:                                                                                                          \
+        mha_fused_kernel<T, I, true><<<grid, 256, smem, st>>>(                                                       \
+            d, H, dh, sh.max_len, pos, static_cast<const T*>(Wp), static_cast<const T*>(x), static_cast<const T*>(Kc), \
+            static_cast<const T*>(Vc), keep_list, n_keep, dev_of_group, n_dev, partials, dev_status,                  \
+            static_cast<const T*>(Wk), static_cast<const T*>(Wv), static_cast<T*>(Kc), static_cast<T*>(Vc));          \
+        break;
+    switch (iters) {
+        HALO_MHA_BLOCK(1)
+        HALO_MHA_BLOCK(2)
+        HALO_MHA_BLOCK(3)
+        HALO_MHA_BLOCK(4)
+        default: return HALO_ERR_SHAPE;
+    }
+#undef HALO_MHA_BLOCK
+    HALO_CHECK_LAUNCH();
+    return HALO_OK;
+}
+
+halo_status halo::launch_mha_block(const halo_mha_shape& sh, const void* W_packed, const void* Wk, const void* Wv, const void* x,
+                                   void* K_cache, void* V_cache, int pos, const int32_t* keep_list, const int32_t* n_keep,
+                                   const int32_t* dev_of_group, int n_dev, float* partials, uint32_t* dev_status,
+                                   cudaStream_t st, bool already_zero) {
+    if (sh.wdtype == HALO_BF16)
+        return mha_block_typed<__nv_bfloat16>(sh, W_packed, Wk, Wv, x, K_cache, V_cache, pos, keep_list, n_keep, dev_of_group,
+                                              n_dev, partials, dev_status, st, already_zero);
+    return mha_block_typed<float>(sh, W_packed, Wk, Wv, x, K_cache, V_cache, pos, keep_list, n_keep, dev_of_group, n_dev,
+                                  partials, dev_status, st, already_zero);
+}
+
+extern "C" halo_status halo_mha_block(const halo_mha_shape* shape, const void* W_packed, const void* Wk, const void* Wv,
+                                      const void* x, void* K_cache, void* V_cache, int pos, const int32_t* keep_list,
+                                      const int32_t* n_keep, const int32_t* dev_of_group, int n_dev, float* partials,
+                                      uint32_t* dev_status, void* stream) {
+    halo_status rc = check_mha_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (!W_packed || !Wk || !Wv || !x || !K_cache || !V_cache || !keep_list || !n_keep || !partials) return HALO_ERR_ARG;
+    if (pos < 0 || pos >= shape->max_len) return HALO_ERR_ARG;
+    if (n_dev < 0 || n_dev > HALO_MAX_DEVICES || (!dev_of_group && n_dev != 0)) return HALO_ERR_ARG;
+    if (shape->head_dim % (2 * kMhaCluster) != 0) return HALO_ERR_SHAPE;
+    if (!aligned16(W_packed) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(x) || !aligned16(K_cache) ||
+        !aligned16(V_cache) || !aligned16(partials))
+        return HALO_ERR_ALIGN;
+    return halo::launch_mha_block(*shape, W_packed, Wk, Wv, x, K_cache, V_cache, pos, keep_list, n_keep, dev_of_group, n_dev,
+                                  partials, dev_status, static_cast<cudaStream_t>(stream), false);
 }

@@ -87,7 +87,7 @@ def test_block_stack_teacher_forced(name, layers, H, dh, steps, pos0):
     V_start = [hb(b["V"]) for b in blocks]
     step0 = 3
     h0, h_out, logits, ta, tf = run(wl, stack, H, vocab, steps, pos0, step0)
-    assert stack.last_launches() > steps * layers * 8
+    assert stack.last_launches() >= steps * layers * 4             # one launch per step of the path
     L, G, d, nf, na = wl.n_layers, wl.n_groups, wl.d_model, wl.n_dev, 3
     Kc, Vc = [k.copy() for k in K_start], [v.copy() for v in V_start]
     lost_a = lost_f = 0

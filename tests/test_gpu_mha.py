@@ -119,3 +119,58 @@ def test_mha_argument_checks():
     ok = B.mha_shape(512, 8, 64, 64, B.BF16)
     with pytest.raises(B.HaloError):
         B.halo_mha_kv_append(ok, t, t, t, 64, t, t)   # position beyond the cache
+
+
+@pytest.mark.parametrize("dtype,d,H,dh,L,positions", [("f32", 64, 4, 16, 40, (0, 7, 39)), ("bf16", 512, 8, 64, 300, (0, 128, 299)),
+                                                      ("bf16", 4096, 32, 128, 1100, (3, 1023, 1099)),
+                                                      ("bf16", 2048, 32, 64, 600, (511,))])
+def test_mha_block_one_launch_matches_oracle_and_the_two_calls(dtype, d, H, dh, L, positions):
+    """halo_mha_block: keys / values of every head appended and the kept heads attended in one launch.  The cache rows
+    it writes are the bits halo_mha_kv_append writes (and within a rounding step of the oracle's); the partials are
+    the oracle's from those cache bytes, also when the token's own position is the only one (pos 0) and for heads
+    that are not kept (their keys and values must still land)."""
+    wl = _wl(dtype, d)
+    code = U.dtype_code(wl)
+    sh = B.mha_shape(d, H, dh, L, code)
+    Wq, Wk, Wv, Wo = synth.mha_matrices(wl, 1, H, DEV)
+    Wp = torch.empty((H, 2, dh, d), dtype=wl.torch_dtype, device=DEV)
+    B.halo_pack_mha_weights(sh, Wq, Wo, Wp)
+    hb = synth.host_bits
+    Wp_ref = hb(Wp)
+    K, V = _caches(wl, H, L, dh, L)
+    tol = U.tol_for(wl)
+    dev = np.array([(-1, 0, 1, 2)[h % 4] for h in range(H)], dtype=np.int32)
+    dg = torch.as_tensor(dev, device=DEV)
+    ws = torch.empty(B.halo_group_mha_workspace_bytes(sh), dtype=torch.uint8, device=DEV)
+    for pos in positions:
+        for keep in (list(range(H)), [h for h in range(H) if h % 3 != 1], [H - 1], []):
+            x = synth.activation(wl, 90 + pos + len(keep), DEV)
+            K2, V2 = K.clone(), V.clone()
+            kl = torch.full((H,), -1, dtype=torch.int32, device=DEV)
+            if keep:
+                kl[: len(keep)] = torch.as_tensor(keep, dtype=torch.int32, device=DEV)
+            nk = torch.tensor([len(keep)], dtype=torch.int32, device=DEV)
+            P = torch.full((4, d), float("nan"), dtype=torch.float32, device=DEV)
+            status = torch.zeros(1, dtype=torch.int32, device=DEV)
+            B.halo_mha_block(sh, Wp, Wk, Wv, x, K, V, pos, kl, nk, dg, 3, P, status)
+            # the two calls, on copies of the caches
+            B.halo_mha_kv_append(sh, Wk, Wv, x, pos, K2, V2)
+            P2 = torch.empty_like(P)
+            B.halo_group_mha(sh, Wp, x, K2, V2, pos, kl, nk, dg, 3, P2, ws, status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            assert torch.equal(K.view(torch.uint8), K2.view(torch.uint8)) and torch.equal(V.view(torch.uint8), V2.view(torch.uint8))
+            Kh, Vh = hb(K), hb(V)
+            Kr, Vr = Kh.copy(), Vh.copy()
+            R.mha_kv_append(hb(Wk), hb(Wv), hb(x)[0], pos, Kr, Vr)
+            kk = R.to_f64(Kr[:, pos])
+            rt = 1e-5 if dtype == "f32" else 2 ** -7
+            assert np.abs(R.to_f64(Kh[:, pos]) - kk).max() <= rt * np.abs(kk).max()
+            assert np.abs(R.to_f64(Vh[:, pos]) - R.to_f64(Vr[:, pos])).max() <= rt * np.abs(kk).max()
+            if not keep:
+                assert (P == 0).all().item()
+                continue
+            ref = R.group_mha(Wp_ref, hb(x)[0], Kh, Vh, pos, keep, dev, 3)
+            rms = np.sqrt(np.mean(ref.sum(0) ** 2))
+            assert np.abs(P.cpu().numpy() - ref).max() <= tol * rms, (pos, len(keep))
+            assert np.abs(P2.cpu().numpy() - ref).max() <= tol * rms

@@ -121,7 +121,8 @@ halo_status launch_group_ffn_decode(const halo_ffn_shape& sh, const void* W, con
                                     bool already_zero = false);
 halo_status launch_group_ffn_stream(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                     const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
-                                    int n_dev, float* partials, uint32_t* dev_status, cudaStream_t st);
+                                    int n_dev, float* partials, uint32_t* dev_status, cudaStream_t st,
+                                    bool zero_first = false);
 // Prefill form (tensor cores); workspace = bf16 [n_tok][d_ffn]; partials must already be zero.
 bool prefill_supported(const halo_ffn_shape& sh, int n_tok);
 size_t prefill_workspace_bytes(const halo_ffn_shape& sh, int n_tok);
@@ -144,6 +145,9 @@ halo_status launch_glue(int d, int n_tok, halo_dtype xdtype, const float* h, con
 halo_status launch_merge_glue(const float* partials, const uint8_t* arrived, int n_dev, int n_tok, int d,
                               halo_dtype xdtype, const float* h, float* h_out, void* x_out, float* y_tap,
                               cudaStream_t st, bool zero_after = false);
+// Zero-fill of partial slots by a kernel that releases a programmatically dependent launch at once (the dependent
+// kernel executes griddepcontrol.wait before it first adds to the slots); n_floats a multiple of 4.
+halo_status launch_zero_partials(float* partials, size_t n_floats, cudaStream_t st);
 // halo_mha_block without argument checks; already_zero: the caller guarantees that `partials` is zero.
 halo_status launch_mha_block(const halo_mha_shape& sh, const void* W_packed, const void* Wk, const void* Wv, const void* x,
                              void* K_cache, void* V_cache, int pos, const int32_t* keep_list, const int32_t* n_keep,

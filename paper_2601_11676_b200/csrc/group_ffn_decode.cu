@@ -220,12 +220,12 @@ static halo_status launch_typed(const halo_ffn_shape& sh, const void* W, const v
 halo_status launch_group_ffn_decode(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                     const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
                                     int n_dev, float* partials, uint32_t* dev_status, cudaStream_t st, bool already_zero) {
+    // bf16 shapes with a streaming configuration take the shared-memory ring kernel (which zeroes under its own stream)
+    const halo_status fast = launch_group_ffn_stream(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials,
+                                                     dev_status, st, !already_zero);
+    if (fast != HALO_ERR_UNIMPLEMENTED) return fast;
     const size_t bytes = sizeof(float) * static_cast<size_t>(n_dev + 1) * n_tok * sh.d_model;
     if (!already_zero && cudaMemsetAsync(partials, 0, bytes, st) != cudaSuccess) return HALO_ERR_CUDA;
-    // bf16 shapes with a streaming configuration take the shared-memory ring kernel
-    const halo_status fast = launch_group_ffn_stream(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials,
-                                                     dev_status, st);
-    if (fast != HALO_ERR_UNIMPLEMENTED) return fast;
     if (sh.wdtype == HALO_BF16)
         return launch_typed<__nv_bfloat16>(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials,
                                            dev_status, st);

@@ -55,6 +55,10 @@ group_ffn_stream_kernel(int d, int S, int G, const __nv_bfloat16* __restrict__ W
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tok = blockIdx.y;
+    // A following launch that declares itself a programmatic dependent (the zero-fill of the next call of this entry
+    // point does) may be scheduled as this kernel's thread blocks retire; it waits for this kernel's completion itself
+    // before it touches anything.  Ordinary launches behind this kernel are not affected.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     int nk = *n_keep_ptr;
     if (nk < 0 || nk > G) {
@@ -141,7 +145,11 @@ group_ffn_stream_kernel(int d, int S, int G, const __nv_bfloat16* __restrict__ W
     int cur_slot = -1;
     const size_t slot_stride = static_cast<size_t>(n_tok) * d;
 
+    bool dep_waited = false;
     auto flush = [&](int slot) {
+        // The zero-fill of `partials` may still be running (this kernel is launched as its programmatic dependent, so
+        // that the weight stream starts under it): nothing is added before it has completed.  A no-op otherwise.
+        if (!dep_waited) { asm volatile("griddepcontrol.wait;" ::: "memory"); dep_waited = true; }
         float* dst = partials + static_cast<size_t>(slot) * slot_stride + static_cast<size_t>(tok) * d;
 #pragma unroll
         for (int p = 0; p < P2; ++p) {
@@ -198,6 +206,32 @@ group_ffn_stream_kernel(int d, int S, int G, const __nv_bfloat16* __restrict__ W
     if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
 }
 
+// Zero-fill of the partial slots; lets the dependent streaming kernel start at once.
+__global__ void __launch_bounds__(256)
+zero_partials_kernel(float4* __restrict__ p, size_t n4) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // itself launched as a programmatic dependent: whatever ran before it on the stream (say the previous call's
+    // streaming kernel, which may still be adding to these very slots) must have completed before anything is zeroed
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < n4) p[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+}
+
+halo_status launch_zero_partials(float* partials, size_t n_floats, cudaStream_t st) {
+    const size_t n4 = n_floats / 4;     // a multiple of 4: d_model % 8 == 0
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>((n4 + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, zero_partials_kernel, reinterpret_cast<float4*>(partials), n4) == cudaSuccess ? HALO_OK
+                                                                                                                 : HALO_ERR_CUDA;
+}
+
 // ---- host side ---------------------------------------------------------------------------------------------
 
 namespace {
@@ -220,7 +254,7 @@ bool pick_stream_config(int d, int S, StreamConfig* cfg) {
 template <int NB, int XC, int P2, int REP, int STAGES>
 halo_status launch_stream_cfg(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                               const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group, int n_dev,
-                              float* partials, uint32_t* dev_status, cudaStream_t st) {
+                              float* partials, uint32_t* dev_status, cudaStream_t st, bool zero_first) {
     auto kernel = group_ffn_stream_kernel<NB, XC, P2, REP, STAGES>;
     const size_t smem = 1024 + static_cast<size_t>(STAGES) * 3 * NB * sh.d_model * 2;
     static bool configured[64] = {};
@@ -230,27 +264,46 @@ halo_status launch_stream_cfg(const halo_ffn_shape& sh, const void* W, const voi
     const int G = sh.d_ffn / sh.group_size;
     const long long max_batches = static_cast<long long>(G) * (sh.group_size / NB);
     dim3 grid(static_cast<unsigned>(std::min<long long>(max_batches, sms)), n_tok);
-    kernel<<<grid, kStreamThreads, smem, st>>>(sh.d_model, sh.group_size, G, static_cast<const __nv_bfloat16*>(W),
-                                               static_cast<const __nv_bfloat16*>(x), keep_list, n_keep, dev_of_group,
-                                               n_dev, n_tok, partials, dev_status);
-    HALO_CHECK_LAUNCH();
-    return HALO_OK;
+    if (!zero_first) {
+        kernel<<<grid, kStreamThreads, smem, st>>>(sh.d_model, sh.group_size, G, static_cast<const __nv_bfloat16*>(W),
+                                                   static_cast<const __nv_bfloat16*>(x), keep_list, n_keep, dev_of_group,
+                                                   n_dev, n_tok, partials, dev_status);
+        HALO_CHECK_LAUNCH();
+        return HALO_OK;
+    }
+    // zero-fill as a kernel that releases its dependent at once, then the streaming kernel as that dependent: its
+    // prologue and its weight stream run under the zero-fill; it waits for it only before it first adds to `partials`
+    if (launch_zero_partials(partials, static_cast<size_t>(n_dev + 1) * n_tok * sh.d_model, st) != HALO_OK) return HALO_ERR_CUDA;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kStreamThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, sh.d_model, sh.group_size, G, static_cast<const __nv_bfloat16*>(W),
+                                               static_cast<const __nv_bfloat16*>(x), keep_list, n_keep, dev_of_group, n_dev,
+                                               n_tok, partials, dev_status);
+    return err == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
 }
 
 }  // namespace
 
 // Returns HALO_ERR_UNIMPLEMENTED when the shape has no streaming configuration (the caller falls back to the
-// generic kernel).  partials must already be zero.
+// generic kernel, having zeroed nothing).  zero_first: the call zeroes partials itself; otherwise they must be zero.
 halo_status launch_group_ffn_stream(const halo_ffn_shape& sh, const void* W, const void* x, int n_tok,
                                     const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
-                                    int n_dev, float* partials, uint32_t* dev_status, cudaStream_t st) {
+                                    int n_dev, float* partials, uint32_t* dev_status, cudaStream_t st, bool zero_first) {
     StreamConfig cfg;
     if (sh.wdtype != HALO_BF16 || !pick_stream_config(sh.d_model, sh.group_size, &cfg)) return HALO_ERR_UNIMPLEMENTED;
     switch (sh.d_model) {
-        case 2048: return launch_stream_cfg<4, 4, 1, 2, 4>(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, st);
-        case 4096: return launch_stream_cfg<2, 4, 1, 1, 4>(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, st);
-        case 5120: return launch_stream_cfg<2, 5, 2, 1, 3>(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, st);
-        case 8192: return launch_stream_cfg<1, 4, 2, 1, 4>(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, st);
+        case 2048: return launch_stream_cfg<4, 4, 1, 2, 4>(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, st, zero_first);
+        case 4096: return launch_stream_cfg<2, 4, 1, 1, 4>(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, st, zero_first);
+        case 5120: return launch_stream_cfg<2, 5, 2, 1, 3>(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, st, zero_first);
+        case 8192: return launch_stream_cfg<1, 4, 2, 1, 4>(sh, W, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, st, zero_first);
     }
     return HALO_ERR_UNIMPLEMENTED;
 }

@@ -346,6 +346,7 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
     const int chunks = d / E;
     int h, slot = 0;
     if constexpr (APPEND) {
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see group_ffn_stream_kernel
         h = blockIdx.y;
         // keys and values of this token for head h, rows j0 .. j0 + rows of each, two rows per warp and turn
         stage_x(x, xs, d);
@@ -534,6 +535,8 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
             }
         }
     }
+    // the zero-fill of the slots may still be running when this kernel was launched as its programmatic dependent
+    if constexpr (APPEND) asm volatile("griddepcontrol.wait;" ::: "memory");
     float* dst = partials + static_cast<size_t>(slot) * d;
 #pragma unroll
     for (int i = 0; i < ITERS; ++i) {
@@ -715,18 +718,29 @@ static halo_status mha_block_typed(const halo_mha_shape& sh, const void* Wp, con
                                    cudaStream_t st, bool already_zero) {
     constexpr int E = Elem<T>::kPerChunk;
     const int d = sh.d_model, H = sh.n_heads, dh = sh.head_dim;
-    if (!already_zero &&
-        cudaMemsetAsync(partials, 0, sizeof(float) * static_cast<size_t>(n_dev + 1) * d, st) != cudaSuccess)
-        return HALO_ERR_CUDA;
+    // the zero-fill releases this launch at once: the row products and the attention run under it
+    if (!already_zero && launch_zero_partials(partials, static_cast<size_t>(n_dev + 1) * d, st) != HALO_OK) return HALO_ERR_CUDA;
     const int iters = (d / E + 255) / 256;
-    const dim3 grid(kMhaCluster, H);
-    const size_t smem = sizeof(float) * d;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(kMhaCluster, H);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = sizeof(float) * d;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = already_zero ? 0 : 1;
+    const T* Wp_t = static_cast<const T*>(Wp); const T* x_t = static_cast<const T*>(x);
+    const T* Kc_t = static_cast<const T*>(Kc); const T* Vc_t = static_cast<const T*>(Vc);
+    const T* Wk_t = static_cast<const T*>(Wk); const T* Wv_t = static_cast<const T*>(Wv);
+    T* Kw_t = static_cast<T*>(Kc); T* Vw_t = static_cast<T*>(Vc);
+    const int Lmax = sh.max_len;
+    cudaError_t err = cudaSuccess;
 #define HALO_MHA_BLOCK(I)                                                                                            \
     case I:                                                                                                          \
-        mha_fused_kernel<T, I, true><<<grid, 256, smem, st>>>(                                                       \
-            d, H, dh, sh.max_len, pos, static_cast<const T*>(Wp), static_cast<const T*>(x), static_cast<const T*>(Kc), \
-            static_cast<const T*>(Vc), keep_list, n_keep, dev_of_group, n_dev, partials, dev_status,                  \
-            static_cast<const T*>(Wk), static_cast<const T*>(Wv), static_cast<T*>(Kc), static_cast<T*>(Vc));          \
+        err = cudaLaunchKernelEx(&cfg, mha_fused_kernel<T, I, true>, d, H, dh, Lmax, pos, Wp_t, x_t, Kc_t, Vc_t,      \
+                                 keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, Wk_t, Wv_t, Kw_t, Vw_t); \
         break;
     switch (iters) {
         HALO_MHA_BLOCK(1)
@@ -736,8 +750,7 @@ static halo_status mha_block_typed(const halo_mha_shape& sh, const void* Wp, con
         default: return HALO_ERR_SHAPE;
     }
 #undef HALO_MHA_BLOCK
-    HALO_CHECK_LAUNCH();
-    return HALO_OK;
+    return err == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
 }
 
 halo_status halo::launch_mha_block(const halo_mha_shape& sh, const void* W_packed, const void* Wk, const void* Wv, const void* x,

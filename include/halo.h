@@ -468,7 +468,8 @@ halo_status halo_stack_set_mode(halo_stack* stack, int mode);
  *   "prefill_kcuts" (1..16), "prefill_kratio_percent" (30..100)   prompt FFN: K runs per down-projection tile and
  *                                     the ratio between consecutive runs
  *   "mha_three_launches" (0/1)        halo_group_mha as three launches instead of one
- *   "i4_no_ring" (0/1/3)              halo_group_ffn_i4: 0 shared-memory ring (default), 1 plain loads, 3 ring with
+ *   "i4_no_ring" (0..3)               halo_group_ffn_i4: 0 shared-memory ring with two thread blocks per SM
+ *                                     (default), 1 plain loads, 2 ring with one thread block per SM, 3 ring with
  *                                     the products on the legacy tensor-core path (mma.sync; slower here)
  * HALO_ERR_ARG for an unknown name or a value outside the stated range. */
 halo_status halo_set_option(const char* name, int value);

@@ -31,6 +31,20 @@ __device__ __forceinline__ uint32_t nibble_pair_bf16(uint32_t word, int k) {
     return ((word >> (4 * k)) & 0x000F000Fu) | 0x43004300u;      // {128 + nibble k, 128 + nibble k+4} as bf16x2
 }
 
+// The same pair with the right shift done as the high half of a product (word * 2^(32 - 4k)), which runs on the
+// multiply-add pipe; the logic pipe, half as wide, is what bounds the unpacking.  `mul` = 2^(32 - 4k) must reach the
+// kernel as a run-time value, else the compiler turns the product back into a shift.
+__device__ __forceinline__ uint32_t nibble_pair_mulhi(uint32_t word, uint32_t mul) {
+    return (__umulhi(word, mul) & 0x000F000Fu) | 0x43004300u;
+}
+
+// Mask and exponent bits as run-time values held in registers: with two immediates the "and, then or" is two logic
+// instructions, with register operands it is one three-input instruction.
+struct PairBits { uint32_t mask, magic; };
+__device__ __forceinline__ uint32_t nibble_pair_r(uint32_t shifted_word, const PairBits& pb) {
+    return (shifted_word & pb.mask) | pb.magic;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 quantize_i4_kernel(int d, long long n_rows, const T* __restrict__ W, uint8_t* __restrict__ Q,
@@ -293,20 +307,25 @@ group_ffn_i4_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, const __
 }
 
 // ------------------------------------------------------------------------------------------------------------
-// Ring form of the same computation for d_model 2048 / 4096 (group size a multiple of 8): one thread block per SM,
-// a producer warp streams batches of 8 neurons (their gate, up and down code rows and the three runs of scales:
-// six bulk copies per stage) into a shared-memory ring, 512 consumer threads work from shared memory, so no
-// consumer ever waits on a global load and the bytes in flight are set by the ring depth.
-//   phase 1  one warp per row (8 gate + 8 up rows); the lane's chunks against x kept in shared memory in the
+// Ring form of the same computation for d_model 2048 / 4096 (group size a multiple of 8): a producer warp streams
+// batches of 8 neurons (their gate, up and down code rows and the three runs of scales: six bulk copies per stage)
+// into a shared-memory ring, the consumer warps work from shared memory, so no consumer ever waits on a global load
+// and the bytes in flight are set by the ring depth.
+//   phase 1  a warp per row (or per gate/up pair of rows); the lane's chunks against x kept in shared memory in the
 //            nibble pairing; the two products of a neuron meet in shared memory;
 //   phase 2  REP replicas of d/16 threads; a replica takes every REP-th down row, a thread owns 16 columns.
+// The unpacking is bound by the logic pipe (half as wide as the multiply-add pipe), so work is moved off it: mask and
+// exponent bits sit in registers (one three-input logic instruction per pair of weights), some right shifts are done
+// as high halves of products, the lower element of a pair is moved up by a multiplication, and the upper element is
+// used without masking the lower one off (its surplus is subtracted once per flush).
 // Every mbarrier wait is bounded; on a timeout the block flags HALO_DEV_TIMEOUT, drains its copies and returns.
 // ------------------------------------------------------------------------------------------------------------
 constexpr int kRingNB = 8;
-constexpr int kRingConsumers = 512;
+constexpr int kRingConsumers = 512;            // consumer threads of the tensor-core form further down
 constexpr int kRingConsumerWarps = kRingConsumers / 32;
-constexpr int kRingThreads = kRingConsumers + 32;
-__device__ __forceinline__ void ring_consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kRingConsumers) : "memory"); }
+template <int N>
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void ring_consumer_barrier() { consumer_barrier<kRingConsumers>(); }
 
 struct RingHeader {
     uint64_t full[8];
@@ -316,15 +335,24 @@ struct RingHeader {
     int pad[3];
     __align__(16) float red[2][2 * kRingNB];
 };
+constexpr int kRingHeaderBytes = 1024;
+static_assert(sizeof(RingHeader) <= kRingHeaderBytes, "ring header region");
 
-template <int XC, int REP, int STAGES>
-__global__ void __launch_bounds__(kRingThreads, 1)
+// NCW consumer warps + one producer warp.  NCW = 8 with two stages is sized so that TWO thread blocks share an SM
+// (2 x 113 KB of shared memory, 2 x 288 threads): while one block sits at the barrier between its phases or waits for
+// a stage, the other one computes, and the blocks of the next launch move in as soon as one of this launch leaves.
+// NCW = 16 with four stages is the one-block-per-SM form.  Phase 1: warp w takes rows w, w + NCW, ... of the 16
+// (8 gate, then 8 up), so with NCW = 8 a warp has the gate and the up row of one neuron and reads x once for both.
+template <int XC, int REP, int STAGES, int NCW>
+__global__ void __launch_bounds__(NCW * 32 + 32, NCW == 8 ? 2 : 1)
 group_ffn_i4_ring_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, const __nv_bfloat16* __restrict__ scales,
                          const __nv_bfloat16* __restrict__ x_all, const int32_t* __restrict__ keep_list,
                          const int32_t* __restrict__ n_keep_ptr, const int32_t* __restrict__ dev_of_group, int n_dev,
                          int n_tok, float* __restrict__ partials, uint32_t* dev_status) {
     constexpr int NB = kRingNB;
-    static_assert(STAGES <= 8 && NB % REP == 0, "ring / replica shape");
+    constexpr int kConsumers = NCW * 32;
+    constexpr int RPW = 2 * NB / NCW;            // rows of phase 1 per warp
+    static_assert(STAGES <= 8 && NB % REP == 0 && (NCW == 8 || NCW == 16), "ring / replica shape");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     RingHeader& hd = *reinterpret_cast<RingHeader*>(smem_raw);
     const int chunks16 = d / 32, chunks8 = d / 16, nb = d / kQBlock;
@@ -332,17 +360,27 @@ group_ffn_i4_ring_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, con
     const uint32_t plane_bytes = row_bytes * NB;                 // codes of one of gate / up / down for a batch
     const uint32_t sc_bytes = static_cast<uint32_t>(nb) * 2u * NB;   // scales of one plane of a batch
     const uint32_t stage_bytes = 3u * (plane_bytes + sc_bytes);
-    uint4* xp = reinterpret_cast<uint4*>(smem_raw + 1024);                                  // [4][chunks16]
-    float* xsum = reinterpret_cast<float*>(smem_raw + 1024 + static_cast<size_t>(d) * 2);   // [chunks16]
-    unsigned char* ring = smem_raw + 1024 + static_cast<size_t>(d) * 2 + ((static_cast<size_t>(chunks16) * 4 + 127) & ~size_t(127));
+    uint4* xp = reinterpret_cast<uint4*>(smem_raw + kRingHeaderBytes);                                  // [4][chunks16]
+    float* xsum = reinterpret_cast<float*>(smem_raw + kRingHeaderBytes + static_cast<size_t>(d) * 2);   // [chunks16]
+    unsigned char* ring =
+        smem_raw + kRingHeaderBytes + static_cast<size_t>(d) * 2 + ((static_cast<size_t>(chunks16) * 4 + 127) & ~size_t(127));
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int tok = blockIdx.y;
+    // Run-time copies of constants (n_tok > 0, so the added term is zero): the multipliers stand in for shifts (see
+    // nibble_pair_mulhi), and mask / exponent bits held in registers make "and, then or" one instruction (PairBits).
+    const uint32_t rt_zero = static_cast<uint32_t>(n_tok) >> 31;
+    const uint32_t mul1 = 0x10000000u + rt_zero, mul2 = 0x01000000u + rt_zero, mul3 = 0x00100000u + rt_zero;
+    const uint32_t mul16 = 0x00010000u + rt_zero;
+    const PairBits pb{0x000F000Fu + rt_zero, 0x43004300u + rt_zero};
     int nk = *n_keep_ptr;
     if (nk < 0 || nk > G) {
         if (tid == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
         nk = nk < 0 ? 0 : G;
     }
+    // the zero-fill of the partial slots runs ahead of this kernel as a programmatic dependency: released here for the
+    // next call's zero-fill, waited for below before the first sum leaves this block
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int per_group = S / NB;
     const long long total = static_cast<long long>(nk) * per_group;  // batches
     const int lo = static_cast<int>(total * blockIdx.x / gridDim.x);
@@ -351,14 +389,14 @@ group_ffn_i4_ring_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, con
     const int n_it = hi - lo;
 
     if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&hd.full[s], 1); mbar_init(&hd.empty[s], kRingConsumerWarps); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&hd.full[s], 1); mbar_init(&hd.empty[s], NCW); }
         hd.abort_flag = 0;
         mbar_fence_init();
     }
     __syncthreads();
     volatile int* abort_flag = &hd.abort_flag;
 
-    if (warp == kRingConsumerWarps) {
+    if (warp == NCW) {
         // ---------------- producer ----------------
         if (lane == 0) {
             int issued = 0;
@@ -406,33 +444,48 @@ group_ffn_i4_ring_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, con
     {   // x in the nibble pairing, and its plain sums per 32 elements
         const uint16_t* xb = reinterpret_cast<const uint16_t*>(x_all + static_cast<size_t>(tok) * d);
         uint32_t* xp_words = reinterpret_cast<uint32_t*>(xp);
-        for (int i = tid; i < d / 2; i += kRingConsumers) {
+        for (int i = tid; i < d / 2; i += kConsumers) {
             const int c = i / 16, r = i - c * 16, w = r >> 2, k = r & 3;
             const uint32_t lo16 = xb[32 * c + 8 * w + k], hi16 = xb[32 * c + 8 * w + k + 4];
             xp_words[(static_cast<size_t>(w) * chunks16 + c) * 4 + k] = lo16 | (hi16 << 16);
         }
-        for (int c = tid; c < chunks16; c += kRingConsumers) {
+        for (int c = tid; c < chunks16; c += kConsumers) {
             float sx = 0.0f;
             for (int e = 0; e < 32; ++e) sx += __bfloat162float(x_all[static_cast<size_t>(tok) * d + 32 * c + e]);
             xsum[c] = sx;
         }
     }
-    ring_consumer_barrier();
-    const int row = warp;                                  // phase 1: rows 0..7 gate, 8..15 up
-    const int rep = tid / (kRingConsumers / REP);          // phase 2 replica and 8-byte column chunk
-    const int col = tid % (kRingConsumers / REP);
+    consumer_barrier<kConsumers>();
+    const int rep = tid / (kConsumers / REP);              // phase 2 replica and 8-byte column chunk
+    const int col = tid % (kConsumers / REP);
     float acc[16], corr = 0.0f;
 #pragma unroll
     for (int e = 0; e < 16; ++e) acc[e] = 0.0f;
     int cur_slot = -1;
     const size_t slot_stride = static_cast<size_t>(n_tok) * d;
 
+    bool dep_waited = false;
     auto flush = [&](int slot) {
+        if (!dep_waited) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            dep_waited = true;
+        }
         if (col < chunks8) {
             float* dst = partials + static_cast<size_t>(slot) * slot_stride + static_cast<size_t>(tok) * d + col * 16;
             const float off = kNibbleBias * corr;
+            // upper elements (e + 4): sum f * (128 + 0x4300 / 65536 + n_hi + n_lo / 65536), n_lo from element e
+            const float off_hi = (kNibbleBias + 17152.0f / 65536.0f) * corr;
 #pragma unroll
-            for (int e = 0; e < 16; e += 4) red_add_v4f(dst + e, acc[e] - off, acc[e + 1] - off, acc[e + 2] - off, acc[e + 3] - off);
+            for (int v = 0; v < 16; v += 8) {
+                float lo4[4], hi4[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    lo4[k] = acc[v + k] - off;
+                    hi4[k] = (acc[v + k + 4] - off_hi) - (acc[v + k] - 128.0f * corr) * (1.0f / 65536.0f);
+                }
+                red_add_v4f(dst + v, lo4[0], lo4[1], lo4[2], lo4[3]);
+                red_add_v4f(dst + v + 4, hi4[0], hi4[1], hi4[2], hi4[3]);
+            }
         }
         corr = 0.0f;
 #pragma unroll
@@ -453,28 +506,44 @@ group_ffn_i4_ring_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, con
                 cur_slot = slot;
             }
             // phase 1: code rows 0..15 of the stage are the 8 gate rows then the 8 up rows (planes 0, 1 adjacent)
-            const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(row) * row_bytes);
-            const __nv_bfloat16* rs = stage_sc + static_cast<size_t>(row) * nb;
-            float a = 0.0f;
+            float a[RPW];
+#pragma unroll
+            for (int r = 0; r < RPW; ++r) a[r] = 0.0f;
 #pragma unroll
             for (int u = 0; u < XC; ++u) {
                 const int c = lane + 32 * u;
-                const uint4 w4 = rp[c];
-                const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
-                float t0 = 0.0f, t1 = 0.0f;
+                uint32_t ww[RPW][4];
+                float t0[RPW], t1[RPW];
+#pragma unroll
+                for (int r = 0; r < RPW; ++r) {
+                    const uint4 w4 = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(warp + r * NCW) * row_bytes)[c];
+                    ww[r][0] = w4.x; ww[r][1] = w4.y; ww[r][2] = w4.z; ww[r][3] = w4.w;
+                    t0[r] = 0.0f; t1[r] = 0.0f;
+                }
 #pragma unroll
                 for (int w = 0; w < 4; ++w) {
                     const uint4 xq = xp[static_cast<size_t>(w) * chunks16 + c];
-                    const uint32_t xk[4] = {xq.x, xq.y, xq.z, xq.w};
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) fma_bf16x2(nibble_pair_bf16(ww[w], k), xk[k], t0, t1);
+                    for (int r = 0; r < RPW; ++r) {
+                        fma_bf16x2(nibble_pair_r(ww[r][w], pb), xq.x, t0[r], t1[r]);
+                        fma_bf16x2(nibble_pair_r(ww[r][w] >> 4, pb), xq.y, t0[r], t1[r]);
+                        fma_bf16x2(nibble_pair_r(ww[r][w] >> 8, pb), xq.z, t0[r], t1[r]);
+                        fma_bf16x2(nibble_pair_r(__umulhi(ww[r][w], mul3), pb), xq.w, t0[r], t1[r]);
+                    }
                 }
-                a = fmaf(__bfloat162float(rs[c >> 2]), (t0 + t1) - kNibbleBias * xsum[c], a);
+                const float off = kNibbleBias * xsum[c];
+#pragma unroll
+                for (int r = 0; r < RPW; ++r)
+                    a[r] = fmaf(__bfloat162float(stage_sc[static_cast<size_t>(warp + r * NCW) * nb + (c >> 2)]),
+                                (t0[r] + t1[r]) - off, a[r]);
             }
-            a = warp_sum(a);
-            if (lane == 0) red[row] = a;
+#pragma unroll
+            for (int r = 0; r < RPW; ++r) {
+                a[r] = warp_sum(a[r]);
+                if (lane == 0) red[warp + r * NCW] = a[r];
+            }
         }
-        ring_consumer_barrier();
+        consumer_barrier<kConsumers>();
         if (slot >= 0 && col < chunks8) {
             // phase 2: this replica's down rows, 16 columns of each
             const unsigned char* down = stage + 2 * plane_bytes;
@@ -487,14 +556,19 @@ group_ffn_i4_ring_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, con
                 corr += f;
                 const uint2 w2 = reinterpret_cast<const uint2*>(down + static_cast<size_t>(j) * row_bytes)[col];
                 const uint32_t words[2] = {w2.x, w2.y};
+                // The pair register itself, read as fp32, is 128 + (upper nibble) + (0x4300 + lower nibble) / 65536: it is
+                // used as it stands for the upper element (no mask), and the surplus is taken off once, at the flush.
 #pragma unroll
-                for (int v = 0; v < 2; ++v)
+                for (int v = 0; v < 2; ++v) {
+                    const uint32_t pk[4] = {nibble_pair_r(words[v], pb), nibble_pair_r(__umulhi(words[v], mul1), pb),
+                                            nibble_pair_r(__umulhi(words[v], mul2), pb),
+                                            nibble_pair_r(__umulhi(words[v], mul3), pb)};
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
-                        const uint32_t p = nibble_pair_bf16(words[v], k);
-                        acc[8 * v + k] = fmaf(f, __uint_as_float(p << 16), acc[8 * v + k]);
-                        acc[8 * v + k + 4] = fmaf(f, __uint_as_float(p & 0xffff0000u), acc[8 * v + k + 4]);
+                        acc[8 * v + k] = fmaf(f, __uint_as_float(pk[k] * mul16), acc[8 * v + k]);
+                        acc[8 * v + k + 4] = fmaf(f, __uint_as_float(pk[k]), acc[8 * v + k + 4]);
                     }
+                }
             }
         }
         __syncwarp();
@@ -502,6 +576,14 @@ group_ffn_i4_ring_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, con
     }
     if (cur_slot >= 0) flush(cur_slot);
     if (tid == 0 && *abort_flag) flag_status(dev_status, HALO_DEV_TIMEOUT);
+}
+
+__device__ __forceinline__ void mma_16816_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -522,14 +604,6 @@ group_ffn_i4_ring_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, con
 //            to bf16 rounding.  The column sums stay in the MMA accumulators across batches.
 // Rows are staged with a pitch of (d/2 + 16) bytes so that the word loads above are free of bank conflicts.
 // ------------------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void mma_16816_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
 struct MmaRingHeader {
     uint64_t full[8];
     uint64_t empty[8];
@@ -827,16 +901,22 @@ extern "C" halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void
     const int d = shape->d_model, S = shape->group_size, G = shape->d_ffn / S;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t bytes = sizeof(float) * static_cast<size_t>(n_dev + 1) * n_tok * d;
-    if (cudaMemsetAsync(partials, 0, bytes, st) != cudaSuccess) return HALO_ERR_CUDA;
+    const int form_early = option_value(OPT_I4_NO_RING);
+    const bool ring_form = (d == 2048 || d == 4096) && S % kRingNB == 0 && form_early != 1 && form_early != 3;
+    if (ring_form) {
+        if (launch_zero_partials(partials, bytes / sizeof(float), st) != HALO_OK) return HALO_ERR_CUDA;
+    } else if (cudaMemsetAsync(partials, 0, bytes, st) != cudaSuccess) {
+        return HALO_ERR_CUDA;
+    }
     const uint8_t* q = static_cast<const uint8_t*>(Q);
     const __nv_bfloat16* sc = static_cast<const __nv_bfloat16*>(scales);
     const __nv_bfloat16* xt = static_cast<const __nv_bfloat16*>(x);
     int dev = 0, sms = kSmCount;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const bool no_ring = option_value(OPT_I4_NO_RING) == 1;
-    // 3: ring with the products on the tensor cores.  Correct, and measured SLOWER than the CUDA-core ring (61 against
-    // 35 us on the 7B block): mma.sync is the legacy tensor path on this GPU, so it is kept as an option only.
-    const int form = option_value(OPT_I4_NO_RING);
+    // 3: ring with the products on the tensor cores.  Correct, and measured SLOWER than the CUDA-core ring: with one
+    // token only one of the 8 columns of an m16n8k16 MMA carries data, and at the rate of the legacy mma.sync path of this
+    // GPU (about 8 cycles per instruction and SM sub-partition) that costs as many cycles per weight as the FMA it replaces.
+    const int form = form_early;
     if ((d == 2048 || d == 4096) && S % kRingNB == 0 && form == 3) {
         constexpr int kStages = 4;
         const size_t nbk = static_cast<size_t>(d) / kQBlock;
@@ -859,28 +939,35 @@ extern "C" halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void
         }
         return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
     }
-    if ((d == 2048 || d == 4096) && S % kRingNB == 0 && !no_ring) {
-        // ring form: one block per SM
-        constexpr int kStages = 4;
+    if (ring_form) {
+        // ring form.  Default: two thread blocks per SM (8 consumer warps, 2 stages each); option value 2: one block
+        // per SM (16 consumer warps, 4 stages).
+        const bool two = form_early != 2;
+        const int stages = two ? 2 : 4;
         const size_t stage = 3 * (static_cast<size_t>(d) / 2 * kRingNB + static_cast<size_t>(d) / kQBlock * 2 * kRingNB);
-        const size_t smem_r = 1024 + static_cast<size_t>(d) * 2 + ((static_cast<size_t>(d) / 32 * 4 + 127) & ~size_t(127)) +
-                              kStages * stage;
+        const size_t smem_r = kRingHeaderBytes + static_cast<size_t>(d) * 2 +
+                              ((static_cast<size_t>(d) / 32 * 4 + 127) & ~size_t(127)) + stages * stage;
         const long long batches = static_cast<long long>(G) * (S / kRingNB);
-        const dim3 grid_r(static_cast<unsigned>(std::min<long long>(batches, sms)), n_tok);
-        if (d == 4096) {
-            auto k = group_ffn_i4_ring_kernel<4, 2, kStages>;
-            static bool once[64] = {};
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(batches, static_cast<long long>(sms) * (two ? 2 : 1))), n_tok);
+        cfg.blockDim = dim3(two ? 8 * 32 + 32 : 16 * 32 + 32);
+        cfg.dynamicSmemBytes = smem_r;
+        cfg.stream = st;
+        cudaLaunchAttribute attr{};
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        auto go = [&](auto k, bool (&once)[64]) {
             if (!ensure_dynamic_smem(k, smem_r, once)) return HALO_ERR_CUDA;
-            k<<<grid_r, kRingThreads, smem_r, st>>>(d, S, G, q, sc, xt, keep_list, n_keep, dev_of_group, n_dev, n_tok,
-                                                   partials, dev_status);
-        } else {
-            auto k = group_ffn_i4_ring_kernel<2, 4, kStages>;
-            static bool once[64] = {};
-            if (!ensure_dynamic_smem(k, smem_r, once)) return HALO_ERR_CUDA;
-            k<<<grid_r, kRingThreads, smem_r, st>>>(d, S, G, q, sc, xt, keep_list, n_keep, dev_of_group, n_dev, n_tok,
-                                                   partials, dev_status);
-        }
-        return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+            return cudaLaunchKernelEx(&cfg, k, d, S, G, q, sc, xt, keep_list, n_keep, dev_of_group, n_dev, n_tok, partials,
+                                      dev_status) == cudaSuccess
+                       ? HALO_OK
+                       : HALO_ERR_CUDA;
+        };
+        static bool once_a[64] = {}, once_b[64] = {}, once_c[64] = {}, once_d[64] = {};
+        if (d == 4096) return two ? go(group_ffn_i4_ring_kernel<4, 1, 2, 8>, once_a) : go(group_ffn_i4_ring_kernel<4, 2, 4, 16>, once_b);
+        return two ? go(group_ffn_i4_ring_kernel<2, 2, 2, 8>, once_c) : go(group_ffn_i4_ring_kernel<2, 4, 4, 16>, once_d);
     }
     const int chunks8 = d / 16;
     const int iters = (chunks8 + kI4Threads - 1) / kI4Threads;

@@ -38,7 +38,8 @@ def _run(sh, Q, Sc, x, keep, dev, n_dev, G):
 
 
 @pytest.mark.parametrize("dtype,d,G,S,n_tok", [("bf16", 256, 5, 16, 1), ("f32", 384, 4, 24, 2), ("bf16", 4096, 6, 128, 1),
-                                               ("bf16", 8192, 3, 40, 1), ("bf16", 1024, 7, 256, 3)])
+                                               ("bf16", 8192, 3, 40, 1), ("bf16", 1024, 7, 256, 3),
+                                               ("bf16", 2048, 9, 64, 2)])
 def test_int4_codes_bit_exact_and_ffn_matches_the_oracle(dtype, d, G, S, n_tok):
     wl = synth.Workload("q", 1, d, G * S, S, 16, dtype, (0.0, 0.3, 0.6), (1, 1, 1), 500, 1)
     Wp = synth.packed_layer(wl, 0, DEV)
@@ -95,7 +96,7 @@ def test_int4_full_size_7b_block_sampled_groups():
     assert np.abs(P - ref).max() <= U.TOL_BF16 * rms
 
 
-@pytest.mark.parametrize("form", [-1, 1, 3])
+@pytest.mark.parametrize("form", [-1, 1, 2, 3])
 def test_int4_full_size_7b_block_all_groups_kept_every_element(form):
     """The case the benchmark times: one 7B-shaped block on int4 weights with all 86 groups kept (the shared-memory
     ring kernel with a full kept set; also the plain-load form and the tensor-core form).  Codes and scales of the

@@ -461,7 +461,9 @@ halo_status halo_stack_set_mode(halo_stack* stack, int mode);
  * ablation can be run through the same library.  value = -1 restores the default.  A stack reads the first three
  * when it is created; the others are read at every call of the entry point they belong to.  No environment
  * variable is read anywhere in the library.
- *   "cross_stages" (0..8)             persistent kernel: stages of the next block fetched across the block barrier
+ *   "cross_stages" (0..16)            persistent kernel: stages of the next block fetched across the block barrier
+ *   "tmem_ring" (0/1)                 persistent kernel, d_model 2048 / 4096: second level of the weight ring in
+ *                                     tensor memory (default 0: measured slower, kept as an option)
  *   "l2_ahead" (0..32)                persistent kernel: batches prefetched to L2 on entering a block
  *   "max_steps_per_launch" (0 = auto) persistent kernel: steps per launch before a run is split
  *   "prefill_two_launches" (0/1)      prompt FFN as two launches (hidden, down) instead of one

@@ -99,7 +99,8 @@ halo_status check_pred_shape(const halo_pred_shape* s);   // argument rules of t
 
 // Process-wide options set through halo_set_option (capi.cu).  A value of -1 means "not set: use the default".
 enum OptionId { OPT_CROSS_STAGES = 0, OPT_L2_AHEAD, OPT_MAX_STEPS_PER_LAUNCH, OPT_PREFILL_TWO_LAUNCHES, OPT_PREFILL_KCUTS,
-                OPT_PREFILL_KRATIO_PERCENT, OPT_MHA_THREE_LAUNCHES, OPT_I4_NO_RING, OPT_PROMPT_KCUTS, OPT_PROMPT_L2_AHEAD, OPT_COUNT };
+                OPT_PREFILL_KRATIO_PERCENT, OPT_MHA_THREE_LAUNCHES, OPT_I4_NO_RING, OPT_PROMPT_KCUTS, OPT_PROMPT_L2_AHEAD, OPT_TMEM_RING,
+                OPT_COUNT };
 int option_value(OptionId id);
 
 halo_status launch_predict(const halo_pred_shape& sh, const void* W1, const void* W2, const void* feat, int n_tok,

@@ -27,15 +27,20 @@
 #include "select_device.cuh"
 #include "stack_persistent.cuh"
 #include "tma.cuh"
+#include "umma.cuh"
 
 namespace halo {
 
 constexpr int kPC = 512;                 // consumer threads
 constexpr int kPCWarps = kPC / 32;
 constexpr int kPThreads = kPC + 32;      // + producer warp
+constexpr int kPThreadsTM = kPC + 64;    // + producer warp + the warp that moves stages into tensor memory
+constexpr int kTSlots = 5;               // stage slots in tensor memory
+constexpr int kTSlotCols = 96;           // 32-bit columns per slot: 128 lanes x 96 x 4 B = 48 KB, one stage
+constexpr int kTCols = 512;              // columns allocated (all of the SM's tensor memory)
 constexpr int kHeaderBytes = 16 * 1024;  // PersistSmem
 constexpr int kAccBufs = 2;              // interleaved accumulation buffers per block of the stack
-constexpr int kFetchAhead = 3;           // batch-counter fetches a producer keeps in flight
+constexpr int kFetchAhead = 6;           // batch-counter claims a producer keeps in flight
 
 enum StageType { ST_FFN = 0, ST_PRED = 1, ST_END = 3 };
 
@@ -53,6 +58,14 @@ struct PersistSmem {
     float score[HALO_MAX_GROUPS];
     int kept_group[HALO_MAX_GROUPS];   // producer's table for the block it is issuing: group id or -1 per kept position
     SelectSmem sel;
+    // second level of the ring, in tensor memory (TM form of the kernel)
+    uint64_t tfull[8];
+    uint64_t tempty[8];
+    uint64_t tdrain;
+    int ttype[8];
+    int targ0[8];
+    int targ1[8];
+    uint32_t tmem_base;
 };
 static_assert(sizeof(PersistSmem) <= kHeaderBytes, "shared-memory header too large");
 
@@ -98,12 +111,62 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 enum TraceSlot { TR_BLOCK_START = 0, TR_FIRST_STAGE = 1, TR_STAGES_DONE = 2, TR_FLUSHED = 3, TR_BARRIER_DONE = 4,
                  TR_MERGED = 5, TR_X_READY = 6, TR_SELECT_NS = 7 };
 
-template <int NB, int XC, int P2, int REP, int STAGES>
-__global__ void __launch_bounds__(kPThreads, 1)
+// consumers + the mover warp, at the end of the TM form: nobody reads tensor memory after it
+__device__ __forceinline__ void tm_join_barrier() { asm volatile("bar.sync 2, %0;" ::"n"(kPC + 32) : "memory"); }
+
+// Shared-memory matrix descriptor without swizzle: 8 x 16-byte core matrices, `sbo` bytes from one group of 8 rows
+// to the next, `lbo` bytes from one 16-byte column of core matrices to the next.
+__device__ __forceinline__ uint64_t smem_desc_plain(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t dsc = 0;
+    dsc |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+    dsc |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    dsc |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    dsc |= 1ull << 46;
+    return dsc;
+}
+// 4 KB of shared memory -> 128 lanes x 8 columns of tensor memory: with sbo = 128 and lbo = 2048, lane i receives the
+// 16-byte chunk i of the first 2 KB in columns 0..3 and chunk i of the second 2 KB in columns 4..7.
+__device__ __forceinline__ void tmem_cp_4k(uint32_t taddr, uint32_t smem_addr) {
+    asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(smem_desc_plain(smem_addr, 2048u, 128u))
+                 : "memory");
+}
+template <int N>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&v)[N]) {
+    static_assert(N == 4 || N == 8 || N == 16, "columns per load");
+    if constexpr (N == 4) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
+                     : "r"(taddr)
+                     : "memory");
+    } else if constexpr (N == 8) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                     : "r"(taddr)
+                     : "memory");
+    } else {
+        tmem_ld_32x16(taddr, v);
+    }
+}
+
+// TM = true: the ring has a second level in tensor memory.  A stage that has landed in shared memory is moved on at
+// once (tcgen05.cp, issued by one thread of a fourth role, the mover warp) into one of kTSlots slots of the SM's
+// 256 KB of tensor memory, which frees the shared-memory stage for the next bulk copy; the consumers read their
+// operands from tensor memory (tcgen05.ld).  Shared memory plus tensor memory hold 9 stages (432 KB) instead of 4,
+// enough for the producer to keep streaming the next block's weights through the whole of the flush / grid barrier /
+// merge at the end of a block, so HBM does not fall idle there and does not have to ramp up again afterwards.
+//   layout   row rho of a stage (gate rows, up rows, down rows), 2 KB piece pi of it: columns (rho * PPR + pi) * 4 .. + 3
+//            of the slot; lane i holds the 16-byte chunk 128 * pi + i of the row.
+//   phase 1  warp w reads lanes 32 * (w % 4) ..; the four warps w / 4 = 0..3 take rows w / 4, w / 4 + 4, ...; a thread
+//            keeps the PPR chunks of x that meet its lane.
+//   phase 2  thread tid owns the same columns as in the plain form (chunk tid % (512 / REP)), piece = chunk / 128.
+template <int NB, int XC, int P2, int REP, int STAGES, bool TM>
+__global__ void __launch_bounds__(TM ? kPThreadsTM : kPThreads, 1)
 stack_decode_kernel(const __grid_constant__ PersistParams P) {
     constexpr int ROWS = 2 * NB;
-    constexpr int WPR = kPCWarps / ROWS;
-    static_assert(WPR * ROWS == kPCWarps && STAGES <= 8 && NB % REP == 0, "shape");
+    constexpr int WPR = TM ? 4 : kPCWarps / ROWS;
+    constexpr int PPR = XC;                       // TM: 2 KB pieces per row = chunks of x per thread
+    static_assert((TM || WPR * ROWS == kPCWarps) && STAGES <= 8 && NB % REP == 0, "shape");
+    static_assert(!TM || (P2 == 1 && ROWS % 4 == 0 && 3 * NB * PPR * 4 == kTSlotCols && (PPR == 2 || PPR == 4)), "TM shape");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     PersistSmem& sm = *reinterpret_cast<PersistSmem*>(smem_raw);
     // one vector buffer, used in turn for the fp32 column sums on their way out and for x (bf16) on its way in
@@ -128,17 +191,30 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
     unsigned* const sync_selready = P.sync + 3;
 
     if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], kPCWarps); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], TM ? 1 : kPCWarps); }
+        if constexpr (TM) {
+            // tfull: one arrival from the copies' completion, one from the mover after it wrote the slot's metadata
+            for (int t = 0; t < kTSlots; ++t) { mbar_init(&sm.tfull[t], 2); mbar_init(&sm.tempty[t], kPCWarps); }
+            mbar_init(&sm.tdrain, 1);
+        }
         sm.abort_flag = 0;
         sm.blocks_done = 0;
         mbar_fence_init();
     }
+    if constexpr (TM) {
+        if (!is_selector && warp == kPCWarps + 1) {
+            tmem_alloc(&sm.tmem_base, kTCols);
+            tmem_relinquish_alloc_permit();
+        }
+        tcgen05_fence_before_sync();
+    }
     __syncthreads();
+    if constexpr (TM) tcgen05_fence_after_sync();
     volatile int* abort_flag = &sm.abort_flag;
 
     // =========================================== selector ===========================================
     if (is_selector) {
-        if (warp == kPCWarps) return;   // only the 512 "consumer" threads are used here
+        if (warp >= kPCWarps) return;   // only the 512 "consumer" threads are used here
         bool bad = false;
         for (int step_i = 0; step_i < P.steps && !bad; ++step_i) {
             for (int lp = 1; lp < L && !bad; ++lp) {
@@ -318,21 +394,23 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 }
                 if (lane == 0) {
                     // (d) batches of kept neurons, handed out by the block's counter
-                    unsigned* const ctr = P.sync + 16 + (qp & 15u);
+                    unsigned* const ctr = P.sync + 32 + (qp & 31u);
                     const __nv_bfloat16* Wl = P.W[l];
-                    // The first batch is fixed, the rest come from the counter.  kFetchAhead fetches are kept in
-                    // flight so that the round trip of the atomic is off the issue path.
-                    long long b = cta;
-                    long long ahead[kFetchAhead];
+                    // The first batch is fixed, the rest come from the counter.  kFetchAhead claims are kept in
+                    // flight so that the round trip of the atomic (a microsecond and more while HBM is saturated) is
+                    // off the issue path: the claims sit in registers with fixed roles (the loop below is unrolled),
+                    // and a claim is read only kFetchAhead batches after it was made.
                     // deterministic: batch cta, cta + workers, ...: every thread block sums the same batches in the
                     // same order in every run
-#pragma unroll
-                    for (int k = 0; k < kFetchAhead; ++k)
-                        ahead[k] = P.deterministic ? static_cast<long long>(cta) + static_cast<long long>(workers) * (k + 1)
-                                                   : static_cast<long long>(workers) + atomicAdd(ctr, 1u);
-                    while (b < U) {
+                    long long ahead[kFetchAhead];
+                    long long det_next = static_cast<long long>(cta) + workers;
+                    auto claim = [&]() -> long long {
+                        if (P.deterministic) { const long long v = det_next; det_next += workers; return v; }
+                        return static_cast<long long>(workers) + atomicAdd(ctr, 1u);
+                    };
+                    auto issue = [&](long long b) -> bool {
                         int s;
-                        if (!acquire(s)) { alive = false; break; }
+                        if (!acquire(s)) return false;
                         const int ki = static_cast<int>(b / per_group), j0 = static_cast<int>(b - static_cast<long long>(ki) * per_group) * NB;
                         const int g = sm.kept_group[ki];
                         sm.type[s] = ST_FFN; sm.arg0[s] = g >= 0 ? 0 : -1; sm.arg1[s] = 0;
@@ -348,11 +426,29 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                                           &sm.full[s]);
                         }
                         ++it;
-                        b = ahead[0];
+                        return true;
+                    };
+                    if (static_cast<long long>(cta) < U) {
 #pragma unroll
-                        for (int k = 0; k + 1 < kFetchAhead; ++k) ahead[k] = ahead[k + 1];
-                        if (P.deterministic) ahead[kFetchAhead - 1] = ahead[kFetchAhead - 2] + workers;
-                        else ahead[kFetchAhead - 1] = (b < U) ? static_cast<long long>(workers) + atomicAdd(ctr, 1u) : U;
+                        for (int k = 0; k < kFetchAhead; ++k) ahead[k] = claim();
+                        if (!issue(cta)) alive = false;
+                        bool more = alive;
+                        while (more) {
+#pragma unroll
+                            for (int k = 0; k < kFetchAhead; ++k) {
+                                if (more) {
+                                    const long long b = ahead[k];
+                                    if (b >= U) {
+                                        more = false;     // claims only grow: every later one is past the end too
+                                    } else if (!issue(b)) {
+                                        alive = false;
+                                        more = false;
+                                    } else {
+                                        ahead[k] = claim();
+                                    }
+                                }
+                            }
+                        }
                     }
                     if (alive) alive = marker(ST_END, 0);
                 }
@@ -371,9 +467,66 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
         return;
     }
 
+    // =========================================== mover (TM) ===========================================
+    if constexpr (TM) {
+        if (warp == kPCWarps + 1) {
+            const uint32_t tbase = sm.tmem_base;
+            if (lane == 0) {
+                long long blocks_left = static_cast<long long>(P.steps) * L;
+                int it = 0;
+                bool cps = false;
+                while (blocks_left > 0) {
+                    const int s = it % STAGES, t = it % kTSlots;
+                    if (!mbar_wait_bounded(&sm.full[s], static_cast<uint32_t>(it / STAGES) & 1u, abort_flag)) { *abort_flag = 1; break; }
+                    if (it >= kTSlots &&
+                        !mbar_wait_bounded(&sm.tempty[t], (static_cast<uint32_t>(it / kTSlots) - 1u) & 1u, abort_flag)) {
+                        *abort_flag = 1;
+                        break;
+                    }
+                    const int type = sm.type[s], a0 = sm.arg0[s], a1 = sm.arg1[s];
+                    sm.ttype[t] = type; sm.targ0[t] = a0; sm.targ1[t] = a1;
+                    int n4k = 0;    // 4 KB pieces to move
+                    if (type == ST_FFN && a0 >= 0) n4k = 3 * NB * PPR / 2;
+                    else if (type == ST_PRED) n4k = a1 * PPR / 2;
+                    if (n4k > 0) {
+                        tcgen05_fence_after_sync();
+                        const uint32_t src = smem_u32(ring + static_cast<size_t>(s) * stage_bytes);
+                        const uint32_t dst = tbase + static_cast<uint32_t>(t * kTSlotCols);
+                        for (int k = 0; k < n4k; ++k) tmem_cp_4k(dst + 8u * k, src + 4096u * k);
+                        umma_commit(&sm.tfull[t]);    // the slot is complete when the copies are
+                        umma_commit(&sm.empty[s]);    // ... and the shared-memory stage is free again
+                        mbar_arrive(&sm.tfull[t]);    // releases the metadata written above
+                        cps = true;
+                    } else {
+                        mbar_arrive(&sm.tfull[t]);
+                        mbar_arrive(&sm.tfull[t]);
+                        mbar_arrive(&sm.empty[s]);
+                    }
+                    ++it;
+                    if (type == ST_END) --blocks_left;
+                }
+                if (cps) {   // every copy issued has completed before tensor memory is given back
+                    umma_commit(&sm.tdrain);
+                    int never = 0;
+                    mbar_wait_bounded(&sm.tdrain, 0u, &never);
+                }
+            }
+            __syncwarp();
+            tcgen05_fence_before_sync();
+            tm_join_barrier();
+            tcgen05_fence_after_sync();
+            tmem_dealloc(tbase, kTCols);
+            return;
+        }
+    }
+
     // =========================================== consumers ===========================================
     const int row = warp / WPR, part = warp % WPR;
-    const int p1_base = part * (XC * 32) + lane;
+    const int tq = warp & 3, tg = warp >> 2;      // TM: quarter of the lanes this warp can read, and its row group
+    const uint32_t tlane = static_cast<uint32_t>(tq * 32) << 16;
+    const uint32_t tbase = TM ? sm.tmem_base : 0u;
+    const int p1_base = TM ? tq * 32 + lane : part * (XC * 32) + lane;
+    constexpr int p1_step = TM ? 128 : 32;        // distance between this thread's chunks of x
     const int rep = (REP > 1) ? tid / (kPC / REP) : 0;
     const int col0 = (REP > 1) ? tid % (kPC / REP) : tid;
     const bool owner = (REP == 1) || (rep == 0);   // threads that carry the residual stream for their columns
@@ -430,7 +583,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
         pc_barrier();  // xs complete; sm.reduce free again
         if (want_x) {
 #pragma unroll
-            for (int i = 0; i < XC; ++i) xq[i] = reinterpret_cast<const uint4*>(xs)[p1_base + 32 * i];
+            for (int i = 0; i < XC; ++i) xq[i] = reinterpret_cast<const uint4*>(xs)[p1_base + p1_step * i];
         }
     };
 
@@ -475,15 +628,42 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
 
             // ------------------------------ stages of this block ------------------------------
             while (true) {
-                const int s = it % STAGES;
-                const uint32_t parity = static_cast<uint32_t>(it / STAGES) & 1u;
-                const bool ok = mbar_wait_bounded(&sm.full[s], parity, abort_flag);
+                const int s = TM ? it % kTSlots : it % STAGES;
+                const uint32_t parity = static_cast<uint32_t>(it / (TM ? kTSlots : STAGES)) & 1u;
+                const bool ok = mbar_wait_bounded(TM ? &sm.tfull[s] : &sm.full[s], parity, abort_flag);
+                if constexpr (TM) tcgen05_fence_after_sync();
                 if (first_stage) { trace(TR_FIRST_STAGE, global_timer_ns()); first_stage = false; }
-                const int type = sm.type[s], a0 = sm.arg0[s], a1 = sm.arg1[s];
-                const unsigned char* stage = ring + static_cast<size_t>(s) * stage_bytes;
+                const int type = TM ? sm.ttype[s] : sm.type[s], a0 = TM ? sm.targ0[s] : sm.arg0[s],
+                          a1 = TM ? sm.targ1[s] : sm.arg1[s];
+                const unsigned char* stage = ring + static_cast<size_t>(TM ? 0 : s) * stage_bytes;
+                const uint32_t tslot = tbase + tlane + static_cast<uint32_t>(s * kTSlotCols);   // TM: this warp's lanes of the slot
                 float* red = sm.red[red_par];
                 // ---- before the barrier: nothing in here may block on other consumers ----
-                if (type == ST_FFN) {
+                if constexpr (TM) {
+                    if ((type == ST_FFN && a0 >= 0) || type == ST_PRED) {
+                        if (type == ST_FFN) any = true;
+                        const int n_rows = type == ST_FFN ? ROWS : a1;
+                        const uint4* xg = reinterpret_cast<const uint4*>(P.x_hist + static_cast<size_t>((l - 1) & 1) * d);
+                        const bool x_global = type == ST_PRED && P.pred_serial;   // this block's own predictor
+#pragma unroll
+                        for (int rr = 0; rr < ROWS / 4; ++rr) {
+                            const int rw = tg + 4 * rr;
+                            if (rw < n_rows) {       // warp-uniform
+                                uint32_t w[4 * PPR];
+                                tmem_ld_cols<4 * PPR>(tslot + static_cast<uint32_t>(rw * PPR * 4), w);
+                                tmem_ld_wait();
+                                float dot0 = 0.0f, dot1 = 0.0f;
+#pragma unroll
+                                for (int i = 0; i < PPR; ++i) {
+                                    const uint4 wv = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+                                    dot_bf16x8(wv, x_global ? __ldcg(xg + p1_base + p1_step * i) : xq[i], dot0, dot1);
+                                }
+                                const float dot = warp_sum(dot0 + dot1);
+                                if (lane == 0) red[rw * WPR + tq] = dot;
+                            }
+                        }
+                    }
+                } else if (type == ST_FFN) {
                     if (a0 >= 0) {
                         any = true;
                         const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(row) * row_bytes);
@@ -520,11 +700,19 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                         for (int jj = 0; jj < NB / REP; ++jj) {
                             const int j = jj * REP + rep;
                             const float h = silu_mul(sum_parts<WPR>(red + j * WPR), sum_parts<WPR>(red + (NB + j) * WPR));
+                            if constexpr (TM) {
+                                // the thread's chunk col0 of down row j: piece col0 / 128, lane col0 % 128 (this warp's quarter)
+                                uint32_t w[4];
+                                tmem_ld_cols<4>(tslot + static_cast<uint32_t>(((ROWS + j) * PPR + (col0 >> 7)) * 4), w);
+                                tmem_ld_wait();
+                                axpy_bf16x8(h, make_uint4(w[0], w[1], w[2], w[3]), acc[0]);
+                            } else {
                             const uint4* dr = reinterpret_cast<const uint4*>(down + static_cast<size_t>(j) * row_bytes);
 #pragma unroll
                             for (int p = 0; p < P2; ++p) {
                                 const int c = col0 + kPC * p;
                                 if (P2 == 1 || c < chunks) axpy_bf16x8(h, dr[c], acc[p]);
+                            }
                             }
                         }
                     }
@@ -545,8 +733,9 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                     }
                     red_par ^= 1;
                 }
+                if constexpr (TM) tcgen05_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.empty[s]);
+                if (lane == 0) mbar_arrive(TM ? &sm.tempty[s] : &sm.empty[s]);
                 ++it;
                 if (type == ST_END) break;
             }
@@ -591,10 +780,11 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                     fence_proxy_async_all();
                 }
                 trace(TR_FLUSHED, global_timer_ns());
-                // Batch counters rotate over 16 words.  A producer leads its consumers by at most the ring depth
-                // (<= 8 stages, every block has at least its END stage), so the counter of the block 8 ahead is
-                // idle now: its last user finished 8 blocks ago and its next user cannot have started.
-                if (cta == 0) P.sync[16 + ((q + 8u) & 15u)] = 0u;
+                // Batch counters rotate over 32 words.  A producer leads its consumers by at most the ring depth
+                // (<= 13 stages with the tensor-memory level, every block has at least its END stage), so the counter
+                // of the block 16 ahead is idle now: its last user finished 16 blocks ago and its next user cannot
+                // have started.
+                if (cta == 0) P.sync[32 + ((q + 16u) & 31u)] = 0u;
                 __threadfence();
                 const unsigned target = (q + 1u) * static_cast<unsigned>(workers);
                 const unsigned before = atomicAdd(sync_barrier, 1u);
@@ -672,6 +862,10 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
         atomicExch(sync_abort, 1u);      // every other thread block follows
         flag_status(P.status, HALO_DEV_TIMEOUT);
     }
+    if constexpr (TM) {
+        tcgen05_fence_before_sync();
+        tm_join_barrier();               // the mover frees the tensor memory behind this
+    }
 }
 
 // ---- host side -----------------------------------------------------------------------------------------
@@ -686,9 +880,10 @@ bool persistent_supported(const halo_ffn_shape& sh, int n_tok, int G) {
     return false;
 }
 
-template <int NB, int XC, int P2, int REP, int STAGES>
+template <int NB, int XC, int P2, int REP, int STAGES, bool TM>
 static halo_status launch_cfg(PersistParams& P, cudaStream_t st) {
-    auto kernel = stack_decode_kernel<NB, XC, P2, REP, STAGES>;
+    auto kernel = stack_decode_kernel<NB, XC, P2, REP, STAGES, TM>;
+    constexpr int kThreads = TM ? kPThreadsTM : kPThreads;
     const size_t smem = kHeaderBytes + static_cast<size_t>(P.d) * 4 * REP + static_cast<size_t>(STAGES) * 3 * NB * P.d * 2;
     static bool configured[64] = {};
     int dev = 0, sms = kSmCount;
@@ -696,11 +891,11 @@ static halo_status launch_cfg(PersistParams& P, cudaStream_t st) {
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (!ensure_dynamic_smem(kernel, smem, configured)) return HALO_ERR_CUDA;
     int blocks_per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, kernel, kPThreads, smem) != cudaSuccess)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, kernel, kThreads, smem) != cudaSuccess)
         return HALO_ERR_CUDA;
     if (blocks_per_sm < 1 || sms < 2) return HALO_ERR_UNIMPLEMENTED;   // cannot be made resident: caller falls back
     void* args[] = {&P};
-    const cudaError_t err = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(sms), dim3(kPThreads), args,
+    const cudaError_t err = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(sms), dim3(kThreads), args,
                                                         smem, st);
     if (err == cudaErrorCooperativeLaunchTooLarge) {
         // the SMs are not all ours (another context on the device): not an error of this call, the caller runs the
@@ -713,10 +908,10 @@ static halo_status launch_cfg(PersistParams& P, cudaStream_t st) {
 
 halo_status launch_stack_persistent(PersistParams& P, cudaStream_t st) {
     switch (P.d) {
-        case 2048: return launch_cfg<4, 4, 1, 2, 4>(P, st);
-        case 4096: return launch_cfg<2, 4, 1, 1, 4>(P, st);
-        case 5120: return launch_cfg<2, 5, 2, 1, 3>(P, st);
-        case 8192: return launch_cfg<1, 4, 2, 1, 3>(P, st);
+        case 2048: return P.tmem_ring ? launch_cfg<4, 2, 1, 2, 4, true>(P, st) : launch_cfg<4, 4, 1, 2, 4, false>(P, st);
+        case 4096: return P.tmem_ring ? launch_cfg<2, 4, 1, 1, 4, true>(P, st) : launch_cfg<2, 4, 1, 1, 4, false>(P, st);
+        case 5120: return launch_cfg<2, 5, 2, 1, 3, false>(P, st);
+        case 8192: return launch_cfg<1, 4, 2, 1, 3, false>(P, st);
     }
     return HALO_ERR_UNIMPLEMENTED;
 }

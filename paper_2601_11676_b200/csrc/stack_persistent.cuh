@@ -24,8 +24,8 @@ struct PersistParams {
     float* partials;                       // [3][2][d] rotating interleaved accumulation buffers, zero at launch
     float* z;                              // [2][r]: hidden values, by parity of the prediction
     PersistSel* sel;                       // [3]: two rotating + the static first-block selection
-    unsigned* sync;                        // [32]: 0 barrier count, 1 abort, 2 hidden rows done, 3 selections
-                                           //       published, 16..31 rotating batch counters; zero at launch
+    unsigned* sync;                        // [64]: 0 barrier count, 1 abort, 2 hidden rows done, 3 selections
+                                           //       published, 32..63 rotating batch counters; zero at launch
     uint32_t* status;
     // optional records (thread block 0 / the selecting thread block write them)
     __nv_bfloat16* tap_x;
@@ -40,6 +40,7 @@ struct PersistParams {
     int cross_stages;                      // stages of the next block a producer may issue before its consumers
                                            // have passed the grid barrier of the current block
     int l2_ahead;                          // batches per thread block prefetched into L2 on entering a block
+    int tmem_ring;                         // 1: stages pass through tensor memory (d_model 2048 / 4096 only)
     int pred_serial;                       // 1: the predictor rows and the selection of block l run at the start of
                                            // block l itself (from the recorded x_{l-1}), not beside block l-1
     int deterministic;                     // 1: fixed batch assignment and fixed-order sums (bitwise repeatable)

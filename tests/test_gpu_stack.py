@@ -392,6 +392,26 @@ def test_long_runs_are_split_into_several_persistent_launches():
     assert (h_out - h_ref).abs().max().item() <= 1e-3 * h_ref.abs().max().item()
 
 
+@pytest.mark.parametrize("mode", [0, B.STACK_PRED_SERIAL, B.STACK_DETERMINISTIC])
+@pytest.mark.parametrize("name,layers,steps", [("tinyllama-1.1b-decode", 5, 4), ("llama2-7b-decode", 4, 3)])
+def test_stack_with_the_ring_extended_into_tensor_memory(name, layers, steps, mode):
+    """Option "tmem_ring": landed stages are moved on into tensor memory (tcgen05.cp) and the consumers read them from
+    there (tcgen05.ld).  Same path, same records: teacher-forced against the oracle, same selections as the default."""
+    wl = synth.small_variant(synth.workload(name), layers, steps)
+    B.halo_set_option("tmem_ring", 1)
+    try:
+        stack, Wp, preds = build_stack(wl)
+    finally:
+        B.halo_set_option("tmem_ring", -1)
+    stack.set_mode(mode)
+    h0, h_out, t = run_with_taps(wl, stack, steps, step0=5)
+    assert stack.last_launches() == 1 and stack.status() == 0
+    check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=5)
+    ref_stack, _, _ = build_stack(wl)
+    _, h_ref, t_ref = run_with_taps(wl, ref_stack, steps, step0=5)
+    assert (t["n_keep"] == t_ref["n_keep"]).all().item() and (t["keep_list"] == t_ref["keep_list"]).all().item()
+
+
 @pytest.mark.parametrize("mode", [B.STACK_PRED_SERIAL, B.STACK_LOAD_SERIAL, B.STACK_PRED_SERIAL | B.STACK_LOAD_SERIAL])
 @pytest.mark.parametrize("name,layers,steps", [("tinyllama-1.1b-decode", 4, 3), ("llama2-7b-decode", 3, 2),
                                                ("llama2-13b-decode", 3, 2)])

@@ -32,9 +32,10 @@ NOMINAL_HBM_GBS = 8000.0
 # 4-block 7B-shaped case (profiles/stack_decode_kernel_llama2-7b_4blocks.md); traffic is proportional to the kept
 # groups processed, so the ratio carries over to the full-size launch.  The figure belongs to the kernel sources with
 # the hash below: when they change the line reports no traffic until the counters have been taken again.
-STACK_KERNEL_TRAFFIC_RATIO = 1.0003
-STACK_KERNEL_SOURCES = ("stack_persistent.cu", "stack_persistent.cuh", "ffn_math.cuh", "tma.cuh", "select_device.cuh")
-STACK_KERNEL_SOURCES_SHA1 = "unset"
+STACK_KERNEL_TRAFFIC_RATIO = 1.0005
+STACK_KERNEL_SOURCES = ("stack_persistent.cu", "stack_persistent.cuh", "ffn_math.cuh", "tma.cuh", "umma.cuh",
+                        "select_device.cuh")
+STACK_KERNEL_SOURCES_SHA1 = "45f77459a6c9ab59f4e93c4f7b4143d6a9bd9f91"
 FALLBACK_HBM_GBS = 6650.0
 
 

@@ -161,6 +161,9 @@ def build_stack(wl, dev):
 def run_halo(args, rank, world, local_rank):
     from paper_2601_11676_b200 import binding as B
     B.lib()  # fail loudly if the CUDA library is missing
+    for item in args.option:
+        name, _, value = item.partition("=")
+        B.halo_set_option(name, int(value))
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     wl = synth.workload(args.workload, keep_permille=args.keep_permille)
@@ -279,6 +282,8 @@ def run_halo(args, rank, world, local_rank):
                 "peak_gbs": peak, "peak_kind": peak_kind},
     }
     persistent = launches == 1
+    if args.option:
+        result["options"] = list(args.option)     # a tuning sweep, not the default configuration
     traffic_valid = STACK_KERNEL_TRAFFIC_RATIO is not None and stack_kernel_sources_sha1() == STACK_KERNEL_SOURCES_SHA1
     if persistent:
         # the timed region is ONE launch of the persistent stack kernel: its duration is the event time itself
@@ -793,6 +798,8 @@ def main():
     ap.add_argument("--no-prefill", action="store_true", help="skip the 512-token prompt report")
     ap.add_argument("--no-extra", action="store_true", help="skip the brief runs of the other decode workloads")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
+                    help="halo_set_option before anything is created (tuning sweeps), e.g. --option cross_stages=4")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "halo" else args.warmup
 

@@ -646,7 +646,7 @@ halo_status stack_create_impl(halo_stack** out, const halo_ffn_shape* ffn, const
     // thread blocks finish a block further apart (the grid barrier waits 6 us instead of 2).  Net: 20 % slower there.
     s->tmem_ring = option_value(OPT_TMEM_RING) == 1;
     // with the tensor-memory level the producer may run as far ahead as the ring lets it
-    s->cross_stages = s->tmem_ring ? 16 : 1;
+    s->cross_stages = s->tmem_ring ? 16 : 2;
     s->l2_ahead = 0;
     if (option_value(OPT_CROSS_STAGES) >= 0) s->cross_stages = option_value(OPT_CROSS_STAGES);
     s->max_steps_per_launch = std::max(0, option_value(OPT_MAX_STEPS_PER_LAUNCH));

@@ -59,28 +59,48 @@ glue_kernel(int d, const float* __restrict__ h, const float* __restrict__ y_in, 
         // four columns per thread and access (every row starts 16-byte aligned)
         const int d4 = d >> 2;
         const float4* h4 = reinterpret_cast<const float4*>(h + base);
-        for (int c = threadIdx.x; c < d4; c += blockDim.x) {
+        // The arrival flags as one mask per warp (lane i reads flag i; the loads below do not wait for it): the slots of
+        // a batch of devices are fetched unconditionally and masked afterwards, so a merge is one round trip to memory
+        // instead of one per device.
+        uint8_t my_flag = 1;
+        if (MERGE && arrived && (threadIdx.x & 31) < n_dev) my_flag = arrived[threadIdx.x & 31];
+        unsigned mask = 0u;
+        bool have_mask = false;
+        for (int c0 = 0; c0 < d4; c0 += blockDim.x) {   // same trip count for every thread: the vote below is warp-wide
+            const int c = c0 + threadIdx.x;
+            const bool on = c < d4;
             float4 y = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             if (MERGE) {
-                y = reinterpret_cast<const float4*>(partials + base)[c];
-                for (int i = 0; i < n_dev; ++i)
-                    if (!arrived || arrived[i]) {
-                        const float4 p =
-                            reinterpret_cast<const float4*>(partials + static_cast<size_t>(i + 1) * slot_stride + base)[c];
-                        y.x += p.x; y.y += p.y; y.z += p.z; y.w += p.w;
+                if (on) y = reinterpret_cast<const float4*>(partials + base)[c];
+                for (int i0 = 0; i0 < n_dev; i0 += 8) {
+                    float4 p[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        if (on && i0 + k < n_dev)
+                            p[k] = reinterpret_cast<const float4*>(partials + static_cast<size_t>(i0 + k + 1) * slot_stride + base)[c];
+                    if (!have_mask) {
+                        mask = __ballot_sync(0xffffffffu, my_flag != 0);
+                        have_mask = true;
                     }
-                if (y_tap) reinterpret_cast<float4*>(y_tap + base)[c] = y;
-                if (zero_slots)   // the slots are left zeroed for the next kernel that adds into them
+                    const unsigned m = mask >> i0;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        if (on && i0 + k < n_dev && ((m >> k) & 1u)) { y.x += p[k].x; y.y += p[k].y; y.z += p[k].z; y.w += p[k].w; }
+                }
+                if (on && y_tap) reinterpret_cast<float4*>(y_tap + base)[c] = y;
+                if (on && zero_slots)   // the slots are left zeroed for the next kernel that adds into them
                     for (int i = 0; i <= n_dev; ++i)
                         reinterpret_cast<float4*>(zero_slots + static_cast<size_t>(i) * slot_stride + base)[c] =
                             make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            } else if (y_in) {
+            } else if (y_in && on) {
                 y = reinterpret_cast<const float4*>(y_in + base)[c];
             }
-            const float4 hh = h4[c];
-            const float4 v = make_float4(hh.x + y.x, hh.y + y.y, hh.z + y.z, hh.w + y.w);
-            reinterpret_cast<float4*>(hv)[c] = v;
-            ss = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, fmaf(v.w, v.w, ss))));
+            if (on) {
+                const float4 hh = h4[c];
+                const float4 v = make_float4(hh.x + y.x, hh.y + y.y, hh.z + y.z, hh.w + y.w);
+                reinterpret_cast<float4*>(hv)[c] = v;
+                ss = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, fmaf(v.w, v.w, ss))));
+            }
         }
     } else {
         for (int c = threadIdx.x; c < d; c += blockDim.x) {

@@ -624,7 +624,7 @@ halo_status stack_create_impl(halo_stack** out, const halo_ffn_shape* ffn, const
     s->set_kl[0] = s->keep_list; s->set_kl[1] = reinterpret_cast<int32_t*>(base + o_kl2);
     s->set_nk[0] = s->n_keep; s->set_nk[1] = reinterpret_cast<int32_t*>(base + o_nk2);
     s->side = nullptr; s->ev_x = nullptr; s->ev_sel = nullptr;
-    if (n_tok > 1 && !i4_scales) {
+    if (n_tok > 1 || i4_scales || !persistent_supported(*ffn, n_tok, G)) {   // every path that is not the persistent kernel
         // best effort: without them the blocks simply run one after the other on the caller's stream
         // highest priority: the short predictor/selection kernels of the next block must get SMs as they free up,
         // ahead of the waiting CTAs of the long FFN launch (which pulls its tiles from a queue and loses nothing)
@@ -925,7 +925,10 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
         s->last_launches = launches;
         return HALO_OK;
     }
-    if (T > 1 && s->side) {
+    // Decode stacks that cannot take the persistent kernel (int4 weights, other widths) get the same overlap from the side
+    // stream, unless the one-launch-per-step arm was asked for.
+    const bool overlapped_decode = T == 1 && !(s->mode & HALO_STACK_PER_STEP_LAUNCHES);
+    if ((T > 1 || overlapped_decode) && s->side) {
         // Prompt path, one launch per step of the path.  The scores of block l+1 need only x_l (one layer ahead, Sec. III-B.2), which exists before
         // block l's FFN starts: predictor + selection of block l+1 go to the side stream and overlap with the
         // tensor-core GEMMs of block l (the paper's Pred || Comp overlap).  Two selection sets alternate by block.
@@ -945,13 +948,22 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                 void* x_next = s->x[nxt];
                 if (l + 1 < L) {
                     HALO_CU(cudaStreamWaitEvent(side, s->ev_x, 0));
-                    HALO_TRY(launch_predict(s->pred, s->W1[l + 1], s->W2[l + 1], x_cur, static_cast<int>(T), 1,
-                                            s->set_scores[nxt], s->pred_ws, s->status, side));
-                    HALO_TRY(launch_select(s->plan.dev, G, s->set_scores[nxt], step, static_cast<uint32_t>(l + 1), 0,
-                                           nullptr, s->set_dev[nxt], s->set_arr[nxt], nullptr, s->set_kl[nxt],
-                                           s->set_nk[nxt], s->status, side));
+                    if (T == 1) {
+                        HALO_TRY(launch_predict_hidden(s->pred, s->W1[l + 1], x_cur, 1, s->pred_ws, side));
+                        HALO_TRY(launch_score_select(s->pred, s->W2[l + 1], s->pred_ws, s->plan.dev, step,
+                                                     static_cast<uint32_t>(l + 1), 0, s->set_scores[nxt], nullptr,
+                                                     s->set_dev[nxt], s->set_arr[nxt], nullptr, s->set_kl[nxt],
+                                                     s->set_nk[nxt], s->status, side));
+                        launches += 2;
+                    } else {
+                        HALO_TRY(launch_predict(s->pred, s->W1[l + 1], s->W2[l + 1], x_cur, static_cast<int>(T), 1,
+                                                s->set_scores[nxt], s->pred_ws, s->status, side));
+                        HALO_TRY(launch_select(s->plan.dev, G, s->set_scores[nxt], step, static_cast<uint32_t>(l + 1), 0,
+                                               nullptr, s->set_dev[nxt], s->set_arr[nxt], nullptr, s->set_kl[nxt],
+                                               s->set_nk[nxt], s->status, side));
+                        launches += 4;
+                    }
                     HALO_CU(cudaEventRecord(s->ev_sel, side));
-                    launches += 4;
                 }
                 float* y_tap = nullptr;
                 if (taps) {
@@ -965,7 +977,13 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                     if (taps->y) y_tap = taps->y + rec * step_elems;
                 }
                 float* h_dst = (l == L - 1) ? h_out + sidx * step_elems : s->h;
-                if (!y_tap && s->ffn_ws && prefill_accumulates(s->ffn, static_cast<int>(T))) {
+                if (!s->i4_scales.empty()) {
+                    HALO_TRY(halo_group_ffn_i4(&s->ffn, s->W[l], s->i4_scales[l], x_cur, static_cast<int>(T), s->set_kl[cur],
+                                               s->set_nk[cur], s->set_dev[cur], n_dev, s->partials, s->status, stream));
+                    HALO_TRY(launch_merge_glue(s->partials, s->set_arr[cur], n_dev, static_cast<int>(T), static_cast<int>(d),
+                                               s->ffn.wdtype, s->h, h_dst, x_next, y_tap, st));
+                    launches += 3;
+                } else if (!y_tap && s->ffn_ws && prefill_accumulates(s->ffn, static_cast<int>(T))) {
                     // only kept (= arrived) groups are computed and nobody asked for y itself: the down projection
                     // adds its tiles straight into the residual stream, and the glue only normalises
                     HALO_TRY(launch_group_ffn_prefill(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->set_kl[cur],

@@ -321,15 +321,28 @@ __device__ __forceinline__ void st_remote_f32(float* local_smem_ptr, uint32_t ta
 // block r first computes dh / 8 rows each of the head's keys and values for this token and writes them into the
 // caches at `pos` (every head, never dropped); clusters of heads that are not kept end there.  The cluster barrier
 // that completes the query also orders those cache writes before the attention reads them.
+// Shared memory for a thread block's K and V rows (see kv_smem in the kernel): used when every block of a cluster has
+// a single piece of positions and the two pieces fit in 64 KB (so that two thread blocks still share an SM).
+constexpr size_t kKvSmemMax = 64 * 1024;
+constexpr size_t kMhaSmemLimit = 32 * 1024 + kKvSmemMax;   // x widened (at most 8192 floats) + the K / V rows
+static size_t kv_smem_bytes(int pos, int dh, size_t elem) {
+    const int n_pos = pos + 1;
+    const int piece = std::min(256, std::max(32, ((n_pos + kMhaCluster - 1) / kMhaCluster + 31) & ~31));
+    if (n_pos > kMhaCluster * piece) return 0;          // several pieces per block: the loop fetches them itself
+    const size_t bytes = 2 * static_cast<size_t>(piece) * dh * elem;
+    return (bytes <= kKvSmemMax && (static_cast<size_t>(dh) * elem) % 16 == 0) ? bytes : 0;
+}
+
 template <typename T, int ITERS, bool APPEND>
 __global__ void __cluster_dims__(kMhaCluster, 1, 1) __launch_bounds__(256)
 mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ Wp, const T* __restrict__ x,
                  const T* Kc, const T* Vc, const int32_t* __restrict__ keep_list,
                  const int32_t* __restrict__ n_keep_ptr, const int32_t* __restrict__ dev_of_group, int n_dev,
                  float* __restrict__ partials, uint32_t* dev_status, const T* __restrict__ Wk, const T* __restrict__ Wv,
-                 T* Kw, T* Vw) {
+                 T* Kw, T* Vw, int kv_smem) {
     constexpr int E = Elem<T>::kPerChunk;
-    extern __shared__ __align__(16) float xs[];          // [d]: x widened
+    extern __shared__ __align__(16) float xs[];          // [d]: x widened; behind it (kv_smem): this block's K and V rows
+    __shared__ uint64_t kv_bar;
     __shared__ float q_s[256];                           // the head's full query (written by all blocks of the cluster)
     __shared__ float o_acc[256];                         // this block's running o over its positions
     __shared__ float w_s[256];                           // softmax weights of the current piece
@@ -399,7 +412,28 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
     // ---- query rows j0 .. j0 + rows, two per warp and turn, sent to every block of the cluster ----
     if constexpr (!APPEND) stage_x(x, xs, d);
     for (int j = tid; j < dh; j += 256) o_acc[j] = 0.0f;
+    // piece = positions a block takes at a time: an eighth of the context (so that all eight blocks work) in
+    // multiples of 32, at most one position per thread
+    const int n_pos = pos + 1;
+    const int piece = min(256, max(32, ((n_pos + kMhaCluster - 1) / kMhaCluster + 31) & ~31));
+    // kv_smem (the host sets it when a block has one piece and it fits): the cached K and V rows of this block's
+    // positions are fetched into shared memory by two bulk copies NOW, under the query rows, instead of by dependent
+    // loads in the position loop.  The row of the current token is not among them when this launch writes it itself.
+    unsigned char* kvs = reinterpret_cast<unsigned char*>(xs + d);
+    const size_t row_b = static_cast<size_t>(dh) * sizeof(T);
+    const int pf_first = r * piece;
+    const int pf_valid = max(0, min(piece, n_pos - pf_first));
+    int pf_rows = pf_valid;
+    if (APPEND && pf_valid > 0 && pf_first + pf_valid - 1 == pos) pf_rows -= 1;
+    const bool pf = kv_smem != 0 && pf_valid > 0;
+    if (pf && tid == 0) { mbar_init(&kv_bar, 1); mbar_fence_init(); }
     __syncthreads();
+    if (pf && tid == 0 && pf_rows > 0) {
+        const uint32_t bytes = static_cast<uint32_t>(pf_rows * row_b);
+        mbar_arrive_expect_tx(&kv_bar, 2u * bytes);
+        bulk_copy_g2s(kvs, Kc + (static_cast<size_t>(h) * Lmax + pf_first) * dh, bytes, &kv_bar);
+        bulk_copy_g2s(kvs + piece * row_b, Vc + (static_cast<size_t>(h) * Lmax + pf_first) * dh, bytes, &kv_bar);
+    }
     const float scale = rsqrtf(static_cast<float>(dh));
     cluster_wait();                                      // every block of the cluster has started
     for (int i = 2 * warp; i < rows; i += 16) {
@@ -415,26 +449,53 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
 
     // ---- this block's positions: pieces r, r + 8, r + 16, ... of 256 positions; running (m, l, o) ----
     float m_run = -INFINITY, l_run = 0.0f;
-    const int n_pos = pos + 1;
     const int col_groups = dh / E;                       // 16-byte groups per value row
     const int pos_groups = 256 / col_groups;             // threads per column group
     const int cg = tid % col_groups, pg = tid / col_groups;
-    // piece = positions a block takes at a time: an eighth of the context (so that all eight blocks work) in
-    // multiples of 32, at most one position per thread
-    const int piece = min(256, max(32, ((n_pos + kMhaCluster - 1) / kMhaCluster + 31) & ~31));
+    if (pf) {
+        if (pf_rows > 0) {
+            int never = 0;
+            if (!mbar_wait_bounded(&kv_bar, 0u, &never) && tid == 0) flag_status(dev_status, HALO_DEV_TIMEOUT);
+        }
+        if (pf_rows < pf_valid) {
+            // the current token's row, written by this cluster before the barrier above: 16 bytes per thread
+            const int rl = pf_valid - 1;
+            if (tid < 2 * col_groups) {
+                const bool is_v = tid >= col_groups;
+                const int c = is_v ? tid - col_groups : tid;
+                const uint4* src = reinterpret_cast<const uint4*>((is_v ? Vc : Kc) + (static_cast<size_t>(h) * Lmax + pos) * dh) + c;
+                reinterpret_cast<uint4*>(kvs + (is_v ? piece * row_b : 0) + rl * row_b)[c] = __ldcg(src);
+            }
+            __syncthreads();
+        }
+    }
     for (int p0 = r * piece; p0 < n_pos; p0 += kMhaCluster * piece) {
         const int p = p0 + tid;
         const bool valid = tid < piece && p < n_pos;
         float sc = -INFINITY;
         if (valid) {
-            const uint4* krow = reinterpret_cast<const uint4*>(Kc + (static_cast<size_t>(h) * Lmax + p) * dh);
             float acc = 0.0f;
+            if (pf) {
+                // a row per thread out of shared memory; the threads of a quarter warp start at different 16-byte groups
+                const uint4* krow = reinterpret_cast<const uint4*>(kvs + tid * row_b);
+#pragma unroll 8
+                for (int c = 0; c < col_groups; ++c) {
+                    int cc = c + tid;
+                    cc -= (cc / col_groups) * col_groups;
+                    float kf[E];
+                    Elem<T>::widen(krow[cc], kf);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc = fmaf(kf[e], q_s[cc * E + e], acc);
+                }
+            } else {
+            const uint4* krow = reinterpret_cast<const uint4*>(Kc + (static_cast<size_t>(h) * Lmax + p) * dh);
 #pragma unroll 8
             for (int c = 0; c < col_groups; ++c) {
                 float kf[E];
                 Elem<T>::widen(APPEND ? __ldcg(krow + c) : __ldg(krow + c), kf);
 #pragma unroll
                 for (int e = 0; e < E; ++e) acc = fmaf(kf[e], q_s[c * E + e], acc);
+            }
             }
             sc = acc;
         }
@@ -464,11 +525,13 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
             float part[E];
 #pragma unroll
             for (int k = 0; k < E; ++k) part[k] = 0.0f;
-            const uint4* vbase = reinterpret_cast<const uint4*>(Vc + (static_cast<size_t>(h) * Lmax + p0) * dh) + cg;
+            const uint4* vbase = pf ? reinterpret_cast<const uint4*>(kvs + piece * row_b) + cg
+                                    : reinterpret_cast<const uint4*>(Vc + (static_cast<size_t>(h) * Lmax + p0) * dh) + cg;
 #pragma unroll 8
             for (int pp = pg; pp < n_valid; pp += pos_groups) {
                 float vf[E];
-                Elem<T>::widen(APPEND ? __ldcg(vbase + static_cast<size_t>(pp) * col_groups) : __ldg(vbase + static_cast<size_t>(pp) * col_groups), vf);
+                const uint4* vp = vbase + static_cast<size_t>(pp) * col_groups;
+                Elem<T>::widen(pf ? *vp : (APPEND ? __ldcg(vp) : __ldg(vp)), vf);
                 const float wp = w_s[pp];
 #pragma unroll
                 for (int k = 0; k < E; ++k) part[k] = fmaf(wp, vf[k], part[k]);
@@ -643,14 +706,18 @@ static halo_status group_mha_typed(const halo_mha_shape& sh, const void* Wp, con
         // one launch: a cluster of eight thread blocks per kept head
         const int iters_f = (d / E + 255) / 256;
         const dim3 grid_f(kMhaCluster, H);
-        const size_t smem_f = sizeof(float) * d;
+        const size_t kv_b = kv_smem_bytes(pos, dh, sizeof(T));
+        const size_t smem_f = sizeof(float) * d + kv_b;
 #define HALO_MHA_FUSED(I)                                                                                            \
-    case I:                                                                                                          \
+    case I: {                                                                                                        \
+        static bool once[64] = {};                                                                                   \
+        if (!ensure_dynamic_smem(mha_fused_kernel<T, I, false>, kMhaSmemLimit, once)) return HALO_ERR_CUDA; \
         mha_fused_kernel<T, I, false><<<grid_f, 256, smem_f, st>>>(                                                   \
             d, H, dh, sh.max_len, pos, static_cast<const T*>(Wp), static_cast<const T*>(x), static_cast<const T*>(Kc), \
             static_cast<const T*>(Vc), keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, nullptr, nullptr,  \
-            nullptr, nullptr);                                                                                       \
-        break;
+            nullptr, nullptr, kv_b ? 1 : 0);                                                                         \
+        break;                                                                                                       \
+    }
         switch (iters_f) {
             HALO_MHA_FUSED(1)
             HALO_MHA_FUSED(2)
@@ -724,7 +791,8 @@ static halo_status mha_block_typed(const halo_mha_shape& sh, const void* Wp, con
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(kMhaCluster, H);
     cfg.blockDim = dim3(256);
-    cfg.dynamicSmemBytes = sizeof(float) * d;
+    const size_t kv_b = kv_smem_bytes(pos, dh, sizeof(T));
+    cfg.dynamicSmemBytes = sizeof(float) * d + kv_b;
     cfg.stream = st;
     cudaLaunchAttribute attr{};
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -737,11 +805,16 @@ static halo_status mha_block_typed(const halo_mha_shape& sh, const void* Wp, con
     T* Kw_t = static_cast<T*>(Kc); T* Vw_t = static_cast<T*>(Vc);
     const int Lmax = sh.max_len;
     cudaError_t err = cudaSuccess;
+    const int kv_flag = kv_b ? 1 : 0;
 #define HALO_MHA_BLOCK(I)                                                                                            \
-    case I:                                                                                                          \
+    case I: {                                                                                                        \
+        static bool once[64] = {};                                                                                   \
+        if (!ensure_dynamic_smem(mha_fused_kernel<T, I, true>, kMhaSmemLimit, once)) return HALO_ERR_CUDA; \
         err = cudaLaunchKernelEx(&cfg, mha_fused_kernel<T, I, true>, d, H, dh, Lmax, pos, Wp_t, x_t, Kc_t, Vc_t,      \
-                                 keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, Wk_t, Wv_t, Kw_t, Vw_t); \
-        break;
+                                 keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, Wk_t, Wv_t, Kw_t, Vw_t, \
+                                 kv_flag);                                                                            \
+        break;                                                                                                       \
+    }
     switch (iters) {
         HALO_MHA_BLOCK(1)
         HALO_MHA_BLOCK(2)

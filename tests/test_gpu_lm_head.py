@@ -31,7 +31,8 @@ def _run(W, x, S, keep, dtype_code, fill=-123.0):
 
 
 @pytest.mark.parametrize("dtype,code,tol", [(torch.bfloat16, B.BF16, U.TOL_BF16), (torch.float32, B.F32, U.TOL_F32)])
-@pytest.mark.parametrize("vocab,d,S,n_tok", [(1000, 512, 256, 1), (777, 1024, 100, 3), (50, 64, 256, 2), (4099, 2048, 256, 1)])
+@pytest.mark.parametrize("vocab,d,S,n_tok", [(1000, 512, 256, 1), (777, 1024, 100, 3), (50, 64, 256, 2), (4099, 2048, 256, 1),
+                                             (1003, 4096, 96, 1), (5, 4096, 256, 1), (300, 2048, 20, 1)])
 def test_lm_head_groups_match_the_oracle(dtype, code, tol, vocab, d, S, n_tok):
     g = torch.Generator().manual_seed(vocab + d)
     W = (torch.randn((vocab, d), generator=g) / np.sqrt(d)).to(dtype).to(DEV)
@@ -52,6 +53,18 @@ def test_lm_head_flags_a_bad_group_index_and_computes_the_rest():
     assert status & 1 or status != 0
     ref = R.group_lm_head(W.cpu().numpy(), x.cpu().numpy(), 64, [0, 2], fill=-123.0)
     assert np.abs(got - ref).max() <= U.TOL_F32 * np.abs(ref[ref != -123.0]).max()
+
+
+def test_lm_head_streaming_form_flags_a_bad_group_index_and_computes_the_rest():
+    """One token, bf16, d 4096: the shared-memory ring form; a bad index in the list costs a status bit, not the call."""
+    g = torch.Generator().manual_seed(3)
+    W = (torch.randn((700, 4096), generator=g) / 64.0).to(torch.bfloat16).to(DEV)
+    x = torch.randn((1, 4096), generator=g).to(torch.bfloat16).to(DEV)
+    got, status = _run(W, x, 64, [0, 99, 10, -1, 2], B.BF16)
+    assert status != 0
+    ref = R.group_lm_head(synth.host_bits(W), synth.host_bits(x), 64, [0, 10, 2], fill=-123.0)
+    rms = np.sqrt(np.mean(R.group_lm_head(synth.host_bits(W), synth.host_bits(x), 64) ** 2))
+    assert np.abs(got - ref).max() <= U.TOL_BF16 * rms
 
 
 def test_lm_head_full_vocabulary_at_7b_width():

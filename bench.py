@@ -340,14 +340,14 @@ def other_blocks_report(dev, peak, reps=12):
             fn()
         torch.cuda.synchronize()
         ts = []
-        for _ in range(reps):          # eight calls back to back per window: launch latency is not what is measured
+        for _ in range(reps):          # 32 calls back to back per window: the first launch's latency is not what is measured
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
-            for _ in range(8):
+            for _ in range(32):
                 fn()
             b.record()
             torch.cuda.synchronize()
-            ts.append(a.elapsed_time(b) * 1e3 / 8)
+            ts.append(a.elapsed_time(b) * 1e3 / 32)
         return float(sorted(ts)[len(ts) // 2])
 
     g = torch.Generator(device="cpu").manual_seed(11)

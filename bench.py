@@ -87,7 +87,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, reasons, mx = [], set(), None
+        sm, reasons, mx, pw = [], set(), None, []
         try:
             for ln in open(self.path):
                 f = [v.strip() for v in ln.split(",")]
@@ -97,6 +97,10 @@ class ClockSampler:
                     sm.append(float(f[1])); mx = float(f[2])
                 except ValueError:
                     continue
+                try:
+                    pw.append(float(f[3]))
+                except ValueError:
+                    pass
                 for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
                     if v.lower().startswith("active"):
                         reasons.add(name)
@@ -106,6 +110,8 @@ class ClockSampler:
         if sm:
             busy = [v for v in sm if v >= 0.5 * max(sm)] or sm
             out.update(sm_mhz=statistics.median(busy), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+            if pw:
+                out.update(power_w_max=max(pw))
         return out
 
 

@@ -469,6 +469,7 @@ struct halo_stack {
     int mode;                      // 0 = automatic, 1 = one launch per step of the path
     bool persistent_ok;
     const void** d_W;              // device pointer tables
+    const void** d_Wsc;            // ... of the int4 scales (int4 stacks)
     const void** d_W1;
     const void** d_W2;
     float* p_partials;             // [3][2][d]
@@ -580,13 +581,14 @@ halo_status stack_create_impl(halo_stack** out, const halo_ffn_shape* ffn, const
     const size_t o_so = carve(sizeof(float) * s->stage_steps * step_elems);
     const size_t o_tw = carve(sizeof(void*) * n_layers), o_tw1 = carve(sizeof(void*) * n_layers);
     const size_t o_tw2 = carve(sizeof(void*) * n_layers);
+    const size_t o_tws = carve(sizeof(void*) * n_layers);
     const size_t o_pp = carve(sizeof(float) * 3 * 2 * d);
     const size_t o_pz = carve(sizeof(float) * 2 * pred->rank);
     const size_t o_ps = carve(sizeof(PersistSel) * 3);
     const size_t o_py = carve(sizeof(unsigned) * 64);
     constexpr size_t kMaxGrid = 192;   // thread blocks of the persistent kernel (one per SM)
     const size_t o_xh = carve(2 * d * 2);
-    const size_t o_dr = carve(persistent_supported(*ffn, n_tok, G) ? sizeof(float) * 2 * kMaxGrid * d : 16);
+    const size_t o_dr = carve(!i4_scales && persistent_supported(*ffn, n_tok, G) ? sizeof(float) * 2 * kMaxGrid * d : 16);
     const size_t ws_bytes = (!i4_scales && prefill_supported(*ffn, n_tok)) ? prefill_workspace_bytes(*ffn, n_tok) : 0;
     const size_t o_ws = carve(ws_bytes ? ws_bytes : 16);
     const size_t o_sc2 = carve(sizeof(float) * G), o_dg2 = carve(sizeof(int32_t) * G);
@@ -611,6 +613,7 @@ halo_status stack_create_impl(halo_stack** out, const halo_ffn_shape* ffn, const
     s->d_W = reinterpret_cast<const void**>(base + o_tw);
     s->d_W1 = reinterpret_cast<const void**>(base + o_tw1);
     s->d_W2 = reinterpret_cast<const void**>(base + o_tw2);
+    s->d_Wsc = reinterpret_cast<const void**>(base + o_tws);
     s->p_partials = reinterpret_cast<float*>(base + o_pp);
     s->p_z = reinterpret_cast<float*>(base + o_pz);
     s->p_sel = reinterpret_cast<PersistSel*>(base + o_ps);
@@ -651,7 +654,7 @@ halo_status stack_create_impl(halo_stack** out, const halo_ffn_shape* ffn, const
     if (option_value(OPT_CROSS_STAGES) >= 0) s->cross_stages = option_value(OPT_CROSS_STAGES);
     s->max_steps_per_launch = std::max(0, option_value(OPT_MAX_STEPS_PER_LAUNCH));
     if (option_value(OPT_L2_AHEAD) >= 0) s->l2_ahead = option_value(OPT_L2_AHEAD);
-    s->persistent_ok = !i4_scales && persistent_supported(*ffn, n_tok, G);
+    s->persistent_ok = i4_scales ? persistent_supported_i4(*ffn, n_tok, G) : persistent_supported(*ffn, n_tok, G);
     {
         // pointer tables, and the first block's selection: reliable block, all scores equal -> the priority
         // order is the group order, everything is kept (Sec. III-B.3, first layer)
@@ -673,6 +676,8 @@ halo_status stack_create_impl(halo_stack** out, const halo_ffn_shape* ffn, const
         ok = ok && cudaMemcpy(s->d_W, s->W.data(), sizeof(void*) * n_layers, cudaMemcpyHostToDevice) == cudaSuccess;
         ok = ok && cudaMemcpy(s->d_W1, s->W1.data(), sizeof(void*) * n_layers, cudaMemcpyHostToDevice) == cudaSuccess;
         ok = ok && cudaMemcpy(s->d_W2, s->W2.data(), sizeof(void*) * n_layers, cudaMemcpyHostToDevice) == cudaSuccess;
+        if (i4_scales)
+            ok = ok && cudaMemcpy(s->d_Wsc, s->i4_scales.data(), sizeof(void*) * n_layers, cudaMemcpyHostToDevice) == cudaSuccess;
         if (!ok) { cudaFree(s->slab); delete s; return HALO_ERR_CUDA; }
         if (n_tok > 1 && !i4_scales && prompt_stack_supported(*ffn, *pred, n_layers, n_tok)) {
             // persistent prompt kernel: tensor maps (encoded once, here), two H buffers, control words, one selection
@@ -758,7 +763,10 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
     const int L = s->n_layers, G = s->G, n_dev = s->n_dev;
     long long launches = 0;
     halo_status rc;
-    if (s->persistent_ok && !(s->mode & HALO_STACK_PER_STEP_LAUNCHES)) {
+    // (the int4 form of the kernel has neither the serialised-predictor arm nor the fixed-order sums)
+    const bool i4_stack = !s->i4_scales.empty();
+    if (s->persistent_ok && !(s->mode & HALO_STACK_PER_STEP_LAUNCHES) &&
+        !(i4_stack && (s->mode & (HALO_STACK_PRED_SERIAL | HALO_STACK_DETERMINISTIC)))) {
         // whole run in one cooperative launch
         if (cudaMemsetAsync(s->p_partials, 0, sizeof(float) * 3 * 2 * d, st) != cudaSuccess ||
             cudaMemsetAsync(s->p_sync, 0, sizeof(unsigned) * 64, st) != cudaSuccess)
@@ -770,6 +778,8 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
         P.W = reinterpret_cast<const __nv_bfloat16* const*>(s->d_W);
         P.W1 = reinterpret_cast<const __nv_bfloat16* const*>(s->d_W1);
         P.W2 = reinterpret_cast<const __nv_bfloat16* const*>(s->d_W2);
+        P.i4 = i4_stack ? 1 : 0;
+        P.Wsc = reinterpret_cast<const __nv_bfloat16* const*>(s->d_Wsc);
         P.h0 = h0; P.h_out = h_out; P.partials = s->p_partials; P.z = s->p_z; P.sel = s->p_sel; P.sync = s->p_sync;
         P.status = s->status;
         P.plan = s->plan.dev;

@@ -16,6 +16,7 @@
 
 #include "common.cuh"
 #include "ffn_math.cuh"
+#include "i4_math.cuh"
 #include "tma.cuh"
 
 namespace halo {
@@ -25,7 +26,6 @@ constexpr int kQBlock = 128;
 constexpr int kI4Threads = 256;
 constexpr int kI4Warps = kI4Threads / 32;
 constexpr int kI4BlocksPerSm = 2;
-constexpr float kNibbleBias = 136.0f;      // 128 from the bf16 trick + 8 from the code's zero point
 
 __device__ __forceinline__ uint32_t nibble_pair_bf16(uint32_t word, int k) {
     return ((word >> (4 * k)) & 0x000F000Fu) | 0x43004300u;      // {128 + nibble k, 128 + nibble k+4} as bf16x2
@@ -38,12 +38,7 @@ __device__ __forceinline__ uint32_t nibble_pair_mulhi(uint32_t word, uint32_t mu
     return (__umulhi(word, mul) & 0x000F000Fu) | 0x43004300u;
 }
 
-// Mask and exponent bits as run-time values held in registers: with two immediates the "and, then or" is two logic
-// instructions, with register operands it is one three-input instruction.
-struct PairBits { uint32_t mask, magic; };
-__device__ __forceinline__ uint32_t nibble_pair_r(uint32_t shifted_word, const PairBits& pb) {
-    return (shifted_word & pb.mask) | pb.magic;
-}
+
 
 template <typename T>
 __global__ void __launch_bounds__(256)

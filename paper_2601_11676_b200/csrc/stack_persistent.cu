@@ -24,6 +24,7 @@
 
 #include "common.cuh"
 #include "ffn_math.cuh"
+#include "i4_math.cuh"
 #include "select_device.cuh"
 #include "stack_persistent.cuh"
 #include "tma.cuh"
@@ -159,9 +160,17 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&v)[N]) {
 //   phase 1  warp w reads lanes 32 * (w % 4) ..; the four warps w / 4 = 0..3 take rows w / 4, w / 4 + 4, ...; a thread
 //            keeps the PPR chunks of x that meet its lane.
 //   phase 2  thread tid owns the same columns as in the plain form (chunk tid % (512 / REP)), piece = chunk / 128.
-template <int NB, int XC, int P2, int REP, int STAGES, bool TM>
+// I4 = true: the FFN weights are int4 codes with one bf16 scale per 128 elements (the layout of halo_group_ffn_i4).
+// A stage is a batch of NB = 8 neurons: three planes of code rows (d / 2 bytes each) and three runs of scales, six bulk
+// copies.  Phase 1: warp w takes code row w of the 16 (8 gate, 8 up) against x kept in shared memory in the nibble
+// pairing (XC = 16-byte chunks per lane); phase 2: 512 / (d / 16) replicas of d / 16 threads, a thread owns 16 columns;
+// the replicas' sums meet in the one vector buffer in turn.  Predictor rows (bf16) ride the same ring, at most
+// stage_bytes / (2 d) of them per stage, two warps per row against x (bf16) in shared memory.  Skeleton (selector,
+// producer, grid barrier, merge, glue) as for bf16; the modes PRED_SERIAL and DETERMINISTIC are not built for it.
+template <int NB, int XC, int P2, int REP, int STAGES, bool TM, bool I4>
 __global__ void __launch_bounds__(TM ? kPThreadsTM : kPThreads, 1)
 stack_decode_kernel(const __grid_constant__ PersistParams P) {
+    static_assert(!I4 || (!TM && NB == 8 && P2 == 1 && REP == 1), "int4 shape");
     constexpr int ROWS = 2 * NB;
     constexpr int WPR = TM ? 4 : kPCWarps / ROWS;
     constexpr int PPR = XC;                       // TM: 2 KB pieces per row = chunks of x per thread
@@ -173,13 +182,20 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
     constexpr int kVecBytesPerCol = 4 * REP;
     unsigned char* vec_buf = smem_raw + kHeaderBytes;
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(vec_buf);
-    unsigned char* ring = smem_raw + kHeaderBytes + static_cast<size_t>(P.d) * kVecBytesPerCol;
+    // I4: behind the vector buffer, x in the nibble pairing [4][d/32] uint4 and its plain sums per 32 elements
+    uint4* xp = reinterpret_cast<uint4*>(smem_raw + kHeaderBytes + static_cast<size_t>(P.d) * kVecBytesPerCol);
+    float* xsum = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(xp) + static_cast<size_t>(P.d) * 2);
+    unsigned char* ring = smem_raw + kHeaderBytes + static_cast<size_t>(P.d) * kVecBytesPerCol +
+                          (I4 ? static_cast<size_t>(P.d) * 2 + ((static_cast<size_t>(P.d) / 32 * 4 + 127) & ~size_t(127)) : 0);
 
     const int d = P.d, S = P.S, G = P.G, L = P.L, r = P.r, n_dev = P.plan.n_dev;
     const int chunks = d >> 3;
-    const uint32_t row_bytes = static_cast<uint32_t>(d) * 2u;
-    const uint32_t plane_bytes = row_bytes * NB;
-    const uint32_t stage_bytes = 3u * plane_bytes;
+    const uint32_t row_bytes = static_cast<uint32_t>(d) * 2u;                 // a bf16 row (predictor rows; FFN rows of the bf16 form)
+    const uint32_t crow_bytes = static_cast<uint32_t>(d) / 2u;                // I4: a row of codes
+    const uint32_t sc_bytes = static_cast<uint32_t>(d / 128) * 2u * NB;       // I4: scales of one plane of a batch
+    const uint32_t plane_bytes = (I4 ? crow_bytes : row_bytes) * NB;
+    const uint32_t stage_bytes = I4 ? 3u * (plane_bytes + sc_bytes) : 3u * plane_bytes;
+    const int pred_rows = I4 ? min(8, static_cast<int>(stage_bytes / row_bytes)) : ROWS;   // predictor rows per stage
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int grid = gridDim.x, cta = blockIdx.x;
     const int workers = grid - 1;                 // thread blocks that stream weights; the last one selects
@@ -340,8 +356,8 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                         const int r0 = static_cast<int>(static_cast<long long>(cta) * r / workers);
                         const int r1 = static_cast<int>(static_cast<long long>(cta + 1) * r / workers);
                         const __nv_bfloat16* W1 = P.W1[lp];
-                        for (int row = r0; row < r1 && alive; row += ROWS) {
-                            const int n = min(ROWS, r1 - row);
+                        for (int row = r0; row < r1 && alive; row += pred_rows) {
+                            const int n = min(pred_rows, r1 - row);
                             int s;
                             if (!acquire(s)) { alive = false; break; }
                             sm.type[s] = ST_PRED; sm.arg0[s] = row; sm.arg1[s] = n;
@@ -379,7 +395,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 const long long U = static_cast<long long>(nk) * per_group;
                 // (c') keep HBM busy while the consumers synchronise: the block's first batches go to L2 now, long
                 //      before ring slots free up for them (whoever ends up consuming them)
-                if (lane < P.l2_ahead) {
+                if (!I4 && lane < P.l2_ahead) {
                     const long long b = cta + static_cast<long long>(workers) * lane;
                     if (b < U) {
                         const int ki = static_cast<int>(b / per_group), j0 = static_cast<int>(b - static_cast<long long>(ki) * per_group) * NB;
@@ -420,10 +436,22 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                             const __nv_bfloat16* group = Wl + static_cast<size_t>(g) * 3 * S * d;
                             unsigned char* dst = ring + static_cast<size_t>(s) * stage_bytes;
                             mbar_arrive_expect_tx(&sm.full[s], stage_bytes);
+                            if constexpr (I4) {
+                                const unsigned char* Q = reinterpret_cast<const unsigned char*>(Wl);
+                                const __nv_bfloat16* Sc = P.Wsc[l];
+                                const int nb = d / 128;
+#pragma unroll
+                                for (int plane = 0; plane < 3; ++plane) {
+                                    const size_t rowi = static_cast<size_t>(g) * 3 * S + static_cast<size_t>(plane) * S + j0;
+                                    bulk_copy_g2s(dst + plane * plane_bytes, Q + rowi * crow_bytes, plane_bytes, &sm.full[s]);
+                                    bulk_copy_g2s(dst + 3 * plane_bytes + plane * sc_bytes, Sc + rowi * nb, sc_bytes, &sm.full[s]);
+                                }
+                            } else {
                             bulk_copy_g2s(dst, group + static_cast<size_t>(j0) * d, plane_bytes, &sm.full[s]);
                             bulk_copy_g2s(dst + plane_bytes, group + static_cast<size_t>(S + j0) * d, plane_bytes, &sm.full[s]);
                             bulk_copy_g2s(dst + 2 * plane_bytes, group + static_cast<size_t>(2 * S + j0) * d, plane_bytes,
                                           &sm.full[s]);
+                            }
                         }
                         ++it;
                         return true;
@@ -533,6 +561,17 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
     uint4 xq[XC];      // this lane's slice of x, packed bf16
     float acc[P2][8];
     float hreg[P2][8];
+    // I4: phase-2 replica and 16-column chunk of this thread, its sums, and the run-time copies of constants that keep
+    // the unpacking off the logic pipe (see group_ffn_i4.cu)
+    constexpr int kI4Acc = I4 ? 16 : 1;
+    float acc16[kI4Acc], corr = 0.0f;
+    const int i4_cols = d >> 4;                                   // 16-column chunks per row
+    const int i4_reps = kPC / max(i4_cols, 1);
+    const int i4_rep = tid / max(i4_cols, 1), i4_col = tid % max(i4_cols, 1);
+    const uint32_t rt_zero = static_cast<uint32_t>(P.steps) >> 31;
+    const uint32_t mul1 = 0x10000000u + rt_zero, mul2 = 0x01000000u + rt_zero, mul3 = 0x00100000u + rt_zero;
+    const uint32_t mul16 = 0x00010000u + rt_zero;
+    const PairBits pb{0x000F000Fu + rt_zero, 0x43004300u + rt_zero};
     int it = 0, red_par = 0;
     unsigned q = 0;  // running block counter over steps: partial buffers rotate with it
     const size_t acc_stride = static_cast<size_t>(d);
@@ -581,7 +620,24 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
             }
         }
         pc_barrier();  // xs complete; sm.reduce free again
-        if (want_x) {
+        if constexpr (I4) {
+            if (want_x) {
+                const uint16_t* xb = reinterpret_cast<const uint16_t*>(xs);
+                uint32_t* xp_words = reinterpret_cast<uint32_t*>(xp);
+                const int chunks16 = d / 32;
+                for (int i = tid; i < d / 2; i += kPC) {
+                    const int c = i / 16, rr = i - c * 16, w = rr >> 2, k = rr & 3;
+                    const uint32_t lo16 = xb[32 * c + 8 * w + k], hi16 = xb[32 * c + 8 * w + k + 4];
+                    xp_words[(static_cast<size_t>(w) * chunks16 + c) * 4 + k] = lo16 | (hi16 << 16);
+                }
+                for (int c = tid; c < chunks16; c += kPC) {
+                    float sx = 0.0f;
+                    for (int e = 0; e < 32; ++e) sx += __bfloat162float(xs[32 * c + e]);
+                    xsum[c] = sx;
+                }
+            }
+            pc_barrier();
+        } else if (want_x) {
 #pragma unroll
             for (int i = 0; i < XC; ++i) xq[i] = reinterpret_cast<const uint4*>(xs)[p1_base + p1_step * i];
         }
@@ -622,6 +678,9 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
             for (int p = 0; p < P2; ++p)
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc[p][e] = 0.0f;
+#pragma unroll
+            for (int e = 0; e < kI4Acc; ++e) acc16[e] = 0.0f;
+            corr = 0.0f;
             bool any = false;
             bool first_stage = true;
             trace(TR_BLOCK_START, global_timer_ns());
@@ -639,7 +698,49 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 const uint32_t tslot = tbase + tlane + static_cast<uint32_t>(s * kTSlotCols);   // TM: this warp's lanes of the slot
                 float* red = sm.red[red_par];
                 // ---- before the barrier: nothing in here may block on other consumers ----
-                if constexpr (TM) {
+                if constexpr (I4) {
+                    if (type == ST_FFN) {
+                        if (a0 >= 0) {
+                            any = true;
+                            // code rows 0..15 of the stage: 8 gate rows, then 8 up rows; this warp's row against xp
+                            const int chunks16 = d / 32, nbk = d / 128;
+                            const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(warp) * crow_bytes);
+                            const __nv_bfloat16* rs =
+                                reinterpret_cast<const __nv_bfloat16*>(stage + 3 * plane_bytes) + static_cast<size_t>(warp) * nbk;
+                            float a = 0.0f;
+#pragma unroll
+                            for (int u = 0; u < XC; ++u) {
+                                const int c = lane + 32 * u;
+                                const uint4 w4 = rp[c];
+                                const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
+                                float t0 = 0.0f, t1 = 0.0f;
+#pragma unroll
+                                for (int w = 0; w < 4; ++w) {
+                                    const uint4 xv = xp[static_cast<size_t>(w) * chunks16 + c];
+                                    fma_bf16x2(nibble_pair_r(ww[w], pb), xv.x, t0, t1);
+                                    fma_bf16x2(nibble_pair_r(ww[w] >> 4, pb), xv.y, t0, t1);
+                                    fma_bf16x2(nibble_pair_r(ww[w] >> 8, pb), xv.z, t0, t1);
+                                    fma_bf16x2(nibble_pair_r(__umulhi(ww[w], mul3), pb), xv.w, t0, t1);
+                                }
+                                a = fmaf(__bfloat162float(rs[c >> 2]), (t0 + t1) - kNibbleBias * xsum[c], a);
+                            }
+                            a = warp_sum(a);
+                            if (lane == 0) red[warp] = a;
+                        }
+                    } else if (type == ST_PRED) {
+                        // bf16 predictor rows: two warps per row, x (bf16) from shared memory
+                        const int prow = warp >> 1, ppart = warp & 1;
+                        if (prow < a1) {
+                            const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(prow) * row_bytes);
+                            const uint4* xv = reinterpret_cast<const uint4*>(xs);
+                            float dot0 = 0.0f, dot1 = 0.0f;
+                            const int half = chunks >> 1;
+                            for (int c = ppart * half + lane; c < (ppart + 1) * half; c += 32) dot_bf16x8(rp[c], xv[c], dot0, dot1);
+                            const float dot = warp_sum(dot0 + dot1);
+                            if (lane == 0) red[prow * 2 + ppart] = dot;
+                        }
+                    }
+                } else if constexpr (TM) {
                     if ((type == ST_FFN && a0 >= 0) || type == ST_PRED) {
                         if (type == ST_FFN) any = true;
                         const int n_rows = type == ST_FFN ? ROWS : a1;
@@ -693,7 +794,34 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 bad = pc_barrier_or(!ok);
                 if (bad) break;
                 // ---- after the barrier ----
-                if (type == ST_FFN) {
+                if (I4 && type == ST_FFN) {
+                    if constexpr (I4) {
+                        if (a0 >= 0 && i4_rep < i4_reps) {
+                            const int nbk = d / 128;
+                            const unsigned char* down = stage + 2 * plane_bytes;
+                            const __nv_bfloat16* ds = reinterpret_cast<const __nv_bfloat16*>(stage + 3 * plane_bytes) + static_cast<size_t>(2 * NB) * nbk;
+                            for (int j = i4_rep; j < NB; j += i4_reps) {
+                                const float h = silu_mul(red[j], red[NB + j]);
+                                const float f = h * __bfloat162float(ds[static_cast<size_t>(j) * nbk + (i4_col >> 3)]);
+                                corr += f;
+                                const uint2 w2 = reinterpret_cast<const uint2*>(down + static_cast<size_t>(j) * crow_bytes)[i4_col];
+                                const uint32_t words[2] = {w2.x, w2.y};
+#pragma unroll
+                                for (int v = 0; v < 2; ++v) {
+                                    const uint32_t pk[4] = {nibble_pair_r(words[v], pb), nibble_pair_r(__umulhi(words[v], mul1), pb),
+                                                            nibble_pair_r(__umulhi(words[v], mul2), pb),
+                                                            nibble_pair_r(__umulhi(words[v], mul3), pb)};
+#pragma unroll
+                                    for (int k = 0; k < 4; ++k) {
+                                        acc16[(8 * v + k) % kI4Acc] = fmaf(f, __uint_as_float(pk[k] * mul16), acc16[(8 * v + k) % kI4Acc]);
+                                        acc16[(8 * v + k + 4) % kI4Acc] = fmaf(f, __uint_as_float(pk[k]), acc16[(8 * v + k + 4) % kI4Acc]);
+                                    }
+                                }
+                            }
+                        }
+                    }
+                    red_par ^= 1;
+                } else if (type == ST_FFN) {
                     if (a0 >= 0) {
                         const unsigned char* down = stage + 2 * plane_bytes;
 #pragma unroll
@@ -724,7 +852,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                         float* zdst = P.z + static_cast<size_t>(n_pred & 1u) * r;
                         for (int i = 0; i < a1; ++i) {
                             float z = 0.0f;
-                            for (int w = 0; w < WPR; ++w) z += red[i * WPR + w];
+                            for (int w = 0; w < (I4 ? 2 : WPR); ++w) z += red[i * (I4 ? 2 : WPR) + w];
                             if (P.act == HALO_ACT_RELU) z = fmaxf(z, 0.0f);
                             zdst[a0 + i] = z;
                         }
@@ -743,7 +871,41 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
 
             // ------------------------------ end of the block: flush, grid barrier, merge + glue ------------------------------
             trace(TR_STAGES_DONE, global_timer_ns());
+            if constexpr (I4) {
+                if (any) {
+                    // the replicas' sums meet in the one vector buffer in turn; the offsets of the unpacking come off here
+                    // (upper elements: sum f * (128 + 0x4300 / 65536 + n_hi + n_lo / 65536), n_lo from the element 4 below)
+                    const float off = kNibbleBias * corr;
+                    const float off_hi = (kNibbleBias + 17152.0f / 65536.0f) * corr;
+                    float* dst = reinterpret_cast<float*>(vec_buf) + static_cast<size_t>(i4_col) * 16;
+                    for (int rr = 0; rr < i4_reps; ++rr) {
+                        if (i4_rep == rr) {
+#pragma unroll
+                            for (int v = 0; v < 16; v += 8) {
+                                float4 lo4, hi4;
+                                float* lo = reinterpret_cast<float*>(&lo4);
+                                float* hi = reinterpret_cast<float*>(&hi4);
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    lo[k] = acc16[(v + k) % kI4Acc] - off;
+                                    hi[k] = (acc16[(v + k + 4) % kI4Acc] - off_hi) - (acc16[(v + k) % kI4Acc] - 128.0f * corr) * (1.0f / 65536.0f);
+                                }
+                                if (rr > 0) {
+                                    const float4 a = reinterpret_cast<const float4*>(dst + v)[0], b = reinterpret_cast<const float4*>(dst + v)[1];
+                                    lo4.x += a.x; lo4.y += a.y; lo4.z += a.z; lo4.w += a.w;
+                                    hi4.x += b.x; hi4.y += b.y; hi4.z += b.z; hi4.w += b.w;
+                                }
+                                reinterpret_cast<float4*>(dst + v)[0] = lo4;
+                                reinterpret_cast<float4*>(dst + v)[1] = hi4;
+                            }
+                            fence_proxy_async_smem();
+                        }
+                        if (rr + 1 < i4_reps) pc_barrier();
+                    }
+                }
+            } else {
             if (any || P.deterministic) stage_sums();
+            }
             pc_barrier();
             if (P.deterministic) {
                 // this thread block's column sums (replicas added in index order) go to its own row
@@ -870,6 +1032,11 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
 
 // ---- host side -----------------------------------------------------------------------------------------
 
+bool persistent_supported_i4(const halo_ffn_shape& sh, int n_tok, int G) {
+    return sh.wdtype == HALO_BF16 && n_tok == 1 && G <= kPC && (sh.d_model == 2048 || sh.d_model == 4096) &&
+           sh.group_size % 8 == 0;
+}
+
 bool persistent_supported(const halo_ffn_shape& sh, int n_tok, int G) {
     if (sh.wdtype != HALO_BF16 || n_tok != 1 || G > kPC) return false;
     switch (sh.d_model) {
@@ -880,11 +1047,14 @@ bool persistent_supported(const halo_ffn_shape& sh, int n_tok, int G) {
     return false;
 }
 
-template <int NB, int XC, int P2, int REP, int STAGES, bool TM>
+template <int NB, int XC, int P2, int REP, int STAGES, bool TM, bool I4 = false>
 static halo_status launch_cfg(PersistParams& P, cudaStream_t st) {
-    auto kernel = stack_decode_kernel<NB, XC, P2, REP, STAGES, TM>;
+    auto kernel = stack_decode_kernel<NB, XC, P2, REP, STAGES, TM, I4>;
     constexpr int kThreads = TM ? kPThreadsTM : kPThreads;
-    const size_t smem = kHeaderBytes + static_cast<size_t>(P.d) * 4 * REP + static_cast<size_t>(STAGES) * 3 * NB * P.d * 2;
+    const size_t dd = static_cast<size_t>(P.d);
+    const size_t smem = I4 ? kHeaderBytes + dd * 4 * REP + dd * 2 + ((dd / 32 * 4 + 127) & ~size_t(127)) +
+                                 static_cast<size_t>(STAGES) * 3 * NB * (dd / 2 + dd / 128 * 2)
+                           : kHeaderBytes + dd * 4 * REP + static_cast<size_t>(STAGES) * 3 * NB * dd * 2;
     static bool configured[64] = {};
     int dev = 0, sms = kSmCount;
     if (cudaGetDevice(&dev) != cudaSuccess) return HALO_ERR_CUDA;
@@ -907,6 +1077,13 @@ static halo_status launch_cfg(PersistParams& P, cudaStream_t st) {
 }
 
 halo_status launch_stack_persistent(PersistParams& P, cudaStream_t st) {
+    if (P.i4) {
+        switch (P.d) {
+            case 2048: return launch_cfg<8, 2, 1, 1, 4, false, true>(P, st);
+            case 4096: return launch_cfg<8, 4, 1, 1, 3, false, true>(P, st);
+        }
+        return HALO_ERR_UNIMPLEMENTED;
+    }
     switch (P.d) {
         case 2048: return P.tmem_ring ? launch_cfg<4, 2, 1, 2, 4, true>(P, st) : launch_cfg<4, 4, 1, 2, 4, false>(P, st);
         case 4096: return P.tmem_ring ? launch_cfg<2, 4, 1, 1, 4, true>(P, st) : launch_cfg<2, 4, 1, 1, 4, false>(P, st);

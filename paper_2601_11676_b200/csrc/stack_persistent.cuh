@@ -41,6 +41,8 @@ struct PersistParams {
                                            // have passed the grid barrier of the current block
     int l2_ahead;                          // batches per thread block prefetched into L2 on entering a block
     int tmem_ring;                         // 1: stages pass through tensor memory (d_model 2048 / 4096 only)
+    int i4;                                // 1: W holds int4 codes (uint8), Wsc their bf16 scales per 128 elements
+    const __nv_bfloat16* const* Wsc;       // device table [L] (i4 only)
     int pred_serial;                       // 1: the predictor rows and the selection of block l run at the start of
                                            // block l itself (from the recorded x_{l-1}), not beside block l-1
     int deterministic;                     // 1: fixed batch assignment and fixed-order sums (bitwise repeatable)
@@ -52,6 +54,7 @@ struct PersistParams {
 };
 
 bool persistent_supported(const halo_ffn_shape& sh, int n_tok, int G);
+bool persistent_supported_i4(const halo_ffn_shape& sh, int n_tok, int G);   // int4 codes + scales
 halo_status launch_stack_persistent(PersistParams& P, cudaStream_t st);
 
 }  // namespace halo

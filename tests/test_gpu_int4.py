@@ -130,10 +130,12 @@ def _full_block_all_groups():
     assert np.sqrt(np.mean(diff ** 2)) <= 0.5 * np.sqrt(np.mean(R.merge(P16) ** 2))
 
 
-@pytest.mark.parametrize("name,layers,steps", [("tinyllama-1.1b-decode", 3, 3), ("llama2-7b-decode", 3, 2)])
-def test_int4_stack_teacher_forced(name, layers, steps):
+@pytest.mark.parametrize("mode", [0, B.STACK_PER_STEP_LAUNCHES, B.STACK_LOAD_SERIAL, B.STACK_DETERMINISTIC])
+@pytest.mark.parametrize("name,layers,steps", [("tinyllama-1.1b-decode", 4, 3), ("llama2-7b-decode", 3, 3)])
+def test_int4_stack_teacher_forced(name, layers, steps, mode):
     """The FFN stack on int4 weights (halo_stack_create_i4): scores and selections as for the bf16 stack, every block's
-    output against the oracle's FFN on the dequantised weights from the recorded input."""
+    output against the oracle's FFN on the dequantised weights from the recorded input.  Mode 0 and LOAD_SERIAL run as
+    one persistent launch, the others as one launch per step of the path."""
     wl = synth.small_variant(synth.workload(name), layers, steps)
     L, G, d, n = wl.n_layers, wl.n_groups, wl.d_model, wl.n_dev
     hb = synth.host_bits
@@ -156,9 +158,14 @@ def test_int4_stack_teacher_forced(name, layers, steps):
              n_keep=torch.zeros((steps, L), dtype=torch.int32, device=DEV),
              y=torch.zeros((steps, L, 1, d), dtype=torch.float32, device=DEV))
     taps = B.Taps(*[t[k].data_ptr() for k in ("x", "scores", "dev_of_group", "arrived", "keep_list", "n_keep", "y")])
+    stack.set_mode(mode)
     stack.decode(h0, steps, 2, h_out, taps)
     torch.cuda.synchronize()
-    assert stack.status() == 0 and stack.last_launches() > steps * L
+    assert stack.status() == 0
+    if mode in (0, B.STACK_LOAD_SERIAL):
+        assert stack.last_launches() == 1                  # the persistent kernel
+    else:
+        assert stack.last_launches() > steps * L
     x_all = hb(t["x"])
     lost = 0
     for s in range(steps):

@@ -33,9 +33,9 @@ NOMINAL_HBM_GBS = 8000.0
 # groups processed, so the ratio carries over to the full-size launch.  The figure belongs to the kernel sources with
 # the hash below: when they change the line reports no traffic until the counters have been taken again.
 STACK_KERNEL_TRAFFIC_RATIO = 1.0005
-STACK_KERNEL_SOURCES = ("stack_persistent.cu", "stack_persistent.cuh", "ffn_math.cuh", "tma.cuh", "umma.cuh",
+STACK_KERNEL_SOURCES = ("stack_persistent.cu", "stack_persistent.cuh", "ffn_math.cuh", "i4_math.cuh", "tma.cuh", "umma.cuh",
                         "select_device.cuh")
-STACK_KERNEL_SOURCES_SHA1 = "45f77459a6c9ab59f4e93c4f7b4143d6a9bd9f91"
+STACK_KERNEL_SOURCES_SHA1 = "13df837cf1ac5e76773b5ef1c6216963b6aa9f89"
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -517,7 +517,8 @@ def overlap_ablation(dev, steps=48, warm=4):
 
 def int4_stack_report(dev, peak, steps=32, warm=4):
     """The 7B-shaped FFN stack on int4 group-quantised weights (the paper's models are 4-bit): tokens/s and GB/s over the
-    int4 bytes of the kept groups (codes + scales) and the predictors.  One launch per step of the path."""
+    int4 bytes of the kept groups (codes + scales) and the predictors.  One persistent launch (the int4 form of the
+    decode kernel)."""
     from paper_2601_11676_b200 import binding as B
     wl = synth.workload("llama2-7b-decode")
     L, G, S, d = wl.n_layers, wl.n_groups, wl.group_size, wl.d_model

@@ -59,6 +59,7 @@ struct PersistSmem {
     float score[HALO_MAX_GROUPS];
     int kept_group[HALO_MAX_GROUPS];   // producer's table for the block it is issuing: group id or -1 per kept position
     SelectSmem sel;
+    float red_h[2][2][32];   // I4 form: [half][parity][row]
     // second level of the ring, in tensor memory (TM form of the kernel)
     uint64_t tfull[8];
     uint64_t tempty[8];
@@ -81,6 +82,19 @@ __device__ __forceinline__ bool pc_barrier_or(bool flag) {
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(out)
         : "r"(static_cast<uint32_t>(flag)), "n"(kPC)
+        : "memory");
+    return out != 0;
+}
+// I4 form: the consumers work as two halves of 256 threads on alternate stages; barrier (with OR) over one half
+__device__ __forceinline__ bool half_barrier_or(int half, bool flag) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"(static_cast<uint32_t>(flag)), "r"(3 + half), "n"(kPC / 2)
         : "memory");
     return out != 0;
 }
@@ -207,7 +221,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
     unsigned* const sync_selready = P.sync + 3;
 
     if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], TM ? 1 : kPCWarps); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], TM ? 1 : (I4 ? kPCWarps / 2 : kPCWarps)); }
         if constexpr (TM) {
             // tfull: one arrival from the copies' completion, one from the mover after it wrote the slot's metadata
             for (int t = 0; t < kTSlots; ++t) { mbar_init(&sm.tfull[t], 2); mbar_init(&sm.tempty[t], kPCWarps); }
@@ -479,6 +493,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                         }
                     }
                     if (alive) alive = marker(ST_END, 0);
+                    if (I4 && alive) alive = marker(ST_END, 0);   // one for each half of the consumers
                 }
                 ++qp;
                 issued_in_block = 0;
@@ -573,6 +588,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
     const uint32_t mul16 = 0x00010000u + rt_zero;
     const PairBits pb{0x000F000Fu + rt_zero, 0x43004300u + rt_zero};
     int it = 0, red_par = 0;
+    int it_half = warp >> 3;       // I4 form: the next stage of this thread's half (stages alternate between the halves)
     unsigned q = 0;  // running block counter over steps: partial buffers rotate with it
     const size_t acc_stride = static_cast<size_t>(d);
     const size_t buf_stride = static_cast<size_t>(kAccBufs) * d;
@@ -622,18 +638,23 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
         pc_barrier();  // xs complete; sm.reduce free again
         if constexpr (I4) {
             if (want_x) {
-                const uint16_t* xb = reinterpret_cast<const uint16_t*>(xs);
-                uint32_t* xp_words = reinterpret_cast<uint32_t*>(xp);
+                // one 16-byte piece of x (8 elements e0..e7) per thread: its nibble pairing is (e0,e4) (e1,e5) (e2,e6) (e3,e7);
+                // the four threads of a 32-element chunk add up its plain sum
                 const int chunks16 = d / 32;
-                for (int i = tid; i < d / 2; i += kPC) {
-                    const int c = i / 16, rr = i - c * 16, w = rr >> 2, k = rr & 3;
-                    const uint32_t lo16 = xb[32 * c + 8 * w + k], hi16 = xb[32 * c + 8 * w + k + 4];
-                    xp_words[(static_cast<size_t>(w) * chunks16 + c) * 4 + k] = lo16 | (hi16 << 16);
-                }
-                for (int c = tid; c < chunks16; c += kPC) {
-                    float sx = 0.0f;
-                    for (int e = 0; e < 32; ++e) sx += __bfloat162float(xs[32 * c + e]);
-                    xsum[c] = sx;
+                for (int i = tid; i < (d >> 3); i += kPC) {
+                    const int c = i >> 2, w = i & 3;
+                    const uint4 v = reinterpret_cast<const uint4*>(xs)[i];
+                    uint4 o;
+                    o.x = __byte_perm(v.x, v.z, 0x5410); o.y = __byte_perm(v.x, v.z, 0x7632);
+                    o.z = __byte_perm(v.y, v.w, 0x5410); o.w = __byte_perm(v.y, v.w, 0x7632);
+                    xp[static_cast<size_t>(w) * chunks16 + c] = o;
+                    float sx = (__uint_as_float(v.x << 16) + __uint_as_float(v.x & 0xffff0000u)) +
+                               (__uint_as_float(v.y << 16) + __uint_as_float(v.y & 0xffff0000u)) +
+                               (__uint_as_float(v.z << 16) + __uint_as_float(v.z & 0xffff0000u)) +
+                               (__uint_as_float(v.w << 16) + __uint_as_float(v.w & 0xffff0000u));
+                    sx += __shfl_xor_sync(0xffffffffu, sx, 1);
+                    sx += __shfl_xor_sync(0xffffffffu, sx, 2);
+                    if (w == 0) xsum[c] = sx;
                 }
             }
             pc_barrier();
@@ -686,6 +707,120 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
             trace(TR_BLOCK_START, global_timer_ns());
 
             // ------------------------------ stages of this block ------------------------------
+            if constexpr (I4) {
+                // Two halves of 8 warps take alternate stages (each with its own barrier), so that one half's phase
+                // change and waits are covered by the other half's arithmetic.  Phase 1: warp w of the half takes the gate
+                // and the up row of neuron w and reads x once for both; phase 2: a thread owns 16 columns, 256 / (d/16)
+                // replicas per half.  The producer ends a block with two END markers, one per half.
+                const int half = warp >> 3, hw = warp & 7, ht = tid & 255;
+                const int chunks16 = d / 32, nbk = d / 128;
+                const int rh = (kPC / 2) / max(i4_cols, 1);           // replicas inside a half
+                const int hrep = ht / max(i4_cols, 1);
+                int hpar = 0;
+                bool hbad = false;
+                while (true) {
+                    const int itx = it_half;
+                    const int s = itx % STAGES;
+                    const uint32_t parity = static_cast<uint32_t>(itx / STAGES) & 1u;
+                    const bool ok = mbar_wait_bounded(&sm.full[s], parity, abort_flag);
+                    if (first_stage && half == 0) { trace(TR_FIRST_STAGE, global_timer_ns()); first_stage = false; }
+                    const int type = sm.type[s], a0 = sm.arg0[s], a1 = sm.arg1[s];
+                    const unsigned char* stage = ring + static_cast<size_t>(s) * stage_bytes;
+                    float* red = sm.red_h[half][hpar];
+                    if (ok && type == ST_FFN && a0 >= 0) {
+                        any = true;
+                        const uint4* rg = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(hw) * crow_bytes);
+                        const uint4* ru = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(NB + hw) * crow_bytes);
+                        const __nv_bfloat16* sc0 = reinterpret_cast<const __nv_bfloat16*>(stage + 3 * plane_bytes);
+                        const __nv_bfloat16* sg = sc0 + static_cast<size_t>(hw) * nbk;
+                        const __nv_bfloat16* su = sc0 + static_cast<size_t>(NB + hw) * nbk;
+                        float ag = 0.0f, au = 0.0f;
+#pragma unroll
+                        for (int u = 0; u < XC; ++u) {
+                            const int c = lane + 32 * u;
+                            const uint4 g4 = rg[c], u4 = ru[c];
+                            const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w};
+                            const uint32_t uw[4] = {u4.x, u4.y, u4.z, u4.w};
+                            float g0 = 0.0f, g1 = 0.0f, u0 = 0.0f, u1 = 0.0f;
+#pragma unroll
+                            for (int w = 0; w < 4; ++w) {
+                                const uint4 xv = xp[static_cast<size_t>(w) * chunks16 + c];
+                                fma_bf16x2(nibble_pair_r(gw[w], pb), xv.x, g0, g1);
+                                fma_bf16x2(nibble_pair_r(uw[w], pb), xv.x, u0, u1);
+                                fma_bf16x2(nibble_pair_r(gw[w] >> 4, pb), xv.y, g0, g1);
+                                fma_bf16x2(nibble_pair_r(uw[w] >> 4, pb), xv.y, u0, u1);
+                                fma_bf16x2(nibble_pair_r(gw[w] >> 8, pb), xv.z, g0, g1);
+                                fma_bf16x2(nibble_pair_r(uw[w] >> 8, pb), xv.z, u0, u1);
+                                fma_bf16x2(nibble_pair_r(__umulhi(gw[w], mul3), pb), xv.w, g0, g1);
+                                fma_bf16x2(nibble_pair_r(__umulhi(uw[w], mul3), pb), xv.w, u0, u1);
+                            }
+                            const float offx = kNibbleBias * xsum[c];
+                            ag = fmaf(__bfloat162float(sg[c >> 2]), (g0 + g1) - offx, ag);
+                            au = fmaf(__bfloat162float(su[c >> 2]), (u0 + u1) - offx, au);
+                        }
+                        ag = warp_sum(ag);
+                        au = warp_sum(au);
+                        if (lane == 0) { red[hw] = ag; red[NB + hw] = au; }
+                    } else if (ok && type == ST_PRED) {
+                        // bf16 predictor rows: a warp per row, x (bf16) from shared memory
+                        if (hw < a1) {
+                            const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(hw) * row_bytes);
+                            const uint4* xv = reinterpret_cast<const uint4*>(xs);
+                            float dot0 = 0.0f, dot1 = 0.0f;
+                            for (int c = lane; c < chunks; c += 32) dot_bf16x8(rp[c], xv[c], dot0, dot1);
+                            const float dot = warp_sum(dot0 + dot1);
+                            if (lane == 0) red[hw] = dot;
+                        }
+                    }
+                    hbad = half_barrier_or(half, !ok);
+                    if (hbad) { *abort_flag = 1; break; }     // the other half's waits give up on this flag
+                    if (type == ST_FFN) {
+                        if (a0 >= 0 && hrep < rh) {
+                            const unsigned char* down = stage + 2 * plane_bytes;
+                            const __nv_bfloat16* ds = reinterpret_cast<const __nv_bfloat16*>(stage + 3 * plane_bytes) + static_cast<size_t>(2 * NB) * nbk;
+                            for (int j = hrep; j < NB; j += rh) {
+                                const float h = silu_mul(red[j], red[NB + j]);
+                                const float f = h * __bfloat162float(ds[static_cast<size_t>(j) * nbk + (i4_col >> 3)]);
+                                corr += f;
+                                const uint2 w2 = reinterpret_cast<const uint2*>(down + static_cast<size_t>(j) * crow_bytes)[i4_col];
+                                const uint32_t words[2] = {w2.x, w2.y};
+#pragma unroll
+                                for (int v = 0; v < 2; ++v) {
+                                    const uint32_t pk[4] = {nibble_pair_r(words[v], pb), nibble_pair_r(__umulhi(words[v], mul1), pb),
+                                                            nibble_pair_r(__umulhi(words[v], mul2), pb),
+                                                            nibble_pair_r(__umulhi(words[v], mul3), pb)};
+#pragma unroll
+                                    for (int k = 0; k < 4; ++k) {
+                                        acc16[(8 * v + k) % kI4Acc] = fmaf(f, __uint_as_float(pk[k] * mul16), acc16[(8 * v + k) % kI4Acc]);
+                                        acc16[(8 * v + k + 4) % kI4Acc] = fmaf(f, __uint_as_float(pk[k]), acc16[(8 * v + k + 4) % kI4Acc]);
+                                    }
+                                }
+                            }
+                        }
+                        hpar ^= 1;
+                    } else if (type == ST_PRED) {
+                        if (ht == 0) {
+                            const unsigned n_pred = static_cast<unsigned>(step_i) * (L - 1) + (l + 1);
+                            float* zdst = P.z + static_cast<size_t>(n_pred & 1u) * r;
+                            for (int i = 0; i < a1; ++i) {
+                                float z = red[i];
+                                if (P.act == HALO_ACT_RELU) z = fmaxf(z, 0.0f);
+                                zdst[a0 + i] = z;
+                            }
+                            __threadfence();
+                            atomicAdd(sync_zcount, static_cast<unsigned>(a1));
+                        }
+                        hpar ^= 1;
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.empty[s]);
+                    it_half += 2;
+                    if (type == ST_END) break;
+                }
+                // both halves are through their END marker (or gave up): one decision for the whole thread block
+                bad = pc_barrier_or(hbad);
+                any = pc_barrier_or(any);
+            } else
             while (true) {
                 const int s = TM ? it % kTSlots : it % STAGES;
                 const uint32_t parity = static_cast<uint32_t>(it / (TM ? kTSlots : STAGES)) & 1u;
@@ -698,49 +833,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 const uint32_t tslot = tbase + tlane + static_cast<uint32_t>(s * kTSlotCols);   // TM: this warp's lanes of the slot
                 float* red = sm.red[red_par];
                 // ---- before the barrier: nothing in here may block on other consumers ----
-                if constexpr (I4) {
-                    if (type == ST_FFN) {
-                        if (a0 >= 0) {
-                            any = true;
-                            // code rows 0..15 of the stage: 8 gate rows, then 8 up rows; this warp's row against xp
-                            const int chunks16 = d / 32, nbk = d / 128;
-                            const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(warp) * crow_bytes);
-                            const __nv_bfloat16* rs =
-                                reinterpret_cast<const __nv_bfloat16*>(stage + 3 * plane_bytes) + static_cast<size_t>(warp) * nbk;
-                            float a = 0.0f;
-#pragma unroll
-                            for (int u = 0; u < XC; ++u) {
-                                const int c = lane + 32 * u;
-                                const uint4 w4 = rp[c];
-                                const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
-                                float t0 = 0.0f, t1 = 0.0f;
-#pragma unroll
-                                for (int w = 0; w < 4; ++w) {
-                                    const uint4 xv = xp[static_cast<size_t>(w) * chunks16 + c];
-                                    fma_bf16x2(nibble_pair_r(ww[w], pb), xv.x, t0, t1);
-                                    fma_bf16x2(nibble_pair_r(ww[w] >> 4, pb), xv.y, t0, t1);
-                                    fma_bf16x2(nibble_pair_r(ww[w] >> 8, pb), xv.z, t0, t1);
-                                    fma_bf16x2(nibble_pair_r(__umulhi(ww[w], mul3), pb), xv.w, t0, t1);
-                                }
-                                a = fmaf(__bfloat162float(rs[c >> 2]), (t0 + t1) - kNibbleBias * xsum[c], a);
-                            }
-                            a = warp_sum(a);
-                            if (lane == 0) red[warp] = a;
-                        }
-                    } else if (type == ST_PRED) {
-                        // bf16 predictor rows: two warps per row, x (bf16) from shared memory
-                        const int prow = warp >> 1, ppart = warp & 1;
-                        if (prow < a1) {
-                            const uint4* rp = reinterpret_cast<const uint4*>(stage + static_cast<size_t>(prow) * row_bytes);
-                            const uint4* xv = reinterpret_cast<const uint4*>(xs);
-                            float dot0 = 0.0f, dot1 = 0.0f;
-                            const int half = chunks >> 1;
-                            for (int c = ppart * half + lane; c < (ppart + 1) * half; c += 32) dot_bf16x8(rp[c], xv[c], dot0, dot1);
-                            const float dot = warp_sum(dot0 + dot1);
-                            if (lane == 0) red[prow * 2 + ppart] = dot;
-                        }
-                    }
-                } else if constexpr (TM) {
+                if constexpr (TM) {
                     if ((type == ST_FFN && a0 >= 0) || type == ST_PRED) {
                         if (type == ST_FFN) any = true;
                         const int n_rows = type == ST_FFN ? ROWS : a1;
@@ -794,34 +887,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 bad = pc_barrier_or(!ok);
                 if (bad) break;
                 // ---- after the barrier ----
-                if (I4 && type == ST_FFN) {
-                    if constexpr (I4) {
-                        if (a0 >= 0 && i4_rep < i4_reps) {
-                            const int nbk = d / 128;
-                            const unsigned char* down = stage + 2 * plane_bytes;
-                            const __nv_bfloat16* ds = reinterpret_cast<const __nv_bfloat16*>(stage + 3 * plane_bytes) + static_cast<size_t>(2 * NB) * nbk;
-                            for (int j = i4_rep; j < NB; j += i4_reps) {
-                                const float h = silu_mul(red[j], red[NB + j]);
-                                const float f = h * __bfloat162float(ds[static_cast<size_t>(j) * nbk + (i4_col >> 3)]);
-                                corr += f;
-                                const uint2 w2 = reinterpret_cast<const uint2*>(down + static_cast<size_t>(j) * crow_bytes)[i4_col];
-                                const uint32_t words[2] = {w2.x, w2.y};
-#pragma unroll
-                                for (int v = 0; v < 2; ++v) {
-                                    const uint32_t pk[4] = {nibble_pair_r(words[v], pb), nibble_pair_r(__umulhi(words[v], mul1), pb),
-                                                            nibble_pair_r(__umulhi(words[v], mul2), pb),
-                                                            nibble_pair_r(__umulhi(words[v], mul3), pb)};
-#pragma unroll
-                                    for (int k = 0; k < 4; ++k) {
-                                        acc16[(8 * v + k) % kI4Acc] = fmaf(f, __uint_as_float(pk[k] * mul16), acc16[(8 * v + k) % kI4Acc]);
-                                        acc16[(8 * v + k + 4) % kI4Acc] = fmaf(f, __uint_as_float(pk[k]), acc16[(8 * v + k + 4) % kI4Acc]);
-                                    }
-                                }
-                            }
-                        }
-                    }
-                    red_par ^= 1;
-                } else if (type == ST_FFN) {
+                if (type == ST_FFN) {
                     if (a0 >= 0) {
                         const unsigned char* down = stage + 2 * plane_bytes;
 #pragma unroll
@@ -852,7 +918,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                         float* zdst = P.z + static_cast<size_t>(n_pred & 1u) * r;
                         for (int i = 0; i < a1; ++i) {
                             float z = 0.0f;
-                            for (int w = 0; w < (I4 ? 2 : WPR); ++w) z += red[i * (I4 ? 2 : WPR) + w];
+                            for (int w = 0; w < WPR; ++w) z += red[i * WPR + w];
                             if (P.act == HALO_ACT_RELU) z = fmaxf(z, 0.0f);
                             zdst[a0 + i] = z;
                         }

@@ -32,10 +32,10 @@ NOMINAL_HBM_GBS = 8000.0
 # 4-block 7B-shaped case (profiles/stack_decode_kernel_llama2-7b_4blocks.md); traffic is proportional to the kept
 # groups processed, so the ratio carries over to the full-size launch.  The figure belongs to the kernel sources with
 # the hash below: when they change the line reports no traffic until the counters have been taken again.
-STACK_KERNEL_TRAFFIC_RATIO = 1.0005
+STACK_KERNEL_TRAFFIC_RATIO = 1.0007
 STACK_KERNEL_SOURCES = ("stack_persistent.cu", "stack_persistent.cuh", "ffn_math.cuh", "i4_math.cuh", "tma.cuh", "umma.cuh",
                         "select_device.cuh")
-STACK_KERNEL_SOURCES_SHA1 = "13df837cf1ac5e76773b5ef1c6216963b6aa9f89"
+STACK_KERNEL_SOURCES_SHA1 = "ed86f5839d047624aa461b171c8af53181582bc1"
 FALLBACK_HBM_GBS = 6650.0
 
 

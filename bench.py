@@ -547,6 +547,7 @@ def int4_stack_report(dev, peak, steps=32, warm=4):
            "weights_gb": L * G * group_bytes_i4 / 1e9, "gpu_launches_per_token": stack.last_launches() / steps,
            "device_status": stack.status()}
     stack.close()
+    res["prefill"] = _int4_prompt_timing(wl, fsh, plan, Q, Sc, preds, dev)
     return res
 
 
@@ -648,6 +649,39 @@ def decode_brief(name, dev, peak, steps=64, warm=4):
            "device_status": stack.status()}
     stack.close()
     return res
+
+
+def _int4_prompt_timing(wl, fsh, plan, Q, Sc, preds, dev, n_tok=512, prompts=8, warm=3):
+    """512-token prompts through the int4 stack: per block the kept groups are turned back into bf16 in a scratch
+    block (on the side stream, under the previous block's FFN) and the tensor-core FFN reads those.  FLOPs as for the
+    bf16 prompt."""
+    from paper_2601_11676_b200 import binding as B
+    L, G, d = wl.n_layers, wl.n_groups, wl.d_model
+    stack = B.Stack(fsh, B.pred_shape(d, wl.pred_rank, G, B.BF16), n_tok, plan, Q, [p[0] for p in preds],
+                    [p[1] for p in preds], i4_scales=Sc)
+    pw = synth.workload(wl.name, n_tok=n_tok)
+    total = warm + prompts
+    h0 = torch.stack([synth.stream_input(pw, 1000 + s, dev) for s in range(total)])
+    h_out = torch.empty_like(h0)
+    nk_rec = torch.zeros((total, L), dtype=torch.int32, device=dev)
+    stack.decode(h0, total, 0, h_out, B.Taps(None, None, None, None, None, nk_rec.data_ptr(), None))
+    torch.cuda.synchronize()
+    reps = []
+    for _ in range(3):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        stack.decode(h0[warm:], prompts, warm, h_out[warm:])
+        b.record()
+        torch.cuda.synchronize()
+        reps.append(a.elapsed_time(b))
+    ms = sorted(reps)[1]
+    kept = int(nk_rec[warm:].sum().item())
+    flops = 6.0 * n_tok * kept * wl.group_size * d + prompts * (L - 1) * 2.0 * n_tok * (d * wl.pred_rank + wl.pred_rank * G)
+    out = {"prompt_tokens": n_tok, "prompts_timed": prompts, "ms_per_prompt": ms / prompts,
+           "ms_per_prompt_runs": [r / prompts for r in reps], "tflops": flops / (ms * 1e-3) / 1e12,
+           "gpu_launches": int(stack.last_launches()), "device_status": stack.status()}
+    stack.close()
+    return out
 
 
 def prefill_report(wl, Wp, preds, plan, ffn, dev, n_tok=512, prompts=16, warm=3):

@@ -338,9 +338,18 @@ halo_status halo_group_mha(const halo_mha_shape* shape, const void* W_packed, co
  *   halo_group_ffn_i4: halo_group_ffn on the dequantised weights; x device bf16 [n_tok][d]; partials device
  *     fp32 [n_dev+1][n_tok][d], zeroed by the call; keep_list / n_keep / dev_of_group / dev_status as there.
  *     Decode form (one pass over the kept groups' weights per token); no workspace.
+ *   halo_dequantize_weights_i4: Q, scales -> W_packed (device bf16, layout of halo_pack_weights, 16-byte aligned,
+ *     caller-owned), every element bf16((nibble - 8) * s): one rounding of the exact value.  keep_list / n_keep
+ *     (device, as for halo_group_ffn) name the groups to write, the others are left as they are; keep_list NULL
+ *     writes all groups.  For prompts: the tensor cores take bf16 operands, so a prompt on int4 weights is this
+ *     call followed by halo_group_ffn on its output (what an int4 stack created for more than one token does per
+ *     block).  shape->wdtype is ignored.  An out-of-range index sets HALO_DEV_BAD_INDEX and that entry is skipped.
  * ---------------------------------------------------------------------- */
 halo_status halo_quantize_weights_i4(const halo_ffn_shape* shape, const void* W_packed, void* Q, void* scales,
                                      void* stream);
+halo_status halo_dequantize_weights_i4(const halo_ffn_shape* shape, const void* Q, const void* scales,
+                                       const int32_t* keep_list, const int32_t* n_keep, void* W_packed,
+                                       uint32_t* dev_status, void* stream);
 halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void* Q, const void* scales, const void* x, int n_tok,
                               const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
                               int n_dev, float* partials, uint32_t* dev_status, void* stream);

@@ -448,6 +448,10 @@ struct halo_stack {
     halo_plan plan;
     std::vector<const void*> W, W1, W2;
     std::vector<const void*> i4_scales;   // non-empty: W holds int4 codes (halo_quantize_weights_i4)
+    // int4 stacks made for prompts: the kept groups of a block are turned back into bf16 (the tensor cores' operand
+    // type) in one of two scratch blocks, alternating by block, and the tensor-core FFN reads those
+    void* i4_deq[2] = {nullptr, nullptr};
+    bool i4_prompt = false;
     void* slab;
     // carved from the slab
     float* h;
@@ -589,7 +593,7 @@ halo_status stack_create_impl(halo_stack** out, const halo_ffn_shape* ffn, const
     constexpr size_t kMaxGrid = 192;   // thread blocks of the persistent kernel (one per SM)
     const size_t o_xh = carve(2 * d * 2);
     const size_t o_dr = carve(!i4_scales && persistent_supported(*ffn, n_tok, G) ? sizeof(float) * 2 * kMaxGrid * d : 16);
-    const size_t ws_bytes = (!i4_scales && prefill_supported(*ffn, n_tok)) ? prefill_workspace_bytes(*ffn, n_tok) : 0;
+    const size_t ws_bytes = prefill_supported(*ffn, n_tok) ? prefill_workspace_bytes(*ffn, n_tok) : 0;
     const size_t o_ws = carve(ws_bytes ? ws_bytes : 16);
     const size_t o_sc2 = carve(sizeof(float) * G), o_dg2 = carve(sizeof(int32_t) * G);
     const size_t o_ar2 = carve(HALO_MAX_DEVICES), o_kl2 = carve(sizeof(int32_t) * G), o_nk2 = carve(sizeof(int32_t));
@@ -655,6 +659,17 @@ halo_status stack_create_impl(halo_stack** out, const halo_ffn_shape* ffn, const
     s->max_steps_per_launch = std::max(0, option_value(OPT_MAX_STEPS_PER_LAUNCH));
     if (option_value(OPT_L2_AHEAD) >= 0) s->l2_ahead = option_value(OPT_L2_AHEAD);
     s->persistent_ok = i4_scales ? persistent_supported_i4(*ffn, n_tok, G) : persistent_supported(*ffn, n_tok, G);
+    if (i4_scales && ws_bytes) {
+        // best effort: without the scratch blocks a prompt runs through the decode form, token by token
+        const size_t block_bytes = static_cast<size_t>(ffn->d_ffn) * 3 * d * 2;
+        if (cudaMalloc(&s->i4_deq[0], block_bytes) == cudaSuccess && cudaMalloc(&s->i4_deq[1], block_bytes) == cudaSuccess) {
+            s->i4_prompt = true;
+        } else {
+            (void)cudaGetLastError();
+            if (s->i4_deq[0]) cudaFree(s->i4_deq[0]);
+            s->i4_deq[0] = s->i4_deq[1] = nullptr;
+        }
+    }
     {
         // pointer tables, and the first block's selection: reliable block, all scores equal -> the priority
         // order is the group order, everything is kept (Sec. III-B.3, first layer)
@@ -749,6 +764,8 @@ extern "C" halo_status halo_stack_destroy(halo_stack* s) {
     }
     cudaFree(s->slab);
     if (s->pp_slab) cudaFree(s->pp_slab);
+    if (s->i4_deq[0]) cudaFree(s->i4_deq[0]);
+    if (s->i4_deq[1]) cudaFree(s->i4_deq[1]);
     delete s;
     return HALO_OK;
 }
@@ -951,6 +968,11 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
             HALO_TRY(launch_select(s->plan.dev, G, s->zero_scores, step, 0u, 1, nullptr, s->set_dev[0], s->set_arr[0],
                                    nullptr, s->set_kl[0], s->set_nk[0], s->status, st));
             launches += 2;
+            if (s->i4_prompt) {
+                HALO_TRY(launch_dequantize_i4(s->ffn, s->W[0], s->i4_scales[0], s->set_kl[0], s->set_nk[0], s->i4_deq[0],
+                                              s->status, st));
+                ++launches;
+            }
             HALO_CU(cudaEventRecord(s->ev_x, st));   // x_0 is ready (and set[1] is no longer in use)
             for (int l = 0; l < L; ++l) {
                 const int cur = l & 1, nxt = (l + 1) & 1;
@@ -973,6 +995,12 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                                                s->set_nk[nxt], s->status, side));
                         launches += 4;
                     }
+                    if (s->i4_prompt) {
+                        // the scratch block of parity nxt was last read by block l-1, which ev_x is behind
+                        HALO_TRY(launch_dequantize_i4(s->ffn, s->W[l + 1], s->i4_scales[l + 1], s->set_kl[nxt], s->set_nk[nxt],
+                                                      s->i4_deq[nxt], s->status, side));
+                        ++launches;
+                    }
                     HALO_CU(cudaEventRecord(s->ev_sel, side));
                 }
                 float* y_tap = nullptr;
@@ -987,7 +1015,8 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                     if (taps->y) y_tap = taps->y + rec * step_elems;
                 }
                 float* h_dst = (l == L - 1) ? h_out + sidx * step_elems : s->h;
-                if (!s->i4_scales.empty()) {
+                const void* W_l = s->i4_prompt ? s->i4_deq[cur] : s->W[l];
+                if (!s->i4_scales.empty() && !s->i4_prompt) {
                     HALO_TRY(halo_group_ffn_i4(&s->ffn, s->W[l], s->i4_scales[l], x_cur, static_cast<int>(T), s->set_kl[cur],
                                                s->set_nk[cur], s->set_dev[cur], n_dev, s->partials, s->status, stream));
                     HALO_TRY(launch_merge_glue(s->partials, s->set_arr[cur], n_dev, static_cast<int>(T), static_cast<int>(d),
@@ -996,7 +1025,7 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                 } else if (!y_tap && s->ffn_ws && prefill_accumulates(s->ffn, static_cast<int>(T))) {
                     // only kept (= arrived) groups are computed and nobody asked for y itself: the down projection
                     // adds its tiles straight into the residual stream, and the glue only normalises
-                    HALO_TRY(launch_group_ffn_prefill(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->set_kl[cur],
+                    HALO_TRY(launch_group_ffn_prefill(s->ffn, W_l, x_cur, static_cast<int>(T), s->set_kl[cur],
                                                       s->set_nk[cur], s->set_dev[cur], n_dev, 1, s->h, s->ffn_ws,
                                                       s->status, st, s->ffn_ws_clean));
                     s->ffn_ws_clean = true;   // every launch on this workspace leaves the control words zeroed
@@ -1005,7 +1034,7 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                     launches += 3;
                 } else {
                     bool collapsed = false;   // the sum over holders is all the glue needs
-                    HALO_TRY(dispatch_group_ffn(s->ffn, s->W[l], x_cur, static_cast<int>(T), s->set_kl[cur],
+                    HALO_TRY(dispatch_group_ffn(s->ffn, W_l, x_cur, static_cast<int>(T), s->set_kl[cur],
                                                 s->set_nk[cur], s->set_dev[cur], n_dev, s->partials, s->ffn_ws,
                                                 s->status, st, &collapsed));
                     HALO_TRY(launch_merge_glue(s->partials, collapsed ? nullptr : s->set_arr[cur],
@@ -1064,7 +1093,13 @@ extern "C" halo_status halo_stack_decode(halo_stack* s, const float* h0, int ste
                 if (taps->n_keep) HALO_COPY(taps->n_keep + rec, s->n_keep, sizeof(int32_t));
                 if (taps->y) y_tap = taps->y + rec * step_elems;
             }
-            if (!s->i4_scales.empty()) {
+            if (s->i4_prompt) {
+                HALO_TRY(launch_dequantize_i4(s->ffn, s->W[l], s->i4_scales[l], s->keep_list, s->n_keep, s->i4_deq[0],
+                                              s->status, st));
+                ++launches;
+                HALO_TRY(dispatch_group_ffn(s->ffn, s->i4_deq[0], x_cur, static_cast<int>(T), s->keep_list, s->n_keep,
+                                            s->dev_of_group, n_dev, s->partials, s->ffn_ws, s->status, st));
+            } else if (!s->i4_scales.empty()) {
                 HALO_TRY(halo_group_ffn_i4(&s->ffn, s->W[l], s->i4_scales[l], x_cur, static_cast<int>(T), s->keep_list,
                                            s->n_keep, s->dev_of_group, n_dev, s->partials, s->status, stream));
                 ++launches;

@@ -70,6 +70,73 @@ quantize_i4_kernel(int d, long long n_rows, const T* __restrict__ W, uint8_t* __
     reinterpret_cast<uint16_t*>(Q)[base / 4] = static_cast<uint16_t>(packed);   // 4 elements = 2 bytes
 }
 
+// Kept groups (or all of them) back to bf16 in the packed layout, for the tensor-core prompt path: a thread turns one
+// word of codes into 8 values = one 16-byte store, neighbouring lanes neighbouring words, so every store instruction
+// of a warp covers 512 contiguous bytes.  value = bf16((nibble - 8) * s) (the product has at most 12 significant bits,
+// so this is ONE rounding of the exact value).  No integer-to-float conversion: nibbles k and k+4 of the word become
+// the bf16 pair {128 + n_k, 128 + n_k+4} by mask and OR, 136 is subtracted (exact) and the pair is multiplied by the
+// scale in bf16x2 (one rounding); a byte permute puts neighbouring elements back side by side.  Groups outside the
+// kept set are not touched.
+__device__ __forceinline__ uint4 dequant_word(uint32_t word, __nv_bfloat16 scale) {
+    const __nv_bfloat162 s2 = __halves2bfloat162(scale, scale);
+    const uint32_t bias_bits = 0x43084308u;                       // {136, 136}
+    const __nv_bfloat162 bias = *reinterpret_cast<const __nv_bfloat162*>(&bias_bits);
+    uint32_t r[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t pr = nibble_pair_bf16(word, k);            // {128 + e_k, 128 + e_k+4}
+        const __nv_bfloat162 v = __hmul2(__hsub2(*reinterpret_cast<const __nv_bfloat162*>(&pr), bias), s2);
+        r[k] = *reinterpret_cast<const uint32_t*>(&v);
+    }
+    return make_uint4(__byte_perm(r[0], r[1], 0x5410), __byte_perm(r[2], r[3], 0x5410),
+                      __byte_perm(r[0], r[1], 0x7632), __byte_perm(r[2], r[3], 0x7632));
+}
+
+__global__ void __launch_bounds__(256)
+dequantize_i4_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, const __nv_bfloat16* __restrict__ scales,
+                     const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
+                     __nv_bfloat16* __restrict__ W, uint32_t* dev_status) {
+    int nk = G;
+    if (keep_list) {
+        nk = *n_keep_ptr;
+        if (nk < 0 || nk > G) {
+            if (threadIdx.x == 0 && blockIdx.x == 0) flag_status(dev_status, HALO_DEV_BAD_INDEX);
+            nk = nk < 0 ? 0 : G;
+        }
+    }
+    // a group's rows are contiguous in all three arrays: word j of the group's codes holds elements 8j..8j+7 of the
+    // group and uses scale j / 16
+    const long long per_group = 3ll * S * (d / 8);               // code words per group
+    const long long total = static_cast<long long>(nk) * per_group;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    constexpr int kU = 4;                                        // loads in flight per thread
+    for (long long i0 = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i0 < total; i0 += kU * stride) {
+        uint32_t word[kU];
+        __nv_bfloat16 sc[kU];
+        uint4* dst[kU];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            dst[u] = nullptr;
+            const long long i = i0 + u * stride;
+            if (i >= total) continue;
+            const int kp = static_cast<int>(i / per_group);
+            const long long j = i - kp * per_group;
+            const int g = keep_list ? keep_list[kp] : kp;
+            if (g < 0 || g >= G) {
+                flag_status(dev_status, HALO_DEV_BAD_INDEX);
+                continue;
+            }
+            const size_t gbase = static_cast<size_t>(g) * per_group;
+            word[u] = __ldg(reinterpret_cast<const uint32_t*>(Q) + gbase + j);
+            sc[u] = scales[(gbase + j) / 16];
+            dst[u] = reinterpret_cast<uint4*>(W) + gbase + j;
+        }
+#pragma unroll
+        for (int u = 0; u < kU; ++u)
+            if (dst[u]) *dst[u] = dequant_word(word[u], sc[u]);
+    }
+}
+
 template <int ITERS>
 __global__ void __launch_bounds__(kI4Threads, kI4BlocksPerSm)
 group_ffn_i4_kernel(int d, int S, int G, const uint8_t* __restrict__ Q, const __nv_bfloat16* __restrict__ scales,
@@ -858,6 +925,19 @@ halo_status check_i4_shape(const halo_ffn_shape* s) {
 }
 }  // namespace
 
+halo_status launch_dequantize_i4(const halo_ffn_shape& sh, const void* Q, const void* scales, const int32_t* keep_list,
+                                 const int32_t* n_keep, void* W_out, uint32_t* dev_status, cudaStream_t st) {
+    const int d = sh.d_model, S = sh.group_size, G = sh.d_ffn / S;
+    int dev = 0, sms = kSmCount;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long long threads = static_cast<long long>(G) * 3 * S * (d / 32);
+    const unsigned blocks = static_cast<unsigned>(std::min<long long>((threads + 255) / 256, static_cast<long long>(sms) * 16));
+    dequantize_i4_kernel<<<blocks, 256, 0, st>>>(d, S, G, static_cast<const uint8_t*>(Q),
+                                                  static_cast<const __nv_bfloat16*>(scales), keep_list, n_keep,
+                                                  static_cast<__nv_bfloat16*>(W_out), dev_status);
+    return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+}
+
 }  // namespace halo
 
 using namespace halo;
@@ -882,6 +962,16 @@ extern "C" halo_status halo_quantize_weights_i4(const halo_ffn_shape* shape, con
         quantize_i4_kernel<float><<<blocks, 256, 0, st>>>(d, n_rows, static_cast<const float*>(W_packed),
                                                           static_cast<uint8_t*>(Q), static_cast<__nv_bfloat16*>(scales));
     return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+}
+
+extern "C" halo_status halo_dequantize_weights_i4(const halo_ffn_shape* shape, const void* Q, const void* scales,
+                                                  const int32_t* keep_list, const int32_t* n_keep, void* W_packed,
+                                                  uint32_t* dev_status, void* stream) {
+    halo_status rc = check_i4_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (!Q || !scales || !W_packed || (keep_list && !n_keep)) return HALO_ERR_ARG;
+    if (!aligned16(Q) || !aligned16(scales) || !aligned16(W_packed)) return HALO_ERR_ALIGN;
+    return launch_dequantize_i4(*shape, Q, scales, keep_list, n_keep, W_packed, dev_status, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void* Q, const void* scales, const void* x,

@@ -8,6 +8,7 @@ from oracle import halo_ref as R
 from paper_2601_11676_b200 import binding as B
 from paper_2601_11676_b200 import synth
 from tests import gpu_util as U
+from tests import test_gpu_stack as TS
 
 pytestmark = pytest.mark.gpu
 DEV = U.DEV
@@ -184,3 +185,81 @@ def test_int4_stack_teacher_forced(name, layers, steps, mode):
             y_ref = R.merge(P)
             assert U.rel_err(t["y"][s, l].cpu().numpy(), y_ref) <= U.TOL_BF16, (s, l)
     assert lost > 0
+
+
+@pytest.mark.parametrize("d,G,S", [(256, 5, 16), (4096, 6, 128), (1024, 7, 256)])
+def test_int4_dequantise_is_one_rounding_of_the_exact_value(d, G, S):
+    """halo_dequantize_weights_i4: every element equals the exact (nibble - 8) * s of the oracle, rounded once to bf16
+    (ties to even: the library cast); with a kept list only the named groups are written, a bad index is reported."""
+    wl = synth.Workload("q", 1, d, G * S, S, 16, "bf16", (), (), 500, 1)
+    Wp = synth.packed_layer(wl, 1, DEV)
+    sh, Q, Sc = _quantize(wl, Wp)
+    exact = R.dequantize_i4(Q.cpu().numpy(), synth.host_bits(Sc))                 # fp32, exact
+    want = synth.host_bits(torch.from_numpy(exact).to(torch.bfloat16))
+    out = torch.full((G, 3, S, d), 7.0, dtype=torch.bfloat16, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.halo_dequantize_weights_i4(sh, Q, Sc, None, None, out, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and (synth.host_bits(out) == want).all()
+    keep = [G - 1, 0, 9, 2]                                                       # 9 is out of range
+    kl = torch.full((G,), -1, dtype=torch.int32, device=DEV)
+    kl[: len(keep)] = torch.tensor(keep, dtype=torch.int32)
+    nk = torch.tensor([len(keep)], dtype=torch.int32, device=DEV)
+    out.fill_(7.0)
+    B.halo_dequantize_weights_i4(sh, Q, Sc, kl, nk, out, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) & B.DEV_BAD_INDEX
+    got = synth.host_bits(out)
+    seven = synth.host_bits(torch.tensor([7.0], dtype=torch.bfloat16))[0]
+    for g in range(G):
+        assert (got[g] == (want[g] if g in keep else seven)).all(), g
+
+
+def _int4_prompt_stack(wl):
+    L, G, d = wl.n_layers, wl.n_groups, wl.d_model
+    quant, host = [], []
+    for l in range(L):
+        Wp = synth.packed_layer(wl, l, DEV)
+        _, Q, Sc = _quantize(wl, Wp)
+        quant.append((Q, Sc))
+        host.append((Q.cpu().numpy(), synth.host_bits(Sc)))
+        del Wp
+    preds = [synth.predictor(wl, l, DEV) for l in range(L)]
+    plan = B.Plan(G, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
+    stack = B.Stack(B.ffn_shape(d, wl.d_ffn, wl.group_size, B.BF16), B.pred_shape(d, wl.pred_rank, G, B.BF16), wl.n_tok,
+                    plan, [q[0] for q in quant], [p[0] for p in preds], [p[1] for p in preds],
+                    i4_scales=[q[1] for q in quant])
+
+    def ffn_ref(l, x, keep, dev):
+        return R.group_ffn_i4(host[l][0], host[l][1], x, keep, dev, wl.n_dev)
+    return stack, preds, ffn_ref
+
+
+@pytest.mark.parametrize("n_tok,d", [(5, 512), (64, 512), (300, 256)])
+def test_int4_stack_prompts(n_tok, d):
+    """An int4 stack made for prompts: five tokens go through the decode form token by token, 64 and 300 through the
+    tensor-core path on the kept groups turned back into bf16.  Teacher-forced against the oracle's FFN on the EXACT
+    dequantised weights through the records; then the run without the y records (down projection adding into the
+    residual stream) chained from the recorded inputs."""
+    wl = synth.Workload("pq", 3, d, 64 * 12, 64, 64, "bf16", (0.0, 0.3, 0.6), (2, 1, 1), 250, 2, n_tok=n_tok)
+    stack, preds, ffn_ref = _int4_prompt_stack(wl)
+    h0, h_out, t = TS.run_with_taps(wl, stack, wl.steps)
+    lost = TS.check_teacher_forced(wl, None, preds, h0, h_out, t, wl.steps, ffn_ref=ffn_ref)
+    assert lost > 0
+    plain, t2 = TS.run_without_y(wl, stack, h0, wl.steps)
+    assert TS.check_chained_without_y(wl, None, preds, h0, plain, t2, wl.steps, 0, list(range(n_tok)), ffn_ref=ffn_ref) == lost
+    upd = float((h_out - h0).double().pow(2).mean().sqrt().item())
+    assert (plain - h_out).abs().max().item() <= U.TOL_BF16 * upd
+
+
+def test_int4_prompt_stack_at_the_benchmarked_shape():
+    """512 tokens, d 4096, groups of 128, lossy devices, int4 weights: teacher-forced on sampled token rows, then the
+    timed form (no y records) chained from the recorded inputs."""
+    wl = synth.workload("llama2-7b-prefill", n_layers=3, steps=1, loss_rate=(0.0, 0.3, 0.5, 0.7))
+    stack, preds, ffn_ref = _int4_prompt_stack(wl)
+    h0, h_out, t = TS.run_with_taps(wl, stack, wl.steps, step0=5)
+    tokens = [0, 127, 128, 300, 511]
+    lost = TS.check_teacher_forced(wl, None, preds, h0, h_out, t, wl.steps, step0=5, tokens=tokens, ffn_ref=ffn_ref)
+    assert lost > 0
+    plain, t2 = TS.run_without_y(wl, stack, h0, wl.steps, step0=5)
+    assert TS.check_chained_without_y(wl, None, preds, h0, plain, t2, wl.steps, 5, tokens, ffn_ref=ffn_ref) == lost

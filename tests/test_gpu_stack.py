@@ -59,9 +59,10 @@ def run_without_y(wl, stack, h0, steps, step0=0):
 
 
 def check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=0, mode=R.SEL_TOPK, threshold=0.0,
-                         act=R.ACT_RELU, tokens=None):
+                         act=R.ACT_RELU, tokens=None, ffn_ref=None):
     """`tokens`: token rows whose FFN output the oracle recomputes (all when None); scores, selection integers and
-    the glue chain are always checked in full."""
+    the glue chain are always checked in full.  `ffn_ref(l, x, keep_list, dev_of_group)`: the oracle's holder slots
+    of block l when the weights are not a packed bf16/fp32 tensor (int4 stacks)."""
     hb = synth.host_bits
     tol = U.tol_for(wl)
     L, n = wl.n_layers, wl.n_dev
@@ -91,7 +92,10 @@ def check_teacher_forced(wl, Wp, preds, h0, h_out, t, steps, step0=0, mode=R.SEL
             lost_layers += int(nk < wl.n_groups)
             y = t["y"][s, l].cpu().numpy()
             x_ffn = x_l if tokens is None else x_l[tokens]
-            P = R.group_ffn(hb(Wp[l]), x_ffn, sel["keep_list"][:nk], sel["dev_of_group"], n)
+            if ffn_ref is not None:
+                P = ffn_ref(l, x_ffn, sel["keep_list"][:nk], sel["dev_of_group"])
+            else:
+                P = R.group_ffn(hb(Wp[l]), x_ffn, sel["keep_list"][:nk], sel["dev_of_group"], n)
             y_ref = R.merge(P)
             assert U.rel_err(y if tokens is None else y[tokens], y_ref) <= tol, (s, l)
             # glue, from the GPU's own y: next input and residual stream
@@ -185,7 +189,7 @@ def test_stack_prompt_on_the_tensor_core_path(n_tok, d):
         assert (plain - h_out).abs().max().item() <= U.TOL_BF16 * upd
 
 
-def check_chained_without_y(wl, Wp, preds, h0, h_out, t, steps, step0, tokens, act=R.ACT_RELU):
+def check_chained_without_y(wl, Wp, preds, h0, h_out, t, steps, step0, tokens, act=R.ACT_RELU, ffn_ref=None):
     """Check of a run that recorded every block's input x, scores and selection but NOT its output y (the form in
     which the prompt path adds the down projection straight into the residual stream).  Scores and selection
     integers are checked as usual.  For the sampled token rows the oracle computes y_l from the recorded x_l and
@@ -218,7 +222,10 @@ def check_chained_without_y(wl, Wp, preds, h0, h_out, t, steps, step0, tokens, a
             if n:
                 assert (t["arrived"][s, l, :n].cpu().numpy() == sel["arrived"]).all()
             lost += int(nk < wl.n_groups)
-            y_ref = R.merge(R.group_ffn(hb(Wp[l]), x_all[s, l][tokens], sel["keep_list"][:nk], sel["dev_of_group"], n))
+            if ffn_ref is not None:
+                y_ref = R.merge(ffn_ref(l, x_all[s, l][tokens], sel["keep_list"][:nk], sel["dev_of_group"]))
+            else:
+                y_ref = R.merge(R.group_ffn(hb(Wp[l]), x_all[s, l][tokens], sel["keep_list"][:nk], sel["dev_of_group"], n))
             bound += tol * float(np.sqrt(np.mean(y_ref ** 2)))
             h, x_next = R.glue(h, y_ref, code)
             if l + 1 < L:

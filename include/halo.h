@@ -418,7 +418,11 @@ halo_status halo_stack_create(halo_stack** out, const halo_ffn_shape* ffn, const
                               const void* const* W1, const void* const* W2);
 /* The same stack on int4 group-quantised FFN weights (Sec. IV-A: the evaluated models are 4-bit): Q[L] and scales[L]
  * as written by halo_quantize_weights_i4 for every block; activations, predictor and everything else as above
- * (ffn->wdtype must be HALO_BF16, d_model % 128 == 0).  Runs one launch per step of the path. */
+ * (ffn->wdtype must be HALO_BF16, d_model % 128 == 0).  One token: the persistent decode kernel for d_model 2048 and
+ * 4096, else one launch per step of the path.  Prompts of 16 tokens or more on shapes the tensor-core FFN takes: the
+ * stack also owns two bf16 scratch blocks (2 x 3 * d_ffn * d_model * 2 bytes), the kept groups of every block are
+ * written there by halo_dequantize_weights_i4's kernel and the tensor-core FFN reads them; other token counts go
+ * through halo_group_ffn_i4 token by token. */
 halo_status halo_stack_create_i4(halo_stack** out, const halo_ffn_shape* ffn, const halo_pred_shape* pred,
                                  int n_layers, int n_tok, const halo_plan* plan, const void* const* Q,
                                  const void* const* scales, const void* const* W1, const void* const* W2);

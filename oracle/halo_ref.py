@@ -399,6 +399,14 @@ def group_lm_head(W: np.ndarray, x: np.ndarray, group_size: int, group_list=None
     return out
 
 
+def group_lm_head_i4(Q: np.ndarray, Sc: np.ndarray, x: np.ndarray, group_size: int, group_list=None,
+                     fill: float = np.nan):
+    """The LM-head groups on int4 rows = the LM-head groups on their dequantised values (x widened exactly to fp32)."""
+    W32 = dequantize_i4(Q, Sc)
+    x32 = to_f64(x).astype(np.float32)          # bf16 -> fp32 is exact
+    return group_lm_head(W32, x32, group_size, group_list, fill)
+
+
 # --- a transformer-block stack: MHA groups, then FFN groups, per layer; LM-head groups at the end --------------
 
 def block_stack_token(h0, pos, step, blocks, lm_W, lm_group_size, plan_mha, plan_ffn, dtype, act=ACT_RELU):

@@ -79,3 +79,27 @@ def test_ffn_on_int4_weights_is_the_ffn_on_the_dequantised_values():
     assert (P4[1] == 0).all() and (P16[1] == 0).all()
     rel = np.abs(P4 - P16).max() / np.abs(P16).max()
     assert 1e-4 < rel < 0.25
+
+
+def test_lm_head_on_int4_rows_is_a_plain_matrix_product_of_the_code_grid():
+    """Rows built ON the int4 grid (integer codes times a power-of-two scale) with integer activations: the logits
+    are integers that a numpy int64 product gives exactly; unlisted groups keep the fill value; a short last group."""
+    rng = np.random.default_rng(5)
+    vocab, d, S = 37, 256, 8
+    codes = rng.integers(-7, 8, size=(vocab, d))
+    codes[:, 0] = 7                                              # amax = 7 * scale in every block ...
+    codes[:, 128] = -7                                           # ... so the scale comes back exactly
+    scale = np.where(np.arange(vocab)[:, None] % 2 == 0, 0.5, 2.0)
+    W = torch.tensor(codes * scale, dtype=torch.float32).numpy()
+    Q, Sc = R.quantize_i4(W)
+    assert (R.dequantize_i4(Q, Sc) == W).all()
+    x_int = rng.integers(-3, 4, size=(2, d))
+    x = torch.tensor(x_int, dtype=torch.float32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    want = (x_int.astype(np.int64) @ (codes * 2).astype(np.int64).T) * np.where(np.arange(vocab) % 2 == 0, 0.25, 1.0)
+    full = R.group_lm_head_i4(Q, Sc, x, S)
+    assert full.shape == (2, vocab) and (full == want).all()
+    part = R.group_lm_head_i4(Q, Sc, x, S, group_list=[4, 0], fill=-1.0)      # group 4 = rows 32..36 (short)
+    listed = np.zeros(vocab, dtype=bool)
+    listed[0:8] = True
+    listed[32:37] = True
+    assert (part[:, listed] == want[:, listed]).all() and (part[:, ~listed] == -1.0).all()

@@ -368,7 +368,24 @@ def other_blocks_report(dev, peak, reps=12):
 
     lm_us = timed(lm_call)
     lm_bytes = vocab * d * 2
+    # the same head on int4 rows (three quantised copies rotate)
+    lmq = []
+    for W in Wl:
+        q = torch.empty((vocab, d // 2), dtype=torch.uint8, device=dev)
+        sc = torch.empty((vocab, d // 128), dtype=torch.bfloat16, device=dev)
+        B.halo_quantize_rows_i4(d, vocab, B.BF16, W, q, sc)
+        lmq.append((q, sc))
+    torch.cuda.synchronize()
     del Wl
+
+    def lm_i4_call():
+        q, sc = lmq[i[0] % 3]
+        B.halo_group_lm_head_i4(lm, q, sc, x, 1, None, None, logits, status)
+        i[0] += 1
+
+    lm_i4_us = timed(lm_i4_call)
+    lm_i4_bytes = vocab * (d // 2 + (d // 128) * 2)
+    del lmq
     mh = B.mha_shape(d, H, dh, Lmax, B.BF16)
     sets = []
     for l in range(6):
@@ -427,6 +444,9 @@ def other_blocks_report(dev, peak, reps=12):
     i4_bytes = G * 3 * S * (d // 2 + (d // 128) * 2)
     return {"lm_head": {"shape": "32000 x 4096 bf16, 125 groups of 256 rows", "us_per_token": lm_us,
                         "achieved_gbs": lm_bytes / lm_us / 1e3, "frac_of_peak": lm_bytes / lm_us / 1e3 / peak},
+            "lm_head_int4": {"shape": "32000 x 4096 int4 rows + bf16 scales per 128", "us_per_token": lm_i4_us,
+                             "achieved_gbs": lm_i4_bytes / lm_i4_us / 1e3,
+                             "frac_of_peak": lm_i4_bytes / lm_i4_us / 1e3 / peak},
             "mha_groups": {"shape": "32 heads x 128, d 4096, 1024 cached positions, all heads kept; halo_mha_block "
                                     "(K/V append + attention + output projection in one launch)",
                            "us_per_block": mha_us, "achieved_gbs": mha_bytes / mha_us / 1e3,

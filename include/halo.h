@@ -347,6 +347,10 @@ halo_status halo_group_mha(const halo_mha_shape* shape, const void* W_packed, co
  * ---------------------------------------------------------------------- */
 halo_status halo_quantize_weights_i4(const halo_ffn_shape* shape, const void* W_packed, void* Q, void* scales,
                                      void* stream);
+/* The same quantiser for any row matrix: W device [n_rows][d_model] in wdtype (d_model % 128 == 0, <= 8192) ->
+ * Q device uint8 [n_rows][d_model/2], scales device bf16 [n_rows][d_model/128]; all 16-byte aligned. */
+halo_status halo_quantize_rows_i4(int d_model, long long n_rows, halo_dtype wdtype, const void* W, void* Q, void* scales,
+                                  void* stream);
 halo_status halo_dequantize_weights_i4(const halo_ffn_shape* shape, const void* Q, const void* scales,
                                        const int32_t* keep_list, const int32_t* n_keep, void* W_packed,
                                        uint32_t* dev_status, void* stream);
@@ -374,6 +378,12 @@ typedef struct {
 halo_status halo_group_lm_head(const halo_lm_shape* shape, const void* W, const void* x, int n_tok,
                                const int32_t* keep_list, const int32_t* n_keep, float* logits, uint32_t* dev_status,
                                void* stream);
+/* halo_group_lm_head on int4 rows (Sec. IV-A: the evaluated models are 4-bit): Q / scales as written by
+ * halo_quantize_rows_i4 for W [vocab][d_model] (d_model % 128 == 0); x device bf16 [n_tok][d_model]; shape->wdtype is
+ * ignored.  logits[t][v] = <dequantised row v, x_t> (fp32 accumulation); everything else as halo_group_lm_head. */
+halo_status halo_group_lm_head_i4(const halo_lm_shape* shape, const void* Q, const void* scales, const void* x, int n_tok,
+                                  const int32_t* keep_list, const int32_t* n_keep, float* logits, uint32_t* dev_status,
+                                  void* stream);
 
 /* ------------------------------------------------------------------------
  * One block, steps a1..a9 in one call (the Pred, Comp and merge of one block of the generation phase,

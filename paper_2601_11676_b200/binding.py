@@ -33,7 +33,8 @@ EXPORTS = [
     "halo_selftest_bounded_wait", "halo_group_importance_workspace_bytes", "halo_group_importance",
     "halo_layer_workspace_bytes", "halo_layer_fused", "halo_read_status",
     "halo_pack_mha_weights", "halo_mha_kv_append", "halo_group_mha_workspace_bytes", "halo_group_mha",
-    "halo_group_lm_head", "halo_late_devices", "halo_quantize_weights_i4", "halo_group_ffn_i4", "halo_dequantize_weights_i4", "halo_set_option",
+    "halo_group_lm_head", "halo_late_devices", "halo_quantize_weights_i4", "halo_group_ffn_i4", "halo_dequantize_weights_i4", "halo_quantize_rows_i4", "halo_group_lm_head_i4",
+    "halo_set_option",
     "halo_block_stack_create", "halo_block_stack_destroy", "halo_block_stack_decode", "halo_block_stack_status",
     "halo_block_stack_last_launches", "halo_stack_create_i4", "halo_mha_block",
 ]
@@ -149,6 +150,9 @@ def lib() -> ctypes.CDLL:
         L.halo_quantize_weights_i4.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_void_p]
         L.halo_group_ffn_i4.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
                                         c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+        L.halo_quantize_rows_i4.argtypes = [c_int, c_longlong, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.halo_group_lm_head_i4.argtypes = [POINTER(LmShape), c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
+                                            c_void_p, c_void_p, c_void_p]
         L.halo_dequantize_weights_i4.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                                  c_void_p, c_void_p]
         L.halo_selftest_bounded_wait.argtypes = [c_void_p, c_longlong, c_void_p, c_void_p, c_void_p]
@@ -365,6 +369,16 @@ def halo_group_lm_head(shape: LmShape, W, x, n_tok, keep_list, n_keep, logits, d
 def halo_quantize_weights_i4(shape: FfnShape, W_packed, Q, scales, stream=None) -> None:
     _chk(lib().halo_quantize_weights_i4(byref(shape), _ptr(W_packed), _ptr(Q), _ptr(scales), _stream(stream)),
          "halo_quantize_weights_i4")
+
+
+def halo_quantize_rows_i4(d_model: int, n_rows: int, wdtype: int, W, Q, scales, stream=None) -> None:
+    _chk(lib().halo_quantize_rows_i4(d_model, n_rows, wdtype, _ptr(W), _ptr(Q), _ptr(scales), _stream(stream)),
+         "halo_quantize_rows_i4")
+
+
+def halo_group_lm_head_i4(shape: LmShape, Q, scales, x, n_tok, keep_list, n_keep, logits, dev_status, stream=None) -> None:
+    _chk(lib().halo_group_lm_head_i4(byref(shape), _ptr(Q), _ptr(scales), _ptr(x), n_tok, _ptr(keep_list), _ptr(n_keep),
+                                     _ptr(logits), _ptr(dev_status), _stream(stream)), "halo_group_lm_head_i4")
 
 
 def halo_dequantize_weights_i4(shape: FfnShape, Q, scales, keep_list, n_keep, W_packed, dev_status=None,

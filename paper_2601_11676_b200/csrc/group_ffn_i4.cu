@@ -27,10 +27,6 @@ constexpr int kI4Threads = 256;
 constexpr int kI4Warps = kI4Threads / 32;
 constexpr int kI4BlocksPerSm = 2;
 
-__device__ __forceinline__ uint32_t nibble_pair_bf16(uint32_t word, int k) {
-    return ((word >> (4 * k)) & 0x000F000Fu) | 0x43004300u;      // {128 + nibble k, 128 + nibble k+4} as bf16x2
-}
-
 // The same pair with the right shift done as the high half of a product (word * 2^(32 - 4k)), which runs on the
 // multiply-add pipe; the logic pipe, half as wide, is what bounds the unpacking.  `mul` = 2^(32 - 4k) must reach the
 // kernel as a run-time value, else the compiler turns the product back into a shift.
@@ -942,26 +938,31 @@ halo_status launch_dequantize_i4(const halo_ffn_shape& sh, const void* Q, const 
 
 using namespace halo;
 
+extern "C" halo_status halo_quantize_rows_i4(int d_model, long long n_rows, halo_dtype wdtype, const void* W, void* Q,
+                                             void* scales, void* stream) {
+    if (d_model <= 0 || d_model % kQBlock != 0 || d_model > 8192 || n_rows <= 0) return HALO_ERR_SHAPE;
+    if (wdtype != HALO_F32 && wdtype != HALO_BF16) return HALO_ERR_DTYPE;
+    if (!W || !Q || !scales) return HALO_ERR_ARG;
+    if (!aligned16(W) || !aligned16(Q) || !aligned16(scales)) return HALO_ERR_ALIGN;
+    const long long warps = n_rows * (d_model / kQBlock);
+    if ((warps + 7) / 8 > 0x7fffffffll) return HALO_ERR_SHAPE;
+    const unsigned blocks = static_cast<unsigned>((warps + 7) / 8);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (wdtype == HALO_BF16)
+        quantize_i4_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(d_model, n_rows, static_cast<const __nv_bfloat16*>(W),
+                                                                  static_cast<uint8_t*>(Q),
+                                                                  static_cast<__nv_bfloat16*>(scales));
+    else
+        quantize_i4_kernel<float><<<blocks, 256, 0, st>>>(d_model, n_rows, static_cast<const float*>(W),
+                                                          static_cast<uint8_t*>(Q), static_cast<__nv_bfloat16*>(scales));
+    return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+}
+
 extern "C" halo_status halo_quantize_weights_i4(const halo_ffn_shape* shape, const void* W_packed, void* Q,
                                                 void* scales, void* stream) {
     halo_status rc = check_i4_shape(shape);
     if (rc != HALO_OK) return rc;
-    if (shape->wdtype != HALO_F32 && shape->wdtype != HALO_BF16) return HALO_ERR_DTYPE;
-    if (!W_packed || !Q || !scales) return HALO_ERR_ARG;
-    if (!aligned16(W_packed) || !aligned16(Q) || !aligned16(scales)) return HALO_ERR_ALIGN;
-    const int d = shape->d_model;
-    const long long n_rows = 3ll * shape->d_ffn;
-    const long long warps = n_rows * (d / kQBlock);
-    const unsigned blocks = static_cast<unsigned>((warps + 7) / 8);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (shape->wdtype == HALO_BF16)
-        quantize_i4_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(d, n_rows, static_cast<const __nv_bfloat16*>(W_packed),
-                                                                  static_cast<uint8_t*>(Q),
-                                                                  static_cast<__nv_bfloat16*>(scales));
-    else
-        quantize_i4_kernel<float><<<blocks, 256, 0, st>>>(d, n_rows, static_cast<const float*>(W_packed),
-                                                          static_cast<uint8_t*>(Q), static_cast<__nv_bfloat16*>(scales));
-    return cudaGetLastError() == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+    return halo_quantize_rows_i4(shape->d_model, 3ll * shape->d_ffn, shape->wdtype, W_packed, Q, scales, stream);
 }
 
 extern "C" halo_status halo_dequantize_weights_i4(const halo_ffn_shape* shape, const void* Q, const void* scales,

@@ -8,6 +8,10 @@ namespace halo {
 
 constexpr float kNibbleBias = 136.0f;      // 128 from the bf16 trick + 8 from the code's zero point
 
+__device__ __forceinline__ uint32_t nibble_pair_bf16(uint32_t word, int k) {
+    return ((word >> (4 * k)) & 0x000F000Fu) | 0x43004300u;      // {128 + nibble k, 128 + nibble k+4} as bf16x2
+}
+
 // Mask and exponent bits as run-time values held in registers: with two immediates the "and, then or" is two logic
 // instructions, with register operands it is one three-input instruction.
 struct PairBits { uint32_t mask, magic; };

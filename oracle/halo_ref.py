@@ -383,6 +383,26 @@ def group_mha(Wpacked: np.ndarray, x: np.ndarray, K_cache: np.ndarray, V_cache: 
     return P
 
 
+def _widen32(a: np.ndarray) -> np.ndarray:
+    """bf16 bits or float32 -> float32 (exact)."""
+    return to_f64(a).astype(np.float32)
+
+
+def mha_kv_append_i4(Qk, Sk, Qv, Sv, x: np.ndarray, pos: int, K_cache32: np.ndarray, V_cache32: np.ndarray):
+    """Keys and values of this token from int4 Wk / Wv (their dequantised values) into float32 caches, unrounded."""
+    mha_kv_append(dequantize_i4(Qk, Sk), dequantize_i4(Qv, Sv), _widen32(x), pos, K_cache32, V_cache32)
+
+
+def group_mha_i4(Qp, Sp, H: int, x: np.ndarray, K_cache: np.ndarray, V_cache: np.ndarray, pos: int, head_list,
+                 dev_of_group=None, n_dev: int = 0):
+    """halo_group_mha on int4 packed weights: Qp [H*2*dh][d/2], Sp [H*2*dh][d/128] -> dequantised [H][2][dh][d]; x and the
+    caches (bf16 bits or float32) widened exactly."""
+    W = dequantize_i4(Qp, Sp)
+    rows, d = W.shape
+    return group_mha(W.reshape(H, 2, rows // (2 * H), d), _widen32(x), _widen32(K_cache), _widen32(V_cache), pos, head_list,
+                     dev_of_group, n_dev)
+
+
 def group_lm_head(W: np.ndarray, x: np.ndarray, group_size: int, group_list=None, fill: float = np.nan):
     """LM-head groups (Sec. II-A, Sec. III-B.3): logits[t][v] = <W[v], x_t> for the rows of the listed groups of
     `group_size` vocabulary rows; the other entries keep `fill`."""

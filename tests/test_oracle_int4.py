@@ -103,3 +103,39 @@ def test_lm_head_on_int4_rows_is_a_plain_matrix_product_of_the_code_grid():
     listed[0:8] = True
     listed[32:37] = True
     assert (part[:, listed] == want[:, listed]).all() and (part[:, ~listed] == -1.0).all()
+
+
+def test_mha_on_int4_weights_is_the_mha_on_the_dequantised_values():
+    """Weights built ON the int4 grid: the int4 wrappers must give exactly what the float32 functions give on the same
+    weights (catches a mixed-up code / scale array, a wrong reshape of the packed rows, a cache that is not widened)."""
+    rng = np.random.default_rng(9)
+    d, H, dh, L = 128, 2, 16, 6
+
+    def on_grid(rows):
+        c = rng.integers(-7, 8, size=(rows, d)).astype(np.float32)
+        c[:, 0] = 7
+        return c * np.where(np.arange(rows)[:, None] % 2 == 0, 2.0 ** -4, 2.0 ** -5).astype(np.float32)
+    Wq, Wk, Wv = on_grid(H * dh), on_grid(H * dh), on_grid(H * dh)
+    Wo_rows = on_grid(H * dh)                                  # row h*dh + j = column h*dh + j of Wo
+    Wp = np.stack([np.stack([Wq[h * dh:(h + 1) * dh], Wo_rows[h * dh:(h + 1) * dh]]) for h in range(H)])   # [H][2][dh][d]
+    assert (R.pack_mha(Wq, np.ascontiguousarray(Wo_rows.T), H) == Wp).all()
+    x = (rng.integers(-4, 5, size=d) / 4.0).astype(np.float32)
+    xb = _bf16_bits(x)
+    Qp, Sp = R.quantize_i4(Wp.reshape(H * 2 * dh, d))
+    Qk, Sk = R.quantize_i4(Wk)
+    Qv, Sv = R.quantize_i4(Wv)
+    K32 = rng.standard_normal((H, L, dh)).astype(np.float32)
+    V32 = rng.standard_normal((H, L, dh)).astype(np.float32)
+    Ka, Va, Kb, Vb = K32.copy(), V32.copy(), K32.copy(), V32.copy()
+    R.mha_kv_append_i4(Qk, Sk, Qv, Sv, xb, 3, Ka, Va)
+    R.mha_kv_append(Wk, Wv, x, 3, Kb, Vb)
+    assert (Ka == Kb).all() and (Va == Vb).all() and not (Ka[:, 3] == K32[:, 3]).all()
+    dev = np.array([0, -1], dtype=np.int32)
+    got = R.group_mha_i4(Qp, Sp, H, xb, Ka, Va, 3, [1, 0], dev, 1)
+    want = R.group_mha(Wp, x, Kb, Vb, 3, [1, 0], dev, 1)
+    assert (got == want).all() and np.abs(want).max() > 0
+    # bf16 caches are widened, not reinterpreted
+    Kbits, Vbits = _bf16_bits(Ka), _bf16_bits(Va)
+    got16 = R.group_mha_i4(Qp, Sp, H, xb, Kbits, Vbits, 3, [0], dev, 1)
+    want16 = R.group_mha(Wp, x, R.to_f64(Kbits).astype(np.float32), R.to_f64(Vbits).astype(np.float32), 3, [0], dev, 1)
+    assert (got16 == want16).all()

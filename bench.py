@@ -324,6 +324,7 @@ def run_halo(args, rank, world, local_rank):
         result["other_blocks"] = other_blocks_report(dev, peak)
         result["int4_stack"] = int4_stack_report(dev, peak)
         result["block_stack"] = block_stack_report(dev, peak)
+        result["block_stack_int4"] = block_stack_report(dev, peak, int4=True)
         result["keep_sweep"] = keep_sweep(dev, peak)
         result["overlap_ablation"] = overlap_ablation(dev)
     if world == 1 and not args.no_cpu_baseline:
@@ -416,7 +417,26 @@ def other_blocks_report(dev, peak, reps=12):
     mha_us = timed(mha_call)
     mha_two_us = timed(mha_two_calls)
     mha_bytes = 2 * d * d * 2 + H * (2 * dh * d * 2 + 2 * (pos + 1) * dh * 2)
+    # the same block on int4 weights (caches stay bf16)
+    def qrows(W2d):
+        rows = W2d.shape[0]
+        q = torch.empty((rows, d // 2), dtype=torch.uint8, device=dev)
+        sc = torch.empty((rows, d // 128), dtype=torch.bfloat16, device=dev)
+        B.halo_quantize_rows_i4(d, rows, B.BF16, W2d, q, sc)
+        return q, sc
+    sets4 = [(qrows(Wp.view(-1, d)), qrows(Wk), qrows(Wv), K, V) for (Wp, Wk, Wv, K, V) in sets]
+    torch.cuda.synchronize()
     del sets
+
+    def mha_i4_call():
+        (Qp, Sp), (Qk, Sk), (Qv, Sv), K, V = sets4[j[0] % 6]
+        j[0] += 1
+        B.halo_mha_block_i4(mh, Qp, Sp, Qk, Sk, Qv, Sv, x, K, V, pos, kl, nk, dg, 3, P, status)
+
+    mha_i4_us = timed(mha_i4_call)
+    wb4 = 0.5 + 2.0 / 128.0
+    mha_i4_bytes = 2 * d * d * wb4 + H * (2 * dh * d * wb4 + 2 * (pos + 1) * dh * 2)
+    del sets4
     # the FFN of one 7B-shaped block on int4 group-quantised weights, all groups kept
     fw = synth.workload("llama2-7b-decode")
     G, S = fw.n_groups, fw.group_size
@@ -452,6 +472,9 @@ def other_blocks_report(dev, peak, reps=12):
                            "us_per_block": mha_us, "achieved_gbs": mha_bytes / mha_us / 1e3,
                            "frac_of_peak": mha_bytes / mha_us / 1e3 / peak,
                            "us_per_block_as_two_calls": mha_two_us},
+            "mha_groups_int4": {"shape": "the same block on int4 weights, bf16 caches; halo_mha_block_i4",
+                                "us_per_block": mha_i4_us, "achieved_gbs": mha_i4_bytes / mha_i4_us / 1e3,
+                                "frac_of_peak": mha_i4_bytes / mha_i4_us / 1e3 / peak},
             "ffn_int4": {"shape": "one 7B block, 86 groups of 128, int4 weights + bf16 scales per 128, all kept",
                          "us_per_block": i4_us, "achieved_gbs": i4_bytes / i4_us / 1e3,
                          "frac_of_peak": i4_bytes / i4_us / 1e3 / peak,
@@ -571,15 +594,25 @@ def int4_stack_report(dev, peak, steps=32, warm=4):
     return res
 
 
-def block_stack_report(dev, peak, steps=24, warm=4, context=1024):
+def block_stack_report(dev, peak, steps=24, warm=4, context=1024, int4=False):
     """The paper's generation loop over whole layers at the 7B shape: per layer the MHA block (keys / values of all 32
     heads appended, kept heads attend over `context` cached positions) and the MLP block, each with its predictor,
     selection and merge, and the LM-head groups at the end (32000 x 4096).  One launch per step of the path.
     Bytes: kept FFN groups + kept heads' query / output rows + K/V projections + K/V cache rows read + predictors +
-    LM head."""
+    LM head.  int4: every weight matrix as int4 codes + one bf16 scale per 128 elements (the paper's models are 4-bit);
+    activations, caches and predictors stay bf16."""
     from paper_2601_11676_b200 import binding as B
     wl = synth.workload("llama2-7b-decode")
     L, d, G, H, dh, vocab, r_mha = wl.n_layers, wl.d_model, wl.n_groups, 32, 128, 32000, 64
+    fsh = B.ffn_shape(d, wl.d_ffn, wl.group_size, B.BF16)
+
+    def qrows(W2d):
+        rows = W2d.shape[0]
+        q = torch.empty((rows, d // 2), dtype=torch.uint8, device=dev)
+        sc = torch.empty((rows, d // 128), dtype=torch.bfloat16, device=dev)
+        B.halo_quantize_rows_i4(d, rows, B.BF16, W2d, q, sc)
+        torch.cuda.synchronize()
+        return q, sc
     max_len = context + warm + steps + 1
     mh = B.mha_shape(d, H, dh, max_len, B.BF16)
     mw = synth.Workload("mha-pred", L, d, H * 8, 8, r_mha, "bf16", (), (), 500, 1, seed=wl.seed + 1)
@@ -596,6 +629,12 @@ def block_stack_report(dev, peak, steps=24, warm=4, context=1024):
         K[:, :context] = torch.randn((H, context, dh), generator=g, device=dev).to(torch.bfloat16)
         V[:, :context] = torch.randn((H, context, dh), generator=g, device=dev).to(torch.bfloat16)
         blk = dict(W_ffn=synth.packed_layer(wl, l, dev), W_mha=Wp, Wk=Wk, Wv=Wv, K=K, V=V)
+        if int4:
+            blk["W_ffn"], blk["S_ffn"] = qrows(blk["W_ffn"].view(-1, d))
+            blk["W_mha"], blk["S_mha"] = qrows(Wp.view(-1, d))
+            blk["Wk"], blk["Sk"] = qrows(Wk)
+            blk["Wv"], blk["Sv"] = qrows(Wv)
+            del Wp, Wk, Wv
         if l > 0:
             blk["W1_ffn"], blk["W2_ffn"] = synth.predictor(wl, l, dev)
             blk["W1_mha"], blk["W2_mha"] = synth.predictor(mw, l, dev)
@@ -604,9 +643,12 @@ def block_stack_report(dev, peak, steps=24, warm=4, context=1024):
     W_lm = (torch.randn((vocab, d), generator=gc) / 64).to(torch.bfloat16).to(dev)
     plan_f = B.Plan(G, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
     plan_a = B.Plan(H, wl.loss_rate, wl.share_weight, B.SEL_TOPK, H // 2, 0.0, wl.seed + 1)
-    stack = B.BlockStack(B.ffn_shape(d, wl.d_ffn, wl.group_size, B.BF16), mh, B.lm_shape(d, vocab, 256, B.BF16),
+    S_lm = None
+    if int4:
+        W_lm, S_lm = qrows(W_lm)
+    stack = B.BlockStack(fsh, mh, B.lm_shape(d, vocab, 256, B.BF16),
                          B.pred_shape(d, wl.pred_rank, G, B.BF16), B.pred_shape(d, r_mha, H, B.BF16), plan_f, plan_a,
-                         blocks, W_lm)
+                         blocks, W_lm, S_lm)
     total = warm + steps
     h0 = torch.stack([synth.stream_input(wl, 500 + s, dev)[0] for s in range(total)])
     logits = torch.empty((total, vocab), dtype=torch.float32, device=dev)
@@ -627,12 +669,14 @@ def block_stack_report(dev, peak, steps=24, warm=4, context=1024):
     ms = sorted(ts)[1]
     kept_f, kept_a = int(nk_f[warm:].sum().item()), int(nk_a[warm:].sum().item())
     pos_sum = sum(context + warm + s + 1 for s in range(steps))
-    byts = (kept_f * wl.group_bytes + steps * (L - 1) * (wl.pred_bytes + (d * r_mha + r_mha * H) * 2)
-            + steps * L * 2 * d * d * 2 + kept_a * 2 * dh * d * 2
+    wb = (0.5 + 2.0 / 128.0) if int4 else 2.0                    # bytes per weight element
+    byts = (kept_f * wl.group_bytes / 2 * wb + steps * (L - 1) * (wl.pred_bytes + (d * r_mha + r_mha * H) * 2)
+            + steps * L * 2 * d * d * wb + kept_a * 2 * dh * d * wb
             + sum(int(nk_a[warm + s].sum().item()) * 2 * (context + warm + s + 1) * dh * 2 for s in range(steps))
-            + steps * vocab * d * 2)
+            + steps * vocab * d * wb)
     gbs = byts / (ms * 1e-3) / 1e9
-    res = {"shape": "32 layers x (32 heads of 128 + 86 FFN groups of 128), d 4096, %d cached positions, LM head 32000" % context,
+    res = {"shape": "32 layers x (32 heads of 128 + 86 FFN groups of 128), d 4096, %d cached positions, LM head 32000%s"
+                    % (context, ", int4 weights" if int4 else ""),
            "steps": steps, "tokens_per_s": steps / (ms * 1e-3), "ms_per_token": ms / steps,
            "kept_fraction_ffn": kept_f / float(steps * L * G), "kept_fraction_heads": kept_a / float(steps * L * H),
            "algorithmic_gb_per_token": byts / steps / 1e9, "achieved_gbs": gbs, "frac_of_peak": gbs / peak,

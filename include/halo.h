@@ -320,6 +320,14 @@ halo_status halo_mha_block(const halo_mha_shape* shape, const void* W_packed, co
                            const void* x, void* K_cache, void* V_cache, int pos, const int32_t* keep_list,
                            const int32_t* n_keep, const int32_t* dev_of_group, int n_dev, float* partials,
                            uint32_t* dev_status, void* stream);
+/* halo_mha_block on int4 weights (Sec. IV-A): Qp / Sp, Qk / Sk, Qv / Sv = codes and scales written by
+ * halo_quantize_rows_i4 for W_packed (as [H*2*head_dim][d_model]), Wk and Wv; x and the caches bf16
+ * (shape->wdtype must be HALO_BF16), d_model % 128 == 0, head_dim % 16 == 0.  Results: halo_mha_block on the
+ * dequantised weights. */
+halo_status halo_mha_block_i4(const halo_mha_shape* shape, const void* Qp, const void* Sp, const void* Qk, const void* Sk,
+                              const void* Qv, const void* Sv, const void* x, void* K_cache, void* V_cache, int pos,
+                              const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group, int n_dev,
+                              float* partials, uint32_t* dev_status, void* stream);
 halo_status halo_group_mha(const halo_mha_shape* shape, const void* W_packed, const void* x, const void* K_cache,
                            const void* V_cache, int pos, const int32_t* keep_list, const int32_t* n_keep,
                            const int32_t* dev_of_group, int n_dev, float* partials, void* workspace,
@@ -550,6 +558,24 @@ halo_status halo_block_stack_create(halo_block_stack** out, const halo_ffn_shape
                                     const halo_lm_shape* lm, const halo_pred_shape* pred_ffn,
                                     const halo_pred_shape* pred_mha, int n_layers, const halo_plan* plan_ffn,
                                     const halo_plan* plan_mha, const halo_block_weights* weights);
+/* The same stack on int4 weights (Sec. IV-A: the evaluated models are 4-bit): `codes` has the layout of
+ * halo_block_weights with W_ffn = codes of halo_quantize_weights_i4, W_mha / Wk / Wv / W_lm = codes of
+ * halo_quantize_rows_i4 of the matrices named there; `scales` holds the matching scale arrays (host arrays of n_layers
+ * device pointers, 16-byte aligned; S_lm NULL without an LM head).  Predictor factors, activations and the K/V caches
+ * stay bf16 (every shape's wdtype must be HALO_BF16); d_model % 128 == 0, head_dim % 16 == 0.  Per layer:
+ * halo_mha_block_i4, halo_group_ffn_i4, and halo_group_lm_head_i4 at the end. */
+typedef struct {
+    const void* const* S_ffn;
+    const void* const* S_mha;
+    const void* const* Sk;
+    const void* const* Sv;
+    const void* S_lm;
+} halo_block_scales;
+halo_status halo_block_stack_create_i4(halo_block_stack** out, const halo_ffn_shape* ffn, const halo_mha_shape* mha,
+                                       const halo_lm_shape* lm, const halo_pred_shape* pred_ffn,
+                                       const halo_pred_shape* pred_mha, int n_layers, const halo_plan* plan_ffn,
+                                       const halo_plan* plan_mha, const halo_block_weights* codes,
+                                       const halo_block_scales* scales);
 halo_status halo_block_stack_destroy(halo_block_stack* stack);
 halo_status halo_block_stack_decode(halo_block_stack* stack, const float* h0, int steps, int pos0, uint32_t step0,
                                     float* logits, float* h_out, const halo_block_taps* taps, void* stream);

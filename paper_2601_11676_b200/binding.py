@@ -33,7 +33,8 @@ EXPORTS = [
     "halo_selftest_bounded_wait", "halo_group_importance_workspace_bytes", "halo_group_importance",
     "halo_layer_workspace_bytes", "halo_layer_fused", "halo_read_status",
     "halo_pack_mha_weights", "halo_mha_kv_append", "halo_group_mha_workspace_bytes", "halo_group_mha",
-    "halo_group_lm_head", "halo_late_devices", "halo_quantize_weights_i4", "halo_group_ffn_i4", "halo_dequantize_weights_i4", "halo_quantize_rows_i4", "halo_group_lm_head_i4",
+    "halo_group_lm_head", "halo_late_devices", "halo_quantize_weights_i4", "halo_group_ffn_i4", "halo_dequantize_weights_i4", "halo_quantize_rows_i4", "halo_group_lm_head_i4", "halo_mha_block_i4",
+    "halo_block_stack_create_i4",
     "halo_set_option",
     "halo_block_stack_create", "halo_block_stack_destroy", "halo_block_stack_decode", "halo_block_stack_status",
     "halo_block_stack_last_launches", "halo_stack_create_i4", "halo_mha_block",
@@ -64,6 +65,10 @@ class Taps(Structure):
 class BlockWeights(Structure):
     _fields_ = [(n, POINTER(c_void_p)) for n in ("W_ffn", "W_mha", "Wk", "Wv", "W1_ffn", "W2_ffn", "W1_mha", "W2_mha",
                                                   "K_cache", "V_cache")] + [("W_lm", c_void_p)]
+
+
+class BlockScales(Structure):
+    _fields_ = [(n, POINTER(c_void_p)) for n in ("S_ffn", "S_mha", "Sk", "Sv")] + [("S_lm", c_void_p)]
 
 
 class BlockTaps(Structure):
@@ -145,6 +150,12 @@ def lib() -> ctypes.CDLL:
                                      c_void_p, c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
         L.halo_mha_block.argtypes = [POINTER(MhaShape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int,
                                      c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+        L.halo_mha_block_i4.argtypes = [POINTER(MhaShape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                        c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int,
+                                        c_void_p, c_void_p, c_void_p]
+        L.halo_block_stack_create_i4.argtypes = [POINTER(c_void_p), POINTER(FfnShape), POINTER(MhaShape), POINTER(LmShape),
+                                                 POINTER(PredShape), POINTER(PredShape), c_int, c_void_p, c_void_p,
+                                                 POINTER(BlockWeights), POINTER(BlockScales)]
         L.halo_group_lm_head.argtypes = [POINTER(LmShape), c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
                                          c_void_p, c_void_p]
         L.halo_quantize_weights_i4.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_void_p]
@@ -357,6 +368,13 @@ def halo_mha_block(shape: MhaShape, W_packed, Wk, Wv, x, K_cache, V_cache, pos, 
                               _stream(stream)), "halo_mha_block")
 
 
+def halo_mha_block_i4(shape: MhaShape, Qp, Sp, Qk, Sk, Qv, Sv, x, K_cache, V_cache, pos, keep_list, n_keep, dev_of_group,
+                      n_dev, partials, dev_status=None, stream=None) -> None:
+    _chk(lib().halo_mha_block_i4(byref(shape), _ptr(Qp), _ptr(Sp), _ptr(Qk), _ptr(Sk), _ptr(Qv), _ptr(Sv), _ptr(x),
+                                 _ptr(K_cache), _ptr(V_cache), pos, _ptr(keep_list), _ptr(n_keep), _ptr(dev_of_group), n_dev,
+                                 _ptr(partials), _ptr(dev_status), _stream(stream)), "halo_mha_block_i4")
+
+
 def lm_shape(d_model, vocab, group_size, dtype) -> LmShape:
     return LmShape(d_model, vocab, group_size, dtype)
 
@@ -517,12 +535,15 @@ class Stack:
 
 class BlockStack:
     """halo_block_stack_create / _decode / _destroy.  Keeps the weight and cache tensors alive.
-    blocks: list of dicts with W_ffn, W_mha, Wk, Wv, K, V and (from the second layer on) W1_ffn, W2_ffn, W1_mha, W2_mha."""
+    blocks: list of dicts with W_ffn, W_mha, Wk, Wv, K, V and (from the second layer on) W1_ffn, W2_ffn, W1_mha, W2_mha.
+    int4 stacks (halo_block_stack_create_i4): the four weight entries hold codes, the dicts also have S_ffn, S_mha, Sk,
+    Sv, and S_lm comes with W_lm."""
 
     def __init__(self, ffn: FfnShape, mha: MhaShape, lm, pred_ffn: PredShape, pred_mha: PredShape, plan_ffn: Plan,
-                 plan_mha: Plan, blocks, W_lm=None):
+                 plan_mha: Plan, blocks, W_lm=None, S_lm=None):
         L = len(blocks)
-        self._keep = (blocks, W_lm, plan_ffn, plan_mha)
+        self._keep = (blocks, W_lm, S_lm)
+        self.plan_ffn, self.plan_mha = plan_ffn, plan_mha
         self.n_layers = L
         arr = lambda key: (c_void_p * L)(*[(b[key].data_ptr() if b.get(key) is not None else None) for b in blocks])
         self._arrays = {k: arr(k) for k in ("W_ffn", "W_mha", "Wk", "Wv", "W1_ffn", "W2_ffn", "W1_mha", "W2_mha", "K", "V")}
@@ -533,6 +554,17 @@ class BlockStack:
         w.V_cache = ctypes.cast(self._arrays["V"], POINTER(c_void_p))
         w.W_lm = c_void_p(W_lm.data_ptr()) if W_lm is not None else None
         self.handle = c_void_p()
+        if blocks[0].get("S_ffn") is not None:
+            self._scale_arrays = {k: arr(k) for k in ("S_ffn", "S_mha", "Sk", "Sv")}
+            sc = BlockScales()
+            for k in ("S_ffn", "S_mha", "Sk", "Sv"):
+                setattr(sc, k, ctypes.cast(self._scale_arrays[k], POINTER(c_void_p)))
+            sc.S_lm = c_void_p(S_lm.data_ptr()) if S_lm is not None else None
+            _chk(lib().halo_block_stack_create_i4(byref(self.handle), byref(ffn), byref(mha),
+                                                  byref(lm) if lm is not None else None, byref(pred_ffn), byref(pred_mha), L,
+                                                  plan_ffn.handle, plan_mha.handle, byref(w), byref(sc)),
+                 "halo_block_stack_create_i4")
+            return
         _chk(lib().halo_block_stack_create(byref(self.handle), byref(ffn), byref(mha), byref(lm) if lm is not None else None,
                                            byref(pred_ffn), byref(pred_mha), L, plan_ffn.handle, plan_mha.handle, byref(w)),
              "halo_block_stack_create")

@@ -27,6 +27,10 @@ struct halo_block_stack {
     std::vector<const void*> W_ffn, W_mha, Wk, Wv, W1_ffn, W2_ffn, W1_mha, W2_mha;
     std::vector<void*> K, V;
     const void* W_lm;
+    // int4 stacks: W_ffn, W_mha, Wk, Wv and W_lm hold codes, these their scales (activations, caches, predictors bf16)
+    bool i4 = false;
+    std::vector<const void*> S_ffn, S_mha, Sk, Sv;
+    const void* S_lm = nullptr;
     void* slab;
     float* h;
     void* x_a[2];
@@ -46,10 +50,46 @@ struct halo_block_stack {
     long long last_launches;
 };
 
+namespace {
+halo_status block_stack_create_impl(halo_block_stack** out, const halo_ffn_shape* ffn, const halo_mha_shape* mha,
+                                    const halo_lm_shape* lm, const halo_pred_shape* pred_ffn,
+                                    const halo_pred_shape* pred_mha, int n_layers, const halo_plan* plan_ffn,
+                                    const halo_plan* plan_mha, const halo_block_weights* w, const halo_block_scales* sc);
+}  // namespace
+
 extern "C" halo_status halo_block_stack_create(halo_block_stack** out, const halo_ffn_shape* ffn, const halo_mha_shape* mha,
                                                const halo_lm_shape* lm, const halo_pred_shape* pred_ffn,
                                                const halo_pred_shape* pred_mha, int n_layers, const halo_plan* plan_ffn,
                                                const halo_plan* plan_mha, const halo_block_weights* w) {
+    return block_stack_create_impl(out, ffn, mha, lm, pred_ffn, pred_mha, n_layers, plan_ffn, plan_mha, w, nullptr);
+}
+
+extern "C" halo_status halo_block_stack_create_i4(halo_block_stack** out, const halo_ffn_shape* ffn, const halo_mha_shape* mha,
+                                                  const halo_lm_shape* lm, const halo_pred_shape* pred_ffn,
+                                                  const halo_pred_shape* pred_mha, int n_layers, const halo_plan* plan_ffn,
+                                                  const halo_plan* plan_mha, const halo_block_weights* codes,
+                                                  const halo_block_scales* scales) {
+    if (!out) return HALO_ERR_ARG;
+    *out = nullptr;
+    if (!ffn || !mha || !scales) return HALO_ERR_ARG;
+    if (ffn->wdtype != HALO_BF16) return HALO_ERR_DTYPE;                   // activations, caches and predictors
+    if (ffn->d_model % 128 != 0 || mha->head_dim % 16 != 0) return HALO_ERR_SHAPE;
+    if (!scales->S_ffn || !scales->S_mha || !scales->Sk || !scales->Sv || (lm && !scales->S_lm)) return HALO_ERR_ARG;
+    for (int l = 0; l < n_layers; ++l) {
+        const void* p[4] = {scales->S_ffn[l], scales->S_mha[l], scales->Sk[l], scales->Sv[l]};
+        for (const void* q : p) {
+            if (!q) return HALO_ERR_ARG;
+            if (!aligned16(q)) return HALO_ERR_ALIGN;
+        }
+    }
+    return block_stack_create_impl(out, ffn, mha, lm, pred_ffn, pred_mha, n_layers, plan_ffn, plan_mha, codes, scales);
+}
+
+namespace {
+halo_status block_stack_create_impl(halo_block_stack** out, const halo_ffn_shape* ffn, const halo_mha_shape* mha,
+                                    const halo_lm_shape* lm, const halo_pred_shape* pred_ffn,
+                                    const halo_pred_shape* pred_mha, int n_layers, const halo_plan* plan_ffn,
+                                    const halo_plan* plan_mha, const halo_block_weights* w, const halo_block_scales* sc) {
     if (!out) return HALO_ERR_ARG;
     *out = nullptr;
     if (!ffn || !mha || !pred_ffn || !pred_mha || !plan_ffn || !plan_mha || !w) return HALO_ERR_ARG;
@@ -86,6 +126,11 @@ extern "C" halo_status halo_block_stack_create(halo_block_stack** out, const hal
     s->K.assign(w->K_cache, w->K_cache + n_layers);
     s->V.assign(w->V_cache, w->V_cache + n_layers);
     s->W_lm = w->W_lm;
+    if (sc) {
+        s->i4 = true;
+        take(s->S_ffn, sc->S_ffn); take(s->S_mha, sc->S_mha); take(s->Sk, sc->Sk); take(s->Sv, sc->Sv);
+        s->S_lm = sc->S_lm;
+    }
     s->last_launches = 0;
 
     const size_t es = bs_elem(ffn->wdtype);
@@ -145,6 +190,7 @@ extern "C" halo_status halo_block_stack_create(halo_block_stack** out, const hal
     *out = s;
     return HALO_OK;
 }
+}  // namespace
 
 extern "C" halo_status halo_block_stack_destroy(halo_block_stack* s) {
     if (!s) return HALO_OK;
@@ -208,7 +254,12 @@ extern "C" halo_status halo_block_stack_decode(halo_block_stack* s, const float*
                 if (fork) BS_CU(cudaEventRecord(s->ev_sa, side));
                 launches += 2;
             }
-            if (s->mha.head_dim % 16 == 0) {
+            if (s->i4) {
+                BS_TRY(launch_mha_block_i4(s->mha, s->W_mha[l], s->S_mha[l], s->Wk[l], s->Sk[l], s->Wv[l], s->Sv[l], xa, s->K[l],
+                                           s->V[l], pos, s->kl_a[cur], s->nk_a[cur], s->dev_a[cur], s->n_dev_a, s->part_a,
+                                           s->status, st, true));
+                ++launches;
+            } else if (s->mha.head_dim % 16 == 0) {
                 BS_TRY(launch_mha_block(s->mha, s->W_mha[l], s->Wk[l], s->Wv[l], xa, s->K[l], s->V[l], pos, s->kl_a[cur],
                                         s->nk_a[cur], s->dev_a[cur], s->n_dev_a, s->part_a, s->status, st, true));
                 ++launches;
@@ -245,9 +296,16 @@ extern "C" halo_status halo_block_stack_decode(halo_block_stack* s, const float*
                 if (fork) BS_CU(cudaEventRecord(s->ev_sf, side));
                 launches += 2;
             }
-            BS_TRY(launch_group_ffn_decode(s->ffn, s->W_ffn[l], xf, 1, s->kl_f[cur], s->nk_f[cur], s->dev_f[cur], s->n_dev_f,
-                                           s->part_f, s->status, st, true));
-            ++launches;
+            if (s->i4) {
+                // (the entry point zeroes the slots itself: one small launch that the streaming kernel overlaps)
+                BS_TRY(halo_group_ffn_i4(&s->ffn, s->W_ffn[l], s->S_ffn[l], xf, 1, s->kl_f[cur], s->nk_f[cur], s->dev_f[cur],
+                                         s->n_dev_f, s->part_f, s->status, stream));
+                launches += 2;
+            } else {
+                BS_TRY(launch_group_ffn_decode(s->ffn, s->W_ffn[l], xf, 1, s->kl_f[cur], s->nk_f[cur], s->dev_f[cur], s->n_dev_f,
+                                               s->part_f, s->status, st, true));
+                ++launches;
+            }
             y_tap = nullptr;
             if (taps) {
                 const halo_taps& t = taps->ffn;
@@ -272,8 +330,12 @@ extern "C" halo_status halo_block_stack_decode(halo_block_stack* s, const float*
         }
         if (logits) {
             // LM head: every vocabulary group, sent reliably (Sec. III-B.3)
-            BS_TRY(halo_group_lm_head(&s->lm, s->W_lm, s->x_a[L & 1], 1, nullptr, nullptr,
-                                      logits + static_cast<size_t>(sidx) * s->lm.vocab, s->status, stream));
+            if (s->i4)
+                BS_TRY(halo_group_lm_head_i4(&s->lm, s->W_lm, s->S_lm, s->x_a[L & 1], 1, nullptr, nullptr,
+                                             logits + static_cast<size_t>(sidx) * s->lm.vocab, s->status, stream));
+            else
+                BS_TRY(halo_group_lm_head(&s->lm, s->W_lm, s->x_a[L & 1], 1, nullptr, nullptr,
+                                          logits + static_cast<size_t>(sidx) * s->lm.vocab, s->status, stream));
             ++launches;
         }
         if (h_out) BS_COPY(h_out + static_cast<size_t>(sidx) * d, s->h, sizeof(float) * d);

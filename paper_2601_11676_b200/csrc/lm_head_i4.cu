@@ -9,9 +9,7 @@
 // in the FFN kernel, changed nothing here: no single pipe is the bound, the issue slots are 55 % busy at 24 warps per SM).
 #include <algorithm>
 
-#include "common.cuh"
-#include "ffn_math.cuh"
-#include "i4_math.cuh"
+#include "i4_rows.cuh"
 
 namespace halo {
 
@@ -21,23 +19,12 @@ constexpr int kLmI4Warps = kLmI4Threads / 32;
 constexpr int kLmI4RowsPerItem = 2 * kLmI4Warps;                     // a warp takes two rows of an item
 constexpr int kLmI4BlocksPerSm = 3;
 
-// Operands of one row pair held by a lane: chunks lane + 32u of both rows and their scales (rows up to 4096 wide), or,
-// for wider rows, the chunks of one 4096-element slice at a time.
-struct PairRegs {
-    uint4 wa[4], wb[4];
-    float sa[4], sb[4];
-    int v0;            // first row, or -1 when this warp has nothing to do in the item
-    bool two;
-};
-
 __global__ void __launch_bounds__(kLmI4Threads, kLmI4BlocksPerSm)
 lm_head_i4_kernel(int d, int vocab, int S, int n_tok, const uint8_t* __restrict__ Q,
                   const __nv_bfloat16* __restrict__ scales, const __nv_bfloat16* __restrict__ x,
                   const int32_t* __restrict__ keep_list, const int32_t* __restrict__ n_keep_ptr,
                   float* __restrict__ logits, uint32_t* dev_status) {
     extern __shared__ __align__(16) unsigned char smem_b[];
-    const int chunks16 = d / 32;                                     // 16-byte code chunks (32 weights) per row
-    const int nb = d / 128;
     uint4* xp = reinterpret_cast<uint4*>(smem_b);                    // [4][chunks16]: x in nibble pairing
     float* xsum = reinterpret_cast<float*>(smem_b + static_cast<size_t>(d) * 2);   // [chunks16]
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -46,7 +33,6 @@ lm_head_i4_kernel(int d, int vocab, int S, int n_tok, const uint8_t* __restrict_
     int nk = n_groups;
     if (keep_list) nk = max(0, min(*n_keep_ptr, n_groups));
     const long long total = static_cast<long long>(nk) * items_per_group;
-    const size_t row_bytes = static_cast<size_t>(d) / 2;
     // rows of this warp in an item (and whether the item is valid at all)
     auto rows_of = [&](long long item, int& v0, bool& two, bool report) {
         v0 = -1;
@@ -65,80 +51,22 @@ lm_head_i4_kernel(int d, int vocab, int S, int n_tok, const uint8_t* __restrict_
             two = v + 1 < v_end;
         }
     };
-    // the chunks c0 + 32u of the pair's rows
-    auto fetch = [&](PairRegs& r, int c0) {
-        if (r.v0 < 0) return;
-        const size_t ra = static_cast<size_t>(r.v0), rb = r.two ? ra + 1 : ra;   // a lone last row: read twice, used once
-        const uint4* a4 = reinterpret_cast<const uint4*>(Q + ra * row_bytes);
-        const uint4* b4 = reinterpret_cast<const uint4*>(Q + rb * row_bytes);
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int c = c0 + 32 * u;
-            if (c < chunks16) {
-                r.wa[u] = ldg_stream16(a4 + c);
-                r.wb[u] = ldg_stream16(b4 + c);
-                r.sa[u] = __bfloat162float(scales[ra * nb + (c >> 2)]);
-                r.sb[u] = __bfloat162float(scales[rb * nb + (c >> 2)]);
-            }
-        }
-    };
-    auto dot = [&](const PairRegs& r, int c0, float& acc_a, float& acc_b) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int c = c0 + 32 * u;
-            if (c < chunks16) {
-                float ta0 = 0.0f, ta1 = 0.0f, tb0 = 0.0f, tb1 = 0.0f;
-                const uint32_t aw[4] = {r.wa[u].x, r.wa[u].y, r.wa[u].z, r.wa[u].w};
-                const uint32_t bw[4] = {r.wb[u].x, r.wb[u].y, r.wb[u].z, r.wb[u].w};
-#pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    const uint4 xq = xp[static_cast<size_t>(w) * chunks16 + c];
-                    const uint32_t xk[4] = {xq.x, xq.y, xq.z, xq.w};
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        fma_bf16x2(nibble_pair_bf16(aw[w], k), xk[k], ta0, ta1);
-                        fma_bf16x2(nibble_pair_bf16(bw[w], k), xk[k], tb0, tb1);
-                    }
-                }
-                const float off = kNibbleBias * xsum[c];
-                acc_a = fmaf(r.sa[u], (ta0 + ta1) - off, acc_a);
-                acc_b = fmaf(r.sb[u], (tb0 + tb1) - off, acc_b);
-            }
-        }
-    };
-
     for (int t = 0; t < n_tok; ++t) {
         if (t > 0) __syncthreads();                                  // everybody is done with the previous x
-        // for chunk c and word w of a code chunk, the four pairs (x[8w+k], x[8w+k+4]), k = 0..3, as bf16x2
-        const uint16_t* xb = reinterpret_cast<const uint16_t*>(x + static_cast<size_t>(t) * d);
-        uint32_t* xp_words = reinterpret_cast<uint32_t*>(xp);
-        PairRegs cur;
-        for (int i = tid; i < d / 2; i += kLmI4Threads) {
-            const int c = i / 16, r = i - c * 16, w = r >> 2, k = r & 3;
-            const uint32_t lo16 = xb[32 * c + 8 * w + k], hi16 = xb[32 * c + 8 * w + k + 4];
-            xp_words[(static_cast<size_t>(w) * chunks16 + c) * 4 + k] = lo16 | (hi16 << 16);
-        }
-        for (int c = tid; c < chunks16; c += kLmI4Threads) {
-            float sx = 0.0f;
-            for (int e = 0; e < 32; ++e) sx += __bfloat162float(x[static_cast<size_t>(t) * d + 32 * c + e]);
-            xsum[c] = sx;
-        }
+        stage_x_paired(x + static_cast<size_t>(t) * d, xp, xsum, d);
         __syncthreads();
 
         for (long long item = blockIdx.x; item < total; item += gridDim.x) {
-            float acc_a = 0.0f, acc_b = 0.0f;
-            rows_of(item, cur.v0, cur.two, t == 0);
-            if (cur.v0 >= 0)
-                for (int c0 = lane; c0 < chunks16; c0 += 128) {
-                    fetch(cur, c0);
-                    dot(cur, c0, acc_a, acc_b);
-                }
-            if (cur.v0 >= 0) {                                       // warp-uniform
-                acc_a = warp_sum(acc_a);
-                acc_b = warp_sum(acc_b);
-                float* out = logits + static_cast<size_t>(t) * vocab + cur.v0;
+            int v0;
+            bool two;
+            rows_of(item, v0, two, t == 0);
+            if (v0 >= 0) {                                           // warp-uniform
+                float acc_a, acc_b;
+                const size_t ra = static_cast<size_t>(v0);           // a lone last row: read twice, used once
+                warp_two_rows_dot_i4(Q, scales, ra, two ? ra + 1 : ra, d, xp, xsum, lane, acc_a, acc_b);
+                float* out = logits + static_cast<size_t>(t) * vocab + v0;
                 if (lane == 0) out[0] = acc_a;
-                if (lane == 1 && cur.two) out[1] = acc_b;
+                if (lane == 1 && two) out[1] = acc_b;
             }
         }
     }

@@ -13,6 +13,7 @@
 #include <cstdlib>
 
 #include "common.cuh"
+#include "i4_rows.cuh"
 #include "tma.cuh"
 
 namespace halo {
@@ -333,15 +334,23 @@ static size_t kv_smem_bytes(int pos, int dh, size_t elem) {
     return (bytes <= kKvSmemMax && (static_cast<size_t>(dh) * elem) % 16 == 0) ? bytes : 0;
 }
 
-template <typename T, int ITERS, bool APPEND>
+// I4 (with APPEND, T = bf16): Wp, Wk and Wv hold int4 codes (halo_quantize_rows_i4 of the same row matrices), Sp, Sk
+// and Sv their scales; x and the caches stay bf16.  The row products go against x in the nibble pairing, the
+// output-projection rows are unpacked into 16 columns per thread; everything between is the same code.
+template <typename T, int ITERS, bool APPEND, bool I4 = false>
 __global__ void __cluster_dims__(kMhaCluster, 1, 1) __launch_bounds__(256)
 mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ Wp, const T* __restrict__ x,
                  const T* Kc, const T* Vc, const int32_t* __restrict__ keep_list,
                  const int32_t* __restrict__ n_keep_ptr, const int32_t* __restrict__ dev_of_group, int n_dev,
                  float* __restrict__ partials, uint32_t* dev_status, const T* __restrict__ Wk, const T* __restrict__ Wv,
-                 T* Kw, T* Vw, int kv_smem) {
+                 T* Kw, T* Vw, int kv_smem, const __nv_bfloat16* __restrict__ Sp = nullptr,
+                 const __nv_bfloat16* __restrict__ Sk = nullptr, const __nv_bfloat16* __restrict__ Sv = nullptr) {
+    static_assert(!I4 || (APPEND && sizeof(T) == 2), "int4 weights: fused block on bf16 activations only");
     constexpr int E = Elem<T>::kPerChunk;
     extern __shared__ __align__(16) float xs[];          // [d]: x widened; behind it (kv_smem): this block's K and V rows
+    // int4: the same d floats hold x in the nibble pairing (2d bytes) and its sums per 32 elements (d/8 bytes)
+    uint4* xp = reinterpret_cast<uint4*>(xs);
+    float* xsum = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(xs) + static_cast<size_t>(d) * 2);
     __shared__ uint64_t kv_bar;
     __shared__ float q_s[256];                           // the head's full query (written by all blocks of the cluster)
     __shared__ float o_acc[256];                         // this block's running o over its positions
@@ -362,14 +371,21 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
         asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see group_ffn_stream_kernel
         h = blockIdx.y;
         // keys and values of this token for head h, rows j0 .. j0 + rows of each, two rows per warp and turn
-        stage_x(x, xs, d);
+        if constexpr (I4) stage_x_paired(reinterpret_cast<const __nv_bfloat16*>(x), xp, xsum, d);
+        else stage_x(x, xs, d);
         __syncthreads();
         for (int i = 2 * warp; i < 2 * rows; i += 16) {
             const bool is_v = i >= rows;
             const int j = j0 + (is_v ? i - rows : i);
-            const T* base = (is_v ? Wv : Wk) + (static_cast<size_t>(h) * dh + j) * d;
             float va, vb;
-            warp_two_rows_dot(base, base + d, xs, chunks, lane, va, vb);
+            if constexpr (I4) {
+                const size_t row = static_cast<size_t>(h) * dh + j;
+                warp_two_rows_dot_i4(reinterpret_cast<const uint8_t*>(is_v ? Wv : Wk), is_v ? Sv : Sk, row, row + 1, d, xp,
+                                     xsum, lane, va, vb);
+            } else {
+                const T* base = (is_v ? Wv : Wk) + (static_cast<size_t>(h) * dh + j) * d;
+                warp_two_rows_dot(base, base + d, xs, chunks, lane, va, vb);
+            }
             if (lane < 2) (is_v ? Vw : Kw)[(static_cast<size_t>(h) * Lmax + pos) * dh + j + lane] = from_float<T>(lane == 0 ? va : vb);
         }
         // is this head kept, and by whom?  (the list is short: one pass of the block over it)
@@ -437,9 +453,14 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
     const float scale = rsqrtf(static_cast<float>(dh));
     cluster_wait();                                      // every block of the cluster has started
     for (int i = 2 * warp; i < rows; i += 16) {
-        const T* base = Wp + ((static_cast<size_t>(h) * 2 + 0) * dh + j0 + i) * d;
         float va, vb;
-        warp_two_rows_dot(base, base + d, xs, chunks, lane, va, vb);
+        if constexpr (I4) {
+            const size_t row = (static_cast<size_t>(h) * 2 + 0) * dh + j0 + i;
+            warp_two_rows_dot_i4(reinterpret_cast<const uint8_t*>(Wp), Sp, row, row + 1, d, xp, xsum, lane, va, vb);
+        } else {
+            const T* base = Wp + ((static_cast<size_t>(h) * 2 + 0) * dh + j0 + i) * d;
+            warp_two_rows_dot(base, base + d, xs, chunks, lane, va, vb);
+        }
         if (lane < kMhaCluster) {
             st_remote_f32(&q_s[j0 + i], lane, va * scale);
             st_remote_f32(&q_s[j0 + i + 1], lane, vb * scale);
@@ -565,6 +586,71 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
     __syncthreads();
 
     // ---- output-projection rows j0 .. j0 + rows of the head's slice: column sums into the holder's slot ----
+    if constexpr (I4) {
+        // a thread owns 8-byte code chunks (16 columns each); sums of f * (128 + nibble) with f = o_j * scale, and of f
+        // alone, whose 136-fold is taken off at the end
+        const int chunks8 = d / 16, nb = d / 128;
+        const size_t row_bytes = static_cast<size_t>(d) / 2;
+        const uint8_t* Qp = reinterpret_cast<const uint8_t*>(Wp);
+        const size_t row0 = (static_cast<size_t>(h) * 2 + 1) * dh + j0;
+        float acc4[ITERS][16], corr[ITERS];
+#pragma unroll
+        for (int i = 0; i < ITERS; ++i) {
+            corr[i] = 0.0f;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) acc4[i][k] = 0.0f;
+        }
+        constexpr int kRowsInFlight = ITERS == 1 ? 8 : 4;
+        for (int jb = 0; jb < rows; jb += kRowsInFlight) {
+            uint2 wv[kRowsInFlight][ITERS];
+            float sv[kRowsInFlight][ITERS];
+#pragma unroll
+            for (int jj = 0; jj < kRowsInFlight; ++jj)
+#pragma unroll
+                for (int i = 0; i < ITERS; ++i) {
+                    const int c = tid + 256 * i;
+                    if (c < chunks8 && jb + jj < rows) {
+                        const size_t rw = row0 + jb + jj;
+                        wv[jj][i] = __ldg(reinterpret_cast<const uint2*>(Qp + rw * row_bytes) + c);
+                        sv[jj][i] = __bfloat162float(Sp[rw * nb + (c >> 3)]);
+                    } else {
+                        wv[jj][i] = make_uint2(0u, 0u);
+                        sv[jj][i] = 0.0f;
+                    }
+                }
+#pragma unroll
+            for (int jj = 0; jj < kRowsInFlight; ++jj) {
+                const float o = jb + jj < rows ? o_s[jb + jj] : 0.0f;
+#pragma unroll
+                for (int i = 0; i < ITERS; ++i) {
+                    const float f = o * sv[jj][i];               // 0 for the padded rows and columns
+                    corr[i] += f;
+                    const uint32_t words[2] = {wv[jj][i].x, wv[jj][i].y};
+#pragma unroll
+                    for (int v = 0; v < 2; ++v)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const uint32_t p = nibble_pair_bf16(words[v], k);
+                            acc4[i][8 * v + k] = fmaf(f, __uint_as_float(p << 16), acc4[i][8 * v + k]);
+                            acc4[i][8 * v + k + 4] = fmaf(f, __uint_as_float(p & 0xffff0000u), acc4[i][8 * v + k + 4]);
+                        }
+                }
+            }
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");       // the zero-fill of the slots (see below)
+        float* dst4 = partials + static_cast<size_t>(slot) * d;
+#pragma unroll
+        for (int i = 0; i < ITERS; ++i) {
+            const int c = tid + 256 * i;
+            if (c < chunks8) {
+                const float off = kNibbleBias * corr[i];
+#pragma unroll
+                for (int k = 0; k < 16; k += 4)
+                    red_add_v4f(dst4 + c * 16 + k, acc4[i][k] - off, acc4[i][k + 1] - off, acc4[i][k + 2] - off,
+                                acc4[i][k + 3] - off);
+            }
+        }
+    } else {
     float acc[ITERS][E];
 #pragma unroll
     for (int i = 0; i < ITERS; ++i)
@@ -608,6 +694,7 @@ mha_fused_kernel(int d, int H, int dh, int Lmax, int pos, const T* __restrict__ 
 #pragma unroll
             for (int k = 0; k < E; k += 4) red_add_v4f(dst + c * E + k, acc[i][k], acc[i][k + 1], acc[i][k + 2], acc[i][k + 3]);
         }
+    }
     }
 }
 
@@ -806,13 +893,14 @@ static halo_status mha_block_typed(const halo_mha_shape& sh, const void* Wp, con
     const int Lmax = sh.max_len;
     cudaError_t err = cudaSuccess;
     const int kv_flag = kv_b ? 1 : 0;
+    const __nv_bfloat16* no_scales = nullptr;
 #define HALO_MHA_BLOCK(I)                                                                                            \
     case I: {                                                                                                        \
         static bool once[64] = {};                                                                                   \
         if (!ensure_dynamic_smem(mha_fused_kernel<T, I, true>, kMhaSmemLimit, once)) return HALO_ERR_CUDA; \
         err = cudaLaunchKernelEx(&cfg, mha_fused_kernel<T, I, true>, d, H, dh, Lmax, pos, Wp_t, x_t, Kc_t, Vc_t,      \
                                  keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, Wk_t, Wv_t, Kw_t, Vw_t, \
-                                 kv_flag);                                                                            \
+                                 kv_flag, no_scales, no_scales, no_scales);                                           \
         break;                                                                                                       \
     }
     switch (iters) {
@@ -823,6 +911,51 @@ static halo_status mha_block_typed(const halo_mha_shape& sh, const void* Wp, con
         default: return HALO_ERR_SHAPE;
     }
 #undef HALO_MHA_BLOCK
+    return err == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
+}
+
+// The fused block on int4 weights (activations and caches bf16).
+halo_status halo::launch_mha_block_i4(const halo_mha_shape& sh, const void* Qp, const void* Sp, const void* Qk, const void* Sk,
+                                      const void* Qv, const void* Sv, const void* x, void* Kc, void* Vc, int pos,
+                                      const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group, int n_dev,
+                                      float* partials, uint32_t* dev_status, cudaStream_t st, bool already_zero) {
+    using T = __nv_bfloat16;
+    const int d = sh.d_model, H = sh.n_heads, dh = sh.head_dim;
+    if (!already_zero && launch_zero_partials(partials, static_cast<size_t>(n_dev + 1) * d, st) != HALO_OK) return HALO_ERR_CUDA;
+    const int iters = (d / 16 + 255) / 256;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(kMhaCluster, H);
+    cfg.blockDim = dim3(256);
+    const size_t kv_b = kv_smem_bytes(pos, dh, sizeof(T));
+    cfg.dynamicSmemBytes = sizeof(float) * d + kv_b;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = already_zero ? 0 : 1;
+    const T* Wp_t = static_cast<const T*>(Qp); const T* x_t = static_cast<const T*>(x);
+    const T* Kc_t = static_cast<const T*>(Kc); const T* Vc_t = static_cast<const T*>(Vc);
+    const T* Wk_t = static_cast<const T*>(Qk); const T* Wv_t = static_cast<const T*>(Qv);
+    T* Kw_t = static_cast<T*>(Kc); T* Vw_t = static_cast<T*>(Vc);
+    const T* Sp_t = static_cast<const T*>(Sp); const T* Sk_t = static_cast<const T*>(Sk); const T* Sv_t = static_cast<const T*>(Sv);
+    const int Lmax = sh.max_len, kv_flag = kv_b ? 1 : 0;
+    cudaError_t err = cudaSuccess;
+#define HALO_MHA_BLOCK_I4(I)                                                                                         \
+    case I: {                                                                                                        \
+        static bool once[64] = {};                                                                                   \
+        if (!ensure_dynamic_smem(mha_fused_kernel<T, I, true, true>, kMhaSmemLimit, once)) return HALO_ERR_CUDA;      \
+        err = cudaLaunchKernelEx(&cfg, mha_fused_kernel<T, I, true, true>, d, H, dh, Lmax, pos, Wp_t, x_t, Kc_t, Vc_t, \
+                                 keep_list, n_keep, dev_of_group, n_dev, partials, dev_status, Wk_t, Wv_t, Kw_t, Vw_t, \
+                                 kv_flag, Sp_t, Sk_t, Sv_t);                                                          \
+        break;                                                                                                       \
+    }
+    switch (iters) {
+        HALO_MHA_BLOCK_I4(1)
+        HALO_MHA_BLOCK_I4(2)
+        default: return HALO_ERR_SHAPE;
+    }
+#undef HALO_MHA_BLOCK_I4
     return err == cudaSuccess ? HALO_OK : HALO_ERR_CUDA;
 }
 
@@ -852,4 +985,24 @@ extern "C" halo_status halo_mha_block(const halo_mha_shape* shape, const void* W
         return HALO_ERR_ALIGN;
     return halo::launch_mha_block(*shape, W_packed, Wk, Wv, x, K_cache, V_cache, pos, keep_list, n_keep, dev_of_group, n_dev,
                                   partials, dev_status, static_cast<cudaStream_t>(stream), false);
+}
+
+extern "C" halo_status halo_mha_block_i4(const halo_mha_shape* shape, const void* Qp, const void* Sp, const void* Qk,
+                                         const void* Sk, const void* Qv, const void* Sv, const void* x, void* K_cache,
+                                         void* V_cache, int pos, const int32_t* keep_list, const int32_t* n_keep,
+                                         const int32_t* dev_of_group, int n_dev, float* partials, uint32_t* dev_status,
+                                         void* stream) {
+    halo_status rc = check_mha_shape(shape);
+    if (rc != HALO_OK) return rc;
+    if (!Qp || !Sp || !Qk || !Sk || !Qv || !Sv || !x || !K_cache || !V_cache || !keep_list || !n_keep || !partials)
+        return HALO_ERR_ARG;
+    if (pos < 0 || pos >= shape->max_len) return HALO_ERR_ARG;
+    if (n_dev < 0 || n_dev > HALO_MAX_DEVICES || (!dev_of_group && n_dev != 0)) return HALO_ERR_ARG;
+    if (shape->wdtype != HALO_BF16) return HALO_ERR_DTYPE;                 // activations and caches
+    if (shape->head_dim % (2 * kMhaCluster) != 0 || shape->d_model % 128 != 0) return HALO_ERR_SHAPE;
+    if (!aligned16(Qp) || !aligned16(Sp) || !aligned16(Qk) || !aligned16(Sk) || !aligned16(Qv) || !aligned16(Sv) ||
+        !aligned16(x) || !aligned16(K_cache) || !aligned16(V_cache) || !aligned16(partials))
+        return HALO_ERR_ALIGN;
+    return halo::launch_mha_block_i4(*shape, Qp, Sp, Qk, Sk, Qv, Sv, x, K_cache, V_cache, pos, keep_list, n_keep, dev_of_group,
+                                     n_dev, partials, dev_status, static_cast<cudaStream_t>(stream), false);
 }

@@ -52,7 +52,7 @@ def run(wl, stack, H, vocab, steps, pos0, step0):
                  keep_list=mk((steps, L, Gx), torch.int32), n_keep=mk((steps, L), torch.int32),
                  y=mk((steps, L, 1, d), torch.float32))
         return t, B.Taps(*[t[k].data_ptr() for k in ("x", "scores", "dev_of_group", "arrived", "keep_list", "n_keep", "y")])
-    ta, Ta = taps(H, stack._keep[3].n_dev)
+    ta, Ta = taps(H, stack.plan_mha.n_dev)
     tf, Tf = taps(G, nf)
     bt = B.BlockTaps(Ta, Tf)
     logits = mk((steps, vocab), torch.float32) if vocab else None
@@ -168,3 +168,118 @@ def test_block_stack_argument_checks():
         stack.decode(h0, 1, 8, 0)                        # position beyond the cache
     with pytest.raises(B.HaloError):
         stack.decode(h0, 1, 0, 0, logits=torch.zeros((1, 10), dtype=torch.float32, device=DEV))   # no LM head given
+
+
+def _qrows(W2d):
+    rows, d = W2d.shape
+    Q = torch.empty((rows, d // 2), dtype=torch.uint8, device=DEV)
+    S = torch.empty((rows, d // 128), dtype=torch.bfloat16, device=DEV)
+    B.halo_quantize_rows_i4(d, rows, B.BF16, W2d, Q, S)
+    torch.cuda.synchronize()
+    return Q, S
+
+
+@pytest.mark.parametrize("name,layers,H,dh,steps,pos0", [("tinyllama-1.1b-decode", 3, 32, 64, 3, 37),
+                                                         ("llama2-7b-decode", 2, 32, 128, 2, 500)])
+def test_block_stack_on_int4_weights_teacher_forced(name, layers, H, dh, steps, pos0):
+    """halo_block_stack_create_i4: every weight matrix of the stack as int4 codes + scales (the paper's models are
+    4-bit), activations, caches and predictors bf16.  Teacher-forced per block against the oracle's functions on the
+    dequantised weights through the recorded taps; logits against the oracle's int4 LM head."""
+    wl = synth.small_variant(synth.workload(name), layers, steps)
+    vocab, lm_group, r_mha, max_len = 1000, 256, 64, pos0 + steps + 3
+    L, G, d, nf, na = wl.n_layers, wl.n_groups, wl.d_model, wl.n_dev, 3
+    tol = U.TOL_BF16
+    pm = dict(loss_rate=(0.0, 0.3, 0.6), share_weight=(2, 1, 1), k=max(1, H // 4), seed=11)
+    mh = B.mha_shape(d, H, dh, max_len, B.BF16)
+    fsh = B.ffn_shape(d, wl.d_ffn, wl.group_size, B.BF16)
+    hb = synth.host_bits
+    blocks, host = [], []
+    g = torch.Generator(device=DEV).manual_seed(5)
+    for l in range(L):
+        Wq, Wk, Wv, Wo = synth.mha_matrices(wl, l, H, DEV)
+        Wp = torch.empty((H, 2, dh, d), dtype=torch.bfloat16, device=DEV)
+        B.halo_pack_mha_weights(mh, Wq, Wo, Wp)
+        Wf = synth.packed_layer(wl, l, DEV)
+        Qf = torch.empty((G, 3, wl.group_size, d // 2), dtype=torch.uint8, device=DEV)
+        Sf = torch.empty((G, 3, wl.group_size, d // 128), dtype=torch.bfloat16, device=DEV)
+        B.halo_quantize_weights_i4(fsh, Wf, Qf, Sf)
+        Qp, Sp = _qrows(Wp.view(H * 2 * dh, d))
+        Qk, Sk = _qrows(Wk)
+        Qv, Sv = _qrows(Wv)
+        K = torch.zeros((H, max_len, dh), dtype=torch.bfloat16, device=DEV)
+        V = torch.zeros((H, max_len, dh), dtype=torch.bfloat16, device=DEV)
+        K[:, :pos0] = torch.randn((H, pos0, dh), generator=g, device=DEV).to(torch.bfloat16)
+        V[:, :pos0] = torch.randn((H, pos0, dh), generator=g, device=DEV).to(torch.bfloat16)
+        blk = dict(W_ffn=Qf, S_ffn=Sf, W_mha=Qp, S_mha=Sp, Wk=Qk, Sk=Sk, Wv=Qv, Sv=Sv, K=K, V=V)
+        if l > 0:
+            blk["W1_ffn"], blk["W2_ffn"] = synth.predictor(wl, l, DEV)
+            mw = synth.Workload("m", L, d, H * 8, 8, r_mha, wl.dtype, (), (), 500, 1, seed=wl.seed + 1)
+            blk["W1_mha"], blk["W2_mha"] = synth.predictor(mw, l, DEV)
+        blocks.append(blk)
+        host.append({k: (v.cpu().numpy() if v.dtype == torch.uint8 else hb(v)) for k, v in blk.items() if k not in ("K", "V")})
+        del Wf, Wp, Wq, Wk, Wv, Wo
+    gl = torch.Generator(device="cpu").manual_seed(17)
+    W_lm = (torch.randn((vocab, d), generator=gl) / 8).to(torch.bfloat16).to(DEV)
+    Q_lm, S_lm = _qrows(W_lm)
+    plan_f = B.Plan(G, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
+    plan_a = B.Plan(H, pm["loss_rate"], pm["share_weight"], B.SEL_TOPK, pm["k"], 0.0, pm["seed"])
+    stack = B.BlockStack(fsh, mh, B.lm_shape(d, vocab, lm_group, B.BF16), B.pred_shape(d, wl.pred_rank, G, B.BF16),
+                         B.pred_shape(d, r_mha, H, B.BF16), plan_f, plan_a, blocks, Q_lm, S_lm)
+    K_start = [hb(b["K"]) for b in blocks]
+    V_start = [hb(b["V"]) for b in blocks]
+    step0 = 3
+    h0, h_out, logits, ta, tf = run(wl, stack, H, vocab, steps, pos0, step0)
+    Kc, Vc = [k.copy() for k in K_start], [v.copy() for v in V_start]
+    lost_a = lost_f = 0
+    for s in range(steps):
+        pos = pos0 + s
+        h = h0[s].cpu().numpy().astype(np.float64).reshape(1, d)
+        xa_all, xf_all = hb(ta["x"]), hb(tf["x"])
+        for l in range(L):
+            b, hw = blocks[l], host[l]
+            x_a, x_f = xa_all[s, l], xf_all[s, l]
+            K32, V32 = R.to_f64(Kc[l]).astype(np.float32), R.to_f64(Vc[l]).astype(np.float32)
+            R.mha_kv_append_i4(hw["Wk"], hw["Sk"], hw["Wv"], hw["Sv"], x_a[0], pos, K32, V32)
+            Kg, Vg = hb(b["K"][:, pos]), hb(b["V"][:, pos])
+            kk = K32[:, pos].astype(np.float64)
+            assert np.abs(R.to_f64(Kg) - kk).max() <= 2 ** -7 * np.abs(kk).max()
+            assert np.abs(R.to_f64(Vg) - V32[:, pos]).max() <= 2 ** -7 * np.abs(kk).max()
+            Kc[l][:, pos], Vc[l][:, pos] = Kg, Vg          # teacher forcing: go on from the GPU's own cache bytes
+            sa = ta["scores"][s, l].cpu().numpy()
+            if l > 0:
+                ref = R.predict(hw["W1_mha"], hw["W2_mha"], xa_all[s, l - 1])
+                assert U.rel_err(sa, ref.astype(np.float64)) <= tol
+            sel = R.select(sa, pm["loss_rate"], pm["share_weight"], R.SEL_TOPK, pm["k"], 0.0, pm["seed"], step0 + s, 2 * l,
+                           force_all=(l == 0))
+            nk = int(ta["n_keep"][s, l].item())
+            assert nk == sel["n_keep"] and (ta["keep_list"][s, l].cpu().numpy() == sel["keep_list"]).all()
+            assert (ta["arrived"][s, l, :na].cpu().numpy() == sel["arrived"]).all()
+            lost_a += int(nk < H)
+            P = R.group_mha_i4(hw["W_mha"], hw["S_mha"], H, x_a[0], Kc[l], Vc[l], pos, sel["keep_list"][:nk],
+                               sel["dev_of_group"], na)
+            y = ta["y"][s, l, 0].cpu().numpy()
+            assert U.rel_err(y, P.sum(0)) <= tol, ("mha", s, l)
+            h, x_next = R.glue(h, y.astype(np.float64).reshape(1, d), B.BF16)
+            assert np.abs(R.to_f64(x_next) - R.to_f64(x_f)).max() <= 2 ** -7 * np.abs(R.to_f64(x_next)).max()
+            sf = tf["scores"][s, l].cpu().numpy()
+            if l > 0:
+                ref = R.predict(hw["W1_ffn"], hw["W2_ffn"], xf_all[s, l - 1])
+                assert U.rel_err(sf, ref.astype(np.float64)) <= tol
+            sel = R.select(sf, wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0, wl.seed, step0 + s, 2 * l + 1,
+                           force_all=(l == 0))
+            nk = int(tf["n_keep"][s, l].item())
+            assert nk == sel["n_keep"] and (tf["keep_list"][s, l].cpu().numpy() == sel["keep_list"]).all()
+            lost_f += int(nk < G)
+            y_ref = R.merge(R.group_ffn_i4(hw["W_ffn"], hw["S_ffn"], x_f, sel["keep_list"][:nk], sel["dev_of_group"], nf))
+            y = tf["y"][s, l].cpu().numpy()
+            assert U.rel_err(y, y_ref) <= tol, ("ffn", s, l)
+            h, x_next = R.glue(h, y.astype(np.float64), B.BF16)
+            if l + 1 < L:
+                xr, xg = R.to_f64(x_next), R.to_f64(xa_all[s, l + 1])
+                assert np.abs(xr - xg).max() <= 2 ** -7 * np.abs(xr).max()
+        assert np.abs(h_out[s].cpu().numpy() - h[0]).max() <= 1e-4 * np.abs(h).max()
+        _, x_o = R.glue(h_out[s].cpu().numpy().astype(np.float64).reshape(1, d), None, B.BF16)
+        ref = R.group_lm_head_i4(Q_lm.cpu().numpy(), hb(S_lm), x_o, lm_group)
+        got = logits[s].cpu().numpy()
+        assert np.abs(got - ref[0]).max() <= tol * np.sqrt(np.mean(ref ** 2)) + 2 ** -6 * np.abs(ref).max()
+    assert lost_a > 0 and lost_f > 0

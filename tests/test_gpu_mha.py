@@ -174,3 +174,59 @@ def test_mha_block_one_launch_matches_oracle_and_the_two_calls(dtype, d, H, dh, 
             rms = np.sqrt(np.mean(ref.sum(0) ** 2))
             assert np.abs(P.cpu().numpy() - ref).max() <= tol * rms, (pos, len(keep))
             assert np.abs(P2.cpu().numpy() - ref).max() <= tol * rms
+
+
+def _quant_rows(W):
+    rows, d = W.shape
+    Q = torch.empty((rows, d // 2), dtype=torch.uint8, device=DEV)
+    S = torch.empty((rows, d // 128), dtype=torch.bfloat16, device=DEV)
+    B.halo_quantize_rows_i4(d, rows, B.BF16, W, Q, S)
+    torch.cuda.synchronize()
+    return Q, S
+
+
+@pytest.mark.parametrize("d,H,dh,L,positions", [(512, 8, 64, 300, (0, 128, 299)), (4096, 32, 128, 1100, (3, 1023, 1099)),
+                                                (2048, 32, 64, 600, (511,)), (8192, 4, 128, 64, (40,)), (128, 3, 16, 20, (0, 19))])
+def test_mha_block_on_int4_weights_matches_the_oracle(d, H, dh, L, positions):
+    """halo_mha_block_i4: the appended cache rows against the oracle's keys and values from the dequantised Wk / Wv
+    (one bf16 rounding apart), the partials against the oracle's attention on the dequantised packed weights from the
+    GPU's cache bytes; heads that are not kept must still append, an empty kept set leaves zeros."""
+    wl = _wl("bf16", d)
+    sh = B.mha_shape(d, H, dh, L, B.BF16)
+    Wq, Wk, Wv, Wo = synth.mha_matrices(wl, 2, H, DEV)
+    Wp = torch.empty((H, 2, dh, d), dtype=torch.bfloat16, device=DEV)
+    B.halo_pack_mha_weights(sh, Wq, Wo, Wp)
+    Qp, Sp = _quant_rows(Wp.view(H * 2 * dh, d))
+    Qk, Sk = _quant_rows(Wk)
+    Qv, Sv = _quant_rows(Wv)
+    hb = synth.host_bits
+    Qp_h, Sp_h, Qk_h, Sk_h, Qv_h, Sv_h = Qp.cpu().numpy(), hb(Sp), Qk.cpu().numpy(), hb(Sk), Qv.cpu().numpy(), hb(Sv)
+    ref_q = R.quantize_i4(hb(Wk))
+    assert (Qk_h == ref_q[0]).all() and (Sk_h == ref_q[1]).all()
+    K, V = _caches(wl, H, L, dh, L)
+    dev = np.array([(-1, 0, 1, 2)[h % 4] for h in range(H)], dtype=np.int32)
+    dg = torch.as_tensor(dev, device=DEV)
+    for pos in positions:
+        for keep in (list(range(H)), [h for h in range(H) if h % 3 != 1], [H - 1], []):
+            x = synth.activation(wl, 190 + pos + len(keep), DEV)
+            kl = torch.full((H,), -1, dtype=torch.int32, device=DEV)
+            if keep:
+                kl[: len(keep)] = torch.as_tensor(keep, dtype=torch.int32, device=DEV)
+            nk = torch.tensor([len(keep)], dtype=torch.int32, device=DEV)
+            P = torch.full((4, d), float("nan"), dtype=torch.float32, device=DEV)
+            status = torch.zeros(1, dtype=torch.int32, device=DEV)
+            B.halo_mha_block_i4(sh, Qp, Sp, Qk, Sk, Qv, Sv, x, K, V, pos, kl, nk, dg, 3, P, status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            Kh, Vh = hb(K), hb(V)
+            K32, V32 = R.to_f64(Kh).astype(np.float32), R.to_f64(Vh).astype(np.float32)
+            R.mha_kv_append_i4(Qk_h, Sk_h, Qv_h, Sv_h, hb(x)[0], pos, K32, V32)      # overwrites row `pos`, unrounded
+            kk = K32[:, pos].astype(np.float64)
+            assert np.abs(R.to_f64(Kh[:, pos]) - kk).max() <= 2 ** -7 * np.abs(kk).max()
+            assert np.abs(R.to_f64(Vh[:, pos]) - V32[:, pos]).max() <= 2 ** -7 * np.abs(V32[:, pos]).max()
+            if not keep:
+                assert (P == 0).all().item()
+                continue
+            ref = R.group_mha_i4(Qp_h, Sp_h, H, hb(x)[0], Kh, Vh, pos, keep, dev, 3)
+            rms = np.sqrt(np.mean(ref.sum(0) ** 2))
+            assert np.abs(P.cpu().numpy() - ref).max() <= U.TOL_BF16 * rms, (pos, len(keep))

@@ -970,7 +970,36 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                     }
                 }
             } else {
-            if (any || P.deterministic) stage_sums();
+                if (REP > 1 && !P.deterministic) {
+                    // the replicas' sums meet in the first vector buffer in turn, so one bulk reduction leaves the thread block
+                    if (any) {
+                        float* dst = reinterpret_cast<float*>(vec_buf);
+                        for (int rr = 0; rr < REP; ++rr) {
+                            if (rep == rr) {
+#pragma unroll
+                                for (int p = 0; p < P2; ++p) {
+                                    const int c = col0 + kPC * p;
+                                    if (c < chunks) {
+                                        float4 a = make_float4(acc[p][0], acc[p][1], acc[p][2], acc[p][3]);
+                                        float4 b = make_float4(acc[p][4], acc[p][5], acc[p][6], acc[p][7]);
+                                        if (rr > 0) {
+                                            const float4 u = reinterpret_cast<const float4*>(dst + c * 8)[0];
+                                            const float4 v = reinterpret_cast<const float4*>(dst + c * 8)[1];
+                                            a.x += u.x; a.y += u.y; a.z += u.z; a.w += u.w;
+                                            b.x += v.x; b.y += v.y; b.z += v.z; b.w += v.w;
+                                        }
+                                        reinterpret_cast<float4*>(dst + c * 8)[0] = a;
+                                        reinterpret_cast<float4*>(dst + c * 8)[1] = b;
+                                    }
+                                }
+                                fence_proxy_async_smem();
+                            }
+                            if (rr + 1 < REP) pc_barrier();
+                        }
+                    }
+                } else if (any || P.deterministic) {
+                    stage_sums();
+                }
             }
             pc_barrier();
             if (P.deterministic) {
@@ -1001,9 +1030,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
             if (tid == 0) {
                 if (any && !P.deterministic) {
                     float* dst = P.partials + (q % 3u) * buf_stride + static_cast<size_t>(cta % kAccBufs) * acc_stride;
-#pragma unroll
-                    for (int k = 0; k < REP; ++k)
-                        bulk_reduce_add_f32_s2g(dst, vec_buf + static_cast<size_t>(k) * d * 4, static_cast<uint32_t>(d) * 4u);
+                    bulk_reduce_add_f32_s2g(dst, vec_buf, static_cast<uint32_t>(d) * 4u);   // (replicas already added up)
                     bulk_commit_and_wait_all();   // the sums are in global memory (and vec_buf is free again)
                     fence_proxy_async_all();
                 }

@@ -35,7 +35,7 @@ NOMINAL_HBM_GBS = 8000.0
 STACK_KERNEL_TRAFFIC_RATIO = 1.0007
 STACK_KERNEL_SOURCES = ("stack_persistent.cu", "stack_persistent.cuh", "ffn_math.cuh", "i4_math.cuh", "tma.cuh", "umma.cuh",
                         "select_device.cuh")
-STACK_KERNEL_SOURCES_SHA1 = "ed86f5839d047624aa461b171c8af53181582bc1"
+STACK_KERNEL_SOURCES_SHA1 = "894a086bae4c112767a568eeea9c682ef7ff8b4c"
 FALLBACK_HBM_GBS = 6650.0
 
 

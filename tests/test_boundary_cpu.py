@@ -99,6 +99,37 @@ def test_host_side_argument_checks_launch_nothing(lib):
     assert lib.halo_select_groups(None, None, 0, 0, 0, None, None, None, None, None, None, None, None) == -1
 
 
+def test_int4_entry_points_check_their_arguments_on_the_host(lib):
+    """The int4 calls reject NULL pointers, shapes outside the format (d_model % 128), misaligned arrays and other
+    element types before anything is launched."""
+    sh = B.ffn_shape(256, 688, 16, B.BF16)
+    assert lib.halo_quantize_rows_i4(256, 10, B.BF16, None, 16, 16, None) == -1
+    assert lib.halo_quantize_rows_i4(200, 10, B.BF16, 16, 16, 16, None) == -2          # not a multiple of 128
+    assert lib.halo_quantize_rows_i4(256, 0, B.BF16, 16, 16, 16, None) == -2
+    assert lib.halo_quantize_rows_i4(256, 10, 5, 16, 16, 16, None) == -4
+    assert lib.halo_quantize_rows_i4(256, 10, B.BF16, 16, 24, 16, None) == -3
+    assert lib.halo_dequantize_weights_i4(ctypes.byref(sh), None, 16, None, None, 16, None, None) == -1
+    assert lib.halo_dequantize_weights_i4(ctypes.byref(sh), 16, 16, 16, None, 16, None, None) == -1   # list without a count
+    assert lib.halo_dequantize_weights_i4(ctypes.byref(sh), 16, 16, None, None, 24, None, None) == -3
+    bad = B.ffn_shape(192, 688, 16, B.BF16)
+    assert lib.halo_dequantize_weights_i4(ctypes.byref(bad), 16, 16, None, None, 16, None, None) == -2
+    lm = B.lm_shape(256, 100, 16, B.BF16)
+    assert lib.halo_group_lm_head_i4(ctypes.byref(lm), 16, 16, 16, 1, None, None, 16, None, None) == -1   # no status word
+    assert lib.halo_group_lm_head_i4(ctypes.byref(lm), 16, 16, 16, 1, 16, None, 16, 16, None) == -1       # list without a count
+    assert lib.halo_group_lm_head_i4(ctypes.byref(B.lm_shape(200, 100, 16, B.BF16)), 16, 16, 16, 1, None, None, 16, 16, None) == -2
+    assert lib.halo_group_lm_head_i4(ctypes.byref(lm), 16, 24, 16, 1, None, None, 16, 16, None) == -3
+    mh = B.mha_shape(256, 4, 32, 64, B.BF16)
+    ptrs = [16] * 9
+    assert lib.halo_mha_block_i4(ctypes.byref(mh), None, *ptrs[1:], 0, 16, 16, None, 0, 16, None, None) == -1
+    assert lib.halo_mha_block_i4(ctypes.byref(mh), *ptrs, 64, 16, 16, None, 0, 16, None, None) == -1       # pos beyond the cache
+    assert lib.halo_mha_block_i4(ctypes.byref(B.mha_shape(256, 4, 32, 64, B.F32)), *ptrs, 0, 16, 16, None, 0, 16, None, None) == -4
+    assert lib.halo_mha_block_i4(ctypes.byref(B.mha_shape(192, 4, 32, 64, B.BF16)), *ptrs, 0, 16, 16, None, 0, 16, None, None) == -2
+    assert lib.halo_mha_block_i4(ctypes.byref(mh), 16, 24, *ptrs[2:], 0, 16, 16, None, 0, 16, None, None) == -3
+    out = ctypes.c_void_p()
+    assert lib.halo_block_stack_create_i4(ctypes.byref(out), ctypes.byref(sh), ctypes.byref(mh), None, None, None, 1, None,
+                                          None, None, None) == -1
+
+
 def test_schedulers_match_oracle_and_feed_the_plan(lib):
     rng = np.random.default_rng(3)
     for _ in range(200):

@@ -297,10 +297,9 @@ extern "C" halo_status halo_block_stack_decode(halo_block_stack* s, const float*
                 launches += 2;
             }
             if (s->i4) {
-                // (the entry point zeroes the slots itself: one small launch that the streaming kernel overlaps)
-                BS_TRY(halo_group_ffn_i4(&s->ffn, s->W_ffn[l], s->S_ffn[l], xf, 1, s->kl_f[cur], s->nk_f[cur], s->dev_f[cur],
-                                         s->n_dev_f, s->part_f, s->status, stream));
-                launches += 2;
+                BS_TRY(launch_group_ffn_i4(s->ffn, s->W_ffn[l], s->S_ffn[l], xf, 1, s->kl_f[cur], s->nk_f[cur], s->dev_f[cur],
+                                           s->n_dev_f, s->part_f, s->status, st, true));
+                ++launches;
             } else {
                 BS_TRY(launch_group_ffn_decode(s->ffn, s->W_ffn[l], xf, 1, s->kl_f[cur], s->nk_f[cur], s->dev_f[cur], s->n_dev_f,
                                                s->part_f, s->status, st, true));

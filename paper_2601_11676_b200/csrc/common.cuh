@@ -157,6 +157,10 @@ halo_status launch_mha_block(const halo_mha_shape& sh, const void* W_packed, con
 // int4 codes + scales of the kept groups (all groups when keep_list is null) -> bf16 rows in the packed layout
 halo_status launch_dequantize_i4(const halo_ffn_shape& sh, const void* Q, const void* scales, const int32_t* keep_list,
                                  const int32_t* n_keep, void* W_out, uint32_t* dev_status, cudaStream_t st);
+// halo_group_ffn_i4 without argument checks; already_zero: the caller guarantees that `partials` is zero
+halo_status launch_group_ffn_i4(const halo_ffn_shape& sh, const void* Q, const void* scales, const void* x, int n_tok,
+                                const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group, int n_dev,
+                                float* partials, uint32_t* dev_status, cudaStream_t st, bool already_zero);
 // the same block on int4 weights: Qp/Sp, Qk/Sk, Qv/Sv = codes and scales of W_packed, Wk, Wv (halo_quantize_rows_i4)
 halo_status launch_mha_block_i4(const halo_mha_shape& sh, const void* Qp, const void* Sp, const void* Qk, const void* Sk,
                                 const void* Qv, const void* Sv, const void* x, void* K_cache, void* V_cache, int pos,

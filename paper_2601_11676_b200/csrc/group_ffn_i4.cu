@@ -984,12 +984,23 @@ extern "C" halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void
     if (!Q || !scales || !x || !keep_list || !n_keep || !partials || n_tok <= 0) return HALO_ERR_ARG;
     if (n_dev < 0 || n_dev > HALO_MAX_DEVICES || (!dev_of_group && n_dev != 0)) return HALO_ERR_ARG;
     if (!aligned16(Q) || !aligned16(scales) || !aligned16(x) || !aligned16(partials)) return HALO_ERR_ALIGN;
+    return launch_group_ffn_i4(*shape, Q, scales, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status,
+                               static_cast<cudaStream_t>(stream), false);
+}
+
+// already_zero: the caller guarantees that `partials` is zero (otherwise the call zeroes it first).  Without the
+// zero-fill in front of it the ring kernel is an ordinary launch: as a programmatic dependent it would start under
+// whatever precedes it in the stream, which may be the kernel that writes x.
+halo_status halo::launch_group_ffn_i4(const halo_ffn_shape& sh, const void* Q, const void* scales, const void* x, int n_tok,
+                                      const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
+                                      int n_dev, float* partials, uint32_t* dev_status, cudaStream_t st, bool already_zero) {
+    const halo_ffn_shape* shape = &sh;
     const int d = shape->d_model, S = shape->group_size, G = shape->d_ffn / S;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t bytes = sizeof(float) * static_cast<size_t>(n_dev + 1) * n_tok * d;
     const int form_early = option_value(OPT_I4_NO_RING);
     const bool ring_form = (d == 2048 || d == 4096) && S % kRingNB == 0 && form_early != 1 && form_early != 3;
-    if (ring_form) {
+    if (already_zero) {
+    } else if (ring_form) {
         if (launch_zero_partials(partials, bytes / sizeof(float), st) != HALO_OK) return HALO_ERR_CUDA;
     } else if (cudaMemsetAsync(partials, 0, bytes, st) != cudaSuccess) {
         return HALO_ERR_CUDA;
@@ -1043,7 +1054,7 @@ extern "C" halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void
         attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr.val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = &attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = already_zero ? 0 : 1;
         auto go = [&](auto k, bool (&once)[64]) {
             if (!ensure_dynamic_smem(k, smem_r, once)) return HALO_ERR_CUDA;
             return cudaLaunchKernelEx(&cfg, k, d, S, G, q, sc, xt, keep_list, n_keep, dev_of_group, n_dev, n_tok, partials,

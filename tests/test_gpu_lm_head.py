@@ -157,3 +157,21 @@ def test_lm_head_int4_full_vocabulary_at_7b_width():
     hb = synth.host_bits
     ref = R.group_lm_head_i4(Q.cpu().numpy(), hb(Sc), hb(x), 256)
     assert np.abs(got - ref).max() <= U.TOL_BF16 * np.sqrt(np.mean(ref ** 2))
+
+
+def test_lm_head_int4_streaming_form_flags_a_bad_group_index_and_ragged_groups():
+    """One token, d 4096: the shared-memory ring form of the int4 head; groups of 40 rows (a full batch of 32 and a
+    ragged one of 8), a short last group, a bad index in the list."""
+    g = torch.Generator().manual_seed(6)
+    vocab, d, S = 1013, 4096, 40
+    W = (torch.randn((vocab, d), generator=g) / 64.0).to(torch.bfloat16).to(DEV)
+    x = torch.randn((1, d), generator=g).to(torch.bfloat16).to(DEV)
+    Q, Sc = _quantize_rows(W, B.BF16)
+    n_groups = (vocab + S - 1) // S
+    keep = [0, 99, n_groups - 1, -1, 7, 3]
+    got, status = _run_i4(Q, Sc, x, vocab, S, keep)
+    assert status & B.DEV_BAD_INDEX
+    hb = synth.host_bits
+    ref = R.group_lm_head_i4(Q.cpu().numpy(), hb(Sc), hb(x), S, [0, n_groups - 1, 7, 3], fill=-123.0)
+    rms = np.sqrt(np.mean(R.group_lm_head_i4(Q.cpu().numpy(), hb(Sc), hb(x), S) ** 2))
+    assert np.abs(got - ref).max() <= U.TOL_BF16 * rms

@@ -337,8 +337,10 @@ halo_status halo_group_mha(const halo_mha_shape* shape, const void* W_packed, co
  * int4 group-quantised weights for the decode FFN (the paper evaluates models "quantized to 4-bit integer
  * precision", Sec. IV-A, and fixes the neuron-group size "for compatibility with quantization", Sec. II-A; it
  * gives no format).  Format used here: symmetric, one bf16 scale per block of 128 consecutive elements of a
- * packed row: s = bf16(amax / 7), q = clamp(rint(w / s), -8, 7) (fp32 division, round half to even; s == 0
- * gives q = 0), stored as nibble q + 8 with element 2i in the low half of byte i.  value = (nibble - 8) * s.
+ * packed row: s = bf16(amax / 7) rounded UP to the next bf16 number with at most 5 significant bits,
+ * q = clamp(rint(w / s), -8, 7) (fp32 division, round half to even; s == 0 gives q = 0), stored as nibble q + 8
+ * with element 2i in the low half of byte i.  value = (nibble - 8) * s, which has at most 8 significant bits: every
+ * dequantised value is exactly a bf16 number.
  *   shape: as for halo_group_ffn, with d_model % 128 == 0 and d_model <= 8192; wdtype = type of the SOURCE
  *     weights for halo_quantize_weights_i4, ignored by halo_group_ffn_i4.
  *   Q device uint8 [G][3][S][d/2]; scales device bf16 [G][3][S][d/128]; both 16-byte aligned, caller-owned.
@@ -347,7 +349,8 @@ halo_status halo_group_mha(const halo_mha_shape* shape, const void* W_packed, co
  *     fp32 [n_dev+1][n_tok][d], zeroed by the call; keep_list / n_keep / dev_of_group / dev_status as there.
  *     Decode form (one pass over the kept groups' weights per token); no workspace.
  *   halo_dequantize_weights_i4: Q, scales -> W_packed (device bf16, layout of halo_pack_weights, 16-byte aligned,
- *     caller-owned), every element bf16((nibble - 8) * s): one rounding of the exact value.  keep_list / n_keep
+ *     caller-owned), every element (nibble - 8) * s, exact for scales written by the quantisers of this library
+ *     (a scale with more than 5 significant bits is rounded once).  keep_list / n_keep
  *     (device, as for halo_group_ffn) name the groups to write, the others are left as they are; keep_list NULL
  *     writes all groups.  For prompts: the tensor cores take bf16 operands, so a prompt on int4 weights is this
  *     call followed by halo_group_ffn on its output (what an int4 stack created for more than one token does per

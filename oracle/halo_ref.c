@@ -627,11 +627,14 @@ int halo_ref_late_devices(int n_dev, const int32_t* units, const double* compute
  * precision" (Sec. IV-A) and picks the neuron-group size "for compatibility with quantization"
  * (Sec. II-A) but gives no format; the reading taken here: symmetric, one scale per block of 128
  * consecutive elements of a stored (packed) row,
- *   s = bf16(amax / 7)   (fp32 division, round-to-nearest-even to bf16; amax = max |w| of the block)
+ *   s = up5(bf16(amax / 7))   (fp32 division, round-to-nearest-even to bf16, then UP to the next bf16 number
+ *                              with at most 5 significant bits; amax = max |w| of the block)
  *   q = clamp(rint(w / s), -8, 7)   (fp32 division, round-half-even; s == 0 -> q = 0)
  * stored as nibble q + 8; element 2i in the low half of byte i, element 2i+1 in the high half.
  * The decisions are taken in fp32 on both sides (here and on the GPU), so codes and scales
- * compare bit for bit.  Dequantised value: (nibble - 8) * s, exact in fp32.
+ * compare bit for bit.  Dequantised value: (nibble - 8) * s.  With 5 significant bits in s and at most 3 (or a
+ * single one, for -8) in the code, the product has at most 8: every dequantised value is a bf16 number, so a
+ * bf16 operand path (tensor cores) carries the weights without any rounding.
  * ------------------------------------------------------------------------------------------- */
 #define REF_QBLOCK 128
 
@@ -657,6 +660,7 @@ int halo_ref_quantize_i4(int d, long long n_rows, int dtype, const void* W, uint
             }
             float s32 = amax / 7.0f;
             uint16_t sb = ref_double_to_bf16((double)s32);
+            if (sb & 7u) sb = (uint16_t)((sb | 7u) + 1u);        /* up to 5 significant bits (may carry into the exponent) */
             float s = ref_bf16_bits_to_float(sb);
             scales[(size_t)r * nb + b] = sb;
             for (int e = 0; e < REF_QBLOCK; e += 2) {
@@ -682,7 +686,7 @@ int halo_ref_dequantize_i4(int d, long long n_rows, const uint8_t* Q, const uint
             size_t i = (size_t)r * d + c;
             int nib = (Q[i / 2] >> ((c & 1) * 4)) & 15;
             float s = ref_bf16_bits_to_float(scales[(size_t)r * nb + c / REF_QBLOCK]);
-            W32[i] = (float)(nib - 8) * s;     /* at most 4 + 8 significant bits: exact */
+            W32[i] = (float)(nib - 8) * s;     /* at most 8 significant bits: exact, and a bf16 number */
         }
     return REF_OK;
 }

@@ -312,7 +312,8 @@ QBLOCK = 128
 
 def quantize_i4(W: np.ndarray):
     """Packed rows [..., d] (float32 or bf16 bits) -> (codes uint8 [..., d/2], scales bf16 bits [..., d/128]);
-    symmetric, s = bf16(amax/7), q = clamp(rint(w/s), -8, 7), nibble = q + 8, element 2i in the low half of byte i."""
+    symmetric, s = bf16(amax/7) rounded up to 5 significant bits, q = clamp(rint(w/s), -8, 7), nibble = q + 8, element
+    2i in the low half of byte i."""
     d = W.shape[-1]
     n_rows = int(np.prod(W.shape[:-1]))
     dt = _dtype_of(W)

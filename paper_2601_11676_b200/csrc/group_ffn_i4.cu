@@ -1,7 +1,8 @@
 // int4 group-quantised weights for the decode FFN (steps a6..a8 on 4-bit weights).  The paper evaluates models
 // quantised to 4-bit integers (Sec. IV-A) without giving a format; the one used here: symmetric, one bf16 scale
-// per block of 128 consecutive elements of a packed row, s = bf16(amax / 7), q = clamp(rint(w / s), -8, 7),
-// nibble = q + 8, element 2i in the low half of byte i.
+// per block of 128 consecutive elements of a packed row, s = bf16(amax / 7) rounded up to 5 significant bits,
+// q = clamp(rint(w / s), -8, 7), nibble = q + 8, element 2i in the low half of byte i.  With 5 bits in the scale every
+// dequantised value (nibble - 8) * s is exactly a bf16 number: the tensor-core prompt path loses nothing on the weights.
 //
 // halo_quantize_weights_i4: one warp per (row, block); decisions in fp32 with IEEE division and round-half-even.
 // halo_group_ffn_i4, generic form: the structure of the generic decode kernel (a thread block walks a contiguous range of kept
@@ -53,7 +54,14 @@ quantize_i4_kernel(int d, long long n_rows, const T* __restrict__ W, uint8_t* __
     float amax = fmaxf(fmaxf(fabsf(w[0]), fabsf(w[1])), fmaxf(fabsf(w[2]), fabsf(w[3])));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    const __nv_bfloat16 sb = __float2bfloat16_rn(__fdiv_rn(amax, 7.0f));
+    __nv_bfloat16 sb = __float2bfloat16_rn(__fdiv_rn(amax, 7.0f));
+    {
+        // up to the next bf16 number with at most 5 significant bits (the carry may reach the exponent): code * scale
+        // then has at most 8 significant bits, i.e. every dequantised value is itself a bf16 number
+        uint16_t bits = __bfloat16_as_ushort(sb);
+        if (bits & 7u) bits = static_cast<uint16_t>((bits | 7u) + 1u);
+        sb = __ushort_as_bfloat16(bits);
+    }
     const float s = __bfloat162float(sb);
     if (lane == 0) scales[static_cast<size_t>(row) * nb + b] = sb;
     uint32_t packed = 0;
@@ -68,11 +76,11 @@ quantize_i4_kernel(int d, long long n_rows, const T* __restrict__ W, uint8_t* __
 
 // Kept groups (or all of them) back to bf16 in the packed layout, for the tensor-core prompt path: a thread turns one
 // word of codes into 8 values = one 16-byte store, neighbouring lanes neighbouring words, so every store instruction
-// of a warp covers 512 contiguous bytes.  value = bf16((nibble - 8) * s) (the product has at most 12 significant bits,
-// so this is ONE rounding of the exact value).  No integer-to-float conversion: nibbles k and k+4 of the word become
-// the bf16 pair {128 + n_k, 128 + n_k+4} by mask and OR, 136 is subtracted (exact) and the pair is multiplied by the
-// scale in bf16x2 (one rounding); a byte permute puts neighbouring elements back side by side.  Groups outside the
-// kept set are not touched.
+// of a warp covers 512 contiguous bytes.  value = (nibble - 8) * s, EXACT in bf16 for scales of the quantiser above (5
+// significant bits; a foreign scale with more bits is rounded once).  No integer-to-float conversion: nibbles k and
+// k+4 of the word become the bf16 pair {128 + n_k, 128 + n_k+4} by mask and OR, 136 is subtracted (exact) and the pair
+// is multiplied by the scale in bf16x2; a byte permute puts neighbouring elements back side by side.  Groups outside
+// the kept set are not touched.
 __device__ __forceinline__ uint4 dequant_word(uint32_t word, __nv_bfloat16 scale) {
     const __nv_bfloat162 s2 = __halves2bfloat162(scale, scale);
     const uint32_t bias_bits = 0x43084308u;                       // {136, 136}

@@ -188,14 +188,17 @@ def test_int4_stack_teacher_forced(name, layers, steps, mode):
 
 
 @pytest.mark.parametrize("d,G,S", [(256, 5, 16), (4096, 6, 128), (1024, 7, 256)])
-def test_int4_dequantise_is_one_rounding_of_the_exact_value(d, G, S):
-    """halo_dequantize_weights_i4: every element equals the exact (nibble - 8) * s of the oracle, rounded once to bf16
-    (ties to even: the library cast); with a kept list only the named groups are written, a bad index is reported."""
+def test_int4_dequantise_is_exact(d, G, S):
+    """halo_dequantize_weights_i4: every element IS the oracle's (nibble - 8) * s (the format's scales have 5
+    significant bits, so the value is a bf16 number and the cast below loses nothing); with a kept list only the named
+    groups are written, a bad index is reported."""
     wl = synth.Workload("q", 1, d, G * S, S, 16, "bf16", (), (), 500, 1)
     Wp = synth.packed_layer(wl, 1, DEV)
     sh, Q, Sc = _quantize(wl, Wp)
     exact = R.dequantize_i4(Q.cpu().numpy(), synth.host_bits(Sc))                 # fp32, exact
-    want = synth.host_bits(torch.from_numpy(exact).to(torch.bfloat16))
+    as_bf16 = torch.from_numpy(exact).to(torch.bfloat16)
+    assert (as_bf16.to(torch.float32).numpy() == exact).all()
+    want = synth.host_bits(as_bf16)
     out = torch.full((G, 3, S, d), 7.0, dtype=torch.bfloat16, device=DEV)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     B.halo_dequantize_weights_i4(sh, Q, Sc, None, None, out, status)
@@ -235,13 +238,15 @@ def _int4_prompt_stack(wl):
     return stack, preds, ffn_ref
 
 
-@pytest.mark.parametrize("n_tok,d", [(5, 512), (64, 512), (300, 256)])
-def test_int4_stack_prompts(n_tok, d):
-    """An int4 stack made for prompts: five tokens go through the decode form token by token, 64 and 300 through the
-    tensor-core path on the kept groups turned back into bf16.  Teacher-forced against the oracle's FFN on the EXACT
-    dequantised weights through the records; then the run without the y records (down projection adding into the
-    residual stream) chained from the recorded inputs."""
-    wl = synth.Workload("pq", 3, d, 64 * 12, 64, 64, "bf16", (0.0, 0.3, 0.6), (2, 1, 1), 250, 2, n_tok=n_tok)
+@pytest.mark.parametrize("n_tok,d,loss", [(5, 512, (0.0, 0.3, 0.6)), (64, 512, (0.0, 0.3, 0.6)), (300, 256, (0.0, 0.3, 0.6)),
+                                          (160, 512, (0.85, 0.9, 0.95))])
+def test_int4_stack_prompts(n_tok, d, loss):
+    """An int4 stack made for prompts: five tokens go through the decode form token by token, 64, 160 and 300 through
+    the tensor-core path on the kept groups turned back into bf16 (exactly: the format's scales have 5 significant
+    bits); the last case has devices that mostly fail, so blocks run with a quarter of their groups.  Teacher-forced
+    against the oracle's FFN on the dequantised weights through the records; then the run without the y records (down
+    projection adding into the residual stream) chained from the recorded inputs."""
+    wl = synth.Workload("pq", 3, d, 64 * 12, 64, 64, "bf16", loss, (2, 1, 1), 250, 2, n_tok=n_tok)
     stack, preds, ffn_ref = _int4_prompt_stack(wl)
     h0, h_out, t = TS.run_with_taps(wl, stack, wl.steps)
     lost = TS.check_teacher_forced(wl, None, preds, h0, h_out, t, wl.steps, ffn_ref=ffn_ref)

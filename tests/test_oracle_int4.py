@@ -31,13 +31,21 @@ def test_zero_block_halfway_cases_and_scale_rounding():
     assert Sc[0, 1] == _bf16_bits([1.0])[0]
     deq = R.dequantize_i4(Q, Sc)[0, 128:136]
     assert deq.tolist() == [7.0, 2.0, 4.0, -2.0, 0.0, 0.0, -7.0, 6.0]
-    # a scale that is not a bf16 number: amax = 1 -> 1/7 = 0.142857.. -> bf16 0.142578125 (nearest of 0.1416, 0.1426)
+    # a scale that is not on the grid: amax = 1 -> 1/7 = 0.142857.. -> bf16 0.142578125 = 1.140625 * 2^-3 -> up to
+    # 5 significant bits (steps of 1/16 in the significand): 1.1875 * 2^-3 = 0.1484375
     W2 = np.zeros((1, 128), dtype=np.float32)
     W2[0, 0] = 1.0
     Q2, Sc2 = R.quantize_i4(W2)
     s = float(R.to_f64(Sc2)[0, 0])
-    assert s == 0.142578125
-    assert (Q2[0, 0] & 15) == 7 + 8                               # 1 / s = 7.01.. -> 7, no clipping trouble
+    assert s == 0.1484375
+    assert (Q2[0, 0] & 15) == 7 + 8                               # 1 / s = 6.74 -> 7, and never above 7
+    # a scale that already has 5 bits stays; the carry of the rounding may reach the exponent:
+    # amax = 7 * 1.96875 -> s = bf16(1.96875) = 1.96875 = 1.1111110b -> up: 2.0
+    for amax, want in ((7 * 1.5, 1.5), (7 * 1.96875, 2.0), (7 * 0.0625, 0.0625)):
+        W3 = np.zeros((1, 128), dtype=np.float32)
+        W3[0, 5] = -amax
+        _, Sc3 = R.quantize_i4(W3)
+        assert float(R.to_f64(Sc3)[0, 0]) == want
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
@@ -50,11 +58,17 @@ def test_error_bound_and_brute_force_python(dtype):
     w = R.to_f64(Wb).reshape(-1, 2, 128)
     s = R.to_f64(Sc).reshape(-1, 2, 1)
     deq = R.dequantize_i4(Q, Sc).astype(np.float64).reshape(-1, 2, 128)
-    # every value within half a step (plus the slack of the rounded scale at the block maximum)
+    # every value within half a step (the scale is never below amax / 7 by more than the bf16 rounding, so only
+    # that rounding can push the block maximum past 7.5 steps)
     assert (np.abs(w - deq) <= 0.5 * s * (1 + 2.0 ** -6)).all()
-    # the scale is amax / 7 to bf16 precision
+    # the scale: bf16(amax / 7) rounded UP to 5 significant bits, so within (-2^-8, +2^-4] of amax / 7 relatively,
+    # with the three low bits of its bf16 significand clear
     amax = np.abs(w).max(axis=2, keepdims=True)
-    assert (np.abs(s - amax / 7) <= amax / 7 * 2.0 ** -8).all()
+    assert (s >= amax / 7 * (1 - 2.0 ** -8)).all() and (s <= amax / 7 * (1 + 2.0 ** -8) * (1 + 2.0 ** -4)).all()
+    assert ((Sc.reshape(-1) & 7) == 0).all()
+    # hence every dequantised value is itself a bf16 number (what a bf16 tensor-core operand can carry exactly)
+    deq32 = R.dequantize_i4(Q, Sc)
+    assert (torch.from_numpy(deq32).to(torch.bfloat16).to(torch.float32).numpy() == deq32).all()
     # brute force in numpy float32 arithmetic, same decisions
     w32 = w.astype(np.float32)
     s32 = s.astype(np.float32)

@@ -368,6 +368,17 @@ halo_status halo_dequantize_weights_i4(const halo_ffn_shape* shape, const void* 
 halo_status halo_group_ffn_i4(const halo_ffn_shape* shape, const void* Q, const void* scales, const void* x, int n_tok,
                               const int32_t* keep_list, const int32_t* n_keep, const int32_t* dev_of_group,
                               int n_dev, float* partials, uint32_t* dev_status, void* stream);
+/* halo_group_ffn_i4 for prompts.  halo_group_ffn_i4_workspace_bytes is non-zero for token counts and shapes the
+ * tensor-core FFN takes (16 tokens or more, d_model % 128 == 0, group size 64 / 128 / 256): the call then writes the
+ * kept groups' dequantised weights (exact in bf16) into the caller's workspace and runs halo_group_ffn's tensor-core
+ * form on them; workspace device, 16-byte aligned, at least that many bytes (one bf16 block of 3 * d_ffn * d_model
+ * elements + halo_group_ffn's own workspace), else HALO_ERR_WORKSPACE.  Where the size is 0 the call is
+ * halo_group_ffn_i4 and the workspace is not used.  Results and every other argument as halo_group_ffn_i4. */
+size_t halo_group_ffn_i4_workspace_bytes(const halo_ffn_shape* shape, int n_tok);
+halo_status halo_group_ffn_i4_prompt(const halo_ffn_shape* shape, const void* Q, const void* scales, const void* x,
+                                     int n_tok, const int32_t* keep_list, const int32_t* n_keep,
+                                     const int32_t* dev_of_group, int n_dev, float* partials, void* workspace,
+                                     size_t workspace_bytes, uint32_t* dev_status, void* stream);
 
 /* ------------------------------------------------------------------------
  * LM-head neuron groups (Sec. II-A: the LM head "only contains up-projection" and is "also a collection of

@@ -34,7 +34,7 @@ EXPORTS = [
     "halo_layer_workspace_bytes", "halo_layer_fused", "halo_read_status",
     "halo_pack_mha_weights", "halo_mha_kv_append", "halo_group_mha_workspace_bytes", "halo_group_mha",
     "halo_group_lm_head", "halo_late_devices", "halo_quantize_weights_i4", "halo_group_ffn_i4", "halo_dequantize_weights_i4", "halo_quantize_rows_i4", "halo_group_lm_head_i4", "halo_mha_block_i4",
-    "halo_block_stack_create_i4",
+    "halo_block_stack_create_i4", "halo_group_ffn_i4_workspace_bytes", "halo_group_ffn_i4_prompt",
     "halo_set_option",
     "halo_block_stack_create", "halo_block_stack_destroy", "halo_block_stack_decode", "halo_block_stack_status",
     "halo_block_stack_last_launches", "halo_stack_create_i4", "halo_mha_block",
@@ -164,6 +164,10 @@ def lib() -> ctypes.CDLL:
         L.halo_quantize_rows_i4.argtypes = [c_int, c_longlong, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
         L.halo_group_lm_head_i4.argtypes = [POINTER(LmShape), c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
                                             c_void_p, c_void_p, c_void_p]
+        L.halo_group_ffn_i4_workspace_bytes.argtypes = [POINTER(FfnShape), c_int]
+        L.halo_group_ffn_i4_workspace_bytes.restype = c_size_t
+        L.halo_group_ffn_i4_prompt.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p,
+                                               c_void_p, c_int, c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
         L.halo_dequantize_weights_i4.argtypes = [POINTER(FfnShape), c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                                                  c_void_p, c_void_p]
         L.halo_selftest_bounded_wait.argtypes = [c_void_p, c_longlong, c_void_p, c_void_p, c_void_p]
@@ -397,6 +401,18 @@ def halo_quantize_rows_i4(d_model: int, n_rows: int, wdtype: int, W, Q, scales, 
 def halo_group_lm_head_i4(shape: LmShape, Q, scales, x, n_tok, keep_list, n_keep, logits, dev_status, stream=None) -> None:
     _chk(lib().halo_group_lm_head_i4(byref(shape), _ptr(Q), _ptr(scales), _ptr(x), n_tok, _ptr(keep_list), _ptr(n_keep),
                                      _ptr(logits), _ptr(dev_status), _stream(stream)), "halo_group_lm_head_i4")
+
+
+def halo_group_ffn_i4_workspace_bytes(shape: FfnShape, n_tok: int) -> int:
+    return int(lib().halo_group_ffn_i4_workspace_bytes(byref(shape), n_tok))
+
+
+def halo_group_ffn_i4_prompt(shape: FfnShape, Q, scales, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials,
+                             workspace, dev_status=None, stream=None) -> None:
+    _chk(lib().halo_group_ffn_i4_prompt(byref(shape), _ptr(Q), _ptr(scales), _ptr(x), n_tok, _ptr(keep_list), _ptr(n_keep),
+                                        _ptr(dev_of_group), n_dev, _ptr(partials), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                        _ptr(dev_status), _stream(stream)), "halo_group_ffn_i4_prompt")
 
 
 def halo_dequantize_weights_i4(shape: FfnShape, Q, scales, keep_list, n_keep, W_packed, dev_status=None,

@@ -354,6 +354,41 @@ extern "C" halo_status halo_group_ffn(const halo_ffn_shape* shape, const void* W
                               need > 0 ? workspace : nullptr, dev_status, static_cast<cudaStream_t>(stream));
 }
 
+// ---- int4 weights, many tokens: kept groups back to bf16 in the caller's workspace, then the tensor-core FFN ----
+
+extern "C" size_t halo_group_ffn_i4_workspace_bytes(const halo_ffn_shape* shape, int n_tok) {
+    if (!shape || n_tok <= 0) return 0;
+    halo_ffn_shape sh = *shape;
+    sh.wdtype = HALO_BF16;                                   // activations; the tensor cores' operand type
+    if (check_ffn_shape(&sh) != HALO_OK || sh.d_model % 128 != 0 || !prefill_supported(sh, n_tok)) return 0;
+    return align_up(static_cast<size_t>(sh.d_ffn) * 3 * sh.d_model * 2, 1024) + prefill_workspace_bytes(sh, n_tok);
+}
+
+extern "C" halo_status halo_group_ffn_i4_prompt(const halo_ffn_shape* shape, const void* Q, const void* scales, const void* x,
+                                                int n_tok, const int32_t* keep_list, const int32_t* n_keep,
+                                                const int32_t* dev_of_group, int n_dev, float* partials, void* workspace,
+                                                size_t workspace_bytes, uint32_t* dev_status, void* stream) {
+    if (!shape) return HALO_ERR_ARG;
+    const size_t need = halo_group_ffn_i4_workspace_bytes(shape, n_tok);
+    if (need == 0)    // few tokens or a shape the tensor-core FFN does not take: the decode form, token by token
+        return halo_group_ffn_i4(shape, Q, scales, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, dev_status,
+                                 stream);
+    if (!Q || !scales || !x || !keep_list || !n_keep || !partials) return HALO_ERR_ARG;
+    if (n_dev < 0 || n_dev > HALO_MAX_DEVICES || (!dev_of_group && n_dev != 0)) return HALO_ERR_ARG;
+    if (!workspace || workspace_bytes < need) return HALO_ERR_WORKSPACE;
+    if (!aligned16(Q) || !aligned16(scales) || !aligned16(x) || !aligned16(partials) || !aligned16(workspace))
+        return HALO_ERR_ALIGN;
+    halo_ffn_shape sh = *shape;
+    sh.wdtype = HALO_BF16;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    const size_t block_bytes = align_up(static_cast<size_t>(sh.d_ffn) * 3 * sh.d_model * 2, 1024);
+    halo_status rc = launch_dequantize_i4(sh, Q, scales, keep_list, n_keep, ws, dev_status, st);
+    if (rc != HALO_OK) return rc;
+    return dispatch_group_ffn(sh, ws, x, n_tok, keep_list, n_keep, dev_of_group, n_dev, partials, ws + block_bytes,
+                              dev_status, st);
+}
+
 // ---- a9 and helpers -----------------------------------------------------------------------------------
 
 extern "C" halo_status halo_merge_partials(const float* partials, const uint8_t* arrived, int n_dev, int n_tok,

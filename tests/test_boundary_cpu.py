@@ -125,6 +125,15 @@ def test_int4_entry_points_check_their_arguments_on_the_host(lib):
     assert lib.halo_mha_block_i4(ctypes.byref(B.mha_shape(256, 4, 32, 64, B.F32)), *ptrs, 0, 16, 16, None, 0, 16, None, None) == -4
     assert lib.halo_mha_block_i4(ctypes.byref(B.mha_shape(192, 4, 32, 64, B.BF16)), *ptrs, 0, 16, 16, None, 0, 16, None, None) == -2
     assert lib.halo_mha_block_i4(ctypes.byref(mh), 16, 24, *ptrs[2:], 0, 16, 16, None, 0, 16, None, None) == -3
+    big = B.ffn_shape(512, 1024, 128, B.BF16)
+    assert B.halo_group_ffn_i4_workspace_bytes(big, 8) == 0                      # too few tokens for the tensor cores
+    need = B.halo_group_ffn_i4_workspace_bytes(big, 64)
+    assert need >= 3 * 1024 * 512 * 2                                             # one bf16 block + the FFN's own
+    assert B.halo_group_ffn_i4_workspace_bytes(B.ffn_shape(512, 1024, 32, B.BF16), 64) == 0   # group size not taken
+    assert lib.halo_group_ffn_i4_prompt(ctypes.byref(big), 16, 16, 16, 64, 16, 16, None, 0, 16, None, 0, None, None) == -8
+    assert lib.halo_group_ffn_i4_prompt(ctypes.byref(big), 16, 16, 16, 64, 16, 16, None, 0, 16, 16, need - 1, None, None) == -8
+    assert lib.halo_group_ffn_i4_prompt(ctypes.byref(big), None, 16, 16, 64, 16, 16, None, 0, 16, 16, need, None, None) == -1
+    assert lib.halo_group_ffn_i4_prompt(ctypes.byref(big), 16, 16, 16, 64, 16, 16, None, 0, 16, 24, need, None, None) == -3
     out = ctypes.c_void_p()
     assert lib.halo_block_stack_create_i4(ctypes.byref(out), ctypes.byref(sh), ctypes.byref(mh), None, None, None, 1, None,
                                           None, None, None) == -1

@@ -268,3 +268,74 @@ def test_int4_prompt_stack_at_the_benchmarked_shape():
     assert lost > 0
     plain, t2 = TS.run_without_y(wl, stack, h0, wl.steps, step0=5)
     assert TS.check_chained_without_y(wl, None, preds, h0, plain, t2, wl.steps, 5, tokens, ffn_ref=ffn_ref) == lost
+
+
+def _run_prompt(sh, Q, Sc, x, keep, dev, n_dev, G):
+    n_tok, d = x.shape
+    kl = torch.full((G,), -1, dtype=torch.int32, device=DEV)
+    if len(keep):
+        kl[: len(keep)] = torch.as_tensor(np.asarray(keep, dtype=np.int32), device=DEV)
+    nk = torch.tensor([len(keep)], dtype=torch.int32, device=DEV)
+    dg = None if dev is None else torch.as_tensor(np.asarray(dev, dtype=np.int32), device=DEV)
+    P = torch.full((n_dev + 1, n_tok, d), float("nan"), dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    need = B.halo_group_ffn_i4_workspace_bytes(sh, n_tok)
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device=DEV)
+    B.halo_group_ffn_i4_prompt(sh, Q, Sc, x, n_tok, kl, nk, dg, n_dev, P, ws, status)
+    torch.cuda.synchronize()
+    return P.cpu().numpy(), int(status.item()), need
+
+
+@pytest.mark.parametrize("d,G,S,n_tok", [(256, 12, 64, 40), (512, 9, 128, 300), (1024, 5, 256, 130), (512, 7, 64, 3),
+                                         (384, 6, 24, 20)])
+def test_int4_prompt_entry_point_matches_the_oracle(d, G, S, n_tok):
+    """halo_group_ffn_i4_prompt: with a workspace the kept groups go through the tensor cores (their dequantised values
+    are exact in bf16), without one (few tokens, a group size the tensor-core form does not take) through the decode
+    form; per-holder slots against the oracle's FFN on the dequantised weights, every token."""
+    wl = synth.Workload("q", 1, d, G * S, S, 16, "bf16", (0.0, 0.3, 0.6), (1, 1, 1), 500, 1)
+    Wp = synth.packed_layer(wl, 0, DEV)
+    sh, Q, Sc = _quantize(wl, Wp)
+    hb = synth.host_bits
+    Qh, Sh = Q.cpu().numpy(), hb(Sc)
+    x = synth.activation(wl, 4, DEV, n_tok=n_tok)
+    dev = (np.arange(G, dtype=np.int32) % 4) - 1
+    needs = set()
+    for keep in (list(range(G)), [g for g in range(G) if g % 3 != 1][::-1], [G - 1], []):
+        P, status, need = _run_prompt(sh, Q, Sc, x, keep, dev, 3, G)
+        needs.add(need > 0)
+        assert status == 0
+        if not keep:
+            assert (P == 0).all()
+            continue
+        ref = R.group_ffn_i4(Qh, Sh, hb(x), keep, dev, 3)
+        rms = np.sqrt(np.mean(R.merge(ref) ** 2))
+        assert np.abs(P - ref).max() <= U.TOL_BF16 * rms, (keep, np.abs(P - ref).max() / rms)
+    assert needs == {n_tok >= 16 and S in (64, 128, 256)}
+    if n_tok >= 16 and S in (64, 128, 256):
+        with pytest.raises(B.HaloError):                              # a workspace that is too small is refused
+            kl = torch.zeros(G, dtype=torch.int32, device=DEV)
+            nk = torch.ones(1, dtype=torch.int32, device=DEV)
+            Pz = torch.empty((1, n_tok, d), dtype=torch.float32, device=DEV)
+            B.halo_group_ffn_i4_prompt(sh, Q, Sc, x, n_tok, kl, nk, None, 0, Pz, torch.empty(1024, dtype=torch.uint8, device=DEV))
+
+
+def test_int4_prompt_entry_point_full_size_7b_block_sampled_tokens():
+    """One 7B-shaped block, 512 tokens, lossy holders, through the tensor cores: sampled token rows of every holder
+    slot against the oracle."""
+    wl = synth.workload("llama2-7b-decode")
+    Wp = synth.packed_layer(wl, 1, DEV)
+    sh, Q, Sc = _quantize(wl, Wp)
+    del Wp
+    hb = synth.host_bits
+    Qh, Sh = Q.cpu().numpy(), hb(Sc)
+    xw = synth.workload("llama2-7b-decode", n_tok=512)
+    x = synth.activation(xw, 8, DEV, n_tok=512)
+    G = wl.n_groups
+    dev = (np.arange(G, dtype=np.int32) % (wl.n_dev + 1)) - 1
+    keep = [g for g in range(G) if g % 7 != 3]
+    P, status, need = _run_prompt(sh, Q, Sc, x, keep, dev, wl.n_dev, G)
+    assert status == 0 and need > 0
+    tokens = [0, 127, 128, 255, 256, 400, 511]
+    ref = R.group_ffn_i4(Qh, Sh, hb(x)[tokens], keep, dev, wl.n_dev)
+    rms = np.sqrt(np.mean(R.merge(ref) ** 2))
+    assert np.abs(P[:, tokens] - ref).max() <= U.TOL_BF16 * rms

@@ -339,3 +339,26 @@ def test_int4_prompt_entry_point_full_size_7b_block_sampled_tokens():
     ref = R.group_ffn_i4(Qh, Sh, hb(x)[tokens], keep, dev, wl.n_dev)
     rms = np.sqrt(np.mean(R.merge(ref) ** 2))
     assert np.abs(P[:, tokens] - ref).max() <= U.TOL_BF16 * rms
+
+
+def test_int4_quantiser_extreme_magnitudes_bit_exact():
+    """Blocks of very small (fp32 subnormal), very large and mixed magnitudes, all-zero blocks and a lone non-zero
+    element: codes and scales of the GPU quantiser equal the oracle's bit for bit (both decide in IEEE fp32 without
+    flushing subnormals); the dequantised values stay finite."""
+    d, rows = 512, 24
+    g = torch.Generator().manual_seed(3)
+    W = torch.randn((rows, d), generator=g)
+    mags = torch.tensor([1e-42, 3e-39, 1e-30, 1e-8, 1.0, 1e8, 1e30, 3e37])
+    W = W * mags.repeat_interleave(3)[:, None]
+    W[5, 128:256] = 0.0                                      # an all-zero block
+    W[6, :128] = 0.0
+    W[6, 77] = -2.5e-41                                      # a lone subnormal
+    W = W.to(DEV)
+    Q = torch.empty((rows, d // 2), dtype=torch.uint8, device=DEV)
+    Sc = torch.empty((rows, d // 128), dtype=torch.bfloat16, device=DEV)
+    B.halo_quantize_rows_i4(d, rows, B.F32, W, Q, Sc)
+    torch.cuda.synchronize()
+    Q_ref, Sc_ref = R.quantize_i4(W.cpu().numpy())
+    assert (synth.host_bits(Sc) == Sc_ref).all()
+    assert (Q.cpu().numpy() == Q_ref).all()
+    assert np.isfinite(R.dequantize_i4(Q_ref, Sc_ref)).all()

@@ -187,6 +187,59 @@ def test_int4_stack_teacher_forced(name, layers, steps, mode):
     assert lost > 0
 
 
+def test_int4_stack_full_size_7b_sampled_blocks():
+    """The configuration bench.py times: 32 blocks at the 7B shape on int4 weights in ONE persistent launch.  Scores
+    and selections of every block (selection integers bit for bit from the recorded scores), the oracle's FFN on the
+    dequantised weights for sampled blocks from the recorded inputs."""
+    wl = synth.small_variant(synth.workload("llama2-7b-decode"), 32, 2)
+    L, G, d, n, steps = wl.n_layers, wl.n_groups, wl.d_model, wl.n_dev, 2
+    sample = {(0, 0), (0, 1), (1, 16), (1, 31)}
+    hb = synth.host_bits
+    quant = []
+    for l in range(L):
+        Wp = synth.packed_layer(wl, l, DEV)
+        _, Q, Sc = _quantize(wl, Wp)
+        quant.append((Q, Sc))
+        del Wp
+    preds = [synth.predictor(wl, l, DEV) for l in range(L)]
+    plan = B.Plan(G, wl.loss_rate, wl.share_weight, B.SEL_TOPK, B.k_of(wl), 0.0, wl.seed)
+    stack = B.Stack(B.ffn_shape(d, wl.d_ffn, wl.group_size, B.BF16), B.pred_shape(d, wl.pred_rank, G, B.BF16), 1, plan,
+                    [q[0] for q in quant], [p[0] for p in preds], [p[1] for p in preds], i4_scales=[q[1] for q in quant])
+    h0 = torch.stack([synth.stream_input(wl, s, DEV) for s in range(steps)])
+    h_out = torch.empty_like(h0)
+    t = dict(x=torch.zeros((steps, L, 1, d), dtype=torch.bfloat16, device=DEV),
+             scores=torch.zeros((steps, L, G), dtype=torch.float32, device=DEV),
+             dev_of_group=torch.zeros((steps, L, G), dtype=torch.int32, device=DEV),
+             arrived=torch.zeros((steps, L, n), dtype=torch.uint8, device=DEV),
+             keep_list=torch.zeros((steps, L, G), dtype=torch.int32, device=DEV),
+             n_keep=torch.zeros((steps, L), dtype=torch.int32, device=DEV),
+             y=torch.zeros((steps, L, 1, d), dtype=torch.float32, device=DEV))
+    taps = B.Taps(*[t[k].data_ptr() for k in ("x", "scores", "dev_of_group", "arrived", "keep_list", "n_keep", "y")])
+    stack.decode(h0, steps, 3, h_out, taps)
+    torch.cuda.synchronize()
+    assert stack.status() == 0 and stack.last_launches() == 1
+    x_all = hb(t["x"])
+    lost = 0
+    for s in range(steps):
+        for l in range(L):
+            scores = t["scores"][s, l].cpu().numpy()
+            sel = R.select(scores, wl.loss_rate, wl.share_weight, R.SEL_TOPK, R.k_of(wl), 0.0, wl.seed, 3 + s, l,
+                           force_all=(l == 0))
+            nk = int(t["n_keep"][s, l].item())
+            assert nk == sel["n_keep"] and (t["keep_list"][s, l].cpu().numpy() == sel["keep_list"]).all()
+            assert (t["dev_of_group"][s, l].cpu().numpy() == sel["dev_of_group"]).all()
+            assert (t["arrived"][s, l, :n].cpu().numpy() == sel["arrived"]).all()
+            lost += int(nk < G)
+            if (s, l) in sample:
+                if l > 0:
+                    ref = R.predict(hb(preds[l][0]), hb(preds[l][1]), x_all[s, l - 1])
+                    assert U.rel_err(scores, ref.astype(np.float64)) <= U.TOL_BF16
+                Q, Sc = quant[l]
+                P = R.group_ffn_i4(Q.cpu().numpy(), hb(Sc), x_all[s, l], sel["keep_list"][:nk], sel["dev_of_group"], n)
+                assert U.rel_err(t["y"][s, l].cpu().numpy(), R.merge(P)) <= U.TOL_BF16, (s, l)
+    assert lost > 0
+
+
 @pytest.mark.parametrize("d,G,S", [(256, 5, 16), (4096, 6, 128), (1024, 7, 256)])
 def test_int4_dequantise_is_exact(d, G, S):
     """halo_dequantize_weights_i4: every element IS the oracle's (nibble - 8) * s (the format's scales have 5

@@ -32,10 +32,10 @@ NOMINAL_HBM_GBS = 8000.0
 # 4-block 7B-shaped case (profiles/stack_decode_kernel_llama2-7b_4blocks.md); traffic is proportional to the kept
 # groups processed, so the ratio carries over to the full-size launch.  The figure belongs to the kernel sources with
 # the hash below: when they change the line reports no traffic until the counters have been taken again.
-STACK_KERNEL_TRAFFIC_RATIO = 1.0006
+STACK_KERNEL_TRAFFIC_RATIO = 1.0007
 STACK_KERNEL_SOURCES = ("stack_persistent.cu", "stack_persistent.cuh", "ffn_math.cuh", "i4_math.cuh", "tma.cuh", "umma.cuh",
                         "select_device.cuh")
-STACK_KERNEL_SOURCES_SHA1 = "c138ed5b9447b4f996c2f7b4f39510b79b0a6898"
+STACK_KERNEL_SOURCES_SHA1 = "7ae621467ca99f174feac17d4c5484231b8f22ea"
 FALLBACK_HBM_GBS = 6650.0
 
 

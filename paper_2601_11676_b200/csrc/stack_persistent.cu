@@ -106,6 +106,12 @@ struct ConsumerSync {
 };
 
 // Bounded spin until *word >= target (acquire); gives up early when the global abort word is set.
+// counter += v with release semantics and no return value: the stores this thread made before it are visible to whoever
+// acquires the counter (spin_until_ge), and the thread does not wait for the round trip
+__device__ __forceinline__ void red_release_add(unsigned* word, unsigned v) {
+    asm volatile("red.release.gpu.add.u32 [%0], %1;" ::"l"(word), "r"(v) : "memory");
+}
+
 __device__ __forceinline__ bool spin_until_ge(const unsigned* word, unsigned target, const unsigned* abort_word) {
     if (ld_acquire_gpu(word) >= target) return true;
     const long long t0 = clock64();
@@ -810,8 +816,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                                 if (P.act == HALO_ACT_RELU) z = fmaxf(z, 0.0f);
                                 zdst[a0 + i] = z;
                             }
-                            __threadfence();
-                            atomicAdd(sync_zcount, static_cast<unsigned>(a1));
+                            red_release_add(sync_zcount, static_cast<unsigned>(a1));   // publishes the values above
                         }
                         hpar ^= 1;
                     }
@@ -925,8 +930,7 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                             if (P.act == HALO_ACT_RELU) z = fmaxf(z, 0.0f);
                             zdst[a0 + i] = z;
                         }
-                        __threadfence();
-                        atomicAdd(sync_zcount, static_cast<unsigned>(a1));
+                        red_release_add(sync_zcount, static_cast<unsigned>(a1));   // publishes the values above
                     }
                     red_par ^= 1;
                 }
@@ -1043,11 +1047,15 @@ stack_decode_kernel(const __grid_constant__ PersistParams P) {
                 // of the block 16 ahead is idle now: its last user finished 16 blocks ago and its next user cannot
                 // have started.
                 if (cta == 0) P.sync[32 + ((q + 16u) & 31u)] = 0u;
-                __threadfence();
+                // Arrival: ONE acquire-release atomic instead of fence + relaxed atomic + fence (0.3 us per block: 3182 ->
+                // 3253 tokens/s on the TinyLlama shape, 784 -> 794 at 7B).  Release: this thread's stores and, through the
+                // thread-block barrier in front of it, the other threads' (whose reductions are complete and proxy-fenced
+                // above).  Acquire: the last arriver reads the head of the others' release sequence on this word; everybody
+                // else acquires in spin_until_ge, and the thread-block barrier behind this passes that on.
                 const unsigned target = (q + 1u) * static_cast<unsigned>(workers);
-                const unsigned before = atomicAdd(sync_barrier, 1u);
+                unsigned before;
+                asm volatile("atom.add.acq_rel.gpu.u32 %0, [%1], 1;" : "=r"(before) : "l"(sync_barrier) : "memory");
                 okb = (before + 1u == target) || spin_until_ge(sync_barrier, target, sync_abort);
-                __threadfence();
             }
             bad = pc_barrier_or(!okb);
             if (bad) break;
